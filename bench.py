@@ -1,0 +1,336 @@
+"""Benchmark of the routed FP4 mixture-of-experts layer on B200.
+
+A step is one pass of the whole hot path (moe_route -> moe_permute -> moe_expert_ffn -> moe_combine)
+over one batch of seeded synthetic input.  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+N > 1 (launched by torch.distributed.run, one rank per GPU) runs independent replicas: the layer
+does not shard in this build, so there is no data-path collective; the barrier and the max over
+ranks are the only communication.  --impl reference times the CPU oracle (rank 0 only).
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "MoE FP4 layer tokens/s"
+DECODE = ("decode_c1", "decode_c64")
+
+# dram__bytes_read.sum + dram__bytes_write.sum per moe_expert_ffn call from one ncu capture of the
+# workload (see profiles/); None until captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def expert_weight_bytes(H, I):
+    return 3 * H * I // 2 + 3 * H * I // 32
+
+
+def ffn_algorithmic_bytes(wl, n_touched):
+    """Bytes moe_expert_ffn must move: each touched expert's packed codes and scale bytes once, the
+    sorted activations in, the bf16 intermediate out and back in, the fp32 per-slot rows out."""
+    S = wl.T * wl.k
+    return n_touched * expert_weight_bytes(wl.H, wl.I) + S * wl.H * 2 + 2 * S * wl.I * 2 + S * wl.H * 4
+
+
+def ffn_flops(wl):
+    return wl.T * wl.k * 6 * wl.I * wl.H
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm=float(p["hbm_gbs"]), tensor_burst=float(p["bf16_tflops"]),
+                    tensor_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm=6650.0, tensor_burst=1590.0, tensor_sustained=1400.0, source="fallback")
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index, period=0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def sample(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        try:
+            self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+            r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)) if hasattr(
+                nv, "nvmlDeviceGetCurrentClocksEventReasons") else int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+            names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+            for bit, name in names.items():
+                if r & bit:
+                    self.reasons.add(name)
+        except Exception:
+            pass
+
+    def run(self):
+        while not self._stop_evt.is_set():
+            self.sample()
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        self.sample()
+        med = int(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_index):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+def max_over_ranks(value, world):
+    """Max of a float over all ranks (identity when not distributed)."""
+    if world == 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device="cuda" if dist.get_backend() == "nccl" else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def oracle_sample(wl, inputs, n_tokens, seed0=1000):
+    """Time the CPU oracle, as it stands, on n_tokens tokens of the workload (per-token definition)."""
+    from oracle import moe_oracle as O
+    logits = inputs.make_logits(max(wl.T, 1), wl.E, seed0, wl.skew)
+    x = inputs.make_x(max(wl.T, 1), wl.H, seed0)
+    if n_tokens > wl.T:
+        logits = np.concatenate([inputs.make_logits(wl.T, wl.E, seed0 + i, wl.skew) for i in range(n_tokens)])[:n_tokens]
+        x = np.concatenate([inputs.make_x(wl.T, wl.H, seed0 + i) for i in range(n_tokens)])[:n_tokens]
+    tokens = np.arange(min(n_tokens, logits.shape[0]), dtype=np.int32)
+    ids, _, _ = O.route(logits, wl.k)
+    need = sorted(set(ids[tokens].ravel().tolist()))
+    w13, s13, w2, s2 = inputs.make_expert_weights(wl.H, wl.I, wl.E, seed=0, experts=need)
+    t0 = time.perf_counter()
+    O.forward_tokens(logits, x, w13, s13, w2, s2, wl.k, tokens)
+    dt = time.perf_counter() - t0
+    return len(tokens) / dt, dt, len(tokens), O.num_threads()
+
+
+def run_reference(args, wl, inputs):
+    """The CPU oracle as the reference arm: each step is a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_tok = {"tiny": 16, "decode_c1": 1, "decode_c64": 8}.get(wl.name, 4)
+    for _ in range(args.warmup):
+        oracle_sample(wl, inputs, n_tok)
+    rates, total_t = [], 0.0
+    cores = 1
+    for i in range(args.steps):
+        r, dt, n, cores = oracle_sample(wl, inputs, n_tok, seed0=2000 + i)
+        rates.append(r)
+        total_t += dt
+    value = n_tok * args.steps / total_t
+    sample = "%d token(s) of %s per step, per-token definition, weights of the touched experts only" % (n_tok, wl.name)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "T": wl.T, "H": wl.H, "I": wl.I, "E": wl.E, "k": wl.k},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--workload", default="decode_c1")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2609_15627_b200 import inputs
+    wl = inputs.WORKLOADS[args.workload]
+    decode = wl.name in DECODE or wl.name == "tiny"
+    if args.impl == "reference":
+        args.steps = args.steps if args.steps is not None else 5
+        args.warmup = args.warmup if args.warmup is not None else 1
+        run_reference(args, wl, inputs)
+        return
+    if args.steps is None:
+        args.steps = 2000 if decode else 10
+    if args.warmup is None:
+        args.warmup = 20 if decode else 3
+    args.warmup = max(args.warmup, 3)
+
+    import torch
+    from paper_2609_15627_b200 import build_ext, moe
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        build_ext.build()
+    if world > 1:
+        torch.distributed.barrier()
+    moe.lib()
+
+    # ---- resident inputs: weights once, a cycle of seeded (logits, x) batches -------------------------
+    def dev(a):
+        if a.dtype == np.uint16:
+            return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+        return torch.from_numpy(a).cuda()
+
+    weights = tuple(dev(a) for a in inputs.make_expert_weights(wl.H, wl.I, wl.E, seed=0))
+    n_cycle = 32 if decode else 2
+    batches_host = [(inputs.make_logits(wl.T, wl.E, 7000 + rank * 100 + i, wl.skew), inputs.make_x(wl.T, wl.H, 7000 + rank * 100 + i))
+                    for i in range(n_cycle)]
+    batches = [(dev(l), dev(x)) for l, x in batches_host]
+    sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
+    buf = moe.LayerBuffers(sh)
+    stream = torch.cuda.current_stream()
+
+    # experts touched per batch of the cycle (from the library's own routing), for the byte count
+    touched = []
+    for l, x in batches:
+        moe.moe_route(l, wl.k, buf.topk_ids, buf.topk_w, buf.expert_offsets, buf.ws)
+        off = buf.expert_offsets.cpu().numpy()
+        touched.append(int(np.count_nonzero(np.diff(off))))
+
+    def step(i, ev=None):
+        l, x = batches[i % n_cycle]
+        moe.moe_route(l, wl.k, buf.topk_ids, buf.topk_w, buf.expert_offsets, buf.ws, stream)
+        moe.moe_permute(x, buf.topk_ids, buf.expert_offsets, sh, buf.x_perm, buf.perm, buf.inv_perm, buf.ws, stream)
+        if ev is not None:
+            ev[0].record(stream)
+        moe.moe_expert_ffn(buf.x_perm, buf.expert_offsets, *weights, sh, buf.y_perm, buf.status, buf.ws, stream)
+        if ev is not None:
+            ev[1].record(stream)
+        moe.moe_combine(buf.y_perm, buf.inv_perm, buf.topk_w, sh, buf.out, stream)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+
+    # ---- timed region: exactly K steps ---------------------------------------------------------------------
+    n_inner = min(args.steps, 256)  # steps whose expert-FFN call is bracketed by its own events
+    inner = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_inner)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(physical_gpu_index(local))
+    launches0 = moe.moe_launch_count()
+    barrier()
+    sampler.start()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i, inner[i] if i < n_inner else None)
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    launches = moe.moe_launch_count() - launches0
+    assert int(buf.status.item()) == 0, "device-side wait timed out"
+    ms_total = max_over_ranks(e0.elapsed_time(e1), world)
+    ms_step = ms_total / args.steps
+    value = wl.T * world / (ms_step * 1e-3)
+
+    # ---- roofline of the dominant call (the expert FFN) --------------------------------------------------------
+    ffn_ms = float(np.mean([a.elapsed_time(b) for a, b in inner]))
+    mean_touched = float(np.mean([touched[i % n_cycle] for i in range(n_inner)]))
+    peaks = load_peaks()
+    if decode:
+        alg = ffn_algorithmic_bytes(wl, mean_touched)
+        achieved = alg / (ffn_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"],
+                "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "algorithmic_bytes": alg}
+    else:
+        fl = ffn_flops(wl)
+        achieved = fl / (ffn_ms * 1e-3) / 1e12
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["tensor_sustained"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["tensor_sustained"], "traffic": NCU_TRAFFIC_BYTES.get(wl.name),
+                "algorithmic_flops": fl}
+    roof.update({"kernel": "moe_expert_ffn",
+                 "ms": ffn_ms, "peak_source": peaks["source"], "experts_touched": mean_touched})
+
+    # ---- end to end through the host-buffer entry point ---------------------------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        ws_h = moe.alloc_workspace(sh, host_path=True)
+        lh = [torch.from_numpy(l).pin_memory() for l, _ in batches_host]
+        xh = [torch.from_numpy(x.view(np.int16)).pin_memory() for _, x in batches_host]
+        oh = torch.empty((wl.T, wl.H), dtype=torch.int16).pin_memory()
+        n_e2e = max(3, min(args.steps, 200 if decode else 5))
+        for i in range(3):
+            moe.moe_forward_host(lh[i % n_cycle], xh[i % n_cycle], *weights, sh, oh, buf.status, ws_h, stream)
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(n_e2e):
+            moe.moe_forward_host(lh[i % n_cycle], xh[i % n_cycle], *weights, sh, oh, buf.status, ws_h, stream)
+        dt = max_over_ranks(time.perf_counter() - t0, world)
+        e2e = {"value": wl.T * world * n_e2e / dt, "unit": "tokens/s",
+               "h2d_bytes_per_step": wl.T * wl.E * 4 + wl.T * wl.H * 2, "d2h_bytes_per_step": wl.T * wl.H * 2,
+               "steps": n_e2e, "call": "moe_forward_host (pinned host logits/x in, bf16 out back, weights resident)"}
+
+    # ---- the oracle on the host cores (rank 0, N = 1 only) ----------------------------------------------------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n_tok = {"tiny": 64, "decode_c1": 32, "decode_c64": 32}.get(wl.name, 32)
+        v, dt, n, cores = oracle_sample(wl, inputs, n_tok)
+        cpu = {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+               "sample": "%d tokens with the %s shape and routing distribution, per-token definition, %.1f s" % (n, wl.name, dt)}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "T": wl.T, "H": wl.H, "I": wl.I, "E": wl.E, "k": wl.k,
+                       "parallelism": "replicas only" if world > 1 else "1 GPU",
+                       "l2": "inputs cycle over %d seeded batches; %.2f GB of expert weights resident (larger than L2)"
+                             % (n_cycle, wl.E * expert_weight_bytes(wl.H, wl.I) / 1e9)},
+            "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+            "kernels": moe.moe_last_kernel_name(),
+        }))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

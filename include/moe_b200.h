@@ -1,0 +1,144 @@
+/*
+ * moe_b200.h - C ABI of the B200 (sm_100a) routed mixture-of-experts layer with FP4 expert weights.
+ *
+ * The layer (paper, figure "Execution structure" and the accepted large-prefill path in the section
+ * "Prefill optimization"): Router Top-k -> route production (expert sorter) -> FP4 routed experts
+ * gate/up -> activation rounded to BF16 -> down projection, FP32 per-slot partials, unique-slot
+ * stores -> fixed-order Top-k FP32 reduction.  One call per stage, in that order.
+ *
+ * Notation: T tokens, H hidden size, I expert intermediate size, E experts, k experts per token,
+ * S = T*k slots, flat slot s = t*k + j (j = rank of the expert for token t, 0 = largest logit).
+ *
+ * Common rules
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer, 16-byte aligned, to a dense
+ *     row-major array (innermost dimension contiguous).  The caller owns every buffer; the library
+ *     allocates, frees and retains nothing.  `ws` is caller-provided scratch of at least
+ *     moe_workspace_bytes() bytes, 256-byte aligned; its contents need not survive between calls
+ *     and need no initialisation.
+ *   - Every call only enqueues work on `cuda_stream` (a cudaStream_t passed as void*, NULL = the
+ *     legacy default stream) and returns; there is no host synchronisation and no device-to-host copy.
+ *   - Return value: a moe_status_t.  Argument errors are found on the host before anything is
+ *     launched.  A device-side bounded wait that runs out writes MOE_ERR_TIMEOUT to *status_word
+ *     (sticky, device memory, may be NULL) and the kernel still terminates normally.
+ *   - Determinism: identical inputs give bit-identical outputs on every launch.  No invariance is
+ *     claimed across different T or batch compositions.
+ *   - bf16 arrays are passed as `const void*` / `void*` (16-bit elements, IEEE bfloat16 bit patterns).
+ *
+ * FP4 weight format (the checkpoint's storage format, kept packed in HBM; paper, section on the
+ * historical decode route: packed 4-bit weights without offline expansion, E2M1 nibbles, E8M0 scales)
+ *   - codes: two E2M1 codes per byte along K, element 2j in bits 3:0 of byte j, element 2j+1 in bits 7:4.
+ *     E2M1: bit 3 sign, bits 2:1 exponent (bias 1), bit 0 mantissa: magnitudes 0,.5,1,1.5,2,3,4,6.
+ *   - scales: one E8M0 byte b per 32 consecutive K elements of a row, meaning 2^(b-127).
+ *     The kernels support b in [0,128] (block scale up to 2); 255 (NaN) and 129..254 are rejected by
+ *     moe_validate_scales and otherwise give unspecified values.
+ *   - w13 [E, 2I, H/2] codes, rows [0,I) gate (w1), rows [I,2I) up (w3); w13_scale [E, 2I, H/32];
+ *     w2 [E, H, I/2] codes; w2_scale [E, H, I/32].
+ */
+#ifndef MOE_B200_H_
+#define MOE_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MOE_OK = 0,
+  MOE_ERR_INVALID_ARG = 1,       /* null or misaligned pointer, non-positive size, k > E */
+  MOE_ERR_UNSUPPORTED_SHAPE = 2, /* H or I not a multiple of 128, E > 1024, k > 32, T*k > 2^30 */
+  MOE_ERR_WORKSPACE = 3,         /* ws is NULL, misaligned or smaller than moe_workspace_bytes() */
+  MOE_ERR_CUDA = 4,              /* a CUDA runtime call or a launch failed */
+  MOE_ERR_TIMEOUT = 5            /* device side only: written to *status_word */
+} moe_status_t;
+
+typedef struct {
+  int32_t T, H, I, E, k;
+} moe_shape_t;
+
+/* Host, pure.  Scratch bytes the four calls need for this shape (0 if the shape is unsupported). */
+size_t moe_workspace_bytes(const moe_shape_t* shape);
+
+/* Host, pure.  Static string for a moe_status_t value. */
+const char* moe_status_string(int status);
+
+/* Host.  Name of the kernel variant the calling thread's last successful moe_* call chose
+ * (the choice is a pure function of the shape); "" before any call. */
+const char* moe_last_kernel_name(void);
+
+/* Host.  Number of kernels launched (memset nodes not counted) by this thread's moe_* calls so far. */
+uint64_t moe_launch_count(void);
+
+/*
+ * Router Top-k (paper: "Router Top-k"; fixed Top-K membership and order is a stated requirement).
+ *   logits [T,E] fp32 (finite).  For each token the k largest logits are selected, slot 0 the
+ *   largest, equal logits in ascending expert id.  topk_w = softmax over the k selected logits,
+ *   computed as e_j = EXP(l_j - l_0), s = ((e_0 + e_1) + ...) in fp32, w_j = e_j / s, where EXP is the
+ *   fixed fp32 sequence: d = max(d,-80); n = rint(d*0x1.715476p+0f); r = fma(n,-0x1.62e4p-1f,d);
+ *   r = fma(n,-0x1.7f7d1cp-20f,r); p = Horner/fma over 1/720,1/120,1/24,1/6,1/2,1,1 in r; EXP = p*2^n.
+ *   expert_offsets [E+1] int32: exclusive prefix sum of the per-expert slot counts, [E] = T*k.
+ * Errors: INVALID_ARG (null/misaligned, T<1, k<1, k>E), UNSUPPORTED_SHAPE (E>1024, k>32), WORKSPACE.
+ */
+int moe_route(const float* logits, int32_t T, int32_t E, int32_t k, int32_t* topk_ids /* [T,k] */,
+              float* topk_w /* [T,k] */, int32_t* expert_offsets /* [E+1] */, void* ws, size_t ws_bytes,
+              void* cuda_stream);
+
+/*
+ * Route production / expert sorter (paper: the sorter that groups assignments into per-expert row
+ * blocks so an expert's packed weights are scanned once).  A stable counting sort of the flat slots
+ * by expert id: perm[p] = slot at sorted position p (expert-major, ascending slot within an expert),
+ * inv_perm[perm[p]] = p, x_perm[p,:] = x[perm[p]/k,:].
+ *   x [T,H] bf16; topk_ids [T,k]; expert_offsets [E+1] as written by moe_route.
+ */
+int moe_permute(const void* x_bf16, const int32_t* topk_ids, const int32_t* expert_offsets,
+                const moe_shape_t* shape, void* x_perm_bf16 /* [T*k,H] */, int32_t* perm /* [T*k] */,
+                int32_t* inv_perm /* [T*k] */, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * FP4 routed experts: gate/up -> activation -> down (paper: stage 1, activation, stage 2).
+ * For every expert e and sorted row p in [expert_offsets[e], expert_offsets[e+1]):
+ *   g = W1_e x_p, u = W3_e x_p            (fp32 accumulation, weights = E2M1 value * 2^(scale-127))
+ *   a = bf16_rne( silu(g) * u )           (the already-rounded BF16 intermediate; kept in ws)
+ *   y_perm[p,:] = W2_e a                  (fp32, one store per (slot, column), no atomics)
+ * The summation order inside a dot product is the kernel's; everything else is as written.
+ *   status_word: device int32, may be NULL; see the common rules.
+ */
+int moe_expert_ffn(const void* x_perm_bf16 /* [T*k,H] */, const int32_t* expert_offsets,
+                   const uint8_t* w13, const uint8_t* w13_scale, const uint8_t* w2, const uint8_t* w2_scale,
+                   const moe_shape_t* shape, float* y_perm /* [T*k,H] */, int32_t* status_word, void* ws,
+                   size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Fixed-order Top-k FP32 reduction (paper: the vectorised fixed-order Top-k FP32 reducer that
+ * replaces cross-expert atomics).  out[t,n] = bf16_rne(acc_k), acc_0 = 0,
+ * acc_{j+1} = fma(topk_w[t,j], y_perm[inv_perm[t*k+j], n], acc_j), j = 0..k-1 ascending.
+ */
+int moe_combine(const float* y_perm, const int32_t* inv_perm, const float* topk_w, const moe_shape_t* shape,
+                void* out_bf16 /* [T,H] */, void* cuda_stream);
+
+/*
+ * One-time load check of E8M0 scale bytes (paper: scale layout and value traps, "test real
+ * nonconstant scales").  Counts bytes outside [0,128] into *bad_count (device int32, overwritten).
+ */
+int moe_validate_scales(const uint8_t* scales, size_t n_bytes, int32_t* bad_count, void* cuda_stream);
+
+/*
+ * The four calls above with HOST input and output for one batch: copies logits_host [T,E] and
+ * x_host [T,H] to the device buffers carved from `ws`, runs route -> permute -> expert_ffn ->
+ * combine on `cuda_stream`, copies out [T,H] bf16 back into out_host and waits for the stream.
+ * Weights stay device-resident (they are model state, not per-batch input).  For page-locked host
+ * buffers the copies are asynchronous until the final wait.  ws must hold
+ * moe_forward_host_workspace_bytes() bytes.  No counterpart in the paper: it is the end-to-end
+ * measurement path of the four calls.
+ */
+size_t moe_forward_host_workspace_bytes(const moe_shape_t* shape);
+int moe_forward_host(const float* logits_host, const void* x_host_bf16, const uint8_t* w13,
+                     const uint8_t* w13_scale, const uint8_t* w2, const uint8_t* w2_scale,
+                     const moe_shape_t* shape, void* out_host_bf16, int32_t* status_word, void* ws,
+                     size_t ws_bytes, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOE_B200_H_ */

@@ -1,0 +1,206 @@
+// extern "C" entry points of include/moe_b200.h: host-side argument checks, workspace carving and
+// kernel selection (a pure function of the shape).  No allocation, no synchronisation, no D2H copy,
+// except in moe_forward_host which is the host-buffer convenience path.
+#include <string.h>
+
+#include "moe_common.cuh"
+
+namespace moe {
+
+namespace {
+thread_local const char* g_last_kernel = "";
+thread_local uint64_t g_launches = 0;
+
+bool aligned(const void* p, size_t a) { return p != nullptr && (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+int check_shape(const moe_shape_t* s) {
+  if (s == nullptr) return MOE_ERR_INVALID_ARG;
+  if (s->T < 1 || s->H < 1 || s->I < 1 || s->E < 1 || s->k < 1 || s->k > s->E) return MOE_ERR_INVALID_ARG;
+  if (s->H % 128 != 0 || s->I % 128 != 0 || s->E > 1024 || s->k > 32) return MOE_ERR_UNSUPPORTED_SHAPE;
+  if (static_cast<long long>(s->T) * s->k > (1LL << 30)) return MOE_ERR_UNSUPPORTED_SHAPE;
+  return MOE_OK;
+}
+
+int check_ws(const void* ws, size_t ws_bytes, size_t need) {
+  if (!aligned(ws, kAlign) || ws_bytes < need) return MOE_ERR_WORKSPACE;
+  return MOE_OK;
+}
+}  // namespace
+
+void note_kernel(const char* name, int launches) {
+  g_last_kernel = name;
+  g_launches += static_cast<uint64_t>(launches);
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        n <= 0)
+      n = 148;
+  }
+  return n;
+}
+
+}  // namespace moe
+
+using namespace moe;
+
+extern "C" {
+
+size_t moe_workspace_bytes(const moe_shape_t* shape) {
+  if (check_shape(shape) != MOE_OK) return 0;
+  return ws_layout(*shape).total;
+}
+
+const char* moe_status_string(int status) {
+  switch (status) {
+    case MOE_OK: return "ok";
+    case MOE_ERR_INVALID_ARG: return "invalid argument";
+    case MOE_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case MOE_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case MOE_ERR_CUDA: return "CUDA runtime or launch error";
+    case MOE_ERR_TIMEOUT: return "device-side bounded wait ran out";
+    default: return "unknown status";
+  }
+}
+
+const char* moe_last_kernel_name(void) { return g_last_kernel; }
+
+uint64_t moe_launch_count(void) { return g_launches; }
+
+int moe_route(const float* logits, int32_t T, int32_t E, int32_t k, int32_t* topk_ids, float* topk_w,
+              int32_t* expert_offsets, void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (T < 1 || E < 1 || k < 1 || k > E) return MOE_ERR_INVALID_ARG;
+  if (E > 1024 || k > 32 || static_cast<long long>(T) * k > (1LL << 30)) return MOE_ERR_UNSUPPORTED_SHAPE;
+  if (!aligned(logits, 16) || !aligned(topk_ids, 16) || !aligned(topk_w, 16) || !aligned(expert_offsets, 16))
+    return MOE_ERR_INVALID_ARG;
+  // route uses only the counter block at the start of the workspace
+  const size_t need = align_up((static_cast<size_t>(E) + 8) * 4, kAlign);
+  if (check_ws(ws, ws_bytes, need) != MOE_OK) return MOE_ERR_WORKSPACE;
+  int* counters = static_cast<int*>(ws);
+  return launch_route(logits, T, E, k, topk_ids, topk_w, expert_offsets, counters, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int moe_permute(const void* x_bf16, const int32_t* topk_ids, const int32_t* expert_offsets, const moe_shape_t* shape,
+                void* x_perm_bf16, int32_t* perm, int32_t* inv_perm, void* ws, size_t ws_bytes, void* cuda_stream) {
+  const int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (!aligned(x_bf16, 16) || !aligned(topk_ids, 16) || !aligned(expert_offsets, 16) || !aligned(x_perm_bf16, 16) ||
+      !aligned(perm, 16) || !aligned(inv_perm, 16))
+    return MOE_ERR_INVALID_ARG;
+  const WsLayout L = ws_layout(*shape);
+  if (check_ws(ws, ws_bytes, L.total) != MOE_OK) return MOE_ERR_WORKSPACE;
+  int* block_counts = reinterpret_cast<int*>(static_cast<char*>(ws) + L.permute_off);
+  return launch_permute(static_cast<const __nv_bfloat16*>(x_bf16), topk_ids, expert_offsets, *shape,
+                        static_cast<__nv_bfloat16*>(x_perm_bf16), perm, inv_perm, block_counts,
+                        static_cast<cudaStream_t>(cuda_stream));
+}
+
+int moe_expert_ffn(const void* x_perm_bf16, const int32_t* expert_offsets, const uint8_t* w13, const uint8_t* w13_scale,
+                   const uint8_t* w2, const uint8_t* w2_scale, const moe_shape_t* shape, float* y_perm,
+                   int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
+  const int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (!aligned(x_perm_bf16, 16) || !aligned(expert_offsets, 16) || !aligned(w13, 16) || !aligned(w13_scale, 16) ||
+      !aligned(w2, 16) || !aligned(w2_scale, 16) || !aligned(y_perm, 16))
+    return MOE_ERR_INVALID_ARG;
+  if (status_word != nullptr && !aligned(status_word, 4)) return MOE_ERR_INVALID_ARG;
+  const WsLayout L = ws_layout(*shape);
+  if (check_ws(ws, ws_bytes, L.total) != MOE_OK) return MOE_ERR_WORKSPACE;
+  __nv_bfloat16* act = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(ws) + L.act_off);
+  return launch_expert_ffn(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w13, w13_scale, w2, w2_scale,
+                           *shape, act, y_perm, status_word, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int moe_combine(const float* y_perm, const int32_t* inv_perm, const float* topk_w, const moe_shape_t* shape,
+                void* out_bf16, void* cuda_stream) {
+  const int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (!aligned(y_perm, 16) || !aligned(inv_perm, 16) || !aligned(topk_w, 16) || !aligned(out_bf16, 16))
+    return MOE_ERR_INVALID_ARG;
+  return launch_combine(y_perm, inv_perm, topk_w, *shape, static_cast<__nv_bfloat16*>(out_bf16),
+                        static_cast<cudaStream_t>(cuda_stream));
+}
+
+int moe_validate_scales(const uint8_t* scales, size_t n_bytes, int32_t* bad_count, void* cuda_stream) {
+  if (scales == nullptr || n_bytes == 0 || !aligned(bad_count, 4)) return MOE_ERR_INVALID_ARG;
+  return launch_validate_scales(scales, n_bytes, bad_count, static_cast<cudaStream_t>(cuda_stream));
+}
+
+// ---- host-buffer path ---------------------------------------------------------------------------
+namespace {
+struct HostLayout {
+  size_t logits, x, ids, w, offsets, x_perm, perm, inv_perm, y_perm, out, inner, total;
+};
+HostLayout host_layout(const moe_shape_t& s) {
+  HostLayout L;
+  const size_t S = static_cast<size_t>(s.T) * s.k;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t o = off;
+    off += align_up(bytes, kAlign);
+    return o;
+  };
+  L.logits = take(static_cast<size_t>(s.T) * s.E * 4);
+  L.x = take(static_cast<size_t>(s.T) * s.H * 2);
+  L.ids = take(S * 4);
+  L.w = take(S * 4);
+  L.offsets = take((static_cast<size_t>(s.E) + 1) * 4);
+  L.x_perm = take(S * s.H * 2);
+  L.perm = take(S * 4);
+  L.inv_perm = take(S * 4);
+  L.y_perm = take(S * s.H * 4);
+  L.out = take(static_cast<size_t>(s.T) * s.H * 2);
+  L.inner = off;
+  off += ws_layout(s).total;
+  L.total = off;
+  return L;
+}
+}  // namespace
+
+size_t moe_forward_host_workspace_bytes(const moe_shape_t* shape) {
+  if (check_shape(shape) != MOE_OK) return 0;
+  return host_layout(*shape).total;
+}
+
+int moe_forward_host(const float* logits_host, const void* x_host_bf16, const uint8_t* w13, const uint8_t* w13_scale,
+                     const uint8_t* w2, const uint8_t* w2_scale, const moe_shape_t* shape, void* out_host_bf16,
+                     int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (logits_host == nullptr || x_host_bf16 == nullptr || out_host_bf16 == nullptr) return MOE_ERR_INVALID_ARG;
+  const HostLayout L = host_layout(*shape);
+  if (check_ws(ws, ws_bytes, L.total) != MOE_OK) return MOE_ERR_WORKSPACE;
+  char* base = static_cast<char*>(ws);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const moe_shape_t& s = *shape;
+  float* d_logits = reinterpret_cast<float*>(base + L.logits);
+  void* d_x = base + L.x;
+  int32_t* d_ids = reinterpret_cast<int32_t*>(base + L.ids);
+  float* d_w = reinterpret_cast<float*>(base + L.w);
+  int32_t* d_off = reinterpret_cast<int32_t*>(base + L.offsets);
+  void* d_xp = base + L.x_perm;
+  int32_t* d_perm = reinterpret_cast<int32_t*>(base + L.perm);
+  int32_t* d_inv = reinterpret_cast<int32_t*>(base + L.inv_perm);
+  float* d_y = reinterpret_cast<float*>(base + L.y_perm);
+  void* d_out = base + L.out;
+  void* inner = base + L.inner;
+  const size_t inner_bytes = ws_bytes - L.inner;
+  if (cudaMemcpyAsync(d_logits, logits_host, static_cast<size_t>(s.T) * s.E * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(d_x, x_host_bf16, static_cast<size_t>(s.T) * s.H * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  if ((rc = moe_route(d_logits, s.T, s.E, s.k, d_ids, d_w, d_off, inner, inner_bytes, st)) != MOE_OK) return rc;
+  if ((rc = moe_permute(d_x, d_ids, d_off, shape, d_xp, d_perm, d_inv, inner, inner_bytes, st)) != MOE_OK) return rc;
+  if ((rc = moe_expert_ffn(d_xp, d_off, w13, w13_scale, w2, w2_scale, shape, d_y, status_word, inner, inner_bytes, st)) !=
+      MOE_OK)
+    return rc;
+  if ((rc = moe_combine(d_y, d_inv, d_w, shape, d_out, st)) != MOE_OK) return rc;
+  if (cudaMemcpyAsync(out_host_bf16, d_out, static_cast<size_t>(s.T) * s.H * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return MOE_ERR_CUDA;
+  return MOE_OK;
+}
+
+}  // extern "C"

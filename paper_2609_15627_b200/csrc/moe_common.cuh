@@ -1,0 +1,72 @@
+// Shared declarations of the sm_100a routed-MoE library (internal; the public ABI is include/moe_b200.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/moe_b200.h"
+
+#define MOE_DEVINL __device__ __forceinline__
+
+namespace moe {
+
+// ---- workspace carving (host) ----------------------------------------------------------------
+// ws = [ route counters (always first) | act bf16 [S,I] | permute block counts | ffn counters ]
+struct WsLayout {
+  size_t act_off, route_off, permute_off, ffn_off, total;
+};
+
+constexpr int kPermuteChunk = 1024;  // slots per CTA in the multi-CTA permute
+constexpr size_t kAlign = 256;
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+inline WsLayout ws_layout(const moe_shape_t& s) {
+  WsLayout L;
+  const size_t S = static_cast<size_t>(s.T) * s.k;
+  size_t off = 0;
+  L.route_off = off;  // moe_route is given only (T, E, k): its block must not depend on H or I
+  off += align_up((static_cast<size_t>(s.E) + 8) * 4, kAlign);
+  L.act_off = off;
+  off += align_up(S * s.I * 2, kAlign);
+  L.permute_off = off;
+  const size_t nblk = (S + kPermuteChunk - 1) / kPermuteChunk;
+  off += align_up(nblk * s.E * 4, kAlign);
+  L.ffn_off = off;
+  off += align_up(1024, kAlign);
+  L.total = off;
+  return L;
+}
+
+// ---- per-thread call record (host) -----------------------------------------------------------
+void note_kernel(const char* name, int launches);
+
+// ---- launchers implemented in the .cu files --------------------------------------------------
+int launch_route(const float* logits, int T, int E, int k, int* ids, float* w, int* offsets, int* counters,
+                 cudaStream_t st);
+int launch_permute(const __nv_bfloat16* x, const int* ids, const int* offsets, const moe_shape_t& s,
+                   __nv_bfloat16* x_perm, int* perm, int* inv_perm, int* block_counts, cudaStream_t st);
+int launch_expert_ffn(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
+                      const uint8_t* w2, const uint8_t* s2, const moe_shape_t& s, __nv_bfloat16* act, float* y_perm,
+                      int* status_word, cudaStream_t st);
+int launch_combine(const float* y_perm, const int* inv_perm, const float* w, const moe_shape_t& s,
+                   __nv_bfloat16* out, cudaStream_t st);
+int launch_validate_scales(const uint8_t* scales, size_t n, int* bad, cudaStream_t st);
+
+int sm_count();
+
+// ---- small device helpers ---------------------------------------------------------------------
+MOE_DEVINL int warp_excl_scan(int v, int lane, int* total) {
+  int incl = v;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += n;
+  }
+  *total = __shfl_sync(0xffffffffu, incl, 31);
+  return incl - v;
+}
+
+}  // namespace moe

@@ -1,0 +1,392 @@
+// Router top-k, route production (stable expert sort + row gather) and the fixed-order fp32 combine.
+// All three are integer / bandwidth work: warp shuffles, shared-memory histograms, prefix scans and
+// 16-byte vector copies.  Results are bit-defined (see include/moe_b200.h).
+#include "moe_common.cuh"
+
+namespace moe {
+
+// =================================================================================================
+// moe_route
+// =================================================================================================
+
+// The fixed fp32 exponential of the routing softmax (sequence stated in the public header).  Every
+// step is an explicitly rounded intrinsic so that the compiler cannot contract or reorder it.
+MOE_DEVINL float exp_fixed(float d) {
+  d = fmaxf(d, -80.0f);
+  const float t = __fmul_rn(d, 0x1.715476p+0f);
+  const float n = rintf(t);
+  float r = __fmaf_rn(n, -0x1.62e4p-1f, d);
+  r = __fmaf_rn(n, -0x1.7f7d1cp-20f, r);
+  float p = 0x1.6c16c2p-10f;               // 1/720
+  p = __fmaf_rn(p, r, 0x1.111112p-7f);     // 1/120
+  p = __fmaf_rn(p, r, 0x1.555556p-5f);     // 1/24
+  p = __fmaf_rn(p, r, 0x1.555556p-3f);     // 1/6
+  p = __fmaf_rn(p, r, 0.5f);
+  p = __fmaf_rn(p, r, 1.0f);
+  p = __fmaf_rn(p, r, 1.0f);
+  const int e = static_cast<int>(n);       // in [-116, 0]
+  return __fmul_rn(p, __int_as_float((e + 127) << 23));
+}
+
+// Exclusive scan of counts[0..E) into offsets[0..E], offsets[E] = total.  Whole block takes part.
+__device__ void block_offsets_scan(const int* counts, int E, int* offsets, int* warp_tot /* smem [32] */) {
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nw = blockDim.x >> 5;
+  const int per = (E + blockDim.x - 1) / blockDim.x;
+  const int base = tid * per;
+  int sum = 0;
+  for (int i = 0; i < per; ++i)
+    if (base + i < E) sum += counts[base + i];
+  int wtotal;
+  const int excl = warp_excl_scan(sum, lane, &wtotal);
+  if (lane == 0) warp_tot[wid] = wtotal;
+  __syncthreads();
+  if (wid == 0) {
+    const int v = (lane < nw) ? warp_tot[lane] : 0;
+    int tot;
+    const int ex = warp_excl_scan(v, lane, &tot);
+    __syncwarp();
+    warp_tot[lane] = ex;
+    if (lane == 0) offsets[E] = tot;
+  }
+  __syncthreads();
+  int run = warp_tot[wid] + excl;
+  for (int i = 0; i < per; ++i) {
+    if (base + i < E) {
+      offsets[base + i] = run;
+      run += counts[base + i];
+    }
+  }
+}
+
+// One warp per token.  row = this warp's copy of the token's logits in shared memory.
+// Returns through lane j (< k) the j-th selected expert and its logit.
+MOE_DEVINL void warp_topk(const float* row, int E, int k, int lane, int* my_id, float* my_v) {
+  unsigned taken = 0u;  // bit i: element lane + 32*i already selected
+  *my_id = 0;
+  *my_v = 0.0f;
+  for (int j = 0; j < k; ++j) {
+    float bv = 0.0f;
+    int bi = -1;
+    for (int i = 0; i * 32 + lane < E; ++i) {
+      if (!((taken >> i) & 1u)) {
+        const float v = row[i * 32 + lane];
+        if (bi < 0 || v > bv) {  // strict '>': the lowest id among this lane's equal values stays
+          bv = v;
+          bi = i * 32 + lane;
+        }
+      }
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, d);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, d);
+      const bool take = (oi >= 0) && (bi < 0 || ov > bv || (ov == bv && oi < bi));
+      if (take) {
+        bv = ov;
+        bi = oi;
+      }
+    }
+    // lane 0's view is authoritative (identical on all lanes for finite logits)
+    bi = __shfl_sync(0xffffffffu, bi, 0);
+    bv = __shfl_sync(0xffffffffu, bv, 0);
+    if (bi >= 0 && (bi & 31) == lane) taken |= 1u << (bi >> 5);
+    if (lane == j) {
+      *my_id = bi;
+      *my_v = bv;
+    }
+  }
+}
+
+MOE_DEVINL float warp_softmax_selected(float my_v, int k, int lane) {
+  const float m = __shfl_sync(0xffffffffu, my_v, 0);
+  const float e = exp_fixed(__fsub_rn(my_v, m));
+  float s = 0.0f;
+  for (int j = 0; j < k; ++j) {
+    const float ej = __shfl_sync(0xffffffffu, e, j);
+    s = (j == 0) ? ej : __fadd_rn(s, ej);
+  }
+  return __fdiv_rn(e, s);
+}
+
+// single_block != 0: one CTA handles every token and builds the histogram in shared memory.
+// Otherwise the histogram is accumulated in g_counts[0..E) (zeroed before the launch) and the last
+// CTA to finish (ticket in g_counts[E]) scans it.
+__global__ void __launch_bounds__(1024) route_kernel(const float* __restrict__ logits, int T, int E, int k,
+                                                     int* __restrict__ ids, float* __restrict__ w,
+                                                     int* __restrict__ offsets, int* g_counts, int single_block) {
+  extern __shared__ float sm_f[];
+  const int nw = blockDim.x >> 5;
+  float* rows = sm_f;                                   // [nw][E]
+  int* s_counts = reinterpret_cast<int*>(sm_f + nw * E);  // [E]
+  int* s_misc = s_counts + E;                           // [32] + flag
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  if (single_block) {
+    for (int e = tid; e < E; e += blockDim.x) s_counts[e] = 0;
+    __syncthreads();
+  }
+  float* row = rows + wid * E;
+  const int t0 = blockIdx.x * nw + wid;
+  const int tstride = gridDim.x * nw;
+  for (int t = t0; t < T; t += tstride) {
+    for (int e = lane; e < E; e += 32) row[e] = logits[static_cast<size_t>(t) * E + e];
+    __syncwarp();
+    int my_id;
+    float my_v;
+    warp_topk(row, E, k, lane, &my_id, &my_v);
+    const float wt = warp_softmax_selected(my_v, k, lane);
+    if (lane < k) {
+      ids[static_cast<size_t>(t) * k + lane] = my_id;
+      w[static_cast<size_t>(t) * k + lane] = wt;
+      if (my_id >= 0) atomicAdd(single_block ? &s_counts[my_id] : &g_counts[my_id], 1);
+    }
+    __syncwarp();
+  }
+  if (single_block) {
+    __syncthreads();
+    block_offsets_scan(s_counts, E, offsets, s_misc);
+    return;
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_misc[32] = (atomicAdd(&g_counts[E], 1) == static_cast<int>(gridDim.x) - 1);
+  __syncthreads();
+  if (s_misc[32]) {
+    __threadfence();
+    for (int e = tid; e < E; e += blockDim.x) s_counts[e] = __ldcg(&g_counts[e]);
+    __syncthreads();
+    block_offsets_scan(s_counts, E, offsets, s_misc);
+  }
+}
+
+int launch_route(const float* logits, int T, int E, int k, int* ids, float* w, int* offsets, int* counters,
+                 cudaStream_t st) {
+  const bool single = T <= 128;
+  const int nw = single ? 32 : 8;
+  const size_t smem = (static_cast<size_t>(nw) * E + E + 40) * 4;
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
+      return MOE_ERR_CUDA;
+    attr_done = true;
+  }
+  int launches = 1;
+  if (single) {
+    route_kernel<<<1, nw * 32, smem, st>>>(logits, T, E, k, ids, w, offsets, counters, 1);
+    note_kernel("route_topk_single_cta", launches);
+  } else {
+    if (cudaMemsetAsync(counters, 0, (static_cast<size_t>(E) + 1) * 4, st) != cudaSuccess) return MOE_ERR_CUDA;
+    const int grid = (T + nw - 1) / nw;
+    route_kernel<<<grid, nw * 32, smem, st>>>(logits, T, E, k, ids, w, offsets, counters, 0);
+    note_kernel("route_topk_multi_cta", launches);
+  }
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+// =================================================================================================
+// moe_permute
+// =================================================================================================
+
+MOE_DEVINL void warp_copy_row(const __nv_bfloat16* src, __nv_bfloat16* dst, int H, int lane) {
+  const uint4* s4 = reinterpret_cast<const uint4*>(src);
+  uint4* d4 = reinterpret_cast<uint4*>(dst);
+  const int n = H / 8;
+  for (int i = lane; i < n; i += 32) d4[i] = __ldg(&s4[i]);
+}
+
+// Small S: one warp per slot.  Rank of slot s inside its expert = number of earlier slots with the
+// same expert (counted directly), so the sort is stable by construction.
+__global__ void __launch_bounds__(256) permute_small_kernel(const __nv_bfloat16* __restrict__ x,
+                                                            const int* __restrict__ ids,
+                                                            const int* __restrict__ offsets, int S, int H, int k,
+                                                            __nv_bfloat16* __restrict__ x_perm,
+                                                            int* __restrict__ perm, int* __restrict__ inv_perm) {
+  const int lane = threadIdx.x & 31;
+  const int s = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (s >= S) return;
+  const int e = ids[s];
+  int c = 0;
+  for (int q = lane; q < s; q += 32) c += (ids[q] == e);
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) c += __shfl_xor_sync(0xffffffffu, c, d);
+  const int p = offsets[e] + c;
+  if (lane == 0) {
+    perm[p] = s;
+    inv_perm[s] = p;
+  }
+  warp_copy_row(x + static_cast<size_t>(s / k) * H, x_perm + static_cast<size_t>(p) * H, H, lane);
+}
+
+// Large S, pass 1: per-chunk histogram.
+__global__ void __launch_bounds__(256) permute_count_kernel(const int* __restrict__ ids, int S, int E,
+                                                            int* __restrict__ block_counts) {
+  extern __shared__ int s_hist[];
+  for (int e = threadIdx.x; e < E; e += blockDim.x) s_hist[e] = 0;
+  __syncthreads();
+  const int base = blockIdx.x * kPermuteChunk;
+  for (int i = threadIdx.x; i < kPermuteChunk; i += blockDim.x) {
+    const int s = base + i;
+    if (s < S) atomicAdd(&s_hist[ids[s]], 1);
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += blockDim.x) block_counts[static_cast<size_t>(blockIdx.x) * E + e] = s_hist[e];
+}
+
+// Large S, pass 2: one warp per expert turns the per-chunk counts into per-chunk start positions.
+__global__ void __launch_bounds__(256) permute_scan_kernel(const int* __restrict__ offsets, int E, int nblk,
+                                                           int* __restrict__ block_counts) {
+  const int lane = threadIdx.x & 31;
+  const int e = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (e >= E) return;
+  int running = offsets[e];
+  for (int b0 = 0; b0 < nblk; b0 += 32) {
+    const int b = b0 + lane;
+    const int v = (b < nblk) ? block_counts[static_cast<size_t>(b) * E + e] : 0;
+    int tot;
+    const int ex = warp_excl_scan(v, lane, &tot);
+    if (b < nblk) block_counts[static_cast<size_t>(b) * E + e] = running + ex;
+    running += tot;
+  }
+}
+
+// Large S, pass 3: stable ranks inside a chunk.  Each warp owns 128 consecutive slots; warps are
+// ordered through a per-warp count table, lanes through a match mask.
+__global__ void __launch_bounds__(256) permute_scatter_kernel(const int* __restrict__ ids, int S, int E,
+                                                              const int* __restrict__ block_base,
+                                                              int* __restrict__ perm, int* __restrict__ inv_perm) {
+  extern __shared__ int s_w[];  // [8][E]
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  constexpr int kWarps = 8, kPerWarp = kPermuteChunk / kWarps;
+  for (int i = tid; i < kWarps * E; i += blockDim.x) s_w[i] = 0;
+  __syncthreads();
+  int* mine = s_w + wid * E;
+  const int base = blockIdx.x * kPermuteChunk + wid * kPerWarp;
+  const unsigned lt = (1u << lane) - 1u;
+  for (int it = 0; it < kPerWarp / 32; ++it) {
+    const int s = base + it * 32 + lane;
+    const int e = (s < S) ? ids[s] : E;
+    const unsigned peers = __match_any_sync(0xffffffffu, e);
+    if (e < E && (peers & lt) == 0u) mine[e] += __popc(peers);
+    __syncwarp();
+  }
+  __syncthreads();
+  for (int e = tid; e < E; e += blockDim.x) {
+    int run = block_base[static_cast<size_t>(blockIdx.x) * E + e];
+    for (int w = 0; w < kWarps; ++w) {
+      const int c = s_w[w * E + e];
+      s_w[w * E + e] = run;
+      run += c;
+    }
+  }
+  __syncthreads();
+  for (int it = 0; it < kPerWarp / 32; ++it) {
+    const int s = base + it * 32 + lane;
+    const int e = (s < S) ? ids[s] : E;
+    const unsigned peers = __match_any_sync(0xffffffffu, e);
+    if (e < E) {
+      const int p = mine[e] + __popc(peers & lt);
+      perm[p] = s;
+      inv_perm[s] = p;
+    }
+    __syncwarp();
+    if (e < E && (peers & lt) == 0u) mine[e] += __popc(peers);
+    __syncwarp();
+  }
+}
+
+// Large S, pass 4: gather rows, one warp per sorted row.
+__global__ void __launch_bounds__(256) permute_gather_kernel(const __nv_bfloat16* __restrict__ x,
+                                                             const int* __restrict__ perm, int S, int H, int k,
+                                                             __nv_bfloat16* __restrict__ x_perm) {
+  const int lane = threadIdx.x & 31;
+  const int wpb = blockDim.x >> 5;
+  for (int p = blockIdx.x * wpb + (threadIdx.x >> 5); p < S; p += gridDim.x * wpb) {
+    const int s = perm[p];
+    warp_copy_row(x + static_cast<size_t>(s / k) * H, x_perm + static_cast<size_t>(p) * H, H, lane);
+  }
+}
+
+int launch_permute(const __nv_bfloat16* x, const int* ids, const int* offsets, const moe_shape_t& sh,
+                   __nv_bfloat16* x_perm, int* perm, int* inv_perm, int* block_counts, cudaStream_t st) {
+  const int S = sh.T * sh.k;
+  if (S <= 4096) {
+    permute_small_kernel<<<(S + 7) / 8, 256, 0, st>>>(x, ids, offsets, S, sh.H, sh.k, x_perm, perm, inv_perm);
+    note_kernel("permute_rank_by_count", 1);
+  } else {
+    const int nblk = (S + kPermuteChunk - 1) / kPermuteChunk;
+    permute_count_kernel<<<nblk, 256, sh.E * 4, st>>>(ids, S, sh.E, block_counts);
+    permute_scan_kernel<<<(sh.E + 7) / 8, 256, 0, st>>>(offsets, sh.E, nblk, block_counts);
+    permute_scatter_kernel<<<nblk, 256, 8 * sh.E * 4, st>>>(ids, S, sh.E, block_counts, perm, inv_perm);
+    const int grid = min((S + 7) / 8, sm_count() * 16);
+    permute_gather_kernel<<<grid, 256, 0, st>>>(x, perm, S, sh.H, sh.k, x_perm);
+    note_kernel("permute_chunked_scan", 4);
+  }
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+// =================================================================================================
+// moe_combine
+// =================================================================================================
+
+// One thread per (token, 8 consecutive columns): k fused multiply-adds per column in slot order.
+__global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ y, const int* __restrict__ inv_perm,
+                                                      const float* __restrict__ w, int T, int H, int k,
+                                                      __nv_bfloat16* __restrict__ out) {
+  const int groups = H / 8;
+  const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= static_cast<size_t>(T) * groups) return;
+  const int t = static_cast<int>(idx / groups);
+  const int c = static_cast<int>(idx % groups) * 8;
+  float acc[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) acc[i] = 0.0f;
+  for (int j = 0; j < k; ++j) {
+    const int p = __ldg(&inv_perm[static_cast<size_t>(t) * k + j]);
+    const float wj = __ldg(&w[static_cast<size_t>(t) * k + j]);
+    const float4* src = reinterpret_cast<const float4*>(y + static_cast<size_t>(p) * H + c);
+    const float4 a = __ldg(src), b = __ldg(src + 1);
+    acc[0] = __fmaf_rn(wj, a.x, acc[0]);
+    acc[1] = __fmaf_rn(wj, a.y, acc[1]);
+    acc[2] = __fmaf_rn(wj, a.z, acc[2]);
+    acc[3] = __fmaf_rn(wj, a.w, acc[3]);
+    acc[4] = __fmaf_rn(wj, b.x, acc[4]);
+    acc[5] = __fmaf_rn(wj, b.y, acc[5]);
+    acc[6] = __fmaf_rn(wj, b.z, acc[6]);
+    acc[7] = __fmaf_rn(wj, b.w, acc[7]);
+  }
+  __nv_bfloat162 o[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) o[i] = __floats2bfloat162_rn(acc[2 * i], acc[2 * i + 1]);
+  *reinterpret_cast<uint4*>(out + static_cast<size_t>(t) * H + c) = *reinterpret_cast<uint4*>(o);
+}
+
+int launch_combine(const float* y_perm, const int* inv_perm, const float* w, const moe_shape_t& sh,
+                   __nv_bfloat16* out, cudaStream_t st) {
+  const size_t n = static_cast<size_t>(sh.T) * (sh.H / 8);
+  combine_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(y_perm, inv_perm, w, sh.T, sh.H, sh.k, out);
+  note_kernel("combine_slot_order_fma", 1);
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+// =================================================================================================
+// moe_validate_scales
+// =================================================================================================
+
+__global__ void __launch_bounds__(256) validate_scales_kernel(const uint8_t* __restrict__ s, size_t n, int* bad) {
+  int c = 0;
+  for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n;
+       i += static_cast<size_t>(gridDim.x) * blockDim.x)
+    c += (s[i] > 128);
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) c += __shfl_xor_sync(0xffffffffu, c, d);
+  if ((threadIdx.x & 31) == 0 && c) atomicAdd(bad, c);
+}
+
+int launch_validate_scales(const uint8_t* scales, size_t n, int* bad, cudaStream_t st) {
+  if (cudaMemsetAsync(bad, 0, 4, st) != cudaSuccess) return MOE_ERR_CUDA;
+  const int grid = static_cast<int>(min(static_cast<size_t>(sm_count()) * 8, (n + 255) / 256));
+  validate_scales_kernel<<<grid > 0 ? grid : 1, 256, 0, st>>>(scales, n, bad);
+  note_kernel("validate_scales", 1);
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+}  // namespace moe

@@ -141,11 +141,11 @@ def index_scales(rows, K, E=1, lo=116, span=8):
     return (lo + (3 * e + 5 * r + 7 * b) % span).astype(np.uint8)
 
 
-def fingerprint_codes(rows, K, E=1):
-    """Codes whose rows are pairwise different in a way a row or tile permutation cannot hide:
-    element (e, r, h) has code (r + 3*h + 5*e + (r // 16)) mod 16."""
-    e = np.arange(E)[:, None, None]
-    r = np.arange(rows)[None, :, None]
-    h = np.arange(K)[None, None, :]
-    c = ((r + 3 * h + 5 * e + r // 16) % 16).astype(np.uint8)
+def fingerprint_codes(rows, K, E=1, seed=0):
+    """Codes in which every row carries its own signature: one seeded random code sequence per expert,
+    shared by all its rows, shifted per row by (7*r + 3*(r // 16)) mod 16.  The 16 rows of a tile all
+    differ and neighbouring tiles differ, so a kernel that swaps rows or row tiles gives a wrong output."""
+    base = _rng(seed, 99).integers(0, 16, size=(E, 1, K), dtype=np.int64)
+    r = np.arange(rows, dtype=np.int64)[None, :, None]
+    c = ((base + 7 * r + 3 * (r // 16)) % 16).astype(np.uint8)
     return (c[..., 0::2] | (c[..., 1::2] << 4)).astype(np.uint8)

@@ -1,0 +1,164 @@
+"""Thin binding over the C-ABI CUDA library (include/moe_b200.h): argument marshalling only.
+
+Every function has the name and meaning of the C entry point it calls; every step of the layer runs
+in the library's CUDA kernels.  torch is used for device memory and streams.  There is no CPU path:
+if libmoe_b200.so is missing or a call fails, a MoeError is raised.
+"""
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmoe_b200.so")
+
+EXPORTS = ("moe_workspace_bytes", "moe_status_string", "moe_last_kernel_name", "moe_launch_count", "moe_route",
+           "moe_permute", "moe_expert_ffn", "moe_combine", "moe_validate_scales",
+           "moe_forward_host_workspace_bytes", "moe_forward_host")
+
+
+class MoeError(RuntimeError):
+    pass
+
+
+class Shape(C.Structure):
+    _fields_ = [("T", C.c_int32), ("H", C.c_int32), ("I", C.c_int32), ("E", C.c_int32), ("k", C.c_int32)]
+
+
+_lib = None
+
+
+def lib():
+    """Load the CUDA library once; raise if it was not built (python paper_2609_15627_b200/build_ext.py)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise MoeError("CUDA library not built: %s is missing (run paper_2609_15627_b200/build_ext.py)" % LIB_PATH)
+        L = C.CDLL(LIB_PATH)
+        vp, i32, sz = C.c_void_p, C.c_int32, C.c_size_t
+        L.moe_workspace_bytes.restype = sz
+        L.moe_workspace_bytes.argtypes = [C.POINTER(Shape)]
+        L.moe_forward_host_workspace_bytes.restype = sz
+        L.moe_forward_host_workspace_bytes.argtypes = [C.POINTER(Shape)]
+        L.moe_status_string.restype = C.c_char_p
+        L.moe_status_string.argtypes = [C.c_int]
+        L.moe_last_kernel_name.restype = C.c_char_p
+        L.moe_launch_count.restype = C.c_uint64
+        L.moe_route.restype = C.c_int
+        L.moe_route.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
+        L.moe_permute.restype = C.c_int
+        L.moe_permute.argtypes = [vp, vp, vp, C.POINTER(Shape), vp, vp, vp, vp, sz, vp]
+        L.moe_expert_ffn.restype = C.c_int
+        L.moe_expert_ffn.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp, sz, vp]
+        L.moe_combine.restype = C.c_int
+        L.moe_combine.argtypes = [vp, vp, vp, C.POINTER(Shape), vp, vp]
+        L.moe_validate_scales.restype = C.c_int
+        L.moe_validate_scales.argtypes = [vp, sz, vp, vp]
+        L.moe_forward_host.restype = C.c_int
+        L.moe_forward_host.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp, sz, vp]
+        _lib = L
+    return _lib
+
+
+def _check(rc, what):
+    if rc != 0:
+        raise MoeError("%s failed: %s (%d)" % (what, lib().moe_status_string(rc).decode(), rc))
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def shape(T, H, I, E, k):
+    return Shape(int(T), int(H), int(I), int(E), int(k))
+
+
+def moe_workspace_bytes(sh):
+    return int(lib().moe_workspace_bytes(C.byref(sh)))
+
+
+def moe_forward_host_workspace_bytes(sh):
+    return int(lib().moe_forward_host_workspace_bytes(C.byref(sh)))
+
+
+def moe_last_kernel_name():
+    return lib().moe_last_kernel_name().decode()
+
+
+def moe_launch_count():
+    return int(lib().moe_launch_count())
+
+
+def alloc_workspace(sh, device="cuda", host_path=False):
+    n = moe_forward_host_workspace_bytes(sh) if host_path else moe_workspace_bytes(sh)
+    if n == 0:
+        raise MoeError("unsupported shape")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def moe_route(logits, k, topk_ids, topk_w, expert_offsets, ws, stream=None):
+    T, E = logits.shape
+    _check(lib().moe_route(_ptr(logits), T, E, k, _ptr(topk_ids), _ptr(topk_w), _ptr(expert_offsets), _ptr(ws),
+                           ws.numel(), _stream(stream)), "moe_route")
+
+
+def moe_permute(x, topk_ids, expert_offsets, sh, x_perm, perm, inv_perm, ws, stream=None):
+    _check(lib().moe_permute(_ptr(x), _ptr(topk_ids), _ptr(expert_offsets), C.byref(sh), _ptr(x_perm), _ptr(perm),
+                             _ptr(inv_perm), _ptr(ws), ws.numel(), _stream(stream)), "moe_permute")
+
+
+def moe_expert_ffn(x_perm, expert_offsets, w13, w13_scale, w2, w2_scale, sh, y_perm, status_word, ws, stream=None):
+    _check(lib().moe_expert_ffn(_ptr(x_perm), _ptr(expert_offsets), _ptr(w13), _ptr(w13_scale), _ptr(w2), _ptr(w2_scale),
+                                C.byref(sh), _ptr(y_perm), _ptr(status_word), _ptr(ws), ws.numel(), _stream(stream)),
+           "moe_expert_ffn")
+
+
+def moe_combine(y_perm, inv_perm, topk_w, sh, out, stream=None):
+    _check(lib().moe_combine(_ptr(y_perm), _ptr(inv_perm), _ptr(topk_w), C.byref(sh), _ptr(out), _stream(stream)),
+           "moe_combine")
+
+
+def moe_validate_scales(scales, bad_count, stream=None):
+    _check(lib().moe_validate_scales(_ptr(scales), scales.numel(), _ptr(bad_count), _stream(stream)),
+           "moe_validate_scales")
+
+
+def moe_forward_host(logits_host, x_host, w13, w13_scale, w2, w2_scale, sh, out_host, status_word, ws, stream=None):
+    _check(lib().moe_forward_host(_ptr(logits_host), _ptr(x_host), _ptr(w13), _ptr(w13_scale), _ptr(w2), _ptr(w2_scale),
+                                  C.byref(sh), _ptr(out_host), _ptr(status_word), _ptr(ws), ws.numel(), _stream(stream)),
+           "moe_forward_host")
+
+
+class LayerBuffers:
+    """Device buffers for the four calls on one shape (allocation only, no arithmetic)."""
+
+    def __init__(self, sh, device="cuda"):
+        S = sh.T * sh.k
+        dev = device
+        self.sh = sh
+        self.topk_ids = torch.empty((sh.T, sh.k), dtype=torch.int32, device=dev)
+        self.topk_w = torch.empty((sh.T, sh.k), dtype=torch.float32, device=dev)
+        self.expert_offsets = torch.empty(sh.E + 1, dtype=torch.int32, device=dev)
+        self.x_perm = torch.empty((S, sh.H), dtype=torch.bfloat16, device=dev)
+        self.perm = torch.empty(S, dtype=torch.int32, device=dev)
+        self.inv_perm = torch.empty(S, dtype=torch.int32, device=dev)
+        self.y_perm = torch.empty((S, sh.H), dtype=torch.float32, device=dev)
+        self.out = torch.empty((sh.T, sh.H), dtype=torch.bfloat16, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.ws = alloc_workspace(sh, dev)
+
+
+def moe_layer(logits, x, weights, buf, stream=None):
+    """route -> permute -> expert_ffn -> combine on device tensors; returns buf.out (enqueue only)."""
+    w13, s13, w2, s2 = weights
+    sh = buf.sh
+    moe_route(logits, sh.k, buf.topk_ids, buf.topk_w, buf.expert_offsets, buf.ws, stream)
+    moe_permute(x, buf.topk_ids, buf.expert_offsets, sh, buf.x_perm, buf.perm, buf.inv_perm, buf.ws, stream)
+    moe_expert_ffn(buf.x_perm, buf.expert_offsets, w13, s13, w2, s2, sh, buf.y_perm, buf.status, buf.ws, stream)
+    moe_combine(buf.y_perm, buf.inv_perm, buf.topk_w, sh, buf.out, stream)
+    return buf.out

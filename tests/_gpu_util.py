@@ -1,0 +1,68 @@
+"""Helpers for the GPU parity tests: numpy <-> torch marshalling and the parity metrics."""
+import numpy as np
+import torch
+
+from paper_2609_15627_b200 import inputs, moe
+
+
+def dev(a):
+    """numpy -> cuda tensor; uint16 arrays are bf16 bit patterns."""
+    if a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+    return torch.from_numpy(a).cuda()
+
+
+def bits(t):
+    """cuda bf16 tensor -> numpy uint16 bit patterns."""
+    return t.view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def weights_dev(d):
+    return tuple(dev(d[n]) for n in ("w13", "s13", "w2", "s2"))
+
+
+def run_layer(wl, d, wdev=None):
+    sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
+    buf = moe.LayerBuffers(sh)
+    wdev = wdev if wdev is not None else weights_dev(d)
+    out = moe.moe_layer(dev(d["logits"]), dev(d["x"]), wdev, buf)
+    torch.cuda.synchronize()
+    assert int(buf.status.item()) == 0
+    return buf, out
+
+
+def check_out(got_bits, ref_bits, ref_f32, what=""):
+    """The stated tolerance: rel-Frobenius <= 5e-3 and max|diff| <= 2e-2 * rms(reference).
+
+    An element over the max bound is accepted only if the GPU value is one of the two bf16
+    neighbours of the oracle's unrounded fp32 result (a rounding flip of one bf16 ulp).
+    """
+    got = inputs.bf16_bits_to_f32(got_bits).astype(np.float64)
+    ref = inputs.bf16_bits_to_f32(ref_bits).astype(np.float64)
+    rel = np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)
+    rms = np.sqrt(np.mean(ref ** 2))
+    diff = np.abs(got - ref)
+    over = diff > 2e-2 * rms
+    flips = 0
+    if over.any():
+        f = ref_f32[over].astype(np.float32)
+        lo = inputs.bf16_bits_to_f32((f.view(np.uint32) >> 16).astype(np.uint16))            # truncation
+        step = np.abs(lo) * 2.0 ** -7
+        hi = lo + np.sign(f) * np.where(step > 0, step, 2.0 ** -133)
+        g = got[over]
+        ok = (g == lo) | (g == hi.astype(np.float32))
+        assert ok.all(), "%s: %d elements beyond 2e-2*rms that are not bf16 rounding flips (max %g, rms %g)" % (
+            what, int((~ok).sum()), diff.max(), rms)
+        flips = int(over.sum())
+    assert rel <= 5e-3, "%s: rel-Frobenius %g" % (what, rel)
+    return dict(rel=rel, max_over_rms=float(diff.max() / rms), flips=flips)
+
+
+def check_y(got, ref, what=""):
+    got = got.astype(np.float64)
+    ref = ref.astype(np.float64)
+    rel = np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)
+    rms = np.sqrt(np.mean(ref ** 2))
+    mx = np.abs(got - ref).max() / max(rms, 1e-30)
+    assert rel <= 5e-4 and mx <= 2e-2, "%s: y_perm rel %g max/rms %g" % (what, rel, mx)
+    return dict(rel=rel, max_over_rms=float(mx))
