@@ -5,11 +5,11 @@
 // stage it is 16 consecutive rows of w2.  Rows of one expert matrix are contiguous in HBM, so a tile is
 // one or two contiguous blocks that the producer warp brings into a shared-memory ring with bulk
 // asynchronous copies (cp.async.bulk, completion on an mbarrier), packed: 4.25 bits per weight all the
-// way to shared memory.  Eight consumer warps split K, expand E2M1 codes to bf16 in registers (the three
+// way to shared memory.  Sixteen consumer warps split K, expand E2M1 codes to bf16 in registers (the three
 // magnitude bits dropped into the exponent/mantissa boundary of a bf16 give value * 2^-126 exactly; one
 // packed multiply by 2^(scale byte - 1) restores value * 2^(scale byte - 127), also exactly), and feed
 // m16n8k16 bf16 tensor-core MMAs whose n dimension holds up to 8 tokens of the expert.  Partial sums of
-// the eight warps are added in a fixed order through shared memory, so the result is deterministic.
+// the sixteen warps are added in a fixed order through shared memory, so the result is deterministic.
 //
 // K elements are assigned to MMA k slots in a permuted order (identically for weights and activations);
 // only the summation order inside the dot product depends on it.
@@ -19,9 +19,9 @@ namespace moe {
 
 namespace {
 
-constexpr int kConsumerWarps = 8;
+constexpr int kConsumerWarps = 16;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;  // + one producer warp
-constexpr int kMaxScPerWarp = 4;                     // 128-element K groups a warp keeps activations for
+constexpr int kMaxScPerWarp = 2;                     // 128-element K groups a warp keeps activations for
 constexpr int kSection = kConsumerWarps * kMaxScPerWarp * 128;  // K elements per register-resident pass
 constexpr long long kWaitLimitCycles = 4000000000LL;  // about two seconds
 
@@ -96,11 +96,15 @@ MOE_DEVINL uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
 // Eight E2M1 codes (one 32-bit word, element i in bits 4i+3:4i) -> four bf16x2 registers holding
 // elements (0,4), (1,5), (2,6), (3,7), each multiplied by `m` = bf16x2 of 2^(scale byte - 1).
 MOE_DEVINL void dequant8(uint32_t wd, uint32_t m, uint32_t (&p)[4]) {
-  constexpr uint32_t kMag = 0x01C001C0u, kSign = 0x80008000u;
-  p[0] = mul_bf16x2(((wd << 6) & kMag) | ((wd << 12) & kSign), m);
-  p[1] = mul_bf16x2(((wd << 2) & kMag) | ((wd << 8) & kSign), m);
-  p[2] = mul_bf16x2(((wd >> 2) & kMag) | ((wd << 4) & kSign), m);
-  p[3] = mul_bf16x2(((wd >> 6) & kMag) | (wd & kSign), m);
+  // A nibble n isolated at bit 0 (or 4) and multiplied by 2^6 + 2^12 (or 2^2 + 2^8) lands twice: its
+  // magnitude bits on bf16 bits 8:6 and its sign bit on bit 15; one mask removes the rest.  The integer
+  // multiply runs on the FMA pipe, which keeps the (half-rate) integer ALU pipe for the two masks.
+  constexpr uint32_t kKeep = 0x81C081C0u;
+  const uint32_t hi = wd >> 8;
+  p[0] = mul_bf16x2(((wd & 0x000F000Fu) * 0x1040u) & kKeep, m);
+  p[1] = mul_bf16x2(((wd & 0x00F000F0u) * 0x0104u) & kKeep, m);
+  p[2] = mul_bf16x2(((hi & 0x000F000Fu) * 0x1040u) & kKeep, m);
+  p[3] = mul_bf16x2(((hi & 0x00F000F0u) * 0x0104u) & kKeep, m);
 }
 
 // bf16x2 of (2^(b-1), 2^(b-1)) for a scale byte b in [0,128]
@@ -232,6 +236,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const FfnArgs a
 
       for (int row0 = row_begin; row0 < row_end; row0 += 8) {
         float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        float c2[4] = {0.0f, 0.0f, 0.0f, 0.0f};  // second chain: consecutive MMAs do not wait on each other
         const int my_row = (row0 + g < row_end) ? row0 + g : -2;
         for (int sec = 0; sec < n_sections; ++sec) {
           // ---- activations of this lane's row for this K section ----
@@ -274,14 +279,14 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const FfnArgs a
                 dequant8(wav[q], ma, pa);
                 dequant8(wbv[q], mb, pb);
                 mma_bf16_16x8x16(c, pa[0], pb[0], pa[1], pb[1], breg[j][4 * q + 0], breg[j][4 * q + 1]);
-                mma_bf16_16x8x16(c, pa[2], pb[2], pa[3], pb[3], breg[j][4 * q + 2], breg[j][4 * q + 3]);
+                mma_bf16_16x8x16(c2, pa[2], pb[2], pa[3], pb[3], breg[j][4 * q + 2], breg[j][4 * q + 3]);
               }
             }
           }
         }
         // ---- cross-warp reduction in fixed warp order, then the epilogue by one warp ----
         float* mine = red + ((red_buf * kConsumerWarps + wid) * 32 + lane) * 4;
-        *reinterpret_cast<float4*>(mine) = make_float4(c[0], c[1], c[2], c[3]);
+        *reinterpret_cast<float4*>(mine) = make_float4(c[0] + c2[0], c[1] + c2[1], c[2] + c2[2], c[3] + c2[3]);
         asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
         if (wid == (item_no & (kConsumerWarps - 1))) {
           float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
