@@ -110,8 +110,13 @@ int moe_expert_ffn(const void* x_perm_bf16, const int32_t* expert_offsets, const
   const WsLayout L = ws_layout(*shape);
   if (check_ws(ws, ws_bytes, L.total) != MOE_OK) return MOE_ERR_WORKSPACE;
   __nv_bfloat16* act = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(ws) + L.act_off);
-  return launch_expert_ffn(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w13, w13_scale, w2, w2_scale,
-                           *shape, act, y_perm, status_word, static_cast<cudaStream_t>(cuda_stream));
+  // kernel choice is a pure function of the shape: tensor-core grouped GEMM for prefill-sized batches,
+  // the weight-streaming kernel otherwise
+  if (umma_shape_ok(*shape))
+    return launch_expert_ffn_umma(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w13, w13_scale, w2,
+                                  w2_scale, *shape, act, y_perm, status_word, static_cast<cudaStream_t>(cuda_stream));
+  return launch_expert_ffn_stream(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w13, w13_scale, w2,
+                                  w2_scale, *shape, act, y_perm, status_word, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int moe_combine(const float* y_perm, const int32_t* inv_perm, const float* topk_w, const moe_shape_t* shape,

@@ -48,9 +48,15 @@ int launch_route(const float* logits, int T, int E, int k, int* ids, float* w, i
                  cudaStream_t st);
 int launch_permute(const __nv_bfloat16* x, const int* ids, const int* offsets, const moe_shape_t& s,
                    __nv_bfloat16* x_perm, int* perm, int* inv_perm, int* block_counts, cudaStream_t st);
-int launch_expert_ffn(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
-                      const uint8_t* w2, const uint8_t* s2, const moe_shape_t& s, __nv_bfloat16* act, float* y_perm,
-                      int* status_word, cudaStream_t st);
+// weight-streaming variant (any shape; the one for decode-sized batches)
+int launch_expert_ffn_stream(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
+                             const uint8_t* w2, const uint8_t* s2, const moe_shape_t& s, __nv_bfloat16* act, float* y_perm,
+                             int* status_word, cudaStream_t st);
+// tcgen05 grouped-GEMM variant (prefill-sized batches); umma_shape_ok says whether it applies
+bool umma_shape_ok(const moe_shape_t& s);
+int launch_expert_ffn_umma(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
+                           const uint8_t* w2, const uint8_t* s2, const moe_shape_t& s, __nv_bfloat16* act, float* y_perm,
+                           int* status_word, cudaStream_t st);
 int launch_combine(const float* y_perm, const int* inv_perm, const float* w, const moe_shape_t& s,
                    __nv_bfloat16* out, cudaStream_t st);
 int launch_validate_scales(const uint8_t* scales, size_t n, int* bad, cudaStream_t st);

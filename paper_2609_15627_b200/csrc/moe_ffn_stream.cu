@@ -13,7 +13,7 @@
 //
 // K elements are assigned to MMA k slots in a permuted order (identically for weights and activations);
 // only the summation order inside the dot product depends on it.
-#include "moe_common.cuh"
+#include "moe_sm100_primitives.cuh"
 
 namespace moe {
 
@@ -23,7 +23,6 @@ constexpr int kConsumerWarps = 16;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;  // + one producer warp
 constexpr int kMaxScPerWarp = 2;                     // 128-element K groups a warp keeps activations for
 constexpr int kSection = kConsumerWarps * kMaxScPerWarp * 128;  // K elements per register-resident pass
-constexpr long long kWaitLimitCycles = 4000000000LL;  // about two seconds
 
 struct FfnArgs {
   const uint8_t* w;           // [E, R, K/2] packed codes
@@ -37,48 +36,6 @@ struct FfnArgs {
   int n_stages;
 };
 
-// ---- mbarrier / bulk copy primitives ---------------------------------------------------------------
-MOE_DEVINL uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-MOE_DEVINL void mbar_init(uint64_t* bar, int count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-MOE_DEVINL void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-MOE_DEVINL void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-MOE_DEVINL bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait: gives up after kWaitLimitCycles, records MOE_ERR_TIMEOUT and lets the caller go on
-// (the data is then wrong, but every warp keeps taking part in every barrier, so nothing hangs).
-MOE_DEVINL void mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
-  if (mbar_try_wait(bar, parity)) return;
-  const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > kWaitLimitCycles) {
-      if (status != nullptr) atomicExch(status, static_cast<int>(MOE_ERR_TIMEOUT));
-      return;
-    }
-  }
-}
-MOE_DEVINL void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   smem_u32(dst)),
-               "l"(src), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
-}
-
 MOE_DEVINL void mma_bf16_16x8x16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                  uint32_t b1) {
   asm volatile(
@@ -86,29 +43,6 @@ MOE_DEVINL void mma_bf16_16x8x16(float (&c)[4], uint32_t a0, uint32_t a1, uint32
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-
-MOE_DEVINL uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
-  uint32_t d;
-  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-  return d;
-}
-
-// Eight E2M1 codes (one 32-bit word, element i in bits 4i+3:4i) -> four bf16x2 registers holding
-// elements (0,4), (1,5), (2,6), (3,7), each multiplied by `m` = bf16x2 of 2^(scale byte - 1).
-MOE_DEVINL void dequant8(uint32_t wd, uint32_t m, uint32_t (&p)[4]) {
-  // A nibble n isolated at bit 0 (or 4) and multiplied by 2^6 + 2^12 (or 2^2 + 2^8) lands twice: its
-  // magnitude bits on bf16 bits 8:6 and its sign bit on bit 15; one mask removes the rest.  The integer
-  // multiply runs on the FMA pipe, which keeps the (half-rate) integer ALU pipe for the two masks.
-  constexpr uint32_t kKeep = 0x81C081C0u;
-  const uint32_t hi = wd >> 8;
-  p[0] = mul_bf16x2(((wd & 0x000F000Fu) * 0x1040u) & kKeep, m);
-  p[1] = mul_bf16x2(((wd & 0x00F000F0u) * 0x0104u) & kKeep, m);
-  p[2] = mul_bf16x2(((hi & 0x000F000Fu) * 0x1040u) & kKeep, m);
-  p[3] = mul_bf16x2(((hi & 0x00F000F0u) * 0x0104u) & kKeep, m);
-}
-
-// bf16x2 of (2^(b-1), 2^(b-1)) for a scale byte b in [0,128]
-MOE_DEVINL uint32_t scale_mult(uint32_t b) { return ((b + 126u) << 7) * 0x00010001u; }
 
 }  // namespace
 
@@ -165,7 +99,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const FfnArgs a
         mbar_init(&full_bar[s], 1);
         mbar_init(&empty_bar[s], kConsumerWarps);
       }
-      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      mbar_fence_init();
     }
     __syncthreads();
   }
@@ -334,7 +268,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const FfnArgs a
   }
 }
 
-int launch_expert_ffn(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
+int launch_expert_ffn_stream(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
                       const uint8_t* w2, const uint8_t* s2, const moe_shape_t& sh, __nv_bfloat16* act, float* y_perm,
                       int* status_word, cudaStream_t st) {
   static bool attr_done = false;

@@ -395,3 +395,51 @@ def test_validate_scales_counts_out_of_range_bytes():
     moe.moe_validate_scales(dev(s), bad)
     torch.cuda.synchronize()
     assert int(bad.item()) == 3
+
+
+# ---- the tensor-core (tcgen05) expert FFN, reached when T*k >= 1024 and H, I are multiples of 256 ----
+
+@pytest.mark.parametrize("T,H,I,E,k,hot,seed", [
+    (600, 512, 256, 8, 2, False, 0),     # ~150 rows per expert: one accumulator, ragged N
+    (700, 512, 256, 4, 2, False, 1),     # ~350 rows per expert: second accumulator and a second pass
+    (1100, 256, 512, 8, 1, True, 2),     # one hot expert with ~1000 rows (4 passes), empty experts
+    (520, 1024, 256, 16, 2, False, 3),   # K = 1024 (several packed stages), few rows per expert
+])
+def test_ffn_tensor_core_path_against_oracle(T, H, I, E, k, hot, seed):
+    wl = inputs.Workload("umma", T, H, I, E, k)
+    w = inputs.make_expert_weights(H, I, E, seed=seed)
+    s13 = inputs.index_scales(2 * I, H, E, lo=117, span=6)
+    s2 = inputs.index_scales(H, I, E, lo=118, span=5)
+    w = (w[0], s13, w[2], s2)
+    logits = inputs.make_logits(T, E, seed=seed)
+    if hot:
+        logits[:, 2] += 8.0
+        logits[:, [5, 6]] -= 50.0
+    x = inputs.make_x(T, H, seed=seed)
+    ids, tw, off = O.route(logits, k)
+    x_perm, perm, inv = O.permute(x, ids, off)
+    sh = moe.shape(T, H, I, E, k)
+    buf = moe.LayerBuffers(sh)
+    moe.moe_expert_ffn(dev(x_perm), dev(off), *[dev(a) for a in w], sh, buf.y_perm, buf.status, buf.ws)
+    torch.cuda.synchronize()
+    assert int(buf.status.item()) == 0
+    assert moe.moe_last_kernel_name() == "ffn_umma_tcgen05_grouped"
+    ry = O.expert_ffn(x_perm, off, *w, k)
+    check_y(buf.y_perm.cpu().numpy(), ry, "tensor-core path")
+
+
+def test_kernel_choice_is_a_function_of_the_shape():
+    for (T, H, I, E, k, want) in [(16, 256, 128, 8, 2, "ffn_stream_bulk_ring_mma16816"),
+                                  (64, 512, 256, 8, 2, "ffn_stream_bulk_ring_mma16816"),
+                                  (512, 512, 256, 8, 2, "ffn_umma_tcgen05_grouped"),
+                                  (512, 384, 256, 8, 2, "ffn_stream_bulk_ring_mma16816")]:
+        wl = inputs.Workload("choice", T, H, I, E, k)
+        w = inputs.make_expert_weights(H, I, E, seed=0)
+        logits, x = inputs.make_logits(T, E, 0), inputs.make_x(T, H, 0)
+        ids, tw, off = O.route(logits, k)
+        x_perm, _, _ = O.permute(x, ids, off)
+        sh = moe.shape(T, H, I, E, k)
+        buf = moe.LayerBuffers(sh)
+        moe.moe_expert_ffn(dev(x_perm), dev(off), *[dev(a) for a in w], sh, buf.y_perm, buf.status, buf.ws)
+        torch.cuda.synchronize()
+        assert moe.moe_last_kernel_name() == want
