@@ -1,18 +1,21 @@
 // Expert FFN, tensor-core variant for prefill-sized batches: a persistent grouped GEMM on tcgen05.
 //
-// Roles inside the MMA: the M dimension (128 lanes of tensor memory) holds 128 weight rows, the N
-// dimension holds up to 320 tokens of one expert (two accumulators, N <= 256 and N <= 64), so the
-// padding of a ragged expert is at most 15 tokens and each packed weight is expanded once per pass.
-// A work item is (expert, pass of <= 320 tokens, tile of 128 weight rows).  For the gate/up stage a tile
-// is 64 gate rows (lanes 0..63) plus the matching 64 up rows (lanes 64..127).
+// Roles inside the MMA: the M dimension (128 lanes of tensor memory) holds weight rows, the N dimension
+// holds up to 256 tokens of one expert.  A work item is (expert, pass of <= 256 tokens, tile of 256 weight
+// rows); the 256 rows are two M=128 MMAs that share one token stage in shared memory (each token tile read
+// from L2 feeds twice the math) and own one 256-column accumulator each: all 512 columns of tensor memory.
+// An expert with more than 256 rows is cut into equal passes, so the padding of a ragged expert is at
+// most 15 tokens per pass.  For the gate/up stage each M=128 tile is 64 gate rows (lanes 0..63) plus the
+// matching 64 up rows (lanes 64..127).
 //
 // Warp roles (one CTA per SM, persistent):
-//   warp 0      producer: TMA loads of the token tile (bf16, 128-byte swizzle) and of the packed codes
-//   warp 1      allocates tensor memory, issues tcgen05.mma (one lane), commits to mbarriers
-//   warps 2..9  expand E2M1 -> bf16 (exact, scaled by the E8M0 block scale) from the packed stage into the
-//               swizzled K-major A stage the tensor core reads
-//   warps 10..13 epilogue: tcgen05.ld the accumulators, SwiGLU + bf16 rounding (stage 1, gate and up meet
-//               through shared memory) or the fp32 store (stage 2)
+//   warp 0       producer: TMA loads of the token tile (bf16, 128-byte swizzle) and of the packed codes
+//   warp 1       allocates tensor memory, issues tcgen05.mma (one lane), commits to mbarriers
+//   warps 2..9   one thread per weight row: packed E2M1 codes from the TMA-fed packed ring, exact expansion
+//                to bf16 scaled by the E8M0 block scale, written into the swizzled K-major A stage the
+//                tensor core reads
+//   warps 10..13 epilogue: tcgen05.ld the accumulators; stage 1 transposes through shared memory so that
+//                gate and up meet and act is stored 16 bytes at a time; stage 2 stores fp32 rows
 // Every mbarrier wait is bounded and reports through the status word.
 #include <cuda.h>
 
@@ -22,13 +25,11 @@ namespace moe {
 
 namespace {
 
-constexpr int kTileM = 128;       // weight rows per tile
+constexpr int kTileRows = 256;    // weight rows per work item: two M=128 MMA tiles
 constexpr int kBlockK = 64;       // K per pipeline stage: one 128-byte row of bf16
-constexpr int kMaxTok = 320;      // tokens per pass
+constexpr int kMaxTok = 256;      // tokens per pass
 constexpr int kTokBox = 64;       // token rows per TMA box
 constexpr int kStages = 3;        // A/B ring depth
-constexpr int kPackK = 256;       // K covered by one packed-code stage
-constexpr int kPackStages = 2;
 constexpr int kDequantWarps = 8;
 constexpr int kEpilogueWarps = 4;
 constexpr int kThreadsUmma = (2 + kDequantWarps + kEpilogueWarps) * 32;  // 448
@@ -36,12 +37,16 @@ constexpr int kFirstDequantWarp = 2;
 constexpr int kFirstEpilogueWarp = 2 + kDequantWarps;  // 10: (warp % 4) = 2,3,0,1 covers the four lane quadrants
 constexpr uint32_t kTmemCols = 512;
 
-constexpr int kABytes = kTileM * kBlockK * 2;        // 16 KB
-constexpr int kBBytes = kMaxTok * kBlockK * 2;       // 40 KB
-constexpr int kPBytes = kTileM * (kPackK / 2);       // 16 KB
-constexpr int kXchgBytes = 64 * 33 * 4;              // SwiGLU exchange: 64 up rows x 32 columns (+1 pad)
+constexpr int kATile = 128 * kBlockK * 2;            // 16 KB: one M=128 tile of a stage
+constexpr int kABytes = 2 * kATile;                  // 32 KB
+constexpr int kBBytes = kMaxTok * kBlockK * 2;       // 32 KB
+constexpr int kTChunk = 16;                          // accumulator columns per stage-1 epilogue step
+constexpr int kTBytes = kTChunk * 128 * 4;           // 8 KB transpose buffer
+constexpr int kPStages = 3;                          // packed-code ring (one K block per stage)
+constexpr int kPBytes = kTileRows * (kBlockK / 2);   // 8 KB: 256 rows x 32 bytes
 
 struct UmmaArgs {
+  const uint8_t* w;        // [E, R, K/2] packed codes
   const uint8_t* sc;       // [E, R, K/32] scale bytes
   const int* offsets;      // [E+1]
   __nv_bfloat16* act;      // stage 1 output [S, I]
@@ -51,7 +56,7 @@ struct UmmaArgs {
 };
 
 struct SmemMap {
-  uint32_t a, b, p, xchg, bars, misc, prefix, total;
+  uint32_t a, b, p, t, bars, misc, prefix, total;
 };
 __host__ __device__ inline SmemMap smem_map(int E) {
   SmemMap m;
@@ -61,9 +66,9 @@ __host__ __device__ inline SmemMap smem_map(int E) {
   m.b = off;
   off += kStages * kBBytes;
   m.p = off;
-  off += kPackStages * kPBytes;
-  m.xchg = off;
-  off += kXchgBytes;
+  off += kPStages * kPBytes;
+  m.t = off;
+  off += kTBytes;
   m.bars = off;
   off += 32 * 8;
   m.misc = off;
@@ -84,6 +89,17 @@ MOE_DEVINL int find_expert(const int* prefix, int E, int g) {
   return lo;
 }
 
+// rows [row0, row0 + ntok) of pass `pass` of an expert with rows [r_begin, r_end): equal passes, 16-aligned
+MOE_DEVINL void pass_rows(int r_begin, int r_end, int pass, int* row0, int* ntok) {
+  const int m = r_end - r_begin;
+  const int np = (m + kMaxTok - 1) / kMaxTok;
+  const int tp = (((m + np - 1) / np) + 15) & ~15;
+  *row0 = r_begin + pass * tp;
+  *ntok = min(tp, m - pass * tp);
+}
+
+MOE_DEVINL float silu_mul(float g, float u) { return __fdividef(g, 1.0f + __expf(-g)) * u; }
+
 }  // namespace
 
 template <bool STAGE1>
@@ -95,14 +111,14 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
   unsigned char* sA = smem + sm.a;
   unsigned char* sB = smem + sm.b;
   unsigned char* sP = smem + sm.p;
-  float* sX = reinterpret_cast<float*>(smem + sm.xchg);
+  float* sT = reinterpret_cast<float*>(smem + sm.t);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bars);
   uint64_t* full_a = bars;                      // [kStages] dequant warps -> MMA
   uint64_t* full_b = bars + kStages;            // [kStages] TMA -> MMA
   uint64_t* empty_ab = bars + 2 * kStages;      // [kStages] MMA done -> producer, dequant warps
-  uint64_t* full_p = bars + 3 * kStages;        // [kPackStages] TMA -> dequant warps
-  uint64_t* empty_p = full_p + kPackStages;     // [kPackStages] dequant warps -> producer
-  uint64_t* acc_full = empty_p + kPackStages;   // MMA -> epilogue
+  uint64_t* full_p = bars + 3 * kStages;        // [kPStages] TMA -> dequant warps
+  uint64_t* empty_p = full_p + kPStages;        // [kPStages] dequant warps -> producer
+  uint64_t* acc_full = empty_p + kPStages;      // MMA -> epilogue
   uint64_t* acc_empty = acc_full + 1;           // epilogue -> MMA
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + sm.misc);
   int* prefix = reinterpret_cast<int*>(smem + sm.prefix);
@@ -110,11 +126,10 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int K = a.K;
   const int num_kb = K / kBlockK;
-  const int tiles_per_expert = a.R / kTileM;
+  const int tiles_per_expert = a.R / kTileRows;
 
   // ---- setup: pass prefix over experts, barriers, tensor memory ----
   if (wid == 2) {
-    // one warp builds the exclusive prefix of ceil(rows / kMaxTok) over experts
     int run = 0;
     for (int e0 = 0; e0 < a.E; e0 += 32) {
       const int e = e0 + lane;
@@ -133,7 +148,7 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
       mbar_init(&full_b[s], 1);
       mbar_init(&empty_ab[s], 1);
     }
-    for (int s = 0; s < kPackStages; ++s) {
+    for (int s = 0; s < kPStages; ++s) {
       mbar_init(&full_p[s], 1);
       mbar_init(&empty_p[s], kDequantWarps);
     }
@@ -149,28 +164,25 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
   const int total_work = prefix[a.E] * tiles_per_expert;
 
   if (wid == 0) {
-    // =========================== producer ===========================
+    // =========================== producer: token tiles ===========================
     if (lane == 0) {
       int s = 0, ps = 0;
       uint32_t ph = 0, pph = 0;
       for (int w = blockIdx.x; w < total_work; w += gridDim.x) {
         const int g = w / tiles_per_expert, rt = w % tiles_per_expert;
         const int e = find_expert(prefix, a.E, g);
-        const int pass = g - prefix[e];
-        const int row0 = a.offsets[e] + pass * kMaxTok;
-        const int ntok = min(kMaxTok, a.offsets[e + 1] - row0);
+        int row0, ntok;
+        pass_rows(a.offsets[e], a.offsets[e + 1], g - prefix[e], &row0, &ntok);
         const int nbox = (ntok + kTokBox - 1) / kTokBox;
-        const int wrow_a = STAGE1 ? e * a.R + rt * 64 : e * a.R + rt * kTileM;
-        const int wrow_b = STAGE1 ? e * a.R + a.I + rt * 64 : wrow_a + 64;
+        // packed rows of the tile: stage 1 = 128 gate rows then the 128 matching up rows; stage 2 = 256 rows
+        const int wrow_a = STAGE1 ? e * a.R + rt * 128 : e * a.R + rt * kTileRows;
+        const int wrow_b = STAGE1 ? e * a.R + a.I + rt * 128 : wrow_a + 128;
         for (int kb = 0; kb < num_kb; ++kb) {
-          if ((kb & 3) == 0) {
-            mbar_wait(&empty_p[ps], pph ^ 1u, a.status);
-            mbar_expect_tx(&full_p[ps], kPBytes);
-            unsigned char* dst = sP + ps * kPBytes;
-            tma_load_2d(dst, &tmap_w, (kb >> 2) * (kPackK / 2), wrow_a, &full_p[ps]);
-            tma_load_2d(dst + 64 * (kPackK / 2), &tmap_w, (kb >> 2) * (kPackK / 2), wrow_b, &full_p[ps]);
-            if (++ps == kPackStages) { ps = 0; pph ^= 1u; }
-          }
+          mbar_wait(&empty_p[ps], pph ^ 1u, a.status);
+          mbar_expect_tx(&full_p[ps], kPBytes);
+          tma_load_2d(sP + ps * kPBytes, &tmap_w, kb * (kBlockK / 2), wrow_a, &full_p[ps]);
+          tma_load_2d(sP + ps * kPBytes + kPBytes / 2, &tmap_w, kb * (kBlockK / 2), wrow_b, &full_p[ps]);
+          if (++ps == kPStages) { ps = 0; pph ^= 1u; }
           mbar_wait(&empty_ab[s], ph ^ 1u, a.status);
           mbar_expect_tx(&full_b[s], static_cast<uint32_t>(nbox) * kTokBox * kBlockK * 2);
           for (int b = 0; b < nbox; ++b)
@@ -188,13 +200,10 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
       for (int w = blockIdx.x; w < total_work; w += gridDim.x) {
         const int g = w / tiles_per_expert;
         const int e = find_expert(prefix, a.E, g);
-        const int pass = g - prefix[e];
-        const int row0 = a.offsets[e] + pass * kMaxTok;
-        const int ntok = min(kMaxTok, a.offsets[e + 1] - row0);
+        int row0, ntok;
+        pass_rows(a.offsets[e], a.offsets[e + 1], g - prefix[e], &row0, &ntok);
         const int n16 = (ntok + 15) & ~15;
-        const int n1 = min(n16, 256), n2 = n16 - n1;
-        const uint32_t idesc1 = umma_idesc_bf16(kTileM, n1);
-        const uint32_t idesc2 = umma_idesc_bf16(kTileM, n2 > 0 ? n2 : 16);
+        const uint32_t idesc = umma_idesc_bf16(128, n16);
         mbar_wait(acc_empty, acc_ph ^ 1u, a.status);
         tc_fence_after_sync();
         for (int kb = 0; kb < num_kb; ++kb) {
@@ -205,10 +214,10 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
           const uint32_t b_addr = smem_u32(sB + s * kBBytes);
 #pragma unroll
           for (int k4 = 0; k4 < kBlockK / 16; ++k4) {
-            const uint64_t adesc = umma_desc_k_sw128(a_addr + k4 * 32);
+            const uint64_t bdesc = umma_desc_k_sw128(b_addr + k4 * 32);
             const uint32_t acc = (kb | k4) != 0 ? 1u : 0u;
-            umma_bf16(tmem_base, adesc, umma_desc_k_sw128(b_addr + k4 * 32), idesc1, acc);
-            if (n2 > 0) umma_bf16(tmem_base + 256, adesc, umma_desc_k_sw128(b_addr + 256 * 128 + k4 * 32), idesc2, acc);
+            umma_bf16(tmem_base, umma_desc_k_sw128(a_addr + k4 * 32), bdesc, idesc, acc);
+            umma_bf16(tmem_base + 256, umma_desc_k_sw128(a_addr + kATile + k4 * 32), bdesc, idesc, acc);
           }
           umma_commit(&empty_ab[s]);
           if (++s == kStages) { s = 0; ph ^= 1u; }
@@ -218,27 +227,49 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
       }
     }
   } else if (wid < kFirstEpilogueWarp) {
-    // =========================== E2M1 -> bf16 expansion ===========================
-    const int dt = tid - kFirstDequantWarp * 32;  // 0..255
-    const int row = dt >> 1, half = dt & 1;       // tile row, which 32 elements of the 64-wide K block
+    // =========================== E2M1 -> bf16 expansion, one thread per weight row ===========================
+    const int r = tid - kFirstDequantWarp * 32;   // 0..255
+    const int t = r >> 7, l = r & 127;            // MMA tile, lane (row) inside it
     int s = 0, ps = 0;
     uint32_t ph = 0, pph = 0;
     for (int w = blockIdx.x; w < total_work; w += gridDim.x) {
       const int g = w / tiles_per_expert, rt = w % tiles_per_expert;
       const int e = find_expert(prefix, a.E, g);
-      const int grow = STAGE1 ? e * a.R + (row < 64 ? rt * 64 + row : a.I + rt * 64 + (row - 64)) : e * a.R + rt * kTileM + row;
+      int grow;
+      if (STAGE1) {
+        const int i = rt * 128 + t * 64 + (l & 63);
+        grow = e * a.R + (l < 64 ? i : a.I + i);
+      } else {
+        grow = e * a.R + rt * kTileRows + r;
+      }
       const uint8_t* srow = a.sc + static_cast<size_t>(grow) * (K / 32);
+      // row of this thread inside the packed stage (stage 1: gate rows 0..127, up rows 128..255)
+      const int prow = STAGE1 ? (l < 64 ? t * 64 + l : 128 + t * 64 + (l - 64)) : r;
+      // scale bytes: 16 bytes cover 8 K blocks; fetched one group ahead
+      uint4 sc_cur = __ldg(reinterpret_cast<const uint4*>(srow));
+      uint4 sc_next = sc_cur;
+      unsigned char* arow_base = sA + t * kATile + l * 128;
       for (int kb = 0; kb < num_kb; ++kb) {
-        if ((kb & 3) == 0) mbar_wait(&full_p[ps], pph, a.status);
-        const uint32_t scale_byte = __ldg(srow + kb * 2 + half);
-        const uint4 codes = *reinterpret_cast<const uint4*>(sP + ps * kPBytes + row * (kPackK / 2) + (kb & 3) * 32 + half * 16);
-        const uint32_t m = scale_mult(scale_byte);
-        const uint32_t wv[4] = {codes.x, codes.y, codes.z, codes.w};
-        uint4 out[4];
+        if ((kb & 7) == 0) {
+          if (kb != 0) sc_cur = sc_next;
+          if (kb + 8 < num_kb) sc_next = __ldg(reinterpret_cast<const uint4*>(srow + (kb + 8) * 2));
+        }
+        const int sidx = (kb & 7) >> 1;  // 32-bit word of the 16 scale bytes; two bytes per K block
+        const uint32_t sword = (sidx == 0) ? sc_cur.x : (sidx == 1) ? sc_cur.y : (sidx == 2) ? sc_cur.z : sc_cur.w;
+        const uint32_t spair = sword >> ((kb & 1) * 16);
+        const uint32_t m_lo = scale_mult(spair & 0xFFu), m_hi = scale_mult((spair >> 8) & 0xFFu);
+        mbar_wait(&full_p[ps], pph, a.status);
+        const uint4 ca = *reinterpret_cast<const uint4*>(sP + ps * kPBytes + prow * 32);
+        const uint4 cb = *reinterpret_cast<const uint4*>(sP + ps * kPBytes + prow * 32 + 16);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty_p[ps]);
+        if (++ps == kPStages) { ps = 0; pph ^= 1u; }
+        const uint32_t wv[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
+        uint4 out[8];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
+        for (int q = 0; q < 8; ++q) {
           uint32_t p[4];
-          dequant8(wv[q], m, p);
+          dequant8(wv[q], q < 4 ? m_lo : m_hi, p);
           // (0,4),(1,5),(2,6),(3,7) -> natural order (0,1),(2,3),(4,5),(6,7)
           out[q].x = __byte_perm(p[0], p[1], 0x5410);
           out[q].y = __byte_perm(p[2], p[3], 0x5410);
@@ -246,66 +277,68 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
           out[q].w = __byte_perm(p[2], p[3], 0x7632);
         }
         mbar_wait(&empty_ab[s], ph ^ 1u, a.status);
-        unsigned char* arow = sA + s * kABytes + row * 128;
+        unsigned char* arow = arow_base + s * kABytes;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int chunk = half * 4 + q;  // 16-byte chunk of the 128-byte row
-          *reinterpret_cast<uint4*>(arow + ((chunk ^ (row & 7)) << 4)) = out[q];
-        }
+        for (int q = 0; q < 8; ++q) *reinterpret_cast<uint4*>(arow + ((q ^ (l & 7)) << 4)) = out[q];
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(&full_a[s]);
-          if ((kb & 3) == 3) mbar_arrive(&empty_p[ps]);
-        }
-        if ((kb & 3) == 3) {
-          if (++ps == kPackStages) { ps = 0; pph ^= 1u; }
-        }
+        if (lane == 0) mbar_arrive(&full_a[s]);
         if (++s == kStages) { s = 0; ph ^= 1u; }
       }
     }
   } else {
     // =========================== epilogue ===========================
-    const int q = wid & 3;  // tensor-memory lane quadrant this warp may read
+    const int q = wid & 3;                         // tensor-memory lane quadrant this warp may read
+    const int te = tid - kFirstEpilogueWarp * 32;  // 0..127
     const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
     uint32_t acc_ph = 0;
     for (int w = blockIdx.x; w < total_work; w += gridDim.x) {
       const int g = w / tiles_per_expert, rt = w % tiles_per_expert;
       const int e = find_expert(prefix, a.E, g);
-      const int pass = g - prefix[e];
-      const int row0 = a.offsets[e] + pass * kMaxTok;
-      const int ntok = min(kMaxTok, a.offsets[e + 1] - row0);
+      int row0, ntok;
+      pass_rows(a.offsets[e], a.offsets[e + 1], g - prefix[e], &row0, &ntok);
       mbar_wait(acc_full, acc_ph, a.status);
       tc_fence_after_sync();
-      for (int c0 = 0; c0 < ntok; c0 += 32) {
-        uint32_t v[32];
-        tmem_ld_32x32(tmem_base + lane_base + static_cast<uint32_t>(c0), v);
-        tmem_ld_wait();
+#pragma unroll 1
+      for (int t = 0; t < 2; ++t) {
+        const uint32_t tcol = tmem_base + lane_base + static_cast<uint32_t>(t * 256);
         if (STAGE1) {
-          // lanes 0..63 hold gate rows, lanes 64..127 the matching up rows: up goes through shared memory
-          if (q >= 2) {
+          // lanes 0..63 hold gate rows, lanes 64..127 the matching up rows.  Transpose 16 columns through
+          // shared memory (sT[column][lane]); then thread (column j, segment) owns 8 consecutive i of token j.
+          const int j = te >> 3, seg = te & 7;
+          const int ibase = rt * 128 + t * 64 + seg * 8;
+          for (int c0 = 0; c0 < ntok; c0 += kTChunk) {
+            uint32_t v[16];
+            tmem_ld_32x16(tcol + static_cast<uint32_t>(c0), v);
+            tmem_ld_wait();
+            float* tb = sT;
+            asm volatile("bar.sync 2, %0;" ::"n"(kEpilogueWarps * 32) : "memory");  // previous chunk fully read
 #pragma unroll
-            for (int j = 0; j < 32; ++j) sX[((q - 2) * 32 + lane) * 33 + j] = __uint_as_float(v[j]);
-          }
-          asm volatile("bar.sync 2, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
-          if (q < 2) {
-            const int i = rt * 64 + q * 32 + lane;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              if (c0 + j < ntok) {
-                const float gv = __uint_as_float(v[j]);
-                const float uv = sX[(q * 32 + lane) * 33 + j];
-                const float r = (gv / (1.0f + __expf(-gv))) * uv;
-                a.act[static_cast<size_t>(row0 + c0 + j) * a.I + i] = __float2bfloat16_rn(r);
-              }
+            for (int jj = 0; jj < 16; ++jj) tb[jj * 128 + q * 32 + lane] = __uint_as_float(v[jj]);
+            asm volatile("bar.sync 2, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
+            if (c0 + j < ntok) {
+              const float4 g0 = *reinterpret_cast<const float4*>(tb + j * 128 + seg * 8);
+              const float4 g1 = *reinterpret_cast<const float4*>(tb + j * 128 + seg * 8 + 4);
+              const float4 u0 = *reinterpret_cast<const float4*>(tb + j * 128 + 64 + seg * 8);
+              const float4 u1 = *reinterpret_cast<const float4*>(tb + j * 128 + 64 + seg * 8 + 4);
+              __nv_bfloat162 o[4];
+              o[0] = __floats2bfloat162_rn(silu_mul(g0.x, u0.x), silu_mul(g0.y, u0.y));
+              o[1] = __floats2bfloat162_rn(silu_mul(g0.z, u0.z), silu_mul(g0.w, u0.w));
+              o[2] = __floats2bfloat162_rn(silu_mul(g1.x, u1.x), silu_mul(g1.y, u1.y));
+              o[3] = __floats2bfloat162_rn(silu_mul(g1.z, u1.z), silu_mul(g1.w, u1.w));
+              *reinterpret_cast<uint4*>(a.act + static_cast<size_t>(row0 + c0 + j) * a.I + ibase) = *reinterpret_cast<uint4*>(o);
             }
           }
-          asm volatile("bar.sync 2, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
         } else {
-          const int n = rt * kTileM + q * 32 + lane;
+          const int n = rt * kTileRows + t * 128 + q * 32 + lane;
+          for (int c0 = 0; c0 < ntok; c0 += 32) {
+            uint32_t v[32];
+            tmem_ld_32x32(tcol + static_cast<uint32_t>(c0), v);
+            tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (c0 + j < ntok) a.y[static_cast<size_t>(row0 + c0 + j) * a.R + n] = __uint_as_float(v[j]);
+            for (int jj = 0; jj < 32; ++jj)
+              if (c0 + jj < ntok) a.y[static_cast<size_t>(row0 + c0 + jj) * a.R + n] = __uint_as_float(v[jj]);
+          }
         }
       }
       tc_fence_before_sync();
@@ -358,7 +391,9 @@ bool make_map_2d(CUtensorMap* m, CUtensorMapDataType dt, int elem_bytes, const v
 }  // namespace
 
 bool umma_shape_ok(const moe_shape_t& sh) {
-  return sh.H % kPackK == 0 && sh.I % kPackK == 0 && static_cast<long long>(sh.T) * sh.k >= 1024 &&
+  // K % 512: a row's scale bytes (K/32 of them) are then 16-byte aligned for the vector prefetch;
+  // rows per expert (2I and H) are then whole 256-row tiles
+  return sh.H % 512 == 0 && sh.I % 512 == 0 && static_cast<long long>(sh.T) * sh.k >= 1024 &&
          smem_map(sh.E).total + 1024 <= 227 * 1024;
 }
 
@@ -377,9 +412,9 @@ int launch_expert_ffn_umma(const __nv_bfloat16* x_perm, const int* offsets, cons
   CUtensorMap tm_x, tm_act, tm_w13, tm_w2;
   if (!make_map_2d(&tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, x_perm, sh.H, S, kBlockK, kTokBox, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !make_map_2d(&tm_act, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, act, sh.I, S, kBlockK, kTokBox, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !make_map_2d(&tm_w13, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w13, sh.H / 2, static_cast<uint64_t>(sh.E) * 2 * sh.I,
-                   kPackK / 2, 64, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-      !make_map_2d(&tm_w2, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w2, sh.I / 2, static_cast<uint64_t>(sh.E) * sh.H, kPackK / 2, 64,
+      !make_map_2d(&tm_w13, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w13, sh.H / 2, static_cast<uint64_t>(sh.E) * 2 * sh.I, kBlockK / 2,
+                   128, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+      !make_map_2d(&tm_w2, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w2, sh.I / 2, static_cast<uint64_t>(sh.E) * sh.H, kBlockK / 2, 128,
                    CU_TENSOR_MAP_SWIZZLE_NONE))
     return MOE_ERR_CUDA;
   const int grid = sm_count();
@@ -390,11 +425,13 @@ int launch_expert_ffn_umma(const __nv_bfloat16* x_perm, const int* offsets, cons
   a.status = status_word;
   a.E = sh.E;
   a.I = sh.I;
+  a.w = w13;
   a.sc = s13;
   a.K = sh.H;
   a.R = 2 * sh.I;
   ffn_umma_kernel<true><<<grid, kThreadsUmma, smem, st>>>(tm_x, tm_w13, a);
   if (cudaGetLastError() != cudaSuccess) return MOE_ERR_CUDA;
+  a.w = w2;
   a.sc = s2;
   a.K = sh.I;
   a.R = sh.H;

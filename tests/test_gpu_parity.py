@@ -397,13 +397,13 @@ def test_validate_scales_counts_out_of_range_bytes():
     assert int(bad.item()) == 3
 
 
-# ---- the tensor-core (tcgen05) expert FFN, reached when T*k >= 1024 and H, I are multiples of 256 ----
+# ---- the tensor-core (tcgen05) expert FFN, reached when T*k >= 1024 and H, I are multiples of 512 ----
 
 @pytest.mark.parametrize("T,H,I,E,k,hot,seed", [
-    (600, 512, 256, 8, 2, False, 0),     # ~150 rows per expert: one accumulator, ragged N
-    (700, 512, 256, 4, 2, False, 1),     # ~350 rows per expert: second accumulator and a second pass
-    (1100, 256, 512, 8, 1, True, 2),     # one hot expert with ~1000 rows (4 passes), empty experts
-    (520, 1024, 256, 16, 2, False, 3),   # K = 1024 (several packed stages), few rows per expert
+    (600, 512, 512, 8, 2, False, 0),     # ~150 rows per expert: one accumulator, ragged N
+    (700, 512, 512, 4, 2, False, 1),     # ~350 rows per expert: second accumulator and a second pass
+    (1100, 512, 512, 8, 1, True, 2),     # one hot expert with ~1000 rows (4 passes), empty experts
+    (520, 1024, 512, 16, 2, False, 3),   # K = 1024 (several packed stages), few rows per expert
 ])
 def test_ffn_tensor_core_path_against_oracle(T, H, I, E, k, hot, seed):
     wl = inputs.Workload("umma", T, H, I, E, k)
@@ -431,8 +431,8 @@ def test_ffn_tensor_core_path_against_oracle(T, H, I, E, k, hot, seed):
 def test_kernel_choice_is_a_function_of_the_shape():
     for (T, H, I, E, k, want) in [(16, 256, 128, 8, 2, "ffn_stream_bulk_ring_mma16816"),
                                   (64, 512, 256, 8, 2, "ffn_stream_bulk_ring_mma16816"),
-                                  (512, 512, 256, 8, 2, "ffn_umma_tcgen05_grouped"),
-                                  (512, 384, 256, 8, 2, "ffn_stream_bulk_ring_mma16816")]:
+                                  (512, 512, 512, 8, 2, "ffn_umma_tcgen05_grouped"),
+                                  (512, 512, 256, 8, 2, "ffn_stream_bulk_ring_mma16816")]:
         wl = inputs.Workload("choice", T, H, I, E, k)
         w = inputs.make_expert_weights(H, I, E, seed=0)
         logits, x = inputs.make_logits(T, E, 0), inputs.make_x(T, H, 0)
