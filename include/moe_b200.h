@@ -138,6 +138,33 @@ int moe_forward_host(const float* logits_host, const void* x_host_bf16, const ui
                      const moe_shape_t* shape, void* out_host_bf16, int32_t* status_word, void* ws,
                      size_t ws_bytes, void* cuda_stream);
 
+/*
+ * moe_expert_ffn without a workspace argument, for callers that cannot allocate device memory
+ * (the paper has no counterpart: this is a packaging variant of moe_expert_ffn, same arithmetic).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - a plug-in called inside another
+ * framework's stream-ordered or graph-managed section, a real-time loop that must not touch the driver's
+ * allocator, a host that hands this library pre-made buffers for inputs and outputs only.  Such a caller
+ * still passes every input and output, but not the scratch: the bf16 intermediate act[T*k, I] is kept in a
+ * fixed array of moe_expert_ffn_noalloc_max_bytes() = 8 MiB inside the library image (each GPU that loads
+ * the library holds those 8 MiB until the process exits).
+ *
+ *   - Sizes: 2*T*k*I bytes must fit the array, else MOE_ERR_WORKSPACE and nothing is launched
+ *     (decode-sized batches: up to 2048 slots at I = 2048).  Other argument rules as moe_expert_ffn.
+ *   - The call allocates and frees nothing and calls no allocating library routine.  Its first call on a
+ *     device looks up the array's device address (one runtime query, cached per device): make that first
+ *     call outside any stream capture.
+ *   - All calls share the one array and it keeps the last call's contents.  Nothing in it needs to start
+ *     at zero (each call writes every row it later reads), but two calls that overlap on the GPU - other
+ *     streams, other host threads - race on it: keep calls on one stream or order them yourself.
+ *   - Result: identical to moe_expert_ffn on the same inputs (same kernels, same kernel choice).
+ */
+size_t moe_expert_ffn_noalloc_max_bytes(void);
+int moe_expert_ffn_noalloc(const void* x_perm_bf16 /* [T*k,H] */, const int32_t* expert_offsets, const uint8_t* w13,
+                           const uint8_t* w13_scale, const uint8_t* w2, const uint8_t* w2_scale,
+                           const moe_shape_t* shape, float* y_perm /* [T*k,H] */, int32_t* status_word,
+                           void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

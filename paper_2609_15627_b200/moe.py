@@ -14,7 +14,8 @@ LIB_PATH = os.path.join(_HERE, "libmoe_b200.so")
 
 EXPORTS = ("moe_workspace_bytes", "moe_status_string", "moe_last_kernel_name", "moe_launch_count", "moe_route",
            "moe_permute", "moe_expert_ffn", "moe_combine", "moe_validate_scales",
-           "moe_forward_host_workspace_bytes", "moe_forward_host")
+           "moe_forward_host_workspace_bytes", "moe_forward_host", "moe_expert_ffn_noalloc_max_bytes",
+           "moe_expert_ffn_noalloc")
 
 
 class MoeError(RuntimeError):
@@ -54,6 +55,9 @@ def lib():
         L.moe_combine.argtypes = [vp, vp, vp, C.POINTER(Shape), vp, vp]
         L.moe_validate_scales.restype = C.c_int
         L.moe_validate_scales.argtypes = [vp, sz, vp, vp]
+        L.moe_expert_ffn_noalloc_max_bytes.restype = sz
+        L.moe_expert_ffn_noalloc.restype = C.c_int
+        L.moe_expert_ffn_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp]
         L.moe_forward_host.restype = C.c_int
         L.moe_forward_host.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp, sz, vp]
         _lib = L
@@ -116,6 +120,18 @@ def moe_expert_ffn(x_perm, expert_offsets, w13, w13_scale, w2, w2_scale, sh, y_p
     _check(lib().moe_expert_ffn(_ptr(x_perm), _ptr(expert_offsets), _ptr(w13), _ptr(w13_scale), _ptr(w2), _ptr(w2_scale),
                                 C.byref(sh), _ptr(y_perm), _ptr(status_word), _ptr(ws), ws.numel(), _stream(stream)),
            "moe_expert_ffn")
+
+
+def moe_expert_ffn_noalloc_max_bytes():
+    return int(lib().moe_expert_ffn_noalloc_max_bytes())
+
+
+def moe_expert_ffn_noalloc(x_perm, expert_offsets, w13, w13_scale, w2, w2_scale, sh, y_perm, status_word, stream=None):
+    """moe_expert_ffn for callers that cannot allocate: no workspace argument, the intermediate lives in a
+    fixed 8 MiB array inside the library (see include/moe_b200.h for the limits and the sharing rules)."""
+    _check(lib().moe_expert_ffn_noalloc(_ptr(x_perm), _ptr(expert_offsets), _ptr(w13), _ptr(w13_scale), _ptr(w2),
+                                        _ptr(w2_scale), C.byref(sh), _ptr(y_perm), _ptr(status_word), _stream(stream)),
+           "moe_expert_ffn_noalloc")
 
 
 def moe_combine(y_perm, inv_perm, topk_w, sh, out, stream=None):
