@@ -110,8 +110,12 @@ int moe_expert_ffn(const void* x_perm_bf16, const int32_t* expert_offsets, const
   const WsLayout L = ws_layout(*shape);
   if (check_ws(ws, ws_bytes, L.total) != MOE_OK) return MOE_ERR_WORKSPACE;
   __nv_bfloat16* act = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(ws) + L.act_off);
-  // kernel choice is a pure function of the shape: tensor-core grouped GEMM for prefill-sized batches,
-  // the weight-streaming kernel otherwise
+  // kernel choice is a pure function of the shape (and of the 32-byte alignment the 4-bit tensor map needs):
+  // native block-scaled FP4 MMA for decode-sized batches, bf16 grouped GEMM for prefill-sized batches, the
+  // register-expansion streaming kernel for every other shape
+  if (native_shape_ok(*shape, w13, w2))
+    return launch_expert_ffn_native(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w13, w13_scale, w2,
+                                    w2_scale, *shape, act, y_perm, status_word, static_cast<cudaStream_t>(cuda_stream));
   if (umma_shape_ok(*shape))
     return launch_expert_ffn_umma(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w13, w13_scale, w2,
                                   w2_scale, *shape, act, y_perm, status_word, static_cast<cudaStream_t>(cuda_stream));

@@ -29,8 +29,8 @@ inline WsLayout ws_layout(const moe_shape_t& s) {
   size_t off = 0;
   L.route_off = off;  // moe_route is given only (T, E, k): its block must not depend on H or I
   off += align_up((static_cast<size_t>(s.E) + 8) * 4, kAlign);
-  L.act_off = off;
-  off += align_up(S * s.I * 2, kAlign);
+  L.act_off = off;  // bf16 act[S,I], or the split E4M3 pair [2S,I] with its scale bytes [2S,I/32]
+  off += align_up(S * s.I * 2, kAlign) + align_up(2 * S * (s.I / 32), kAlign) + kAlign;
   L.permute_off = off;
   const size_t nblk = (S + kPermuteChunk - 1) / kPermuteChunk;
   off += align_up(nblk * s.E * 4, kAlign);
@@ -60,6 +60,13 @@ int launch_expert_ffn_umma(const __nv_bfloat16* x_perm, const int* offsets, cons
 int launch_combine(const float* y_perm, const int* inv_perm, const float* w, const moe_shape_t& s,
                    __nv_bfloat16* out, cudaStream_t st);
 int launch_validate_scales(const uint8_t* scales, size_t n, int* bad, cudaStream_t st);
+
+// native block-scaled FP4 variant (decode-sized batches); scratch holds the split activations
+bool native_shape_ok(const moe_shape_t& s, const void* w13, const void* w2);
+size_t native_scratch_bytes(const moe_shape_t& s);
+int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
+                             const uint8_t* w2, const uint8_t* s2, const moe_shape_t& s, void* scratch, float* y_perm,
+                             int* status_word, cudaStream_t st);
 
 int sm_count();
 

@@ -1,0 +1,583 @@
+// Expert FFN for decode-sized batches on the native block-scaled FP4 tensor-core path:
+// packed E2M1 codes and E8M0 scales go HBM -> TMA -> shared memory -> tcgen05.mma with no ALU expansion.
+//
+// tcgen05.mma kind::mxf8f6f4.block_scale multiplies an E2M1 operand by an E4M3 operand with one UE8M0 scale per
+// 32 K elements on both sides - the checkpoint format of the expert weights is exactly its A operand.  The
+// activations are bf16, so each row is split on the fly into two E4M3 rows with their own block scales,
+//   x = 2^s * hi + 2^(s-3) * lo,   hi = e4m3(x / 2^s),   lo = e4m3((x / 2^s - hi) * 8),
+// which is exact for every element within 2^14 of its block's maximum (8 significant bits = 4 + 4) and loses
+// less than 2^-19 of the block maximum otherwise; products are exact and accumulate in fp32 in tensor memory.
+// An MMA has M = 128 weight rows, N = 16 (8 tokens x {hi, lo}), K = 32; the two halves are added in the epilogue.
+//
+// Work item = (touched expert, tile of 128 weight rows) over the full K (stage 1: 64 gate + 64 up rows).
+// Warp roles (one persistent CTA per SM):
+//   warp 0      producer: TMA loads of the weight tile (4-bit tensor map that unpacks to the 16-byte-aligned
+//               operand layout, 128-byte swizzle) and of the scale bytes
+//   warp 1      allocates tensor memory, issues the MMAs, commits to mbarriers
+//   warps 2..5  move scale bytes into tensor memory (tcgen05.st), and at an expert change split that expert's
+//               token rows into the E4M3 pair and lay them out as the B operand
+//   warps 6..9  epilogue: hi + lo, SwiGLU + bf16 rounding + re-split for stage 2 (stage 1) or fp32 store (stage 2)
+// Every wait is bounded and reports through the status word.
+#include <cuda.h>
+#include <cuda_fp8.h>
+
+#include "moe_sm100_primitives.cuh"
+
+namespace moe {
+
+namespace {
+
+constexpr int kTile = 128;            // weight rows per item
+constexpr int kKStep = 128;           // K elements per A stage (one 128-byte swizzled row per weight row)
+constexpr int kAStage = kTile * 128;  // 16 KB of shared memory per stage (8 KB of HBM bytes)
+constexpr int kAStages = 8;
+constexpr int kScStages = 3;          // scale-byte ring: one stage = 128 rows x 16 bytes = 4 K steps
+constexpr int kScStage = kTile * 16;
+constexpr int kSfGroups = 3;          // tensor-memory groups for the A scale factors: 4 K steps x 4 columns each
+constexpr int kMaxTokPass = 8;        // tokens per pass (N = 16)
+constexpr int kMaxK = 4096;           // B operand of one expert stays resident: 16 rows x K bytes
+constexpr int kNatThreads = 10 * 32;
+constexpr uint32_t kNatTmemCols = 256;
+// tensor-memory columns: two 16-column accumulators, 3 A-scale groups of 16 columns, and 4 columns per K step for
+// the B scales (a scale-factor block is 4 columns wide - rows 32c..32c+31 in column c - and must start on a
+// multiple of 4 columns; with N = 16 only its first column carries data)
+constexpr uint32_t kColD = 0, kColSfa = 32, kColSfb = 96;
+
+struct NatArgs {
+  const __nv_bfloat16* x;    // stage 1: sorted token rows [S, K]
+  const uint8_t* aq;         // stage 2 input / stage 1 output: split activations [2S, I] (row 2p hi, 2p+1 lo)
+  const uint8_t* aq_sf;      //   and their scale bytes [2S, I/32]
+  uint8_t* aq_out;
+  uint8_t* aq_sf_out;
+  const int* offsets;
+  float* y;                  // stage 2 output [S, R]
+  int* status;
+  int E, K, R, I;
+};
+
+struct NatSmem {
+  uint32_t a, b, sc, sfb, xchg, bars, misc, touched, total;
+};
+__host__ __device__ inline NatSmem nat_smem(int E, int K) {
+  NatSmem m;
+  uint32_t off = 0;
+  m.a = off;
+  off += kAStages * kAStage;
+  m.b = off;
+  off += 16 * static_cast<uint32_t>(K);
+  m.sc = off;
+  off += kScStages * kScStage;
+  m.sfb = off;
+  off += 16 * (static_cast<uint32_t>(K) / 32);  // multiple of 256 for K % 512 == 0: keeps 16-byte alignment
+  m.xchg = off;
+  off += 64 * 9 * 4;
+  m.bars = off;
+  off += 64 * 8;
+  m.misc = off;
+  off += 64;
+  m.touched = off;
+  off += (static_cast<uint32_t>(E) + 8) * 4;
+  m.total = off;
+  return m;
+}
+
+MOE_DEVINL void tmem_st_32x4(uint32_t taddr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1,%2,%3,%4};" ::"r"(taddr), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
+               : "memory");
+}
+MOE_DEVINL void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem, E2M1] * B[smem, E4M3]^T with UE8M0 block scales held in tensor memory
+MOE_DEVINL void umma_mxf4(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t sfa, uint32_t sfb,
+                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+      :
+      : "r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
+      : "memory");
+}
+// instruction descriptor: A E2M1, B E4M3, UE8M0 scales, M = 128, N = 16; `j` picks byte j of the scale words
+MOE_DEVINL uint32_t idesc_mxf4(uint32_t j) {
+  return (5u << 7) | (0u << 10) | ((16u >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24) | (j << 29) | (j << 4);
+}
+
+MOE_DEVINL float e4m3_to_float(uint32_t byte) {
+  const __half_raw h = __nv_cvt_fp8_to_halfraw(static_cast<__nv_fp8_storage_t>(byte), __NV_E4M3);
+  return __half2float(*reinterpret_cast<const __half*>(&h));
+}
+MOE_DEVINL uint32_t float_to_e4m3(float v) {
+  return static_cast<uint32_t>(__nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E4M3));
+}
+// Block scale exponent for a block whose largest magnitude is amax (> 0): values / 2^s lie in [128, 256)
+MOE_DEVINL int block_exp(float amax) { return static_cast<int>((__float_as_uint(amax) >> 23) & 0xFFu) - 127 - 7; }
+// v (already divided by the block scale) -> (hi, lo) E4M3 bytes with v = hi + lo / 8
+MOE_DEVINL void split_e4m3(float v, uint32_t* hi, uint32_t* lo) {
+  const uint32_t h = float_to_e4m3(v);
+  *hi = h;
+  *lo = float_to_e4m3((v - e4m3_to_float(h)) * 8.0f);
+}
+MOE_DEVINL float pow2f(int e) { return __uint_as_float(static_cast<uint32_t>(e + 127) << 23); }  // e in [-126, 127]
+
+}  // namespace
+
+template <bool STAGE1>
+__global__ void __launch_bounds__(kNatThreads, 1)
+ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_sc, const NatArgs a) {
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  const int K = a.K;
+  const NatSmem sm = nat_smem(a.E, K);
+  unsigned char* sA = smem + sm.a;
+  unsigned char* sB = smem + sm.b;      // [K/128 steps][16 rows][128 bytes], 128-byte swizzle
+  unsigned char* sSc = smem + sm.sc;    // ring of [128 rows][16 bytes]
+  unsigned char* sSfb = smem + sm.sfb;  // [16 rows][K/32] scale bytes of the B rows
+  float* sX = reinterpret_cast<float*>(smem + sm.xchg);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bars);
+  uint64_t* full_a = bars;                       // [kAStages]  TMA -> MMA
+  uint64_t* empty_a = full_a + kAStages;         // [kAStages]  MMA done -> producer
+  uint64_t* full_sc = empty_a + kAStages;        // [kScStages] TMA -> scale warps
+  uint64_t* empty_sc = full_sc + kScStages;      // [kScStages] scale warps -> producer
+  uint64_t* sf_full = empty_sc + kScStages;      // [kSfGroups] scale warps -> MMA
+  uint64_t* sf_free = sf_full + kSfGroups;       // [kSfGroups] MMA done -> scale warps
+  uint64_t* acc_full = sf_free + kSfGroups;      // [2] MMA -> epilogue
+  uint64_t* acc_empty = acc_full + 2;            // [2] epilogue -> MMA
+  uint64_t* b_ready = acc_empty + 2;             // scale warps -> MMA: B operand of the current (expert, pass) is in place
+  uint64_t* b_free = b_ready + 1;                // MMA done with the B operand -> scale warps
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + sm.misc);
+  int* touched = reinterpret_cast<int*>(smem + sm.touched);
+  int* s_misc = touched + a.E;
+
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int n_steps = K / kKStep;
+  const int tiles_per_expert = a.R / kTile;
+
+  // ---- setup: touched experts, barriers, tensor memory ----
+  if (wid == 2) {
+    int run = 0;
+    for (int e0 = 0; e0 < a.E; e0 += 32) {
+      const int e = e0 + lane;
+      const int has = (e < a.E && a.offsets[e + 1] > a.offsets[e]) ? 1 : 0;
+      int tot;
+      const int ex = warp_excl_scan(has, lane, &tot);
+      if (has) touched[run + ex] = e;
+      run += tot;
+    }
+    if (lane == 0) s_misc[0] = run;
+  }
+  if (tid == 0) {
+    for (int s = 0; s < kAStages; ++s) { mbar_init(&full_a[s], 1); mbar_init(&empty_a[s], 1); }
+    for (int s = 0; s < kScStages; ++s) { mbar_init(&full_sc[s], 1); mbar_init(&empty_sc[s], 4); }
+    for (int s = 0; s < kSfGroups; ++s) { mbar_init(&sf_full[s], 4); mbar_init(&sf_free[s], 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4); }
+    mbar_init(b_ready, 4);
+    mbar_init(b_free, 1);
+    mbar_fence_init();
+  }
+  if (wid == 1) tmem_alloc(tmem_holder, kNatTmemCols);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_holder;
+  const int n_touched = s_misc[0];
+  const long long total_items = static_cast<long long>(n_touched) * tiles_per_expert;
+  const long long per_cta = (total_items + gridDim.x - 1) / gridDim.x;
+  const long long item_begin = static_cast<long long>(blockIdx.x) * per_cta;
+  const long long item_end = min(item_begin + per_cta, total_items);
+  // Every role walks the same sequence: for each item, for each pass of up to 8 tokens, all K steps.
+
+  if (wid == 0) {
+    // =========================== producer ===========================
+    if (lane == 0) {
+      int s = 0, cs = 0;
+      uint32_t ph = 0, cph = 0;
+      for (long long it = item_begin; it < item_end; ++it) {
+        const int e = touched[it / tiles_per_expert];
+        const int tile = static_cast<int>(it % tiles_per_expert);
+        const int rows = a.offsets[e + 1] - a.offsets[e];
+        const int n_pass = (rows + kMaxTokPass - 1) / kMaxTokPass;
+        const int wrow_a = STAGE1 ? e * a.R + tile * 64 : e * a.R + tile * kTile;
+        const int wrow_b = STAGE1 ? e * a.R + a.I + tile * 64 : wrow_a + 64;
+        for (int pass = 0; pass < n_pass; ++pass) {
+          for (int ks = 0; ks < n_steps; ++ks) {
+            if ((ks & 3) == 0) {
+              mbar_wait(&empty_sc[cs], cph ^ 1u, a.status);
+              mbar_expect_tx(&full_sc[cs], kScStage);
+              tma_load_2d(sSc + cs * kScStage, &tmap_sc, ks * 4, wrow_a, &full_sc[cs]);
+              tma_load_2d(sSc + cs * kScStage + 64 * 16, &tmap_sc, ks * 4, wrow_b, &full_sc[cs]);
+              if (++cs == kScStages) { cs = 0; cph ^= 1u; }
+            }
+            mbar_wait(&empty_a[s], ph ^ 1u, a.status);
+            mbar_expect_tx(&full_a[s], kAStage / 2);  // the transaction count is in packed (global) bytes
+            tma_load_2d(sA + s * kAStage, &tmap_w, ks * kKStep, wrow_a, &full_a[s]);
+            tma_load_2d(sA + s * kAStage + 64 * 128, &tmap_w, ks * kKStep, wrow_b, &full_a[s]);
+            if (++s == kAStages) { s = 0; ph ^= 1u; }
+          }
+        }
+      }
+    }
+  } else if (wid == 1) {
+    // =========================== MMA issuer ===========================
+    if (lane == 0) {
+      int s = 0, slot = 0, buf = 0;
+      uint32_t ph = 0, sph = 0, bph = 0;
+      uint32_t acc_ph[2] = {0u, 0u};
+      int prev_e = -1;
+      const uint32_t b_base = smem_u32(sB);
+      for (long long it = item_begin; it < item_end; ++it) {
+        const int e = touched[it / tiles_per_expert];
+        const int rows = a.offsets[e + 1] - a.offsets[e];
+        const int n_pass = (rows + kMaxTokPass - 1) / kMaxTokPass;
+        for (int pass = 0; pass < n_pass; ++pass) {
+          // The B operand is shared by consecutive items of an expert whose rows fit one pass; otherwise
+          // every (item, pass) has its own.  The scale warps follow the same rule.
+          const bool new_operand = (prev_e != e) || (n_pass > 1);
+          prev_e = e;
+          if (new_operand) {
+            mbar_wait(b_ready, bph, a.status);
+            bph ^= 1u;
+          }
+          mbar_wait(&acc_empty[buf], acc_ph[buf] ^ 1u, a.status);
+          tc_fence_after_sync();
+          const uint32_t d_addr = tmem_base + kColD + static_cast<uint32_t>(buf * 16);
+          for (int ks = 0; ks < n_steps; ++ks) {
+            if ((ks & 3) == 0) mbar_wait(&sf_full[slot], sph, a.status);  // scale factors of 4 K steps at a time
+            mbar_wait(&full_a[s], ph, a.status);
+            tc_fence_after_sync();
+            const uint32_t a_addr = smem_u32(sA + s * kAStage);
+            const uint32_t sfa = tmem_base + kColSfa + static_cast<uint32_t>(slot * 16 + (ks & 3) * 4);
+            const uint32_t sfb = tmem_base + kColSfb + static_cast<uint32_t>(ks * 4);
+#pragma unroll
+            for (uint32_t j = 0; j < 4; ++j)
+              umma_mxf4(d_addr, umma_desc_k_sw128(a_addr + j * 32), umma_desc_k_sw128(b_base + ks * 2048 + j * 32),
+                        idesc_mxf4(j), sfa, sfb, (ks | static_cast<int>(j)) != 0 ? 1u : 0u);
+            umma_commit(&empty_a[s]);
+            if (++s == kAStages) { s = 0; ph ^= 1u; }
+            if ((ks & 3) == 3) {
+              umma_commit(&sf_free[slot]);
+              if (++slot == kSfGroups) { slot = 0; sph ^= 1u; }
+            }
+          }
+          umma_commit(&acc_full[buf]);
+          acc_ph[buf] ^= 1u;
+          buf ^= 1;
+          bool next_new = true;  // is this the last use of the operand?
+          if (pass + 1 >= n_pass && it + 1 < item_end) next_new = (touched[(it + 1) / tiles_per_expert] != e) || (n_pass > 1);
+          if (next_new) umma_commit(b_free);
+        }
+      }
+    }
+  } else if (wid < 6) {
+    // =========================== scale factors and the B operand ===========================
+    const int qq = wid & 3;                      // tensor-memory lane quadrant written by this warp (warps 2..5 -> 2,3,0,1)
+    const uint32_t lane_base = static_cast<uint32_t>(qq * 32) << 16;
+    const int st = tid - 64;                     // 0..127
+    int cs = 0, slot = 0;
+    uint32_t cph = 0, sfree_ph = 0, bfree_ph = 0;
+    int prev_e = -1;
+    bool first_b = true;
+    for (long long it = item_begin; it < item_end; ++it) {
+      const int e = touched[it / tiles_per_expert];
+      const int row_begin = a.offsets[e], row_end = a.offsets[e + 1];
+      const int n_pass = (row_end - row_begin + kMaxTokPass - 1) / kMaxTokPass;
+      for (int pass = 0; pass < n_pass; ++pass) {
+        const bool new_operand = (prev_e != e) || (n_pass > 1);
+        prev_e = e;
+        if (new_operand) {
+          // ---- lay out the B operand of (expert, pass): 8 token rows -> 16 E4M3 rows + their scale bytes ----
+          if (!first_b) {
+            mbar_wait(b_free, bfree_ph, a.status);  // MMAs that read the previous operand are done
+            bfree_ph ^= 1u;
+          }
+          first_b = false;
+          const int row0 = row_begin + pass * kMaxTokPass;
+          const int n_blk = K / 32;
+          if (STAGE1) {
+            // task = (token j, 32-element block b): 8 * K/32 tasks over 128 threads
+            for (int task = st; task < kMaxTokPass * n_blk; task += 128) {
+              const int j = task / n_blk, b = task % n_blk;
+              uint32_t hi_w[8], lo_w[8];
+              uint32_t sb_hi = 127u, sb_lo = 127u;
+              if (row0 + j < row_end) {
+                const uint4* src = reinterpret_cast<const uint4*>(a.x + static_cast<size_t>(row0 + j) * K + b * 32);
+                uint4 v[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) v[c] = __ldcg(src + c);
+                const uint32_t* w32 = reinterpret_cast<const uint32_t*>(v);
+                float f[32];
+                float amax = 0.0f;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                  f[2 * i] = __uint_as_float(w32[i] << 16);
+                  f[2 * i + 1] = __uint_as_float(w32[i] & 0xFFFF0000u);
+                  amax = fmaxf(amax, fmaxf(fabsf(f[2 * i]), fabsf(f[2 * i + 1])));
+                }
+                int se = (amax > 0.0f) ? block_exp(amax) : 0;
+                se = max(-120, min(se, 120));
+                const float inv = pow2f(-se);
+                sb_hi = static_cast<uint32_t>(se + 127);
+                sb_lo = static_cast<uint32_t>(se - 3 + 127);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  uint32_t hw = 0u, lw = 0u;
+#pragma unroll
+                  for (int t = 0; t < 4; ++t) {
+                    uint32_t h, l;
+                    split_e4m3(f[4 * i + t] * inv, &h, &l);
+                    hw |= h << (8 * t);
+                    lw |= l << (8 * t);
+                  }
+                  hi_w[i] = hw;
+                  lo_w[i] = lw;
+                }
+              } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) { hi_w[i] = 0u; lo_w[i] = 0u; }
+              }
+              const int ks = b >> 2, c16 = (b & 3) * 2;  // K step, first 16-byte chunk of the 128-byte row
+              unsigned char* base = sB + ks * 2048;
+              const int rh = 2 * j, rl = 2 * j + 1;
+              *reinterpret_cast<uint4*>(base + rh * 128 + (((c16) ^ (rh & 7)) << 4)) = make_uint4(hi_w[0], hi_w[1], hi_w[2], hi_w[3]);
+              *reinterpret_cast<uint4*>(base + rh * 128 + (((c16 + 1) ^ (rh & 7)) << 4)) = make_uint4(hi_w[4], hi_w[5], hi_w[6], hi_w[7]);
+              *reinterpret_cast<uint4*>(base + rl * 128 + (((c16) ^ (rl & 7)) << 4)) = make_uint4(lo_w[0], lo_w[1], lo_w[2], lo_w[3]);
+              *reinterpret_cast<uint4*>(base + rl * 128 + (((c16 + 1) ^ (rl & 7)) << 4)) = make_uint4(lo_w[4], lo_w[5], lo_w[6], lo_w[7]);
+              sSfb[rh * n_blk + b] = static_cast<unsigned char>(sb_hi);
+              sSfb[rl * n_blk + b] = static_cast<unsigned char>(sb_lo);
+            }
+          } else {
+            // stage 2: the split rows were written by stage 1; copy 16-byte chunks into the swizzled layout
+            const int chunks_per_row = K / 16;
+            for (int task = st; task < 16 * chunks_per_row; task += 128) {
+              const int r = task / chunks_per_row, c = task % chunks_per_row;
+              const int p = row0 + (r >> 1);
+              uint4 v = make_uint4(0u, 0u, 0u, 0u);
+              if (p < row_end) v = __ldcg(reinterpret_cast<const uint4*>(a.aq + (static_cast<size_t>(2 * p + (r & 1))) * K + c * 16));
+              const int ks = c >> 3, c16 = c & 7;
+              *reinterpret_cast<uint4*>(sB + ks * 2048 + r * 128 + ((c16 ^ (r & 7)) << 4)) = v;
+            }
+            for (int task = st; task < 16 * n_blk; task += 128) {
+              const int r = task / n_blk, b = task % n_blk;
+              const int p = row0 + (r >> 1);
+              sSfb[r * n_blk + b] = (p < row_end) ? a.aq_sf[(static_cast<size_t>(2 * p + (r & 1))) * n_blk + b] : static_cast<unsigned char>(127);
+            }
+          }
+          fence_proxy_async_smem();
+          asm volatile("bar.sync 3, 128;" ::: "memory");
+          __syncwarp();
+          // B scale factors -> tensor memory: the block of K step ks holds, in lane n (< 16) of every quadrant, the
+          // 4 scale bytes of B row n for that step
+          for (int ks = 0; ks < n_steps; ++ks) {
+            const uint32_t w = (lane < 16) ? *reinterpret_cast<const uint32_t*>(sSfb + lane * n_blk + ks * 4) : 0u;
+            tmem_st_32x4(tmem_base + lane_base + kColSfb + static_cast<uint32_t>(ks * 4), w, 0u, 0u, 0u);
+          }
+          tmem_st_wait();
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(b_ready);
+        }
+        // ---- A scale factors: one scale stage (128 rows x 16 bytes = 4 K steps) -> one 16-column group ----
+        for (int ks = 0; ks < n_steps; ks += 4) {
+          mbar_wait(&full_sc[cs], cph, a.status);
+          mbar_wait(&sf_free[slot], sfree_ph ^ 1u, a.status);
+          __syncwarp();  // the spins may leave lanes diverged; tcgen05.st is warp-collective
+          const unsigned char* blk = sSc + cs * kScStage;
+          const uint4 r0 = *reinterpret_cast<const uint4*>(blk + (lane) * 16);
+          const uint4 r1 = *reinterpret_cast<const uint4*>(blk + (lane + 32) * 16);
+          const uint4 r2 = *reinterpret_cast<const uint4*>(blk + (lane + 64) * 16);
+          const uint4 r3 = *reinterpret_cast<const uint4*>(blk + (lane + 96) * 16);
+          // column 4t + c of the group: scale bytes of K step t for row lane + 32c
+          asm volatile(
+              "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(
+                  tmem_base + lane_base + kColSfa + static_cast<uint32_t>(slot * 16)),
+              "r"(r0.x), "r"(r1.x), "r"(r2.x), "r"(r3.x), "r"(r0.y), "r"(r1.y), "r"(r2.y), "r"(r3.y), "r"(r0.z), "r"(r1.z),
+              "r"(r2.z), "r"(r3.z), "r"(r0.w), "r"(r1.w), "r"(r2.w), "r"(r3.w)
+              : "memory");
+          tmem_st_wait();
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive(&sf_full[slot]);
+            mbar_arrive(&empty_sc[cs]);
+          }
+          if (++cs == kScStages) { cs = 0; cph ^= 1u; }
+          if (++slot == kSfGroups) { slot = 0; sfree_ph ^= 1u; }
+        }
+      }
+    }
+  } else {
+    // =========================== epilogue ===========================
+    const int q = wid & 3;  // warps 6..9 -> quadrants 2,3,0,1
+    const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
+    int buf = 0;
+    uint32_t acc_ph[2] = {0u, 0u};
+    for (long long it = item_begin; it < item_end; ++it) {
+      const int e = touched[it / tiles_per_expert];
+      const int tile = static_cast<int>(it % tiles_per_expert);
+      const int row_begin = a.offsets[e], row_end = a.offsets[e + 1];
+      const int n_pass = (row_end - row_begin + kMaxTokPass - 1) / kMaxTokPass;
+      for (int pass = 0; pass < n_pass; ++pass) {
+        const int row0 = row_begin + pass * kMaxTokPass;
+        mbar_wait(&acc_full[buf], acc_ph[buf], a.status);
+        __syncwarp();  // tcgen05.ld is warp-collective
+        acc_ph[buf] ^= 1u;
+        tc_fence_after_sync();
+        uint32_t v[16];
+        tmem_ld_32x16(tmem_base + lane_base + kColD + static_cast<uint32_t>(buf * 16), v);
+        tmem_ld_wait();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[buf]);  // values are in registers: the accumulator may be reused
+        buf ^= 1;
+        float r[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) r[j] = __uint_as_float(v[2 * j]) + __uint_as_float(v[2 * j + 1]);
+        if (STAGE1) {
+          // lanes 0..63 gate, 64..127 up: up values go through shared memory, then each gate thread owns
+          // (i, 8 tokens); a warp holds 32 consecutive i = one scale block of the stage-2 operand
+          if (q >= 2) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) sX[((q - 2) * 32 + lane) * 9 + j] = r[j];
+          }
+          asm volatile("bar.sync 2, 128;" ::: "memory");
+          if (q < 2) {
+            const int i = tile * 64 + q * 32 + lane;
+            const int n_blk = a.I / 32;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const int p = row0 + j;
+              const float u = sX[(q * 32 + lane) * 9 + j];
+              const float g = r[j];
+              float av = __fdividef(g, 1.0f + __expf(-g)) * u;
+              av = __bfloat162float(__float2bfloat16_rn(av));  // the intermediate is defined as a bf16 value
+              float amax = fabsf(av);
+#pragma unroll
+              for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
+              int se = (amax > 0.0f) ? block_exp(amax) : 0;
+              se = max(-120, min(se, 120));
+              uint32_t h, l;
+              split_e4m3(av * pow2f(-se), &h, &l);
+              if (p < row_end) {
+                a.aq_out[static_cast<size_t>(2 * p) * a.I + i] = static_cast<uint8_t>(h);
+                a.aq_out[static_cast<size_t>(2 * p + 1) * a.I + i] = static_cast<uint8_t>(l);
+                if (lane == 0) {
+                  a.aq_sf_out[static_cast<size_t>(2 * p) * n_blk + (i >> 5)] = static_cast<uint8_t>(se + 127);
+                  a.aq_sf_out[static_cast<size_t>(2 * p + 1) * n_blk + (i >> 5)] = static_cast<uint8_t>(se - 3 + 127);
+                }
+              }
+            }
+          }
+          asm volatile("bar.sync 2, 128;" ::: "memory");
+        } else {
+          const int n = tile * kTile + q * 32 + lane;
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (row0 + j < row_end) a.y[static_cast<size_t>(row0 + j) * a.R + n] = r[j];
+        }
+      }
+    }
+  }
+
+  // ---- teardown ----
+  tc_fence_before_sync();
+  __syncthreads();
+  if (wid == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kNatTmemCols);
+  }
+}
+
+// ---- host side ---------------------------------------------------------------------------------------
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn nat_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+bool nat_map(CUtensorMap* m, CUtensorMapDataType dt, const void* base, uint64_t inner_elems, uint64_t row_bytes, uint64_t rows,
+             uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle sw) {
+  EncodeTiledFn fn = nat_encode_fn();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[2] = {inner_elems, rows};
+  const cuuint64_t strides[1] = {row_bytes};
+  const cuuint32_t box[2] = {box_inner, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool native_shape_ok(const moe_shape_t& sh, const void* w13, const void* w2) {
+  // decode-sized: on average at most 32 rows per expert (4 passes of 8 tokens over the weight stream)
+  const long long S = static_cast<long long>(sh.T) * sh.k;
+  return S <= 4096 && S <= 32LL * sh.E && sh.H % 128 == 0 && sh.I % 128 == 0 && sh.H <= kMaxK && sh.I <= kMaxK && sh.H % 512 == 0 &&
+         sh.I % 512 == 0 && (reinterpret_cast<uintptr_t>(w13) & 31u) == 0 && (reinterpret_cast<uintptr_t>(w2) & 31u) == 0 &&
+         nat_smem(sh.E, sh.H > sh.I ? sh.H : sh.I).total + 1024 <= 227 * 1024;
+}
+
+size_t native_scratch_bytes(const moe_shape_t& sh) {
+  const size_t S = static_cast<size_t>(sh.T) * sh.k;
+  return align_up(2 * S * sh.I, kAlign) + align_up(2 * S * (sh.I / 32), kAlign);
+}
+
+int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
+                             const uint8_t* w2, const uint8_t* s2, const moe_shape_t& sh, void* scratch, float* y_perm,
+                             int* status_word, cudaStream_t st) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(ffn_native_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(ffn_native_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+      return MOE_ERR_CUDA;
+    attr_done = true;
+  }
+  const size_t S = static_cast<size_t>(sh.T) * sh.k;
+  uint8_t* aq = static_cast<uint8_t*>(scratch);
+  uint8_t* aq_sf = aq + align_up(2 * S * sh.I, kAlign);
+  CUtensorMap tm_w13, tm_w2, tm_s13, tm_s2;
+  if (!nat_map(&tm_w13, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, w13, sh.H, sh.H / 2, static_cast<uint64_t>(sh.E) * 2 * sh.I, kKStep,
+               64, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !nat_map(&tm_w2, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, w2, sh.I, sh.I / 2, static_cast<uint64_t>(sh.E) * sh.H, kKStep, 64,
+               CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !nat_map(&tm_s13, CU_TENSOR_MAP_DATA_TYPE_UINT8, s13, sh.H / 32, sh.H / 32, static_cast<uint64_t>(sh.E) * 2 * sh.I, 16, 64,
+               CU_TENSOR_MAP_SWIZZLE_NONE) ||
+      !nat_map(&tm_s2, CU_TENSOR_MAP_DATA_TYPE_UINT8, s2, sh.I / 32, sh.I / 32, static_cast<uint64_t>(sh.E) * sh.H, 16, 64,
+               CU_TENSOR_MAP_SWIZZLE_NONE))
+    return MOE_ERR_CUDA;
+  const int grid = sm_count();
+  NatArgs a;
+  a.x = x_perm;
+  a.aq = aq;
+  a.aq_sf = aq_sf;
+  a.aq_out = aq;
+  a.aq_sf_out = aq_sf;
+  a.offsets = offsets;
+  a.y = y_perm;
+  a.status = status_word;
+  a.E = sh.E;
+  a.I = sh.I;
+  a.K = sh.H;
+  a.R = 2 * sh.I;
+  ffn_native_kernel<true><<<grid, kNatThreads, nat_smem(sh.E, sh.H).total + 1024, st>>>(tm_w13, tm_s13, a);
+  if (cudaGetLastError() != cudaSuccess) return MOE_ERR_CUDA;
+  a.K = sh.I;
+  a.R = sh.H;
+  ffn_native_kernel<false><<<grid, kNatThreads, nat_smem(sh.E, sh.I).total + 1024, st>>>(tm_w2, tm_s2, a);
+  if (cudaGetLastError() != cudaSuccess) return MOE_ERR_CUDA;
+  note_kernel("ffn_native_mxf4_block_scaled", 2);
+  return MOE_OK;
+}
+
+}  // namespace moe

@@ -32,6 +32,7 @@ struct FfnArgs {
   __nv_bfloat16* act;         // stage 1 output [S, I]
   float* y;                   // stage 2 output [S, Hout]
   int* status;
+  uint32_t k1, k2;         // 0x1040, 0x0104: multipliers of the E2M1 expansion, kept opaque to the compiler
   int E, K, R, I;             // R rows per expert (2I for stage 1, H for stage 2); I used by stage 1 only
   int n_stages;
 };
@@ -210,8 +211,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const FfnArgs a
 #pragma unroll
               for (int q = 0; q < 4; ++q) {
                 uint32_t pa[4], pb[4];
-                dequant8(wav[q], ma, pa);
-                dequant8(wbv[q], mb, pb);
+                dequant8(wav[q], ma, a.k1, a.k2, pa);
+                dequant8(wbv[q], mb, a.k1, a.k2, pb);
                 mma_bf16_16x8x16(c, pa[0], pb[0], pa[1], pb[1], breg[j][4 * q + 0], breg[j][4 * q + 1]);
                 mma_bf16_16x8x16(c2, pa[2], pb[2], pa[3], pb[3], breg[j][4 * q + 2], breg[j][4 * q + 3]);
               }
@@ -288,6 +289,10 @@ int launch_expert_ffn_stream(const __nv_bfloat16* x_perm, const int* offsets, co
     a.act = act;
     a.y = y_perm;
     a.status = status_word;
+  a.k1 = 0x1040u;
+  a.k2 = 0x0104u;
+    a.k1 = 0x1040u;
+    a.k2 = 0x0104u;
     a.E = sh.E;
     a.I = sh.I;
     if (stage1) {

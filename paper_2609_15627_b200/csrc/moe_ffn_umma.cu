@@ -52,6 +52,7 @@ struct UmmaArgs {
   __nv_bfloat16* act;      // stage 1 output [S, I]
   float* y;                // stage 2 output [S, R]
   int* status;
+  uint32_t k1, k2;         // 0x1040, 0x0104: multipliers of the E2M1 expansion, kept opaque to the compiler
   int E, K, R, I;          // R weight rows per expert (2I or H)
 };
 
@@ -269,7 +270,7 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
           uint32_t p[4];
-          dequant8(wv[q], q < 4 ? m_lo : m_hi, p);
+          dequant8(wv[q], q < 4 ? m_lo : m_hi, a.k1, a.k2, p);
           // (0,4),(1,5),(2,6),(3,7) -> natural order (0,1),(2,3),(4,5),(6,7)
           out[q].x = __byte_perm(p[0], p[1], 0x5410);
           out[q].y = __byte_perm(p[2], p[3], 0x5410);
@@ -298,6 +299,7 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
       int row0, ntok;
       pass_rows(a.offsets[e], a.offsets[e + 1], g - prefix[e], &row0, &ntok);
       mbar_wait(acc_full, acc_ph, a.status);
+      __syncwarp();  // tcgen05.ld is warp-collective
       tc_fence_after_sync();
 #pragma unroll 1
       for (int t = 0; t < 2; ++t) {
@@ -423,6 +425,8 @@ int launch_expert_ffn_umma(const __nv_bfloat16* x_perm, const int* offsets, cons
   a.act = act;
   a.y = y_perm;
   a.status = status_word;
+  a.k1 = 0x1040u;
+  a.k2 = 0x0104u;
   a.E = sh.E;
   a.I = sh.I;
   a.w = w13;

@@ -51,7 +51,8 @@ int moe_expert_ffn_noalloc(const void* x_perm_bf16, const int32_t* expert_offset
       !aligned16(w2_scale) || !aligned16(y_perm))
     return MOE_ERR_INVALID_ARG;
   // the intermediate act[T*k, I] bf16 must fit the fixed array
-  const unsigned long long need = 2ull * static_cast<unsigned long long>(s.T) * s.k * s.I;
+  // (bf16 act[T*k, I], or the same rows split into two E4M3 rows plus scale bytes: a little over 2 bytes per element)
+  const unsigned long long need = native_scratch_bytes(s) + kAlign;
   if (need > kStaticScratchBytes) return MOE_ERR_WORKSPACE;
   void* scratch = nullptr;
   const int rc = static_scratch(&scratch);  // first call on a device looks the address up
@@ -60,6 +61,9 @@ int moe_expert_ffn_noalloc(const void* x_perm_bf16, const int32_t* expert_offset
   // to start at zero.  Same kernels and the same kernel choice as moe_expert_ffn.
   __nv_bfloat16* act = static_cast<__nv_bfloat16*>(scratch);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (native_shape_ok(s, w13, w2))
+    return launch_expert_ffn_native(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w13, w13_scale, w2,
+                                    w2_scale, s, scratch, y_perm, status_word, st);
   if (umma_shape_ok(s))
     return launch_expert_ffn_umma(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w13, w13_scale, w2,
                                   w2_scale, s, act, y_perm, status_word, st);

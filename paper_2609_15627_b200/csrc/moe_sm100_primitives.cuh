@@ -151,13 +151,16 @@ MOE_DEVINL uint32_t scale_mult(uint32_t b) { return ((b + 126u) << 7) * 0x000100
 // elements (0,4), (1,5), (2,6), (3,7), each multiplied by `m` = bf16x2 of 2^(scale byte - 1).
 // A nibble isolated at bit 0 (or 4) and multiplied by 2^6 + 2^12 (or 2^2 + 2^8) lands twice: its
 // magnitude bits on bf16 bits 8:6 (value * 2^-126 exactly) and its sign on bit 15; one mask removes the rest.
-MOE_DEVINL void dequant8(uint32_t wd, uint32_t m, uint32_t (&p)[4]) {
+// k1 = 0x1040 and k2 = 0x0104 are passed in registers the compiler cannot see through (kernel
+// parameters), so that each product stays one integer multiply on the FMA pipe instead of being
+// rewritten into shift/add pairs on the half-rate integer pipe.
+MOE_DEVINL void dequant8(uint32_t wd, uint32_t m, uint32_t k1, uint32_t k2, uint32_t (&p)[4]) {
   constexpr uint32_t kKeep = 0x81C081C0u;
   const uint32_t hi = wd >> 8;
-  p[0] = mul_bf16x2(((wd & 0x000F000Fu) * 0x1040u) & kKeep, m);
-  p[1] = mul_bf16x2(((wd & 0x00F000F0u) * 0x0104u) & kKeep, m);
-  p[2] = mul_bf16x2(((hi & 0x000F000Fu) * 0x1040u) & kKeep, m);
-  p[3] = mul_bf16x2(((hi & 0x00F000F0u) * 0x0104u) & kKeep, m);
+  p[0] = mul_bf16x2(((wd & 0x000F000Fu) * k1) & kKeep, m);
+  p[1] = mul_bf16x2(((wd & 0x00F000F0u) * k2) & kKeep, m);
+  p[2] = mul_bf16x2(((hi & 0x000F000Fu) * k1) & kKeep, m);
+  p[3] = mul_bf16x2(((hi & 0x00F000F0u) * k2) & kKeep, m);
 }
 
 }  // namespace moe

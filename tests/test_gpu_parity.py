@@ -431,6 +431,7 @@ def test_ffn_tensor_core_path_against_oracle(T, H, I, E, k, hot, seed):
 def test_kernel_choice_is_a_function_of_the_shape():
     for (T, H, I, E, k, want) in [(16, 256, 128, 8, 2, "ffn_stream_bulk_ring_mma16816"),
                                   (64, 512, 256, 8, 2, "ffn_stream_bulk_ring_mma16816"),
+                                  (64, 512, 512, 8, 2, "ffn_native_mxf4_block_scaled"),
                                   (512, 512, 512, 8, 2, "ffn_umma_tcgen05_grouped"),
                                   (512, 512, 256, 8, 2, "ffn_stream_bulk_ring_mma16816")]:
         wl = inputs.Workload("choice", T, H, I, E, k)
@@ -443,3 +444,38 @@ def test_kernel_choice_is_a_function_of_the_shape():
         moe.moe_expert_ffn(dev(x_perm), dev(off), *[dev(a) for a in w], sh, buf.y_perm, buf.status, buf.ws)
         torch.cuda.synchronize()
         assert moe.moe_last_kernel_name() == want
+
+
+# ---- the native block-scaled FP4 expert FFN, reached when T*k <= 32*E (decode-sized) and H, I are multiples of 512 ----
+
+@pytest.mark.parametrize("T,H,I,E,k,hot,seed", [
+    (16, 512, 512, 8, 2, False, 0),      # a few rows per expert
+    (1, 512, 512, 16, 4, False, 1),      # one token: every expert has one row
+    (64, 1024, 512, 8, 2, False, 2),     # ~16 rows per expert: two passes of 8 tokens
+    (40, 512, 1024, 8, 1, True, 3),      # one hot expert with most rows, several empty experts
+])
+def test_ffn_native_fp4_path_against_oracle(T, H, I, E, k, hot, seed):
+    w = inputs.make_expert_weights(H, I, E, seed=seed)
+    s13 = inputs.index_scales(2 * I, H, E, lo=117, span=6)
+    s2 = inputs.index_scales(H, I, E, lo=118, span=5)
+    w = (w[0], s13, w[2], s2)
+    logits = inputs.make_logits(T, E, seed=seed)
+    if hot:
+        logits[:, 2] += 8.0
+        logits[:, [5, 6]] -= 50.0
+    x = inputs.make_x(T, H, seed=seed)
+    # activations with a wide dynamic range inside a 32-block exercise the hi/lo split
+    xf = inputs.bf16_bits_to_f32(x)
+    xf[:, ::7] *= 2.0 ** -9
+    xf[:, 5::11] *= 64.0
+    x = inputs.f32_to_bf16_bits(xf)
+    ids, tw, off = O.route(logits, k)
+    x_perm, perm, inv = O.permute(x, ids, off)
+    sh = moe.shape(T, H, I, E, k)
+    buf = moe.LayerBuffers(sh)
+    moe.moe_expert_ffn(dev(x_perm), dev(off), *[dev(a) for a in w], sh, buf.y_perm, buf.status, buf.ws)
+    torch.cuda.synchronize()
+    assert int(buf.status.item()) == 0
+    assert moe.moe_last_kernel_name() == "ffn_native_mxf4_block_scaled"
+    ry = O.expert_ffn(x_perm, off, *w, k)
+    check_y(buf.y_perm.cpu().numpy(), ry, "native fp4 path")
