@@ -1,22 +1,29 @@
 // Expert FFN for decode-sized batches on the native block-scaled FP4 tensor-core path:
 // packed E2M1 codes and E8M0 scales go HBM -> TMA -> shared memory -> tcgen05.mma with no ALU expansion.
 //
-// tcgen05.mma kind::mxf8f6f4.block_scale multiplies an E2M1 operand by an E4M3 operand with one UE8M0 scale per
-// 32 K elements on both sides - the checkpoint format of the expert weights is exactly its A operand.  The
+// tcgen05.mma kind::mxf8f6f4.block_scale multiplies an E4M3 operand by an E2M1 operand with one UE8M0 scale per
+// 32 K elements on both sides - the checkpoint format of the expert weights is exactly such an operand.  The
 // activations are bf16, so each row is split on the fly into two E4M3 rows with their own block scales,
 //   x = 2^s * hi + 2^(s-3) * lo,   hi = e4m3(x / 2^s),   lo = e4m3((x / 2^s - hi) * 8),
 // which is exact for every element within 2^14 of its block's maximum (8 significant bits = 4 + 4) and loses
 // less than 2^-19 of the block maximum otherwise; products are exact and accumulate in fp32 in tensor memory.
-// An MMA has M = 128 weight rows, N = 16 (8 tokens x {hi, lo}), K = 32; the two halves are added in the epilogue.
 //
-// Work item = (touched expert, tile of 128 weight rows) over the full K (stage 1: 64 gate + 64 up rows).
+// Operand roles: the tensor core walks the M rows of its A operand one per cycle and all N columns in parallel,
+// so the weights are the B operand (N = 256 weight rows per MMA, K = 32) and the tokens the A operand (M = 128
+// rows of which 16 are used: 8 tokens x {hi, lo}; the other rows read whatever follows in shared memory and
+// their accumulator lanes are never looked at).  With the weights on M the MMA rate capped the stream at
+// about 3 TB/s.
+//
+// Work item = (touched expert, tile of 256 weight rows) over the full K (stage 1: 128 gate + 128 up rows, so
+// gate and up of the same i are two columns of the same accumulator lane).
 // Warp roles (one persistent CTA per SM):
 //   warp 0      producer: TMA loads of the weight tile (4-bit tensor map that unpacks to the 16-byte-aligned
 //               operand layout, 128-byte swizzle) and of the scale bytes
 //   warp 1      allocates tensor memory, issues the MMAs, commits to mbarriers
-//   warps 2..5  move scale bytes into tensor memory (tcgen05.st), and at an expert change split that expert's
-//               token rows into the E4M3 pair and lay them out as the B operand
-//   warps 6..9  epilogue: hi + lo, SwiGLU + bf16 rounding + re-split for stage 2 (stage 1) or fp32 store (stage 2)
+//   warps 2..5  move weight scale bytes into tensor memory (tcgen05.st), and at an expert change split that
+//               expert's token rows into the E4M3 pair and lay them out as the A operand
+//   warp 8      epilogue (lane quadrant 0 holds the 16 used rows): hi + lo, SwiGLU + bf16 rounding + re-split
+//               for stage 2 (stage 1) or the fp32 store (stage 2)
 // Every wait is bounded and reports through the status word.
 #include <cuda.h>
 #include <cuda_fp8.h>
@@ -27,21 +34,22 @@ namespace moe {
 
 namespace {
 
-constexpr int kTile = 128;            // weight rows per item
-constexpr int kKStep = 128;           // K elements per A stage (one 128-byte swizzled row per weight row)
-constexpr int kAStage = kTile * 128;  // 16 KB of shared memory per stage (8 KB of HBM bytes)
-constexpr int kAStages = 8;
-constexpr int kScStages = 3;          // scale-byte ring: one stage = 128 rows x 16 bytes = 4 K steps
+constexpr int kTile = 256;            // weight rows per item (N of the MMA)
+constexpr int kKStep = 128;           // K elements per stage (one 128-byte swizzled row per weight row)
+constexpr int kWStage = kTile * 128;  // 32 KB of shared memory per stage (16 KB of HBM bytes)
+constexpr int kWStages = 4;
+constexpr int kScStages = 3;          // scale-byte ring: one stage = 256 rows x 16 bytes = 4 K steps
 constexpr int kScStage = kTile * 16;
-constexpr int kSfGroups = 3;          // tensor-memory groups for the A scale factors: 4 K steps x 4 columns each
-constexpr int kMaxTokPass = 8;        // tokens per pass (N = 16)
-constexpr int kMaxK = 4096;           // B operand of one expert stays resident: 16 rows x K bytes
-constexpr int kNatThreads = 10 * 32;
-constexpr uint32_t kNatTmemCols = 256;
-// tensor-memory columns: two 16-column accumulators, 3 A-scale groups of 16 columns, and 4 columns per K step for
-// the B scales (a scale-factor block is 4 columns wide - rows 32c..32c+31 in column c - and must start on a
-// multiple of 4 columns; with N = 16 only its first column carries data)
-constexpr uint32_t kColD = 0, kColSfa = 32, kColSfb = 96;
+constexpr int kSfGroups = 3;          // tensor-memory groups for the weight scale factors: 4 K steps x 8 columns
+constexpr int kMaxTokPass = 8;        // tokens per pass (16 operand rows)
+constexpr int kMaxK = 4096;           // activation operand of one expert stays resident: 16 rows x K bytes
+constexpr int kNatThreads = 9 * 32;
+constexpr int kEpiWarp = 8;           // warp 8: (8 % 4) == 0 -> may read tensor-memory lanes 0..31
+constexpr uint32_t kNatTmemCols = 512;
+// tensor-memory columns: one 256-column accumulator; 4 columns per K step for the activation scales (a scale-factor
+// block covers 128 rows in 4 columns - rows 32c..32c+31 in column c - and must start on a multiple of 4 columns; only
+// lanes 0..15 of its first column carry data here); 3 groups of 4 K steps x 8 columns for the weight scales
+constexpr uint32_t kColD = 0, kColSfAct = 256, kColSfW = 384;
 
 struct NatArgs {
   const __nv_bfloat16* x;    // stage 1: sorted token rows [S, K]
@@ -56,21 +64,19 @@ struct NatArgs {
 };
 
 struct NatSmem {
-  uint32_t a, b, sc, sfb, xchg, bars, misc, touched, total;
+  uint32_t act, w, sc, sfa, bars, misc, touched, total;
 };
 __host__ __device__ inline NatSmem nat_smem(int E, int K) {
   NatSmem m;
   uint32_t off = 0;
-  m.a = off;
-  off += kAStages * kAStage;
-  m.b = off;
+  m.act = off;  // first: an MMA reads 128 operand rows from a 16-row tile, i.e. up to 14 KB past it, into the ring
   off += 16 * static_cast<uint32_t>(K);
+  m.w = off;
+  off += kWStages * kWStage;
   m.sc = off;
   off += kScStages * kScStage;
-  m.sfb = off;
-  off += 16 * (static_cast<uint32_t>(K) / 32);  // multiple of 256 for K % 512 == 0: keeps 16-byte alignment
-  m.xchg = off;
-  off += 64 * 9 * 4;
+  m.sfa = off;
+  off += 16 * (static_cast<uint32_t>(K) / 32);
   m.bars = off;
   off += 64 * 8;
   m.misc = off;
@@ -87,7 +93,7 @@ MOE_DEVINL void tmem_st_32x4(uint32_t taddr, uint32_t r0, uint32_t r1, uint32_t 
 }
 MOE_DEVINL void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// D[tmem] (+)= A[smem, E2M1] * B[smem, E4M3]^T with UE8M0 block scales held in tensor memory
+// D[tmem] (+)= A[smem, E4M3] * B[smem, E2M1]^T with UE8M0 block scales held in tensor memory
 MOE_DEVINL void umma_mxf4(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t sfa, uint32_t sfb,
                           uint32_t accumulate) {
   asm volatile(
@@ -98,9 +104,9 @@ MOE_DEVINL void umma_mxf4(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint3
       : "r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
       : "memory");
 }
-// instruction descriptor: A E2M1, B E4M3, UE8M0 scales, M = 128, N = 16; `j` picks byte j of the scale words
+// instruction descriptor: A E4M3, B E2M1, UE8M0 scales, M = 128, N = 256; `j` picks byte j of the scale words
 MOE_DEVINL uint32_t idesc_mxf4(uint32_t j) {
-  return (5u << 7) | (0u << 10) | ((16u >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24) | (j << 29) | (j << 4);
+  return (0u << 7) | (5u << 10) | ((256u >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24) | (j << 29) | (j << 4);
 }
 
 MOE_DEVINL float e4m3_to_float(uint32_t byte) {
@@ -129,22 +135,21 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   const int K = a.K;
   const NatSmem sm = nat_smem(a.E, K);
-  unsigned char* sA = smem + sm.a;
-  unsigned char* sB = smem + sm.b;      // [K/128 steps][16 rows][128 bytes], 128-byte swizzle
-  unsigned char* sSc = smem + sm.sc;    // ring of [128 rows][16 bytes]
-  unsigned char* sSfb = smem + sm.sfb;  // [16 rows][K/32] scale bytes of the B rows
-  float* sX = reinterpret_cast<float*>(smem + sm.xchg);
+  unsigned char* sAct = smem + sm.act;  // [K/128 steps][16 rows][128 bytes], 128-byte swizzle
+  unsigned char* sW = smem + sm.w;      // ring of [256 rows][128 bytes]
+  unsigned char* sSc = smem + sm.sc;    // ring of [256 rows][16 bytes]
+  unsigned char* sSfa = smem + sm.sfa;  // [16 rows][K/32] scale bytes of the activation rows
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bars);
-  uint64_t* full_a = bars;                       // [kAStages]  TMA -> MMA
-  uint64_t* empty_a = full_a + kAStages;         // [kAStages]  MMA done -> producer
-  uint64_t* full_sc = empty_a + kAStages;        // [kScStages] TMA -> scale warps
+  uint64_t* full_w = bars;                       // [kWStages]  TMA -> MMA
+  uint64_t* empty_w = full_w + kWStages;         // [kWStages]  MMA done -> producer
+  uint64_t* full_sc = empty_w + kWStages;        // [kScStages] TMA -> scale warps
   uint64_t* empty_sc = full_sc + kScStages;      // [kScStages] scale warps -> producer
   uint64_t* sf_full = empty_sc + kScStages;      // [kSfGroups] scale warps -> MMA
   uint64_t* sf_free = sf_full + kSfGroups;       // [kSfGroups] MMA done -> scale warps
-  uint64_t* acc_full = sf_free + kSfGroups;      // [2] MMA -> epilogue
-  uint64_t* acc_empty = acc_full + 2;            // [2] epilogue -> MMA
-  uint64_t* b_ready = acc_empty + 2;             // scale warps -> MMA: B operand of the current (expert, pass) is in place
-  uint64_t* b_free = b_ready + 1;                // MMA done with the B operand -> scale warps
+  uint64_t* acc_full = sf_free + kSfGroups;      // MMA -> epilogue
+  uint64_t* acc_empty = acc_full + 1;            // epilogue -> MMA
+  uint64_t* act_ready = acc_empty + 1;           // scale warps -> MMA: activation operand of the current (expert, pass)
+  uint64_t* act_free = act_ready + 1;            // MMA done with the activation operand -> scale warps
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + sm.misc);
   int* touched = reinterpret_cast<int*>(smem + sm.touched);
   int* s_misc = touched + a.E;
@@ -167,12 +172,13 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     if (lane == 0) s_misc[0] = run;
   }
   if (tid == 0) {
-    for (int s = 0; s < kAStages; ++s) { mbar_init(&full_a[s], 1); mbar_init(&empty_a[s], 1); }
+    for (int s = 0; s < kWStages; ++s) { mbar_init(&full_w[s], 1); mbar_init(&empty_w[s], 1); }
     for (int s = 0; s < kScStages; ++s) { mbar_init(&full_sc[s], 1); mbar_init(&empty_sc[s], 4); }
     for (int s = 0; s < kSfGroups; ++s) { mbar_init(&sf_full[s], 4); mbar_init(&sf_free[s], 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4); }
-    mbar_init(b_ready, 4);
-    mbar_init(b_free, 1);
+    mbar_init(acc_full, 1);
+    mbar_init(acc_empty, 1);
+    mbar_init(act_ready, 4);
+    mbar_init(act_free, 1);
     mbar_fence_init();
   }
   if (wid == 1) tmem_alloc(tmem_holder, kNatTmemCols);
@@ -197,22 +203,22 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         const int tile = static_cast<int>(it % tiles_per_expert);
         const int rows = a.offsets[e + 1] - a.offsets[e];
         const int n_pass = (rows + kMaxTokPass - 1) / kMaxTokPass;
-        const int wrow_a = STAGE1 ? e * a.R + tile * 64 : e * a.R + tile * kTile;
-        const int wrow_b = STAGE1 ? e * a.R + a.I + tile * 64 : wrow_a + 64;
+        const int wrow_a = STAGE1 ? e * a.R + tile * 128 : e * a.R + tile * kTile;
+        const int wrow_b = STAGE1 ? e * a.R + a.I + tile * 128 : wrow_a + 128;
         for (int pass = 0; pass < n_pass; ++pass) {
           for (int ks = 0; ks < n_steps; ++ks) {
             if ((ks & 3) == 0) {
               mbar_wait(&empty_sc[cs], cph ^ 1u, a.status);
               mbar_expect_tx(&full_sc[cs], kScStage);
               tma_load_2d(sSc + cs * kScStage, &tmap_sc, ks * 4, wrow_a, &full_sc[cs]);
-              tma_load_2d(sSc + cs * kScStage + 64 * 16, &tmap_sc, ks * 4, wrow_b, &full_sc[cs]);
+              tma_load_2d(sSc + cs * kScStage + 128 * 16, &tmap_sc, ks * 4, wrow_b, &full_sc[cs]);
               if (++cs == kScStages) { cs = 0; cph ^= 1u; }
             }
-            mbar_wait(&empty_a[s], ph ^ 1u, a.status);
-            mbar_expect_tx(&full_a[s], kAStage / 2);  // the transaction count is in packed (global) bytes
-            tma_load_2d(sA + s * kAStage, &tmap_w, ks * kKStep, wrow_a, &full_a[s]);
-            tma_load_2d(sA + s * kAStage + 64 * 128, &tmap_w, ks * kKStep, wrow_b, &full_a[s]);
-            if (++s == kAStages) { s = 0; ph ^= 1u; }
+            mbar_wait(&empty_w[s], ph ^ 1u, a.status);
+            mbar_expect_tx(&full_w[s], kWStage / 2);  // the transaction count is in packed (global) bytes
+            tma_load_2d(sW + s * kWStage, &tmap_w, ks * kKStep, wrow_a, &full_w[s]);
+            tma_load_2d(sW + s * kWStage + 128 * 128, &tmap_w, ks * kKStep, wrow_b, &full_w[s]);
+            if (++s == kWStages) { s = 0; ph ^= 1u; }
           }
         }
       }
@@ -220,63 +226,61 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   } else if (wid == 1) {
     // =========================== MMA issuer ===========================
     if (lane == 0) {
-      int s = 0, slot = 0, buf = 0;
-      uint32_t ph = 0, sph = 0, bph = 0;
-      uint32_t acc_ph[2] = {0u, 0u};
+      int s = 0, slot = 0;
+      uint32_t ph = 0, sph = 0, aph = 0, acc_ph = 0;
       int prev_e = -1;
-      const uint32_t b_base = smem_u32(sB);
+      const uint32_t act_base = smem_u32(sAct);
+      const uint32_t d_addr = tmem_base + kColD;
       for (long long it = item_begin; it < item_end; ++it) {
         const int e = touched[it / tiles_per_expert];
         const int rows = a.offsets[e + 1] - a.offsets[e];
         const int n_pass = (rows + kMaxTokPass - 1) / kMaxTokPass;
         for (int pass = 0; pass < n_pass; ++pass) {
-          // The B operand is shared by consecutive items of an expert whose rows fit one pass; otherwise
-          // every (item, pass) has its own.  The scale warps follow the same rule.
+          // The activation operand is shared by consecutive items of an expert whose rows fit one pass;
+          // otherwise every (item, pass) has its own.  The scale warps follow the same rule.
           const bool new_operand = (prev_e != e) || (n_pass > 1);
           prev_e = e;
           if (new_operand) {
-            mbar_wait(b_ready, bph, a.status);
-            bph ^= 1u;
+            mbar_wait(act_ready, aph, a.status);
+            aph ^= 1u;
           }
-          mbar_wait(&acc_empty[buf], acc_ph[buf] ^ 1u, a.status);
+          mbar_wait(acc_empty, acc_ph ^ 1u, a.status);
           tc_fence_after_sync();
-          const uint32_t d_addr = tmem_base + kColD + static_cast<uint32_t>(buf * 16);
           for (int ks = 0; ks < n_steps; ++ks) {
-            if ((ks & 3) == 0) mbar_wait(&sf_full[slot], sph, a.status);  // scale factors of 4 K steps at a time
-            mbar_wait(&full_a[s], ph, a.status);
+            if ((ks & 3) == 0) mbar_wait(&sf_full[slot], sph, a.status);  // weight scale factors of 4 K steps at a time
+            mbar_wait(&full_w[s], ph, a.status);
             tc_fence_after_sync();
-            const uint32_t a_addr = smem_u32(sA + s * kAStage);
-            const uint32_t sfa = tmem_base + kColSfa + static_cast<uint32_t>(slot * 16 + (ks & 3) * 4);
-            const uint32_t sfb = tmem_base + kColSfb + static_cast<uint32_t>(ks * 4);
+            const uint32_t w_addr = smem_u32(sW + s * kWStage);
+            const uint32_t sf_act = tmem_base + kColSfAct + static_cast<uint32_t>(ks * 4);
+            const uint32_t sf_w = tmem_base + kColSfW + static_cast<uint32_t>(slot * 32 + (ks & 3) * 8);
 #pragma unroll
             for (uint32_t j = 0; j < 4; ++j)
-              umma_mxf4(d_addr, umma_desc_k_sw128(a_addr + j * 32), umma_desc_k_sw128(b_base + ks * 2048 + j * 32),
-                        idesc_mxf4(j), sfa, sfb, (ks | static_cast<int>(j)) != 0 ? 1u : 0u);
-            umma_commit(&empty_a[s]);
-            if (++s == kAStages) { s = 0; ph ^= 1u; }
+              umma_mxf4(d_addr, umma_desc_k_sw128(act_base + ks * 2048 + j * 32), umma_desc_k_sw128(w_addr + j * 32),
+                        idesc_mxf4(j), sf_act, sf_w, (ks | static_cast<int>(j)) != 0 ? 1u : 0u);
+            umma_commit(&empty_w[s]);
+            if (++s == kWStages) { s = 0; ph ^= 1u; }
             if ((ks & 3) == 3) {
               umma_commit(&sf_free[slot]);
               if (++slot == kSfGroups) { slot = 0; sph ^= 1u; }
             }
           }
-          umma_commit(&acc_full[buf]);
-          acc_ph[buf] ^= 1u;
-          buf ^= 1;
-          bool next_new = true;  // is this the last use of the operand?
+          umma_commit(acc_full);
+          acc_ph ^= 1u;
+          bool next_new = true;  // is this the last use of the activation operand?
           if (pass + 1 >= n_pass && it + 1 < item_end) next_new = (touched[(it + 1) / tiles_per_expert] != e) || (n_pass > 1);
-          if (next_new) umma_commit(b_free);
+          if (next_new) umma_commit(act_free);
         }
       }
     }
-  } else if (wid < 6) {
-    // =========================== scale factors and the B operand ===========================
+  } else if (wid >= 2 && wid < 6) {
+    // =========================== scale factors and the activation operand ===========================
     const int qq = wid & 3;                      // tensor-memory lane quadrant written by this warp (warps 2..5 -> 2,3,0,1)
     const uint32_t lane_base = static_cast<uint32_t>(qq * 32) << 16;
     const int st = tid - 64;                     // 0..127
     int cs = 0, slot = 0;
-    uint32_t cph = 0, sfree_ph = 0, bfree_ph = 0;
+    uint32_t cph = 0, sfree_ph = 0, afree_ph = 0;
     int prev_e = -1;
-    bool first_b = true;
+    bool first_op = true;
     for (long long it = item_begin; it < item_end; ++it) {
       const int e = touched[it / tiles_per_expert];
       const int row_begin = a.offsets[e], row_end = a.offsets[e + 1];
@@ -285,12 +289,12 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         const bool new_operand = (prev_e != e) || (n_pass > 1);
         prev_e = e;
         if (new_operand) {
-          // ---- lay out the B operand of (expert, pass): 8 token rows -> 16 E4M3 rows + their scale bytes ----
-          if (!first_b) {
-            mbar_wait(b_free, bfree_ph, a.status);  // MMAs that read the previous operand are done
-            bfree_ph ^= 1u;
+          // ---- lay out the activation operand of (expert, pass): 8 token rows -> 16 E4M3 rows + scale bytes ----
+          if (!first_op) {
+            mbar_wait(act_free, afree_ph, a.status);  // MMAs that read the previous operand are done
+            afree_ph ^= 1u;
           }
-          first_b = false;
+          first_op = false;
           const int row0 = row_begin + pass * kMaxTokPass;
           const int n_blk = K / 32;
           if (STAGE1) {
@@ -336,14 +340,14 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
                 for (int i = 0; i < 8; ++i) { hi_w[i] = 0u; lo_w[i] = 0u; }
               }
               const int ks = b >> 2, c16 = (b & 3) * 2;  // K step, first 16-byte chunk of the 128-byte row
-              unsigned char* base = sB + ks * 2048;
+              unsigned char* base = sAct + ks * 2048;
               const int rh = 2 * j, rl = 2 * j + 1;
               *reinterpret_cast<uint4*>(base + rh * 128 + (((c16) ^ (rh & 7)) << 4)) = make_uint4(hi_w[0], hi_w[1], hi_w[2], hi_w[3]);
               *reinterpret_cast<uint4*>(base + rh * 128 + (((c16 + 1) ^ (rh & 7)) << 4)) = make_uint4(hi_w[4], hi_w[5], hi_w[6], hi_w[7]);
               *reinterpret_cast<uint4*>(base + rl * 128 + (((c16) ^ (rl & 7)) << 4)) = make_uint4(lo_w[0], lo_w[1], lo_w[2], lo_w[3]);
               *reinterpret_cast<uint4*>(base + rl * 128 + (((c16 + 1) ^ (rl & 7)) << 4)) = make_uint4(lo_w[4], lo_w[5], lo_w[6], lo_w[7]);
-              sSfb[rh * n_blk + b] = static_cast<unsigned char>(sb_hi);
-              sSfb[rl * n_blk + b] = static_cast<unsigned char>(sb_lo);
+              sSfa[rh * n_blk + b] = static_cast<unsigned char>(sb_hi);
+              sSfa[rl * n_blk + b] = static_cast<unsigned char>(sb_lo);
             }
           } else {
             // stage 2: the split rows were written by stage 1; copy 16-byte chunks into the swizzled layout
@@ -354,44 +358,46 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
               uint4 v = make_uint4(0u, 0u, 0u, 0u);
               if (p < row_end) v = __ldcg(reinterpret_cast<const uint4*>(a.aq + (static_cast<size_t>(2 * p + (r & 1))) * K + c * 16));
               const int ks = c >> 3, c16 = c & 7;
-              *reinterpret_cast<uint4*>(sB + ks * 2048 + r * 128 + ((c16 ^ (r & 7)) << 4)) = v;
+              *reinterpret_cast<uint4*>(sAct + ks * 2048 + r * 128 + ((c16 ^ (r & 7)) << 4)) = v;
             }
             for (int task = st; task < 16 * n_blk; task += 128) {
               const int r = task / n_blk, b = task % n_blk;
               const int p = row0 + (r >> 1);
-              sSfb[r * n_blk + b] = (p < row_end) ? a.aq_sf[(static_cast<size_t>(2 * p + (r & 1))) * n_blk + b] : static_cast<unsigned char>(127);
+              sSfa[r * n_blk + b] = (p < row_end) ? a.aq_sf[(static_cast<size_t>(2 * p + (r & 1))) * n_blk + b] : static_cast<unsigned char>(127);
             }
           }
           fence_proxy_async_smem();
           asm volatile("bar.sync 3, 128;" ::: "memory");
           __syncwarp();
-          // B scale factors -> tensor memory: the block of K step ks holds, in lane n (< 16) of every quadrant, the
-          // 4 scale bytes of B row n for that step
+          // activation scale factors -> tensor memory: the block of K step ks holds, in lane n (< 16) of every
+          // quadrant, the 4 scale bytes of operand row n for that step
           for (int ks = 0; ks < n_steps; ++ks) {
-            const uint32_t w = (lane < 16) ? *reinterpret_cast<const uint32_t*>(sSfb + lane * n_blk + ks * 4) : 0u;
-            tmem_st_32x4(tmem_base + lane_base + kColSfb + static_cast<uint32_t>(ks * 4), w, 0u, 0u, 0u);
+            const uint32_t w = (lane < 16) ? *reinterpret_cast<const uint32_t*>(sSfa + lane * n_blk + ks * 4) : 0u;
+            tmem_st_32x4(tmem_base + lane_base + kColSfAct + static_cast<uint32_t>(ks * 4), w, 0u, 0u, 0u);
           }
           tmem_st_wait();
           tc_fence_before_sync();
           __syncwarp();
-          if (lane == 0) mbar_arrive(b_ready);
+          if (lane == 0) mbar_arrive(act_ready);
         }
-        // ---- A scale factors: one scale stage (128 rows x 16 bytes = 4 K steps) -> one 16-column group ----
+        // ---- weight scale factors: one scale stage (256 rows x 16 bytes = 4 K steps) -> one 32-column group ----
         for (int ks = 0; ks < n_steps; ks += 4) {
           mbar_wait(&full_sc[cs], cph, a.status);
           mbar_wait(&sf_free[slot], sfree_ph ^ 1u, a.status);
           __syncwarp();  // the spins may leave lanes diverged; tcgen05.st is warp-collective
           const unsigned char* blk = sSc + cs * kScStage;
-          const uint4 r0 = *reinterpret_cast<const uint4*>(blk + (lane) * 16);
-          const uint4 r1 = *reinterpret_cast<const uint4*>(blk + (lane + 32) * 16);
-          const uint4 r2 = *reinterpret_cast<const uint4*>(blk + (lane + 64) * 16);
-          const uint4 r3 = *reinterpret_cast<const uint4*>(blk + (lane + 96) * 16);
-          // column 4t + c of the group: scale bytes of K step t for row lane + 32c
+          uint4 r[8];
+#pragma unroll
+          for (int c = 0; c < 8; ++c) r[c] = *reinterpret_cast<const uint4*>(blk + (lane + 32 * c) * 16);
+          // column 8t + c of the group: scale bytes of K step t for weight row lane + 32c
           asm volatile(
-              "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(
-                  tmem_base + lane_base + kColSfa + static_cast<uint32_t>(slot * 16)),
-              "r"(r0.x), "r"(r1.x), "r"(r2.x), "r"(r3.x), "r"(r0.y), "r"(r1.y), "r"(r2.y), "r"(r3.y), "r"(r0.z), "r"(r1.z),
-              "r"(r2.z), "r"(r3.z), "r"(r0.w), "r"(r1.w), "r"(r2.w), "r"(r3.w)
+              "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+              "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};" ::"r"(
+                  tmem_base + lane_base + kColSfW + static_cast<uint32_t>(slot * 32)),
+              "r"(r[0].x), "r"(r[1].x), "r"(r[2].x), "r"(r[3].x), "r"(r[4].x), "r"(r[5].x), "r"(r[6].x), "r"(r[7].x),
+              "r"(r[0].y), "r"(r[1].y), "r"(r[2].y), "r"(r[3].y), "r"(r[4].y), "r"(r[5].y), "r"(r[6].y), "r"(r[7].y),
+              "r"(r[0].z), "r"(r[1].z), "r"(r[2].z), "r"(r[3].z), "r"(r[4].z), "r"(r[5].z), "r"(r[6].z), "r"(r[7].z),
+              "r"(r[0].w), "r"(r[1].w), "r"(r[2].w), "r"(r[3].w), "r"(r[4].w), "r"(r[5].w), "r"(r[6].w), "r"(r[7].w)
               : "memory");
           tmem_st_wait();
           tc_fence_before_sync();
@@ -405,74 +411,98 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         }
       }
     }
-  } else {
-    // =========================== epilogue ===========================
-    const int q = wid & 3;  // warps 6..9 -> quadrants 2,3,0,1
-    const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
-    int buf = 0;
-    uint32_t acc_ph[2] = {0u, 0u};
+  } else if (wid == kEpiWarp) {
+    // =========================== epilogue (tensor-memory lanes 0..15: row 2j = hi, 2j+1 = lo of token j) ===========================
+    uint32_t acc_ph = 0;
+    const bool writer = (lane < 16) && ((lane & 1) == 0);
+    const int j = lane >> 1;
     for (long long it = item_begin; it < item_end; ++it) {
       const int e = touched[it / tiles_per_expert];
       const int tile = static_cast<int>(it % tiles_per_expert);
       const int row_begin = a.offsets[e], row_end = a.offsets[e + 1];
       const int n_pass = (row_end - row_begin + kMaxTokPass - 1) / kMaxTokPass;
       for (int pass = 0; pass < n_pass; ++pass) {
-        const int row0 = row_begin + pass * kMaxTokPass;
-        mbar_wait(&acc_full[buf], acc_ph[buf], a.status);
+        const int p = row_begin + pass * kMaxTokPass + j;  // sorted row of this lane pair's token
+        mbar_wait(acc_full, acc_ph, a.status);
         __syncwarp();  // tcgen05.ld is warp-collective
-        acc_ph[buf] ^= 1u;
+        acc_ph ^= 1u;
         tc_fence_after_sync();
-        uint32_t v[16];
-        tmem_ld_32x16(tmem_base + lane_base + kColD + static_cast<uint32_t>(buf * 16), v);
-        tmem_ld_wait();
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&acc_empty[buf]);  // values are in registers: the accumulator may be reused
-        buf ^= 1;
-        float r[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) r[j] = __uint_as_float(v[2 * j]) + __uint_as_float(v[2 * j + 1]);
         if (STAGE1) {
-          // lanes 0..63 gate, 64..127 up: up values go through shared memory, then each gate thread owns
-          // (i, 8 tokens); a warp holds 32 consecutive i = one scale block of the stage-2 operand
-          if (q >= 2) {
+          const int n_blk = a.I / 32;
+#pragma unroll 1
+          for (int m = 0; m < 4; ++m) {  // 32 consecutive i: gate in columns 32m.., up in columns 128 + 32m..
+            uint32_t g[32], u[32];
+            tmem_ld_32x32(tmem_base + kColD + static_cast<uint32_t>(32 * m), g);
+            tmem_ld_32x32(tmem_base + kColD + static_cast<uint32_t>(128 + 32 * m), u);
+            tmem_ld_wait();
+            if (m == 3) {
+              tc_fence_before_sync();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(acc_empty);  // last read of this accumulator
+            }
+            float av[32];
+            float amax = 0.0f;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) sX[((q - 2) * 32 + lane) * 9 + j] = r[j];
-          }
-          asm volatile("bar.sync 2, 128;" ::: "memory");
-          if (q < 2) {
-            const int i = tile * 64 + q * 32 + lane;
-            const int n_blk = a.I / 32;
+            for (int c = 0; c < 32; ++c) {
+              float gv = __uint_as_float(g[c]), uv = __uint_as_float(u[c]);
+              gv += __shfl_xor_sync(0xffffffffu, gv, 1);  // hi + lo
+              uv += __shfl_xor_sync(0xffffffffu, uv, 1);
+              const float t = __fdividef(gv, 1.0f + __expf(-gv)) * uv;
+              av[c] = __bfloat162float(__float2bfloat16_rn(t));  // the intermediate is defined as a bf16 value
+              amax = fmaxf(amax, fabsf(av[c]));
+            }
+            int se = (amax > 0.0f) ? block_exp(amax) : 0;
+            se = max(-120, min(se, 120));
+            const float inv = pow2f(-se);
+            uint32_t hw[8], lw[8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const int p = row0 + j;
-              const float u = sX[(q * 32 + lane) * 9 + j];
-              const float g = r[j];
-              float av = __fdividef(g, 1.0f + __expf(-g)) * u;
-              av = __bfloat162float(__float2bfloat16_rn(av));  // the intermediate is defined as a bf16 value
-              float amax = fabsf(av);
+            for (int i = 0; i < 8; ++i) {
+              uint32_t hacc = 0u, lacc = 0u;
 #pragma unroll
-              for (int d = 16; d > 0; d >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, d));
-              int se = (amax > 0.0f) ? block_exp(amax) : 0;
-              se = max(-120, min(se, 120));
-              uint32_t h, l;
-              split_e4m3(av * pow2f(-se), &h, &l);
-              if (p < row_end) {
-                a.aq_out[static_cast<size_t>(2 * p) * a.I + i] = static_cast<uint8_t>(h);
-                a.aq_out[static_cast<size_t>(2 * p + 1) * a.I + i] = static_cast<uint8_t>(l);
-                if (lane == 0) {
-                  a.aq_sf_out[static_cast<size_t>(2 * p) * n_blk + (i >> 5)] = static_cast<uint8_t>(se + 127);
-                  a.aq_sf_out[static_cast<size_t>(2 * p + 1) * n_blk + (i >> 5)] = static_cast<uint8_t>(se - 3 + 127);
-                }
+              for (int t = 0; t < 4; ++t) {
+                uint32_t h, l;
+                split_e4m3(av[4 * i + t] * inv, &h, &l);
+                hacc |= h << (8 * t);
+                lacc |= l << (8 * t);
               }
+              hw[i] = hacc;
+              lw[i] = lacc;
+            }
+            if (writer && p < row_end) {
+              const int i0 = tile * 128 + 32 * m;
+              uint4* dh = reinterpret_cast<uint4*>(a.aq_out + static_cast<size_t>(2 * p) * a.I + i0);
+              uint4* dl = reinterpret_cast<uint4*>(a.aq_out + static_cast<size_t>(2 * p + 1) * a.I + i0);
+              dh[0] = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+              dh[1] = make_uint4(hw[4], hw[5], hw[6], hw[7]);
+              dl[0] = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+              dl[1] = make_uint4(lw[4], lw[5], lw[6], lw[7]);
+              a.aq_sf_out[static_cast<size_t>(2 * p) * n_blk + (i0 >> 5)] = static_cast<uint8_t>(se + 127);
+              a.aq_sf_out[static_cast<size_t>(2 * p + 1) * n_blk + (i0 >> 5)] = static_cast<uint8_t>(se - 3 + 127);
             }
           }
-          asm volatile("bar.sync 2, 128;" ::: "memory");
         } else {
-          const int n = tile * kTile + q * 32 + lane;
+#pragma unroll 1
+          for (int m = 0; m < 8; ++m) {  // 32 consecutive output columns
+            uint32_t v[32];
+            tmem_ld_32x32(tmem_base + kColD + static_cast<uint32_t>(32 * m), v);
+            tmem_ld_wait();
+            if (m == 7) {
+              tc_fence_before_sync();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(acc_empty);
+            }
+            float r[32];
 #pragma unroll
-          for (int j = 0; j < 8; ++j)
-            if (row0 + j < row_end) a.y[static_cast<size_t>(row0 + j) * a.R + n] = r[j];
+            for (int c = 0; c < 32; ++c) {
+              const float t = __uint_as_float(v[c]);
+              r[c] = t + __shfl_xor_sync(0xffffffffu, t, 1);  // hi + lo
+            }
+            if (writer && p < row_end) {
+              float4* dst = reinterpret_cast<float4*>(a.y + static_cast<size_t>(p) * a.R + tile * kTile + 32 * m);
+#pragma unroll
+              for (int c = 0; c < 8; ++c) dst[c] = make_float4(r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
+            }
+          }
         }
       }
     }
@@ -548,12 +578,12 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
   uint8_t* aq_sf = aq + align_up(2 * S * sh.I, kAlign);
   CUtensorMap tm_w13, tm_w2, tm_s13, tm_s2;
   if (!nat_map(&tm_w13, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, w13, sh.H, sh.H / 2, static_cast<uint64_t>(sh.E) * 2 * sh.I, kKStep,
-               64, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !nat_map(&tm_w2, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, w2, sh.I, sh.I / 2, static_cast<uint64_t>(sh.E) * sh.H, kKStep, 64,
+               128, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !nat_map(&tm_w2, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, w2, sh.I, sh.I / 2, static_cast<uint64_t>(sh.E) * sh.H, kKStep, 128,
                CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !nat_map(&tm_s13, CU_TENSOR_MAP_DATA_TYPE_UINT8, s13, sh.H / 32, sh.H / 32, static_cast<uint64_t>(sh.E) * 2 * sh.I, 16, 64,
+      !nat_map(&tm_s13, CU_TENSOR_MAP_DATA_TYPE_UINT8, s13, sh.H / 32, sh.H / 32, static_cast<uint64_t>(sh.E) * 2 * sh.I, 16, 128,
                CU_TENSOR_MAP_SWIZZLE_NONE) ||
-      !nat_map(&tm_s2, CU_TENSOR_MAP_DATA_TYPE_UINT8, s2, sh.I / 32, sh.I / 32, static_cast<uint64_t>(sh.E) * sh.H, 16, 64,
+      !nat_map(&tm_s2, CU_TENSOR_MAP_DATA_TYPE_UINT8, s2, sh.I / 32, sh.I / 32, static_cast<uint64_t>(sh.E) * sh.H, 16, 128,
                CU_TENSOR_MAP_SWIZZLE_NONE))
     return MOE_ERR_CUDA;
   const int grid = sm_count();
