@@ -176,6 +176,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="decode workloads: launch the four calls eagerly instead of replaying CUDA graphs")
     args = ap.parse_args()
 
     from paper_2609_15627_b200 import inputs
@@ -231,16 +232,17 @@ def main():
         off = buf.expert_offsets.cpu().numpy()
         touched.append(int(np.count_nonzero(np.diff(off))))
 
-    def step(i, ev=None):
+    def step(i, ev=None, st=stream):
+        """The four C-ABI calls on batch i of the cycle (st=None: torch's current stream, used during capture)."""
         l, x = batches[i % n_cycle]
-        moe.moe_route(l, wl.k, buf.topk_ids, buf.topk_w, buf.expert_offsets, buf.ws, stream)
-        moe.moe_permute(x, buf.topk_ids, buf.expert_offsets, sh, buf.x_perm, buf.perm, buf.inv_perm, buf.ws, stream)
+        moe.moe_route(l, wl.k, buf.topk_ids, buf.topk_w, buf.expert_offsets, buf.ws, st)
+        moe.moe_permute(x, buf.topk_ids, buf.expert_offsets, sh, buf.x_perm, buf.perm, buf.inv_perm, buf.ws, st)
         if ev is not None:
-            ev[0].record(stream)
-        moe.moe_expert_ffn(buf.x_perm, buf.expert_offsets, *weights, sh, buf.y_perm, buf.status, buf.ws, stream)
+            ev[0].record(st)
+        moe.moe_expert_ffn(buf.x_perm, buf.expert_offsets, *weights, sh, buf.y_perm, buf.status, buf.ws, st)
         if ev is not None:
-            ev[1].record(stream)
-        moe.moe_combine(buf.y_perm, buf.inv_perm, buf.topk_w, sh, buf.out, stream)
+            ev[1].record(st)
+        moe.moe_combine(buf.y_perm, buf.inv_perm, buf.topk_w, sh, buf.out, st)
 
     def barrier():
         if world > 1:
@@ -251,6 +253,29 @@ def main():
         step(i)
     barrier()
 
+    # Decode-sized steps are a handful of short kernels: like the paper's decode tiers they are replayed as CUDA
+    # graphs (one graph per batch of the cycle, each the four C-ABI calls captured as they are).
+    use_graph = decode and not args.no_graph
+    graphs, launches_per_step = [], None
+    if use_graph:
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            for i in range(3):
+                step(i, st=None)
+        stream.wait_stream(side)
+        barrier()
+        for i in range(n_cycle):
+            g = torch.cuda.CUDAGraph()
+            c0 = moe.moe_launch_count()
+            with torch.cuda.graph(g):
+                step(i, st=None)
+            launches_per_step = moe.moe_launch_count() - c0
+            graphs.append(g)
+        for i in range(max(args.warmup, 3)):
+            graphs[i % n_cycle].replay()
+        barrier()
+
     # ---- timed region: exactly K steps ---------------------------------------------------------------------
     n_inner = min(args.steps, 256)  # steps whose expert-FFN call is bracketed by its own events
     inner = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_inner)]
@@ -260,16 +285,31 @@ def main():
     barrier()
     sampler.start()
     e0.record(stream)
-    for i in range(args.steps):
-        step(i, inner[i] if i < n_inner else None)
+    if use_graph:
+        for i in range(args.steps):
+            graphs[i % n_cycle].replay()
+    else:
+        for i in range(args.steps):
+            step(i, inner[i] if i < n_inner else None)
     e1.record(stream)
     barrier()
     clocks = sampler.stop()
-    launches = moe.moe_launch_count() - launches0
+    launches = launches_per_step * args.steps if use_graph else moe.moe_launch_count() - launches0
     assert int(buf.status.item()) == 0, "device-side wait timed out"
     ms_total = max_over_ranks(e0.elapsed_time(e1), world)
     ms_step = ms_total / args.steps
     value = wl.T * world / (ms_step * 1e-3)
+    eager_ms_step = None
+    if use_graph:
+        # the expert-FFN call cannot be bracketed by events inside a graph: time it in a second region of eager
+        # steps on the same batches, right after the timed one
+        ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ee0.record(stream)
+        for i in range(n_inner):
+            step(i, inner[i])
+        ee1.record(stream)
+        barrier()
+        eager_ms_step = ee0.elapsed_time(ee1) / n_inner
 
     # ---- roofline of the dominant call (the expert FFN) --------------------------------------------------------
     ffn_ms = float(np.mean([a.elapsed_time(b) for a, b in inner]))
@@ -287,7 +327,8 @@ def main():
                 "frac": achieved / peaks["tensor_sustained"], "traffic": NCU_TRAFFIC_BYTES.get(wl.name),
                 "algorithmic_flops": fl}
     roof.update({"kernel": "moe_expert_ffn",
-                 "ms": ffn_ms, "peak_source": peaks["source"], "experts_touched": mean_touched})
+                 "ms": ffn_ms, "peak_source": peaks["source"], "experts_touched": mean_touched,
+                 "timed_in": "eager steps right after the graph-replayed region" if use_graph else "the timed region"})
 
     # ---- end to end through the host-buffer entry point ---------------------------------------------------------
     e2e = None
@@ -323,6 +364,8 @@ def main():
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": wl.name, "T": wl.T, "H": wl.H, "I": wl.I, "E": wl.E, "k": wl.k,
                        "parallelism": "replicas only" if world > 1 else "1 GPU",
+                       "launch": "cuda graph replay, one graph per batch of the cycle" if use_graph else "eager",
+                       "eager_ms_per_step": eager_ms_step,
                        "l2": "inputs cycle over %d seeded batches; %.2f GB of expert weights resident (larger than L2)"
                              % (n_cycle, wl.E * expert_weight_bytes(wl.H, wl.I) / 1e9)},
             "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
