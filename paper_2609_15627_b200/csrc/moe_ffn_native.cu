@@ -160,13 +160,21 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
 
   // ---- setup: touched experts, barriers, tensor memory ----
   if (wid == 2) {
+    // lane l looks at experts l, l + 32, ...: all loads are issued before any is used (one memory round trip)
+    unsigned has_mask = 0u;
+#pragma unroll 8
+    for (int i = 0; i < (a.E + 31) / 32; ++i) {
+      const int e = i * 32 + lane;
+      const int lo = (e < a.E) ? __ldg(a.offsets + e) : 0;
+      const int hi = (e < a.E) ? __ldg(a.offsets + e + 1) : 0;
+      has_mask |= (hi > lo ? 1u : 0u) << i;
+    }
     int run = 0;
-    for (int e0 = 0; e0 < a.E; e0 += 32) {
-      const int e = e0 + lane;
-      const int has = (e < a.E && a.offsets[e + 1] > a.offsets[e]) ? 1 : 0;
+    for (int i = 0; i < (a.E + 31) / 32; ++i) {
+      const int has = static_cast<int>((has_mask >> i) & 1u);
       int tot;
       const int ex = warp_excl_scan(has, lane, &tot);
-      if (has) touched[run + ex] = e;
+      if (has) touched[run + ex] = i * 32 + lane;
       run += tot;
     }
     if (lane == 0) s_misc[0] = run;
@@ -186,6 +194,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_holder;
+  // Programmatic dependent launch: the down-projection grid may start its set-up and its weight stream while this
+  // grid is still running; it waits (griddepcontrol.wait) before it reads what this grid writes.
+  if (STAGE1) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int n_touched = s_misc[0];
   const long long total_items = static_cast<long long>(n_touched) * tiles_per_expert;
   const long long per_cta = (total_items + gridDim.x - 1) / gridDim.x;
@@ -350,6 +361,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
               sSfa[rl * n_blk + b] = static_cast<unsigned char>(sb_lo);
             }
           } else {
+            asm volatile("griddepcontrol.wait;" ::: "memory");  // stage 1 is complete and its writes are visible
             // stage 2: the split rows were written by stage 1; copy 16-byte chunks into the swizzled layout
             const int chunks_per_row = K / 16;
             for (int task = st; task < 16 * chunks_per_row; task += 128) {
@@ -604,8 +616,20 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
   if (cudaGetLastError() != cudaSuccess) return MOE_ERR_CUDA;
   a.K = sh.I;
   a.R = sh.H;
-  ffn_native_kernel<false><<<grid, kNatThreads, nat_smem(sh.E, sh.I).total + 1024, st>>>(tm_w2, tm_s2, a);
-  if (cudaGetLastError() != cudaSuccess) return MOE_ERR_CUDA;
+  {
+    // launched as a programmatic dependent of stage 1 (see the kernel)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kNatThreads);
+    cfg.dynamicSmemBytes = nat_smem(sh.E, sh.I).total + 1024;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, ffn_native_kernel<false>, tm_w2, tm_s2, a) != cudaSuccess) return MOE_ERR_CUDA;
+  }
   note_kernel("ffn_native_mxf4_block_scaled", 2);
   return MOE_OK;
 }
