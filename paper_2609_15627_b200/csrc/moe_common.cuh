@@ -70,7 +70,29 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
 
 int sm_count();
 
+// ---- programmatic dependent launch (host) ------------------------------------------------------
+// The kernel may start while its predecessor in the stream is still running; it must execute
+// griddepcontrol.wait before it touches anything the predecessor writes or reads.  Every kernel launched
+// this way here waits first and only then lets its own dependent start, so at most two neighbours overlap.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---- small device helpers ---------------------------------------------------------------------
+MOE_DEVINL void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+MOE_DEVINL void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 MOE_DEVINL int warp_excl_scan(int v, int lane, int* total) {
   int incl = v;
 #pragma unroll

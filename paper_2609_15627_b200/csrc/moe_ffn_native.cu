@@ -194,9 +194,12 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_holder;
-  // Programmatic dependent launch: the down-projection grid may start its set-up and its weight stream while this
-  // grid is still running; it waits (griddepcontrol.wait) before it reads what this grid writes.
-  if (STAGE1) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // Programmatic dependent launch: the next grid (down projection after gate/up, combine after down) may start its
+  // set-up - and the down projection its weight stream - while this grid is still running; it waits
+  // (griddepcontrol.wait) before it reads what this grid writes.  This grid in turn reads nothing of its own
+  // predecessor before its scale warps have waited (below), apart from expert_offsets, which the router finished
+  // before that predecessor was allowed to start this grid.
+  pdl_launch_dependents();
   const int n_touched = s_misc[0];
   const long long total_items = static_cast<long long>(n_touched) * tiles_per_expert;
   const long long per_cta = (total_items + gridDim.x - 1) / gridDim.x;
@@ -309,6 +312,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
           const int row0 = row_begin + pass * kMaxTokPass;
           const int n_blk = K / 32;
           if (STAGE1) {
+            pdl_wait();  // the sorted token rows of moe_permute are complete
             // task = (token j, 32-element block b): 8 * K/32 tasks over 128 threads
             for (int task = st; task < kMaxTokPass * n_blk; task += 128) {
               const int j = task / n_blk, b = task % n_blk;
@@ -361,7 +365,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
               sSfa[rl * n_blk + b] = static_cast<unsigned char>(sb_lo);
             }
           } else {
-            asm volatile("griddepcontrol.wait;" ::: "memory");  // stage 1 is complete and its writes are visible
+            pdl_wait();  // stage 1 is complete and its writes are visible
             // stage 2: the split rows were written by stage 1; copy 16-byte chunks into the swizzled layout
             const int chunks_per_row = K / 16;
             for (int task = st; task < 16 * chunks_per_row; task += 128) {
@@ -612,24 +616,14 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
   a.I = sh.I;
   a.K = sh.H;
   a.R = 2 * sh.I;
-  ffn_native_kernel<true><<<grid, kNatThreads, nat_smem(sh.E, sh.H).total + 1024, st>>>(tm_w13, tm_s13, a);
-  if (cudaGetLastError() != cudaSuccess) return MOE_ERR_CUDA;
+  if (launch_pdl(ffn_native_kernel<true>, dim3(grid), dim3(kNatThreads), nat_smem(sh.E, sh.H).total + 1024, st, tm_w13, tm_s13,
+                 a) != cudaSuccess)
+    return MOE_ERR_CUDA;
   a.K = sh.I;
   a.R = sh.H;
-  {
-    // launched as a programmatic dependent of stage 1 (see the kernel)
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(kNatThreads);
-    cfg.dynamicSmemBytes = nat_smem(sh.E, sh.I).total + 1024;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, ffn_native_kernel<false>, tm_w2, tm_s2, a) != cudaSuccess) return MOE_ERR_CUDA;
-  }
+  if (launch_pdl(ffn_native_kernel<false>, dim3(grid), dim3(kNatThreads), nat_smem(sh.E, sh.I).total + 1024, st, tm_w2, tm_s2,
+                 a) != cudaSuccess)
+    return MOE_ERR_CUDA;
   note_kernel("ffn_native_mxf4_block_scaled", 2);
   return MOE_OK;
 }

@@ -120,6 +120,7 @@ __global__ void __launch_bounds__(1024) route_kernel(const float* __restrict__ l
   int* s_counts = reinterpret_cast<int*>(sm_f + nw * E);  // [E]
   int* s_misc = s_counts + E;                           // [32] + flag
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  pdl_launch_dependents();  // route itself is launched in plain stream order; its dependent waits before it reads
   if (single_block) {
     for (int e = tid; e < E; e += blockDim.x) s_counts[e] = 0;
     __syncthreads();
@@ -202,6 +203,8 @@ __global__ void __launch_bounds__(256) permute_small_kernel(const __nv_bfloat16*
                                                             int* __restrict__ perm, int* __restrict__ inv_perm) {
   const int lane = threadIdx.x & 31;
   const int s = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  pdl_wait();                // the router's ids and offsets are complete
+  pdl_launch_dependents();   // the expert FFN may set up and start its weight stream
   if (s >= S) return;
   const int e = ids[s];
   int c = 0;
@@ -309,7 +312,9 @@ int launch_permute(const __nv_bfloat16* x, const int* ids, const int* offsets, c
                    __nv_bfloat16* x_perm, int* perm, int* inv_perm, int* block_counts, cudaStream_t st) {
   const int S = sh.T * sh.k;
   if (S <= 4096) {
-    permute_small_kernel<<<(S + 7) / 8, 256, 0, st>>>(x, ids, offsets, S, sh.H, sh.k, x_perm, perm, inv_perm);
+    if (launch_pdl(permute_small_kernel, dim3((S + 7) / 8), dim3(256), 0, st, x, ids, offsets, S, sh.H, sh.k, x_perm, perm,
+                   inv_perm) != cudaSuccess)
+      return MOE_ERR_CUDA;
     note_kernel("permute_rank_by_count", 1);
   } else {
     const int nblk = (S + kPermuteChunk - 1) / kPermuteChunk;
@@ -333,6 +338,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
                                                       __nv_bfloat16* __restrict__ out) {
   const int groups = H / 8;
   const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  pdl_wait();  // the per-slot rows of the expert FFN are complete
   if (idx >= static_cast<size_t>(T) * groups) return;
   const int t = static_cast<int>(idx / groups);
   const int c = static_cast<int>(idx % groups) * 8;
@@ -362,7 +368,9 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
 int launch_combine(const float* y_perm, const int* inv_perm, const float* w, const moe_shape_t& sh,
                    __nv_bfloat16* out, cudaStream_t st) {
   const size_t n = static_cast<size_t>(sh.T) * (sh.H / 8);
-  combine_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(y_perm, inv_perm, w, sh.T, sh.H, sh.k, out);
+  if (launch_pdl(combine_kernel, dim3(static_cast<unsigned>((n + 255) / 256)), dim3(256), 0, st, y_perm, inv_perm, w, sh.T,
+                 sh.H, sh.k, out) != cudaSuccess)
+    return MOE_ERR_CUDA;
   note_kernel("combine_slot_order_fma", 1);
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
