@@ -103,6 +103,15 @@ int moe_permute(const void* x_bf16, const int32_t* topk_ids, const int32_t* expe
  *   y_perm[p,:] = W2_e a                  (fp32, one store per (slot, column), no atomics)
  * The summation order inside a dot product is the kernel's; everything else is as written.
  *   status_word: device int32, may be NULL; see the common rules.
+ * Three kernel variants, chosen by the shape alone (moe_last_kernel_name names the one that ran): for
+ * decode-sized batches (T*k <= 32*E, H and I multiples of 512) the packed weights feed the block-scaled FP4
+ * tensor-core instruction directly and each bf16 activation row is split into two E4M3 rows that add up to it
+ * (exact unless an element is more than 2^14 below its 32-block's maximum; then off by < 2^-19 of that maximum);
+ * for prefill-sized batches (T*k >= 1024) weights are expanded to bf16 exactly on chip for a bf16 grouped GEMM;
+ * every other supported shape uses a register-expansion streaming kernel.
+ * Launch order: the decode-sized kernels use programmatic dependent launch.  They read expert_offsets and the
+ * weights before waiting for the kernel launched just before them on the stream, and x_perm only after it has
+ * completed: expert_offsets must not be written by that immediately preceding kernel (moe_permute does not).
  */
 int moe_expert_ffn(const void* x_perm_bf16 /* [T*k,H] */, const int32_t* expert_offsets,
                    const uint8_t* w13, const uint8_t* w13_scale, const uint8_t* w2, const uint8_t* w2_scale,
