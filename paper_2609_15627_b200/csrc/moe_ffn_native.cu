@@ -356,7 +356,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
               }
               const int ks = b >> 2, c16 = (b & 3) * 2;  // K step, first 16-byte chunk of the 128-byte row
               unsigned char* base = sAct + ks * 2048;
-              const int rh = 2 * j, rl = 2 * j + 1;
+              const int rh = j, rl = 8 + j;  // operand rows 0..7 = hi, 8..15 = lo of tokens 0..7
               *reinterpret_cast<uint4*>(base + rh * 128 + (((c16) ^ (rh & 7)) << 4)) = make_uint4(hi_w[0], hi_w[1], hi_w[2], hi_w[3]);
               *reinterpret_cast<uint4*>(base + rh * 128 + (((c16 + 1) ^ (rh & 7)) << 4)) = make_uint4(hi_w[4], hi_w[5], hi_w[6], hi_w[7]);
               *reinterpret_cast<uint4*>(base + rl * 128 + (((c16) ^ (rl & 7)) << 4)) = make_uint4(lo_w[0], lo_w[1], lo_w[2], lo_w[3]);
@@ -370,16 +370,16 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
             const int chunks_per_row = K / 16;
             for (int task = st; task < 16 * chunks_per_row; task += 128) {
               const int r = task / chunks_per_row, c = task % chunks_per_row;
-              const int p = row0 + (r >> 1);
+              const int p = row0 + (r & 7);  // operand row r: token r & 7, hi (r < 8) or lo
               uint4 v = make_uint4(0u, 0u, 0u, 0u);
-              if (p < row_end) v = __ldcg(reinterpret_cast<const uint4*>(a.aq + (static_cast<size_t>(2 * p + (r & 1))) * K + c * 16));
+              if (p < row_end) v = __ldcg(reinterpret_cast<const uint4*>(a.aq + (static_cast<size_t>(2 * p + (r >> 3))) * K + c * 16));
               const int ks = c >> 3, c16 = c & 7;
               *reinterpret_cast<uint4*>(sAct + ks * 2048 + r * 128 + ((c16 ^ (r & 7)) << 4)) = v;
             }
             for (int task = st; task < 16 * n_blk; task += 128) {
               const int r = task / n_blk, b = task % n_blk;
-              const int p = row0 + (r >> 1);
-              sSfa[r * n_blk + b] = (p < row_end) ? a.aq_sf[(static_cast<size_t>(2 * p + (r & 1))) * n_blk + b] : static_cast<unsigned char>(127);
+              const int p = row0 + (r & 7);
+              sSfa[r * n_blk + b] = (p < row_end) ? a.aq_sf[(static_cast<size_t>(2 * p + (r >> 3))) * n_blk + b] : static_cast<unsigned char>(127);
             }
           }
           fence_proxy_async_smem();
@@ -428,17 +428,17 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       }
     }
   } else if (wid == kEpiWarp) {
-    // =========================== epilogue (tensor-memory lanes 0..15: row 2j = hi, 2j+1 = lo of token j) ===========================
+    // =========================== epilogue (tensor-memory lanes 0..7 = hi, 8..15 = lo of tokens 0..7) ===========================
+    // The 16x256b load hands thread t lane t/4 and lane t/4 + 8 of the same two columns: hi + lo is thread-local.
     uint32_t acc_ph = 0;
-    const bool writer = (lane < 16) && ((lane & 1) == 0);
-    const int j = lane >> 1;
+    const int j = lane >> 2, cp = lane & 3;  // token of this thread, column pair inside a group of 8 columns
     for (long long it = item_begin; it < item_end; ++it) {
       const int e = touched[it / tiles_per_expert];
       const int tile = static_cast<int>(it % tiles_per_expert);
       const int row_begin = a.offsets[e], row_end = a.offsets[e + 1];
       const int n_pass = (row_end - row_begin + kMaxTokPass - 1) / kMaxTokPass;
       for (int pass = 0; pass < n_pass; ++pass) {
-        const int p = row_begin + pass * kMaxTokPass + j;  // sorted row of this lane pair's token
+        const int p = row_begin + pass * kMaxTokPass + j;  // sorted row of this thread's token
         mbar_wait(acc_full, acc_ph, a.status);
         __syncwarp();  // tcgen05.ld is warp-collective
         acc_ph ^= 1u;
@@ -447,76 +447,70 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
           const int n_blk = a.I / 32;
 #pragma unroll 1
           for (int m = 0; m < 4; ++m) {  // 32 consecutive i: gate in columns 32m.., up in columns 128 + 32m..
-            uint32_t g[32], u[32];
-            tmem_ld_32x32(tmem_base + kColD + static_cast<uint32_t>(32 * m), g);
-            tmem_ld_32x32(tmem_base + kColD + static_cast<uint32_t>(128 + 32 * m), u);
+            uint32_t g[16], u[16];
+            tmem_ld_16x256b_x4(tmem_base + kColD + static_cast<uint32_t>(32 * m), g);
+            tmem_ld_16x256b_x4(tmem_base + kColD + static_cast<uint32_t>(128 + 32 * m), u);
             tmem_ld_wait();
             if (m == 3) {
               tc_fence_before_sync();
               __syncwarp();
               if (lane == 0) mbar_arrive(acc_empty);  // last read of this accumulator
             }
-            float av[32];
+            float av[8];
             float amax = 0.0f;
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-              float gv = __uint_as_float(g[c]), uv = __uint_as_float(u[c]);
-              gv += __shfl_xor_sync(0xffffffffu, gv, 1);  // hi + lo
-              uv += __shfl_xor_sync(0xffffffffu, uv, 1);
-              const float t = __fdividef(gv, 1.0f + __expf(-gv)) * uv;
-              av[c] = __bfloat162float(__float2bfloat16_rn(t));  // the intermediate is defined as a bf16 value
-              amax = fmaxf(amax, fabsf(av[c]));
+            for (int i = 0; i < 4; ++i) {
+#pragma unroll
+              for (int t = 0; t < 2; ++t) {
+                const float gv = __uint_as_float(g[4 * i + t]) + __uint_as_float(g[4 * i + 2 + t]);  // hi + lo
+                const float uv = __uint_as_float(u[4 * i + t]) + __uint_as_float(u[4 * i + 2 + t]);
+                const float sv = __fdividef(gv, 1.0f + __expf(-gv)) * uv;
+                av[2 * i + t] = __bfloat162float(__float2bfloat16_rn(sv));  // the intermediate is defined as a bf16 value
+                amax = fmaxf(amax, fabsf(av[2 * i + t]));
+              }
             }
+            // the 32 values of this token's scale block sit in the 4 threads of the token
+            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
             int se = (amax > 0.0f) ? block_exp(amax) : 0;
             se = max(-120, min(se, 120));
             const float inv = pow2f(-se);
-            uint32_t hw[8], lw[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              uint32_t hacc = 0u, lacc = 0u;
-#pragma unroll
-              for (int t = 0; t < 4; ++t) {
-                uint32_t h, l;
-                split_e4m3(av[4 * i + t] * inv, &h, &l);
-                hacc |= h << (8 * t);
-                lacc |= l << (8 * t);
-              }
-              hw[i] = hacc;
-              lw[i] = lacc;
-            }
-            if (writer && p < row_end) {
+            if (p < row_end) {
               const int i0 = tile * 128 + 32 * m;
-              uint4* dh = reinterpret_cast<uint4*>(a.aq_out + static_cast<size_t>(2 * p) * a.I + i0);
-              uint4* dl = reinterpret_cast<uint4*>(a.aq_out + static_cast<size_t>(2 * p + 1) * a.I + i0);
-              dh[0] = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-              dh[1] = make_uint4(hw[4], hw[5], hw[6], hw[7]);
-              dl[0] = make_uint4(lw[0], lw[1], lw[2], lw[3]);
-              dl[1] = make_uint4(lw[4], lw[5], lw[6], lw[7]);
-              a.aq_sf_out[static_cast<size_t>(2 * p) * n_blk + (i0 >> 5)] = static_cast<uint8_t>(se + 127);
-              a.aq_sf_out[static_cast<size_t>(2 * p + 1) * n_blk + (i0 >> 5)] = static_cast<uint8_t>(se - 3 + 127);
+              uint8_t* dh = a.aq_out + static_cast<size_t>(2 * p) * a.I + i0 + 2 * cp;
+              uint8_t* dl = a.aq_out + static_cast<size_t>(2 * p + 1) * a.I + i0 + 2 * cp;
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                uint32_t h0, l0, h1, l1;
+                split_e4m3(av[2 * i] * inv, &h0, &l0);
+                split_e4m3(av[2 * i + 1] * inv, &h1, &l1);
+                *reinterpret_cast<uint16_t*>(dh + 8 * i) = static_cast<uint16_t>(h0 | (h1 << 8));
+                *reinterpret_cast<uint16_t*>(dl + 8 * i) = static_cast<uint16_t>(l0 | (l1 << 8));
+              }
+              if (cp == 0) {
+                a.aq_sf_out[static_cast<size_t>(2 * p) * n_blk + (i0 >> 5)] = static_cast<uint8_t>(se + 127);
+                a.aq_sf_out[static_cast<size_t>(2 * p + 1) * n_blk + (i0 >> 5)] = static_cast<uint8_t>(se - 3 + 127);
+              }
             }
           }
         } else {
 #pragma unroll 1
-          for (int m = 0; m < 8; ++m) {  // 32 consecutive output columns
+          for (int m = 0; m < 4; ++m) {  // 64 consecutive output columns
             uint32_t v[32];
-            tmem_ld_32x32(tmem_base + kColD + static_cast<uint32_t>(32 * m), v);
+            tmem_ld_16x256b_x8(tmem_base + kColD + static_cast<uint32_t>(64 * m), v);
             tmem_ld_wait();
-            if (m == 7) {
+            if (m == 3) {
               tc_fence_before_sync();
               __syncwarp();
               if (lane == 0) mbar_arrive(acc_empty);
             }
-            float r[32];
+            if (p < row_end) {
+              float* dst = a.y + static_cast<size_t>(p) * a.R + tile * kTile + 64 * m + 2 * cp;
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-              const float t = __uint_as_float(v[c]);
-              r[c] = t + __shfl_xor_sync(0xffffffffu, t, 1);  // hi + lo
-            }
-            if (writer && p < row_end) {
-              float4* dst = reinterpret_cast<float4*>(a.y + static_cast<size_t>(p) * a.R + tile * kTile + 32 * m);
-#pragma unroll
-              for (int c = 0; c < 8; ++c) dst[c] = make_float4(r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
+              for (int i = 0; i < 8; ++i)
+                *reinterpret_cast<float2*>(dst + 8 * i) =
+                    make_float2(__uint_as_float(v[4 * i]) + __uint_as_float(v[4 * i + 2]),
+                                __uint_as_float(v[4 * i + 1]) + __uint_as_float(v[4 * i + 3]));
             }
           }
         }
