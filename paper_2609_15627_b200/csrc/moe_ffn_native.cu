@@ -310,15 +310,17 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
           }
           first_op = false;
           const int row0 = row_begin + pass * kMaxTokPass;
+          const int n_tok = min(kMaxTokPass, row_end - row0);
           const int n_blk = K / 32;
           if (STAGE1) {
             pdl_wait();  // the sorted token rows of moe_permute are complete
-            // task = (token j, 32-element block b): 8 * K/32 tasks over 128 threads
-            for (int task = st; task < kMaxTokPass * n_blk; task += 128) {
+            // task = (token j, 32-element block b) over the tokens that exist: operand rows of absent tokens keep
+            // whatever shared memory holds - their accumulator lanes are never read and rows do not mix
+            for (int task = st; task < n_tok * n_blk; task += 128) {
               const int j = task / n_blk, b = task % n_blk;
               uint32_t hi_w[8], lo_w[8];
-              uint32_t sb_hi = 127u, sb_lo = 127u;
-              if (row0 + j < row_end) {
+              uint32_t sb_hi, sb_lo;
+              {
                 const uint4* src = reinterpret_cast<const uint4*>(a.x + static_cast<size_t>(row0 + j) * K + b * 32);
                 uint4 v[4];
 #pragma unroll
@@ -350,9 +352,6 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
                   hi_w[i] = hw;
                   lo_w[i] = lw;
                 }
-              } else {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) { hi_w[i] = 0u; lo_w[i] = 0u; }
               }
               const int ks = b >> 2, c16 = (b & 3) * 2;  // K step, first 16-byte chunk of the 128-byte row
               unsigned char* base = sAct + ks * 2048;
@@ -367,19 +366,36 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
           } else {
             pdl_wait();  // stage 1 is complete and its writes are visible
             // stage 2: the split rows were written by stage 1; copy 16-byte chunks into the swizzled layout
+            // operand row r = 8 * half + j (half 0 = hi, 1 = lo) comes from row 2 * (row0 + j) + half of the split
+            // activations; only the rows of tokens that exist are copied, four 16-byte chunks in flight per thread
             const int chunks_per_row = K / 16;
-            for (int task = st; task < 16 * chunks_per_row; task += 128) {
-              const int r = task / chunks_per_row, c = task % chunks_per_row;
-              const int p = row0 + (r & 7);  // operand row r: token r & 7, hi (r < 8) or lo
-              uint4 v = make_uint4(0u, 0u, 0u, 0u);
-              if (p < row_end) v = __ldcg(reinterpret_cast<const uint4*>(a.aq + (static_cast<size_t>(2 * p + (r >> 3))) * K + c * 16));
-              const int ks = c >> 3, c16 = c & 7;
-              *reinterpret_cast<uint4*>(sAct + ks * 2048 + r * 128 + ((c16 ^ (r & 7)) << 4)) = v;
+            const int n_chunks = 2 * n_tok * chunks_per_row;
+            for (int base = st; base < n_chunks; base += 4 * 128) {
+              uint4 v[4];
+#pragma unroll
+              for (int u = 0; u < 4; ++u) {
+                const int task = base + u * 128;
+                if (task < n_chunks) {
+                  const int jj = task / chunks_per_row, c = task % chunks_per_row;
+                  const int half = jj >= n_tok ? 1 : 0, j = jj - half * n_tok;
+                  v[u] = __ldcg(reinterpret_cast<const uint4*>(a.aq + (static_cast<size_t>(2 * (row0 + j) + half)) * K + c * 16));
+                }
+              }
+#pragma unroll
+              for (int u = 0; u < 4; ++u) {
+                const int task = base + u * 128;
+                if (task < n_chunks) {
+                  const int jj = task / chunks_per_row, c = task % chunks_per_row;
+                  const int half = jj >= n_tok ? 1 : 0, r = 8 * half + jj - half * n_tok;
+                  const int ks = c >> 3, c16 = c & 7;
+                  *reinterpret_cast<uint4*>(sAct + ks * 2048 + r * 128 + ((c16 ^ (r & 7)) << 4)) = v[u];
+                }
+              }
             }
-            for (int task = st; task < 16 * n_blk; task += 128) {
-              const int r = task / n_blk, b = task % n_blk;
-              const int p = row0 + (r & 7);
-              sSfa[r * n_blk + b] = (p < row_end) ? a.aq_sf[(static_cast<size_t>(2 * p + (r >> 3))) * n_blk + b] : static_cast<unsigned char>(127);
+            for (int task = st; task < 2 * n_tok * n_blk; task += 128) {
+              const int jj = task / n_blk, b = task % n_blk;
+              const int half = jj >= n_tok ? 1 : 0, j = jj - half * n_tok;
+              sSfa[(8 * half + j) * n_blk + b] = a.aq_sf[(static_cast<size_t>(2 * (row0 + j) + half)) * n_blk + b];
             }
           }
           fence_proxy_async_smem();
