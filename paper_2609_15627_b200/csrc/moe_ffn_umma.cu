@@ -5,8 +5,8 @@
 // rows); the 256 rows are two M=128 MMAs that share one token stage in shared memory (each token tile read
 // from L2 feeds twice the math) and own one 256-column accumulator each: all 512 columns of tensor memory.
 // An expert with more than 256 rows is cut into equal passes, so the padding of a ragged expert is at
-// most 15 tokens per pass.  For the gate/up stage each M=128 tile is 64 gate rows (lanes 0..63) plus the
-// matching 64 up rows (lanes 64..127).
+// most 15 tokens per pass.  For the gate/up stage the first M=128 tile is 128 gate rows and the second the 128
+// matching up rows, so gate and up of one i sit in the same tensor-memory lane of the two accumulators.
 //
 // Warp roles (one CTA per SM, persistent):
 //   warp 0       producer: TMA loads of the token tile (bf16, 128-byte swizzle) and of the packed codes
@@ -14,8 +14,9 @@
 //   warps 2..9   one thread per weight row: packed E2M1 codes from the TMA-fed packed ring, exact expansion
 //                to bf16 scaled by the E8M0 block scale, written into the swizzled K-major A stage the
 //                tensor core reads
-//   warps 10..13 epilogue: tcgen05.ld the accumulators; stage 1 transposes through shared memory so that
-//                gate and up meet and act is stored 16 bytes at a time; stage 2 stores fp32 rows
+//   warps 10..17 epilogue, two warps per lane quadrant taking alternate column chunks: tcgen05.ld the
+//                accumulators; stage 1 applies SwiGLU thread-locally (gate and up share a lane) and stores bf16
+//                pairs; stage 2 stores fp32 rows
 // Every mbarrier wait is bounded and reports through the status word.
 #include <cuda.h>
 
@@ -31,8 +32,8 @@ constexpr int kMaxTok = 256;      // tokens per pass
 constexpr int kTokBox = 64;       // token rows per TMA box
 constexpr int kStages = 3;        // A/B ring depth
 constexpr int kDequantWarps = 8;
-constexpr int kEpilogueWarps = 4;
-constexpr int kThreadsUmma = (2 + kDequantWarps + kEpilogueWarps) * 32;  // 448
+constexpr int kEpilogueWarps = 8;
+constexpr int kThreadsUmma = (2 + kDequantWarps + kEpilogueWarps) * 32;  // 576
 constexpr int kFirstDequantWarp = 2;
 constexpr int kFirstEpilogueWarp = 2 + kDequantWarps;  // 10: (warp % 4) = 2,3,0,1 covers the four lane quadrants
 constexpr uint32_t kTmemCols = 512;
@@ -40,8 +41,6 @@ constexpr uint32_t kTmemCols = 512;
 constexpr int kATile = 128 * kBlockK * 2;            // 16 KB: one M=128 tile of a stage
 constexpr int kABytes = 2 * kATile;                  // 32 KB
 constexpr int kBBytes = kMaxTok * kBlockK * 2;       // 32 KB
-constexpr int kTChunk = 16;                          // accumulator columns per stage-1 epilogue step
-constexpr int kTBytes = kTChunk * 128 * 4;           // 8 KB transpose buffer
 constexpr int kPStages = 3;                          // packed-code ring (one K block per stage)
 constexpr int kPBytes = kTileRows * (kBlockK / 2);   // 8 KB: 256 rows x 32 bytes
 
@@ -57,7 +56,7 @@ struct UmmaArgs {
 };
 
 struct SmemMap {
-  uint32_t a, b, p, t, bars, misc, prefix, total;
+  uint32_t a, b, p, bars, misc, prefix, total;
 };
 __host__ __device__ inline SmemMap smem_map(int E) {
   SmemMap m;
@@ -68,8 +67,6 @@ __host__ __device__ inline SmemMap smem_map(int E) {
   off += kStages * kBBytes;
   m.p = off;
   off += kPStages * kPBytes;
-  m.t = off;
-  off += kTBytes;
   m.bars = off;
   off += 32 * 8;
   m.misc = off;
@@ -112,7 +109,6 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
   unsigned char* sA = smem + sm.a;
   unsigned char* sB = smem + sm.b;
   unsigned char* sP = smem + sm.p;
-  float* sT = reinterpret_cast<float*>(smem + sm.t);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sm.bars);
   uint64_t* full_a = bars;                      // [kStages] dequant warps -> MMA
   uint64_t* full_b = bars + kStages;            // [kStages] TMA -> MMA
@@ -236,16 +232,10 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
     for (int w = blockIdx.x; w < total_work; w += gridDim.x) {
       const int g = w / tiles_per_expert, rt = w % tiles_per_expert;
       const int e = find_expert(prefix, a.E, g);
-      int grow;
-      if (STAGE1) {
-        const int i = rt * 128 + t * 64 + (l & 63);
-        grow = e * a.R + (l < 64 ? i : a.I + i);
-      } else {
-        grow = e * a.R + rt * kTileRows + r;
-      }
+      // stage 1: tile 0 = gate rows rt*128.., tile 1 = the matching up rows; stage 2: 256 consecutive rows
+      const int grow = STAGE1 ? e * a.R + t * a.I + rt * 128 + l : e * a.R + rt * kTileRows + r;
       const uint8_t* srow = a.sc + static_cast<size_t>(grow) * (K / 32);
-      // row of this thread inside the packed stage (stage 1: gate rows 0..127, up rows 128..255)
-      const int prow = STAGE1 ? (l < 64 ? t * 64 + l : 128 + t * 64 + (l - 64)) : r;
+      const int prow = r;  // row of this thread inside the packed stage (stage 1: gate rows 0..127, up rows 128..255)
       // scale bytes: 16 bytes cover 8 K blocks; fetched one group ahead
       uint4 sc_cur = __ldg(reinterpret_cast<const uint4*>(srow));
       uint4 sc_next = sc_cur;
@@ -289,8 +279,8 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
     }
   } else {
     // =========================== epilogue ===========================
-    const int q = wid & 3;                         // tensor-memory lane quadrant this warp may read
-    const int te = tid - kFirstEpilogueWarp * 32;  // 0..127
+    const int q = wid & 3;                                // tensor-memory lane quadrant this warp may read
+    const int half = (wid - kFirstEpilogueWarp) >> 2;     // the two warps of a quadrant take alternate column chunks
     const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
     uint32_t acc_ph = 0;
     for (int w = blockIdx.x; w < total_work; w += gridDim.x) {
@@ -301,39 +291,36 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
       mbar_wait(acc_full, acc_ph, a.status);
       __syncwarp();  // tcgen05.ld is warp-collective
       tc_fence_after_sync();
+      if (STAGE1) {
+        // lane = i inside the tile: gate in the first accumulator, up in the second, one token per column.
+        // Neighbouring lanes swap one value per token pair so that each thread stores a bf16 pair (i, i + 1).
+        const int i = rt * 128 + q * 32 + lane;
+        const int odd = lane & 1;
 #pragma unroll 1
-      for (int t = 0; t < 2; ++t) {
-        const uint32_t tcol = tmem_base + lane_base + static_cast<uint32_t>(t * 256);
-        if (STAGE1) {
-          // lanes 0..63 hold gate rows, lanes 64..127 the matching up rows.  Transpose 16 columns through
-          // shared memory (sT[column][lane]); then thread (column j, segment) owns 8 consecutive i of token j.
-          const int j = te >> 3, seg = te & 7;
-          const int ibase = rt * 128 + t * 64 + seg * 8;
-          for (int c0 = 0; c0 < ntok; c0 += kTChunk) {
-            uint32_t v[16];
-            tmem_ld_32x16(tcol + static_cast<uint32_t>(c0), v);
-            tmem_ld_wait();
-            float* tb = sT;
-            asm volatile("bar.sync 2, %0;" ::"n"(kEpilogueWarps * 32) : "memory");  // previous chunk fully read
+        for (int c0 = half * 16; c0 < ntok; c0 += 32) {
+          uint32_t gv[16], uv[16];
+          tmem_ld_32x16(tmem_base + lane_base + static_cast<uint32_t>(c0), gv);
+          tmem_ld_32x16(tmem_base + lane_base + static_cast<uint32_t>(256 + c0), uv);
+          tmem_ld_wait();
 #pragma unroll
-            for (int jj = 0; jj < 16; ++jj) tb[jj * 128 + q * 32 + lane] = __uint_as_float(v[jj]);
-            asm volatile("bar.sync 2, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
-            if (c0 + j < ntok) {
-              const float4 g0 = *reinterpret_cast<const float4*>(tb + j * 128 + seg * 8);
-              const float4 g1 = *reinterpret_cast<const float4*>(tb + j * 128 + seg * 8 + 4);
-              const float4 u0 = *reinterpret_cast<const float4*>(tb + j * 128 + 64 + seg * 8);
-              const float4 u1 = *reinterpret_cast<const float4*>(tb + j * 128 + 64 + seg * 8 + 4);
-              __nv_bfloat162 o[4];
-              o[0] = __floats2bfloat162_rn(silu_mul(g0.x, u0.x), silu_mul(g0.y, u0.y));
-              o[1] = __floats2bfloat162_rn(silu_mul(g0.z, u0.z), silu_mul(g0.w, u0.w));
-              o[2] = __floats2bfloat162_rn(silu_mul(g1.x, u1.x), silu_mul(g1.y, u1.y));
-              o[3] = __floats2bfloat162_rn(silu_mul(g1.z, u1.z), silu_mul(g1.w, u1.w));
-              *reinterpret_cast<uint4*>(a.act + static_cast<size_t>(row0 + c0 + j) * a.I + ibase) = *reinterpret_cast<uint4*>(o);
-            }
+          for (int jj = 0; jj < 16; jj += 2) {
+            const float v0 = silu_mul(__uint_as_float(gv[jj]), __uint_as_float(uv[jj]));          // token c0 + jj
+            const float v1 = silu_mul(__uint_as_float(gv[jj + 1]), __uint_as_float(uv[jj + 1]));  // token c0 + jj + 1
+            const float got = __shfl_xor_sync(0xffffffffu, odd ? v0 : v1, 1);
+            // even lane: token c0 + jj, rows (i, i + 1); odd lane: token c0 + jj + 1, rows (i - 1, i)
+            const __nv_bfloat162 o = odd ? __floats2bfloat162_rn(got, v1) : __floats2bfloat162_rn(v0, got);
+            const int tok = c0 + jj + odd;
+            if (tok < ntok)
+              *reinterpret_cast<__nv_bfloat162*>(a.act + static_cast<size_t>(row0 + tok) * a.I + (i & ~1)) = o;
           }
-        } else {
+        }
+      } else {
+#pragma unroll 1
+        for (int t = 0; t < 2; ++t) {
+          const uint32_t tcol = tmem_base + lane_base + static_cast<uint32_t>(t * 256);
           const int n = rt * kTileRows + t * 128 + q * 32 + lane;
-          for (int c0 = 0; c0 < ntok; c0 += 32) {
+#pragma unroll 1
+          for (int c0 = half * 32; c0 < ntok; c0 += 64) {
             uint32_t v[32];
             tmem_ld_32x32(tcol + static_cast<uint32_t>(c0), v);
             tmem_ld_wait();
