@@ -23,14 +23,29 @@ constexpr size_t kAlign = 256;
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// native block-scaled FP4 variant (decode-sized batches): on average at most 32 rows per expert (8 passes of 4
+// tokens over the weight stream).  Its scratch holds the E2M1 term rows (8 per row) of both projections' inputs:
+// [8S, I/2] + [8S, I/32] scale bytes and [8S, H/2] + [8S, H/32].
+inline bool native_batch_ok(const moe_shape_t& s) {
+  const long long S = static_cast<long long>(s.T) * s.k;
+  return S <= 4096 && S <= 32LL * s.E;
+}
+inline size_t native_scratch_bytes(const moe_shape_t& s) {
+  const size_t S = static_cast<size_t>(s.T) * s.k;
+  return align_up(8 * S * (s.I / 2), kAlign) + align_up(8 * S * (s.I / 32), kAlign) + align_up(8 * S * (s.H / 2), kAlign) +
+         align_up(8 * S * (s.H / 32), kAlign);
+}
+
 inline WsLayout ws_layout(const moe_shape_t& s) {
   WsLayout L;
   const size_t S = static_cast<size_t>(s.T) * s.k;
   size_t off = 0;
   L.route_off = off;  // moe_route is given only (T, E, k): its block must not depend on H or I
   off += align_up((static_cast<size_t>(s.E) + 8) * 4, kAlign);
-  L.act_off = off;  // bf16 act[S,I], or the split E4M3 pair [2S,I] with its scale bytes [2S,I/32]
-  off += align_up(S * s.I * 2, kAlign) + align_up(2 * S * (s.I / 32), kAlign) + kAlign;
+  L.act_off = off;  // bf16 act[S,I], or the scratch of the native variant
+  const size_t act_bytes = align_up(S * s.I * 2, kAlign);
+  const size_t nat_bytes = native_batch_ok(s) ? native_scratch_bytes(s) : 0;
+  off += (act_bytes > nat_bytes ? act_bytes : nat_bytes) + kAlign;
   L.permute_off = off;
   const size_t nblk = (S + kPermuteChunk - 1) / kPermuteChunk;
   off += align_up(nblk * s.E * 4, kAlign);
@@ -61,9 +76,8 @@ int launch_combine(const float* y_perm, const int* inv_perm, const float* w, con
                    __nv_bfloat16* out, cudaStream_t st);
 int launch_validate_scales(const uint8_t* scales, size_t n, int* bad, cudaStream_t st);
 
-// native block-scaled FP4 variant (decode-sized batches); scratch holds the split activations
+// native block-scaled FP4 variant; scratch of native_scratch_bytes
 bool native_shape_ok(const moe_shape_t& s, const void* w13, const void* w2);
-size_t native_scratch_bytes(const moe_shape_t& s);
 int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
                              const uint8_t* w2, const uint8_t* s2, const moe_shape_t& s, void* scratch, float* y_perm,
                              int* status_word, cudaStream_t st);
