@@ -90,8 +90,8 @@ __host__ __device__ inline NatSmem nat_smem(int E, int K) {
   off += 64 * 8;
   m.misc = off;
   off += 64;
-  m.touched = off;
-  off += (static_cast<uint32_t>(E) + 8) * 4;
+  m.touched = off;  // touched experts: id, first row, end row
+  off += (3 * static_cast<uint32_t>(E) + 8) * 4;
   m.total = off;
   return m;
 }
@@ -216,8 +216,10 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   uint64_t* act_ready = acc_empty + 1;           // scale warps -> MMA: activation operand of the current (expert, pass)
   uint64_t* act_free = act_ready + 1;            // MMA done with the activation operand -> scale warps
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + sm.misc);
-  int* touched = reinterpret_cast<int*>(smem + sm.touched);
-  int* s_misc = touched + a.E;
+  int* touched = reinterpret_cast<int*>(smem + sm.touched);  // ids of the experts that have rows
+  int* t_begin = touched + a.E;                              // their first sorted row
+  int* t_end = t_begin + a.E;                                // and the row after their last
+  int* s_misc = t_end + a.E;
 
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int n_steps = K / kKStep;
@@ -226,21 +228,28 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
 
   // ---- setup: touched experts, barriers, tensor memory ----
   if (wid == 2) {
-    // lane l looks at experts l, l + 32, ...: all loads are issued before any is used (one memory round trip)
+    // lane l looks at experts l, l + 32, ...: all loads are issued before any is used (one memory round trip);
+    // the second loop's loads hit L1
+    const int n_it = (a.E + 31) / 32;
     unsigned has_mask = 0u;
 #pragma unroll 8
-    for (int i = 0; i < (a.E + 31) / 32; ++i) {
+    for (int i = 0; i < n_it; ++i) {
       const int e = i * 32 + lane;
       const int lo = (e < a.E) ? __ldg(a.offsets + e) : 0;
       const int hi = (e < a.E) ? __ldg(a.offsets + e + 1) : 0;
       has_mask |= (hi > lo ? 1u : 0u) << i;
     }
     int run = 0;
-    for (int i = 0; i < (a.E + 31) / 32; ++i) {
+    for (int i = 0; i < n_it; ++i) {
       const int has = static_cast<int>((has_mask >> i) & 1u);
       int tot;
       const int ex = warp_excl_scan(has, lane, &tot);
-      if (has) touched[run + ex] = i * 32 + lane;
+      if (has) {
+        const int e = i * 32 + lane;
+        touched[run + ex] = e;
+        t_begin[run + ex] = __ldg(a.offsets + e);
+        t_end[run + ex] = __ldg(a.offsets + e + 1);
+      }
       run += tot;
     }
     if (lane == 0) s_misc[0] = run;
@@ -283,10 +292,10 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       bool waited = false;
       int n_pend = 0, pend_s[kWStages], pend_x[kWStages], pend_y[kWStages];
       for (long long it = item_begin; it < item_end; ++it) {
-        const int e = touched[it / tiles_per_expert];
+        const int ti = static_cast<int>(it / tiles_per_expert), e = touched[ti];
         const int tile = static_cast<int>(it % tiles_per_expert);
-        const int row_begin = a.offsets[e];
-        const int n_pass = (a.offsets[e + 1] - row_begin + tok_pass - 1) / tok_pass;
+        const int row_begin = t_begin[ti];
+        const int n_pass = (t_end[ti] - row_begin + tok_pass - 1) / tok_pass;
         const int wrow_a = STAGE1 ? e * a.R + tile * 128 : e * a.R + tile * kTile;
         const int wrow_b = STAGE1 ? e * a.R + a.I + tile * 128 : wrow_a + 128;
         for (int pass = 0; pass < n_pass; ++pass) {
@@ -335,9 +344,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
       int prev_e = -1;
       const uint32_t d_addr = tmem_base + kColD;
       for (long long it = item_begin; it < item_end; ++it) {
-        const int e = touched[it / tiles_per_expert];
-        const int rows = a.offsets[e + 1] - a.offsets[e];
-        const int n_pass = (rows + tok_pass - 1) / tok_pass;
+        const int ti = static_cast<int>(it / tiles_per_expert), e = touched[ti];
+        const int n_pass = (t_end[ti] - t_begin[ti] + tok_pass - 1) / tok_pass;
         for (int pass = 0; pass < n_pass; ++pass) {
           // The scale factors of the term rows (tensor memory) are shared by consecutive items of an expert whose
           // rows fit one pass; otherwise every (item, pass) has its own.  The scale warps follow the same rule.
@@ -387,8 +395,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     bool first_op = true;
     const int n_blk = K / 32;
     for (long long it = item_begin; it < item_end; ++it) {
-      const int e = touched[it / tiles_per_expert];
-      const int row_begin = a.offsets[e], row_end = a.offsets[e + 1];
+      const int ti = static_cast<int>(it / tiles_per_expert), e = touched[ti];
+      const int row_begin = t_begin[ti], row_end = t_end[ti];
       const int n_pass = (row_end - row_begin + tok_pass - 1) / tok_pass;
       for (int pass = 0; pass < n_pass; ++pass) {
         const bool new_operand = (prev_e != e) || (n_pass > 1);
@@ -475,9 +483,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     const int cb = 16 * (tl & 1) + 8 * ((tl >> 1) & 1) + 4 * (tl >> 2);
     uint32_t acc_ph = 0;
     for (long long it = item_begin; it < item_end; ++it) {
-      const int e = touched[it / tiles_per_expert];
+      const int ti = static_cast<int>(it / tiles_per_expert);
       const int tile = static_cast<int>(it % tiles_per_expert);
-      const int row_begin = a.offsets[e], row_end = a.offsets[e + 1];
+      const int row_begin = t_begin[ti], row_end = t_end[ti];
       const int n_pass = (row_end - row_begin + tok_pass - 1) / tok_pass;
       for (int pass = 0; pass < n_pass; ++pass) {
         const int row0 = row_begin + pass * tok_pass;
@@ -514,24 +522,39 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
         if (lane == 0) mbar_arrive(acc_empty);  // the accumulator is free: the rest overlaps the next item's MMAs
         if (4 * q >= n_tok) continue;
         if (STAGE1) {
+          // SwiGLU and the 8-term split, one (token, block of 32 consecutive i) per group of 8 lanes: in round rd
+          // the four lane groups take the four blocks of the quadrant's token rd (gate in chunk m, up in chunk m + 4),
+          // so that a quadrant with one token finishes in one round
           const int n_blk_i = a.I / 32;
-          float r[4][4];  // 4 blocks of 32 consecutive i: gate in chunk m, up in chunk m + 4
+          const int n_q = min(4, n_tok - 4 * q);
+#pragma unroll 1
+          for (int rd = 0; rd < n_q; ++rd) {
+            float gsel[4], usel[4];
 #pragma unroll
-          for (int m = 0; m < 4; ++m)
+            for (int m = 0; m < 4; ++m)
+#pragma unroll
+              for (int c = 0; c < 4; ++c) {
+                const float tg = __shfl_sync(0xffffffffu, acc[m][c], rd * 8 + tl);
+                const float tu = __shfl_sync(0xffffffffu, acc[m + 4][c], rd * 8 + tl);
+                if (jl == m) {
+                  gsel[c] = tg;
+                  usel[c] = tu;
+                }
+              }
+            float r[1][4];
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-              const float gv = acc[m][c], uv = acc[m + 4][c];
-              const float sv = __fdividef(gv, 1.0f + __expf(-gv)) * uv;
-              r[m][c] = __bfloat162float(__float2bfloat16_rn(sv));  // the intermediate is defined as a bf16 value
+              const float sv = __fdividef(gsel[c], 1.0f + __expf(-gsel[c])) * usel[c];
+              r[0][c] = __bfloat162float(__float2bfloat16_rn(sv));  // the intermediate is defined as a bf16 value
             }
-          split_terms<4>(r, [&](int m, int t, uint32_t bytes, int se) {
-            if (tok_live) {
-              const int i0 = tile * 128 + 32 * m;
-              const size_t row = static_cast<size_t>(p) * kTerms + t;
-              *reinterpret_cast<uint16_t*>(a.aq_out + row * (a.I / 2) + ((i0 + cb) >> 1)) = static_cast<uint16_t>(bytes);
-              if (tl == 0) a.aq_sf_out[row * n_blk_i + (i0 >> 5)] = static_cast<uint8_t>(se + 127);
-            }
-          });
+            const int i0 = tile * 128 + 32 * jl;
+            uint8_t* qrow = a.aq_out + static_cast<size_t>(row0 + 4 * q + rd) * kTerms * (a.I / 2) + ((i0 + cb) >> 1);
+            uint8_t* srow = a.aq_sf_out + static_cast<size_t>(row0 + 4 * q + rd) * kTerms * n_blk_i + (i0 >> 5);
+            split_terms<1>(r, [&](int, int t, uint32_t bytes, int se) {
+              *reinterpret_cast<uint16_t*>(qrow + static_cast<size_t>(t) * (a.I / 2)) = static_cast<uint16_t>(bytes);
+              if (tl == 0) srow[static_cast<size_t>(t) * n_blk_i] = static_cast<uint8_t>(se + 127);
+            });
+          }
         } else {
           if (tok_live) {
             float* dst = a.y + static_cast<size_t>(p) * a.R + tile * kTile + cb;
