@@ -28,8 +28,8 @@ DECODE = ("decode_c1", "decode_c64")
 # dram__bytes_read.sum + dram__bytes_write.sum per moe_expert_ffn call from one ncu capture of the
 # workload (see profiles/); None until captured.
 NCU_TRAFFIC_BYTES = {
-    "decode_c1": 108632320,      # ffn_native_kernel<true> 71.44 + 1.46 MB, <false> 35.73 MB (profiles/ffn_native_decode.md)
-    "decode_c64": 3023868248,    # 2003.5 + 7.2 MB and 1002.1 + 11.0 MB
+    "decode_c1": 108907776,      # ffn_native_kernel<true> 71.52 + 1.60 MB, <false> 35.79 MB (profiles/ffn_native_decode.md)
+    "decode_c64": 3058403336,    # 2033.1 + 10.5 MB and 1003.6 + 11.1 MB
     "prefill_8k": 5611119000,    # ffn_umma_kernel<true> 2.882 + 0.263 GB, <false> 1.431 + 1.034 GB (profiles/ffn_umma_prefill_8k.md)
 }
 

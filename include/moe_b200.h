@@ -105,8 +105,9 @@ int moe_permute(const void* x_bf16, const int32_t* topk_ids, const int32_t* expe
  *   status_word: device int32, may be NULL; see the common rules.
  * Three kernel variants, chosen by the shape alone (moe_last_kernel_name names the one that ran): for
  * decode-sized batches (T*k <= 32*E, H and I multiples of 512) the packed weights feed the block-scaled FP4
- * tensor-core instruction directly and each bf16 activation row is split into two E4M3 rows that add up to it
- * (exact unless an element is more than 2^14 below its 32-block's maximum; then off by < 2^-19 of that maximum);
+ * tensor-core instruction directly and each bf16 activation row is written as a sum of eight E2M1 rows with their
+ * own block scales (exact for elements within 2^-10 of their 32-block's largest magnitude; the others are off by
+ * less than 2^-16 of that magnitude);
  * for prefill-sized batches (T*k >= 1024) weights are expanded to bf16 exactly on chip for a bf16 grouped GEMM;
  * every other supported shape uses a register-expansion streaming kernel.
  * Launch order: the decode-sized kernels use programmatic dependent launch.  They read expert_offsets and the
@@ -154,12 +155,13 @@ int moe_forward_host(const float* logits_host, const void* x_host_bf16, const ui
  * Who needs it: code that runs where cudaMalloc is off limits - a plug-in called inside another
  * framework's stream-ordered or graph-managed section, a real-time loop that must not touch the driver's
  * allocator, a host that hands this library pre-made buffers for inputs and outputs only.  Such a caller
- * still passes every input and output, but not the scratch: the bf16 intermediate act[T*k, I] is kept in a
- * fixed array of moe_expert_ffn_noalloc_max_bytes() = 8 MiB inside the library image (each GPU that loads
- * the library holds those 8 MiB until the process exits).
+ * still passes every input and output, but not the scratch: what the kernels keep between their launches sits
+ * in a fixed array of moe_expert_ffn_noalloc_max_bytes() = 16 MiB inside the library image (each GPU that loads
+ * the library holds those 16 MiB until the process exits).
  *
- *   - Sizes: 2*T*k*I bytes must fit the array, else MOE_ERR_WORKSPACE and nothing is launched
- *     (decode-sized batches: up to 2048 slots at I = 2048).  Other argument rules as moe_expert_ffn.
+ *   - Sizes: the bf16 intermediate (2*T*k*I bytes) - for the decode-sized kernel variant the E2M1 term rows of
+ *     both projections' inputs, 4.25*T*k*(H+I) bytes - must fit the array, else MOE_ERR_WORKSPACE and nothing is
+ *     launched (up to 640 slots at H = 4096, I = 2048).  Other argument rules as moe_expert_ffn.
  *   - The call allocates and frees nothing and calls no allocating library routine.  Its first call on a
  *     device looks up the array's device address (one runtime query, cached per device): make that first
  *     call outside any stream capture.

@@ -1,12 +1,13 @@
-// moe_expert_ffn for callers that cannot allocate device memory: the bf16 intermediate lives in a
-// fixed array inside the library image instead of a caller-provided workspace.
+// moe_expert_ffn for callers that cannot allocate device memory: the intermediate (and, for decode-sized
+// batches, the E2M1 term rows of the activations) lives in a fixed array inside the library image instead of a
+// caller-provided workspace.
 #include "moe_common.cuh"
 
 namespace moe {
 
 namespace {
 
-constexpr size_t kStaticScratchBytes = 8u << 20;  // 8 MiB: T*k*I <= 4,194,304 intermediate elements
+constexpr size_t kStaticScratchBytes = 16u << 20;  // 16 MiB
 constexpr int kMaxDevices = 64;
 
 // Lives in every GPU context that loads the library, until the process exits.
@@ -50,9 +51,11 @@ int moe_expert_ffn_noalloc(const void* x_perm_bf16, const int32_t* expert_offset
   if (!aligned16(x_perm_bf16) || !aligned16(expert_offsets) || !aligned16(w13) || !aligned16(w13_scale) || !aligned16(w2) ||
       !aligned16(w2_scale) || !aligned16(y_perm))
     return MOE_ERR_INVALID_ARG;
-  // the intermediate act[T*k, I] bf16 must fit the fixed array
-  // (bf16 act[T*k, I], or the same rows split into two E4M3 rows plus scale bytes: a little over 2 bytes per element)
-  const unsigned long long need = native_scratch_bytes(s) + kAlign;
+  // what the chosen kernel keeps between its launches must fit the fixed array: the bf16 intermediate act[T*k, I],
+  // or for the native variant the E2M1 term rows and scale bytes of both projections' inputs (4.25 (H + I) bytes per slot)
+  const unsigned long long S = static_cast<unsigned long long>(s.T) * s.k;
+  const unsigned long long need =
+      (native_shape_ok(s, w13, w2) ? static_cast<unsigned long long>(native_scratch_bytes(s)) : S * s.I * 2ULL) + kAlign;
   if (need > kStaticScratchBytes) return MOE_ERR_WORKSPACE;
   void* scratch = nullptr;
   const int rc = static_scratch(&scratch);  // first call on a device looks the address up

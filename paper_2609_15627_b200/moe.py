@@ -128,7 +128,7 @@ def moe_expert_ffn_noalloc_max_bytes():
 
 def moe_expert_ffn_noalloc(x_perm, expert_offsets, w13, w13_scale, w2, w2_scale, sh, y_perm, status_word, stream=None):
     """moe_expert_ffn for callers that cannot allocate: no workspace argument, the intermediate lives in a
-    fixed 8 MiB array inside the library (see include/moe_b200.h for the limits and the sharing rules)."""
+    fixed 16 MiB array inside the library (see include/moe_b200.h for the limits and the sharing rules)."""
     _check(lib().moe_expert_ffn_noalloc(_ptr(x_perm), _ptr(expert_offsets), _ptr(w13), _ptr(w13_scale), _ptr(w2),
                                         _ptr(w2_scale), C.byref(sh), _ptr(y_perm), _ptr(status_word), _stream(stream)),
            "moe_expert_ffn_noalloc")

@@ -449,9 +449,11 @@ def test_kernel_choice_is_a_function_of_the_shape():
 # ---- the native block-scaled FP4 expert FFN, reached when T*k <= 32*E (decode-sized) and H, I are multiples of 512 ----
 
 @pytest.mark.parametrize("T,H,I,E,k,hot,seed", [
-    (16, 512, 512, 8, 2, False, 0),      # a few rows per expert
-    (1, 512, 512, 16, 4, False, 1),      # one token: every expert has one row
-    (64, 1024, 512, 8, 2, False, 2),     # ~16 rows per expert: two passes of 8 tokens
+    (16, 512, 512, 8, 2, False, 0),      # a few rows per expert, passes of 16 tokens
+    (1, 512, 512, 16, 4, False, 1),      # one token: every expert has one row; passes of 4 tokens (4 slots in all)
+    (4, 512, 512, 8, 2, False, 4),       # 8 slots: passes of 8 tokens
+    (64, 1024, 512, 8, 2, False, 2),     # ~16 rows per expert: some experts need two passes of 16 tokens
+    (64, 512, 512, 4, 2, False, 5),      # ~32 rows per expert: two or three passes each
     (40, 512, 1024, 8, 1, True, 3),      # one hot expert with most rows, several empty experts
 ])
 def test_ffn_native_fp4_path_against_oracle(T, H, I, E, k, hot, seed):
@@ -464,7 +466,7 @@ def test_ffn_native_fp4_path_against_oracle(T, H, I, E, k, hot, seed):
         logits[:, 2] += 8.0
         logits[:, [5, 6]] -= 50.0
     x = inputs.make_x(T, H, seed=seed)
-    # activations with a wide dynamic range inside a 32-block exercise the hi/lo split
+    # activations with a wide dynamic range inside a 32-block exercise the split into E2M1 terms
     xf = inputs.bf16_bits_to_f32(x)
     xf[:, ::7] *= 2.0 ** -9
     xf[:, 5::11] *= 64.0

@@ -35,7 +35,7 @@ def _case(T, H, I, E, k, seed):
 
 def test_noalloc_matches_regular_entry_point_on_two_calls_in_a_row():
     assert torch.cuda.is_available()
-    assert moe.moe_expert_ffn_noalloc_max_bytes() == 8 << 20
+    assert moe.moe_expert_ffn_noalloc_max_bytes() == 16 << 20
     # two different shapes back to back: the second call finds the first call's data in the array
     for (T, H, I, E, k, seed) in [(64, 512, 256, 8, 2, 0), (16, 256, 128, 8, 2, 1), (64, 512, 256, 8, 2, 2)]:
         w, x_perm, off, sh = _case(T, H, I, E, k, seed)
@@ -58,6 +58,6 @@ def test_noalloc_matches_regular_entry_point_on_two_calls_in_a_row():
 def test_noalloc_rejects_sizes_beyond_the_fixed_array():
     L = moe.lib()
     fake = C.c_void_p(0x1000)  # never dereferenced: the size check comes first
-    big = moe.shape(4096, 4096, 2048, 256, 8)   # 2*T*k*I = 128 MiB > 8 MiB
+    big = moe.shape(4096, 4096, 2048, 256, 8)   # 2*T*k*I = 128 MiB > 16 MiB
     assert L.moe_expert_ffn_noalloc(fake, fake, fake, fake, fake, fake, C.byref(big), fake, None, None) == 3
     assert L.moe_expert_ffn_noalloc(fake, fake, fake, fake, fake, fake, None, fake, None, None) == 1
