@@ -127,8 +127,9 @@ def max_over_ranks(value, world):
     return float(t.item())
 
 
-def oracle_sample(wl, inputs, n_tokens, seed0=1000):
-    """Time the CPU oracle, as it stands, on n_tokens tokens of the workload (per-token definition)."""
+def oracle_sample(wl, inputs, n_tokens, seed0=1000, weights=None):
+    """Time the CPU oracle, as it stands, on n_tokens tokens of the workload (per-token definition).
+    `weights`: the full host arrays if the caller has them; else the touched experts are generated here."""
     from oracle import moe_oracle as O
     logits = inputs.make_logits(max(wl.T, 1), wl.E, seed0, wl.skew)
     x = inputs.make_x(max(wl.T, 1), wl.H, seed0)
@@ -137,8 +138,11 @@ def oracle_sample(wl, inputs, n_tokens, seed0=1000):
         x = np.concatenate([inputs.make_x(wl.T, wl.H, seed0 + i) for i in range(n_tokens)])[:n_tokens]
     tokens = np.arange(min(n_tokens, logits.shape[0]), dtype=np.int32)
     ids, _, _ = O.route(logits, wl.k)
-    need = sorted(set(ids[tokens].ravel().tolist()))
-    w13, s13, w2, s2 = inputs.make_expert_weights(wl.H, wl.I, wl.E, seed=0, experts=need)
+    if weights is not None:
+        w13, s13, w2, s2 = weights
+    else:
+        need = sorted(set(ids[tokens].ravel().tolist()))
+        w13, s13, w2, s2 = inputs.make_expert_weights(wl.H, wl.I, wl.E, seed=0, experts=need)
     t0 = time.perf_counter()
     O.forward_tokens(logits, x, w13, s13, w2, s2, wl.k, tokens)
     dt = time.perf_counter() - t0
@@ -220,7 +224,8 @@ def main():
             return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
         return torch.from_numpy(a).cuda()
 
-    weights = tuple(dev(a) for a in inputs.make_expert_weights(wl.H, wl.I, wl.E, seed=0))
+    weights_host = inputs.make_expert_weights(wl.H, wl.I, wl.E, seed=0)
+    weights = tuple(dev(a) for a in weights_host)
     n_cycle = 32 if decode else 2
     batches_host = [(inputs.make_logits(wl.T, wl.E, 7000 + rank * 100 + i, wl.skew), inputs.make_x(wl.T, wl.H, 7000 + rank * 100 + i))
                     for i in range(n_cycle)]
@@ -356,8 +361,9 @@ def main():
     # ---- the oracle on the host cores (rank 0, N = 1 only) ----------------------------------------------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        n_tok = {"tiny": 64, "decode_c1": 32, "decode_c64": 32}.get(wl.name, 32)
-        v, dt, n, cores = oracle_sample(wl, inputs, n_tok)
+        # about 10-20 s of host work at the production shape (the oracle does roughly 50 tokens/s on 16 cores)
+        n_tok = {"tiny": 4096}.get(wl.name, 640)
+        v, dt, n, cores = oracle_sample(wl, inputs, n_tok, weights=weights_host)
         cpu = {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle",
                "sample": "%d tokens with the %s shape and routing distribution, per-token definition, %.1f s" % (n, wl.name, dt)}
 

@@ -120,6 +120,8 @@ MOE_DEVINL uint32_t idesc_mxf4(uint32_t half) {
   return (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24) | ((2u * half) << 29) | ((2u * half) << 4);
 }
 
+MOE_DEVINL void prefetch_tmap(const void* tmap) { asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory"); }
+
 MOE_DEVINL float pow2f(int e) { return __uint_as_float(static_cast<uint32_t>(e + 127) << 23); }  // e in [-126, 127]
 // Block exponent of a term: the smallest s with amax <= 6 * 2^s (amax > 0), kept inside the UE8M0 range
 MOE_DEVINL int term_exp(float amax) {
@@ -227,6 +229,11 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   const int tok_pass = a.tok_pass;
 
   // ---- setup: touched experts, barriers, tensor memory ----
+  if (tid == 32 * 6) {  // an idle warp fetches the tensor maps while the others set up
+    prefetch_tmap(&tmap_w);
+    prefetch_tmap(&tmap_sc);
+    prefetch_tmap(&tmap_a);
+  }
   if (wid == 2) {
     // lane l looks at experts l, l + 32, ...: all loads are issued before any is used (one memory round trip);
     // the second loop's loads hit L1
