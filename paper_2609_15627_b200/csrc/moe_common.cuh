@@ -25,7 +25,7 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // native block-scaled FP4 variant (decode-sized batches): on average at most 32 rows per expert (8 passes of 4
 // tokens over the weight stream).  Its scratch holds the E2M1 term rows (8 per row) of both projections' inputs:
-// [8S, I/2] + [8S, I/32] scale bytes and [8S, H/2] + [8S, H/32].
+// [8S, I/2] + [8S, I/32] scale bytes and [8S, H/2] + [8S, H/32]; and one completion counter per expert.
 inline bool native_batch_ok(const moe_shape_t& s) {
   const long long S = static_cast<long long>(s.T) * s.k;
   return S <= 4096 && S <= 32LL * s.E;
@@ -33,7 +33,7 @@ inline bool native_batch_ok(const moe_shape_t& s) {
 inline size_t native_scratch_bytes(const moe_shape_t& s) {
   const size_t S = static_cast<size_t>(s.T) * s.k;
   return align_up(8 * S * (s.I / 2), kAlign) + align_up(8 * S * (s.I / 32), kAlign) + align_up(8 * S * (s.H / 2), kAlign) +
-         align_up(8 * S * (s.H / 32), kAlign);
+         align_up(8 * S * (s.H / 32), kAlign) + align_up(static_cast<size_t>(s.E) * 4, kAlign);
 }
 
 inline WsLayout ws_layout(const moe_shape_t& s) {

@@ -19,10 +19,15 @@
 // Both operands ride the same shared-memory ring: a stage is one K step (256 elements) of the weight tile plus
 // the same K step of the pass's term rows, each fetched by TMA with the 128-byte swizzle the MMA reads.
 //
-// Launches per call: native_split_kernel (token rows -> E2M1 terms, once per row), then the gate/up kernel and
-// the down kernel.  Work item = (touched expert, tile of 256 weight rows) over the full K (gate/up: 128 gate +
-// 128 up rows, so gate and up of the same i are two columns of the same accumulator lane).
-// Warp roles (one persistent CTA per SM):
+// Launches per call: native_split_kernel (token rows -> E2M1 terms, once per row; clears the per-expert completion
+// counters), then ffn_native_kernel, in which one persistent CTA per SM runs both projections back to back:
+// phase 0 = gate/up + SwiGLU (work item = touched expert x 128 gate rows + the 128 matching up rows, so gate and up of
+// one i are two columns of the same accumulator lane), phase 1 = down (item = touched expert x 256 rows).  The weight
+// stream runs on across the phase change; a down item loads its term rows once the gate/up items of its expert - its
+// own and other CTAs' - have published theirs (one counter per expert, release/acquire through L2, bounded wait).
+// All CTAs of the grid are resident (grid = number of SMs, one CTA each) and no gate/up item ever waits for another
+// CTA, so the waits cannot form a cycle.
+// Warp roles:
 //   warp 0      producer: TMA loads of the weight tile, of the term rows and of the weight scale bytes
 //   warp 1      allocates tensor memory, issues the MMAs, commits to mbarriers
 //   warps 2..5  move weight scale bytes into tensor memory (tcgen05.st), and at a change of (expert, pass) the
@@ -61,17 +66,34 @@ constexpr uint32_t kNatTmemCols = 512;
 constexpr uint32_t kColD = 0, kColSfAct = 256, kColSfW = 384;
 
 struct NatArgs {
-  const __nv_bfloat16* x;    // split kernel input: sorted token rows [S, H]
-  const uint8_t* aq;         // this projection's input terms [S * 8, K/2] (row p * 8 + t), packed E2M1
-  const uint8_t* aq_sf;      //   and their scale bytes [S * 8, K/32]
-  uint8_t* aq_out;           // gate/up output: terms of the bf16 intermediate [S * 8, I/2]
-  uint8_t* aq_sf_out;        //   [S * 8, I/32]
+  const uint8_t* sf1;        // scale bytes of the token rows' terms [S * 8, H/32] (terms: row p * 8 + t, packed E2M1)
+  uint8_t* aq2;              // terms of the bf16 intermediate [S * 8, I/2]: written by phase 0, read by phase 1
+  uint8_t* sf2;              //   and their scale bytes [S * 8, I/32]
+  int* done;                 // [E] epilogue warps that have published a gate/up item of the expert
   const int* offsets;
-  float* y;                  // down output [S, R]
+  float* y;                  // output [S, H]
   int* status;
-  int E, K, R, I, S;
+  int E, H, I, S;
   int tok_pass;              // tokens per pass: 4, 8 or 16 (the row count of the term-row TMA box / 8)
 };
+
+// One projection as the kernel sees it
+struct Phase {
+  int K, R, n_steps, tiles;  // reduction length, weight rows per expert, K steps, items per expert
+  long long begin, end;      // this CTA's items
+};
+MOE_DEVINL Phase phase_of(int ph, const NatArgs& a, int n_touched) {
+  Phase p;
+  p.K = ph == 0 ? a.H : a.I;
+  p.R = ph == 0 ? 2 * a.I : a.H;
+  p.n_steps = p.K / kKStep;
+  p.tiles = p.R / kTile;
+  const long long total = static_cast<long long>(n_touched) * p.tiles;
+  const long long per_cta = (total + gridDim.x - 1) / gridDim.x;
+  p.begin = min(static_cast<long long>(blockIdx.x) * per_cta, total);
+  p.end = min(p.begin + per_cta, total);
+  return p;
+}
 
 struct NatSmem {
   uint32_t act, w, sc, sfa, bars, misc, touched, total;
@@ -120,6 +142,25 @@ MOE_DEVINL uint32_t idesc_mxf4(uint32_t half) {
   return (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24) | ((2u * half) << 29) | ((2u * half) << 4);
 }
 
+// Bounded wait until *p >= need (acquire at GPU scope); same give-up rules as mbar_wait
+MOE_DEVINL void counter_wait_ge(const int* p, int need, int* status) {
+  const long long t0 = clock64();
+  int spins = 0;
+  while (true) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    if (v >= need) return;
+    const long long waited = clock64() - t0;
+    if (waited > kWaitLimitCycles) {
+      if (status != nullptr) atomicExch(status, static_cast<int>(MOE_ERR_TIMEOUT));
+      return;
+    }
+    if (((++spins) & 63) == 0 && waited > 2000000 && status != nullptr && *reinterpret_cast<volatile int*>(status) != 0) return;
+    __nanosleep(64);
+  }
+}
+// orders this thread's generic-proxy accesses with its asynchronous-proxy (TMA) accesses, global memory included
+MOE_DEVINL void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 MOE_DEVINL void prefetch_tmap(const void* tmap) { asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory"); }
 
 MOE_DEVINL float pow2f(int e) { return __uint_as_float(static_cast<uint32_t>(e + 127) << 23); }  // e in [-126, 127]
@@ -174,11 +215,13 @@ MOE_DEVINL void split_terms(float (&r)[NB][4], Store store) {
 
 // ---- split kernel: bf16 token rows -> 8 E2M1 term rows with their scale bytes; 8 threads per 32-element block ----
 __global__ void __launch_bounds__(256) native_split_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict__ aq,
-                                                           uint8_t* __restrict__ aq_sf, int S, int H) {
-  pdl_launch_dependents();  // the gate/up grid may set up and start its weight stream; it waits before it reads aq
-  pdl_wait();               // the sorted token rows of moe_permute are complete
+                                                           uint8_t* __restrict__ aq_sf, int* __restrict__ done, int S, int H,
+                                                           int E) {
+  pdl_launch_dependents();  // the FFN grid may set up and start its weight stream; it waits before it reads aq or done
+  pdl_wait();               // the sorted token rows of moe_permute are complete, and every earlier kernel on the stream
   const int n_blk = H / 32;
   const long long gt = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (gt < E) done[gt] = 0;
   const long long task = gt >> 3;  // (row, block); the grid is padded to whole warps, so whole tasks are in or out
   const int sub = static_cast<int>(gt & 7);
   const bool live = task < static_cast<long long>(S) * n_blk;
@@ -195,14 +238,13 @@ __global__ void __launch_bounds__(256) native_split_kernel(const __nv_bfloat16* 
   });
 }
 
-template <bool STAGE1>
 __global__ void __launch_bounds__(kNatThreads, 1)
-ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_sc,
-                  const __grid_constant__ CUtensorMap tmap_a, const NatArgs a) {
+ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_constant__ CUtensorMap tmap_s13,
+                  const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_w2,
+                  const __grid_constant__ CUtensorMap tmap_s2, const __grid_constant__ CUtensorMap tmap_a2, const NatArgs a) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
-  const int K = a.K;
-  const NatSmem sm = nat_smem(a.E, K);
+  const NatSmem sm = nat_smem(a.E, a.H > a.I ? a.H : a.I);
   unsigned char* sW = smem + sm.w;      // ring of stages: [256 weight rows][128 bytes] then [128 term rows][128 bytes]
   unsigned char* sSc = smem + sm.sc;    // ring of [256 rows][16 bytes]
   unsigned char* sSfa = smem + sm.sfa;  // [128 term rows][K/32] scale bytes of the current pass
@@ -215,8 +257,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   uint64_t* sf_free = sf_full + kSfGroups;       // [kSfGroups] MMA done -> scale warps
   uint64_t* acc_full = sf_free + kSfGroups;      // MMA -> epilogue
   uint64_t* acc_empty = acc_full + 1;            // epilogue -> MMA
-  uint64_t* act_ready = acc_empty + 1;           // scale warps -> MMA: activation operand of the current (expert, pass)
-  uint64_t* act_free = act_ready + 1;            // MMA done with the activation operand -> scale warps
+  uint64_t* act_ready = acc_empty + 1;           // scale warps -> MMA: term-row scale factors of the current (expert, pass)
+  uint64_t* act_free = act_ready + 1;            // MMA done with them -> scale warps
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + sm.misc);
   int* touched = reinterpret_cast<int*>(smem + sm.touched);  // ids of the experts that have rows
   int* t_begin = touched + a.E;                              // their first sorted row
@@ -224,19 +266,21 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   int* s_misc = t_end + a.E;
 
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  const int n_steps = K / kKStep;
-  const int tiles_per_expert = a.R / kTile;
   const int tok_pass = a.tok_pass;
+  const int need_done = 4 * (2 * a.I / kTile);  // four epilogue warps publish each gate/up item of an expert
 
   // ---- setup: touched experts, barriers, tensor memory ----
   if (tid == 32 * 6) {  // an idle warp fetches the tensor maps while the others set up
-    prefetch_tmap(&tmap_w);
-    prefetch_tmap(&tmap_sc);
-    prefetch_tmap(&tmap_a);
+    prefetch_tmap(&tmap_w13);
+    prefetch_tmap(&tmap_s13);
+    prefetch_tmap(&tmap_a1);
+    prefetch_tmap(&tmap_w2);
+    prefetch_tmap(&tmap_s2);
+    prefetch_tmap(&tmap_a2);
   }
   if (wid == 2) {
     // lane l looks at experts l, l + 32, ...: all loads are issued before any is used (one memory round trip);
-    // the second loop's loads hit L1
+    // the second loop's loads hit L1.  expert_offsets was complete before the permute kernel let this chain start.
     const int n_it = (a.E + 31) / 32;
     unsigned has_mask = 0u;
 #pragma unroll 8
@@ -276,206 +320,234 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_holder;
-  // Programmatic dependent launch: the next grid (down projection after gate/up, combine after down) may start its
-  // set-up - and the down projection its weight stream - while this grid is still running; it waits
-  // (griddepcontrol.wait) before it reads what this grid writes.  This grid in turn reads nothing of its own
-  // predecessor before its scale warps have waited (below), apart from expert_offsets, which the router finished
-  // before the permute kernel let this chain start.
+  // Programmatic dependent launch: the next grid on the stream (moe_combine) may start its set-up now; it waits
+  // (griddepcontrol.wait) for this grid to complete before it reads the output.  This grid in turn reads nothing
+  // of the split kernel before it has waited itself, apart from expert_offsets (see above).
   pdl_launch_dependents();
   const int n_touched = s_misc[0];
-  const long long total_items = static_cast<long long>(n_touched) * tiles_per_expert;
-  const long long per_cta = (total_items + gridDim.x - 1) / gridDim.x;
-  const long long item_begin = static_cast<long long>(blockIdx.x) * per_cta;
-  const long long item_end = min(item_begin + per_cta, total_items);
-  // Every role walks the same sequence: for each item, for each pass of up to tok_pass tokens, all K steps.
+  // Every role walks the same sequence: both phases; in each, this CTA's items; per item, passes of up to tok_pass
+  // tokens; per pass, all K steps.
 
   if (wid == 0) {
     // =========================== producer ===========================
     if (lane == 0) {
       int s = 0, cs = 0;
       uint32_t ph = 0, cph = 0;
-      // The weights do not depend on the kernel before this one, the term rows do: the weight loads of the first
-      // kWStages steps go out at once, their term-row loads follow when that kernel is complete.
-      bool waited = false;
+      // The weights depend on nothing, the term rows do: on the split kernel (phase 0) or on the gate/up items of
+      // their expert (phase 1).  While a dependency is open, the weight loads go out and the term-row loads of up to
+      // kWStages steps are held back; they follow once the dependency is met.
+      bool pdl_done = false, dep_ok = false;
+      int dep_phase = 0, dep_e = -1;
       int n_pend = 0, pend_s[kWStages], pend_x[kWStages], pend_y[kWStages];
-      for (long long it = item_begin; it < item_end; ++it) {
-        const int ti = static_cast<int>(it / tiles_per_expert), e = touched[ti];
-        const int tile = static_cast<int>(it % tiles_per_expert);
-        const int row_begin = t_begin[ti];
-        const int n_pass = (t_end[ti] - row_begin + tok_pass - 1) / tok_pass;
-        const int wrow_a = STAGE1 ? e * a.R + tile * 128 : e * a.R + tile * kTile;
-        const int wrow_b = STAGE1 ? e * a.R + a.I + tile * 128 : wrow_a + 128;
-        for (int pass = 0; pass < n_pass; ++pass) {
-          for (int ks = 0; ks < n_steps; ++ks) {
-            if ((ks & 1) == 0) {  // 16 scale bytes per weight row cover two K steps
-              mbar_wait(&empty_sc[cs], cph ^ 1u, a.status);
-              mbar_expect_tx(&full_sc[cs], kScStage);
-              tma_load_2d(sSc + cs * kScStage, &tmap_sc, ks * 8, wrow_a, &full_sc[cs]);
-              tma_load_2d(sSc + cs * kScStage + 128 * 16, &tmap_sc, ks * 8, wrow_b, &full_sc[cs]);
-              if (++cs == kScStages) { cs = 0; cph ^= 1u; }
-            }
-            mbar_wait(&empty_w[s], ph ^ 1u, a.status);
-            mbar_expect_tx(&full_w[s], static_cast<uint32_t>(kWStage + tok_pass * kTerms * 128));
-            tma_load_2d(sW + s * kStage, &tmap_w, ks * 128, wrow_a, &full_w[s]);
-            tma_load_2d(sW + s * kStage + 128 * 128, &tmap_w, ks * 128, wrow_b, &full_w[s]);
-            // the pass's term rows (8 per token, consecutive); rows past the end of the tensor arrive as zeros
-            const int arow = (row_begin + pass * tok_pass) * kTerms;
-            if (waited) {
-              tma_load_2d(sW + s * kStage + kWStage, &tmap_a, ks * 128, arow, &full_w[s]);
-            } else {
-              pend_s[n_pend] = s;
-              pend_x[n_pend] = ks * 128;
-              pend_y[n_pend] = arow;
-              if (++n_pend == kWStages) {
-                pdl_wait();
-                for (int i = 0; i < n_pend; ++i)
-                  tma_load_2d(sW + pend_s[i] * kStage + kWStage, &tmap_a, pend_x[i], pend_y[i], &full_w[pend_s[i]]);
-                waited = true;
+      auto meet = [&]() {  // wait for the open dependency and send the held-back loads
+        if (!pdl_done) {
+          pdl_wait();  // the split kernel is complete: term rows of the tokens, cleared counters
+          pdl_done = true;
+        }
+        if (dep_phase == 1) {
+          counter_wait_ge(a.done + dep_e, need_done, a.status);
+          fence_proxy_async_all();  // the rows were written through the generic proxy, TMA reads through the async one
+        }
+        const CUtensorMap* ma = dep_phase == 0 ? &tmap_a1 : &tmap_a2;
+        for (int i = 0; i < n_pend; ++i)
+          tma_load_2d(sW + pend_s[i] * kStage + kWStage, ma, pend_x[i], pend_y[i], &full_w[pend_s[i]]);
+        n_pend = 0;
+        dep_ok = true;
+      };
+      for (int phase = 0; phase < 2; ++phase) {
+        const Phase P = phase_of(phase, a, n_touched);
+        const CUtensorMap* mw = phase == 0 ? &tmap_w13 : &tmap_w2;
+        const CUtensorMap* msc = phase == 0 ? &tmap_s13 : &tmap_s2;
+        const CUtensorMap* ma = phase == 0 ? &tmap_a1 : &tmap_a2;
+        for (long long it = P.begin; it < P.end; ++it) {
+          const int ti = static_cast<int>(it / P.tiles), e = touched[ti];
+          const int tile = static_cast<int>(it % P.tiles);
+          const int row_begin = t_begin[ti];
+          const int n_pass = (t_end[ti] - row_begin + tok_pass - 1) / tok_pass;
+          const int wrow_a = phase == 0 ? e * P.R + tile * 128 : e * P.R + tile * kTile;
+          const int wrow_b = phase == 0 ? e * P.R + a.I + tile * 128 : wrow_a + 128;
+          if (phase == 1 && (dep_phase != 1 || dep_e != e)) {  // a new dependency: settle the old one first
+            if (n_pend > 0) meet();
+            dep_phase = 1;
+            dep_e = e;
+            dep_ok = false;
+          }
+          for (int pass = 0; pass < n_pass; ++pass) {
+            for (int ks = 0; ks < P.n_steps; ++ks) {
+              if ((ks & 1) == 0) {  // 16 scale bytes per weight row cover two K steps
+                mbar_wait(&empty_sc[cs], cph ^ 1u, a.status);
+                mbar_expect_tx(&full_sc[cs], kScStage);
+                tma_load_2d(sSc + cs * kScStage, msc, ks * 8, wrow_a, &full_sc[cs]);
+                tma_load_2d(sSc + cs * kScStage + 128 * 16, msc, ks * 8, wrow_b, &full_sc[cs]);
+                if (++cs == kScStages) { cs = 0; cph ^= 1u; }
               }
+              mbar_wait(&empty_w[s], ph ^ 1u, a.status);
+              mbar_expect_tx(&full_w[s], static_cast<uint32_t>(kWStage + tok_pass * kTerms * 128));
+              tma_load_2d(sW + s * kStage, mw, ks * 128, wrow_a, &full_w[s]);
+              tma_load_2d(sW + s * kStage + 128 * 128, mw, ks * 128, wrow_b, &full_w[s]);
+              // the pass's term rows (8 per token, consecutive); rows past the end of the tensor arrive as zeros
+              const int arow = (row_begin + pass * tok_pass) * kTerms;
+              if (dep_ok) {
+                tma_load_2d(sW + s * kStage + kWStage, ma, ks * 128, arow, &full_w[s]);
+              } else {
+                pend_s[n_pend] = s;
+                pend_x[n_pend] = ks * 128;
+                pend_y[n_pend] = arow;
+                if (++n_pend == kWStages) meet();
+              }
+              if (++s == kWStages) { s = 0; ph ^= 1u; }
             }
-            if (++s == kWStages) { s = 0; ph ^= 1u; }
           }
         }
       }
-      if (!waited && n_pend > 0) {
-        pdl_wait();
-        for (int i = 0; i < n_pend; ++i)
-          tma_load_2d(sW + pend_s[i] * kStage + kWStage, &tmap_a, pend_x[i], pend_y[i], &full_w[pend_s[i]]);
-      }
+      if (n_pend > 0) meet();
     }
   } else if (wid == 1) {
     // =========================== MMA issuer ===========================
     if (lane == 0) {
       int s = 0, slot = 0;
       uint32_t ph = 0, sph = 0, aph = 0, acc_ph = 0;
-      int prev_e = -1;
       const uint32_t d_addr = tmem_base + kColD;
-      for (long long it = item_begin; it < item_end; ++it) {
-        const int ti = static_cast<int>(it / tiles_per_expert), e = touched[ti];
-        const int n_pass = (t_end[ti] - t_begin[ti] + tok_pass - 1) / tok_pass;
-        for (int pass = 0; pass < n_pass; ++pass) {
-          // The scale factors of the term rows (tensor memory) are shared by consecutive items of an expert whose
-          // rows fit one pass; otherwise every (item, pass) has its own.  The scale warps follow the same rule.
-          const bool new_operand = (prev_e != e) || (n_pass > 1);
-          prev_e = e;
-          if (new_operand) {
-            mbar_wait(act_ready, aph, a.status);
-            aph ^= 1u;
-          }
-          mbar_wait(acc_empty, acc_ph ^ 1u, a.status);
-          tc_fence_after_sync();
-          for (int ks = 0; ks < n_steps; ++ks) {
-            if ((ks & 1) == 0) mbar_wait(&sf_full[slot], sph, a.status);  // weight scale factors of 2 K steps at a time
-            mbar_wait(&full_w[s], ph, a.status);
+      for (int phase = 0; phase < 2; ++phase) {
+        const Phase P = phase_of(phase, a, n_touched);
+        int prev_ti = -1;
+        for (long long it = P.begin; it < P.end; ++it) {
+          const int ti = static_cast<int>(it / P.tiles);
+          const int n_pass = (t_end[ti] - t_begin[ti] + tok_pass - 1) / tok_pass;
+          for (int pass = 0; pass < n_pass; ++pass) {
+            // The scale factors of the term rows (tensor memory) are shared by consecutive items of an expert whose
+            // rows fit one pass; otherwise every (item, pass) has its own.  The scale warps follow the same rule.
+            const bool new_operand = (prev_ti != ti) || (n_pass > 1);
+            prev_ti = ti;
+            if (new_operand) {
+              mbar_wait(act_ready, aph, a.status);
+              aph ^= 1u;
+            }
+            mbar_wait(acc_empty, acc_ph ^ 1u, a.status);
             tc_fence_after_sync();
-            const uint32_t w_addr = smem_u32(sW + s * kStage);
+            for (int ks = 0; ks < P.n_steps; ++ks) {
+              if ((ks & 1) == 0) mbar_wait(&sf_full[slot], sph, a.status);  // weight scale factors of 2 K steps at a time
+              mbar_wait(&full_w[s], ph, a.status);
+              tc_fence_after_sync();
+              const uint32_t w_addr = smem_u32(sW + s * kStage);
 #pragma unroll
-            for (uint32_t j = 0; j < 4; ++j) {  // K = 64 each; scale word (ks & 1) * 2 + j / 2 of the group, half j & 1
-              const uint32_t sf_act = tmem_base + kColSfAct + static_cast<uint32_t>(ks * 8) + (j >> 1) * 4;
-              const uint32_t sf_w = tmem_base + kColSfW + static_cast<uint32_t>(slot * 32 + ((ks & 1) * 2 + (j >> 1)) * 8);
-              umma_mxf4(d_addr, umma_desc_k_sw128(w_addr + kWStage + j * 32), umma_desc_k_sw128(w_addr + j * 32),
-                        idesc_mxf4(j & 1u), sf_act, sf_w, (ks | static_cast<int>(j)) != 0 ? 1u : 0u);
+              for (uint32_t j = 0; j < 4; ++j) {  // K = 64 each; scale word (ks & 1) * 2 + j / 2 of the group, half j & 1
+                const uint32_t sf_act = tmem_base + kColSfAct + static_cast<uint32_t>(ks * 8) + (j >> 1) * 4;
+                const uint32_t sf_w = tmem_base + kColSfW + static_cast<uint32_t>(slot * 32 + ((ks & 1) * 2 + (j >> 1)) * 8);
+                umma_mxf4(d_addr, umma_desc_k_sw128(w_addr + kWStage + j * 32), umma_desc_k_sw128(w_addr + j * 32),
+                          idesc_mxf4(j & 1u), sf_act, sf_w, (ks | static_cast<int>(j)) != 0 ? 1u : 0u);
+              }
+              umma_commit(&empty_w[s]);
+              if (++s == kWStages) { s = 0; ph ^= 1u; }
+              if ((ks & 1) == 1) {
+                umma_commit(&sf_free[slot]);
+                if (++slot == kSfGroups) { slot = 0; sph ^= 1u; }
+              }
             }
-            umma_commit(&empty_w[s]);
-            if (++s == kWStages) { s = 0; ph ^= 1u; }
-            if ((ks & 1) == 1) {
-              umma_commit(&sf_free[slot]);
-              if (++slot == kSfGroups) { slot = 0; sph ^= 1u; }
-            }
+            umma_commit(acc_full);
+            acc_ph ^= 1u;
+            // last use of these scale factors?  (always at the end of a phase)
+            bool next_new = true;
+            if (pass + 1 >= n_pass && it + 1 < P.end) next_new = (static_cast<int>((it + 1) / P.tiles) != ti) || (n_pass > 1);
+            if (next_new) umma_commit(act_free);
           }
-          umma_commit(acc_full);
-          acc_ph ^= 1u;
-          bool next_new = true;  // is this the last use of the activation operand?
-          if (pass + 1 >= n_pass && it + 1 < item_end) next_new = (touched[(it + 1) / tiles_per_expert] != e) || (n_pass > 1);
-          if (next_new) umma_commit(act_free);
         }
       }
     }
   } else if (wid >= 2 && wid < 6) {
-    // =========================== scale factors and the activation operand ===========================
+    // =========================== scale factors of the weights and of the term rows ===========================
     const int qq = wid & 3;                      // tensor-memory lane quadrant written by this warp (warps 2..5 -> 2,3,0,1)
     const uint32_t lane_base = static_cast<uint32_t>(qq * 32) << 16;
     const int st = tid - 64;                     // 0..127
     int cs = 0, slot = 0;
     uint32_t cph = 0, sfree_ph = 0, afree_ph = 0;
-    int prev_e = -1;
     bool first_op = true;
-    const int n_blk = K / 32;
-    for (long long it = item_begin; it < item_end; ++it) {
-      const int ti = static_cast<int>(it / tiles_per_expert), e = touched[ti];
-      const int row_begin = t_begin[ti], row_end = t_end[ti];
-      const int n_pass = (row_end - row_begin + tok_pass - 1) / tok_pass;
-      for (int pass = 0; pass < n_pass; ++pass) {
-        const bool new_operand = (prev_e != e) || (n_pass > 1);
-        prev_e = e;
-        if (new_operand) {
-          // ---- scale factors of the pass's term rows: global -> shared memory -> tensor memory ----
-          if (first_op) {
-            pdl_wait();  // the kernel before this one (split or gate/up) is complete and its term rows are visible
-          } else {
-            mbar_wait(act_free, afree_ph, a.status);  // MMAs that read the previous scale factors are done
-            afree_ph ^= 1u;
-          }
-          first_op = false;
-          const int row0 = row_begin + pass * tok_pass;
-          const int n_rows = min(tok_pass, row_end - row0) * kTerms;  // term rows that exist
-          // rows are n_blk bytes each and consecutive: one contiguous range, copied 16 bytes at a time
-          // (the 16-byte chunks of a row are XOR-swizzled with the row number against bank conflicts)
-          const int n_chunk = n_blk / 16, cmask = min(n_chunk, 8) - 1;
-          const int n_vec = n_rows * n_chunk;
-          const uint4* src = reinterpret_cast<const uint4*>(a.aq_sf + static_cast<size_t>(row0) * kTerms * n_blk);
-          for (int i = st; i < n_vec; i += 128) {
-            const int r = i / n_chunk, c = i % n_chunk;
-            reinterpret_cast<uint4*>(sSfa)[r * n_chunk + (c ^ (r & cmask))] = __ldcg(src + i);
-          }
-          asm volatile("bar.sync 3, 128;" ::: "memory");
-          __syncwarp();
-          // K step ks owns two scale-factor blocks (its two scale words); column c of a block holds, in lane l of
-          // every quadrant, the word of term row 32c + l (rows that do not exist: any value)
-          for (int ks = 0; ks < n_steps; ++ks) {
-            uint32_t w[8];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              const int r = 32 * c + lane;
-              const uint2 v = *reinterpret_cast<const uint2*>(sSfa + (r * n_chunk + ((ks >> 1) ^ (r & cmask))) * 16 + (ks & 1) * 8);
-              w[c] = v.x;
-              w[4 + c] = v.y;
+    for (int phase = 0; phase < 2; ++phase) {
+      const Phase P = phase_of(phase, a, n_touched);
+      const int n_blk = P.K / 32;
+      const uint8_t* src_sf = phase == 0 ? a.sf1 : a.sf2;
+      int prev_ti = -1;
+      for (long long it = P.begin; it < P.end; ++it) {
+        const int ti = static_cast<int>(it / P.tiles);
+        const int row_begin = t_begin[ti], row_end = t_end[ti];
+        const int n_pass = (row_end - row_begin + tok_pass - 1) / tok_pass;
+        for (int pass = 0; pass < n_pass; ++pass) {
+          const bool new_operand = (prev_ti != ti) || (n_pass > 1);
+          prev_ti = ti;
+          if (new_operand) {
+            // ---- scale factors of the pass's term rows: global -> shared memory -> tensor memory ----
+            if (first_op) {
+              pdl_wait();  // the split kernel is complete: scale bytes of the tokens' terms, cleared counters
+            } else {
+              mbar_wait(act_free, afree_ph, a.status);  // MMAs that read the previous scale factors are done
+              afree_ph ^= 1u;
             }
-            tmem_st_32x8(tmem_base + lane_base + kColSfAct + static_cast<uint32_t>(ks * 8), w);
-          }
-          tmem_st_wait();
-          tc_fence_before_sync();
-          asm volatile("bar.sync 3, 128;" ::: "memory");  // sSfa may be overwritten only after every warp has read it
-          if (lane == 0) mbar_arrive(act_ready);
-        }
-        // ---- weight scale factors: one scale stage (256 rows x 16 bytes = 2 K steps) -> one 32-column group ----
-        for (int ks = 0; ks < n_steps; ks += 2) {
-          mbar_wait(&full_sc[cs], cph, a.status);
-          mbar_wait(&sf_free[slot], sfree_ph ^ 1u, a.status);
-          __syncwarp();  // the spins may leave lanes diverged; tcgen05.st is warp-collective
-          const unsigned char* blk = sSc + cs * kScStage;
-          uint4 r[8];
+            first_op = false;
+            if (phase == 1) {
+              // every gate/up item of this expert has published its rows of the intermediate
+              if (st == 0) counter_wait_ge(a.done + touched[ti], need_done, a.status);
+              asm volatile("bar.sync 3, 128;" ::: "memory");
+            }
+            const int row0 = row_begin + pass * tok_pass;
+            const int n_rows = min(tok_pass, row_end - row0) * kTerms;  // term rows that exist
+            // rows are n_blk bytes each and consecutive: one contiguous range, copied 16 bytes at a time
+            // (the 16-byte chunks of a row are XOR-swizzled with the row number against bank conflicts)
+            const int n_chunk = n_blk / 16, cmask = min(n_chunk, 8) - 1;
+            const int n_vec = n_rows * n_chunk;
+            const uint4* src = reinterpret_cast<const uint4*>(src_sf + static_cast<size_t>(row0) * kTerms * n_blk);
+            for (int i = st; i < n_vec; i += 128) {
+              const int r = i / n_chunk, c = i % n_chunk;
+              reinterpret_cast<uint4*>(sSfa)[r * n_chunk + (c ^ (r & cmask))] = __ldcg(src + i);
+            }
+            asm volatile("bar.sync 3, 128;" ::: "memory");
+            __syncwarp();
+            // K step ks owns two scale-factor blocks (its two scale words); column c of a block holds, in lane l of
+            // every quadrant, the word of term row 32c + l (rows that do not exist: any value)
+            for (int ks = 0; ks < P.n_steps; ++ks) {
+              uint32_t w[8];
 #pragma unroll
-          for (int c = 0; c < 8; ++c) r[c] = *reinterpret_cast<const uint4*>(blk + (lane + 32 * c) * 16);
-          // column 8t + c of the group: scale word t (K blocks 4t..4t+3 of the 16) for weight row lane + 32c
-          asm volatile(
-              "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
-              "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};" ::"r"(
-                  tmem_base + lane_base + kColSfW + static_cast<uint32_t>(slot * 32)),
-              "r"(r[0].x), "r"(r[1].x), "r"(r[2].x), "r"(r[3].x), "r"(r[4].x), "r"(r[5].x), "r"(r[6].x), "r"(r[7].x),
-              "r"(r[0].y), "r"(r[1].y), "r"(r[2].y), "r"(r[3].y), "r"(r[4].y), "r"(r[5].y), "r"(r[6].y), "r"(r[7].y),
-              "r"(r[0].z), "r"(r[1].z), "r"(r[2].z), "r"(r[3].z), "r"(r[4].z), "r"(r[5].z), "r"(r[6].z), "r"(r[7].z),
-              "r"(r[0].w), "r"(r[1].w), "r"(r[2].w), "r"(r[3].w), "r"(r[4].w), "r"(r[5].w), "r"(r[6].w), "r"(r[7].w)
-              : "memory");
-          tmem_st_wait();
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) {
-            mbar_arrive(&sf_full[slot]);
-            mbar_arrive(&empty_sc[cs]);
+              for (int c = 0; c < 4; ++c) {
+                const int r = 32 * c + lane;
+                const uint2 v = *reinterpret_cast<const uint2*>(sSfa + (r * n_chunk + ((ks >> 1) ^ (r & cmask))) * 16 + (ks & 1) * 8);
+                w[c] = v.x;
+                w[4 + c] = v.y;
+              }
+              tmem_st_32x8(tmem_base + lane_base + kColSfAct + static_cast<uint32_t>(ks * 8), w);
+            }
+            tmem_st_wait();
+            tc_fence_before_sync();
+            asm volatile("bar.sync 3, 128;" ::: "memory");  // sSfa may be overwritten only after every warp has read it
+            if (lane == 0) mbar_arrive(act_ready);
           }
-          if (++cs == kScStages) { cs = 0; cph ^= 1u; }
-          if (++slot == kSfGroups) { slot = 0; sfree_ph ^= 1u; }
+          // ---- weight scale factors: one scale stage (256 rows x 16 bytes = 2 K steps) -> one 32-column group ----
+          for (int ks = 0; ks < P.n_steps; ks += 2) {
+            mbar_wait(&full_sc[cs], cph, a.status);
+            mbar_wait(&sf_free[slot], sfree_ph ^ 1u, a.status);
+            __syncwarp();  // the spins may leave lanes diverged; tcgen05.st is warp-collective
+            const unsigned char* blk = sSc + cs * kScStage;
+            uint4 r[8];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) r[c] = *reinterpret_cast<const uint4*>(blk + (lane + 32 * c) * 16);
+            // column 8t + c of the group: scale word t (K blocks 4t..4t+3 of the 16) for weight row lane + 32c
+            asm volatile(
+                "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+                "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};" ::"r"(
+                    tmem_base + lane_base + kColSfW + static_cast<uint32_t>(slot * 32)),
+                "r"(r[0].x), "r"(r[1].x), "r"(r[2].x), "r"(r[3].x), "r"(r[4].x), "r"(r[5].x), "r"(r[6].x), "r"(r[7].x),
+                "r"(r[0].y), "r"(r[1].y), "r"(r[2].y), "r"(r[3].y), "r"(r[4].y), "r"(r[5].y), "r"(r[6].y), "r"(r[7].y),
+                "r"(r[0].z), "r"(r[1].z), "r"(r[2].z), "r"(r[3].z), "r"(r[4].z), "r"(r[5].z), "r"(r[6].z), "r"(r[7].z),
+                "r"(r[0].w), "r"(r[1].w), "r"(r[2].w), "r"(r[3].w), "r"(r[4].w), "r"(r[5].w), "r"(r[6].w), "r"(r[7].w)
+                : "memory");
+            tmem_st_wait();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+              mbar_arrive(&sf_full[slot]);
+              mbar_arrive(&empty_sc[cs]);
+            }
+            if (++cs == kScStages) { cs = 0; cph ^= 1u; }
+            if (++slot == kSfGroups) { slot = 0; sfree_ph ^= 1u; }
+          }
         }
       }
     }
@@ -489,86 +561,99 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_const
     const int jl = lane >> 3, tl = lane & 7;
     const int cb = 16 * (tl & 1) + 8 * ((tl >> 1) & 1) + 4 * (tl >> 2);
     uint32_t acc_ph = 0;
-    for (long long it = item_begin; it < item_end; ++it) {
-      const int ti = static_cast<int>(it / tiles_per_expert);
-      const int tile = static_cast<int>(it % tiles_per_expert);
-      const int row_begin = t_begin[ti], row_end = t_end[ti];
-      const int n_pass = (row_end - row_begin + tok_pass - 1) / tok_pass;
-      for (int pass = 0; pass < n_pass; ++pass) {
-        const int row0 = row_begin + pass * tok_pass;
-        const int n_tok = min(tok_pass, row_end - row0);
-        const int p = row0 + 4 * q + jl;                 // sorted row of this lane's token
-        const bool tok_live = 4 * q + jl < n_tok;
-        mbar_wait(acc_full, acc_ph, a.status);
-        __syncwarp();  // tcgen05.ld is warp-collective
-        acc_ph ^= 1u;
-        tc_fence_after_sync();
-        float acc[8][4];  // [chunk of 32 columns][column cb + c]
-        if (4 * q < n_tok) {
+    for (int phase = 0; phase < 2; ++phase) {
+      const Phase P = phase_of(phase, a, n_touched);
+      for (long long it = P.begin; it < P.end; ++it) {
+        const int ti = static_cast<int>(it / P.tiles), tile = static_cast<int>(it % P.tiles);
+        const int row_begin = t_begin[ti], row_end = t_end[ti];
+        const int n_pass = (row_end - row_begin + tok_pass - 1) / tok_pass;
+        for (int pass = 0; pass < n_pass; ++pass) {
+          const int row0 = row_begin + pass * tok_pass;
+          const int n_tok = min(tok_pass, row_end - row0);
+          const int p = row0 + 4 * q + jl;                 // sorted row of this lane's token
+          const bool tok_live = 4 * q + jl < n_tok;
+          mbar_wait(acc_full, acc_ph, a.status);
+          __syncwarp();  // tcgen05.ld is warp-collective
+          acc_ph ^= 1u;
+          tc_fence_after_sync();
+          float acc[8][4];  // [chunk of 32 columns][column cb + c]
+          if (4 * q < n_tok) {
+            // two loads in flight: chunk m + 1 is on its way while chunk m is reduced
+            uint32_t v[2][32];
+            tmem_ld_32x32(tmem_base + lane_base + kColD, v[0]);
 #pragma unroll
-          for (int m = 0; m < 8; ++m) {
-            uint32_t v[32];
-            tmem_ld_32x32(tmem_base + lane_base + kColD + static_cast<uint32_t>(32 * m), v);
-            tmem_ld_wait();
-            float a16[16], a8[8];
+            for (int m = 0; m < 8; ++m) {
+              tmem_ld_wait();
+              if (m + 1 < 8) tmem_ld_32x32(tmem_base + lane_base + kColD + static_cast<uint32_t>(32 * (m + 1)), v[(m + 1) & 1]);
+              const uint32_t(&vc)[32] = v[m & 1];
+              float a16[16], a8[8];
 #pragma unroll
-            for (int k = 0; k < 16; ++k) {
-              const float lo = __uint_as_float(v[k]), hi = __uint_as_float(v[16 + k]);
-              a16[k] = ((tl & 1) ? hi : lo) + __shfl_xor_sync(0xffffffffu, (tl & 1) ? lo : hi, 1);
+              for (int k = 0; k < 16; ++k) {
+                const float lo = __uint_as_float(vc[k]), hi = __uint_as_float(vc[16 + k]);
+                a16[k] = ((tl & 1) ? hi : lo) + __shfl_xor_sync(0xffffffffu, (tl & 1) ? lo : hi, 1);
+              }
+#pragma unroll
+              for (int k = 0; k < 8; ++k)
+                a8[k] = ((tl & 2) ? a16[8 + k] : a16[k]) + __shfl_xor_sync(0xffffffffu, (tl & 2) ? a16[k] : a16[8 + k], 2);
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                acc[m][k] = ((tl & 4) ? a8[4 + k] : a8[k]) + __shfl_xor_sync(0xffffffffu, (tl & 4) ? a8[k] : a8[4 + k], 4);
             }
-#pragma unroll
-            for (int k = 0; k < 8; ++k)
-              a8[k] = ((tl & 2) ? a16[8 + k] : a16[k]) + __shfl_xor_sync(0xffffffffu, (tl & 2) ? a16[k] : a16[8 + k], 2);
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              acc[m][k] = ((tl & 4) ? a8[4 + k] : a8[k]) + __shfl_xor_sync(0xffffffffu, (tl & 4) ? a8[k] : a8[4 + k], 4);
           }
-        }
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(acc_empty);  // the accumulator is free: the rest overlaps the next item's MMAs
-        if (4 * q >= n_tok) continue;
-        if (STAGE1) {
-          // SwiGLU and the 8-term split, one (token, block of 32 consecutive i) per group of 8 lanes: in round rd
-          // the four lane groups take the four blocks of the quadrant's token rd (gate in chunk m, up in chunk m + 4),
-          // so that a quadrant with one token finishes in one round
-          const int n_blk_i = a.I / 32;
-          const int n_q = min(4, n_tok - 4 * q);
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(acc_empty);  // the accumulator is free: the rest overlaps the next item's MMAs
+          if (4 * q >= n_tok) continue;
+          if (phase == 0) {
+            // SwiGLU and the 8-term split, one (token, block of 32 consecutive i) per group of 8 lanes: in round rd
+            // the four lane groups take the four blocks of the quadrant's token rd (gate in chunk m, up in chunk m + 4),
+            // so that a quadrant with one token finishes in one round
+            const int n_blk_i = a.I / 32;
+            const int n_q = min(4, n_tok - 4 * q);
 #pragma unroll 1
-          for (int rd = 0; rd < n_q; ++rd) {
-            float gsel[4], usel[4];
+            for (int rd = 0; rd < n_q; ++rd) {
+              float gsel[4], usel[4];
 #pragma unroll
-            for (int m = 0; m < 4; ++m)
+              for (int m = 0; m < 4; ++m)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                  const float tg = __shfl_sync(0xffffffffu, acc[m][c], rd * 8 + tl);
+                  const float tu = __shfl_sync(0xffffffffu, acc[m + 4][c], rd * 8 + tl);
+                  if (jl == m) {
+                    gsel[c] = tg;
+                    usel[c] = tu;
+                  }
+                }
+              float r[1][4];
 #pragma unroll
               for (int c = 0; c < 4; ++c) {
-                const float tg = __shfl_sync(0xffffffffu, acc[m][c], rd * 8 + tl);
-                const float tu = __shfl_sync(0xffffffffu, acc[m + 4][c], rd * 8 + tl);
-                if (jl == m) {
-                  gsel[c] = tg;
-                  usel[c] = tu;
-                }
+                const float sv = __fdividef(gsel[c], 1.0f + __expf(-gsel[c])) * usel[c];
+                r[0][c] = __bfloat162float(__float2bfloat16_rn(sv));  // the intermediate is defined as a bf16 value
               }
-            float r[1][4];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              const float sv = __fdividef(gsel[c], 1.0f + __expf(-gsel[c])) * usel[c];
-              r[0][c] = __bfloat162float(__float2bfloat16_rn(sv));  // the intermediate is defined as a bf16 value
+              const int i0 = tile * 128 + 32 * jl;
+              uint8_t* qrow = a.aq2 + static_cast<size_t>(row0 + 4 * q + rd) * kTerms * (a.I / 2) + ((i0 + cb) >> 1);
+              uint8_t* srow = a.sf2 + static_cast<size_t>(row0 + 4 * q + rd) * kTerms * n_blk_i + (i0 >> 5);
+              split_terms<1>(r, [&](int, int t, uint32_t bytes, int se) {
+                *reinterpret_cast<uint16_t*>(qrow + static_cast<size_t>(t) * (a.I / 2)) = static_cast<uint16_t>(bytes);
+                if (tl == 0) srow[static_cast<size_t>(t) * n_blk_i] = static_cast<uint8_t>(se + 127);
+              });
             }
-            const int i0 = tile * 128 + 32 * jl;
-            uint8_t* qrow = a.aq_out + static_cast<size_t>(row0 + 4 * q + rd) * kTerms * (a.I / 2) + ((i0 + cb) >> 1);
-            uint8_t* srow = a.aq_sf_out + static_cast<size_t>(row0 + 4 * q + rd) * kTerms * n_blk_i + (i0 >> 5);
-            split_terms<1>(r, [&](int, int t, uint32_t bytes, int se) {
-              *reinterpret_cast<uint16_t*>(qrow + static_cast<size_t>(t) * (a.I / 2)) = static_cast<uint16_t>(bytes);
-              if (tl == 0) srow[static_cast<size_t>(t) * n_blk_i] = static_cast<uint8_t>(se + 127);
-            });
-          }
-        } else {
-          if (tok_live) {
-            float* dst = a.y + static_cast<size_t>(p) * a.R + tile * kTile + cb;
+          } else {
+            if (tok_live) {
+              float* dst = a.y + static_cast<size_t>(p) * P.R + tile * kTile + cb;
 #pragma unroll
-            for (int m = 0; m < 8; ++m)
-              *reinterpret_cast<float4*>(dst + 32 * m) = make_float4(acc[m][0], acc[m][1], acc[m][2], acc[m][3]);
+              for (int m = 0; m < 8; ++m)
+                *reinterpret_cast<float4*>(dst + 32 * m) = make_float4(acc[m][0], acc[m][1], acc[m][2], acc[m][3]);
+            }
           }
+        }
+        if (phase == 0) {
+          // publish: this warp's rows of the item (all passes) are written; TMA (asynchronous proxy) and plain loads
+          // of other CTAs will read them
+          fence_proxy_async_all();
+          __threadfence();
+          __syncwarp();
+          if (lane == 0) atomicAdd(a.done + touched[ti], 1);
         }
       }
     }
@@ -628,17 +713,17 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
                              int* status_word, cudaStream_t st) {
   static bool attr_done = false;
   if (!attr_done) {
-    if (cudaFuncSetAttribute(ffn_native_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-        cudaFuncSetAttribute(ffn_native_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+    if (cudaFuncSetAttribute(ffn_native_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
       return MOE_ERR_CUDA;
     attr_done = true;
   }
   const size_t S = static_cast<size_t>(sh.T) * sh.k;
-  // scratch: term rows of the intermediate and of the token rows, each followed by its scale bytes
+  // scratch: term rows of the intermediate and of the token rows, each followed by its scale bytes; the counters
   uint8_t* aq2 = static_cast<uint8_t*>(scratch);
   uint8_t* sf2 = aq2 + align_up(S * kTerms * (sh.I / 2), kAlign);
   uint8_t* aq1 = sf2 + align_up(S * kTerms * (sh.I / 32), kAlign);
   uint8_t* sf1 = aq1 + align_up(S * kTerms * (sh.H / 2), kAlign);
+  int* done = reinterpret_cast<int*>(sf1 + align_up(S * kTerms * (sh.H / 32), kAlign));
   // tokens per pass: the term-row box is 8 * tok_pass rows; small batches fetch less
   const int tok_pass = S <= 4 ? 4 : (S <= 8 ? 8 : kMaxTokPass);
   CUtensorMap tm_w13, tm_w2, tm_s13, tm_s2, tm_a1, tm_a2;
@@ -650,37 +735,27 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
       !nat_map(&tm_s13, s13, sh.H / 32, static_cast<uint64_t>(sh.E) * 2 * sh.I, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE) ||
       !nat_map(&tm_s2, s2, sh.I / 32, static_cast<uint64_t>(sh.E) * sh.H, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE))
     return MOE_ERR_CUDA;
-  const size_t split_threads = S * (sh.H / 32) * 8;
+  const size_t split_threads = S * (sh.H / 32) * 8 > static_cast<size_t>(sh.E) ? S * (sh.H / 32) * 8 : static_cast<size_t>(sh.E);
   if (launch_pdl(native_split_kernel, dim3(static_cast<unsigned>((split_threads + 255) / 256)), dim3(256), 0, st, x_perm, aq1, sf1,
-                 static_cast<int>(S), sh.H) != cudaSuccess)
+                 done, static_cast<int>(S), sh.H, sh.E) != cudaSuccess)
     return MOE_ERR_CUDA;
-  const int grid = sm_count();
   NatArgs a;
-  a.x = x_perm;
+  a.sf1 = sf1;
+  a.aq2 = aq2;
+  a.sf2 = sf2;
+  a.done = done;
   a.offsets = offsets;
   a.y = y_perm;
   a.status = status_word;
   a.E = sh.E;
+  a.H = sh.H;
   a.I = sh.I;
   a.S = static_cast<int>(S);
   a.tok_pass = tok_pass;
-  a.aq = aq1;
-  a.aq_sf = sf1;
-  a.aq_out = aq2;
-  a.aq_sf_out = sf2;
-  a.K = sh.H;
-  a.R = 2 * sh.I;
-  if (launch_pdl(ffn_native_kernel<true>, dim3(grid), dim3(kNatThreads), nat_smem(sh.E, sh.H).total + 1024, st, tm_w13, tm_s13,
-                 tm_a1, a) != cudaSuccess)
+  if (launch_pdl(ffn_native_kernel, dim3(sm_count()), dim3(kNatThreads), nat_smem(sh.E, sh.H > sh.I ? sh.H : sh.I).total + 1024,
+                 st, tm_w13, tm_s13, tm_a1, tm_w2, tm_s2, tm_a2, a) != cudaSuccess)
     return MOE_ERR_CUDA;
-  a.aq = aq2;
-  a.aq_sf = sf2;
-  a.K = sh.I;
-  a.R = sh.H;
-  if (launch_pdl(ffn_native_kernel<false>, dim3(grid), dim3(kNatThreads), nat_smem(sh.E, sh.I).total + 1024, st, tm_w2, tm_s2,
-                 tm_a2, a) != cudaSuccess)
-    return MOE_ERR_CUDA;
-  note_kernel("ffn_native_mxf4_block_scaled", 3);
+  note_kernel("ffn_native_mxf4_block_scaled", 2);
   return MOE_OK;
 }
 

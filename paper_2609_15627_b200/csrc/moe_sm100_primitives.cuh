@@ -32,6 +32,19 @@ MOE_DEVINL bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// The same with a suspend-time hint: the thread may sleep in the instruction, up to about `hint_ns`, until the
+// phase completes, instead of spinning - a spinning warp takes issue slots from the warps that share its scheduler.
+MOE_DEVINL bool mbar_try_wait_sleepy(uint64_t* bar, uint32_t parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok != 0;
+}
 // Bounded wait: gives up after kWaitLimitCycles, records MOE_ERR_TIMEOUT in *status and lets the caller
 // go on (the data is then wrong, but every warp keeps taking part in every barrier, so nothing hangs).
 // Once the status word is set, every later wait in the grid gives up after a short spin, so that one
@@ -40,7 +53,7 @@ MOE_DEVINL void mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
   if (mbar_try_wait(bar, parity)) return;
   const long long t0 = clock64();
   int spins = 0;
-  while (!mbar_try_wait(bar, parity)) {
+  while (!mbar_try_wait_sleepy(bar, parity, 2000u)) {
     const long long waited = clock64() - t0;
     if (waited > kWaitLimitCycles) {
       if (status != nullptr) atomicExch(status, static_cast<int>(MOE_ERR_TIMEOUT));
