@@ -320,9 +320,55 @@ def main():
         barrier()
         eager_ms_step = ee0.elapsed_time(ee1) / n_inner
 
+    # ---- the expert-FFN call alone, graph-replayed like the step (decode) ------------------------------------------
+    # Eager launches of kernels this short leave the GPU idle between the event and the launch, which the bracketing
+    # events count.  So the call is also captured alone, one graph per batch of the cycle on that batch's own routed
+    # and permuted inputs, and the replays are timed back to back: consecutive calls touch different experts, as in
+    # the step.
+    ffn_graph_ms, n_ffn = None, 0
+    if use_graph:
+        fbufs = []
+        for i in range(n_cycle):
+            b = moe.LayerBuffers(sh)
+            l, x = batches[i]
+            moe.moe_route(l, wl.k, b.topk_ids, b.topk_w, b.expert_offsets, b.ws, stream)
+            moe.moe_permute(x, b.topk_ids, b.expert_offsets, sh, b.x_perm, b.perm, b.inv_perm, b.ws, stream)
+            fbufs.append(b)
+        barrier()
+
+        def ffn_only(b, st=stream):
+            moe.moe_expert_ffn(b.x_perm, b.expert_offsets, *weights, sh, b.y_perm, b.status, b.ws, st)
+
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            ffn_only(fbufs[0], None)
+        stream.wait_stream(side)
+        barrier()
+        fgraphs = []
+        for b in fbufs:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                ffn_only(b, None)
+            fgraphs.append(g)
+        for i in range(max(args.warmup, 3)):
+            fgraphs[i % n_cycle].replay()
+        barrier()
+        n_ffn = max(n_cycle, min(args.steps, 512))
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        for i in range(n_ffn):
+            fgraphs[i % n_cycle].replay()
+        f1.record(stream)
+        barrier()
+        ffn_graph_ms = f0.elapsed_time(f1) / n_ffn
+        assert all(int(b.status.item()) == 0 for b in fbufs), "device-side wait timed out"
+
     # ---- roofline of the dominant call (the expert FFN) --------------------------------------------------------
-    ffn_ms = float(np.mean([a.elapsed_time(b) for a, b in inner]))
-    mean_touched = float(np.mean([touched[i % n_cycle] for i in range(n_inner)]))
+    ffn_eager_ms = float(np.mean([a.elapsed_time(b) for a, b in inner]))
+    ffn_ms = ffn_graph_ms if ffn_graph_ms is not None else ffn_eager_ms
+    n_avg = n_ffn if ffn_graph_ms is not None else n_inner
+    mean_touched = float(np.mean([touched[i % n_cycle] for i in range(n_avg)]))
     peaks = load_peaks()
     if decode:
         alg = ffn_algorithmic_bytes(wl, mean_touched)
@@ -337,7 +383,9 @@ def main():
                 "algorithmic_flops": fl}
     roof.update({"kernel": "moe_expert_ffn",
                  "ms": ffn_ms, "peak_source": peaks["source"], "experts_touched": mean_touched,
-                 "timed_in": "eager steps right after the graph-replayed region" if use_graph else "the timed region"})
+                 "timed_in": ("graph replays of the call alone, one graph per batch of the cycle, right after the timed region"
+                              if use_graph else "the timed region"),
+                 "ms_between_events_in_eager_steps": ffn_eager_ms})
 
     # ---- end to end through the host-buffer entry point ---------------------------------------------------------
     e2e = None

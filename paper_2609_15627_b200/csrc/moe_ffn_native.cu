@@ -32,7 +32,7 @@
 //   warp 1      allocates tensor memory, issues the MMAs, commits to mbarriers
 //   warps 2..5  move weight scale bytes into tensor memory (tcgen05.st), and at a change of (expert, pass) the
 //               scale bytes of its term rows
-//   warps 8..11 epilogue, one warp per tensor-memory lane quadrant (4 tokens each): sum the 8 term rows of each
+//   warps 6..9  epilogue, one warp per tensor-memory lane quadrant (4 tokens each): sum the 8 term rows of each
 //               token, then SwiGLU + bf16 rounding + the 8-term split for the down projection (gate/up) or the
 //               fp32 store (down)
 // Every wait is bounded and reports through the status word.
@@ -57,8 +57,8 @@ constexpr int kSfGroups = 3;          // tensor-memory groups for the weight sca
 constexpr int kTerms = 8;             // E2M1 terms per activation value
 constexpr int kMaxTokPass = 16;       // tokens per pass (16 x 8 = 128 operand rows)
 constexpr int kMaxK = 4096;           // scale factors of one pass's term rows stay in tensor memory: 8 columns per K step
-constexpr int kNatThreads = 12 * 32;
-constexpr int kEpiWarp = 8;           // warps 8..11: warp % 4 = 0..3 -> one tensor-memory lane quadrant each
+constexpr int kNatThreads = 10 * 32;
+constexpr int kEpiWarp = 6;           // warps 6..9: warp % 4 = 2, 3, 0, 1 -> one tensor-memory lane quadrant each
 constexpr uint32_t kNatTmemCols = 512;
 // tensor-memory columns: one 256-column accumulator; per K step two scale words per operand row, each its own
 // scale-factor block of 4 columns (a block covers 128 rows - rows 32c..32c+31 in column c - and must start on a
@@ -214,7 +214,9 @@ MOE_DEVINL void split_terms(float (&r)[NB][4], Store store) {
 }  // namespace
 
 // ---- split kernel: bf16 token rows -> 8 E2M1 term rows with their scale bytes; 8 threads per 32-element block ----
-__global__ void __launch_bounds__(256) native_split_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict__ aq,
+// Few, large CTAs: the FFN grid's CTAs need a whole SM each and are handed out in blockIdx order, so every SM this
+// grid still occupies delays one of them - with at most (SMs - working FFN CTAs) CTAs here, only idle ones.
+__global__ void __launch_bounds__(1024) native_split_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict__ aq,
                                                            uint8_t* __restrict__ aq_sf, int* __restrict__ done, int S, int H,
                                                            int E) {
   pdl_launch_dependents();  // the FFN grid may set up and start its weight stream; it waits before it reads aq or done
@@ -270,7 +272,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   const int need_done = 4 * (2 * a.I / kTile);  // four epilogue warps publish each gate/up item of an expert
 
   // ---- setup: touched experts, barriers, tensor memory ----
-  if (tid == 32 * 6) {  // an idle warp fetches the tensor maps while the others set up
+  if (tid == 32 * 3) {  // a warp with nothing to set up fetches the tensor maps
     prefetch_tmap(&tmap_w13);
     prefetch_tmap(&tmap_s13);
     prefetch_tmap(&tmap_a1);
@@ -561,99 +563,110 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     const int jl = lane >> 3, tl = lane & 7;
     const int cb = 16 * (tl & 1) + 8 * ((tl >> 1) & 1) + 4 * (tl >> 2);
     uint32_t acc_ph = 0;
-    for (int phase = 0; phase < 2; ++phase) {
-      const Phase P = phase_of(phase, a, n_touched);
-      for (long long it = P.begin; it < P.end; ++it) {
-        const int ti = static_cast<int>(it / P.tiles), tile = static_cast<int>(it % P.tiles);
-        const int row_begin = t_begin[ti], row_end = t_end[ti];
-        const int n_pass = (row_end - row_begin + tok_pass - 1) / tok_pass;
-        for (int pass = 0; pass < n_pass; ++pass) {
-          const int row0 = row_begin + pass * tok_pass;
-          const int n_tok = min(tok_pass, row_end - row0);
-          const int p = row0 + 4 * q + jl;                 // sorted row of this lane's token
-          const bool tok_live = 4 * q + jl < n_tok;
-          mbar_wait(acc_full, acc_ph, a.status);
-          __syncwarp();  // tcgen05.ld is warp-collective
-          acc_ph ^= 1u;
-          tc_fence_after_sync();
-          float acc[8][4];  // [chunk of 32 columns][column cb + c]
-          if (4 * q < n_tok) {
-            // two loads in flight: chunk m + 1 is on its way while chunk m is reduced
-            uint32_t v[2][32];
-            tmem_ld_32x32(tmem_base + lane_base + kColD, v[0]);
+    // One pass of one item.  `dry` runs the same instructions on whatever tensor memory holds, with every wait, signal
+    // and store left out: each CTA executes this code only a few times, so its first real use would otherwise pay
+    // for fetching it - on the critical path of a one-item CTA - while the warp has nothing to do before the first
+    // accumulator is complete.
+    auto run_pass = [&](const int phase, const int out_stride, const int tile, const int row0, const int n_tok, const bool dry) {
+      const int p = row0 + 4 * q + jl;                 // sorted row of this lane's token
+      const bool tok_live = !dry && 4 * q + jl < n_tok;
+      if (!dry) {
+        mbar_wait(acc_full, acc_ph, a.status);
+        acc_ph ^= 1u;
+      }
+      __syncwarp();  // tcgen05.ld is warp-collective
+      tc_fence_after_sync();
+      float acc[8][4];  // [chunk of 32 columns][column cb + c]
+      if (dry || 4 * q < n_tok) {
 #pragma unroll
-            for (int m = 0; m < 8; ++m) {
-              tmem_ld_wait();
-              if (m + 1 < 8) tmem_ld_32x32(tmem_base + lane_base + kColD + static_cast<uint32_t>(32 * (m + 1)), v[(m + 1) & 1]);
-              const uint32_t(&vc)[32] = v[m & 1];
-              float a16[16], a8[8];
+        for (int m = 0; m < 8; ++m) {
+          uint32_t vc[32];
+          tmem_ld_32x32(tmem_base + lane_base + kColD + static_cast<uint32_t>(32 * m), vc);
+          tmem_ld_wait();
+          float a16[16], a8[8];
 #pragma unroll
-              for (int k = 0; k < 16; ++k) {
-                const float lo = __uint_as_float(vc[k]), hi = __uint_as_float(vc[16 + k]);
-                a16[k] = ((tl & 1) ? hi : lo) + __shfl_xor_sync(0xffffffffu, (tl & 1) ? lo : hi, 1);
-              }
-#pragma unroll
-              for (int k = 0; k < 8; ++k)
-                a8[k] = ((tl & 2) ? a16[8 + k] : a16[k]) + __shfl_xor_sync(0xffffffffu, (tl & 2) ? a16[k] : a16[8 + k], 2);
-#pragma unroll
-              for (int k = 0; k < 4; ++k)
-                acc[m][k] = ((tl & 4) ? a8[4 + k] : a8[k]) + __shfl_xor_sync(0xffffffffu, (tl & 4) ? a8[k] : a8[4 + k], 4);
-            }
+          for (int k = 0; k < 16; ++k) {
+            const float lo = __uint_as_float(vc[k]), hi = __uint_as_float(vc[16 + k]);
+            a16[k] = ((tl & 1) ? hi : lo) + __shfl_xor_sync(0xffffffffu, (tl & 1) ? lo : hi, 1);
           }
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(acc_empty);  // the accumulator is free: the rest overlaps the next item's MMAs
-          if (4 * q >= n_tok) continue;
-          if (phase == 0) {
-            // SwiGLU and the 8-term split, one (token, block of 32 consecutive i) per group of 8 lanes: in round rd
-            // the four lane groups take the four blocks of the quadrant's token rd (gate in chunk m, up in chunk m + 4),
-            // so that a quadrant with one token finishes in one round
-            const int n_blk_i = a.I / 32;
-            const int n_q = min(4, n_tok - 4 * q);
-#pragma unroll 1
-            for (int rd = 0; rd < n_q; ++rd) {
-              float gsel[4], usel[4];
 #pragma unroll
-              for (int m = 0; m < 4; ++m)
+          for (int k = 0; k < 8; ++k)
+            a8[k] = ((tl & 2) ? a16[8 + k] : a16[k]) + __shfl_xor_sync(0xffffffffu, (tl & 2) ? a16[k] : a16[8 + k], 2);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                  const float tg = __shfl_sync(0xffffffffu, acc[m][c], rd * 8 + tl);
-                  const float tu = __shfl_sync(0xffffffffu, acc[m + 4][c], rd * 8 + tl);
-                  if (jl == m) {
-                    gsel[c] = tg;
-                    usel[c] = tu;
-                  }
-                }
-              float r[1][4];
-#pragma unroll
-              for (int c = 0; c < 4; ++c) {
-                const float sv = __fdividef(gsel[c], 1.0f + __expf(-gsel[c])) * usel[c];
-                r[0][c] = __bfloat162float(__float2bfloat16_rn(sv));  // the intermediate is defined as a bf16 value
-              }
-              const int i0 = tile * 128 + 32 * jl;
-              uint8_t* qrow = a.aq2 + static_cast<size_t>(row0 + 4 * q + rd) * kTerms * (a.I / 2) + ((i0 + cb) >> 1);
-              uint8_t* srow = a.sf2 + static_cast<size_t>(row0 + 4 * q + rd) * kTerms * n_blk_i + (i0 >> 5);
-              split_terms<1>(r, [&](int, int t, uint32_t bytes, int se) {
-                *reinterpret_cast<uint16_t*>(qrow + static_cast<size_t>(t) * (a.I / 2)) = static_cast<uint16_t>(bytes);
-                if (tl == 0) srow[static_cast<size_t>(t) * n_blk_i] = static_cast<uint8_t>(se + 127);
-              });
-            }
-          } else {
-            if (tok_live) {
-              float* dst = a.y + static_cast<size_t>(p) * P.R + tile * kTile + cb;
-#pragma unroll
-              for (int m = 0; m < 8; ++m)
-                *reinterpret_cast<float4*>(dst + 32 * m) = make_float4(acc[m][0], acc[m][1], acc[m][2], acc[m][3]);
-            }
-          }
+          for (int k = 0; k < 4; ++k)
+            acc[m][k] = ((tl & 4) ? a8[4 + k] : a8[k]) + __shfl_xor_sync(0xffffffffu, (tl & 4) ? a8[k] : a8[4 + k], 4);
         }
-        if (phase == 0) {
-          // publish: this warp's rows of the item (all passes) are written; TMA (asynchronous proxy) and plain loads
-          // of other CTAs will read them
-          fence_proxy_async_all();
-          __threadfence();
-          __syncwarp();
-          if (lane == 0) atomicAdd(a.done + touched[ti], 1);
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (!dry && lane == 0) mbar_arrive(acc_empty);  // the accumulator is free: the rest overlaps the next item's MMAs
+      if (!dry && 4 * q >= n_tok) return;
+      if (phase == 0) {
+        // SwiGLU and the 8-term split, one (token, block of 32 consecutive i) per group of 8 lanes: in round rd
+        // the four lane groups take the four blocks of the quadrant's token rd (gate in chunk m, up in chunk m + 4),
+        // so that a quadrant with one token finishes in one round
+        const int n_blk_i = a.I / 32;
+        const int n_q = dry ? 1 : min(4, n_tok - 4 * q);
+#pragma unroll 1
+        for (int rd = 0; rd < n_q; ++rd) {
+          float gsel[4], usel[4];
+#pragma unroll
+          for (int m = 0; m < 4; ++m)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              const float tg = __shfl_sync(0xffffffffu, acc[m][c], rd * 8 + tl);
+              const float tu = __shfl_sync(0xffffffffu, acc[m + 4][c], rd * 8 + tl);
+              if (jl == m) {
+                gsel[c] = tg;
+                usel[c] = tu;
+              }
+            }
+          float r[1][4];
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const float sv = __fdividef(gsel[c], 1.0f + __expf(-gsel[c])) * usel[c];
+            r[0][c] = __bfloat162float(__float2bfloat16_rn(sv));  // the intermediate is defined as a bf16 value
+          }
+          const int i0 = tile * 128 + 32 * jl;
+          uint8_t* qrow = a.aq2 + static_cast<size_t>(row0 + 4 * q + rd) * kTerms * (a.I / 2) + ((i0 + cb) >> 1);
+          uint8_t* srow = a.sf2 + static_cast<size_t>(row0 + 4 * q + rd) * kTerms * n_blk_i + (i0 >> 5);
+          split_terms<1>(r, [&](int, int t, uint32_t bytes, int se) {
+            if (!dry) {
+              *reinterpret_cast<uint16_t*>(qrow + static_cast<size_t>(t) * (a.I / 2)) = static_cast<uint16_t>(bytes);
+              if (tl == 0) srow[static_cast<size_t>(t) * n_blk_i] = static_cast<uint8_t>(se + 127);
+            }
+          });
+        }
+      } else {
+        if (tok_live) {
+          float* dst = a.y + static_cast<size_t>(p) * out_stride + tile * kTile + cb;
+#pragma unroll
+          for (int m = 0; m < 8; ++m)
+            *reinterpret_cast<float4*>(dst + 32 * m) = make_float4(acc[m][0], acc[m][1], acc[m][2], acc[m][3]);
+        }
+      }
+    };
+    for (int round = 0; round < 2; ++round) {  // round 0 is the dry run: one pass through the one call site below
+      const bool dry = round == 0;
+      for (int phase = 0; phase < (dry ? 1 : 2); ++phase) {
+        const Phase P = phase_of(phase, a, n_touched);
+        const long long it_begin = dry ? 0 : P.begin, it_end = dry ? 1 : P.end;
+        for (long long it = it_begin; it < it_end; ++it) {
+          const int ti = static_cast<int>(it / P.tiles), tile = static_cast<int>(it % P.tiles);
+          const int row_begin = dry ? 0 : t_begin[ti], row_end = dry ? 1 : t_end[ti];
+          const int n_pass = (row_end - row_begin + tok_pass - 1) / tok_pass;
+          for (int pass = 0; pass < n_pass; ++pass) {
+            const int row0 = row_begin + pass * tok_pass;
+            run_pass(phase, P.R, tile, row0, min(tok_pass, row_end - row0), dry);
+          }
+          if (!dry && phase == 0) {
+            // publish: this warp's rows of the item (all passes) are written; TMA (asynchronous proxy) and plain
+            // loads of other CTAs will read them
+            fence_proxy_async_all();
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) atomicAdd(a.done + touched[ti], 1);
+          }
         }
       }
     }
@@ -736,7 +749,7 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
       !nat_map(&tm_s2, s2, sh.I / 32, static_cast<uint64_t>(sh.E) * sh.H, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE))
     return MOE_ERR_CUDA;
   const size_t split_threads = S * (sh.H / 32) * 8 > static_cast<size_t>(sh.E) ? S * (sh.H / 32) * 8 : static_cast<size_t>(sh.E);
-  if (launch_pdl(native_split_kernel, dim3(static_cast<unsigned>((split_threads + 255) / 256)), dim3(256), 0, st, x_perm, aq1, sf1,
+  if (launch_pdl(native_split_kernel, dim3(static_cast<unsigned>((split_threads + 1023) / 1024)), dim3(1024), 0, st, x_perm, aq1, sf1,
                  done, static_cast<int>(S), sh.H, sh.E) != cudaSuccess)
     return MOE_ERR_CUDA;
   NatArgs a;
