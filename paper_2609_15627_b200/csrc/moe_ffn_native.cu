@@ -663,9 +663,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             // publish: this warp's rows of the item (all passes) are written; TMA (asynchronous proxy) and plain
             // loads of other CTAs will read them
             fence_proxy_async_all();
-            __threadfence();
-            __syncwarp();
-            if (lane == 0) atomicAdd(a.done + touched[ti], 1);
+            __syncwarp();  // orders the lanes' stores before lane 0's release
+            if (lane == 0) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(a.done + touched[ti]) : "memory");
           }
         }
       }
