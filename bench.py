@@ -28,8 +28,8 @@ DECODE = ("decode_c1", "decode_c64")
 # dram__bytes_read.sum + dram__bytes_write.sum per moe_expert_ffn call from one ncu capture of the
 # workload (see profiles/); None until captured.
 NCU_TRAFFIC_BYTES = {
-    "decode_c1": 108907776,      # ffn_native_kernel<true> 71.52 + 1.60 MB, <false> 35.79 MB (profiles/ffn_native_decode.md)
-    "decode_c64": 3058403336,    # 2033.1 + 10.5 MB and 1003.6 + 11.1 MB
+    "decode_c1": 111177216,      # ffn_native_kernel: 107.21 MB read + 3.97 MB written (profiles/ffn_native_decode.md)
+    "decode_c64": 3060525584,    # 3041.8 MB read + 18.8 MB written
     "prefill_8k": 5611119000,    # ffn_umma_kernel<true> 2.882 + 0.263 GB, <false> 1.431 + 1.034 GB (profiles/ffn_umma_prefill_8k.md)
 }
 
@@ -320,13 +320,13 @@ def main():
         barrier()
         eager_ms_step = ee0.elapsed_time(ee1) / n_inner
 
-    # ---- the expert-FFN call alone, graph-replayed like the step (decode) ------------------------------------------
+    # ---- the expert-FFN call alone, graph-replayed like the step (calls shorter than 100 us) -------------------------
     # Eager launches of kernels this short leave the GPU idle between the event and the launch, which the bracketing
-    # events count.  So the call is also captured alone, one graph per batch of the cycle on that batch's own routed
+    # events count.  So such a call is also captured alone, one graph per batch of the cycle on that batch's own routed
     # and permuted inputs, and the replays are timed back to back: consecutive calls touch different experts, as in
-    # the step.
+    # the step.  Longer calls keep the time between their events inside the eager steps.
     ffn_graph_ms, n_ffn = None, 0
-    if use_graph:
+    if use_graph and float(np.mean([a.elapsed_time(b) for a, b in inner])) < 0.1:
         fbufs = []
         for i in range(n_cycle):
             b = moe.LayerBuffers(sh)
@@ -384,7 +384,8 @@ def main():
     roof.update({"kernel": "moe_expert_ffn",
                  "ms": ffn_ms, "peak_source": peaks["source"], "experts_touched": mean_touched,
                  "timed_in": ("graph replays of the call alone, one graph per batch of the cycle, right after the timed region"
-                              if use_graph else "the timed region"),
+                              if ffn_graph_ms is not None else
+                              ("eager steps right after the graph-replayed region" if use_graph else "the timed region")),
                  "ms_between_events_in_eager_steps": ffn_eager_ms})
 
     # ---- end to end through the host-buffer entry point ---------------------------------------------------------
