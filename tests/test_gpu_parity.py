@@ -308,6 +308,17 @@ def test_layer_tiny():
     _check_layer_full(wl, d, None)
 
 
+@pytest.mark.parametrize("T,H,I,E,k,kernel", [
+    (8, 1024, 512, 32, 6, "ffn_native_mxf4_block_scaled"),   # the paper's own top-k (6), decode-sized
+    (24, 512, 256, 16, 6, "ffn_stream_bulk_ring_mma16816"),  # top-6 with I = 256, the paper's TP8 shard of I
+    (256, 512, 512, 8, 6, "ffn_umma_tcgen05_grouped"),       # top-6, prefill-sized
+])
+def test_layer_full_with_top6(T, H, I, E, k, kernel):
+    wl = inputs.Workload("top6", T, H, I, E, k)
+    d = inputs.make_workload(wl, seed=3)
+    _check_layer_full(wl, d, None)   # `kernel`: the expert-FFN variant this shape selects (see the kernel-choice test)
+
+
 @pytest.mark.parametrize("name", ["decode_c1", "decode_c64"])
 def test_layer_decode_full(name, prod_weights):
     wl = inputs.WORKLOADS[name]
