@@ -191,7 +191,16 @@ MOE_DEVINL void warp_copy_row(const __nv_bfloat16* src, __nv_bfloat16* dst, int 
   const uint4* s4 = reinterpret_cast<const uint4*>(src);
   uint4* d4 = reinterpret_cast<uint4*>(dst);
   const int n = H / 8;
-  for (int i = lane; i < n; i += 32) d4[i] = __ldg(&s4[i]);
+  // eight loads in flight per lane: a row is a few KB and one warp moves it, so latency is what counts
+  for (int i0 = lane; i0 < n; i0 += 32 * 8) {
+    uint4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      if (i0 + 32 * u < n) v[u] = __ldg(&s4[i0 + 32 * u]);
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      if (i0 + 32 * u < n) d4[i0 + 32 * u] = v[u];
+  }
 }
 
 // Small S: one warp per slot.  Rank of slot s inside its expert = number of earlier slots with the
@@ -345,19 +354,37 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
   float acc[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) acc[i] = 0.0f;
-  for (int j = 0; j < k; ++j) {
-    const int p = __ldg(&inv_perm[static_cast<size_t>(t) * k + j]);
-    const float wj = __ldg(&w[static_cast<size_t>(t) * k + j]);
-    const float4* src = reinterpret_cast<const float4*>(y + static_cast<size_t>(p) * H + c);
-    const float4 a = __ldg(src), b = __ldg(src + 1);
-    acc[0] = __fmaf_rn(wj, a.x, acc[0]);
-    acc[1] = __fmaf_rn(wj, a.y, acc[1]);
-    acc[2] = __fmaf_rn(wj, a.z, acc[2]);
-    acc[3] = __fmaf_rn(wj, a.w, acc[3]);
-    acc[4] = __fmaf_rn(wj, b.x, acc[4]);
-    acc[5] = __fmaf_rn(wj, b.y, acc[5]);
-    acc[6] = __fmaf_rn(wj, b.z, acc[6]);
-    acc[7] = __fmaf_rn(wj, b.w, acc[7]);
+  // slots in groups of four: the four row indices, then the eight row loads, are in flight together; the
+  // multiply-adds stay in slot order
+  for (int j0 = 0; j0 < k; j0 += 4) {
+    int p[4];
+    float wj[4];
+    float4 a[4], b[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (j0 + u < k) {
+        p[u] = __ldg(&inv_perm[static_cast<size_t>(t) * k + j0 + u]);
+        wj[u] = __ldg(&w[static_cast<size_t>(t) * k + j0 + u]);
+      }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (j0 + u < k) {
+        const float4* src = reinterpret_cast<const float4*>(y + static_cast<size_t>(p[u]) * H + c);
+        a[u] = __ldg(src);
+        b[u] = __ldg(src + 1);
+      }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (j0 + u < k) {
+        acc[0] = __fmaf_rn(wj[u], a[u].x, acc[0]);
+        acc[1] = __fmaf_rn(wj[u], a[u].y, acc[1]);
+        acc[2] = __fmaf_rn(wj[u], a[u].z, acc[2]);
+        acc[3] = __fmaf_rn(wj[u], a[u].w, acc[3]);
+        acc[4] = __fmaf_rn(wj[u], b[u].x, acc[4]);
+        acc[5] = __fmaf_rn(wj[u], b[u].y, acc[5]);
+        acc[6] = __fmaf_rn(wj[u], b[u].z, acc[6]);
+        acc[7] = __fmaf_rn(wj[u], b[u].w, acc[7]);
+      }
   }
   __nv_bfloat162 o[4];
 #pragma unroll
