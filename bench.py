@@ -263,9 +263,12 @@ def main():
     barrier()
 
     # Decode-sized steps are a handful of short kernels: like the paper's decode tiers they are replayed as CUDA
-    # graphs (one graph per batch of the cycle, each the four C-ABI calls captured as they are).
+    # graphs (the four C-ABI calls captured as they are).  A serving graph holds many layers back to back; here a
+    # graph holds kGraphSteps consecutive batches of the cycle (one layer call each), plus one single-step graph per
+    # batch for a step count that is not a multiple of kGraphSteps.
     use_graph = decode and not args.no_graph
-    graphs, launches_per_step = [], None
+    kGraphSteps = 8
+    graphs, multi_graphs, launches_per_step = [], [], None
     if use_graph:
         side = torch.cuda.Stream()
         side.wait_stream(stream)
@@ -281,8 +284,16 @@ def main():
                 step(i, st=None)
             launches_per_step = moe.moe_launch_count() - c0
             graphs.append(g)
+        for i0 in range(0, n_cycle, kGraphSteps):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for i in range(i0, i0 + kGraphSteps):
+                    step(i, st=None)
+            multi_graphs.append(g)
         for i in range(max(args.warmup, 3)):
             graphs[i % n_cycle].replay()
+        for g in multi_graphs:
+            g.replay()
         barrier()
 
     # ---- timed region: exactly K steps ---------------------------------------------------------------------
@@ -295,7 +306,10 @@ def main():
     sampler.start()
     e0.record(stream)
     if use_graph:
-        for i in range(args.steps):
+        n_multi = args.steps // kGraphSteps
+        for i in range(n_multi):
+            multi_graphs[i % len(multi_graphs)].replay()
+        for i in range(n_multi * kGraphSteps, args.steps):
             graphs[i % n_cycle].replay()
     else:
         for i in range(args.steps):
@@ -423,7 +437,7 @@ def main():
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": wl.name, "T": wl.T, "H": wl.H, "I": wl.I, "E": wl.E, "k": wl.k,
                        "parallelism": "replicas only" if world > 1 else "1 GPU",
-                       "launch": "cuda graph replay, one graph per batch of the cycle" if use_graph else "eager",
+                       "launch": "cuda graph replay, %d consecutive batches of the cycle per graph" % kGraphSteps if use_graph else "eager",
                        "eager_ms_per_step": eager_ms_step,
                        "l2": "inputs cycle over %d seeded batches; %.2f GB of expert weights resident (larger than L2)"
                              % (n_cycle, wl.E * expert_weight_bytes(wl.H, wl.I) / 1e9)},

@@ -78,6 +78,11 @@ uint64_t moe_launch_count(void);
  *   fixed fp32 sequence: d = max(d,-80); n = rint(d*0x1.715476p+0f); r = fma(n,-0x1.62e4p-1f,d);
  *   r = fma(n,-0x1.7f7d1cp-20f,r); p = Horner/fma over 1/720,1/120,1/24,1/6,1/2,1,1 in r; EXP = p*2^n.
  *   expert_offsets [E+1] int32: exclusive prefix sum of the per-expert slot counts, [E] = T*k.
+ * Launch order: for T <= 128 the kernel uses programmatic dependent launch.  It reads logits before it waits
+ * for the kernel launched just before it on the stream, and writes its outputs only after that kernel has
+ * completed (so the outputs of one layer call may be the buffers the previous call's moe_combine still reads).
+ * If that preceding kernel releases its dependents early (cudaTriggerProgrammaticLaunchCompletion /
+ * griddepcontrol.launch_dependents), logits must not be among its outputs; moe_combine's are not.
  * Errors: INVALID_ARG (null/misaligned, T<1, k<1, k>E), UNSUPPORTED_SHAPE (E>1024, k>32), WORKSPACE.
  */
 int moe_route(const float* logits, int32_t T, int32_t E, int32_t k, int32_t* topk_ids /* [T,k] */,

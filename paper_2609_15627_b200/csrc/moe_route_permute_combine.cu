@@ -120,7 +120,12 @@ __global__ void __launch_bounds__(1024) route_kernel(const float* __restrict__ l
   int* s_counts = reinterpret_cast<int*>(sm_f + nw * E);  // [E]
   int* s_misc = s_counts + E;                           // [32] + flag
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  pdl_launch_dependents();  // route itself is launched in plain stream order; its dependent waits before it reads
+  // Programmatic dependent launch on both sides: moe_permute may start and waits before it reads; this kernel may
+  // itself have started while the kernel before it (the previous layer call's moe_combine, which still reads the
+  // routing weights this kernel is about to overwrite) is running, so it reads only its input before it waits and
+  // writes nothing to global memory until then.
+  pdl_launch_dependents();
+  bool waited = false;
   if (single_block) {
     for (int e = tid; e < E; e += blockDim.x) s_counts[e] = 0;
     __syncthreads();
@@ -135,6 +140,10 @@ __global__ void __launch_bounds__(1024) route_kernel(const float* __restrict__ l
     float my_v;
     warp_topk(row, E, k, lane, &my_id, &my_v);
     const float wt = warp_softmax_selected(my_v, k, lane);
+    if (!waited) {
+      pdl_wait();
+      waited = true;
+    }
     if (lane < k) {
       ids[static_cast<size_t>(t) * k + lane] = my_id;
       w[static_cast<size_t>(t) * k + lane] = wt;
@@ -142,6 +151,7 @@ __global__ void __launch_bounds__(1024) route_kernel(const float* __restrict__ l
     }
     __syncwarp();
   }
+  if (!waited) pdl_wait();  // warps without a token
   if (single_block) {
     __syncthreads();
     block_offsets_scan(s_counts, E, offsets, s_misc);
@@ -172,7 +182,8 @@ int launch_route(const float* logits, int T, int E, int k, int* ids, float* w, i
   }
   int launches = 1;
   if (single) {
-    route_kernel<<<1, nw * 32, smem, st>>>(logits, T, E, k, ids, w, offsets, counters, 1);
+    if (launch_pdl(route_kernel, dim3(1), dim3(nw * 32), smem, st, logits, T, E, k, ids, w, offsets, counters, 1) != cudaSuccess)
+      return MOE_ERR_CUDA;
     note_kernel("route_topk_single_cta", launches);
   } else {
     if (cudaMemsetAsync(counters, 0, (static_cast<size_t>(E) + 1) * 4, st) != cudaSuccess) return MOE_ERR_CUDA;
@@ -347,7 +358,8 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
                                                       __nv_bfloat16* __restrict__ out) {
   const int groups = H / 8;
   const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  pdl_wait();  // the per-slot rows of the expert FFN are complete
+  pdl_wait();                // the per-slot rows of the expert FFN are complete
+  pdl_launch_dependents();   // the next call on the stream (the next layer call's router) may start its set-up
   if (idx >= static_cast<size_t>(T) * groups) return;
   const int t = static_cast<int>(idx / groups);
   const int c = static_cast<int>(idx % groups) * 8;

@@ -492,3 +492,38 @@ def test_ffn_native_fp4_path_against_oracle(T, H, I, E, k, hot, seed):
     assert moe.moe_last_kernel_name() == "ffn_native_mxf4_block_scaled"
     ry = O.expert_ffn(x_perm, off, *w, k)
     check_y(buf.y_perm.cpu().numpy(), ry, "native fp4 path")
+
+
+# ---- consecutive layer calls on one stream, sharing every buffer but the output ----
+# With programmatic dependent launch the next call's router may start while this call's combine is still
+# running; it must not overwrite the routing weights and the inverse permutation that combine reads.
+
+@pytest.mark.parametrize("T,H,I,E,k", [(4, 512, 512, 8, 2), (1, 4096, 2048, 256, 8)])
+def test_back_to_back_calls_sharing_buffers(T, H, I, E, k, prod_weights):
+    if (H, I, E) == (4096, 2048, 256):
+        wdev = prod_weights[1]
+    else:
+        wdev = tuple(dev(a) for a in inputs.make_expert_weights(H, I, E, seed=1))
+    sh = moe.shape(T, H, I, E, k)
+    buf = moe.LayerBuffers(sh)
+    n = 12
+    batches = [(dev(inputs.make_logits(T, E, 300 + i)), dev(inputs.make_x(T, H, 300 + i))) for i in range(n)]
+
+    def run(outs, sync_each):
+        for (l, x), o in zip(batches, outs):
+            moe.moe_route(l, k, buf.topk_ids, buf.topk_w, buf.expert_offsets, buf.ws)
+            moe.moe_permute(x, buf.topk_ids, buf.expert_offsets, sh, buf.x_perm, buf.perm, buf.inv_perm, buf.ws)
+            moe.moe_expert_ffn(buf.x_perm, buf.expert_offsets, *wdev, sh, buf.y_perm, buf.status, buf.ws)
+            moe.moe_combine(buf.y_perm, buf.inv_perm, buf.topk_w, sh, o)
+            if sync_each:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        assert int(buf.status.item()) == 0
+
+    ref = [torch.empty_like(buf.out) for _ in range(n)]
+    got = [torch.empty_like(buf.out) for _ in range(n)]
+    run(ref, True)
+    for rep in range(3):
+        run(got, False)
+        for i in range(n):
+            assert torch.equal(got[i].view(torch.int16), ref[i].view(torch.int16)), "call %d of a back-to-back run differs" % i
