@@ -646,8 +646,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         }
       }
     };
-    for (int round = 0; round < 2; ++round) {  // round 0 is the dry run: one pass through the one call site below
-      const bool dry = round == 0;
+    for (int sweep = 0; sweep < 2; ++sweep) {  // sweep 0 is the dry run: one pass through the one call site below
+      const bool dry = sweep == 0;
       for (int phase = 0; phase < (dry ? 1 : 2); ++phase) {
         const Phase P = phase_of(phase, a, n_touched);
         const long long it_begin = dry ? 0 : P.begin, it_end = dry ? 1 : P.end;

@@ -41,7 +41,7 @@ constexpr uint32_t kTmemCols = 512;
 constexpr int kATile = 128 * kBlockK * 2;            // 16 KB: one M=128 tile of a stage
 constexpr int kABytes = 2 * kATile;                  // 32 KB
 constexpr int kBBytes = kMaxTok * kBlockK * 2;       // 32 KB
-constexpr int kPStages = 3;                          // packed-code ring (one K block per stage)
+constexpr int kPStages = 4;                          // packed-code ring (one K block per stage)
 constexpr int kPBytes = kTileRows * (kBlockK / 2);   // 8 KB: 256 rows x 32 bytes
 
 struct UmmaArgs {
