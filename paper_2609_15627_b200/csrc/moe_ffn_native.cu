@@ -39,6 +39,8 @@
 #include <cuda.h>
 #include <cuda_fp4.h>
 
+#include <algorithm>
+
 #include "moe_sm100_primitives.cuh"
 
 namespace moe {
@@ -317,6 +319,14 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     mbar_init(act_free, 1);
     mbar_fence_init();
   }
+  // Operand rows past the term-row box are never written by TMA: zero them once, so that the tensor core multiplies
+  // zeros there instead of stale shared memory (their results are never read; zeros cost less power).
+  for (int s = 0; s < kWStages; ++s) {
+    uint4* z = reinterpret_cast<uint4*>(sW + s * kStage + kWStage + tok_pass * kTerms * 128);
+    const int n = (kAStage - tok_pass * kTerms * 128) / 16;
+    for (int i = tid; i < n; i += kNatThreads) z[i] = make_uint4(0u, 0u, 0u, 0u);
+  }
+  fence_proxy_async_smem();
   if (wid == 1) tmem_alloc(tmem_holder, kNatTmemCols);
   tc_fence_before_sync();
   __syncthreads();
@@ -736,8 +746,11 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
   uint8_t* aq1 = sf2 + align_up(S * kTerms * (sh.I / 32), kAlign);
   uint8_t* sf1 = aq1 + align_up(S * kTerms * (sh.H / 2), kAlign);
   int* done = reinterpret_cast<int*>(sf1 + align_up(S * kTerms * (sh.H / 32), kAlign));
-  // tokens per pass: the term-row box is 8 * tok_pass rows; small batches fetch less
-  const int tok_pass = S <= 4 ? 4 : (S <= 8 ? 8 : kMaxTokPass);
+  // tokens per pass: the term-row box is 8 * tok_pass rows.  An expert has at most T rows and on average S / E:
+  // four times the average covers nearly every expert in one pass, and a smaller box fetches fewer foreign rows
+  // (the rare expert with more rows takes another pass over its weights).
+  const size_t want = std::min(static_cast<size_t>(sh.T), 4 * ((S + sh.E - 1) / sh.E));
+  const int tok_pass = want <= 4 ? 4 : (want <= 8 ? 8 : kMaxTokPass);
   CUtensorMap tm_w13, tm_w2, tm_s13, tm_s2, tm_a1, tm_a2;
   if (!nat_map(&tm_a1, aq1, sh.H / 2, S * kTerms, 128, static_cast<uint32_t>(tok_pass * kTerms), CU_TENSOR_MAP_SWIZZLE_128B) ||
       !nat_map(&tm_a2, aq2, sh.I / 2, S * kTerms, 128, static_cast<uint32_t>(tok_pass * kTerms), CU_TENSOR_MAP_SWIZZLE_128B))
