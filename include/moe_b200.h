@@ -70,6 +70,13 @@ const char* moe_last_kernel_name(void);
 /* Host.  Number of kernels launched (memset nodes not counted) by this thread's moe_* calls so far. */
 uint64_t moe_launch_count(void);
 
+/* Host, pure, diagnostic.  Work split of the decode-sized expert-FFN kernel: which items (touched expert x tile of
+ * 256 weight rows, in expert order) CTA `cta` of `n_ctas` takes when `n_touched` experts have rows.  out4 = first
+ * and one-past-last gate/up item, first and one-past-last down item.  A down item waits, on the device, for all
+ * gate/up items of its expert; the split keeps those in CTAs with a lower or equal index.  INVALID_ARG on
+ * nonsense (cta outside [0, n_ctas), n_touched outside [0, 1024], H or 2I not a multiple of 256). */
+int moe_debug_native_cta_share(int32_t n_ctas, int32_t cta, int32_t n_touched, int32_t H, int32_t I, int32_t* out4);
+
 /*
  * Router Top-k (paper: "Router Top-k"; fixed Top-K membership and order is a stated requirement).
  *   logits [T,E] fp32 (finite).  For each token the k largest logits are selected, slot 0 the

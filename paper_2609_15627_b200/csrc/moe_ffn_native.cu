@@ -25,8 +25,8 @@
 // one i are two columns of the same accumulator lane), phase 1 = down (item = touched expert x 256 rows).  The weight
 // stream runs on across the phase change; a down item loads its term rows once the gate/up items of its expert - its
 // own and other CTAs' - have published theirs (one counter per expert, release/acquire through L2, bounded wait).
-// All CTAs of the grid are resident (grid = number of SMs, one CTA each) and no gate/up item ever waits for another
-// CTA, so the waits cannot form a cycle.
+// No gate/up item ever waits for another CTA, and a down item waits only for gate/up items of CTAs with a lower or
+// equal index (see phase_of), so the waits cannot form a cycle and do not need the whole grid to be resident.
 // Warp roles:
 //   warp 0      producer: TMA loads of the weight tile, of the term rows and of the weight scale bytes
 //   warp 1      allocates tensor memory, issues the MMAs, commits to mbarriers
@@ -84,16 +84,45 @@ struct Phase {
   int K, R, n_steps, tiles;  // reduction length, weight rows per expert, K steps, items per expert
   long long begin, end;      // this CTA's items
 };
-MOE_DEVINL Phase phase_of(int ph, const NatArgs& a, int n_touched) {
+// Items go to CTAs in contiguous shares: gate/up items evenly, per0 each.  A down item of expert t is placed as if it
+// followed that expert's last gate/up item in the gate/up list, its expert's down items spread over the span of the
+// next expert's gate/up items: with t = i1 / tiles1 and j = i1 % tiles1,
+//   u(i1) = (t + 1) * tiles0 - 1 + ceil((j + 1) * tiles0 / tiles1),   CTA(i1) = min(grid - 1, u(i1) / per0).
+// So a down item only ever waits for gate/up items of CTAs with a lower or equal index: CTAs are handed out in index
+// order, hence whatever a running CTA waits for has been started before it, whether or not the whole grid is
+// resident at once.  The shares stay within one expert's items of even.
+//
+// The smallest down item (of total1) that reaches CTA c, i.e. with u(i1) >= c * per0
+__host__ __device__ inline int first_down_item_of_cta(int c, int total1, int tiles0, int tiles1, int per0) {
+  const int U = c * per0;
+  int t = (U + tiles0) / tiles0 - 2;
+  if (t < 0) t = 0;
+  const int V = U - (t + 1) * tiles0 + 1;  // need ceil((j + 1) * tiles0 / tiles1) >= V
+  int j = V <= 1 ? 0 : ((V - 1) * tiles1) / tiles0;
+  if (j >= tiles1) {
+    t += 1;
+    j = 0;
+  }
+  const int i1 = t * tiles1 + j;
+  return i1 < total1 ? i1 : total1;
+}
+// CTA c's share of either phase (item counts fit 32 bits: at most 1024 experts x 32 tiles): begin0, end0, begin1, end1
+__host__ __device__ inline void cta_shares(int grid, int c, int n_touched, int tiles0, int tiles1, int* out) {
+  const int total0 = n_touched * tiles0, total1 = n_touched * tiles1;
+  const int per0 = (total0 + grid - 1) / grid;
+  out[0] = c * per0 < total0 ? c * per0 : total0;
+  out[1] = out[0] + per0 < total0 ? out[0] + per0 : total0;
+  out[2] = total1 == 0 ? 0 : first_down_item_of_cta(c, total1, tiles0, tiles1, per0);
+  out[3] = total1 == 0 ? 0 : (c + 1 >= grid ? total1 : first_down_item_of_cta(c + 1, total1, tiles0, tiles1, per0));
+}
+MOE_DEVINL Phase phase_of(int ph, const NatArgs& a, const int* shares) {
   Phase p;
   p.K = ph == 0 ? a.H : a.I;
   p.R = ph == 0 ? 2 * a.I : a.H;
   p.n_steps = p.K / kKStep;
   p.tiles = p.R / kTile;
-  const long long total = static_cast<long long>(n_touched) * p.tiles;
-  const long long per_cta = (total + gridDim.x - 1) / gridDim.x;
-  p.begin = min(static_cast<long long>(blockIdx.x) * per_cta, total);
-  p.end = min(p.begin + per_cta, total);
+  p.begin = shares[2 * ph];
+  p.end = shares[2 * ph + 1];
   return p;
 }
 
@@ -307,7 +336,10 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       }
       run += tot;
     }
-    if (lane == 0) s_misc[0] = run;
+    if (lane == 0) {
+      s_misc[0] = run;
+      cta_shares(static_cast<int>(gridDim.x), static_cast<int>(blockIdx.x), run, 2 * a.I / kTile, a.H / kTile, s_misc + 1);
+    }
   }
   if (tid == 0) {
     for (int s = 0; s < kWStages; ++s) { mbar_init(&full_w[s], 1); mbar_init(&empty_w[s], 1); }
@@ -336,7 +368,6 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   // (griddepcontrol.wait) for this grid to complete before it reads the output.  This grid in turn reads nothing
   // of the split kernel before it has waited itself, apart from expert_offsets (see above).
   pdl_launch_dependents();
-  const int n_touched = s_misc[0];
   // Every role walks the same sequence: both phases; in each, this CTA's items; per item, passes of up to tok_pass
   // tokens; per pass, all K steps.
 
@@ -367,7 +398,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         dep_ok = true;
       };
       for (int phase = 0; phase < 2; ++phase) {
-        const Phase P = phase_of(phase, a, n_touched);
+        const Phase P = phase_of(phase, a, s_misc + 1);
         const CUtensorMap* mw = phase == 0 ? &tmap_w13 : &tmap_w2;
         const CUtensorMap* msc = phase == 0 ? &tmap_s13 : &tmap_s2;
         const CUtensorMap* ma = phase == 0 ? &tmap_a1 : &tmap_a2;
@@ -421,7 +452,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       uint32_t ph = 0, sph = 0, aph = 0, acc_ph = 0;
       const uint32_t d_addr = tmem_base + kColD;
       for (int phase = 0; phase < 2; ++phase) {
-        const Phase P = phase_of(phase, a, n_touched);
+        const Phase P = phase_of(phase, a, s_misc + 1);
         int prev_ti = -1;
         for (long long it = P.begin; it < P.end; ++it) {
           const int ti = static_cast<int>(it / P.tiles);
@@ -475,7 +506,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     uint32_t cph = 0, sfree_ph = 0, afree_ph = 0;
     bool first_op = true;
     for (int phase = 0; phase < 2; ++phase) {
-      const Phase P = phase_of(phase, a, n_touched);
+      const Phase P = phase_of(phase, a, s_misc + 1);
       const int n_blk = P.K / 32;
       const uint8_t* src_sf = phase == 0 ? a.sf1 : a.sf2;
       int prev_ti = -1;
@@ -659,7 +690,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     for (int sweep = 0; sweep < 2; ++sweep) {  // sweep 0 is the dry run: one pass through the one call site below
       const bool dry = sweep == 0;
       for (int phase = 0; phase < (dry ? 1 : 2); ++phase) {
-        const Phase P = phase_of(phase, a, n_touched);
+        const Phase P = phase_of(phase, a, s_misc + 1);
         const long long it_begin = dry ? 0 : P.begin, it_end = dry ? 1 : P.end;
         for (long long it = it_begin; it < it_end; ++it) {
           const int ti = static_cast<int>(it / P.tiles), tile = static_cast<int>(it % P.tiles);
@@ -785,3 +816,11 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
 }
 
 }  // namespace moe
+
+extern "C" int moe_debug_native_cta_share(int32_t n_ctas, int32_t cta, int32_t n_touched, int32_t H, int32_t I, int32_t* out4) {
+  if (out4 == nullptr || n_ctas < 1 || cta < 0 || cta >= n_ctas || n_touched < 0 || n_touched > 1024 || H < moe::kTile ||
+      I < moe::kTile / 2 || H % moe::kTile != 0 || (2 * I) % moe::kTile != 0)
+    return MOE_ERR_INVALID_ARG;
+  moe::cta_shares(n_ctas, cta, n_touched, 2 * I / moe::kTile, H / moe::kTile, out4);
+  return MOE_OK;
+}

@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libmoe_b200.so")
 EXPORTS = ("moe_workspace_bytes", "moe_status_string", "moe_last_kernel_name", "moe_launch_count", "moe_route",
            "moe_permute", "moe_expert_ffn", "moe_combine", "moe_validate_scales",
            "moe_forward_host_workspace_bytes", "moe_forward_host", "moe_expert_ffn_noalloc_max_bytes",
-           "moe_expert_ffn_noalloc")
+           "moe_expert_ffn_noalloc", "moe_debug_native_cta_share")
 
 
 class MoeError(RuntimeError):
@@ -58,6 +58,8 @@ def lib():
         L.moe_expert_ffn_noalloc_max_bytes.restype = sz
         L.moe_expert_ffn_noalloc.restype = C.c_int
         L.moe_expert_ffn_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp]
+        L.moe_debug_native_cta_share.restype = C.c_int
+        L.moe_debug_native_cta_share.argtypes = [i32, i32, i32, i32, i32, C.POINTER(C.c_int32)]
         L.moe_forward_host.restype = C.c_int
         L.moe_forward_host.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp, sz, vp]
         _lib = L
@@ -132,6 +134,13 @@ def moe_expert_ffn_noalloc(x_perm, expert_offsets, w13, w13_scale, w2, w2_scale,
     _check(lib().moe_expert_ffn_noalloc(_ptr(x_perm), _ptr(expert_offsets), _ptr(w13), _ptr(w13_scale), _ptr(w2),
                                         _ptr(w2_scale), C.byref(sh), _ptr(y_perm), _ptr(status_word), _stream(stream)),
            "moe_expert_ffn_noalloc")
+
+
+def moe_debug_native_cta_share(n_ctas, cta, n_touched, H, I):
+    """(first, end) gate/up items and (first, end) down items of one CTA of the decode-sized expert-FFN kernel."""
+    out = (C.c_int32 * 4)()
+    _check(lib().moe_debug_native_cta_share(n_ctas, cta, n_touched, H, I, out), "moe_debug_native_cta_share")
+    return tuple(out)
 
 
 def moe_combine(y_perm, inv_perm, topk_w, sh, out, stream=None):

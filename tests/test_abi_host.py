@@ -67,3 +67,37 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(moe, "LIB_PATH", "/nonexistent/libmoe_b200.so")
     with pytest.raises(moe.MoeError):
         moe.lib()
+
+
+def test_decode_ffn_work_split_keeps_waits_pointing_down(L):
+    """The decode-sized expert-FFN kernel runs both projections in one grid: a down item waits on the device for the
+    gate/up items of its expert.  The split must cover every item exactly once, and every gate/up item an expert's
+    down items wait for must belong to a CTA with a lower or equal index than theirs (CTAs start in index order, so
+    such a wait can always end), with shares close to even."""
+    n_ctas = 148
+    for (H, I) in [(4096, 2048), (512, 512), (1024, 512), (512, 1024), (4096, 4096), (512, 4096)]:
+        tiles0, tiles1 = 2 * I // 256, H // 256
+        for n_touched in [0, 1, 2, 3, 7, 8, 9, 37, 74, 147, 148, 149, 224, 256, 1024]:
+            shares = [moe.moe_debug_native_cta_share(n_ctas, c, n_touched, H, I) for c in range(n_ctas)]
+            for ph, tiles in ((0, tiles0), (1, tiles1)):
+                pos = 0
+                for sh in shares:
+                    b, e = sh[2 * ph], sh[2 * ph + 1]
+                    assert b == min(pos, n_touched * tiles) or b == pos, (H, I, n_touched, ph, sh, pos)
+                    assert e >= b
+                    pos = e
+                assert pos == n_touched * tiles
+            owner0 = {}
+            for c, sh in enumerate(shares):
+                for it in range(sh[0], sh[1]):
+                    owner0[it] = c
+            for c, sh in enumerate(shares):
+                for it in range(sh[2], sh[3]):
+                    t = it // tiles1
+                    assert max(owner0[g] for g in range(t * tiles0, (t + 1) * tiles0)) <= c, (H, I, n_touched, c, it)
+            if n_touched:
+                even1 = -(-n_touched * tiles1 // n_ctas)
+                assert max(sh[3] - sh[2] for sh in shares) <= even1 + tiles1
+    out = (C.c_int32 * 4)()
+    assert L.moe_debug_native_cta_share(148, 148, 8, 4096, 2048, out) == 1
+    assert L.moe_debug_native_cta_share(148, 0, 8, 4096, 100, out) == 1
