@@ -26,7 +26,7 @@
 // stream runs on across the phase change; a down item loads its term rows once the gate/up items of its expert - its
 // own and other CTAs' - have published theirs (one counter per expert, release/acquire through L2, bounded wait).
 // No gate/up item ever waits for another CTA, and a down item waits only for gate/up items of CTAs with a lower or
-// equal index (see phase_of), so the waits cannot form a cycle and do not need the whole grid to be resident.
+// equal index (see cta_shares), so the waits cannot form a cycle and do not need the whole grid to be resident.
 // Warp roles:
 //   warp 0      producer: TMA loads of the weight tile, of the term rows and of the weight scale bytes
 //   warp 1      allocates tensor memory, issues the MMAs, commits to mbarriers
