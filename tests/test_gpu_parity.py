@@ -347,9 +347,16 @@ def _sample_tokens(wl, ids, off, n):
     return np.array(sorted(pick)[:max(n, len(pick))], np.int32)
 
 
-@pytest.mark.parametrize("name,n_tokens", [("prefill_8k", 24), ("prefill_32k_skewed", 24)])
+# decode_c256 / decode_c512: not benchmark workloads; the largest batches the decode-sized expert-FFN kernel takes at the
+# production shape (8 and 16 rows per expert on average: passes of 16 tokens, some experts with two passes)
+_EXTRA = {"decode_c256": inputs.Workload("decode_c256", 256, 4096, 2048, 256, 8),
+          "decode_c512": inputs.Workload("decode_c512", 512, 4096, 2048, 256, 8)}
+
+
+@pytest.mark.parametrize("name,n_tokens", [("prefill_8k", 24), ("prefill_32k_skewed", 24), ("decode_c256", 16),
+                                           ("decode_c512", 16)])
 def test_layer_prefill_sampled(name, n_tokens, prod_weights):
-    wl = inputs.WORKLOADS[name]
+    wl = inputs.WORKLOADS[name] if name in inputs.WORKLOADS else _EXTRA[name]
     (w13, s13, w2, s2), wdev = prod_weights
     logits = inputs.make_logits(wl.T, wl.E, 0, wl.skew)
     x = inputs.make_x(wl.T, wl.H, 0)
@@ -363,8 +370,9 @@ def test_layer_prefill_sampled(name, n_tokens, prod_weights):
     _, rperm, rinv = O.permute(x, rids, roff)
     assert np.array_equal(buf.perm.cpu().numpy(), rperm)
     assert np.array_equal(buf.inv_perm.cpu().numpy(), rinv)
-    xp = bits(buf.x_perm[:4096]), bits(buf.x_perm[-4096:])
-    assert np.array_equal(xp[0], x[rperm[:4096] // wl.k]) and np.array_equal(xp[1], x[rperm[-4096:] // wl.k])
+    nx = min(4096, wl.T * wl.k)
+    xp = bits(buf.x_perm[:nx]), bits(buf.x_perm[-nx:])
+    assert np.array_equal(xp[0], x[rperm[:nx] // wl.k]) and np.array_equal(xp[1], x[rperm[-nx:] // wl.k])
     # FFN + combine on sampled tokens by the per-token definition
     tokens = _sample_tokens(wl, rids, roff, n_tokens)
     r = O.forward_tokens(logits, x, w13, s13, w2, s2, wl.k, tokens)
