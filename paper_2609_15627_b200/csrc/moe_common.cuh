@@ -23,7 +23,7 @@ constexpr size_t kAlign = 256;
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// native block-scaled FP4 variant (decode-sized batches): on average at most 32 rows per expert (8 passes of 4
+// native block-scaled FP4 variant (decode-sized batches): on average at most 32 rows per expert (2 passes of 16
 // tokens over the weight stream).  Its scratch holds the E2M1 term rows (8 per row) of both projections' inputs:
 // [8S, I/2] + [8S, I/32] scale bytes and [8S, H/2] + [8S, H/32]; and one completion counter per expert.
 inline bool native_batch_ok(const moe_shape_t& s) {

@@ -76,8 +76,14 @@ struct NatArgs {
   float* y;                  // output [S, H]
   int* status;
   int E, H, I, S;
-  int tok_pass;              // tokens per pass: 4, 8 or 16 (the row count of the term-row TMA box / 8)
 };
+
+// Term-row tensor maps of one projection's input: the same tensor with boxes of 32, 64 and 128 rows (4, 8, 16 tokens);
+// a pass fetches the smallest box that holds its tokens
+struct alignas(64) TermMaps {
+  CUtensorMap box[3];
+};
+MOE_DEVINL int term_box(int n_tok) { return n_tok <= 4 ? 0 : (n_tok <= 8 ? 1 : 2); }
 
 // One projection as the kernel sees it
 struct Phase {
@@ -273,8 +279,8 @@ __global__ void __launch_bounds__(1024) native_split_kernel(const __nv_bfloat16*
 
 __global__ void __launch_bounds__(kNatThreads, 1)
 ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_constant__ CUtensorMap tmap_s13,
-                  const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_w2,
-                  const __grid_constant__ CUtensorMap tmap_s2, const __grid_constant__ CUtensorMap tmap_a2, const NatArgs a) {
+                  const __grid_constant__ TermMaps tmap_a1, const __grid_constant__ CUtensorMap tmap_w2,
+                  const __grid_constant__ CUtensorMap tmap_s2, const __grid_constant__ TermMaps tmap_a2, const NatArgs a) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   const NatSmem sm = nat_smem(a.E, a.H > a.I ? a.H : a.I);
@@ -299,17 +305,19 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   int* s_misc = t_end + a.E;
 
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  const int tok_pass = a.tok_pass;
+  constexpr int tok_pass = kMaxTokPass;
   const int need_done = 4 * (2 * a.I / kTile);  // four epilogue warps publish each gate/up item of an expert
 
   // ---- setup: touched experts, barriers, tensor memory ----
   if (tid == 32 * 3) {  // a warp with nothing to set up fetches the tensor maps
     prefetch_tmap(&tmap_w13);
     prefetch_tmap(&tmap_s13);
-    prefetch_tmap(&tmap_a1);
     prefetch_tmap(&tmap_w2);
     prefetch_tmap(&tmap_s2);
-    prefetch_tmap(&tmap_a2);
+    for (int i = 0; i < 3; ++i) {
+      prefetch_tmap(&tmap_a1.box[i]);
+      prefetch_tmap(&tmap_a2.box[i]);
+    }
   }
   if (wid == 2) {
     // lane l looks at experts l, l + 32, ...: all loads are issued before any is used (one memory round trip);
@@ -351,12 +359,11 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     mbar_init(act_free, 1);
     mbar_fence_init();
   }
-  // Operand rows past the term-row box are never written by TMA: zero them once, so that the tensor core multiplies
-  // zeros there instead of stale shared memory (their results are never read; zeros cost less power).
+  // Operand rows that no term-row box has written yet read as zeros instead of whatever shared memory held (their
+  // results are never looked at; zeros cost less power)
   for (int s = 0; s < kWStages; ++s) {
-    uint4* z = reinterpret_cast<uint4*>(sW + s * kStage + kWStage + tok_pass * kTerms * 128);
-    const int n = (kAStage - tok_pass * kTerms * 128) / 16;
-    for (int i = tid; i < n; i += kNatThreads) z[i] = make_uint4(0u, 0u, 0u, 0u);
+    uint4* z = reinterpret_cast<uint4*>(sW + s * kStage + kWStage);
+    for (int i = tid; i < kAStage / 16; i += kNatThreads) z[i] = make_uint4(0u, 0u, 0u, 0u);
   }
   fence_proxy_async_smem();
   if (wid == 1) tmem_alloc(tmem_holder, kNatTmemCols);
@@ -381,7 +388,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       // kWStages steps are held back; they follow once the dependency is met.
       bool pdl_done = false, dep_ok = false;
       int dep_phase = 0, dep_e = -1;
-      int n_pend = 0, pend_s[kWStages], pend_x[kWStages], pend_y[kWStages];
+      int n_pend = 0, pend_s[kWStages], pend_x[kWStages], pend_y[kWStages], pend_b[kWStages];
       auto meet = [&]() {  // wait for the open dependency and send the held-back loads
         if (!pdl_done) {
           pdl_wait();  // the split kernel is complete: term rows of the tokens, cleared counters
@@ -391,9 +398,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
           counter_wait_ge(a.done + dep_e, need_done, a.status);
           fence_proxy_async_all();  // the rows were written through the generic proxy, TMA reads through the async one
         }
-        const CUtensorMap* ma = dep_phase == 0 ? &tmap_a1 : &tmap_a2;
+        const TermMaps* ma = dep_phase == 0 ? &tmap_a1 : &tmap_a2;
         for (int i = 0; i < n_pend; ++i)
-          tma_load_2d(sW + pend_s[i] * kStage + kWStage, ma, pend_x[i], pend_y[i], &full_w[pend_s[i]]);
+          tma_load_2d(sW + pend_s[i] * kStage + kWStage, &ma->box[pend_b[i]], pend_x[i], pend_y[i], &full_w[pend_s[i]]);
         n_pend = 0;
         dep_ok = true;
       };
@@ -401,12 +408,13 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         const Phase P = phase_of(phase, a, s_misc + 1);
         const CUtensorMap* mw = phase == 0 ? &tmap_w13 : &tmap_w2;
         const CUtensorMap* msc = phase == 0 ? &tmap_s13 : &tmap_s2;
-        const CUtensorMap* ma = phase == 0 ? &tmap_a1 : &tmap_a2;
+        const TermMaps* ma = phase == 0 ? &tmap_a1 : &tmap_a2;
         for (long long it = P.begin; it < P.end; ++it) {
           const int ti = static_cast<int>(it / P.tiles), e = touched[ti];
           const int tile = static_cast<int>(it % P.tiles);
           const int row_begin = t_begin[ti];
-          const int n_pass = (t_end[ti] - row_begin + tok_pass - 1) / tok_pass;
+          const int n_rows_e = t_end[ti] - row_begin;
+          const int n_pass = (n_rows_e + tok_pass - 1) / tok_pass;
           const int wrow_a = phase == 0 ? e * P.R + tile * 128 : e * P.R + tile * kTile;
           const int wrow_b = phase == 0 ? e * P.R + a.I + tile * 128 : wrow_a + 128;
           if (phase == 1 && (dep_phase != 1 || dep_e != e)) {  // a new dependency: settle the old one first
@@ -416,6 +424,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             dep_ok = false;
           }
           for (int pass = 0; pass < n_pass; ++pass) {
+            const int bi = term_box(min(tok_pass, n_rows_e - pass * tok_pass));  // 32, 64 or 128 term rows
             for (int ks = 0; ks < P.n_steps; ++ks) {
               if ((ks & 1) == 0) {  // 16 scale bytes per weight row cover two K steps
                 mbar_wait(&empty_sc[cs], cph ^ 1u, a.status);
@@ -425,17 +434,18 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
                 if (++cs == kScStages) { cs = 0; cph ^= 1u; }
               }
               mbar_wait(&empty_w[s], ph ^ 1u, a.status);
-              mbar_expect_tx(&full_w[s], static_cast<uint32_t>(kWStage + tok_pass * kTerms * 128));
+              mbar_expect_tx(&full_w[s], static_cast<uint32_t>(kWStage + (32 << bi) * 128));
               tma_load_2d(sW + s * kStage, mw, ks * 128, wrow_a, &full_w[s]);
               tma_load_2d(sW + s * kStage + 128 * 128, mw, ks * 128, wrow_b, &full_w[s]);
               // the pass's term rows (8 per token, consecutive); rows past the end of the tensor arrive as zeros
               const int arow = (row_begin + pass * tok_pass) * kTerms;
               if (dep_ok) {
-                tma_load_2d(sW + s * kStage + kWStage, ma, ks * 128, arow, &full_w[s]);
+                tma_load_2d(sW + s * kStage + kWStage, &ma->box[bi], ks * 128, arow, &full_w[s]);
               } else {
                 pend_s[n_pend] = s;
                 pend_x[n_pend] = ks * 128;
                 pend_y[n_pend] = arow;
+                pend_b[n_pend] = bi;
                 if (++n_pend == kWStages) meet();
               }
               if (++s == kWStages) { s = 0; ph ^= 1u; }
@@ -777,15 +787,12 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
   uint8_t* aq1 = sf2 + align_up(S * kTerms * (sh.I / 32), kAlign);
   uint8_t* sf1 = aq1 + align_up(S * kTerms * (sh.H / 2), kAlign);
   int* done = reinterpret_cast<int*>(sf1 + align_up(S * kTerms * (sh.H / 32), kAlign));
-  // tokens per pass: the term-row box is 8 * tok_pass rows.  An expert has at most T rows and on average S / E:
-  // four times the average covers nearly every expert in one pass, and a smaller box fetches fewer foreign rows
-  // (the rare expert with more rows takes another pass over its weights).
-  const size_t want = std::min(static_cast<size_t>(sh.T), 4 * ((S + sh.E - 1) / sh.E));
-  const int tok_pass = want <= 4 ? 4 : (want <= 8 ? 8 : kMaxTokPass);
-  CUtensorMap tm_w13, tm_w2, tm_s13, tm_s2, tm_a1, tm_a2;
-  if (!nat_map(&tm_a1, aq1, sh.H / 2, S * kTerms, 128, static_cast<uint32_t>(tok_pass * kTerms), CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !nat_map(&tm_a2, aq2, sh.I / 2, S * kTerms, 128, static_cast<uint32_t>(tok_pass * kTerms), CU_TENSOR_MAP_SWIZZLE_128B))
-    return MOE_ERR_CUDA;
+  CUtensorMap tm_w13, tm_w2, tm_s13, tm_s2;
+  TermMaps tm_a1, tm_a2;
+  for (int i = 0; i < 3; ++i)
+    if (!nat_map(&tm_a1.box[i], aq1, sh.H / 2, S * kTerms, 128, 32u << i, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !nat_map(&tm_a2.box[i], aq2, sh.I / 2, S * kTerms, 128, 32u << i, CU_TENSOR_MAP_SWIZZLE_128B))
+      return MOE_ERR_CUDA;
   if (!nat_map(&tm_w13, w13, sh.H / 2, static_cast<uint64_t>(sh.E) * 2 * sh.I, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !nat_map(&tm_w2, w2, sh.I / 2, static_cast<uint64_t>(sh.E) * sh.H, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !nat_map(&tm_s13, s13, sh.H / 32, static_cast<uint64_t>(sh.E) * 2 * sh.I, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE) ||
@@ -807,7 +814,6 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
   a.H = sh.H;
   a.I = sh.I;
   a.S = static_cast<int>(S);
-  a.tok_pass = tok_pass;
   if (launch_pdl(ffn_native_kernel, dim3(sm_count()), dim3(kNatThreads), nat_smem(sh.E, sh.H > sh.I ? sh.H : sh.I).total + 1024,
                  st, tm_w13, tm_s13, tm_a1, tm_w2, tm_s2, tm_a2, a) != cudaSuccess)
     return MOE_ERR_CUDA;
