@@ -78,12 +78,14 @@ struct NatArgs {
   int E, H, I, S;
 };
 
-// Term-row tensor maps of one projection's input: the same tensor with boxes of 32, 64 and 128 rows (4, 8, 16 tokens);
-// a pass fetches the smallest box that holds its tokens
+// Term-row tensor maps of one projection's input: the same tensor with boxes of 8, 16, 32, 64 and 128 rows (1, 2, 4, 8,
+// 16 tokens); a pass fetches the smallest box that holds its tokens - every byte of term rows competes with the weights
+// for the path from L2
+constexpr int kTermBoxes = 5;
 struct alignas(64) TermMaps {
-  CUtensorMap box[3];
+  CUtensorMap box[kTermBoxes];
 };
-MOE_DEVINL int term_box(int n_tok) { return n_tok <= 4 ? 0 : (n_tok <= 8 ? 1 : 2); }
+MOE_DEVINL int term_box(int n_tok) { return n_tok <= 1 ? 0 : (n_tok <= 2 ? 1 : (n_tok <= 4 ? 2 : (n_tok <= 8 ? 3 : 4))); }
 
 // One projection as the kernel sees it
 struct Phase {
@@ -314,7 +316,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     prefetch_tmap(&tmap_s13);
     prefetch_tmap(&tmap_w2);
     prefetch_tmap(&tmap_s2);
-    for (int i = 0; i < 3; ++i) {
+    for (int i = 0; i < kTermBoxes; ++i) {
       prefetch_tmap(&tmap_a1.box[i]);
       prefetch_tmap(&tmap_a2.box[i]);
     }
@@ -424,7 +426,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             dep_ok = false;
           }
           for (int pass = 0; pass < n_pass; ++pass) {
-            const int bi = term_box(min(tok_pass, n_rows_e - pass * tok_pass));  // 32, 64 or 128 term rows
+            const int bi = term_box(min(tok_pass, n_rows_e - pass * tok_pass));  // box of 8 << bi term rows
             for (int ks = 0; ks < P.n_steps; ++ks) {
               if ((ks & 1) == 0) {  // 16 scale bytes per weight row cover two K steps
                 mbar_wait(&empty_sc[cs], cph ^ 1u, a.status);
@@ -434,7 +436,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
                 if (++cs == kScStages) { cs = 0; cph ^= 1u; }
               }
               mbar_wait(&empty_w[s], ph ^ 1u, a.status);
-              mbar_expect_tx(&full_w[s], static_cast<uint32_t>(kWStage + (32 << bi) * 128));
+              mbar_expect_tx(&full_w[s], static_cast<uint32_t>(kWStage + (8 << bi) * 128));
               tma_load_2d(sW + s * kStage, mw, ks * 128, wrow_a, &full_w[s]);
               tma_load_2d(sW + s * kStage + 128 * 128, mw, ks * 128, wrow_b, &full_w[s]);
               // the pass's term rows (8 per token, consecutive); rows past the end of the tensor arrive as zeros
@@ -789,9 +791,9 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
   int* done = reinterpret_cast<int*>(sf1 + align_up(S * kTerms * (sh.H / 32), kAlign));
   CUtensorMap tm_w13, tm_w2, tm_s13, tm_s2;
   TermMaps tm_a1, tm_a2;
-  for (int i = 0; i < 3; ++i)
-    if (!nat_map(&tm_a1.box[i], aq1, sh.H / 2, S * kTerms, 128, 32u << i, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !nat_map(&tm_a2.box[i], aq2, sh.I / 2, S * kTerms, 128, 32u << i, CU_TENSOR_MAP_SWIZZLE_128B))
+  for (int i = 0; i < kTermBoxes; ++i)
+    if (!nat_map(&tm_a1.box[i], aq1, sh.H / 2, S * kTerms, 128, 8u << i, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !nat_map(&tm_a2.box[i], aq2, sh.I / 2, S * kTerms, 128, 8u << i, CU_TENSOR_MAP_SWIZZLE_128B))
       return MOE_ERR_CUDA;
   if (!nat_map(&tm_w13, w13, sh.H / 2, static_cast<uint64_t>(sh.E) * 2 * sh.I, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !nat_map(&tm_w2, w2, sh.I / 2, static_cast<uint64_t>(sh.E) * sh.H, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||

@@ -468,7 +468,7 @@ def test_kernel_choice_is_a_function_of_the_shape():
 # ---- the native block-scaled FP4 expert FFN, reached when T*k <= 32*E (decode-sized) and H, I are multiples of 512 ----
 
 @pytest.mark.parametrize("T,H,I,E,k,hot,seed", [
-    (16, 512, 512, 8, 2, False, 0),      # a few rows per expert: term-row boxes of 32 and 64 rows
+    (16, 512, 512, 8, 2, False, 0),      # a few rows per expert: term-row boxes of 16 to 64 rows
     (1, 512, 512, 16, 4, False, 1),      # one token: every expert has at most one row
     (8, 512, 512, 8, 2, False, 4),       # two rows per expert on average
     (64, 1024, 512, 8, 2, False, 2),     # ~16 rows per expert: 128-row boxes, some experts need two passes of 16 tokens
