@@ -85,6 +85,10 @@ constexpr int kTermBoxes = 5;
 struct alignas(64) TermMaps {
   CUtensorMap box[kTermBoxes];
 };
+// A pass of at most kRepTok tokens fills one lane quadrant of the accumulator (32 operand rows).  Its term rows are
+// then loaded once per quadrant, so that each of the four epilogue warps finds every token in its own quadrant and
+// takes a quarter of the columns instead of one warp taking them all.
+constexpr int kRepTok = 4, kRepBox = 2;  // boxes 0..kRepBox hold at most kRepTok tokens
 MOE_DEVINL int term_box(int n_tok) { return n_tok <= 1 ? 0 : (n_tok <= 2 ? 1 : (n_tok <= 4 ? 2 : (n_tok <= 8 ? 3 : 4))); }
 
 // One projection as the kernel sees it
@@ -391,6 +395,12 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       bool pdl_done = false, dep_ok = false;
       int dep_phase = 0, dep_e = -1;
       int n_pend = 0, pend_s[kWStages], pend_x[kWStages], pend_y[kWStages], pend_b[kWStages];
+      // term rows of one K step; a pass of at most kRepTok tokens gets them once per lane quadrant of the accumulator
+      auto load_terms = [&](const TermMaps* ma, int stage, int bi, int x, int y) {
+        const int n_rep = bi <= kRepBox ? 4 : 1;
+        for (int r = 0; r < n_rep; ++r)
+          tma_load_2d(sW + stage * kStage + kWStage + r * (32 * 128), &ma->box[bi], x, y, &full_w[stage]);
+      };
       auto meet = [&]() {  // wait for the open dependency and send the held-back loads
         if (!pdl_done) {
           pdl_wait();  // the split kernel is complete: term rows of the tokens, cleared counters
@@ -401,8 +411,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
           fence_proxy_async_all();  // the rows were written through the generic proxy, TMA reads through the async one
         }
         const TermMaps* ma = dep_phase == 0 ? &tmap_a1 : &tmap_a2;
-        for (int i = 0; i < n_pend; ++i)
-          tma_load_2d(sW + pend_s[i] * kStage + kWStage, &ma->box[pend_b[i]], pend_x[i], pend_y[i], &full_w[pend_s[i]]);
+        for (int i = 0; i < n_pend; ++i) load_terms(ma, pend_s[i], pend_b[i], pend_x[i], pend_y[i]);
         n_pend = 0;
         dep_ok = true;
       };
@@ -436,13 +445,13 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
                 if (++cs == kScStages) { cs = 0; cph ^= 1u; }
               }
               mbar_wait(&empty_w[s], ph ^ 1u, a.status);
-              mbar_expect_tx(&full_w[s], static_cast<uint32_t>(kWStage + (8 << bi) * 128));
+              mbar_expect_tx(&full_w[s], static_cast<uint32_t>(kWStage + (bi <= kRepBox ? 4 : 1) * (8 << bi) * 128));
               tma_load_2d(sW + s * kStage, mw, ks * 128, wrow_a, &full_w[s]);
               tma_load_2d(sW + s * kStage + 128 * 128, mw, ks * 128, wrow_b, &full_w[s]);
               // the pass's term rows (8 per token, consecutive); rows past the end of the tensor arrive as zeros
               const int arow = (row_begin + pass * tok_pass) * kTerms;
               if (dep_ok) {
-                tma_load_2d(sW + s * kStage + kWStage, &ma->box[bi], ks * 128, arow, &full_w[s]);
+                load_terms(ma, s, bi, ks * 128, arow);
               } else {
                 pend_s[n_pend] = s;
                 pend_x[n_pend] = ks * 128;
@@ -545,6 +554,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             }
             const int row0 = row_begin + pass * tok_pass;
             const int n_rows = min(tok_pass, row_end - row0) * kTerms;  // term rows that exist
+            const bool rep = n_rows <= kRepTok * kTerms;                // the operand repeats in every lane quadrant
             // rows are n_blk bytes each and consecutive: one contiguous range, copied 16 bytes at a time
             // (the 16-byte chunks of a row are XOR-swizzled with the row number against bank conflicts)
             const int n_chunk = n_blk / 16, cmask = min(n_chunk, 8) - 1;
@@ -562,7 +572,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
               uint32_t w[8];
 #pragma unroll
               for (int c = 0; c < 4; ++c) {
-                const int r = 32 * c + lane;
+                const int r = rep ? lane : 32 * c + lane;
                 const uint2 v = *reinterpret_cast<const uint2*>(sSfa + (r * n_chunk + ((ks >> 1) ^ (r & cmask))) * 16 + (ks & 1) * 8);
                 w[c] = v.x;
                 w[4 + c] = v.y;
@@ -607,10 +617,12 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       }
     }
   } else if (wid >= kEpiWarp) {
-    // =========================== epilogue: warp of quadrant q owns tokens 4q..4q+3 of the pass ===========================
+    // =========================== epilogue ===========================
     // Accumulator lane = term row = 8 * token + term.  A 32x32b load hands each lane 32 columns of its row; three
     // exchange rounds over the 8 lanes of a token (each halves the columns a lane keeps) leave lane (token, t) with
     // the 8-term sums of 4 consecutive columns, at offset 16 (t & 1) + 8 (t >> 1 & 1) + 4 (t >> 2) of the 32.
+    // A pass of more than kRepTok tokens: the warp of quadrant q owns tokens 4q..4q+3 and all 256 columns.  A smaller
+    // pass has all its tokens in every quadrant: the warp of quadrant q owns a quarter of the columns of every token.
     const int q = wid & 3;
     const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
     const int jl = lane >> 3, tl = lane & 7;
@@ -621,93 +633,111 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     // for fetching it - on the critical path of a one-item CTA - while the warp has nothing to do before the first
     // accumulator is complete.
     auto run_pass = [&](const int phase, const int out_stride, const int tile, const int row0, const int n_tok, const bool dry) {
-      const int p = row0 + 4 * q + jl;                 // sorted row of this lane's token
-      const bool tok_live = !dry && 4 * q + jl < n_tok;
+      const bool rep = n_tok <= kRepTok;
+      const bool active = rep || 4 * q < n_tok;
+      // 32-column chunks this warp sums: all 8, or (small pass) gate chunk q and up chunk 4 + q of a gate/up item,
+      // chunks 2q and 2q + 1 of a down item
+      const int n_ch = rep ? 2 : 8;
+      const int ch0 = rep ? (phase == 0 ? q : 2 * q) : 0, ch_step = rep ? (phase == 0 ? 4 : 1) : 1;
       if (!dry) {
         mbar_wait(acc_full, acc_ph, a.status);
         acc_ph ^= 1u;
       }
       __syncwarp();  // tcgen05.ld is warp-collective
       tc_fence_after_sync();
-      float acc[8][4];  // [chunk of 32 columns][column cb + c]
-      if (dry || 4 * q < n_tok) {
+      float acc[8][4];  // [chunk][column cb + c of the chunk]
+      if (active) {
 #pragma unroll
-        for (int m = 0; m < 8; ++m) {
-          uint32_t vc[32];
-          tmem_ld_32x32(tmem_base + lane_base + kColD + static_cast<uint32_t>(32 * m), vc);
-          tmem_ld_wait();
-          float a16[16], a8[8];
+        for (int mm = 0; mm < 8; ++mm) {
+          if (mm < n_ch) {
+            uint32_t vc[32];
+            tmem_ld_32x32(tmem_base + lane_base + kColD + static_cast<uint32_t>(32 * (ch0 + mm * ch_step)), vc);
+            tmem_ld_wait();
+            float a16[16], a8[8];
 #pragma unroll
-          for (int k = 0; k < 16; ++k) {
-            const float lo = __uint_as_float(vc[k]), hi = __uint_as_float(vc[16 + k]);
-            a16[k] = ((tl & 1) ? hi : lo) + __shfl_xor_sync(0xffffffffu, (tl & 1) ? lo : hi, 1);
+            for (int k = 0; k < 16; ++k) {
+              const float lo = __uint_as_float(vc[k]), hi = __uint_as_float(vc[16 + k]);
+              a16[k] = ((tl & 1) ? hi : lo) + __shfl_xor_sync(0xffffffffu, (tl & 1) ? lo : hi, 1);
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              a8[k] = ((tl & 2) ? a16[8 + k] : a16[k]) + __shfl_xor_sync(0xffffffffu, (tl & 2) ? a16[k] : a16[8 + k], 2);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              acc[mm][k] = ((tl & 4) ? a8[4 + k] : a8[k]) + __shfl_xor_sync(0xffffffffu, (tl & 4) ? a8[k] : a8[4 + k], 4);
           }
-#pragma unroll
-          for (int k = 0; k < 8; ++k)
-            a8[k] = ((tl & 2) ? a16[8 + k] : a16[k]) + __shfl_xor_sync(0xffffffffu, (tl & 2) ? a16[k] : a16[8 + k], 2);
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
-            acc[m][k] = ((tl & 4) ? a8[4 + k] : a8[k]) + __shfl_xor_sync(0xffffffffu, (tl & 4) ? a8[k] : a8[4 + k], 4);
         }
       }
       tc_fence_before_sync();
       __syncwarp();
       if (!dry && lane == 0) mbar_arrive(acc_empty);  // the accumulator is free: the rest overlaps the next item's MMAs
-      if (!dry && 4 * q >= n_tok) return;
+      if (!active) return;
       if (phase == 0) {
-        // SwiGLU and the 8-term split, one (token, block of 32 consecutive i) per group of 8 lanes: in round rd
-        // the four lane groups take the four blocks of the quadrant's token rd (gate in chunk m, up in chunk m + 4),
-        // so that a quadrant with one token finishes in one round
+        // SwiGLU, bf16 rounding and the 8-term split, one (token, block of 32 consecutive i) per group of 8 lanes
         const int n_blk_i = a.I / 32;
-        const int n_q = dry ? 1 : min(4, n_tok - 4 * q);
+        // small pass: lane group jl has token jl, block q of the item's four, gate in acc[0] and up in acc[1] - one
+        // round.  Otherwise round rd hands the four blocks of the quadrant's token rd (gate in chunk m, up in chunk
+        // m + 4) to the four lane groups.
+        const int n_rd = rep ? 1 : min(4, n_tok - 4 * q);
 #pragma unroll 1
-        for (int rd = 0; rd < n_q; ++rd) {
+        for (int rd = 0; rd < n_rd; ++rd) {
           float gsel[4], usel[4];
-#pragma unroll
-          for (int m = 0; m < 4; ++m)
+          if (rep) {
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-              const float tg = __shfl_sync(0xffffffffu, acc[m][c], rd * 8 + tl);
-              const float tu = __shfl_sync(0xffffffffu, acc[m + 4][c], rd * 8 + tl);
-              if (jl == m) {
-                gsel[c] = tg;
-                usel[c] = tu;
-              }
+              gsel[c] = acc[0][c];
+              usel[c] = acc[1][c];
             }
+          } else {
+#pragma unroll
+            for (int m = 0; m < 4; ++m)
+#pragma unroll
+              for (int c = 0; c < 4; ++c) {
+                const float tg = __shfl_sync(0xffffffffu, acc[m][c], rd * 8 + tl);
+                const float tu = __shfl_sync(0xffffffffu, acc[m + 4][c], rd * 8 + tl);
+                if (jl == m) {
+                  gsel[c] = tg;
+                  usel[c] = tu;
+                }
+              }
+          }
           float r[1][4];
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             const float sv = __fdividef(gsel[c], 1.0f + __expf(-gsel[c])) * usel[c];
             r[0][c] = __bfloat162float(__float2bfloat16_rn(sv));  // the intermediate is defined as a bf16 value
           }
-          const int i0 = tile * 128 + 32 * jl;
-          uint8_t* qrow = a.aq2 + static_cast<size_t>(row0 + 4 * q + rd) * kTerms * (a.I / 2) + ((i0 + cb) >> 1);
-          uint8_t* srow = a.sf2 + static_cast<size_t>(row0 + 4 * q + rd) * kTerms * n_blk_i + (i0 >> 5);
+          const int tok = rep ? jl : 4 * q + rd;  // token of the pass whose block this lane group splits
+          const int i0 = tile * 128 + 32 * (rep ? q : jl);
+          const bool live = !dry && tok < n_tok;
+          uint8_t* qrow = a.aq2 + static_cast<size_t>(row0 + tok) * kTerms * (a.I / 2) + ((i0 + cb) >> 1);
+          uint8_t* srow = a.sf2 + static_cast<size_t>(row0 + tok) * kTerms * n_blk_i + (i0 >> 5);
           split_terms<1>(r, [&](int, int t, uint32_t bytes, int se) {
-            if (!dry) {
+            if (live) {
               *reinterpret_cast<uint16_t*>(qrow + static_cast<size_t>(t) * (a.I / 2)) = static_cast<uint16_t>(bytes);
               if (tl == 0) srow[static_cast<size_t>(t) * n_blk_i] = static_cast<uint8_t>(se + 127);
             }
           });
         }
       } else {
-        if (tok_live) {
-          float* dst = a.y + static_cast<size_t>(p) * out_stride + tile * kTile + cb;
+        const int tok = rep ? jl : 4 * q + jl;
+        if (!dry && tok < n_tok) {
+          float* dst = a.y + static_cast<size_t>(row0 + tok) * out_stride + tile * kTile + 32 * ch0 + cb;
 #pragma unroll
-          for (int m = 0; m < 8; ++m)
-            *reinterpret_cast<float4*>(dst + 32 * m) = make_float4(acc[m][0], acc[m][1], acc[m][2], acc[m][3]);
+          for (int mm = 0; mm < 8; ++mm)
+            if (mm < n_ch) *reinterpret_cast<float4*>(dst + 32 * mm) = make_float4(acc[mm][0], acc[mm][1], acc[mm][2], acc[mm][3]);
         }
       }
     };
-    for (int sweep = 0; sweep < 2; ++sweep) {  // sweep 0 is the dry run: one pass through the one call site below
+    for (int sweep = 0; sweep < 2; ++sweep) {  // sweep 0 is the dry run of this CTA's first pass, through the one call site below
       const bool dry = sweep == 0;
       for (int phase = 0; phase < (dry ? 1 : 2); ++phase) {
         const Phase P = phase_of(phase, a, s_misc + 1);
-        const long long it_begin = dry ? 0 : P.begin, it_end = dry ? 1 : P.end;
-        for (long long it = it_begin; it < it_end; ++it) {
+        const long long it_end = dry ? min(P.begin + 1, P.end) : P.end;
+        for (long long it = P.begin; it < it_end; ++it) {
           const int ti = static_cast<int>(it / P.tiles), tile = static_cast<int>(it % P.tiles);
-          const int row_begin = dry ? 0 : t_begin[ti], row_end = dry ? 1 : t_end[ti];
-          const int n_pass = (row_end - row_begin + tok_pass - 1) / tok_pass;
+          const int row_begin = t_begin[ti], row_end = t_end[ti];
+          const int n_pass = dry ? 1 : (row_end - row_begin + tok_pass - 1) / tok_pass;
           for (int pass = 0; pass < n_pass; ++pass) {
             const int row0 = row_begin + pass * tok_pass;
             run_pass(phase, P.R, tile, row0, min(tok_pass, row_end - row0), dry);
