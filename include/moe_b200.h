@@ -147,13 +147,39 @@ int moe_combine(const float* y_perm, const int32_t* inv_perm, const float* topk_
 int moe_validate_scales(const uint8_t* scales, size_t n_bytes, int32_t* bad_count, void* cuda_stream);
 
 /*
- * The four calls above with HOST input and output for one batch: copies logits_host [T,E] and
- * x_host [T,H] to the device buffers carved from `ws`, runs route -> permute -> expert_ffn ->
- * combine on `cuda_stream`, copies out [T,H] bf16 back into out_host and waits for the stream.
+ * The whole layer in one call on DEVICE buffers: route -> permute -> expert_ffn -> combine of the same inputs, with
+ * every intermediate (sorted rows, per-slot outputs) kept in `ws`.  The paper's own decode gains came from cutting
+ * passes and launches around the expert kernels (its optimisation history and the section on the down-projection
+ * consumer); this is that step for this library.  Result: out [T,H] bf16 exactly as moe_combine would write it after
+ * the three calls before it, and - where the pointers are not NULL - topk_ids / topk_w [T,k] exactly as moe_route
+ * writes them.
+ *
+ *   - For T <= 4 tokens (T*k <= 32 slots, T*E*4 <= 4*max(H,I) bytes) on shapes the decode-sized expert kernel takes,
+ *     the call is ONE kernel launch: every CTA routes the T tokens itself, sorts the slots, writes its own E2M1 term
+ *     rows of the tokens, runs its share of the gate/up and down items, and the CTA that finishes a column tile's last
+ *     expert reduces that tile over the slots.  Any other shape runs the four calls back to back.
+ *   - ws: moe_forward_workspace_bytes() bytes, 256-byte aligned.  Its first moe_forward_sync_bytes() bytes are the
+ *     kernel's completion counters: they must be ZERO when a call starts.  Clear them once (cudaMemsetAsync) before
+ *     the first call that uses this ws; every call that returns MOE_OK and whose kernels ran to completion leaves them
+ *     zero, also when *status_word reports a device-side timeout.  The rest of ws is scratch.  Calls that share a ws
+ *     must be ordered on one stream.
+ *   - Asynchronous, no allocation, capturable into a CUDA graph, bounded device-side waits as moe_expert_ffn.
+ */
+size_t moe_forward_workspace_bytes(const moe_shape_t* shape);
+size_t moe_forward_sync_bytes(void);
+int moe_forward(const float* logits /* [T,E] */, const void* x_bf16 /* [T,H] */, const uint8_t* w13, const uint8_t* w13_scale,
+                const uint8_t* w2, const uint8_t* w2_scale, const moe_shape_t* shape, void* out_bf16 /* [T,H] */,
+                int32_t* topk_ids /* [T,k] or NULL */, float* topk_w /* [T,k] or NULL */, int32_t* status_word, void* ws,
+                size_t ws_bytes, void* cuda_stream);
+
+/*
+ * moe_forward with HOST input and output for one batch: copies logits_host [T,E] and x_host [T,H] to
+ * device buffers carved from `ws`, clears moe_forward's counters, runs moe_forward on `cuda_stream`,
+ * copies out [T,H] bf16 back into out_host and waits for the stream.
  * Weights stay device-resident (they are model state, not per-batch input).  For page-locked host
  * buffers the copies are asynchronous until the final wait.  ws must hold
  * moe_forward_host_workspace_bytes() bytes.  No counterpart in the paper: it is the end-to-end
- * measurement path of the four calls.
+ * measurement path of the layer.
  */
 size_t moe_forward_host_workspace_bytes(const moe_shape_t* shape);
 int moe_forward_host(const float* logits_host, const void* x_host_bf16, const uint8_t* w13,

@@ -138,14 +138,91 @@ int moe_validate_scales(const uint8_t* scales, size_t n_bytes, int32_t* bad_coun
   return launch_validate_scales(scales, n_bytes, bad_count, static_cast<cudaStream_t>(cuda_stream));
 }
 
+// ---- whole layer, device buffers -------------------------------------------------------------------
+namespace {
+// ws of moe_forward = [ sync block | one-launch scratch, or the buffers between the four calls and their workspace ]
+struct ForwardLayout {
+  size_t ids, w, offsets, x_perm, perm, inv_perm, y_perm, inner, total;
+};
+ForwardLayout forward_layout(const moe_shape_t& s) {
+  ForwardLayout L;
+  const size_t S = static_cast<size_t>(s.T) * s.k;
+  size_t off = kForwardSyncBytes;
+  auto take = [&](size_t bytes) {
+    const size_t o = off;
+    off += align_up(bytes, kAlign);
+    return o;
+  };
+  L.ids = take(S * 4);
+  L.w = take(S * 4);
+  L.offsets = take((static_cast<size_t>(s.E) + 1) * 4);
+  L.x_perm = take(S * s.H * 2);
+  L.perm = take(S * 4);
+  L.inv_perm = take(S * 4);
+  L.y_perm = take(S * s.H * 4);
+  L.inner = off;
+  off += ws_layout(s).total;
+  // whether the one-launch kernel applies also depends on the weights' alignment; the size allows for it whenever
+  // the shape does
+  const size_t fused = forward_fused_ok(s, reinterpret_cast<const void*>(uintptr_t(256)), reinterpret_cast<const void*>(uintptr_t(256)))
+                           ? kForwardSyncBytes + forward_fused_scratch_bytes(s)
+                           : 0;
+  L.total = off > fused ? off : fused;
+  return L;
+}
+}  // namespace
+
+size_t moe_forward_workspace_bytes(const moe_shape_t* shape) {
+  if (check_shape(shape) != MOE_OK) return 0;
+  return forward_layout(*shape).total;
+}
+
+size_t moe_forward_sync_bytes(void) { return kForwardSyncBytes; }
+
+int moe_forward(const float* logits, const void* x_bf16, const uint8_t* w13, const uint8_t* w13_scale, const uint8_t* w2,
+                const uint8_t* w2_scale, const moe_shape_t* shape, void* out_bf16, int32_t* topk_ids, float* topk_w,
+                int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (!aligned(logits, 16) || !aligned(x_bf16, 16) || !aligned(w13, 16) || !aligned(w13_scale, 16) || !aligned(w2, 16) ||
+      !aligned(w2_scale, 16) || !aligned(out_bf16, 16))
+    return MOE_ERR_INVALID_ARG;
+  if ((topk_ids != nullptr && !aligned(topk_ids, 16)) || (topk_w != nullptr && !aligned(topk_w, 16)) ||
+      (status_word != nullptr && !aligned(status_word, 4)))
+    return MOE_ERR_INVALID_ARG;
+  const ForwardLayout L = forward_layout(*shape);
+  if (check_ws(ws, ws_bytes, L.total) != MOE_OK) return MOE_ERR_WORKSPACE;
+  char* base = static_cast<char*>(ws);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (forward_fused_ok(*shape, w13, w2))
+    return launch_forward_fused(logits, static_cast<const __nv_bfloat16*>(x_bf16), w13, w13_scale, w2, w2_scale, *shape,
+                                static_cast<__nv_bfloat16*>(out_bf16), topk_ids, topk_w, reinterpret_cast<int*>(base),
+                                base + kForwardSyncBytes, status_word, st);
+  int32_t* d_ids = topk_ids != nullptr ? topk_ids : reinterpret_cast<int32_t*>(base + L.ids);
+  float* d_w = topk_w != nullptr ? topk_w : reinterpret_cast<float*>(base + L.w);
+  int32_t* d_off = reinterpret_cast<int32_t*>(base + L.offsets);
+  void* d_xp = base + L.x_perm;
+  int32_t* d_perm = reinterpret_cast<int32_t*>(base + L.perm);
+  int32_t* d_inv = reinterpret_cast<int32_t*>(base + L.inv_perm);
+  float* d_y = reinterpret_cast<float*>(base + L.y_perm);
+  void* inner = base + L.inner;
+  const size_t inner_bytes = ws_bytes - L.inner;
+  const moe_shape_t& s = *shape;
+  if ((rc = moe_route(logits, s.T, s.E, s.k, d_ids, d_w, d_off, inner, inner_bytes, st)) != MOE_OK) return rc;
+  if ((rc = moe_permute(x_bf16, d_ids, d_off, shape, d_xp, d_perm, d_inv, inner, inner_bytes, st)) != MOE_OK) return rc;
+  if ((rc = moe_expert_ffn(d_xp, d_off, w13, w13_scale, w2, w2_scale, shape, d_y, status_word, inner, inner_bytes, st)) !=
+      MOE_OK)
+    return rc;
+  return moe_combine(d_y, d_inv, d_w, shape, out_bf16, st);
+}
+
 // ---- host-buffer path ---------------------------------------------------------------------------
 namespace {
 struct HostLayout {
-  size_t logits, x, ids, w, offsets, x_perm, perm, inv_perm, y_perm, out, inner, total;
+  size_t logits, x, out, inner, total;
 };
 HostLayout host_layout(const moe_shape_t& s) {
   HostLayout L;
-  const size_t S = static_cast<size_t>(s.T) * s.k;
   size_t off = 0;
   auto take = [&](size_t bytes) {
     const size_t o = off;
@@ -154,16 +231,9 @@ HostLayout host_layout(const moe_shape_t& s) {
   };
   L.logits = take(static_cast<size_t>(s.T) * s.E * 4);
   L.x = take(static_cast<size_t>(s.T) * s.H * 2);
-  L.ids = take(S * 4);
-  L.w = take(S * 4);
-  L.offsets = take((static_cast<size_t>(s.E) + 1) * 4);
-  L.x_perm = take(S * s.H * 2);
-  L.perm = take(S * 4);
-  L.inv_perm = take(S * 4);
-  L.y_perm = take(S * s.H * 4);
   L.out = take(static_cast<size_t>(s.T) * s.H * 2);
   L.inner = off;
-  off += ws_layout(s).total;
+  off += forward_layout(s).total;
   L.total = off;
   return L;
 }
@@ -187,25 +257,15 @@ int moe_forward_host(const float* logits_host, const void* x_host_bf16, const ui
   const moe_shape_t& s = *shape;
   float* d_logits = reinterpret_cast<float*>(base + L.logits);
   void* d_x = base + L.x;
-  int32_t* d_ids = reinterpret_cast<int32_t*>(base + L.ids);
-  float* d_w = reinterpret_cast<float*>(base + L.w);
-  int32_t* d_off = reinterpret_cast<int32_t*>(base + L.offsets);
-  void* d_xp = base + L.x_perm;
-  int32_t* d_perm = reinterpret_cast<int32_t*>(base + L.perm);
-  int32_t* d_inv = reinterpret_cast<int32_t*>(base + L.inv_perm);
-  float* d_y = reinterpret_cast<float*>(base + L.y_perm);
   void* d_out = base + L.out;
-  void* inner = base + L.inner;
-  const size_t inner_bytes = ws_bytes - L.inner;
-  if (cudaMemcpyAsync(d_logits, logits_host, static_cast<size_t>(s.T) * s.E * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+  // this call owns its workspace's contents: it clears the sync block of moe_forward itself
+  if (cudaMemsetAsync(base + L.inner, 0, kForwardSyncBytes, st) != cudaSuccess ||
+      cudaMemcpyAsync(d_logits, logits_host, static_cast<size_t>(s.T) * s.E * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
       cudaMemcpyAsync(d_x, x_host_bf16, static_cast<size_t>(s.T) * s.H * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
     return MOE_ERR_CUDA;
-  if ((rc = moe_route(d_logits, s.T, s.E, s.k, d_ids, d_w, d_off, inner, inner_bytes, st)) != MOE_OK) return rc;
-  if ((rc = moe_permute(d_x, d_ids, d_off, shape, d_xp, d_perm, d_inv, inner, inner_bytes, st)) != MOE_OK) return rc;
-  if ((rc = moe_expert_ffn(d_xp, d_off, w13, w13_scale, w2, w2_scale, shape, d_y, status_word, inner, inner_bytes, st)) !=
-      MOE_OK)
+  if ((rc = moe_forward(d_logits, d_x, w13, w13_scale, w2, w2_scale, shape, d_out, nullptr, nullptr, status_word,
+                        base + L.inner, ws_bytes - L.inner, st)) != MOE_OK)
     return rc;
-  if ((rc = moe_combine(d_y, d_inv, d_w, shape, d_out, st)) != MOE_OK) return rc;
   if (cudaMemcpyAsync(out_host_bf16, d_out, static_cast<size_t>(s.T) * s.H * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return MOE_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return MOE_ERR_CUDA;

@@ -41,6 +41,7 @@
 
 #include <algorithm>
 
+#include "moe_route_device.cuh"
 #include "moe_sm100_primitives.cuh"
 
 namespace moe {
@@ -76,6 +77,29 @@ struct NatArgs {
   float* y;                  // output [S, H]
   int* status;
   int E, H, I, S;
+};
+
+// The one-launch layer (moe_forward on a handful of tokens): what the kernel needs beyond the expert FFN's arguments.
+// Every CTA routes all T tokens itself (same arithmetic, same result everywhere), sorts the T * k slots by expert in
+// shared memory and splits the T token rows into its own copy of their term rows; the gate/up items then take all T
+// tokens as operand rows (row = 8 * token + term) whatever their expert, and the epilogue keeps the tokens that were
+// routed to the item's expert.  After the down projection the CTA that runs the last expert's item of a column tile
+// reduces that tile over the slots of every token.
+constexpr int kFusedMaxTok = 4;    // tokens of a fused call: one lane quadrant of operand rows
+constexpr int kFusedMaxSlots = 32; // T * k: one warp sorts them
+constexpr int kFusedMaxCtas = 256; // the scratch holds this many CTAs' term rows (more SMs than that: a smaller grid)
+constexpr int kSyncDone2 = 1024;   // int index in the sync block: per column tile, warps that stored a down item
+constexpr int kSyncExit = 1024 + 64;  // CTAs that have finished; the last one clears the block
+struct FusedArgs {
+  const float* logits;       // [T, E]
+  const __nv_bfloat16* x;    // [T, H]
+  __nv_bfloat16* out;        // [T, H]
+  int* ids_out;              // [T, k] or null
+  float* w_out;              // [T, k] or null
+  uint8_t* aq1;              // [grid][T * 8, H/2] each CTA's term rows of the tokens
+  uint8_t* sf1;              // [grid][T * 8, H/32]
+  int* sync;                 // sync block: [0, E) = NatArgs::done, then the indices above; zero between calls
+  int T, k;
 };
 
 // Term-row tensor maps of one projection's input: the same tensor with boxes of 8, 16, 32, 64 and 128 rows (1, 2, 4, 8,
@@ -139,7 +163,7 @@ MOE_DEVINL Phase phase_of(int ph, const NatArgs& a, const int* shares) {
 }
 
 struct NatSmem {
-  uint32_t act, w, sc, sfa, bars, misc, touched, total;
+  uint32_t act, w, sc, sfa, bars, misc, touched, route, total;
 };
 __host__ __device__ inline NatSmem nat_smem(int E, int K) {
   NatSmem m;
@@ -157,6 +181,8 @@ __host__ __device__ inline NatSmem nat_smem(int E, int K) {
   off += 64;
   m.touched = off;  // touched experts: id, first row, end row
   off += (3 * static_cast<uint32_t>(E) + 8) * 4;
+  m.route = off;    // one-launch layer: expert and weight of every slot, sorted row of every slot, row of (touched expert, token)
+  off += (3 * kFusedMaxSlots + kFusedMaxSlots * kFusedMaxTok) * 4;
   m.total = off;
   return m;
 }
@@ -283,10 +309,15 @@ __global__ void __launch_bounds__(1024) native_split_kernel(const __nv_bfloat16*
   });
 }
 
+// kFused = false: the expert FFN (moe_expert_ffn).  kFused = true: the whole layer in this one launch (see FusedArgs);
+// the differences are the set-up, where the gate/up items' operand rows come from, which rows their epilogue writes,
+// and the reduction over slots after the down items.
+template <bool kFused>
 __global__ void __launch_bounds__(kNatThreads, 1)
 ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_constant__ CUtensorMap tmap_s13,
                   const __grid_constant__ TermMaps tmap_a1, const __grid_constant__ CUtensorMap tmap_w2,
-                  const __grid_constant__ CUtensorMap tmap_s2, const __grid_constant__ TermMaps tmap_a2, const NatArgs a) {
+                  const __grid_constant__ CUtensorMap tmap_s2, const __grid_constant__ TermMaps tmap_a2, const NatArgs a,
+                  const FusedArgs f) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   const NatSmem sm = nat_smem(a.E, a.H > a.I ? a.H : a.I);
@@ -309,6 +340,10 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   int* t_begin = touched + a.E;                              // their first sorted row
   int* t_end = t_begin + a.E;                                // and the row after their last
   int* s_misc = t_end + a.E;
+  int* s_ids = reinterpret_cast<int*>(smem + sm.route);                 // [T * k] expert of every slot (one-launch layer only)
+  float* s_w = reinterpret_cast<float*>(s_ids + kFusedMaxSlots);        // [T * k] routing weight
+  int* s_row = reinterpret_cast<int*>(s_w + kFusedMaxSlots);            // [T * k] sorted row of every slot
+  int* row_of = s_row + kFusedMaxSlots;                                 // [touched expert][token] sorted row, or -1
 
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   constexpr int tok_pass = kMaxTokPass;
@@ -325,7 +360,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       prefetch_tmap(&tmap_a2.box[i]);
     }
   }
-  if (wid == 2) {
+  if (!kFused && wid == 2) {
     // lane l looks at experts l, l + 32, ...: all loads are issued before any is used (one memory round trip);
     // the second loop's loads hit L1.  expert_offsets was complete before the permute kernel let this chain start.
     const int n_it = (a.E + 31) / 32;
@@ -381,6 +416,94 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   // (griddepcontrol.wait) for this grid to complete before it reads the output.  This grid in turn reads nothing
   // of the split kernel before it has waited itself, apart from expert_offsets (see above).
   pdl_launch_dependents();
+  if constexpr (kFused) {
+    // ---- the layer's first steps, the same in every CTA: route, sort the slots, split the token rows ----
+    pdl_wait();  // logits and token rows may come from the kernel before this one; the sync block is clear
+    if (wid >= 2 && wid < 6) {
+      // one warp per token: top-k by logit (ties to the lower expert), softmax over the selected logits
+      const int t = wid - 2;
+      if (t < f.T) {
+        float* row = reinterpret_cast<float*>(sSfa) + t * a.E;  // this region is not in use yet
+        for (int e = lane; e < a.E; e += 32) row[e] = f.logits[static_cast<size_t>(t) * a.E + e];
+        __syncwarp();
+        int my_id;
+        float my_v;
+        warp_topk(row, a.E, f.k, lane, &my_id, &my_v);
+        const float wt = warp_softmax_selected(my_v, f.k, lane);
+        if (lane < f.k) {
+          s_ids[t * f.k + lane] = my_id;
+          s_w[t * f.k + lane] = wt;
+          if (blockIdx.x == 0 && f.ids_out != nullptr) f.ids_out[t * f.k + lane] = my_id;
+          if (blockIdx.x == 0 && f.w_out != nullptr) f.w_out[t * f.k + lane] = wt;
+        }
+      }
+    } else {
+      // the other six warps: token rows -> this CTA's term rows, four 32-element blocks per group of 8 lanes at a
+      // time; a warp takes 16 consecutive blocks per round, so its lanes run the same number of rounds
+      const int sw = wid < 2 ? wid : wid - 4;  // 0..5
+      const int n_blk = a.H / 32, n_all = f.T * n_blk;
+      uint8_t* my_aq = f.aq1 + static_cast<size_t>(blockIdx.x) * f.T * kTerms * (a.H / 2);
+      uint8_t* my_sf = f.sf1 + static_cast<size_t>(blockIdx.x) * f.T * kTerms * n_blk;
+      const int sub = lane & 7;
+      for (int b0 = sw * 16 + (lane >> 3) * 4; b0 < n_all; b0 += 6 * 16) {
+        float r[4][4];
+#pragma unroll
+        for (int nb = 0; nb < 4; ++nb) {
+          const int b = b0 + nb, t = b / n_blk, blk = b % n_blk;
+          const uint2 v = *reinterpret_cast<const uint2*>(f.x + static_cast<size_t>(t) * a.H + blk * 32 + sub * 4);
+          r[nb][0] = __uint_as_float(v.x << 16);
+          r[nb][1] = __uint_as_float(v.x & 0xFFFF0000u);
+          r[nb][2] = __uint_as_float(v.y << 16);
+          r[nb][3] = __uint_as_float(v.y & 0xFFFF0000u);
+        }
+        split_terms<4>(r, [&](int nb, int t8, uint32_t bytes, int se) {
+          const int b = b0 + nb, t = b / n_blk, blk = b % n_blk;
+          const size_t trow = static_cast<size_t>(t) * kTerms + t8;
+          *reinterpret_cast<uint16_t*>(my_aq + trow * (a.H / 2) + blk * 16 + sub * 2) = static_cast<uint16_t>(bytes);
+          if (sub == 0) my_sf[trow * n_blk + blk] = static_cast<uint8_t>(se + 127);
+        });
+      }
+      fence_proxy_async_all();  // TMA will read these rows
+    }
+    __syncthreads();
+    if (wid == 2) {
+      // Stable sort of the slots by expert, S <= 32: lane s is slot s.  Its sorted row = slots of smaller experts +
+      // earlier slots of its own expert; the touched experts are the distinct ids in ascending order.
+      const int S = f.T * f.k;
+      const int id = lane < S ? s_ids[lane] : 0x7fffffff;
+      int less = 0, eq_all = 0, eq_before = 0;
+      for (int o = 0; o < S; ++o) {
+        const int oid = __shfl_sync(0xffffffffu, id, o);
+        less += oid < id;
+        eq_all += oid == id;
+        eq_before += (oid == id) && (o < lane);
+      }
+      const bool first = lane < S && eq_before == 0;
+      int ti = 0;  // touched experts with a smaller id
+      for (int o = 0; o < S; ++o) {
+        const int oid = __shfl_sync(0xffffffffu, id, o);
+        const int of = __shfl_sync(0xffffffffu, static_cast<int>(first), o);
+        ti += of && (oid < id);
+      }
+      const int n_t = __popc(__ballot_sync(0xffffffffu, first));
+      for (int i = lane; i < kFusedMaxSlots * kFusedMaxTok; i += 32) row_of[i] = -1;
+      __syncwarp();
+      if (lane < S) {
+        s_row[lane] = less + eq_before;
+        row_of[ti * kFusedMaxTok + lane / f.k] = less + eq_before;
+      }
+      if (first) {
+        touched[ti] = id;
+        t_begin[ti] = less;
+        t_end[ti] = less + eq_all;
+      }
+      if (lane == 0) {
+        s_misc[0] = n_t;
+        cta_shares(static_cast<int>(gridDim.x), static_cast<int>(blockIdx.x), n_t, 2 * a.I / kTile, a.H / kTile, s_misc + 1);
+      }
+    }
+    __syncthreads();
+  }
   // Every role walks the same sequence: both phases; in each, this CTA's items; per item, passes of up to tok_pass
   // tokens; per pass, all K steps.
 
@@ -392,7 +515,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       // The weights depend on nothing, the term rows do: on the split kernel (phase 0) or on the gate/up items of
       // their expert (phase 1).  While a dependency is open, the weight loads go out and the term-row loads of up to
       // kWStages steps are held back; they follow once the dependency is met.
-      bool pdl_done = false, dep_ok = false;
+      // (one-launch layer: the gate/up items read this CTA's own term rows, complete since the set-up)
+      bool pdl_done = kFused, dep_ok = kFused;
       int dep_phase = 0, dep_e = -1;
       int n_pend = 0, pend_s[kWStages], pend_x[kWStages], pend_y[kWStages], pend_b[kWStages];
       // term rows of one K step; a pass of at most kRepTok tokens gets them once per lane quadrant of the accumulator
@@ -435,7 +559,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             dep_ok = false;
           }
           for (int pass = 0; pass < n_pass; ++pass) {
-            const int bi = term_box(min(tok_pass, n_rows_e - pass * tok_pass));  // box of 8 << bi term rows
+            const bool own_rows = kFused && phase == 0;  // all T tokens, from this CTA's copy
+            const int bi = term_box(own_rows ? f.T : min(tok_pass, n_rows_e - pass * tok_pass));  // box of 8 << bi term rows
             for (int ks = 0; ks < P.n_steps; ++ks) {
               if ((ks & 1) == 0) {  // 16 scale bytes per weight row cover two K steps
                 mbar_wait(&empty_sc[cs], cph ^ 1u, a.status);
@@ -449,7 +574,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
               tma_load_2d(sW + s * kStage, mw, ks * 128, wrow_a, &full_w[s]);
               tma_load_2d(sW + s * kStage + 128 * 128, mw, ks * 128, wrow_b, &full_w[s]);
               // the pass's term rows (8 per token, consecutive); rows past the end of the tensor arrive as zeros
-              const int arow = (row_begin + pass * tok_pass) * kTerms;
+              const int arow = own_rows ? static_cast<int>(blockIdx.x) * f.T * kTerms : (row_begin + pass * tok_pass) * kTerms;
               if (dep_ok) {
                 load_terms(ma, s, bi, ks * 128, arow);
               } else {
@@ -481,7 +606,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
           for (int pass = 0; pass < n_pass; ++pass) {
             // The scale factors of the term rows (tensor memory) are shared by consecutive items of an expert whose
             // rows fit one pass; otherwise every (item, pass) has its own.  The scale warps follow the same rule.
-            const bool new_operand = (prev_ti != ti) || (n_pass > 1);
+            // (One-launch layer: every gate/up item has the same operand, all T tokens.)
+            const bool new_operand = (kFused && phase == 0) ? (it == P.begin) : ((prev_ti != ti) || (n_pass > 1));
             prev_ti = ti;
             if (new_operand) {
               mbar_wait(act_ready, aph, a.status);
@@ -512,7 +638,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             acc_ph ^= 1u;
             // last use of these scale factors?  (always at the end of a phase)
             bool next_new = true;
-            if (pass + 1 >= n_pass && it + 1 < P.end) next_new = (static_cast<int>((it + 1) / P.tiles) != ti) || (n_pass > 1);
+            if (pass + 1 >= n_pass && it + 1 < P.end)
+              next_new = (kFused && phase == 0) ? false : ((static_cast<int>((it + 1) / P.tiles) != ti) || (n_pass > 1));
             if (next_new) umma_commit(act_free);
           }
         }
@@ -529,19 +656,19 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     for (int phase = 0; phase < 2; ++phase) {
       const Phase P = phase_of(phase, a, s_misc + 1);
       const int n_blk = P.K / 32;
-      const uint8_t* src_sf = phase == 0 ? a.sf1 : a.sf2;
+      const uint8_t* src_sf = phase == 0 ? (kFused ? f.sf1 : a.sf1) : a.sf2;
       int prev_ti = -1;
       for (long long it = P.begin; it < P.end; ++it) {
         const int ti = static_cast<int>(it / P.tiles);
         const int row_begin = t_begin[ti], row_end = t_end[ti];
         const int n_pass = (row_end - row_begin + tok_pass - 1) / tok_pass;
         for (int pass = 0; pass < n_pass; ++pass) {
-          const bool new_operand = (prev_ti != ti) || (n_pass > 1);
+          const bool new_operand = (kFused && phase == 0) ? (it == P.begin) : ((prev_ti != ti) || (n_pass > 1));
           prev_ti = ti;
           if (new_operand) {
             // ---- scale factors of the pass's term rows: global -> shared memory -> tensor memory ----
             if (first_op) {
-              pdl_wait();  // the split kernel is complete: scale bytes of the tokens' terms, cleared counters
+              if (!kFused) pdl_wait();  // the split kernel is complete: scale bytes of the tokens' terms, cleared counters
             } else {
               mbar_wait(act_free, afree_ph, a.status);  // MMAs that read the previous scale factors are done
               afree_ph ^= 1u;
@@ -552,8 +679,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
               if (st == 0) counter_wait_ge(a.done + touched[ti], need_done, a.status);
               asm volatile("bar.sync 3, 128;" ::: "memory");
             }
-            const int row0 = row_begin + pass * tok_pass;
-            const int n_rows = min(tok_pass, row_end - row0) * kTerms;  // term rows that exist
+            const bool own_rows = kFused && phase == 0;
+            const int row0 = own_rows ? static_cast<int>(blockIdx.x) * f.T : row_begin + pass * tok_pass;
+            const int n_rows = (own_rows ? f.T : min(tok_pass, row_end - row0)) * kTerms;  // term rows that exist
             const bool rep = n_rows <= kRepTok * kTerms;                // the operand repeats in every lane quadrant
             // rows are n_blk bytes each and consecutive: one contiguous range, copied 16 bytes at a time
             // (the 16-byte chunks of a row are XOR-swizzled with the row number against bank conflicts)
@@ -632,7 +760,10 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     // and store left out: each CTA executes this code only a few times, so its first real use would otherwise pay
     // for fetching it - on the critical path of a one-item CTA - while the warp has nothing to do before the first
     // accumulator is complete.
-    auto run_pass = [&](const int phase, const int out_stride, const int tile, const int row0, const int n_tok, const bool dry) {
+    // `rowmap` (one-launch layer, gate/up items): sorted row of each operand token for this item's expert, -1 for the
+    // tokens that were not routed to it; otherwise operand token i is sorted row row0 + i.
+    auto run_pass = [&](const int phase, const int out_stride, const int tile, const int row0, const int n_tok, const int* rowmap,
+                        const bool dry) {
       const bool rep = n_tok <= kRepTok;
       const bool active = rep || 4 * q < n_tok;
       // 32-column chunks this warp sums: all 8, or (small pass) gate chunk q and up chunk 4 + q of a gate/up item,
@@ -709,9 +840,10 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
           }
           const int tok = rep ? jl : 4 * q + rd;  // token of the pass whose block this lane group splits
           const int i0 = tile * 128 + 32 * (rep ? q : jl);
-          const bool live = !dry && tok < n_tok;
-          uint8_t* qrow = a.aq2 + static_cast<size_t>(row0 + tok) * kTerms * (a.I / 2) + ((i0 + cb) >> 1);
-          uint8_t* srow = a.sf2 + static_cast<size_t>(row0 + tok) * kTerms * n_blk_i + (i0 >> 5);
+          const int prow = tok < n_tok ? (rowmap != nullptr ? rowmap[tok] : row0 + tok) : -1;
+          const bool live = !dry && prow >= 0;
+          uint8_t* qrow = a.aq2 + static_cast<size_t>(live ? prow : 0) * kTerms * (a.I / 2) + ((i0 + cb) >> 1);
+          uint8_t* srow = a.sf2 + static_cast<size_t>(live ? prow : 0) * kTerms * n_blk_i + (i0 >> 5);
           split_terms<1>(r, [&](int, int t, uint32_t bytes, int se) {
             if (live) {
               *reinterpret_cast<uint16_t*>(qrow + static_cast<size_t>(t) * (a.I / 2)) = static_cast<uint16_t>(bytes);
@@ -738,9 +870,42 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
           const int ti = static_cast<int>(it / P.tiles), tile = static_cast<int>(it % P.tiles);
           const int row_begin = t_begin[ti], row_end = t_end[ti];
           const int n_pass = dry ? 1 : (row_end - row_begin + tok_pass - 1) / tok_pass;
+          const bool own_rows = kFused && phase == 0;
           for (int pass = 0; pass < n_pass; ++pass) {
             const int row0 = row_begin + pass * tok_pass;
-            run_pass(phase, P.R, tile, row0, min(tok_pass, row_end - row0), dry);
+            run_pass(phase, P.R, tile, row0, own_rows ? f.T : min(tok_pass, row_end - row0),
+                     own_rows ? row_of + ti * kFusedMaxTok : nullptr, dry);
+          }
+          if constexpr (kFused) {
+            if (!dry && phase == 1) {
+              // this warp's columns of the item are stored: count it for the column tile, and after the last
+              // expert's item reduce the tile over the slots of every token (in slot order, as moe_combine does)
+              __syncwarp();
+              if (lane == 0) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(f.sync + kSyncDone2 + tile) : "memory");
+              if (ti == s_misc[0] - 1) {
+                if (lane == 0) counter_wait_ge(f.sync + kSyncDone2 + tile, 4 * s_misc[0], a.status);
+                __syncwarp();
+                const int col = tile * kTile + (wid - kEpiWarp) * 64 + lane * 2;
+                for (int t = 0; t < f.T; ++t) {
+                  float2 acc = make_float2(0.0f, 0.0f);
+                  for (int j0 = 0; j0 < f.k; j0 += 4) {  // four slots' loads in flight; the multiply-adds stay in slot order
+                    float2 v[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                      if (j0 + u < f.k)
+                        v[u] = __ldcg(reinterpret_cast<const float2*>(a.y + static_cast<size_t>(s_row[t * f.k + j0 + u]) * a.H + col));
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                      if (j0 + u < f.k) {
+                        const float wj = s_w[t * f.k + j0 + u];
+                        acc.x = __fmaf_rn(wj, v[u].x, acc.x);
+                        acc.y = __fmaf_rn(wj, v[u].y, acc.y);
+                      }
+                  }
+                  *reinterpret_cast<__nv_bfloat162*>(f.out + static_cast<size_t>(t) * a.H + col) = __floats2bfloat162_rn(acc.x, acc.y);
+                }
+              }
+            }
           }
           if (!dry && phase == 0) {
             // publish: this warp's rows of the item (all passes) are written; TMA (asynchronous proxy) and plain
@@ -760,6 +925,24 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   if (wid == 1) {
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, kNatTmemCols);
+  }
+  if constexpr (kFused) {
+    // The last CTA to get here clears the sync block for the next call: by then every CTA has made its last read of
+    // and its last addition to the counters.
+    if (wid == 0) {
+      int last = 0;
+      if (lane == 0) {
+        __threadfence();
+        last = atomicAdd(f.sync + kSyncExit, 1) == static_cast<int>(gridDim.x) - 1;
+      }
+      last = __shfl_sync(0xffffffffu, last, 0);
+      if (last) {
+        __threadfence();
+        for (int i = lane; i < a.E; i += 32) f.sync[i] = 0;
+        for (int i = lane; i < a.H / kTile; i += 32) f.sync[kSyncDone2 + i] = 0;
+        if (lane == 0) f.sync[kSyncExit] = 0;
+      }
+    }
   }
 }
 
@@ -797,6 +980,19 @@ bool nat_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint64_t rows
 
 }  // namespace
 
+namespace {
+bool nat_attr_once() {
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(ffn_native_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(ffn_native_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+      return false;
+    attr_done = true;
+  }
+  return true;
+}
+}  // namespace
+
 bool native_shape_ok(const moe_shape_t& sh, const void* w13, const void* w2) {
   return native_batch_ok(sh) && sh.H <= kMaxK && sh.I <= kMaxK && sh.H % 512 == 0 && sh.I % 512 == 0 &&
          (reinterpret_cast<uintptr_t>(w13) & 15u) == 0 && (reinterpret_cast<uintptr_t>(w2) & 15u) == 0 &&
@@ -806,12 +1002,7 @@ bool native_shape_ok(const moe_shape_t& sh, const void* w13, const void* w2) {
 int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
                              const uint8_t* w2, const uint8_t* s2, const moe_shape_t& sh, void* scratch, float* y_perm,
                              int* status_word, cudaStream_t st) {
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(ffn_native_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
-      return MOE_ERR_CUDA;
-    attr_done = true;
-  }
+  if (!nat_attr_once()) return MOE_ERR_CUDA;
   const size_t S = static_cast<size_t>(sh.T) * sh.k;
   // scratch: term rows of the intermediate and of the token rows, each followed by its scale bytes; the counters
   uint8_t* aq2 = static_cast<uint8_t*>(scratch);
@@ -846,10 +1037,81 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
   a.H = sh.H;
   a.I = sh.I;
   a.S = static_cast<int>(S);
-  if (launch_pdl(ffn_native_kernel, dim3(sm_count()), dim3(kNatThreads), nat_smem(sh.E, sh.H > sh.I ? sh.H : sh.I).total + 1024,
-                 st, tm_w13, tm_s13, tm_a1, tm_w2, tm_s2, tm_a2, a) != cudaSuccess)
+  if (launch_pdl(ffn_native_kernel<false>, dim3(sm_count()), dim3(kNatThreads),
+                 nat_smem(sh.E, sh.H > sh.I ? sh.H : sh.I).total + 1024, st, tm_w13, tm_s13, tm_a1, tm_w2, tm_s2, tm_a2, a,
+                 FusedArgs{}) != cudaSuccess)
     return MOE_ERR_CUDA;
   note_kernel("ffn_native_mxf4_block_scaled", 2);
+  return MOE_OK;
+}
+
+// ---- the one-launch layer ----
+// Applies to a handful of tokens on shapes the native variant takes; the router's scratch (T rows of E logits)
+// borrows the shared memory that later holds the term rows' scale bytes.
+bool forward_fused_ok(const moe_shape_t& sh, const void* w13, const void* w2) {
+  const int K = sh.H > sh.I ? sh.H : sh.I;
+  return native_shape_ok(sh, w13, w2) && sh.T <= kFusedMaxTok && sh.T * sh.k <= kFusedMaxSlots &&
+         static_cast<size_t>(sh.T) * sh.E * 4 <= static_cast<size_t>(128) * (K / 32) && sh.E <= kSyncDone2 &&
+         sh.H / kTile <= kSyncExit - kSyncDone2;
+}
+int forward_fused_ctas() { return sm_count() < kFusedMaxCtas ? sm_count() : kFusedMaxCtas; }
+size_t forward_fused_scratch_bytes(const moe_shape_t& sh) {
+  const size_t S = static_cast<size_t>(sh.T) * sh.k, own = static_cast<size_t>(kFusedMaxCtas) * sh.T * kTerms;
+  return align_up(S * sh.H * 4, kAlign) + align_up(S * kTerms * (sh.I / 2), kAlign) + align_up(S * kTerms * (sh.I / 32), kAlign) +
+         align_up(own * (sh.H / 2), kAlign) + align_up(own * (sh.H / 32), kAlign);
+}
+int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const uint8_t* w13, const uint8_t* s13, const uint8_t* w2,
+                         const uint8_t* s2, const moe_shape_t& sh, __nv_bfloat16* out, int* ids_out, float* w_out, int* sync,
+                         void* scratch, int* status_word, cudaStream_t st) {
+  if (!nat_attr_once()) return MOE_ERR_CUDA;
+  const size_t S = static_cast<size_t>(sh.T) * sh.k;
+  const int grid = forward_fused_ctas();
+  const size_t own = static_cast<size_t>(kFusedMaxCtas) * sh.T * kTerms;
+  // scratch: per-slot output rows of the down projection, term rows of the intermediate with their scale bytes, and
+  // every CTA's term rows of the tokens with theirs
+  float* y = static_cast<float*>(scratch);
+  uint8_t* aq2 = reinterpret_cast<uint8_t*>(y) + align_up(S * sh.H * 4, kAlign);
+  uint8_t* sf2 = aq2 + align_up(S * kTerms * (sh.I / 2), kAlign);
+  uint8_t* aq1 = sf2 + align_up(S * kTerms * (sh.I / 32), kAlign);
+  uint8_t* sf1 = aq1 + align_up(own * (sh.H / 2), kAlign);
+  CUtensorMap tm_w13, tm_w2, tm_s13, tm_s2;
+  TermMaps tm_a1, tm_a2;
+  for (int i = 0; i < kTermBoxes; ++i)
+    if (!nat_map(&tm_a1.box[i], aq1, sh.H / 2, static_cast<uint64_t>(grid) * sh.T * kTerms, 128, 8u << i, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !nat_map(&tm_a2.box[i], aq2, sh.I / 2, S * kTerms, 128, 8u << i, CU_TENSOR_MAP_SWIZZLE_128B))
+      return MOE_ERR_CUDA;
+  if (!nat_map(&tm_w13, w13, sh.H / 2, static_cast<uint64_t>(sh.E) * 2 * sh.I, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !nat_map(&tm_w2, w2, sh.I / 2, static_cast<uint64_t>(sh.E) * sh.H, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !nat_map(&tm_s13, s13, sh.H / 32, static_cast<uint64_t>(sh.E) * 2 * sh.I, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+      !nat_map(&tm_s2, s2, sh.I / 32, static_cast<uint64_t>(sh.E) * sh.H, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE))
+    return MOE_ERR_CUDA;
+  NatArgs a;
+  a.sf1 = nullptr;
+  a.aq2 = aq2;
+  a.sf2 = sf2;
+  a.done = sync;
+  a.offsets = nullptr;
+  a.y = y;
+  a.status = status_word;
+  a.E = sh.E;
+  a.H = sh.H;
+  a.I = sh.I;
+  a.S = static_cast<int>(S);
+  FusedArgs f;
+  f.logits = logits;
+  f.x = x;
+  f.out = out;
+  f.ids_out = ids_out;
+  f.w_out = w_out;
+  f.aq1 = aq1;
+  f.sf1 = sf1;
+  f.sync = sync;
+  f.T = sh.T;
+  f.k = sh.k;
+  if (launch_pdl(ffn_native_kernel<true>, dim3(grid), dim3(kNatThreads), nat_smem(sh.E, sh.H > sh.I ? sh.H : sh.I).total + 1024, st,
+                 tm_w13, tm_s13, tm_a1, tm_w2, tm_s2, tm_a2, a, f) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  note_kernel("layer_one_launch_mxf4_block_scaled", 1);
   return MOE_OK;
 }
 

@@ -14,6 +14,7 @@ LIB_PATH = os.path.join(_HERE, "libmoe_b200.so")
 
 EXPORTS = ("moe_workspace_bytes", "moe_status_string", "moe_last_kernel_name", "moe_launch_count", "moe_route",
            "moe_permute", "moe_expert_ffn", "moe_combine", "moe_validate_scales",
+           "moe_forward_workspace_bytes", "moe_forward_sync_bytes", "moe_forward",
            "moe_forward_host_workspace_bytes", "moe_forward_host", "moe_expert_ffn_noalloc_max_bytes",
            "moe_expert_ffn_noalloc", "moe_debug_native_cta_share")
 
@@ -60,6 +61,12 @@ def lib():
         L.moe_expert_ffn_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp]
         L.moe_debug_native_cta_share.restype = C.c_int
         L.moe_debug_native_cta_share.argtypes = [i32, i32, i32, i32, i32, C.POINTER(C.c_int32)]
+        L.moe_forward_workspace_bytes.restype = sz
+        L.moe_forward_workspace_bytes.argtypes = [C.POINTER(Shape)]
+        L.moe_forward_sync_bytes.restype = sz
+        L.moe_forward_sync_bytes.argtypes = []
+        L.moe_forward.restype = C.c_int
+        L.moe_forward.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp, vp, vp, sz, vp]
         L.moe_forward_host.restype = C.c_int
         L.moe_forward_host.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp, sz, vp]
         _lib = L
@@ -151,6 +158,30 @@ def moe_combine(y_perm, inv_perm, topk_w, sh, out, stream=None):
 def moe_validate_scales(scales, bad_count, stream=None):
     _check(lib().moe_validate_scales(_ptr(scales), scales.numel(), _ptr(bad_count), _stream(stream)),
            "moe_validate_scales")
+
+
+def moe_forward_workspace_bytes(sh):
+    return int(lib().moe_forward_workspace_bytes(C.byref(sh)))
+
+
+def moe_forward_sync_bytes():
+    return int(lib().moe_forward_sync_bytes())
+
+
+def alloc_forward_workspace(sh, device="cuda"):
+    """Workspace of moe_forward with its counter block cleared (the one-time clear the call asks for)."""
+    n = moe_forward_workspace_bytes(sh)
+    if n == 0:
+        raise MoeError("unsupported shape")
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    ws[:moe_forward_sync_bytes()].zero_()
+    return ws
+
+
+def moe_forward(logits, x, w13, w13_scale, w2, w2_scale, sh, out, topk_ids, topk_w, status_word, ws, stream=None):
+    _check(lib().moe_forward(_ptr(logits), _ptr(x), _ptr(w13), _ptr(w13_scale), _ptr(w2), _ptr(w2_scale), C.byref(sh),
+                             _ptr(out), _ptr(topk_ids), _ptr(topk_w), _ptr(status_word), _ptr(ws), ws.numel(),
+                             _stream(stream)), "moe_forward")
 
 
 def moe_forward_host(logits_host, x_host, w13, w13_scale, w2, w2_scale, sh, out_host, status_word, ws, stream=None):
