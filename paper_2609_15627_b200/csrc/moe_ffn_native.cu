@@ -80,24 +80,27 @@ struct NatArgs {
 };
 
 // The one-launch layer (moe_forward on a handful of tokens): what the kernel needs beyond the expert FFN's arguments.
-// Every CTA routes all T tokens itself (same arithmetic, same result everywhere), sorts the T * k slots by expert in
-// shared memory and splits the T token rows into its own copy of their term rows; the gate/up items then take all T
-// tokens as operand rows (row = 8 * token + term) whatever their expert, and the epilogue keeps the tokens that were
-// routed to the item's expert.  After the down projection the CTA that runs the last expert's item of a column tile
+// Every CTA routes all T tokens itself (same arithmetic, same result everywhere) and sorts the T * k slots by expert in
+// shared memory, so its weight stream starts without waiting for anyone.  The first kSplitCtas CTAs meanwhile split
+// the T token rows into E2M1 term rows, a few 32-element blocks each, and count themselves in; the term-row loads of
+// the gate/up items wait for that count (CTAs are handed out in index order, so those CTAs are running).  The gate/up
+// items take all T tokens as operand rows (row = 8 * token + term) whatever their expert, and the epilogue keeps the
+// tokens that were routed to the item's expert.  After the down projection the CTA that runs the last expert's item of a column tile
 // reduces that tile over the slots of every token.
 constexpr int kFusedMaxTok = 4;    // tokens of a fused call: one lane quadrant of operand rows
 constexpr int kFusedMaxSlots = 32; // T * k: one warp sorts them
-constexpr int kFusedMaxCtas = 256; // the scratch holds this many CTAs' term rows (more SMs than that: a smaller grid)
 constexpr int kSyncDone2 = 1024;   // int index in the sync block: per column tile, warps that stored a down item
 constexpr int kSyncExit = 1024 + 64;  // CTAs that have finished; the last one clears the block
+constexpr int kSyncSplit = 1024 + 65; // CTAs that have written their share of the tokens' term rows
+constexpr int kSplitCtas = 32;
 struct FusedArgs {
   const float* logits;       // [T, E]
   const __nv_bfloat16* x;    // [T, H]
   __nv_bfloat16* out;        // [T, H]
   int* ids_out;              // [T, k] or null
   float* w_out;              // [T, k] or null
-  uint8_t* aq1;              // [grid][T * 8, H/2] each CTA's term rows of the tokens
-  uint8_t* sf1;              // [grid][T * 8, H/32]
+  uint8_t* aq1;              // [T * 8, H/2] term rows of the tokens
+  uint8_t* sf1;              // [T * 8, H/32]
   int* sync;                 // sync block: [0, E) = NatArgs::done, then the indices above; zero between calls
   int T, k;
 };
@@ -419,6 +422,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   if constexpr (kFused) {
     // ---- the layer's first steps, the same in every CTA: route, sort the slots, split the token rows ----
     pdl_wait();  // logits and token rows may come from the kernel before this one; the sync block is clear
+    const int n_split = min(static_cast<int>(gridDim.x), kSplitCtas);
     if (wid >= 2 && wid < 6) {
       // one warp per token: top-k by logit (ties to the lower expert), softmax over the selected logits
       const int t = wid - 2;
@@ -437,35 +441,30 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
           if (blockIdx.x == 0 && f.w_out != nullptr) f.w_out[t * f.k + lane] = wt;
         }
       }
-    } else {
-      // the other six warps: token rows -> this CTA's term rows, four 32-element blocks per group of 8 lanes at a
-      // time; a warp takes 16 consecutive blocks per round, so its lanes run the same number of rounds
-      const int sw = wid < 2 ? wid : wid - 4;  // 0..5
+    } else if (wid != 0 && static_cast<int>(blockIdx.x) < n_split) {
+      // warps 1 and 6..9 of the first CTAs: token rows -> term rows, one 32-element block per group of 8 lanes;
+      // CTA c takes blocks c, c + n_split, ... (at most 16 of them: one round)
+      const int sw = wid == 1 ? 0 : wid - 5;  // 0..4
       const int n_blk = a.H / 32, n_all = f.T * n_blk;
-      uint8_t* my_aq = f.aq1 + static_cast<size_t>(blockIdx.x) * f.T * kTerms * (a.H / 2);
-      uint8_t* my_sf = f.sf1 + static_cast<size_t>(blockIdx.x) * f.T * kTerms * n_blk;
       const int sub = lane & 7;
-      for (int b0 = sw * 16 + (lane >> 3) * 4; b0 < n_all; b0 += 6 * 16) {
-        float r[4][4];
-#pragma unroll
-        for (int nb = 0; nb < 4; ++nb) {
-          const int b = b0 + nb, t = b / n_blk, blk = b % n_blk;
-          const uint2 v = *reinterpret_cast<const uint2*>(f.x + static_cast<size_t>(t) * a.H + blk * 32 + sub * 4);
-          r[nb][0] = __uint_as_float(v.x << 16);
-          r[nb][1] = __uint_as_float(v.x & 0xFFFF0000u);
-          r[nb][2] = __uint_as_float(v.y << 16);
-          r[nb][3] = __uint_as_float(v.y & 0xFFFF0000u);
-        }
-        split_terms<4>(r, [&](int nb, int t8, uint32_t bytes, int se) {
-          const int b = b0 + nb, t = b / n_blk, blk = b % n_blk;
+      const int b = static_cast<int>(blockIdx.x) + n_split * (sw * 4 + (lane >> 3));
+      const bool live = b < n_all;
+      const int t = live ? b / n_blk : 0, blk = live ? b % n_blk : 0;
+      const uint2 v = *reinterpret_cast<const uint2*>(f.x + static_cast<size_t>(t) * a.H + blk * 32 + sub * 4);
+      float r[1][4] = {{__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u), __uint_as_float(v.y << 16),
+                       __uint_as_float(v.y & 0xFFFF0000u)}};
+      split_terms<1>(r, [&](int, int t8, uint32_t bytes, int se) {
+        if (live) {
           const size_t trow = static_cast<size_t>(t) * kTerms + t8;
-          *reinterpret_cast<uint16_t*>(my_aq + trow * (a.H / 2) + blk * 16 + sub * 2) = static_cast<uint16_t>(bytes);
-          if (sub == 0) my_sf[trow * n_blk + blk] = static_cast<uint8_t>(se + 127);
-        });
-      }
+          *reinterpret_cast<uint16_t*>(f.aq1 + trow * (a.H / 2) + blk * 16 + sub * 2) = static_cast<uint16_t>(bytes);
+          if (sub == 0) f.sf1[trow * n_blk + blk] = static_cast<uint8_t>(se + 127);
+        }
+      });
       fence_proxy_async_all();  // TMA will read these rows
     }
     __syncthreads();
+    if (tid == 32 && static_cast<int>(blockIdx.x) < n_split)
+      asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(f.sync + kSyncSplit) : "memory");
     if (wid == 2) {
       // Stable sort of the slots by expert, S <= 32: lane s is slot s.  Its sorted row = slots of smaller experts +
       // earlier slots of its own expert; the touched experts are the distinct ids in ascending order.
@@ -515,8 +514,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       // The weights depend on nothing, the term rows do: on the split kernel (phase 0) or on the gate/up items of
       // their expert (phase 1).  While a dependency is open, the weight loads go out and the term-row loads of up to
       // kWStages steps are held back; they follow once the dependency is met.
-      // (one-launch layer: the gate/up items read this CTA's own term rows, complete since the set-up)
-      bool pdl_done = kFused, dep_ok = kFused;
+      // (one-launch layer: the gate/up items' dependency is the count of CTAs that have split the tokens)
+      bool pdl_done = kFused, dep_ok = false;
       int dep_phase = 0, dep_e = -1;
       int n_pend = 0, pend_s[kWStages], pend_x[kWStages], pend_y[kWStages], pend_b[kWStages];
       // term rows of one K step; a pass of at most kRepTok tokens gets them once per lane quadrant of the accumulator
@@ -529,6 +528,10 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         if (!pdl_done) {
           pdl_wait();  // the split kernel is complete: term rows of the tokens, cleared counters
           pdl_done = true;
+        }
+        if (kFused && dep_phase == 0) {
+          counter_wait_ge(f.sync + kSyncSplit, min(static_cast<int>(gridDim.x), kSplitCtas), a.status);
+          fence_proxy_async_all();
         }
         if (dep_phase == 1) {
           counter_wait_ge(a.done + dep_e, need_done, a.status);
@@ -559,7 +562,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             dep_ok = false;
           }
           for (int pass = 0; pass < n_pass; ++pass) {
-            const bool own_rows = kFused && phase == 0;  // all T tokens, from this CTA's copy
+            const bool own_rows = kFused && phase == 0;  // all T tokens
             const int bi = term_box(own_rows ? f.T : min(tok_pass, n_rows_e - pass * tok_pass));  // box of 8 << bi term rows
             for (int ks = 0; ks < P.n_steps; ++ks) {
               if ((ks & 1) == 0) {  // 16 scale bytes per weight row cover two K steps
@@ -574,7 +577,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
               tma_load_2d(sW + s * kStage, mw, ks * 128, wrow_a, &full_w[s]);
               tma_load_2d(sW + s * kStage + 128 * 128, mw, ks * 128, wrow_b, &full_w[s]);
               // the pass's term rows (8 per token, consecutive); rows past the end of the tensor arrive as zeros
-              const int arow = own_rows ? static_cast<int>(blockIdx.x) * f.T * kTerms : (row_begin + pass * tok_pass) * kTerms;
+              const int arow = own_rows ? 0 : (row_begin + pass * tok_pass) * kTerms;
               if (dep_ok) {
                 load_terms(ma, s, bi, ks * 128, arow);
               } else {
@@ -678,9 +681,12 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
               // every gate/up item of this expert has published its rows of the intermediate
               if (st == 0) counter_wait_ge(a.done + touched[ti], need_done, a.status);
               asm volatile("bar.sync 3, 128;" ::: "memory");
+            } else if (kFused) {
+              if (st == 0) counter_wait_ge(f.sync + kSyncSplit, min(static_cast<int>(gridDim.x), kSplitCtas), a.status);
+              asm volatile("bar.sync 3, 128;" ::: "memory");
             }
             const bool own_rows = kFused && phase == 0;
-            const int row0 = own_rows ? static_cast<int>(blockIdx.x) * f.T : row_begin + pass * tok_pass;
+            const int row0 = own_rows ? 0 : row_begin + pass * tok_pass;
             const int n_rows = (own_rows ? f.T : min(tok_pass, row_end - row0)) * kTerms;  // term rows that exist
             const bool rep = n_rows <= kRepTok * kTerms;                // the operand repeats in every lane quadrant
             // rows are n_blk bytes each and consecutive: one contiguous range, copied 16 bytes at a time
@@ -888,14 +894,14 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
                 const int col = tile * kTile + (wid - kEpiWarp) * 64 + lane * 2;
                 for (int t = 0; t < f.T; ++t) {
                   float2 acc = make_float2(0.0f, 0.0f);
-                  for (int j0 = 0; j0 < f.k; j0 += 4) {  // four slots' loads in flight; the multiply-adds stay in slot order
-                    float2 v[4];
+                  for (int j0 = 0; j0 < f.k; j0 += 8) {  // eight slots' loads in flight; the multiply-adds stay in slot order
+                    float2 v[8];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u)
+                    for (int u = 0; u < 8; ++u)
                       if (j0 + u < f.k)
                         v[u] = __ldcg(reinterpret_cast<const float2*>(a.y + static_cast<size_t>(s_row[t * f.k + j0 + u]) * a.H + col));
 #pragma unroll
-                    for (int u = 0; u < 4; ++u)
+                    for (int u = 0; u < 8; ++u)
                       if (j0 + u < f.k) {
                         const float wj = s_w[t * f.k + j0 + u];
                         acc.x = __fmaf_rn(wj, v[u].x, acc.x);
@@ -940,7 +946,10 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         __threadfence();
         for (int i = lane; i < a.E; i += 32) f.sync[i] = 0;
         for (int i = lane; i < a.H / kTile; i += 32) f.sync[kSyncDone2 + i] = 0;
-        if (lane == 0) f.sync[kSyncExit] = 0;
+        if (lane == 0) {
+          f.sync[kSyncExit] = 0;
+          f.sync[kSyncSplit] = 0;
+        }
       }
     }
   }
@@ -1050,13 +1059,12 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
 // borrows the shared memory that later holds the term rows' scale bytes.
 bool forward_fused_ok(const moe_shape_t& sh, const void* w13, const void* w2) {
   const int K = sh.H > sh.I ? sh.H : sh.I;
-  return native_shape_ok(sh, w13, w2) && sh.T <= kFusedMaxTok && sh.T * sh.k <= kFusedMaxSlots &&
+  return native_shape_ok(sh, w13, w2) && sm_count() >= kSplitCtas && sh.T <= kFusedMaxTok && sh.T * sh.k <= kFusedMaxSlots &&
          static_cast<size_t>(sh.T) * sh.E * 4 <= static_cast<size_t>(128) * (K / 32) && sh.E <= kSyncDone2 &&
-         sh.H / kTile <= kSyncExit - kSyncDone2;
+         sh.H / kTile <= kSyncExit - kSyncDone2 && static_cast<size_t>(sh.T) * (sh.H / 32) <= static_cast<size_t>(kSplitCtas) * 16;
 }
-int forward_fused_ctas() { return sm_count() < kFusedMaxCtas ? sm_count() : kFusedMaxCtas; }
 size_t forward_fused_scratch_bytes(const moe_shape_t& sh) {
-  const size_t S = static_cast<size_t>(sh.T) * sh.k, own = static_cast<size_t>(kFusedMaxCtas) * sh.T * kTerms;
+  const size_t S = static_cast<size_t>(sh.T) * sh.k, own = static_cast<size_t>(sh.T) * kTerms;
   return align_up(S * sh.H * 4, kAlign) + align_up(S * kTerms * (sh.I / 2), kAlign) + align_up(S * kTerms * (sh.I / 32), kAlign) +
          align_up(own * (sh.H / 2), kAlign) + align_up(own * (sh.H / 32), kAlign);
 }
@@ -1065,10 +1073,10 @@ int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const uint
                          void* scratch, int* status_word, cudaStream_t st) {
   if (!nat_attr_once()) return MOE_ERR_CUDA;
   const size_t S = static_cast<size_t>(sh.T) * sh.k;
-  const int grid = forward_fused_ctas();
-  const size_t own = static_cast<size_t>(kFusedMaxCtas) * sh.T * kTerms;
+  const int grid = sm_count();
+  const size_t own = static_cast<size_t>(sh.T) * kTerms;
   // scratch: per-slot output rows of the down projection, term rows of the intermediate with their scale bytes, and
-  // every CTA's term rows of the tokens with theirs
+  // the term rows of the tokens with theirs
   float* y = static_cast<float*>(scratch);
   uint8_t* aq2 = reinterpret_cast<uint8_t*>(y) + align_up(S * sh.H * 4, kAlign);
   uint8_t* sf2 = aq2 + align_up(S * kTerms * (sh.I / 2), kAlign);
@@ -1077,7 +1085,7 @@ int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const uint
   CUtensorMap tm_w13, tm_w2, tm_s13, tm_s2;
   TermMaps tm_a1, tm_a2;
   for (int i = 0; i < kTermBoxes; ++i)
-    if (!nat_map(&tm_a1.box[i], aq1, sh.H / 2, static_cast<uint64_t>(grid) * sh.T * kTerms, 128, 8u << i, CU_TENSOR_MAP_SWIZZLE_128B) ||
+    if (!nat_map(&tm_a1.box[i], aq1, sh.H / 2, own, 128, 8u << i, CU_TENSOR_MAP_SWIZZLE_128B) ||
         !nat_map(&tm_a2.box[i], aq2, sh.I / 2, S * kTerms, 128, 8u << i, CU_TENSOR_MAP_SWIZZLE_128B))
       return MOE_ERR_CUDA;
   if (!nat_map(&tm_w13, w13, sh.H / 2, static_cast<uint64_t>(sh.E) * 2 * sh.I, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||

@@ -26,40 +26,46 @@ MOE_DEVINL float exp_fixed(float d) {
 }
 
 // One warp per token.  row = this warp's copy of the token's logits in shared memory.
-// Returns through lane j (< k) the j-th selected expert and its logit.
+// Returns through lane j (< k) the j-th selected expert and its logit: experts in the order (logit descending by
+// IEEE comparison, so -0 ties with +0; expert id ascending among equals).
 MOE_DEVINL void warp_topk(const float* row, int E, int k, int lane, int* my_id, float* my_v) {
   unsigned taken = 0u;  // bit i: element lane + 32*i already selected
   *my_id = 0;
   *my_v = 0.0f;
   for (int j = 0; j < k; ++j) {
+    // this lane's best remaining element; strict '>': the lowest id among this lane's equal values stays
     float bv = 0.0f;
     int bi = -1;
-    for (int i = 0; i * 32 + lane < E; ++i) {
-      if (!((taken >> i) & 1u)) {
-        const float v = row[i * 32 + lane];
-        if (bi < 0 || v > bv) {  // strict '>': the lowest id among this lane's equal values stays
-          bv = v;
-          bi = i * 32 + lane;
+    for (int i0 = 0; i0 * 32 < E; i0 += 8) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int idx = (i0 + u) * 32 + lane;
+        v[u] = idx < E ? row[idx] : 0.0f;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int idx = (i0 + u) * 32 + lane;
+        if (idx < E && !((taken >> (i0 + u)) & 1u) && (bi < 0 || v[u] > bv)) {
+          bv = v[u];
+          bi = idx;
         }
       }
     }
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, bv, d);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, d);
-      const bool take = (oi >= 0) && (bi < 0 || ov > bv || (ov == bv && oi < bi));
-      if (take) {
-        bv = ov;
-        bi = oi;
-      }
+    // the warp's best: the largest value (as an integer key that orders floats, -0 counted as +0), then the lowest
+    // id among the lanes that hold it; a lane with nothing left sends the lowest key and no id
+    unsigned key = 0u;
+    if (bi >= 0) {
+      const unsigned u = __float_as_uint(bv == 0.0f ? 0.0f : bv);
+      key = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
     }
-    // lane 0's view is authoritative (identical on all lanes for finite logits)
-    bi = __shfl_sync(0xffffffffu, bi, 0);
-    bv = __shfl_sync(0xffffffffu, bv, 0);
-    if (bi >= 0 && (bi & 31) == lane) taken |= 1u << (bi >> 5);
+    const unsigned best_key = __reduce_max_sync(0xffffffffu, key);
+    const unsigned win = __reduce_min_sync(0xffffffffu, (bi >= 0 && key == best_key) ? static_cast<unsigned>(bi) : 0xffffffffu);
+    const float win_v = __shfl_sync(0xffffffffu, bv, static_cast<int>(win & 31u));
+    if ((win & 31u) == static_cast<unsigned>(lane)) taken |= 1u << (win >> 5);
     if (lane == j) {
-      *my_id = bi;
-      *my_v = bv;
+      *my_id = static_cast<int>(win);
+      *my_v = win_v;
     }
   }
 }
