@@ -82,8 +82,8 @@ struct NatArgs {
 // The one-launch layer (moe_forward on a handful of tokens): what the kernel needs beyond the expert FFN's arguments.
 // Every CTA routes all T tokens itself (same arithmetic, same result everywhere) and sorts the T * k slots by expert in
 // shared memory, so its weight stream starts without waiting for anyone.  The first kSplitCtas CTAs meanwhile split
-// the T token rows into E2M1 term rows, a few 32-element blocks each, and count themselves in; the term-row loads of
-// the gate/up items wait for that count (CTAs are handed out in index order, so those CTAs are running).  The gate/up
+// the T token rows into E2M1 term rows, a few 32-element blocks each, and count themselves in; every CTA sees that
+// count complete before its set-up ends (CTAs are handed out in index order, so those CTAs are running).  The gate/up
 // items take all T tokens as operand rows (row = 8 * token + term) whatever their expert, and the epilogue keeps the
 // tokens that were routed to the item's expert.  After the down projection the CTA that runs the last expert's item of a column tile
 // reduces that tile over the slots of every token.
@@ -428,7 +428,19 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       const int t = wid - 2;
       if (t < f.T) {
         float* row = reinterpret_cast<float*>(sSfa) + t * a.E;  // this region is not in use yet
-        for (int e = lane; e < a.E; e += 32) row[e] = f.logits[static_cast<size_t>(t) * a.E + e];
+        for (int e0 = 0; e0 < a.E; e0 += 256) {  // eight loads in flight per lane
+          float lv[8];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int e = e0 + 32 * u + lane;
+            lv[u] = e < a.E ? __ldg(f.logits + static_cast<size_t>(t) * a.E + e) : 0.0f;
+          }
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int e = e0 + 32 * u + lane;
+            if (e < a.E) row[e] = lv[u];
+          }
+        }
         __syncwarp();
         int my_id;
         float my_v;
@@ -461,10 +473,12 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         }
       });
       fence_proxy_async_all();  // TMA will read these rows
+      asm volatile("bar.sync 2, 160;" ::: "memory");  // the five splitting warps
+      if (tid == 32) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(f.sync + kSyncSplit) : "memory");
     }
+    // the term rows are complete long before the routing above is: one thread makes sure while it runs
+    if (tid == 32) counter_wait_ge(f.sync + kSyncSplit, n_split, a.status);
     __syncthreads();
-    if (tid == 32 && static_cast<int>(blockIdx.x) < n_split)
-      asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(f.sync + kSyncSplit) : "memory");
     if (wid == 2) {
       // Stable sort of the slots by expert, S <= 32: lane s is slot s.  Its sorted row = slots of smaller experts +
       // earlier slots of its own expert; the touched experts are the distinct ids in ascending order.
@@ -514,8 +528,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       // The weights depend on nothing, the term rows do: on the split kernel (phase 0) or on the gate/up items of
       // their expert (phase 1).  While a dependency is open, the weight loads go out and the term-row loads of up to
       // kWStages steps are held back; they follow once the dependency is met.
-      // (one-launch layer: the gate/up items' dependency is the count of CTAs that have split the tokens)
-      bool pdl_done = kFused, dep_ok = false;
+      // (one-launch layer: the tokens' term rows were seen complete during the set-up)
+      bool pdl_done = kFused, dep_ok = kFused;
+      if (kFused) fence_proxy_async_all();  // they were written through the generic proxy
       int dep_phase = 0, dep_e = -1;
       int n_pend = 0, pend_s[kWStages], pend_x[kWStages], pend_y[kWStages], pend_b[kWStages];
       // term rows of one K step; a pass of at most kRepTok tokens gets them once per lane quadrant of the accumulator
@@ -528,10 +543,6 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         if (!pdl_done) {
           pdl_wait();  // the split kernel is complete: term rows of the tokens, cleared counters
           pdl_done = true;
-        }
-        if (kFused && dep_phase == 0) {
-          counter_wait_ge(f.sync + kSyncSplit, min(static_cast<int>(gridDim.x), kSplitCtas), a.status);
-          fence_proxy_async_all();
         }
         if (dep_phase == 1) {
           counter_wait_ge(a.done + dep_e, need_done, a.status);
@@ -680,9 +691,6 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             if (phase == 1) {
               // every gate/up item of this expert has published its rows of the intermediate
               if (st == 0) counter_wait_ge(a.done + touched[ti], need_done, a.status);
-              asm volatile("bar.sync 3, 128;" ::: "memory");
-            } else if (kFused) {
-              if (st == 0) counter_wait_ge(f.sync + kSyncSplit, min(static_cast<int>(gridDim.x), kSplitCtas), a.status);
               asm volatile("bar.sync 3, 128;" ::: "memory");
             }
             const bool own_rows = kFused && phase == 0;
