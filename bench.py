@@ -1,7 +1,9 @@
 """Benchmark of the routed FP4 mixture-of-experts layer on B200.
 
 A step is one pass of the whole hot path (moe_route -> moe_permute -> moe_expert_ffn -> moe_combine)
-over one batch of seeded synthetic input.  Prints ONE JSON line (rank 0).
+over one batch of seeded synthetic input.  For a handful of tokens (decode_c1) the library runs that path
+as ONE kernel launch behind moe_forward; the step is then that call, and the four calls are timed beside
+it.  Prints ONE JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
 
@@ -28,6 +30,7 @@ DECODE = ("decode_c1", "decode_c64")
 # dram__bytes_read.sum + dram__bytes_write.sum per moe_expert_ffn call from one ncu capture of the
 # workload (see profiles/); None until captured.
 NCU_TRAFFIC_BYTES = {
+    "decode_c1_one_launch": None,  # ffn_native_kernel<true>, the whole layer
     "decode_c1": 111177216,      # ffn_native_kernel: 107.21 MB read + 3.97 MB written (profiles/ffn_native_decode.md)
     "decode_c64": 3060525584,    # 3041.8 MB read + 18.8 MB written
     "prefill_8k": 5611119000,    # ffn_umma_kernel<true> 2.882 + 0.263 GB, <false> 1.431 + 1.034 GB (profiles/ffn_umma_prefill_8k.md)
@@ -43,6 +46,12 @@ def ffn_algorithmic_bytes(wl, n_touched):
     sorted activations in, the bf16 intermediate out and back in, the fp32 per-slot rows out."""
     S = wl.T * wl.k
     return n_touched * expert_weight_bytes(wl.H, wl.I) + S * wl.H * 2 + 2 * S * wl.I * 2 + S * wl.H * 4
+
+
+def layer_algorithmic_bytes(wl, n_touched):
+    """Bytes the whole layer must move when nothing between its steps is materialised: each touched
+    expert's packed codes and scale bytes once, logits and token rows in, the output rows out."""
+    return n_touched * expert_weight_bytes(wl.H, wl.I) + wl.T * wl.E * 4 + 2 * wl.T * wl.H * 2
 
 
 def ffn_flops(wl):
@@ -184,7 +193,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--no-graph", action="store_true", help="decode workloads: launch the four calls eagerly instead of replaying CUDA graphs")
+    ap.add_argument("--no-graph", action="store_true", help="decode workloads: launch the calls eagerly instead of replaying CUDA graphs")
+    ap.add_argument("--four-calls", action="store_true", help="time the four calls even where moe_forward is one launch")
     args = ap.parse_args()
 
     from paper_2609_15627_b200 import inputs
@@ -241,7 +251,13 @@ def main():
         off = buf.expert_offsets.cpu().numpy()
         touched.append(int(np.count_nonzero(np.diff(off))))
 
-    def step(i, ev=None, st=stream):
+    # Does moe_forward run this shape as one launch?  (Asked of the library: one call, then the name of its kernel.)
+    fws = moe.alloc_forward_workspace(sh)
+    moe.moe_forward(batches[0][0], batches[0][1], *weights, sh, buf.out, None, None, buf.status, fws, stream)
+    torch.cuda.synchronize()
+    one_launch = moe.moe_last_kernel_name().startswith("layer_one_launch") and not args.four_calls
+
+    def step4(i, ev=None, st=stream):
         """The four C-ABI calls on batch i of the cycle (st=None: torch's current stream, used during capture)."""
         l, x = batches[i % n_cycle]
         moe.moe_route(l, wl.k, buf.topk_ids, buf.topk_w, buf.expert_offsets, buf.ws, st)
@@ -252,6 +268,13 @@ def main():
         if ev is not None:
             ev[1].record(st)
         moe.moe_combine(buf.y_perm, buf.inv_perm, buf.topk_w, sh, buf.out, st)
+
+    def step1(i, ev=None, st=stream):
+        """The same path as one call (one kernel launch for this shape)."""
+        l, x = batches[i % n_cycle]
+        moe.moe_forward(l, x, *weights, sh, buf.out, None, None, buf.status, fws, st)
+
+    step = step1 if one_launch else step4
 
     def barrier():
         if world > 1:
@@ -313,7 +336,7 @@ def main():
             graphs[i % n_cycle].replay()
     else:
         for i in range(args.steps):
-            step(i, inner[i] if i < n_inner else None)
+            step(i, inner[i] if i < n_inner and not one_launch else None)
     e1.record(stream)
     barrier()
     clocks = sampler.stop()
@@ -323,16 +346,48 @@ def main():
     ms_step = ms_total / args.steps
     value = wl.T * world / (ms_step * 1e-3)
     eager_ms_step = None
-    if use_graph:
-        # the expert-FFN call cannot be bracketed by events inside a graph: time it in a second region of eager
-        # steps on the same batches, right after the timed one
+    if use_graph or one_launch:
+        # the expert-FFN call cannot be bracketed by events inside a graph (nor inside the one-launch layer): time it
+        # in a second region of eager steps of the four calls on the same batches, right after the timed one
+        for i in range(3):
+            step4(i)
+        barrier()
         ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ee0.record(stream)
         for i in range(n_inner):
-            step(i, inner[i])
+            step4(i, inner[i])
         ee1.record(stream)
         barrier()
         eager_ms_step = ee0.elapsed_time(ee1) / n_inner
+
+    # ---- one-launch workloads: the four calls, graph-replayed the same way, for comparison -----------------------
+    four_calls_ms_step = None
+    if one_launch and use_graph:
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            for i in range(3):
+                step4(i, st=None)
+        stream.wait_stream(side)
+        barrier()
+        mg4 = []
+        for i0 in range(0, n_cycle, kGraphSteps):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for i in range(i0, i0 + kGraphSteps):
+                    step4(i, st=None)
+            mg4.append(g)
+        for g in mg4:
+            g.replay()
+        barrier()
+        n4 = max(len(mg4), min(args.steps // kGraphSteps, 64))
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record(stream)
+        for i in range(n4):
+            mg4[i % len(mg4)].replay()
+        g1.record(stream)
+        barrier()
+        four_calls_ms_step = g0.elapsed_time(g1) / (n4 * kGraphSteps)
 
     # ---- the expert-FFN call alone, graph-replayed like the step (calls shorter than 100 us) -------------------------
     # Eager launches of kernels this short leave the GPU idle between the event and the launch, which the bracketing
@@ -399,8 +454,18 @@ def main():
                  "ms": ffn_ms, "peak_source": peaks["source"], "experts_touched": mean_touched,
                  "timed_in": ("graph replays of the call alone, one graph per batch of the cycle, right after the timed region"
                               if ffn_graph_ms is not None else
-                              ("eager steps right after the graph-replayed region" if use_graph else "the timed region")),
+                              ("eager steps right after the graph-replayed region" if use_graph or one_launch else "the timed region")),
                  "ms_between_events_in_eager_steps": ffn_eager_ms})
+    if one_launch:
+        # the dominant kernel is the step itself: one launch per step, timed by the events of the timed region
+        touched_steps = float(np.mean([touched[i % n_cycle] for i in range(args.steps)]))
+        alg = layer_algorithmic_bytes(wl, touched_steps)
+        achieved = alg / (ms_step * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"],
+                "traffic": NCU_TRAFFIC_BYTES.get(wl.name + "_one_launch"), "algorithmic_bytes": alg,
+                "kernel": "moe_forward (route, term split, expert FFN and combine in one launch)", "ms": ms_step,
+                "peak_source": peaks["source"], "experts_touched": touched_steps, "timed_in": "the timed region",
+                "four_calls": {"ms_per_step": four_calls_ms_step, "eager_ms_per_step": eager_ms_step, "expert_ffn": roof}}
 
     # ---- end to end through the host-buffer entry point ---------------------------------------------------------
     e2e = None
@@ -437,8 +502,9 @@ def main():
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": wl.name, "T": wl.T, "H": wl.H, "I": wl.I, "E": wl.E, "k": wl.k,
                        "parallelism": "replicas only" if world > 1 else "1 GPU",
+                       "call": "moe_forward (one kernel launch per step)" if one_launch else "moe_route, moe_permute, moe_expert_ffn, moe_combine",
                        "launch": "cuda graph replay, %d consecutive batches of the cycle per graph" % kGraphSteps if use_graph else "eager",
-                       "eager_ms_per_step": eager_ms_step,
+                       "eager_ms_per_step": None if one_launch else eager_ms_step,
                        "l2": "inputs cycle over %d seeded batches; %.2f GB of expert weights resident (larger than L2)"
                              % (n_cycle, wl.E * expert_weight_bytes(wl.H, wl.I) / 1e9)},
             "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,

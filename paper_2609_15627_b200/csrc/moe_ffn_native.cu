@@ -476,9 +476,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       asm volatile("bar.sync 2, 160;" ::: "memory");  // the five splitting warps
       if (tid == 32) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(f.sync + kSyncSplit) : "memory");
     }
-    // the term rows are complete long before the routing above is: one thread makes sure while it runs
-    if (tid == 32) counter_wait_ge(f.sync + kSyncSplit, n_split, a.status);
     __syncthreads();
+    // the term rows are complete by the time the routing above is: one thread makes sure while the slots are sorted
+    if (tid == 32) counter_wait_ge(f.sync + kSyncSplit, n_split, a.status);
     if (wid == 2) {
       // Stable sort of the slots by expert, S <= 32: lane s is slot s.  Its sorted row = slots of smaller experts +
       // earlier slots of its own expert; the touched experts are the distinct ids in ascending order.

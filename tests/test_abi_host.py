@@ -60,6 +60,28 @@ def test_argument_errors_are_found_on_the_host(L):
     assert L.moe_combine(fake, fake, fake, None, fake, null) == 1
     assert L.moe_validate_scales(null, 16, fake, null) == 1
     assert L.moe_forward_host(null, fake, fake, fake, fake, fake, C.byref(sh), fake, null, fake, 1 << 30, null) == 1
+    big = C.c_void_p(0x10000)
+    assert L.moe_forward(null, fake, fake, fake, fake, fake, C.byref(sh), fake, null, null, null, big, 1 << 30, null) == 1
+    assert L.moe_forward(fake, fake, fake, fake, fake, fake, C.byref(sh), odd, null, null, null, big, 1 << 30, null) == 1
+    assert L.moe_forward(fake, fake, fake, fake, fake, fake, C.byref(sh), fake, odd, null, null, big, 1 << 30, null) == 1   # topk_ids
+    assert L.moe_forward(fake, fake, fake, fake, fake, fake, C.byref(bad), fake, null, null, null, big, 1 << 30, null) == 2
+    assert L.moe_forward(fake, fake, fake, fake, fake, fake, C.byref(sh), fake, null, null, null, big, 64, null) == 3
+    assert L.moe_forward(fake, fake, fake, fake, fake, fake, C.byref(sh), fake, null, null, null, null, 1 << 30, null) == 3
+
+
+def test_forward_workspace_sizes(L):
+    """The workspace of moe_forward: the counter block, then room for the one-launch scratch or the four calls' buffers."""
+    sync = moe.moe_forward_sync_bytes()
+    assert sync >= 4 * (1024 + 64 + 2) and sync % 256 == 0
+    for T, H, I, E, k in ((1, 4096, 2048, 256, 8), (4, 4096, 2048, 256, 8), (64, 4096, 2048, 256, 8), (16, 256, 128, 8, 2)):
+        sh = moe.shape(T, H, I, E, k)
+        S = T * k
+        n = moe.moe_forward_workspace_bytes(sh)
+        four = S * H * 2 + S * H * 4 + moe.moe_workspace_bytes(sh)        # x_perm, y_perm, the calls' own workspace
+        one = S * H * 4 + 8 * S * (I // 2 + I // 32) + 8 * T * (H // 2 + H // 32)
+        assert n >= sync + four and n >= sync + one and n % 256 == 0
+        assert moe.moe_forward_host_workspace_bytes(sh) >= n + T * E * 4 + 2 * T * H * 2
+    assert moe.moe_forward_workspace_bytes(moe.shape(64, 4000, 2048, 256, 8)) == 0
 
 
 def test_missing_library_fails_loudly(monkeypatch):

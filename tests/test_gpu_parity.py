@@ -327,6 +327,124 @@ def test_layer_decode_full(name, prod_weights):
     _check_layer_full(wl, d, wdev)
 
 
+# ---- moe_forward: the whole layer as one call (one kernel launch for a handful of tokens) -------------------
+
+_ONE_LAUNCH = "layer_one_launch_mxf4_block_scaled"
+
+
+def _run_forward(wl, d, wdev, reps=1):
+    sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
+    ws = moe.alloc_forward_workspace(sh)
+    out = torch.empty((wl.T, wl.H), dtype=torch.bfloat16, device="cuda")
+    ids = torch.empty((wl.T, wl.k), dtype=torch.int32, device="cuda")
+    w = torch.empty((wl.T, wl.k), dtype=torch.float32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    lg, x = dev(d["logits"]), dev(d["x"])
+    for _ in range(reps):
+        out.fill_(float("nan"))
+        moe.moe_forward(lg, x, *wdev, sh, out, ids, w, st, ws)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0
+        # the counter block is left clear for the next call
+        assert int(ws[:moe.moe_forward_sync_bytes()].view(torch.int32).abs().sum().item()) == 0
+    return out, ids, w, moe.moe_last_kernel_name()
+
+
+def _check_forward(wl, d, wdev, one_launch):
+    wdev = wdev if wdev is not None else weights_dev(d)
+    out, ids, w, kernel = _run_forward(wl, d, wdev, reps=3)
+    assert (kernel == _ONE_LAUNCH) == one_launch, kernel
+    # against the oracle: routing bit for bit, the output within the stated tolerance
+    r = O.forward_staged(d["logits"], d["x"], d["w13"], d["s13"], d["w2"], d["s2"], wl.k)
+    assert np.array_equal(ids.cpu().numpy(), r["ids"])
+    assert np.array_equal(w.cpu().numpy().view(np.uint32), r["w"].view(np.uint32))
+    check_out(bits(out), r["out"], r["out_f32"], wl.name)
+    # against the four calls: the same arithmetic in the same order, so the same bits
+    buf, out4 = run_layer(wl, d, wdev)
+    assert np.array_equal(bits(out), bits(out4))
+
+
+@pytest.mark.parametrize("T,H,I,E,k,one_launch", [
+    (1, 512, 512, 8, 2, True), (4, 1024, 512, 16, 4, True), (2, 2048, 1024, 64, 8, True), (3, 1024, 512, 32, 6, True),
+    (1, 512, 512, 4, 4, True),      # every expert touched
+    (4, 512, 512, 256, 8, False),   # the logits of 4 tokens do not fit the router's shared memory at this H
+    (5, 512, 512, 8, 2, False),     # more than 4 tokens
+    (16, 256, 128, 8, 2, False),    # not a shape of the decode-sized expert kernel
+    (64, 1024, 512, 32, 6, False)])
+def test_forward_small_shapes(T, H, I, E, k, one_launch):
+    wl = inputs.Workload("fwd", T, H, I, E, k)
+    d = inputs.make_workload(wl, seed=5)
+    _check_forward(wl, d, None, one_launch)
+
+
+@pytest.mark.parametrize("T,k,seed", [(1, 8, 0), (1, 8, 1), (2, 8, 0), (3, 6, 2), (4, 8, 3)])
+def test_forward_production_shape(T, k, seed, prod_weights):
+    wl = inputs.Workload("fwd_prod", T, 4096, 2048, 256, k)
+    (w13, s13, w2, s2), wdev = prod_weights
+    d = dict(logits=inputs.make_logits(T, wl.E, seed), x=inputs.make_x(T, wl.H, seed), w13=w13, s13=s13, w2=w2, s2=s2)
+    _check_forward(wl, d, wdev, True)
+
+
+def test_forward_tokens_sharing_experts():
+    """Four tokens with the same logits: every touched expert gets all four rows."""
+    wl = inputs.Workload("fwd_same", 4, 1024, 512, 16, 4)
+    d = inputs.make_workload(wl, seed=6)
+    d["logits"][:] = d["logits"][0]
+    _check_forward(wl, d, None, True)
+
+
+def test_forward_without_routing_outputs_and_in_a_graph(prod_weights):
+    """topk_ids / topk_w may be NULL; graph replays of several calls sharing one workspace give the eager result."""
+    wl = inputs.WORKLOADS["decode_c1"]
+    (w13, s13, w2, s2), wdev = prod_weights
+    sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
+    ws = moe.alloc_forward_workspace(sh)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    batches = [(dev(inputs.make_logits(wl.T, wl.E, 40 + i)), dev(inputs.make_x(wl.T, wl.H, 40 + i))) for i in range(4)]
+    outs = [torch.empty((wl.T, wl.H), dtype=torch.bfloat16, device="cuda") for _ in batches]
+    eager = []
+    for (lg, x), o in zip(batches, outs):
+        moe.moe_forward(lg, x, *wdev, sh, o, None, None, st, ws)
+        torch.cuda.synchronize()
+        eager.append(bits(o).copy())
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        moe.moe_forward(batches[0][0], batches[0][1], *wdev, sh, outs[0], None, None, st, ws, None)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for (lg, x), o in zip(batches, outs):
+            moe.moe_forward(lg, x, *wdev, sh, o, None, None, st, ws, None)
+    for _ in range(3):
+        for o in outs:
+            o.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0
+        for o, e in zip(outs, eager):
+            assert np.array_equal(bits(o), e)
+
+
+def test_forward_host_uses_it():
+    """moe_forward_host clears the counter block itself: a workspace full of ones still gives the layer's result."""
+    wl = inputs.Workload("fwd_host", 2, 1024, 512, 16, 4)
+    d = inputs.make_workload(wl, seed=8)
+    wdev = weights_dev(d)
+    sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
+    ws = moe.alloc_workspace(sh, host_path=True)
+    ws.fill_(1)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    lh = torch.from_numpy(d["logits"]).pin_memory()
+    xh = torch.from_numpy(d["x"].view(np.int16)).pin_memory()
+    oh = torch.empty((wl.T, wl.H), dtype=torch.int16).pin_memory()
+    moe.moe_forward_host(lh, xh, *wdev, sh, oh, st, ws)
+    assert int(st.item()) == 0 and moe.moe_last_kernel_name() == _ONE_LAUNCH
+    buf, out4 = run_layer(wl, d, wdev)
+    assert np.array_equal(oh.numpy().view(np.uint16), bits(out4))
+
+
 def _sample_tokens(wl, ids, off, n):
     """Tokens covering the first and last row of the heaviest expert, a row of many experts, and
     rows at tile boundaries; the rest seeded."""
