@@ -154,7 +154,7 @@ int moe_validate_scales(const uint8_t* scales, size_t n_bytes, int32_t* bad_coun
  * the three calls before it, and - where the pointers are not NULL - topk_ids / topk_w [T,k] exactly as moe_route
  * writes them.
  *
- *   - For T <= 4 tokens (T*k <= 32 slots, T*E*4 <= 4*max(H,I) bytes) on shapes the decode-sized expert kernel takes,
+ *   - For T <= 2 tokens (T*k <= 32 slots, T*E*4 <= 4*max(H,I) bytes) on shapes the decode-sized expert kernel takes,
  *     the call is ONE kernel launch: every CTA routes the T tokens itself, sorts the slots, writes its own E2M1 term
  *     rows of the tokens, runs its share of the gate/up and down items, and the CTA that finishes a column tile's last
  *     expert reduces that tile over the slots.  Any other shape runs the four calls back to back.

@@ -87,7 +87,10 @@ struct NatArgs {
 // items take all T tokens as operand rows (row = 8 * token + term) whatever their expert, and the epilogue keeps the
 // tokens that were routed to the item's expert.  After the down projection the CTA that runs the last expert's item of a column tile
 // reduces that tile over the slots of every token.
-constexpr int kFusedMaxTok = 4;    // tokens of a fused call: one lane quadrant of operand rows
+// tokens of a fused call.  Every gate/up item fetches the term rows of all of them, once per lane quadrant: 4 KB per
+// K step and token beside the 32 KB of weights.  From 3 tokens on that traffic costs more than the launches save
+// (production shape: 86 against 74 us for 3 tokens, 104 against 91 us for 4), so those batches take the four calls.
+constexpr int kFusedMaxTok = 2;
 constexpr int kFusedMaxSlots = 32; // T * k: one warp sorts them
 constexpr int kSyncDone2 = 1024;   // int index in the sync block: per column tile, warps that stored a down item
 constexpr int kSyncExit = 1024 + 64;  // CTAs that have finished; the last one clears the block
