@@ -341,6 +341,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   uint64_t* acc_empty = acc_full + 1;            // epilogue -> MMA
   uint64_t* act_ready = acc_empty + 1;           // scale warps -> MMA: term-row scale factors of the current (expert, pass)
   uint64_t* act_free = act_ready + 1;            // MMA done with them -> scale warps
+  uint64_t* ctr_done = act_free + 1;             // one-launch layer: epilogue warps that are through with the global counters
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + sm.misc);
   int* touched = reinterpret_cast<int*>(smem + sm.touched);  // ids of the experts that have rows
   int* t_begin = touched + a.E;                              // their first sorted row
@@ -404,6 +405,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     mbar_init(acc_empty, 4);
     mbar_init(act_ready, 4);
     mbar_init(act_free, 1);
+    mbar_init(ctr_done, 4);
     mbar_fence_init();
   }
   // Operand rows that no term-row box has written yet read as zeros instead of whatever shared memory held (their
@@ -608,6 +610,27 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       }
       if (n_pend > 0) meet();
     }
+    if constexpr (kFused) {
+      // Once this CTA's last addition to and last read of the counters are behind it (the epilogue warps say so;
+      // every other warp's reads come before the MMAs those warps have waited for), it counts itself out, and the last
+      // CTA to do so clears the sync block for the next call.  This runs beside the final reduction, not after it.
+      int last = 0;
+      if (lane == 0) {
+        mbar_wait(ctr_done, 0u, a.status);
+        __threadfence();
+        last = atomicAdd(f.sync + kSyncExit, 1) == static_cast<int>(gridDim.x) - 1;
+      }
+      last = __shfl_sync(0xffffffffu, last, 0);
+      if (last) {
+        __threadfence();
+        for (int i = lane; i < a.E; i += 32) f.sync[i] = 0;
+        for (int i = lane; i < a.H / kTile; i += 32) f.sync[kSyncDone2 + i] = 0;
+        if (lane == 0) {
+          f.sync[kSyncExit] = 0;
+          f.sync[kSyncSplit] = 0;
+        }
+      }
+    }
   } else if (wid == 1) {
     // =========================== MMA issuer ===========================
     if (lane == 0) {
@@ -773,6 +796,12 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     const int jl = lane >> 3, tl = lane & 7;
     const int cb = 16 * (tl & 1) + 8 * ((tl >> 1) & 1) + 4 * (tl >> 2);
     uint32_t acc_ph = 0;
+    bool told = false;  // one-launch layer: this warp has said that it is through with the global counters
+    auto tell = [&]() {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(ctr_done);
+      told = true;
+    };
     // One pass of one item.  `dry` runs the same instructions on whatever tensor memory holds, with every wait, signal
     // and store left out: each CTA executes this code only a few times, so its first real use would otherwise pay
     // for fetching it - on the critical path of a one-item CTA - while the warp has nothing to do before the first
@@ -901,6 +930,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
               if (lane == 0) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(f.sync + kSyncDone2 + tile) : "memory");
               if (ti == s_misc[0] - 1) {
                 if (lane == 0) counter_wait_ge(f.sync + kSyncDone2 + tile, 4 * s_misc[0], a.status);
+                if (it + 1 == P.end) tell();
                 __syncwarp();
                 const int col = tile * kTile + (wid - kEpiWarp) * 64 + lane * 2;
                 for (int t = 0; t < f.T; ++t) {
@@ -934,6 +964,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         }
       }
     }
+    if (kFused && !told) tell();
   }
 
   // ---- teardown ----
@@ -942,27 +973,6 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   if (wid == 1) {
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, kNatTmemCols);
-  }
-  if constexpr (kFused) {
-    // The last CTA to get here clears the sync block for the next call: by then every CTA has made its last read of
-    // and its last addition to the counters.
-    if (wid == 0) {
-      int last = 0;
-      if (lane == 0) {
-        __threadfence();
-        last = atomicAdd(f.sync + kSyncExit, 1) == static_cast<int>(gridDim.x) - 1;
-      }
-      last = __shfl_sync(0xffffffffu, last, 0);
-      if (last) {
-        __threadfence();
-        for (int i = lane; i < a.E; i += 32) f.sync[i] = 0;
-        for (int i = lane; i < a.H / kTile; i += 32) f.sync[kSyncDone2 + i] = 0;
-        if (lane == 0) {
-          f.sync[kSyncExit] = 0;
-          f.sync[kSyncSplit] = 0;
-        }
-      }
-    }
   }
 }
 
