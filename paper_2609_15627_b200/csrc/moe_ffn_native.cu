@@ -530,6 +530,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     if (lane == 0) {
       int s = 0, cs = 0;
       uint32_t ph = 0, cph = 0;
+      const uint64_t stream_once = l2_policy_evict_first();  // every weight byte is read once per call
       // The weights depend on nothing, the term rows do: on the split kernel (phase 0) or on the gate/up items of
       // their expert (phase 1).  While a dependency is open, the weight loads go out and the term-row loads of up to
       // kWStages steps are held back; they follow once the dependency is met.
@@ -584,14 +585,14 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
               if ((ks & 1) == 0) {  // 16 scale bytes per weight row cover two K steps
                 mbar_wait(&empty_sc[cs], cph ^ 1u, a.status);
                 mbar_expect_tx(&full_sc[cs], kScStage);
-                tma_load_2d(sSc + cs * kScStage, msc, ks * 8, wrow_a, &full_sc[cs]);
-                tma_load_2d(sSc + cs * kScStage + 128 * 16, msc, ks * 8, wrow_b, &full_sc[cs]);
+                tma_load_2d_hint(sSc + cs * kScStage, msc, ks * 8, wrow_a, &full_sc[cs], stream_once);
+                tma_load_2d_hint(sSc + cs * kScStage + 128 * 16, msc, ks * 8, wrow_b, &full_sc[cs], stream_once);
                 if (++cs == kScStages) { cs = 0; cph ^= 1u; }
               }
               mbar_wait(&empty_w[s], ph ^ 1u, a.status);
               mbar_expect_tx(&full_w[s], static_cast<uint32_t>(kWStage + (bi <= kRepBox ? 4 : 1) * (8 << bi) * 128));
-              tma_load_2d(sW + s * kStage, mw, ks * 128, wrow_a, &full_w[s]);
-              tma_load_2d(sW + s * kStage + 128 * 128, mw, ks * 128, wrow_b, &full_w[s]);
+              tma_load_2d_hint(sW + s * kStage, mw, ks * 128, wrow_a, &full_w[s], stream_once);
+              tma_load_2d_hint(sW + s * kStage + 128 * 128, mw, ks * 128, wrow_b, &full_w[s], stream_once);
               // the pass's term rows (8 per token, consecutive); rows past the end of the tensor arrive as zeros
               const int arow = own_rows ? 0 : (row_begin + pass * tok_pass) * kTerms;
               if (dep_ok) {
