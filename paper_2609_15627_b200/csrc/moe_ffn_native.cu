@@ -124,7 +124,7 @@ MOE_DEVINL int term_box(int n_tok) { return n_tok <= 1 ? 0 : (n_tok <= 2 ? 1 : (
 // One projection as the kernel sees it
 struct Phase {
   int K, R, n_steps, tiles;  // reduction length, weight rows per expert, K steps, items per expert
-  long long begin, end;      // this CTA's items
+  int begin, end;            // this CTA's items (at most 1024 experts x 32 tiles)
 };
 // Items go to CTAs in contiguous shares: gate/up items evenly, per0 each.  A down item of expert t is placed as if it
 // followed that expert's last gate/up item in the gate/up list, its expert's down items spread over the span of the
@@ -564,9 +564,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         const CUtensorMap* mw = phase == 0 ? &tmap_w13 : &tmap_w2;
         const CUtensorMap* msc = phase == 0 ? &tmap_s13 : &tmap_s2;
         const TermMaps* ma = phase == 0 ? &tmap_a1 : &tmap_a2;
-        for (long long it = P.begin; it < P.end; ++it) {
-          const int ti = static_cast<int>(it / P.tiles), e = touched[ti];
-          const int tile = static_cast<int>(it % P.tiles);
+        for (int it = P.begin; it < P.end; ++it) {
+          const int ti = it / P.tiles, e = touched[ti];
+          const int tile = it % P.tiles;
           const int row_begin = t_begin[ti];
           const int n_rows_e = t_end[ti] - row_begin;
           const int n_pass = (n_rows_e + tok_pass - 1) / tok_pass;
@@ -641,8 +641,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       for (int phase = 0; phase < 2; ++phase) {
         const Phase P = phase_of(phase, a, s_misc + 1);
         int prev_ti = -1;
-        for (long long it = P.begin; it < P.end; ++it) {
-          const int ti = static_cast<int>(it / P.tiles);
+        for (int it = P.begin; it < P.end; ++it) {
+          const int ti = it / P.tiles;
           const int n_pass = (t_end[ti] - t_begin[ti] + tok_pass - 1) / tok_pass;
           for (int pass = 0; pass < n_pass; ++pass) {
             // The scale factors of the term rows (tensor memory) are shared by consecutive items of an expert whose
@@ -680,7 +680,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             // last use of these scale factors?  (always at the end of a phase)
             bool next_new = true;
             if (pass + 1 >= n_pass && it + 1 < P.end)
-              next_new = (kFused && phase == 0) ? false : ((static_cast<int>((it + 1) / P.tiles) != ti) || (n_pass > 1));
+              next_new = (kFused && phase == 0) ? false : (((it + 1) / P.tiles != ti) || (n_pass > 1));
             if (next_new) umma_commit(act_free);
           }
         }
@@ -699,8 +699,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       const int n_blk = P.K / 32;
       const uint8_t* src_sf = phase == 0 ? (kFused ? f.sf1 : a.sf1) : a.sf2;
       int prev_ti = -1;
-      for (long long it = P.begin; it < P.end; ++it) {
-        const int ti = static_cast<int>(it / P.tiles);
+      for (int it = P.begin; it < P.end; ++it) {
+        const int ti = it / P.tiles;
         const int row_begin = t_begin[ti], row_end = t_end[ti];
         const int n_pass = (row_end - row_begin + tok_pass - 1) / tok_pass;
         for (int pass = 0; pass < n_pass; ++pass) {
@@ -912,9 +912,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       const bool dry = sweep == 0;
       for (int phase = 0; phase < (dry ? 1 : 2); ++phase) {
         const Phase P = phase_of(phase, a, s_misc + 1);
-        const long long it_end = dry ? min(P.begin + 1, P.end) : P.end;
-        for (long long it = P.begin; it < it_end; ++it) {
-          const int ti = static_cast<int>(it / P.tiles), tile = static_cast<int>(it % P.tiles);
+        const int it_end = dry ? min(P.begin + 1, P.end) : P.end;
+        for (int it = P.begin; it < it_end; ++it) {
+          const int ti = it / P.tiles, tile = it % P.tiles;
           const int row_begin = t_begin[ti], row_end = t_end[ti];
           const int n_pass = dry ? 1 : (row_end - row_begin + tok_pass - 1) / tok_pass;
           const bool own_rows = kFused && phase == 0;
