@@ -48,7 +48,7 @@ typedef enum {
   MOE_OK = 0,
   MOE_ERR_INVALID_ARG = 1,       /* null or misaligned pointer, non-positive size, k > E */
   MOE_ERR_UNSUPPORTED_SHAPE = 2, /* H or I not a multiple of 128, E > 1024, k > 32, T*k > 2^30 */
-  MOE_ERR_WORKSPACE = 3,         /* ws is NULL, misaligned or smaller than moe_workspace_bytes() */
+  MOE_ERR_WORKSPACE = 3,         /* ws is NULL, misaligned or too small; device side: moe_forward's counters not cleared */
   MOE_ERR_CUDA = 4,              /* a CUDA runtime call or a launch failed */
   MOE_ERR_TIMEOUT = 5            /* device side only: written to *status_word */
 } moe_status_t;
@@ -162,7 +162,9 @@ int moe_validate_scales(const uint8_t* scales, size_t n_bytes, int32_t* bad_coun
  *     kernel's completion counters: they must be ZERO when a call starts.  Clear them once (cudaMemsetAsync) before
  *     the first call that uses this ws; every call that returns MOE_OK and whose kernels ran to completion leaves them
  *     zero, also when *status_word reports a device-side timeout.  The rest of ws is scratch.  Calls that share a ws
- *     must be ordered on one stream.
+ *     must be ordered on one stream.  Two words of the block are never written by any kernel; a one-launch call that
+ *     finds one of them non-zero writes MOE_ERR_WORKSPACE to *status_word and leaves `out` untouched (this catches a block
+ *     that was never cleared, not one that was cleared and then damaged).
  *   - Asynchronous, no allocation, capturable into a CUDA graph, bounded device-side waits as moe_expert_ffn.
  */
 size_t moe_forward_workspace_bytes(const moe_shape_t* shape);

@@ -96,6 +96,10 @@ constexpr int kSyncDone2 = 1024;   // int index in the sync block: per column ti
 constexpr int kSyncExit = 1024 + 64;  // CTAs that have finished; the last one clears the block
 constexpr int kSyncSplit = 1024 + 65; // CTAs that have written their share of the tokens' term rows
 constexpr int kSplitCtas = 32;
+// two words of the sync block that no kernel ever writes: a call that finds one of them non-zero was given a block
+// that was never cleared, reports MOE_ERR_WORKSPACE through the status word and does nothing (every CTA takes the same
+// decision, since nobody changes these words)
+constexpr int kSyncCanary0 = 1024 + 66, kSyncCanary1 = 2047;
 struct FusedArgs {
   const float* logits;       // [T, E]
   const __nv_bfloat16* x;    // [T, H]
@@ -428,6 +432,14 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     // ---- the layer's first steps, the same in every CTA: route, sort the slots, split the token rows ----
     pdl_wait();  // logits and token rows may come from the kernel before this one; the sync block is clear
     const int n_split = min(static_cast<int>(gridDim.x), kSplitCtas);
+    if (tid == 0) {
+      const int dirty = __ldcg(f.sync + kSyncCanary0) | __ldcg(f.sync + kSyncCanary1);
+      s_misc[5] = dirty;
+      if (dirty != 0 && a.status != nullptr) atomicExch(a.status, static_cast<int>(MOE_ERR_WORKSPACE));
+    }
+    // the thread that adds to and polls the split count looks for itself (it runs before the CTA's first barrier)
+    int dirty32 = 0;
+    if (tid == 32) dirty32 = __ldcg(f.sync + kSyncCanary0) | __ldcg(f.sync + kSyncCanary1);
     if (wid >= 2 && wid < 6) {
       // one warp per token: top-k by logit (ties to the lower expert), softmax over the selected logits
       const int t = wid - 2;
@@ -479,11 +491,11 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       });
       fence_proxy_async_all();  // TMA will read these rows
       asm volatile("bar.sync 2, 160;" ::: "memory");  // the five splitting warps
-      if (tid == 32) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(f.sync + kSyncSplit) : "memory");
+      if (tid == 32 && dirty32 == 0) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(f.sync + kSyncSplit) : "memory");
     }
     __syncthreads();
     // the term rows are complete by the time the routing above is: one thread makes sure while the slots are sorted
-    if (tid == 32) counter_wait_ge(f.sync + kSyncSplit, n_split, a.status);
+    if (tid == 32 && dirty32 == 0) counter_wait_ge(f.sync + kSyncSplit, n_split, a.status);
     if (wid == 2) {
       // Stable sort of the slots by expert, S <= 32: lane s is slot s.  Its sorted row = slots of smaller experts +
       // earlier slots of its own expert; the touched experts are the distinct ids in ascending order.
@@ -525,7 +537,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   // Every role walks the same sequence: both phases; in each, this CTA's items; per item, passes of up to tok_pass
   // tokens; per pass, all K steps.
 
-  if (wid == 0) {
+  const int role = (kFused && s_misc[5] != 0) ? -1 : wid;  // a sync block that was never cleared: no work at all
+  if (role == 0) {
     // =========================== producer ===========================
     if (lane == 0) {
       int s = 0, cs = 0;
@@ -632,7 +645,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         }
       }
     }
-  } else if (wid == 1) {
+  } else if (role == 1) {
     // =========================== MMA issuer ===========================
     if (lane == 0) {
       int s = 0, slot = 0;
@@ -686,7 +699,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         }
       }
     }
-  } else if (wid >= 2 && wid < 6) {
+  } else if (role >= 2 && role < 6) {
     // =========================== scale factors of the weights and of the term rows ===========================
     const int qq = wid & 3;                      // tensor-memory lane quadrant written by this warp (warps 2..5 -> 2,3,0,1)
     const uint32_t lane_base = static_cast<uint32_t>(qq * 32) << 16;
@@ -785,7 +798,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         }
       }
     }
-  } else if (wid >= kEpiWarp) {
+  } else if (role >= kEpiWarp) {
     // =========================== epilogue ===========================
     // Accumulator lane = term row = 8 * token + term.  A 32x32b load hands each lane 32 columns of its row; three
     // exchange rounds over the 8 lanes of a token (each halves the columns a lane keeps) leave lane (token, t) with

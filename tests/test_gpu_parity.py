@@ -429,6 +429,31 @@ def test_forward_without_routing_outputs_and_in_a_graph(prod_weights):
             assert np.array_equal(bits(o), e)
 
 
+def test_forward_with_a_workspace_that_was_never_cleared():
+    """The one-launch kernel finds its two untouched words non-zero, reports it and does nothing; after a clear the
+    same workspace works."""
+    wl = inputs.Workload("fwd_dirty", 2, 1024, 512, 16, 4)
+    d = inputs.make_workload(wl, seed=9)
+    wdev = weights_dev(d)
+    sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
+    ws = moe.alloc_forward_workspace(sh)
+    ws.fill_(0x5A)
+    out = torch.zeros((wl.T, wl.H), dtype=torch.bfloat16, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    moe.moe_forward(dev(d["logits"]), dev(d["x"]), *wdev, sh, out, None, None, st, ws)
+    torch.cuda.synchronize()
+    assert moe.moe_last_kernel_name() == _ONE_LAUNCH
+    assert int(st.item()) == 3                      # MOE_ERR_WORKSPACE
+    assert int(out.view(torch.int16).abs().sum().item()) == 0
+    ws[:moe.moe_forward_sync_bytes()].zero_()
+    st.zero_()
+    moe.moe_forward(dev(d["logits"]), dev(d["x"]), *wdev, sh, out, None, None, st, ws)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    buf, out4 = run_layer(wl, d, wdev)
+    assert np.array_equal(bits(out), bits(out4))
+
+
 def test_forward_host_uses_it():
     """moe_forward_host clears the counter block itself: a workspace full of ones still gives the layer's result."""
     wl = inputs.Workload("fwd_host", 2, 1024, 512, 16, 4)
