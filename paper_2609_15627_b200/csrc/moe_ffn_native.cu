@@ -95,7 +95,10 @@ constexpr int kFusedMaxSlots = 32; // T * k: one warp sorts them
 constexpr int kSyncDone2 = 1024;   // int index in the sync block: per column tile, warps that stored a down item
 constexpr int kSyncExit = 1024 + 64;  // CTAs that have finished; the last one clears the block
 constexpr int kSyncSplit = 1024 + 65; // CTAs that have written their share of the tokens' term rows
-constexpr int kSplitCtas = 32;
+// These CTAs wait for one another (every other wait in the kernel points to CTAs with a lower index), so the grid
+// needs this many SMs to itself at the start; 16 CTAs x 20 groups of 8 lanes cover the 256 blocks of two 4096-wide rows
+// in one round, more CTAs would not make it shorter.
+constexpr int kSplitCtas = 16;
 // two words of the sync block that no kernel ever writes: a call that finds one of them non-zero was given a block
 // that was never cleared, reports MOE_ERR_WORKSPACE through the status word and does nothing (every CTA takes the same
 // decision, since nobody changes these words)
