@@ -467,6 +467,22 @@ def main():
                 "peak_source": peaks["source"], "experts_touched": touched_steps, "timed_in": "the timed region",
                 "four_calls": {"ms_per_step": four_calls_ms_step, "eager_ms_per_step": eager_ms_step, "expert_ffn": roof}}
 
+    # ---- read-only ceiling: the decode kernel's load mechanism alone over the resident gate/up weights ------------
+    # (2.1 GB at the production shape, larger than L2; context for the HBM-bound workloads, not the denominator)
+    if decode and weights[0].numel() >= (1 << 28):
+        sink = torch.empty(4096, dtype=torch.int32, device="cuda")
+        for _ in range(2):
+            moe.moe_debug_read_probe(weights[0], sink, buf.status, stream)
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        p0.record(stream)
+        for _ in range(5):
+            moe.moe_debug_read_probe(weights[0], sink, buf.status, stream)
+        p1.record(stream)
+        barrier()
+        read_gbs = 5 * weights[0].numel() / (p0.elapsed_time(p1) * 1e-3) / 1e9
+        roof["read_only_stream_gbs"] = read_gbs
+        roof["frac_of_read_only_stream"] = roof["achieved"] / read_gbs
+
     # ---- end to end through the host-buffer entry point ---------------------------------------------------------
     e2e = None
     if not args.no_e2e:

@@ -70,6 +70,17 @@ const char* moe_last_kernel_name(void);
 /* Host.  Number of kernels launched (memset nodes not counted) by this thread's moe_* calls so far. */
 uint64_t moe_launch_count(void);
 
+/*
+ * Measurement aid (no counterpart in the paper): one persistent CTA per SM pulls `bytes` of device memory at `src`
+ * (128-byte aligned, at least 32 KB) through a shared-memory ring of 32 KB bulk copies and does nothing with them -
+ * the decode-sized expert kernel's weight stream without the tensor-core work.  Timed by the caller with CUDA events
+ * over a buffer larger than L2 it gives the read-only bandwidth such a stream can reach on this GPU, which bench.py
+ * reports beside the roofline.  `sink` receives one word per CTA (4 * number of SMs bytes at least).  Enqueue only;
+ * bounded waits as everywhere.
+ */
+int moe_debug_read_probe(const void* src, size_t bytes, void* sink, size_t sink_bytes, int32_t* status_word,
+                         void* cuda_stream);
+
 /* Host, pure, diagnostic.  Work split of the decode-sized expert-FFN kernel: which items (touched expert x tile of
  * 256 weight rows, in expert order) CTA `cta` of `n_ctas` takes when `n_touched` experts have rows.  out4 = first
  * and one-past-last gate/up item, first and one-past-last down item.  A down item waits, on the device, for all

@@ -16,7 +16,7 @@ EXPORTS = ("moe_workspace_bytes", "moe_status_string", "moe_last_kernel_name", "
            "moe_permute", "moe_expert_ffn", "moe_combine", "moe_validate_scales",
            "moe_forward_workspace_bytes", "moe_forward_sync_bytes", "moe_forward",
            "moe_forward_host_workspace_bytes", "moe_forward_host", "moe_expert_ffn_noalloc_max_bytes",
-           "moe_expert_ffn_noalloc", "moe_debug_native_cta_share")
+           "moe_expert_ffn_noalloc", "moe_debug_native_cta_share", "moe_debug_read_probe")
 
 
 class MoeError(RuntimeError):
@@ -61,6 +61,8 @@ def lib():
         L.moe_expert_ffn_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp]
         L.moe_debug_native_cta_share.restype = C.c_int
         L.moe_debug_native_cta_share.argtypes = [i32, i32, i32, i32, i32, C.POINTER(C.c_int32)]
+        L.moe_debug_read_probe.restype = C.c_int
+        L.moe_debug_read_probe.argtypes = [vp, sz, vp, sz, vp, vp]
         L.moe_forward_workspace_bytes.restype = sz
         L.moe_forward_workspace_bytes.argtypes = [C.POINTER(Shape)]
         L.moe_forward_sync_bytes.restype = sz
@@ -158,6 +160,13 @@ def moe_combine(y_perm, inv_perm, topk_w, sh, out, stream=None):
 def moe_validate_scales(scales, bad_count, stream=None):
     _check(lib().moe_validate_scales(_ptr(scales), scales.numel(), _ptr(bad_count), _stream(stream)),
            "moe_validate_scales")
+
+
+def moe_debug_read_probe(src, sink, status_word, stream=None):
+    """Enqueue one read-only pass over the tensor `src` (see the header); time it with events around the call."""
+    _check(lib().moe_debug_read_probe(_ptr(src), src.numel() * src.element_size(), _ptr(sink),
+                                      sink.numel() * sink.element_size(), _ptr(status_word), _stream(stream)),
+           "moe_debug_read_probe")
 
 
 def moe_forward_workspace_bytes(sh):
