@@ -158,6 +158,32 @@ int moe_combine(const float* y_perm, const int32_t* inv_perm, const float* topk_
 int moe_validate_scales(const uint8_t* scales, size_t n_bytes, int32_t* bad_count, void* cuda_stream);
 
 /*
+ * One-time load transform of the expert weights, and moe_expert_ffn on its result.  The paper applies transforms of
+ * this kind when a checkpoint is loaded (its section on load-time weight layouts) and warns that the scales must
+ * follow the same address map as the codes and that expanded weights cost more traffic than they save: here the
+ * packed buffer holds exactly the same bytes (4.25 bits per weight; moe_prepack_bytes() = the four tensors' sizes
+ * rounded up to 256 bytes each), in another order.
+ *
+ *   - Layout (private to the library; for H and I multiples of 512): the codes of 128 consecutive rows x 128
+ *     consecutive bytes (256 K elements) form one contiguous 16 KB tile, the tiles of a row block following each other
+ *     along K; the scale bytes likewise in tiles of 128 rows x 16 bytes.  A kernel's pipeline step then reads whole
+ *     contiguous runs instead of 128 pieces one row pitch apart.  For every other shape the packed buffer is a plain
+ *     copy of the four tensors.
+ *   - moe_prepack: device to device, asynchronous on the stream, out of place (packed_out must not overlap the
+ *     inputs), 256-byte aligned, packed_bytes >= moe_prepack_bytes() else MOE_ERR_WORKSPACE.  Not part of the timed
+ *     path: weights are packed once per model load.  The caller may free the four tensors afterwards.
+ *   - moe_expert_ffn_packed: moe_expert_ffn with `packed` in place of the four weight arguments; same arithmetic, same
+ *     result bit for bit.  Kernel choice as moe_expert_ffn, except that shapes with the tiled layout that would fall to
+ *     the row-streaming fallback kernel (neither decode-sized nor prefill-sized) run the grouped-GEMM kernel.
+ */
+size_t moe_prepack_bytes(const moe_shape_t* shape);
+int moe_prepack(const uint8_t* w13, const uint8_t* w13_scale, const uint8_t* w2, const uint8_t* w2_scale,
+                const moe_shape_t* shape, void* packed_out, size_t packed_bytes, void* cuda_stream);
+int moe_expert_ffn_packed(const void* x_perm_bf16 /* [T*k,H] */, const int32_t* expert_offsets, const void* packed,
+                          const moe_shape_t* shape, float* y_perm /* [T*k,H] */, int32_t* status_word, void* ws,
+                          size_t ws_bytes, void* cuda_stream);
+
+/*
  * The whole layer in one call on DEVICE buffers: route -> permute -> expert_ffn -> combine of the same inputs, with
  * every intermediate (sorted rows, per-slot outputs) kept in `ws`.  The paper's own decode gains came from cutting
  * passes and launches around the expert kernels (its optimisation history and the section on the down-projection
@@ -184,6 +210,11 @@ int moe_forward(const float* logits /* [T,E] */, const void* x_bf16 /* [T,H] */,
                 const uint8_t* w2, const uint8_t* w2_scale, const moe_shape_t* shape, void* out_bf16 /* [T,H] */,
                 int32_t* topk_ids /* [T,k] or NULL */, float* topk_w /* [T,k] or NULL */, int32_t* status_word, void* ws,
                 size_t ws_bytes, void* cuda_stream);
+/* The same on weights written by moe_prepack (same workspace, same rules, same result). */
+int moe_forward_packed(const float* logits /* [T,E] */, const void* x_bf16 /* [T,H] */, const void* packed,
+                       const moe_shape_t* shape, void* out_bf16 /* [T,H] */, int32_t* topk_ids /* [T,k] or NULL */,
+                       float* topk_w /* [T,k] or NULL */, int32_t* status_word, void* ws, size_t ws_bytes,
+                       void* cuda_stream);
 
 /*
  * moe_forward with HOST input and output for one batch: copies logits_host [T,E] and x_host [T,H] to
@@ -199,6 +230,10 @@ int moe_forward_host(const float* logits_host, const void* x_host_bf16, const ui
                      const uint8_t* w13_scale, const uint8_t* w2, const uint8_t* w2_scale,
                      const moe_shape_t* shape, void* out_host_bf16, int32_t* status_word, void* ws,
                      size_t ws_bytes, void* cuda_stream);
+/* The same on weights written by moe_prepack. */
+int moe_forward_host_packed(const float* logits_host, const void* x_host_bf16, const void* packed,
+                            const moe_shape_t* shape, void* out_host_bf16, int32_t* status_word, void* ws,
+                            size_t ws_bytes, void* cuda_stream);
 
 /*
  * moe_expert_ffn without a workspace argument, for callers that cannot allocate device memory

@@ -98,29 +98,66 @@ int moe_permute(const void* x_bf16, const int32_t* topk_ids, const int32_t* expe
                         static_cast<cudaStream_t>(cuda_stream));
 }
 
-int moe_expert_ffn(const void* x_perm_bf16, const int32_t* expert_offsets, const uint8_t* w13, const uint8_t* w13_scale,
-                   const uint8_t* w2, const uint8_t* w2_scale, const moe_shape_t* shape, float* y_perm,
-                   int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
-  const int rc = check_shape(shape);
-  if (rc != MOE_OK) return rc;
-  if (!aligned(x_perm_bf16, 16) || !aligned(expert_offsets, 16) || !aligned(w13, 16) || !aligned(w13_scale, 16) ||
-      !aligned(w2, 16) || !aligned(w2_scale, 16) || !aligned(y_perm, 16))
+namespace {
+int expert_ffn_impl(const void* x_perm_bf16, const int32_t* expert_offsets, const ExpertWeights& w, const moe_shape_t* shape,
+                    float* y_perm, int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (!aligned(x_perm_bf16, 16) || !aligned(expert_offsets, 16) || !aligned(w.w13, 16) || !aligned(w.s13, 16) ||
+      !aligned(w.w2, 16) || !aligned(w.s2, 16) || !aligned(y_perm, 16))
     return MOE_ERR_INVALID_ARG;
   if (status_word != nullptr && !aligned(status_word, 4)) return MOE_ERR_INVALID_ARG;
   const WsLayout L = ws_layout(*shape);
   if (check_ws(ws, ws_bytes, L.total) != MOE_OK) return MOE_ERR_WORKSPACE;
   __nv_bfloat16* act = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(ws) + L.act_off);
-  // kernel choice is a pure function of the shape (and of the 32-byte alignment the 4-bit tensor map needs):
-  // native block-scaled FP4 MMA for decode-sized batches, bf16 grouped GEMM for prefill-sized batches, the
-  // register-expansion streaming kernel for every other shape
-  if (native_shape_ok(*shape, w13, w2))
-    return launch_expert_ffn_native(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w13, w13_scale, w2,
-                                    w2_scale, *shape, act, y_perm, status_word, static_cast<cudaStream_t>(cuda_stream));
-  if (umma_shape_ok(*shape))
-    return launch_expert_ffn_umma(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w13, w13_scale, w2,
-                                  w2_scale, *shape, act, y_perm, status_word, static_cast<cudaStream_t>(cuda_stream));
-  return launch_expert_ffn_stream(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w13, w13_scale, w2,
-                                  w2_scale, *shape, act, y_perm, status_word, static_cast<cudaStream_t>(cuda_stream));
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const __nv_bfloat16* xp = static_cast<const __nv_bfloat16*>(x_perm_bf16);
+  // kernel choice is a pure function of the shape (and of the alignment the tensor maps need): native block-scaled
+  // FP4 MMA for decode-sized batches, bf16 grouped GEMM for prefill-sized batches, the register-expansion streaming
+  // kernel for every other shape.  The streaming kernel reads whole rows, so with the tile-contiguous weight layout
+  // (which only shapes the first two kernels take can have) the grouped GEMM also takes what is left.
+  if (native_shape_ok(*shape, w.w13, w.w2)) return launch_expert_ffn_native(xp, expert_offsets, w, *shape, act, y_perm, status_word, st);
+  if (umma_shape_ok(*shape) || w.blocked) return launch_expert_ffn_umma(xp, expert_offsets, w, *shape, act, y_perm, status_word, st);
+  return launch_expert_ffn_stream(xp, expert_offsets, w.w13, w.s13, w.w2, w.s2, *shape, act, y_perm, status_word, st);
+}
+
+// the four tensors inside a buffer written by moe_prepack
+ExpertWeights packed_view(const void* packed, const moe_shape_t& s) {
+  const PackedLayout L = packed_layout(s);
+  const uint8_t* b = static_cast<const uint8_t*>(packed);
+  return ExpertWeights{b + L.w13, b + L.s13, b + L.w2, b + L.s2, blocked_shape(s)};
+}
+}  // namespace
+
+int moe_expert_ffn(const void* x_perm_bf16, const int32_t* expert_offsets, const uint8_t* w13, const uint8_t* w13_scale,
+                   const uint8_t* w2, const uint8_t* w2_scale, const moe_shape_t* shape, float* y_perm,
+                   int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
+  const int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  return expert_ffn_impl(x_perm_bf16, expert_offsets, ExpertWeights{w13, w13_scale, w2, w2_scale, false}, shape, y_perm,
+                         status_word, ws, ws_bytes, cuda_stream);
+}
+
+size_t moe_prepack_bytes(const moe_shape_t* shape) {
+  if (check_shape(shape) != MOE_OK) return 0;
+  return packed_layout(*shape).total;
+}
+
+int moe_prepack(const uint8_t* w13, const uint8_t* w13_scale, const uint8_t* w2, const uint8_t* w2_scale,
+                const moe_shape_t* shape, void* packed_out, size_t packed_bytes, void* cuda_stream) {
+  const int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (!aligned(w13, 16) || !aligned(w13_scale, 16) || !aligned(w2, 16) || !aligned(w2_scale, 16)) return MOE_ERR_INVALID_ARG;
+  if (!aligned(packed_out, kAlign) || packed_bytes < packed_layout(*shape).total) return MOE_ERR_WORKSPACE;
+  return launch_prepack(w13, w13_scale, w2, w2_scale, *shape, static_cast<uint8_t*>(packed_out),
+                        static_cast<cudaStream_t>(cuda_stream));
+}
+
+int moe_expert_ffn_packed(const void* x_perm_bf16, const int32_t* expert_offsets, const void* packed, const moe_shape_t* shape,
+                          float* y_perm, int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
+  const int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (!aligned(packed, kAlign)) return MOE_ERR_INVALID_ARG;
+  return expert_ffn_impl(x_perm_bf16, expert_offsets, packed_view(packed, *shape), shape, y_perm, status_word, ws, ws_bytes,
+                         cuda_stream);
 }
 
 int moe_combine(const float* y_perm, const int32_t* inv_perm, const float* topk_w, const moe_shape_t* shape,
@@ -179,13 +216,12 @@ size_t moe_forward_workspace_bytes(const moe_shape_t* shape) {
 
 size_t moe_forward_sync_bytes(void) { return kForwardSyncBytes; }
 
-int moe_forward(const float* logits, const void* x_bf16, const uint8_t* w13, const uint8_t* w13_scale, const uint8_t* w2,
-                const uint8_t* w2_scale, const moe_shape_t* shape, void* out_bf16, int32_t* topk_ids, float* topk_w,
-                int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
-  int rc = check_shape(shape);
-  if (rc != MOE_OK) return rc;
-  if (!aligned(logits, 16) || !aligned(x_bf16, 16) || !aligned(w13, 16) || !aligned(w13_scale, 16) || !aligned(w2, 16) ||
-      !aligned(w2_scale, 16) || !aligned(out_bf16, 16))
+namespace {
+int forward_impl(const float* logits, const void* x_bf16, const ExpertWeights& w, const moe_shape_t* shape, void* out_bf16,
+                 int32_t* topk_ids, float* topk_w, int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
+  int rc;
+  if (!aligned(logits, 16) || !aligned(x_bf16, 16) || !aligned(w.w13, 16) || !aligned(w.s13, 16) || !aligned(w.w2, 16) ||
+      !aligned(w.s2, 16) || !aligned(out_bf16, 16))
     return MOE_ERR_INVALID_ARG;
   if ((topk_ids != nullptr && !aligned(topk_ids, 16)) || (topk_w != nullptr && !aligned(topk_w, 16)) ||
       (status_word != nullptr && !aligned(status_word, 4)))
@@ -194,8 +230,8 @@ int moe_forward(const float* logits, const void* x_bf16, const uint8_t* w13, con
   if (check_ws(ws, ws_bytes, L.total) != MOE_OK) return MOE_ERR_WORKSPACE;
   char* base = static_cast<char*>(ws);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  if (forward_fused_ok(*shape, w13, w2))
-    return launch_forward_fused(logits, static_cast<const __nv_bfloat16*>(x_bf16), w13, w13_scale, w2, w2_scale, *shape,
+  if (forward_fused_ok(*shape, w.w13, w.w2))
+    return launch_forward_fused(logits, static_cast<const __nv_bfloat16*>(x_bf16), w, *shape,
                                 static_cast<__nv_bfloat16*>(out_bf16), topk_ids, topk_w, reinterpret_cast<int*>(base),
                                 base + kForwardSyncBytes, status_word, st);
   int32_t* d_ids = topk_ids != nullptr ? topk_ids : reinterpret_cast<int32_t*>(base + L.ids);
@@ -210,10 +246,27 @@ int moe_forward(const float* logits, const void* x_bf16, const uint8_t* w13, con
   const moe_shape_t& s = *shape;
   if ((rc = moe_route(logits, s.T, s.E, s.k, d_ids, d_w, d_off, inner, inner_bytes, st)) != MOE_OK) return rc;
   if ((rc = moe_permute(x_bf16, d_ids, d_off, shape, d_xp, d_perm, d_inv, inner, inner_bytes, st)) != MOE_OK) return rc;
-  if ((rc = moe_expert_ffn(d_xp, d_off, w13, w13_scale, w2, w2_scale, shape, d_y, status_word, inner, inner_bytes, st)) !=
-      MOE_OK)
-    return rc;
+  if ((rc = expert_ffn_impl(d_xp, d_off, w, shape, d_y, status_word, inner, inner_bytes, st)) != MOE_OK) return rc;
   return moe_combine(d_y, d_inv, d_w, shape, out_bf16, st);
+}
+}  // namespace
+
+int moe_forward(const float* logits, const void* x_bf16, const uint8_t* w13, const uint8_t* w13_scale, const uint8_t* w2,
+                const uint8_t* w2_scale, const moe_shape_t* shape, void* out_bf16, int32_t* topk_ids, float* topk_w,
+                int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
+  const int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  return forward_impl(logits, x_bf16, ExpertWeights{w13, w13_scale, w2, w2_scale, false}, shape, out_bf16, topk_ids, topk_w,
+                      status_word, ws, ws_bytes, cuda_stream);
+}
+
+int moe_forward_packed(const float* logits, const void* x_bf16, const void* packed, const moe_shape_t* shape, void* out_bf16,
+                       int32_t* topk_ids, float* topk_w, int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
+  const int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (!aligned(packed, kAlign)) return MOE_ERR_INVALID_ARG;
+  return forward_impl(logits, x_bf16, packed_view(packed, *shape), shape, out_bf16, topk_ids, topk_w, status_word, ws, ws_bytes,
+                      cuda_stream);
 }
 
 // ---- host-buffer path ---------------------------------------------------------------------------
@@ -244,11 +297,10 @@ size_t moe_forward_host_workspace_bytes(const moe_shape_t* shape) {
   return host_layout(*shape).total;
 }
 
-int moe_forward_host(const float* logits_host, const void* x_host_bf16, const uint8_t* w13, const uint8_t* w13_scale,
-                     const uint8_t* w2, const uint8_t* w2_scale, const moe_shape_t* shape, void* out_host_bf16,
-                     int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
-  int rc = check_shape(shape);
-  if (rc != MOE_OK) return rc;
+namespace {
+int forward_host_impl(const float* logits_host, const void* x_host_bf16, const ExpertWeights& w, const moe_shape_t* shape,
+                      void* out_host_bf16, int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
+  int rc;
   if (logits_host == nullptr || x_host_bf16 == nullptr || out_host_bf16 == nullptr) return MOE_ERR_INVALID_ARG;
   const HostLayout L = host_layout(*shape);
   if (check_ws(ws, ws_bytes, L.total) != MOE_OK) return MOE_ERR_WORKSPACE;
@@ -263,13 +315,32 @@ int moe_forward_host(const float* logits_host, const void* x_host_bf16, const ui
       cudaMemcpyAsync(d_logits, logits_host, static_cast<size_t>(s.T) * s.E * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
       cudaMemcpyAsync(d_x, x_host_bf16, static_cast<size_t>(s.T) * s.H * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
     return MOE_ERR_CUDA;
-  if ((rc = moe_forward(d_logits, d_x, w13, w13_scale, w2, w2_scale, shape, d_out, nullptr, nullptr, status_word,
-                        base + L.inner, ws_bytes - L.inner, st)) != MOE_OK)
+  if ((rc = forward_impl(d_logits, d_x, w, shape, d_out, nullptr, nullptr, status_word, base + L.inner, ws_bytes - L.inner,
+                         st)) != MOE_OK)
     return rc;
   if (cudaMemcpyAsync(out_host_bf16, d_out, static_cast<size_t>(s.T) * s.H * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return MOE_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return MOE_ERR_CUDA;
   return MOE_OK;
+}
+}  // namespace
+
+int moe_forward_host(const float* logits_host, const void* x_host_bf16, const uint8_t* w13, const uint8_t* w13_scale,
+                     const uint8_t* w2, const uint8_t* w2_scale, const moe_shape_t* shape, void* out_host_bf16,
+                     int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
+  const int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  return forward_host_impl(logits_host, x_host_bf16, ExpertWeights{w13, w13_scale, w2, w2_scale, false}, shape, out_host_bf16,
+                           status_word, ws, ws_bytes, cuda_stream);
+}
+
+int moe_forward_host_packed(const float* logits_host, const void* x_host_bf16, const void* packed, const moe_shape_t* shape,
+                            void* out_host_bf16, int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
+  const int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (!aligned(packed, kAlign)) return MOE_ERR_INVALID_ARG;
+  return forward_host_impl(logits_host, x_host_bf16, packed_view(packed, *shape), shape, out_host_bf16, status_word, ws,
+                           ws_bytes, cuda_stream);
 }
 
 }  // extern "C"

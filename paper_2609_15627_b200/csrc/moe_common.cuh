@@ -55,6 +55,40 @@ inline WsLayout ws_layout(const moe_shape_t& s) {
   return L;
 }
 
+// ---- expert weights as the kernels see them --------------------------------------------------------
+// Either the checkpoint's logical layout (rows of H/2 or I/2 packed bytes, rows of K/32 scale bytes), or the layout
+// moe_prepack writes for shapes with H and I multiples of 512: the same bytes in tiles that are contiguous in memory,
+//   codes:  tile (row / 128, byte / 128) = [128 rows][128 bytes], tiles of one row block consecutive along K
+//   scales: tile (row / 128, byte / 16)  = [128 rows][16 bytes]
+// so that what a CTA fetches per pipeline step (128 rows x 128 bytes of codes, 128 rows x 16 scale bytes) is one
+// contiguous 16 KB / 2 KB run instead of 128 pieces 2 KB apart: DRAM pages are read whole (the decode_c64 expert-FFN
+// call went from 0.516 to 0.48 ms on the same bytes).
+struct ExpertWeights {
+  const uint8_t *w13, *s13, *w2, *s2;
+  bool blocked;
+};
+inline bool blocked_shape(const moe_shape_t& s) { return s.H % 512 == 0 && s.I % 512 == 0; }
+struct PackedLayout {
+  size_t w13, s13, w2, s2, total;
+};
+inline PackedLayout packed_layout(const moe_shape_t& s) {
+  PackedLayout L;
+  const size_t n = static_cast<size_t>(s.E) * s.H * s.I;  // weights of one projection pair half: E * H * I
+  size_t off = 0;
+  L.w13 = off;
+  off += align_up(n, kAlign);        // E * 2I * H/2
+  L.s13 = off;
+  off += align_up(n / 16, kAlign);   // E * 2I * H/32
+  L.w2 = off;
+  off += align_up(n / 2, kAlign);    // E * H * I/2
+  L.s2 = off;
+  off += align_up(n / 32, kAlign);   // E * H * I/32
+  L.total = off;
+  return L;
+}
+int launch_prepack(const uint8_t* w13, const uint8_t* s13, const uint8_t* w2, const uint8_t* s2, const moe_shape_t& s,
+                   uint8_t* packed, cudaStream_t st);
+
 // ---- per-thread call record (host) -----------------------------------------------------------
 void note_kernel(const char* name, int launches);
 
@@ -69,27 +103,25 @@ int launch_expert_ffn_stream(const __nv_bfloat16* x_perm, const int* offsets, co
                              int* status_word, cudaStream_t st);
 // tcgen05 grouped-GEMM variant (prefill-sized batches); umma_shape_ok says whether it applies
 bool umma_shape_ok(const moe_shape_t& s);
-int launch_expert_ffn_umma(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
-                           const uint8_t* w2, const uint8_t* s2, const moe_shape_t& s, __nv_bfloat16* act, float* y_perm,
-                           int* status_word, cudaStream_t st);
+int launch_expert_ffn_umma(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& s,
+                           __nv_bfloat16* act, float* y_perm, int* status_word, cudaStream_t st);
 int launch_combine(const float* y_perm, const int* inv_perm, const float* w, const moe_shape_t& s,
                    __nv_bfloat16* out, cudaStream_t st);
 int launch_validate_scales(const uint8_t* scales, size_t n, int* bad, cudaStream_t st);
 
 // native block-scaled FP4 variant; scratch of native_scratch_bytes
 bool native_shape_ok(const moe_shape_t& s, const void* w13, const void* w2);
-int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
-                             const uint8_t* w2, const uint8_t* s2, const moe_shape_t& s, void* scratch, float* y_perm,
-                             int* status_word, cudaStream_t st);
+int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& s,
+                             void* scratch, float* y_perm, int* status_word, cudaStream_t st);
 
 // the whole layer in one launch, for a handful of tokens on shapes the native variant takes (moe_forward);
 // `sync` is the zeroed block of kForwardSyncBytes, `scratch` holds forward_fused_scratch_bytes
 constexpr size_t kForwardSyncBytes = 8192;
 bool forward_fused_ok(const moe_shape_t& s, const void* w13, const void* w2);
 size_t forward_fused_scratch_bytes(const moe_shape_t& s);
-int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const uint8_t* w13, const uint8_t* s13, const uint8_t* w2,
-                         const uint8_t* s2, const moe_shape_t& s, __nv_bfloat16* out, int* ids_out, float* w_out, int* sync,
-                         void* scratch, int* status_word, cudaStream_t st);
+int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const ExpertWeights& w, const moe_shape_t& s,
+                         __nv_bfloat16* out, int* ids_out, float* w_out, int* sync, void* scratch, int* status_word,
+                         cudaStream_t st);
 
 int sm_count();
 

@@ -77,6 +77,7 @@ struct NatArgs {
   float* y;                  // output [S, H]
   int* status;
   int E, H, I, S;
+  int blocked;               // weights in moe_prepack's tile-contiguous layout (see ExpertWeights)
 };
 
 // The one-launch layer (moe_forward on a handful of tokens): what the kernel needs beyond the expert FFN's arguments.
@@ -601,14 +602,22 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
               if ((ks & 1) == 0) {  // 16 scale bytes per weight row cover two K steps
                 mbar_wait(&empty_sc[cs], cph ^ 1u, a.status);
                 mbar_expect_tx(&full_sc[cs], kScStage);
-                tma_load_2d_hint(sSc + cs * kScStage, msc, ks * 8, wrow_a, &full_sc[cs], stream_once);
-                tma_load_2d_hint(sSc + cs * kScStage + 128 * 16, msc, ks * 8, wrow_b, &full_sc[cs], stream_once);
+                // 128 rows x 16 scale bytes; tile-contiguous layout: tile (row / 128, ks / 2) is 128 consecutive rows of 16 bytes
+                const int sx = a.blocked ? 0 : ks * 8;
+                const int sya = a.blocked ? ((wrow_a >> 7) * (P.n_steps >> 1) + (ks >> 1)) * 128 : wrow_a;
+                const int syb = a.blocked ? ((wrow_b >> 7) * (P.n_steps >> 1) + (ks >> 1)) * 128 : wrow_b;
+                tma_load_2d_hint(sSc + cs * kScStage, msc, sx, sya, &full_sc[cs], stream_once);
+                tma_load_2d_hint(sSc + cs * kScStage + 128 * 16, msc, sx, syb, &full_sc[cs], stream_once);
                 if (++cs == kScStages) { cs = 0; cph ^= 1u; }
               }
               mbar_wait(&empty_w[s], ph ^ 1u, a.status);
               mbar_expect_tx(&full_w[s], static_cast<uint32_t>(kWStage + (bi <= kRepBox ? 4 : 1) * (8 << bi) * 128));
-              tma_load_2d_hint(sW + s * kStage, mw, ks * 128, wrow_a, &full_w[s], stream_once);
-              tma_load_2d_hint(sW + s * kStage + 128 * 128, mw, ks * 128, wrow_b, &full_w[s], stream_once);
+              // 128 rows x 128 bytes of codes; tile-contiguous layout: tile (row / 128, ks) is 128 consecutive rows of 128 bytes
+              const int wx = a.blocked ? 0 : ks * 128;
+              const int wya = a.blocked ? ((wrow_a >> 7) * P.n_steps + ks) * 128 : wrow_a;
+              const int wyb = a.blocked ? ((wrow_b >> 7) * P.n_steps + ks) * 128 : wrow_b;
+              tma_load_2d_hint(sW + s * kStage, mw, wx, wya, &full_w[s], stream_once);
+              tma_load_2d_hint(sW + s * kStage + 128 * 128, mw, wx, wyb, &full_w[s], stream_once);
               // the pass's term rows (8 per token, consecutive); rows past the end of the tensor arrive as zeros
               const int arow = own_rows ? 0 : (row_begin + pass * tok_pass) * kTerms;
               if (dep_ok) {
@@ -1040,15 +1049,31 @@ bool nat_attr_once() {
 }
 }  // namespace
 
+namespace {
+// tensor maps of the weights and their scale bytes, in either layout
+bool weight_maps(const ExpertWeights& w, const moe_shape_t& sh, CUtensorMap* tm_w13, CUtensorMap* tm_s13, CUtensorMap* tm_w2,
+                 CUtensorMap* tm_s2) {
+  const uint64_t r13 = static_cast<uint64_t>(sh.E) * 2 * sh.I, r2 = static_cast<uint64_t>(sh.E) * sh.H;
+  if (w.blocked)  // every tile is [128 rows][128 or 16 bytes], tiles one after the other
+    return nat_map(tm_w13, w.w13, 128, r13 * (sh.H / 256), 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
+           nat_map(tm_w2, w.w2, 128, r2 * (sh.I / 256), 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
+           nat_map(tm_s13, w.s13, 16, r13 * (sh.H / 512), 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE) &&
+           nat_map(tm_s2, w.s2, 16, r2 * (sh.I / 512), 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
+  return nat_map(tm_w13, w.w13, sh.H / 2, r13, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
+         nat_map(tm_w2, w.w2, sh.I / 2, r2, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
+         nat_map(tm_s13, w.s13, sh.H / 32, r13, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE) &&
+         nat_map(tm_s2, w.s2, sh.I / 32, r2, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
+}
+}  // namespace
+
 bool native_shape_ok(const moe_shape_t& sh, const void* w13, const void* w2) {
   return native_batch_ok(sh) && sh.H <= kMaxK && sh.I <= kMaxK && sh.H % 512 == 0 && sh.I % 512 == 0 &&
          (reinterpret_cast<uintptr_t>(w13) & 15u) == 0 && (reinterpret_cast<uintptr_t>(w2) & 15u) == 0 &&
          nat_smem(sh.E, sh.H > sh.I ? sh.H : sh.I).total + 1024 <= 227 * 1024;
 }
 
-int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
-                             const uint8_t* w2, const uint8_t* s2, const moe_shape_t& sh, void* scratch, float* y_perm,
-                             int* status_word, cudaStream_t st) {
+int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& sh,
+                             void* scratch, float* y_perm, int* status_word, cudaStream_t st) {
   if (!nat_attr_once()) return MOE_ERR_CUDA;
   const size_t S = static_cast<size_t>(sh.T) * sh.k;
   // scratch: term rows of the intermediate and of the token rows, each followed by its scale bytes; the counters
@@ -1063,11 +1088,7 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
     if (!nat_map(&tm_a1.box[i], aq1, sh.H / 2, S * kTerms, 128, 8u << i, CU_TENSOR_MAP_SWIZZLE_128B) ||
         !nat_map(&tm_a2.box[i], aq2, sh.I / 2, S * kTerms, 128, 8u << i, CU_TENSOR_MAP_SWIZZLE_128B))
       return MOE_ERR_CUDA;
-  if (!nat_map(&tm_w13, w13, sh.H / 2, static_cast<uint64_t>(sh.E) * 2 * sh.I, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !nat_map(&tm_w2, w2, sh.I / 2, static_cast<uint64_t>(sh.E) * sh.H, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !nat_map(&tm_s13, s13, sh.H / 32, static_cast<uint64_t>(sh.E) * 2 * sh.I, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-      !nat_map(&tm_s2, s2, sh.I / 32, static_cast<uint64_t>(sh.E) * sh.H, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE))
-    return MOE_ERR_CUDA;
+  if (!weight_maps(w, sh, &tm_w13, &tm_s13, &tm_w2, &tm_s2)) return MOE_ERR_CUDA;
   const size_t split_threads = S * (sh.H / 32) * 8 > static_cast<size_t>(sh.E) ? S * (sh.H / 32) * 8 : static_cast<size_t>(sh.E);
   if (launch_pdl(native_split_kernel, dim3(static_cast<unsigned>((split_threads + 1023) / 1024)), dim3(1024), 0, st, x_perm, aq1, sf1,
                  done, static_cast<int>(S), sh.H, sh.E) != cudaSuccess)
@@ -1084,6 +1105,7 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
   a.H = sh.H;
   a.I = sh.I;
   a.S = static_cast<int>(S);
+  a.blocked = w.blocked ? 1 : 0;
   if (launch_pdl(ffn_native_kernel<false>, dim3(sm_count()), dim3(kNatThreads),
                  nat_smem(sh.E, sh.H > sh.I ? sh.H : sh.I).total + 1024, st, tm_w13, tm_s13, tm_a1, tm_w2, tm_s2, tm_a2, a,
                  FusedArgs{}) != cudaSuccess)
@@ -1106,9 +1128,9 @@ size_t forward_fused_scratch_bytes(const moe_shape_t& sh) {
   return align_up(S * sh.H * 4, kAlign) + align_up(S * kTerms * (sh.I / 2), kAlign) + align_up(S * kTerms * (sh.I / 32), kAlign) +
          align_up(own * (sh.H / 2), kAlign) + align_up(own * (sh.H / 32), kAlign);
 }
-int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const uint8_t* w13, const uint8_t* s13, const uint8_t* w2,
-                         const uint8_t* s2, const moe_shape_t& sh, __nv_bfloat16* out, int* ids_out, float* w_out, int* sync,
-                         void* scratch, int* status_word, cudaStream_t st) {
+int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const ExpertWeights& w, const moe_shape_t& sh,
+                         __nv_bfloat16* out, int* ids_out, float* w_out, int* sync, void* scratch, int* status_word,
+                         cudaStream_t st) {
   if (!nat_attr_once()) return MOE_ERR_CUDA;
   const size_t S = static_cast<size_t>(sh.T) * sh.k;
   const int grid = sm_count();
@@ -1126,11 +1148,7 @@ int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const uint
     if (!nat_map(&tm_a1.box[i], aq1, sh.H / 2, own, 128, 8u << i, CU_TENSOR_MAP_SWIZZLE_128B) ||
         !nat_map(&tm_a2.box[i], aq2, sh.I / 2, S * kTerms, 128, 8u << i, CU_TENSOR_MAP_SWIZZLE_128B))
       return MOE_ERR_CUDA;
-  if (!nat_map(&tm_w13, w13, sh.H / 2, static_cast<uint64_t>(sh.E) * 2 * sh.I, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !nat_map(&tm_w2, w2, sh.I / 2, static_cast<uint64_t>(sh.E) * sh.H, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !nat_map(&tm_s13, s13, sh.H / 32, static_cast<uint64_t>(sh.E) * 2 * sh.I, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-      !nat_map(&tm_s2, s2, sh.I / 32, static_cast<uint64_t>(sh.E) * sh.H, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE))
-    return MOE_ERR_CUDA;
+  if (!weight_maps(w, sh, &tm_w13, &tm_s13, &tm_w2, &tm_s2)) return MOE_ERR_CUDA;
   NatArgs a;
   a.sf1 = nullptr;
   a.aq2 = aq2;
@@ -1143,6 +1161,7 @@ int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const uint
   a.H = sh.H;
   a.I = sh.I;
   a.S = static_cast<int>(S);
+  a.blocked = w.blocked ? 1 : 0;
   FusedArgs f;
   f.logits = logits;
   f.x = x;

@@ -46,7 +46,8 @@ constexpr int kPBytes = kTileRows * (kBlockK / 2);   // 8 KB: 256 rows x 32 byte
 
 struct UmmaArgs {
   const uint8_t* w;        // [E, R, K/2] packed codes
-  const uint8_t* sc;       // [E, R, K/32] scale bytes
+  const uint8_t* sc;       // [E, R, K/32] scale bytes (or moe_prepack's tiles of [128 rows][16 bytes])
+  int blocked;             // weights in moe_prepack's tile-contiguous layout (see ExpertWeights)
   const int* offsets;      // [E+1]
   __nv_bfloat16* act;      // stage 1 output [S, I]
   float* y;                // stage 2 output [S, R]
@@ -177,8 +178,12 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
         for (int kb = 0; kb < num_kb; ++kb) {
           mbar_wait(&empty_p[ps], pph ^ 1u, a.status);
           mbar_expect_tx(&full_p[ps], kPBytes);
-          tma_load_2d(sP + ps * kPBytes, &tmap_w, kb * (kBlockK / 2), wrow_a, &full_p[ps]);
-          tma_load_2d(sP + ps * kPBytes + kPBytes / 2, &tmap_w, kb * (kBlockK / 2), wrow_b, &full_p[ps]);
+          // 128 rows x 32 bytes of codes; tile-contiguous layout: a quarter of the 128-byte rows of tile (row / 128, kb / 4)
+          const int wx = a.blocked ? (kb & 3) * (kBlockK / 2) : kb * (kBlockK / 2);
+          const int wya = a.blocked ? ((wrow_a >> 7) * (num_kb >> 2) + (kb >> 2)) * 128 : wrow_a;
+          const int wyb = a.blocked ? ((wrow_b >> 7) * (num_kb >> 2) + (kb >> 2)) * 128 : wrow_b;
+          tma_load_2d(sP + ps * kPBytes, &tmap_w, wx, wya, &full_p[ps]);
+          tma_load_2d(sP + ps * kPBytes + kPBytes / 2, &tmap_w, wx, wyb, &full_p[ps]);
           if (++ps == kPStages) { ps = 0; pph ^= 1u; }
           mbar_wait(&empty_ab[s], ph ^ 1u, a.status);
           mbar_expect_tx(&full_b[s], static_cast<uint32_t>(nbox) * kTokBox * kBlockK * 2);
@@ -234,7 +239,11 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
       const int e = find_expert(prefix, a.E, g);
       // stage 1: tile 0 = gate rows rt*128.., tile 1 = the matching up rows; stage 2: 256 consecutive rows
       const int grow = STAGE1 ? e * a.R + t * a.I + rt * 128 + l : e * a.R + rt * kTileRows + r;
-      const uint8_t* srow = a.sc + static_cast<size_t>(grow) * (K / 32);
+      // this row's scale bytes, 16 (= 8 K blocks) per load: K/32 consecutive bytes, or in the tile-contiguous layout
+      // its 16 bytes of tile (row / 128, group of 8 K blocks), the tiles of a row block 2 KB apart
+      const uint8_t* srow = a.blocked ? a.sc + (static_cast<size_t>(grow >> 7) * (K / 512)) * 2048 + (grow & 127) * 16
+                                      : a.sc + static_cast<size_t>(grow) * (K / 32);
+      const int sgroup = a.blocked ? 2048 : 16;  // bytes from one group of 8 K blocks to the next
       const int prow = r;  // row of this thread inside the packed stage (stage 1: gate rows 0..127, up rows 128..255)
       // scale bytes: 16 bytes cover 8 K blocks; fetched one group ahead
       uint4 sc_cur = __ldg(reinterpret_cast<const uint4*>(srow));
@@ -243,7 +252,7 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
       for (int kb = 0; kb < num_kb; ++kb) {
         if ((kb & 7) == 0) {
           if (kb != 0) sc_cur = sc_next;
-          if (kb + 8 < num_kb) sc_next = __ldg(reinterpret_cast<const uint4*>(srow + (kb + 8) * 2));
+          if (kb + 8 < num_kb) sc_next = __ldg(reinterpret_cast<const uint4*>(srow + ((kb + 8) >> 3) * sgroup));
         }
         const int sidx = (kb & 7) >> 1;  // 32-bit word of the 16 scale bytes; two bytes per K block
         const uint32_t sword = (sidx == 0) ? sc_cur.x : (sidx == 1) ? sc_cur.y : (sidx == 2) ? sc_cur.z : sc_cur.w;
@@ -386,9 +395,8 @@ bool umma_shape_ok(const moe_shape_t& sh) {
          smem_map(sh.E).total + 1024 <= 227 * 1024;
 }
 
-int launch_expert_ffn_umma(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
-                           const uint8_t* w2, const uint8_t* s2, const moe_shape_t& sh, __nv_bfloat16* act, float* y_perm,
-                           int* status_word, cudaStream_t st) {
+int launch_expert_ffn_umma(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& sh,
+                           __nv_bfloat16* act, float* y_perm, int* status_word, cudaStream_t st) {
   const size_t smem = smem_map(sh.E).total + 1024;
   static bool attr_done = false;
   if (!attr_done) {
@@ -401,10 +409,12 @@ int launch_expert_ffn_umma(const __nv_bfloat16* x_perm, const int* offsets, cons
   CUtensorMap tm_x, tm_act, tm_w13, tm_w2;
   if (!make_map_2d(&tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, x_perm, sh.H, S, kBlockK, kTokBox, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !make_map_2d(&tm_act, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, act, sh.I, S, kBlockK, kTokBox, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !make_map_2d(&tm_w13, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w13, sh.H / 2, static_cast<uint64_t>(sh.E) * 2 * sh.I, kBlockK / 2,
-                   128, CU_TENSOR_MAP_SWIZZLE_NONE) ||
-      !make_map_2d(&tm_w2, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w2, sh.I / 2, static_cast<uint64_t>(sh.E) * sh.H, kBlockK / 2, 128,
-                   CU_TENSOR_MAP_SWIZZLE_NONE))
+      // codes: rows of K/2 bytes, or (tile-contiguous layout) tiles of [128 rows][128 bytes] one after the other
+      !make_map_2d(&tm_w13, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w.w13, w.blocked ? 128 : sh.H / 2,
+                   static_cast<uint64_t>(sh.E) * 2 * sh.I * (w.blocked ? sh.H / 256 : 1), kBlockK / 2, 128,
+                   CU_TENSOR_MAP_SWIZZLE_NONE) ||
+      !make_map_2d(&tm_w2, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w.w2, w.blocked ? 128 : sh.I / 2,
+                   static_cast<uint64_t>(sh.E) * sh.H * (w.blocked ? sh.I / 256 : 1), kBlockK / 2, 128, CU_TENSOR_MAP_SWIZZLE_NONE))
     return MOE_ERR_CUDA;
   const int grid = sm_count();
   UmmaArgs a;
@@ -416,14 +426,15 @@ int launch_expert_ffn_umma(const __nv_bfloat16* x_perm, const int* offsets, cons
   a.k2 = 0x0104u;
   a.E = sh.E;
   a.I = sh.I;
-  a.w = w13;
-  a.sc = s13;
+  a.blocked = w.blocked ? 1 : 0;
+  a.w = w.w13;
+  a.sc = w.s13;
   a.K = sh.H;
   a.R = 2 * sh.I;
   ffn_umma_kernel<true><<<grid, kThreadsUmma, smem, st>>>(tm_x, tm_w13, a);
   if (cudaGetLastError() != cudaSuccess) return MOE_ERR_CUDA;
-  a.w = w2;
-  a.sc = s2;
+  a.w = w.w2;
+  a.sc = w.s2;
   a.K = sh.I;
   a.R = sh.H;
   ffn_umma_kernel<false><<<grid, kThreadsUmma, smem, st>>>(tm_act, tm_w2, a);

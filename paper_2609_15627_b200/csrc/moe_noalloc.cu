@@ -64,12 +64,13 @@ int moe_expert_ffn_noalloc(const void* x_perm_bf16, const int32_t* expert_offset
   // to start at zero.  Same kernels and the same kernel choice as moe_expert_ffn.
   __nv_bfloat16* act = static_cast<__nv_bfloat16*>(scratch);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const ExpertWeights w{w13, w13_scale, w2, w2_scale, false};
   if (native_shape_ok(s, w13, w2))
-    return launch_expert_ffn_native(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w13, w13_scale, w2,
-                                    w2_scale, s, scratch, y_perm, status_word, st);
+    return launch_expert_ffn_native(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w, s, scratch, y_perm,
+                                    status_word, st);
   if (umma_shape_ok(s))
-    return launch_expert_ffn_umma(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w13, w13_scale, w2,
-                                  w2_scale, s, act, y_perm, status_word, st);
+    return launch_expert_ffn_umma(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w, s, act, y_perm,
+                                  status_word, st);
   return launch_expert_ffn_stream(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w13, w13_scale, w2,
                                   w2_scale, s, act, y_perm, status_word, st);
 }

@@ -16,7 +16,8 @@ EXPORTS = ("moe_workspace_bytes", "moe_status_string", "moe_last_kernel_name", "
            "moe_permute", "moe_expert_ffn", "moe_combine", "moe_validate_scales",
            "moe_forward_workspace_bytes", "moe_forward_sync_bytes", "moe_forward",
            "moe_forward_host_workspace_bytes", "moe_forward_host", "moe_expert_ffn_noalloc_max_bytes",
-           "moe_expert_ffn_noalloc", "moe_debug_native_cta_share", "moe_debug_read_probe")
+           "moe_expert_ffn_noalloc", "moe_debug_native_cta_share", "moe_debug_read_probe", "moe_prepack_bytes", "moe_prepack",
+           "moe_expert_ffn_packed", "moe_forward_packed", "moe_forward_host_packed")
 
 
 class MoeError(RuntimeError):
@@ -61,6 +62,16 @@ def lib():
         L.moe_expert_ffn_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp]
         L.moe_debug_native_cta_share.restype = C.c_int
         L.moe_debug_native_cta_share.argtypes = [i32, i32, i32, i32, i32, C.POINTER(C.c_int32)]
+        L.moe_prepack_bytes.restype = sz
+        L.moe_prepack_bytes.argtypes = [C.POINTER(Shape)]
+        L.moe_prepack.restype = C.c_int
+        L.moe_prepack.argtypes = [vp, vp, vp, vp, C.POINTER(Shape), vp, sz, vp]
+        L.moe_expert_ffn_packed.restype = C.c_int
+        L.moe_expert_ffn_packed.argtypes = [vp, vp, vp, C.POINTER(Shape), vp, vp, vp, sz, vp]
+        L.moe_forward_packed.restype = C.c_int
+        L.moe_forward_packed.argtypes = [vp, vp, vp, C.POINTER(Shape), vp, vp, vp, vp, vp, sz, vp]
+        L.moe_forward_host_packed.restype = C.c_int
+        L.moe_forward_host_packed.argtypes = [vp, vp, vp, C.POINTER(Shape), vp, vp, vp, sz, vp]
         L.moe_debug_read_probe.restype = C.c_int
         L.moe_debug_read_probe.argtypes = [vp, sz, vp, sz, vp, vp]
         L.moe_forward_workspace_bytes.restype = sz
@@ -162,11 +173,44 @@ def moe_validate_scales(scales, bad_count, stream=None):
            "moe_validate_scales")
 
 
+def moe_prepack_bytes(sh):
+    return int(lib().moe_prepack_bytes(C.byref(sh)))
+
+
+def moe_prepack(w13, w13_scale, w2, w2_scale, sh, stream=None):
+    """One-time re-layout of the expert weights; returns the packed buffer (allocation + the call)."""
+    n = moe_prepack_bytes(sh)
+    if n == 0:
+        raise MoeError("unsupported shape")
+    packed = torch.empty(n, dtype=torch.uint8, device=w13.device)
+    _check(lib().moe_prepack(_ptr(w13), _ptr(w13_scale), _ptr(w2), _ptr(w2_scale), C.byref(sh), _ptr(packed), n,
+                             _stream(stream)), "moe_prepack")
+    return packed
+
+
+def moe_expert_ffn_packed(x_perm, expert_offsets, packed, sh, y_perm, status_word, ws, stream=None):
+    _check(lib().moe_expert_ffn_packed(_ptr(x_perm), _ptr(expert_offsets), _ptr(packed), C.byref(sh), _ptr(y_perm),
+                                       _ptr(status_word), _ptr(ws), ws.numel(), _stream(stream)), "moe_expert_ffn_packed")
+
+
+def moe_forward_packed(logits, x, packed, sh, out, topk_ids, topk_w, status_word, ws, stream=None):
+    _check(lib().moe_forward_packed(_ptr(logits), _ptr(x), _ptr(packed), C.byref(sh), _ptr(out), _ptr(topk_ids),
+                                    _ptr(topk_w), _ptr(status_word), _ptr(ws), ws.numel(), _stream(stream)),
+           "moe_forward_packed")
+
+
+def moe_forward_host_packed(logits_host, x_host, packed, sh, out_host, status_word, ws, stream=None):
+    _check(lib().moe_forward_host_packed(_ptr(logits_host), _ptr(x_host), _ptr(packed), C.byref(sh), _ptr(out_host),
+                                         _ptr(status_word), _ptr(ws), ws.numel(), _stream(stream)),
+           "moe_forward_host_packed")
+
+
 def moe_debug_read_probe(src, sink, status_word, stream=None):
     """Enqueue one read-only pass over the tensor `src` (see the header); time it with events around the call."""
     _check(lib().moe_debug_read_probe(_ptr(src), src.numel() * src.element_size(), _ptr(sink),
                                       sink.numel() * sink.element_size(), _ptr(status_word), _stream(stream)),
-           "moe_debug_read_probe")
+           "moe_debug_read_probe", "moe_prepack_bytes", "moe_prepack",
+           "moe_expert_ffn_packed", "moe_forward_packed", "moe_forward_host_packed")
 
 
 def moe_forward_workspace_bytes(sh):

@@ -69,6 +69,21 @@ def test_argument_errors_are_found_on_the_host(L):
     assert L.moe_forward(fake, fake, fake, fake, fake, fake, C.byref(sh), fake, null, null, null, null, 1 << 30, null) == 3
 
 
+def test_prepack_sizes_and_argument_errors(L):
+    sh = moe.shape(4, 1024, 512, 4, 2)
+    n = 4 * 1024 * 512
+    assert moe.moe_prepack_bytes(sh) == n + n // 16 + n // 2 + n // 32        # the same bytes, each tensor a multiple of 256
+    assert moe.moe_prepack_bytes(moe.shape(4, 1000, 512, 4, 2)) == 0
+    fake, odd, null = C.c_void_p(0x1000), C.c_void_p(0x1004), C.c_void_p(0)
+    assert L.moe_prepack(null, fake, fake, fake, C.byref(sh), fake, 1 << 30, null) == 1
+    assert L.moe_prepack(fake, fake, fake, fake, C.byref(sh), odd, 1 << 30, null) == 3
+    assert L.moe_prepack(fake, fake, fake, fake, C.byref(sh), fake, 64, null) == 3
+    assert L.moe_expert_ffn_packed(fake, fake, odd, C.byref(sh), fake, null, fake, 1 << 30, null) == 1
+    assert L.moe_expert_ffn_packed(fake, fake, fake, C.byref(sh), fake, null, fake, 64, null) == 3
+    assert L.moe_forward_packed(fake, fake, odd, C.byref(sh), fake, null, null, null, C.c_void_p(0x10000), 1 << 30, null) == 1
+    assert L.moe_forward_host_packed(null, fake, fake, C.byref(sh), fake, null, fake, 1 << 30, null) == 1
+
+
 def test_forward_workspace_sizes(L):
     """The workspace of moe_forward: the counter block, then room for the one-launch scratch or the four calls' buffers."""
     sync = moe.moe_forward_sync_bytes()

@@ -472,6 +472,97 @@ def test_forward_host_uses_it():
     assert np.array_equal(oh.numpy().view(np.uint16), bits(out4))
 
 
+# ---- moe_prepack and the calls that take its result ------------------------------------------------------
+
+def _tiles(a, tile_bytes):
+    """[R, B] bytes -> tiles of [128 rows][tile_bytes], tile (row // 128, byte // tile_bytes), flattened in that order."""
+    R, B = a.shape
+    return a.reshape(R // 128, 128, B // tile_bytes, tile_bytes).transpose(0, 2, 1, 3).ravel()
+
+
+def _align(n, a=256):
+    return (n + a - 1) // a * a
+
+
+@pytest.mark.parametrize("H,I,E,tiled", [(1024, 512, 4, True), (512, 1536, 3, True), (256, 128, 8, False), (512, 384, 2, False)])
+def test_prepack_layout(H, I, E, tiled):
+    w13, s13, w2, s2 = inputs.make_expert_weights(H, I, E, seed=11)
+    sh = moe.shape(4, H, I, E, 1)
+    packed = moe.moe_prepack(dev(w13), dev(s13), dev(w2), dev(s2), sh)
+    torch.cuda.synchronize()
+    got = packed.cpu().numpy()
+    parts = [(w13.reshape(E * 2 * I, H // 2), 128), (s13.reshape(E * 2 * I, H // 32), 16),
+             (w2.reshape(E * H, I // 2), 128), (s2.reshape(E * H, I // 32), 16)]
+    off = 0
+    for a, tb in parts:
+        want = _tiles(a, tb) if tiled else a.ravel()
+        assert np.array_equal(got[off:off + want.size], want)
+        off += _align(want.size)
+    assert moe.moe_prepack_bytes(sh) == off == got.size
+
+
+@pytest.mark.parametrize("T,H,I,E,k,same_kernel", [
+    (8, 1024, 512, 32, 6, True),      # decode-sized kernel
+    (3, 512, 512, 8, 2, True),
+    (256, 512, 512, 8, 6, True),      # prefill-sized kernel
+    (300, 1024, 1024, 4, 4, True),
+    (64, 512, 512, 2, 2, False),      # raw: row-streaming kernel; packed: grouped GEMM
+    (16, 256, 128, 8, 2, True),       # no tiled layout for this shape: plain copy, same kernel
+])
+def test_expert_ffn_packed(T, H, I, E, k, same_kernel):
+    wl = inputs.Workload("packed", T, H, I, E, k)
+    d = inputs.make_workload(wl, seed=12)
+    wdev = weights_dev(d)
+    buf, out = run_layer(wl, d, wdev)
+    sh = buf.sh
+    raw_kernel_y = buf.y_perm.clone()
+    packed = moe.moe_prepack(*wdev, sh)
+    y = torch.empty_like(buf.y_perm)
+    moe.moe_expert_ffn(buf.x_perm, buf.expert_offsets, *wdev, sh, raw_kernel_y, buf.status, buf.ws)
+    k_raw = moe.moe_last_kernel_name()
+    moe.moe_expert_ffn_packed(buf.x_perm, buf.expert_offsets, packed, sh, y, buf.status, buf.ws)
+    k_packed = moe.moe_last_kernel_name()
+    torch.cuda.synchronize()
+    assert int(buf.status.item()) == 0
+    assert (k_raw == k_packed) == same_kernel, (k_raw, k_packed)
+    r = O.forward_staged(d["logits"], d["x"], d["w13"], d["s13"], d["w2"], d["s2"], wl.k)
+    check_y(y.cpu().numpy(), r["y_perm"], wl.name)
+    if same_kernel:
+        assert torch.equal(y.view(torch.int32), raw_kernel_y.view(torch.int32))
+
+
+@pytest.mark.parametrize("T,k,seed", [(1, 8, 0), (2, 6, 1), (64, 8, 2)])
+def test_forward_packed_production_shape(T, k, seed, prod_weights):
+    wl = inputs.Workload("fwd_packed", T, 4096, 2048, 256, k)
+    (w13, s13, w2, s2), wdev = prod_weights
+    sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
+    packed = moe.moe_prepack(*wdev, sh)
+    lg, x = dev(inputs.make_logits(T, wl.E, seed)), dev(inputs.make_x(T, wl.H, seed))
+    ws = moe.alloc_forward_workspace(sh)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out_raw = torch.empty((T, wl.H), dtype=torch.bfloat16, device="cuda")
+    out_packed = torch.empty_like(out_raw)
+    ids = torch.empty((T, k), dtype=torch.int32, device="cuda")
+    w = torch.empty((T, k), dtype=torch.float32, device="cuda")
+    moe.moe_forward(lg, x, *wdev, sh, out_raw, None, None, st, ws)
+    k_raw = moe.moe_last_kernel_name()
+    moe.moe_forward_packed(lg, x, packed, sh, out_packed, ids, w, st, ws)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0 and moe.moe_last_kernel_name() == k_raw
+    assert (k_raw == _ONE_LAUNCH) == (T <= 2)
+    assert torch.equal(out_raw.view(torch.int16), out_packed.view(torch.int16))
+    d = dict(logits=lg.cpu().numpy(), x=bits(x), w13=w13, s13=s13, w2=w2, s2=s2)
+    r = O.forward_staged(d["logits"], d["x"], w13, s13, w2, s2, k)
+    assert np.array_equal(ids.cpu().numpy(), r["ids"])
+    check_out(bits(out_packed), r["out"], r["out_f32"], wl.name)
+    # and through the host-buffer call
+    ws_h = moe.alloc_workspace(sh, host_path=True)
+    oh = torch.empty((T, wl.H), dtype=torch.int16).pin_memory()
+    moe.moe_forward_host_packed(lg.cpu().pin_memory(), x.view(torch.int16).cpu().pin_memory(), packed, sh, oh, st, ws_h)
+    assert int(st.item()) == 0
+    assert np.array_equal(oh.numpy().view(np.uint16), bits(out_packed))
+
+
 def _sample_tokens(wl, ids, off, n):
     """Tokens covering the first and last row of the heaviest expert, a row of many experts, and
     rows at tile boundaries; the rest seeded."""
