@@ -195,6 +195,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="decode workloads: launch the calls eagerly instead of replaying CUDA graphs")
     ap.add_argument("--four-calls", action="store_true", help="time the four calls even where moe_forward is one launch")
+    ap.add_argument("--raw-weights", action="store_true", help="read the weights in the checkpoint's row layout instead of moe_prepack's tiles")
     args = ap.parse_args()
 
     from paper_2609_15627_b200 import inputs
@@ -236,6 +237,13 @@ def main():
 
     weights_host = inputs.make_expert_weights(wl.H, wl.I, wl.E, seed=0)
     weights = tuple(dev(a) for a in weights_host)
+    # One-time load transform (untimed, as in the paper's load path): the same bytes in tiles that are contiguous in
+    # memory.  The row-layout tensors are dropped afterwards: one copy of the weights is resident.
+    packed = None
+    if not args.raw_weights:
+        packed = moe.moe_prepack(*weights, moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k))
+        torch.cuda.synchronize()
+        weights = None
     n_cycle = 32 if decode else 2
     batches_host = [(inputs.make_logits(wl.T, wl.E, 7000 + rank * 100 + i, wl.skew), inputs.make_x(wl.T, wl.H, 7000 + rank * 100 + i))
                     for i in range(n_cycle)]
@@ -253,7 +261,19 @@ def main():
 
     # Does moe_forward run this shape as one launch?  (Asked of the library: one call, then the name of its kernel.)
     fws = moe.alloc_forward_workspace(sh)
-    moe.moe_forward(batches[0][0], batches[0][1], *weights, sh, buf.out, None, None, buf.status, fws, stream)
+    def forward(l, x, st):
+        if packed is not None:
+            moe.moe_forward_packed(l, x, packed, sh, buf.out, None, None, buf.status, fws, st)
+        else:
+            moe.moe_forward(l, x, *weights, sh, buf.out, None, None, buf.status, fws, st)
+
+    def expert_ffn(b, st):
+        if packed is not None:
+            moe.moe_expert_ffn_packed(b.x_perm, b.expert_offsets, packed, sh, b.y_perm, b.status, b.ws, st)
+        else:
+            moe.moe_expert_ffn(b.x_perm, b.expert_offsets, *weights, sh, b.y_perm, b.status, b.ws, st)
+
+    forward(batches[0][0], batches[0][1], stream)
     torch.cuda.synchronize()
     one_launch = moe.moe_last_kernel_name().startswith("layer_one_launch") and not args.four_calls
 
@@ -264,7 +284,7 @@ def main():
         moe.moe_permute(x, buf.topk_ids, buf.expert_offsets, sh, buf.x_perm, buf.perm, buf.inv_perm, buf.ws, st)
         if ev is not None:
             ev[0].record(st)
-        moe.moe_expert_ffn(buf.x_perm, buf.expert_offsets, *weights, sh, buf.y_perm, buf.status, buf.ws, st)
+        expert_ffn(buf, st)
         if ev is not None:
             ev[1].record(st)
         moe.moe_combine(buf.y_perm, buf.inv_perm, buf.topk_w, sh, buf.out, st)
@@ -272,7 +292,7 @@ def main():
     def step1(i, ev=None, st=stream):
         """The same path as one call (one kernel launch for this shape)."""
         l, x = batches[i % n_cycle]
-        moe.moe_forward(l, x, *weights, sh, buf.out, None, None, buf.status, fws, st)
+        forward(l, x, st)
 
     step = step1 if one_launch else step4
 
@@ -406,7 +426,7 @@ def main():
         barrier()
 
         def ffn_only(b, st=stream):
-            moe.moe_expert_ffn(b.x_perm, b.expert_offsets, *weights, sh, b.y_perm, b.status, b.ws, st)
+            expert_ffn(b, st)
 
         side = torch.cuda.Stream()
         side.wait_stream(stream)
@@ -469,17 +489,18 @@ def main():
 
     # ---- read-only ceiling: the decode kernel's load mechanism alone over the resident gate/up weights ------------
     # (2.1 GB at the production shape, larger than L2; context for the HBM-bound workloads, not the denominator)
-    if decode and weights[0].numel() >= (1 << 28):
+    probe_src = packed if packed is not None else weights[0]
+    if decode and probe_src.numel() >= (1 << 28):
         sink = torch.empty(4096, dtype=torch.int32, device="cuda")
         for _ in range(2):
-            moe.moe_debug_read_probe(weights[0], sink, buf.status, stream)
+            moe.moe_debug_read_probe(probe_src, sink, buf.status, stream)
         p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         p0.record(stream)
         for _ in range(5):
-            moe.moe_debug_read_probe(weights[0], sink, buf.status, stream)
+            moe.moe_debug_read_probe(probe_src, sink, buf.status, stream)
         p1.record(stream)
         barrier()
-        read_gbs = 5 * weights[0].numel() / (p0.elapsed_time(p1) * 1e-3) / 1e9
+        read_gbs = 5 * probe_src.numel() / (p0.elapsed_time(p1) * 1e-3) / 1e9
         roof["read_only_stream_gbs"] = read_gbs
         roof["frac_of_read_only_stream"] = roof["achieved"] / read_gbs
 
@@ -491,16 +512,23 @@ def main():
         xh = [torch.from_numpy(x.view(np.int16)).pin_memory() for _, x in batches_host]
         oh = torch.empty((wl.T, wl.H), dtype=torch.int16).pin_memory()
         n_e2e = max(3, min(args.steps, 200 if decode else 5))
+        def forward_host(i):
+            if packed is not None:
+                moe.moe_forward_host_packed(lh[i % n_cycle], xh[i % n_cycle], packed, sh, oh, buf.status, ws_h, stream)
+            else:
+                moe.moe_forward_host(lh[i % n_cycle], xh[i % n_cycle], *weights, sh, oh, buf.status, ws_h, stream)
+
         for i in range(3):
-            moe.moe_forward_host(lh[i % n_cycle], xh[i % n_cycle], *weights, sh, oh, buf.status, ws_h, stream)
+            forward_host(i)
         barrier()
         t0 = time.perf_counter()
         for i in range(n_e2e):
-            moe.moe_forward_host(lh[i % n_cycle], xh[i % n_cycle], *weights, sh, oh, buf.status, ws_h, stream)
+            forward_host(i)
         dt = max_over_ranks(time.perf_counter() - t0, world)
         e2e = {"value": wl.T * world * n_e2e / dt, "unit": "tokens/s",
                "h2d_bytes_per_step": wl.T * wl.E * 4 + wl.T * wl.H * 2, "d2h_bytes_per_step": wl.T * wl.H * 2,
-               "steps": n_e2e, "call": "moe_forward_host (pinned host logits/x in, bf16 out back, weights resident)"}
+               "steps": n_e2e, "call": "%s (pinned host logits/x in, bf16 out back, weights resident)"
+                       % ("moe_forward_host_packed" if packed is not None else "moe_forward_host")}
 
     # ---- the oracle on the host cores (rank 0, N = 1 only) ----------------------------------------------------------
     cpu = None
@@ -518,7 +546,10 @@ def main():
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": wl.name, "T": wl.T, "H": wl.H, "I": wl.I, "E": wl.E, "k": wl.k,
                        "parallelism": "replicas only" if world > 1 else "1 GPU",
-                       "call": "moe_forward (one kernel launch per step)" if one_launch else "moe_route, moe_permute, moe_expert_ffn, moe_combine",
+                       "call": ("moe_forward%s (one kernel launch per step)" if one_launch else
+                                "moe_route, moe_permute, moe_expert_ffn%s, moe_combine") % ("_packed" if packed is not None else ""),
+                       "weights": ("moe_prepack's tile-contiguous layout (one-time transform, same bytes)" if packed is not None
+                                   else "checkpoint row layout"),
                        "launch": "cuda graph replay, %d consecutive batches of the cycle per graph" % kGraphSteps if use_graph else "eager",
                        "eager_ms_per_step": None if one_launch else eager_ms_step,
                        "l2": "inputs cycle over %d seeded batches; %.2f GB of expert weights resident (larger than L2)"

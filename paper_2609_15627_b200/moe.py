@@ -209,8 +209,7 @@ def moe_debug_read_probe(src, sink, status_word, stream=None):
     """Enqueue one read-only pass over the tensor `src` (see the header); time it with events around the call."""
     _check(lib().moe_debug_read_probe(_ptr(src), src.numel() * src.element_size(), _ptr(sink),
                                       sink.numel() * sink.element_size(), _ptr(status_word), _stream(stream)),
-           "moe_debug_read_probe", "moe_prepack_bytes", "moe_prepack",
-           "moe_expert_ffn_packed", "moe_forward_packed", "moe_forward_host_packed")
+           "moe_debug_read_probe")
 
 
 def moe_forward_workspace_bytes(sh):
