@@ -32,10 +32,18 @@
 //   warp 1      allocates tensor memory, issues the MMAs, commits to mbarriers
 //   warps 2..5  move weight scale bytes into tensor memory (tcgen05.st), and at a change of (expert, pass) the
 //               scale bytes of its term rows
-//   warps 6..9  epilogue, one warp per tensor-memory lane quadrant (4 tokens each): sum the 8 term rows of each
-//               token, then SwiGLU + bf16 rounding + the 8-term split for the down projection (gate/up) or the
-//               fp32 store (down)
+//   warps 6..9  epilogue, one warp per tensor-memory lane quadrant: sum the 8 term rows of each token, then SwiGLU +
+//               bf16 rounding + the 8-term split for the down projection (gate/up) or the fp32 store (down).  A pass
+//               of more than 4 tokens: quadrant q holds tokens 4q..4q+3, its warp takes all 256 columns.  A pass of
+//               at most 4 tokens is loaded into every quadrant, and each warp takes a quarter of the columns.
 // Every wait is bounded and reports through the status word.
+//
+// The weights are read either in the checkpoint's row layout or in moe_prepack's tile-contiguous layout (one tensor
+// map box = one contiguous run; see ExpertWeights), always with the L2 evict-first policy: each byte is used once.
+//
+// The same kernel, instantiated with kFused = true, is the whole layer in one launch for one or two tokens
+// (moe_forward): it routes, sorts the slots and splits the token rows itself, and reduces over the slots at the end
+// (see FusedArgs).
 #include <cuda.h>
 #include <cuda_fp4.h>
 
