@@ -26,9 +26,15 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // native block-scaled FP4 variant (decode-sized batches): on average at most 32 rows per expert (2 passes of 16
 // tokens over the weight stream).  Its scratch holds the E2M1 term rows (8 per row) of both projections' inputs:
 // [8S, I/2] + [8S, I/32] scale bytes and [8S, H/2] + [8S, H/32]; and one completion counter per expert.
+#ifndef MOE_NATIVE_MAX_SLOTS
+#define MOE_NATIVE_MAX_SLOTS 6144            // measured crossover to the prefill-sized kernel at the production shape
+#endif
+#ifndef MOE_NATIVE_MAX_ROWS_PER_EXPERT
+#define MOE_NATIVE_MAX_ROWS_PER_EXPERT 32    // on average: two passes of 16 tokens over an expert's weights
+#endif
 inline bool native_batch_ok(const moe_shape_t& s) {
   const long long S = static_cast<long long>(s.T) * s.k;
-  return S <= 4096 && S <= 32LL * s.E;
+  return S <= MOE_NATIVE_MAX_SLOTS && S <= static_cast<long long>(MOE_NATIVE_MAX_ROWS_PER_EXPERT) * s.E;
 }
 inline size_t native_scratch_bytes(const moe_shape_t& s) {
   const size_t S = static_cast<size_t>(s.T) * s.k;

@@ -583,14 +583,15 @@ def _sample_tokens(wl, ids, off, n):
     return np.array(sorted(pick)[:max(n, len(pick))], np.int32)
 
 
-# decode_c256 / decode_c512: not benchmark workloads; the largest batches the decode-sized expert-FFN kernel takes at the
-# production shape (8 and 16 rows per expert on average: passes of 16 tokens, some experts with two passes)
+# decode_c256 / c512 / c768: not benchmark workloads; mid-size batches up to the largest the decode-sized expert-FFN kernel takes at the
+# production shape (8, 16 and 24 rows per expert on average: passes of 16 tokens, experts with two or three passes)
 _EXTRA = {"decode_c256": inputs.Workload("decode_c256", 256, 4096, 2048, 256, 8),
-          "decode_c512": inputs.Workload("decode_c512", 512, 4096, 2048, 256, 8)}
+          "decode_c512": inputs.Workload("decode_c512", 512, 4096, 2048, 256, 8),
+          "decode_c768": inputs.Workload("decode_c768", 768, 4096, 2048, 256, 8)}
 
 
 @pytest.mark.parametrize("name,n_tokens", [("prefill_8k", 24), ("prefill_32k_skewed", 24), ("decode_c256", 16),
-                                           ("decode_c512", 16)])
+                                           ("decode_c512", 16), ("decode_c768", 16)])
 def test_layer_prefill_sampled(name, n_tokens, prod_weights):
     wl = inputs.WORKLOADS[name] if name in inputs.WORKLOADS else _EXTRA[name]
     (w13, s13, w2, s2), wdev = prod_weights
