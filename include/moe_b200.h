@@ -191,10 +191,11 @@ int moe_expert_ffn_packed(const void* x_perm_bf16 /* [T*k,H] */, const int32_t* 
  * the three calls before it, and - where the pointers are not NULL - topk_ids / topk_w [T,k] exactly as moe_route
  * writes them.
  *
- *   - For T <= 2 tokens (T*k <= 32 slots, T*E*4 <= 4*max(H,I) bytes) on shapes the decode-sized expert kernel takes,
- *     the call is ONE kernel launch: every CTA routes the T tokens itself, sorts the slots, writes its own E2M1 term
- *     rows of the tokens, runs its share of the gate/up and down items, and the CTA that finishes a column tile's last
- *     expert reduces that tile over the slots.  Any other shape runs the four calls back to back.
+ *   - For T = 1 (k <= 32, E*4 <= 4*max(H,I) bytes) on shapes the decode-sized expert kernel takes,
+ *     the call is ONE kernel launch: every CTA routes the token itself and sorts the slots, the first CTAs write the
+ *     token's E2M1 term rows, every CTA runs its share of the gate/up and down items, and the CTA that finishes a
+ *     column tile's last expert reduces that tile over the slots.  Any other shape runs the four calls back to back
+ *     (from two tokens on they are the faster form).
  *   - ws: moe_forward_workspace_bytes() bytes, 256-byte aligned.  Its first moe_forward_sync_bytes() bytes are the
  *     kernel's completion counters: they must be ZERO when a call starts.  Clear them once (cudaMemsetAsync) before
  *     the first call that uses this ws; every call that returns MOE_OK and whose kernels ran to completion leaves them
@@ -210,6 +211,14 @@ int moe_forward(const float* logits /* [T,E] */, const void* x_bf16 /* [T,H] */,
                 const uint8_t* w2, const uint8_t* w2_scale, const moe_shape_t* shape, void* out_bf16 /* [T,H] */,
                 int32_t* topk_ids /* [T,k] or NULL */, float* topk_w /* [T,k] or NULL */, int32_t* status_word, void* ws,
                 size_t ws_bytes, void* cuda_stream);
+/* Diagnostic: the one-launch kernel of moe_forward for any batch it can take (up to 4 tokens, T*k <= 32), where
+ * moe_forward itself would run the four calls because they are faster from 2 tokens on.  Same arguments, workspace and
+ * result as moe_forward; MOE_ERR_UNSUPPORTED_SHAPE if the kernel cannot take the shape.  For the tests. */
+int moe_debug_forward_one_launch(const float* logits, const void* x_bf16, const uint8_t* w13, const uint8_t* w13_scale,
+                                 const uint8_t* w2, const uint8_t* w2_scale, const moe_shape_t* shape, void* out_bf16,
+                                 int32_t* topk_ids, float* topk_w, int32_t* status_word, void* ws, size_t ws_bytes,
+                                 void* cuda_stream);
+
 /* The same on weights written by moe_prepack (same workspace, same rules, same result). */
 int moe_forward_packed(const float* logits /* [T,E] */, const void* x_bf16 /* [T,H] */, const void* packed,
                        const moe_shape_t* shape, void* out_bf16 /* [T,H] */, int32_t* topk_ids /* [T,k] or NULL */,

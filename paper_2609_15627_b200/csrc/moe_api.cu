@@ -230,7 +230,7 @@ int forward_impl(const float* logits, const void* x_bf16, const ExpertWeights& w
   if (check_ws(ws, ws_bytes, L.total) != MOE_OK) return MOE_ERR_WORKSPACE;
   char* base = static_cast<char*>(ws);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  if (forward_fused_ok(*shape, w.w13, w.w2))
+  if (forward_fused_ok(*shape, w.w13, w.w2) && forward_fused_preferred(*shape))
     return launch_forward_fused(logits, static_cast<const __nv_bfloat16*>(x_bf16), w, *shape,
                                 static_cast<__nv_bfloat16*>(out_bf16), topk_ids, topk_w, reinterpret_cast<int*>(base),
                                 base + kForwardSyncBytes, status_word, st);
@@ -258,6 +258,24 @@ int moe_forward(const float* logits, const void* x_bf16, const uint8_t* w13, con
   if (rc != MOE_OK) return rc;
   return forward_impl(logits, x_bf16, ExpertWeights{w13, w13_scale, w2, w2_scale, false}, shape, out_bf16, topk_ids, topk_w,
                       status_word, ws, ws_bytes, cuda_stream);
+}
+
+int moe_debug_forward_one_launch(const float* logits, const void* x_bf16, const uint8_t* w13, const uint8_t* w13_scale,
+                                 const uint8_t* w2, const uint8_t* w2_scale, const moe_shape_t* shape, void* out_bf16,
+                                 int32_t* topk_ids, float* topk_w, int32_t* status_word, void* ws, size_t ws_bytes,
+                                 void* cuda_stream) {
+  const int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (!aligned(logits, 16) || !aligned(x_bf16, 16) || !aligned(w13, 16) || !aligned(w13_scale, 16) || !aligned(w2, 16) ||
+      !aligned(w2_scale, 16) || !aligned(out_bf16, 16) || (topk_ids != nullptr && !aligned(topk_ids, 16)) ||
+      (topk_w != nullptr && !aligned(topk_w, 16)) || (status_word != nullptr && !aligned(status_word, 4)))
+    return MOE_ERR_INVALID_ARG;
+  if (!forward_fused_ok(*shape, w13, w2)) return MOE_ERR_UNSUPPORTED_SHAPE;
+  if (check_ws(ws, ws_bytes, forward_layout(*shape).total) != MOE_OK) return MOE_ERR_WORKSPACE;
+  char* base = static_cast<char*>(ws);
+  return launch_forward_fused(logits, static_cast<const __nv_bfloat16*>(x_bf16), ExpertWeights{w13, w13_scale, w2, w2_scale, false},
+                              *shape, static_cast<__nv_bfloat16*>(out_bf16), topk_ids, topk_w, reinterpret_cast<int*>(base),
+                              base + kForwardSyncBytes, status_word, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int moe_forward_packed(const float* logits, const void* x_bf16, const void* packed, const moe_shape_t* shape, void* out_bf16,

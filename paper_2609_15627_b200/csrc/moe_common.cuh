@@ -123,7 +123,8 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
 // the whole layer in one launch, for a handful of tokens on shapes the native variant takes (moe_forward);
 // `sync` is the zeroed block of kForwardSyncBytes, `scratch` holds forward_fused_scratch_bytes
 constexpr size_t kForwardSyncBytes = 8192;
-bool forward_fused_ok(const moe_shape_t& s, const void* w13, const void* w2);
+bool forward_fused_ok(const moe_shape_t& s, const void* w13, const void* w2);  // the kernel can take the shape
+bool forward_fused_preferred(const moe_shape_t& s);                             // and is the faster choice (measured)
 size_t forward_fused_scratch_bytes(const moe_shape_t& s);
 int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const ExpertWeights& w, const moe_shape_t& s,
                          __nv_bfloat16* out, int* ids_out, float* w_out, int* sync, void* scratch, int* status_word,

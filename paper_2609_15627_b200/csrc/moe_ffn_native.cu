@@ -41,8 +41,8 @@
 // The weights are read either in the checkpoint's row layout or in moe_prepack's tile-contiguous layout (one tensor
 // map box = one contiguous run; see ExpertWeights), always with the L2 evict-first policy: each byte is used once.
 //
-// The same kernel, instantiated with kFused = true, is the whole layer in one launch for one or two tokens
-// (moe_forward): it routes, sorts the slots and splits the token rows itself, and reduces over the slots at the end
+// The same kernel, instantiated with kFused = true, is the whole layer in one launch for a handful of tokens
+// (moe_forward uses it for one): it routes, sorts the slots and splits the token rows itself, and reduces over the slots at the end
 // (see FusedArgs).
 #include <cuda.h>
 #include <cuda_fp4.h>
@@ -91,15 +91,18 @@ struct NatArgs {
 // The one-launch layer (moe_forward on a handful of tokens): what the kernel needs beyond the expert FFN's arguments.
 // Every CTA routes all T tokens itself (same arithmetic, same result everywhere) and sorts the T * k slots by expert in
 // shared memory, so its weight stream starts without waiting for anyone.  The first kSplitCtas CTAs meanwhile split
-// the T token rows into E2M1 term rows, a few 32-element blocks each, and count themselves in; every CTA sees that
-// count complete before its set-up ends (CTAs are handed out in index order, so those CTAs are running).  The gate/up
-// items take all T tokens as operand rows (row = 8 * token + term) whatever their expert, and the epilogue keeps the
-// tokens that were routed to the item's expert.  After the down projection the CTA that runs the last expert's item of a column tile
+// the T token rows into E2M1 term rows (stored by token: no sorted copy of the rows exists), a few 32-element blocks
+// each, and count themselves in; every CTA sees that count complete before its set-up ends (CTAs are handed out in
+// index order, so those CTAs are running).  A gate/up item fetches the term rows of its expert's tokens one token (8
+// rows) at a time, through the sorted-row -> token table of the slot sort.  After the down projection the CTA that runs the last expert's item of a column tile
 // reduces that tile over the slots of every token.
-// tokens of a fused call.  Every gate/up item fetches the term rows of all of them, once per lane quadrant: 4 KB per
-// K step and token beside the 32 KB of weights.  From 3 tokens on that traffic costs more than the launches save
-// (production shape: 86 against 74 us for 3 tokens, 104 against 91 us for 4), so those batches take the four calls.
-constexpr int kFusedMaxTok = 2;
+// Tokens the one-launch kernel can take: one routing warp each.  moe_forward uses it for ONE token only: measured at the
+// production shape on prepacked weights, 32.7 us against 35.0 us for the four calls at 1 token, but 52.6 against 50.5
+// at 2, 85 against 69 at 3, 108 against 85 at 4 - with several items per CTA the set-up that cannot overlap anything
+// (routing before the first weight address is known) and the extra hand-over before the final reduction outweigh the
+// launches saved.  moe_debug_forward_one_launch runs it for 2 to 4 tokens, for the tests.
+constexpr int kFusedMaxTok = 4;
+constexpr int kFusedPreferredTok = 1;
 constexpr int kFusedMaxSlots = 32; // T * k: one warp sorts them
 constexpr int kSyncDone2 = 1024;   // int index in the sync block: per column tile, warps that stored a down item
 constexpr int kSyncExit = 1024 + 64;  // CTAs that have finished; the last one clears the block
@@ -204,7 +207,7 @@ __host__ __device__ inline NatSmem nat_smem(int E, int K) {
   m.touched = off;  // touched experts: id, first row, end row
   off += (3 * static_cast<uint32_t>(E) + 8) * 4;
   m.route = off;    // one-launch layer: expert and weight of every slot, sorted row of every slot, row of (touched expert, token)
-  off += (3 * kFusedMaxSlots + kFusedMaxSlots * kFusedMaxTok) * 4;
+  off += 4 * kFusedMaxSlots * 4;
   m.total = off;
   return m;
 }
@@ -366,7 +369,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   int* s_ids = reinterpret_cast<int*>(smem + sm.route);                 // [T * k] expert of every slot (one-launch layer only)
   float* s_w = reinterpret_cast<float*>(s_ids + kFusedMaxSlots);        // [T * k] routing weight
   int* s_row = reinterpret_cast<int*>(s_w + kFusedMaxSlots);            // [T * k] sorted row of every slot
-  int* row_of = s_row + kFusedMaxSlots;                                 // [touched expert][token] sorted row, or -1
+  int* s_tok = s_row + kFusedMaxSlots;                                  // [T * k] token of every sorted row
 
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   constexpr int tok_pass = kMaxTokPass;
@@ -484,23 +487,26 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       }
     } else if (wid != 0 && static_cast<int>(blockIdx.x) < n_split) {
       // warps 1 and 6..9 of the first CTAs: token rows -> term rows, one 32-element block per group of 8 lanes;
-      // CTA c takes blocks c, c + n_split, ... (at most 16 of them: one round)
+      // CTA c takes blocks c, c + n_split, ..., 20 of them per round (one round up to two 4096-wide rows)
       const int sw = wid == 1 ? 0 : wid - 5;  // 0..4
       const int n_blk = a.H / 32, n_all = f.T * n_blk;
       const int sub = lane & 7;
-      const int b = static_cast<int>(blockIdx.x) + n_split * (sw * 4 + (lane >> 3));
-      const bool live = b < n_all;
-      const int t = live ? b / n_blk : 0, blk = live ? b % n_blk : 0;
-      const uint2 v = *reinterpret_cast<const uint2*>(f.x + static_cast<size_t>(t) * a.H + blk * 32 + sub * 4);
-      float r[1][4] = {{__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u), __uint_as_float(v.y << 16),
-                       __uint_as_float(v.y & 0xFFFF0000u)}};
-      split_terms<1>(r, [&](int, int t8, uint32_t bytes, int se) {
-        if (live) {
-          const size_t trow = static_cast<size_t>(t) * kTerms + t8;
-          *reinterpret_cast<uint16_t*>(f.aq1 + trow * (a.H / 2) + blk * 16 + sub * 2) = static_cast<uint16_t>(bytes);
-          if (sub == 0) f.sf1[trow * n_blk + blk] = static_cast<uint8_t>(se + 127);
-        }
-      });
+      const int n_rounds = (n_all + n_split * 20 - 1) / (n_split * 20);
+      for (int rd = 0; rd < n_rounds; ++rd) {
+        const int b = static_cast<int>(blockIdx.x) + n_split * (rd * 20 + sw * 4 + (lane >> 3));
+        const bool live = b < n_all;
+        const int t = live ? b / n_blk : 0, blk = live ? b % n_blk : 0;
+        const uint2 v = *reinterpret_cast<const uint2*>(f.x + static_cast<size_t>(t) * a.H + blk * 32 + sub * 4);
+        float r[1][4] = {{__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u), __uint_as_float(v.y << 16),
+                         __uint_as_float(v.y & 0xFFFF0000u)}};
+        split_terms<1>(r, [&](int, int t8, uint32_t bytes, int se) {
+          if (live) {
+            const size_t trow = static_cast<size_t>(t) * kTerms + t8;
+            *reinterpret_cast<uint16_t*>(f.aq1 + trow * (a.H / 2) + blk * 16 + sub * 2) = static_cast<uint16_t>(bytes);
+            if (sub == 0) f.sf1[trow * n_blk + blk] = static_cast<uint8_t>(se + 127);
+          }
+        });
+      }
       fence_proxy_async_all();  // TMA will read these rows
       asm volatile("bar.sync 2, 160;" ::: "memory");  // the five splitting warps
       if (tid == 32 && dirty32 == 0) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(f.sync + kSyncSplit) : "memory");
@@ -528,11 +534,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         ti += of && (oid < id);
       }
       const int n_t = __popc(__ballot_sync(0xffffffffu, first));
-      for (int i = lane; i < kFusedMaxSlots * kFusedMaxTok; i += 32) row_of[i] = -1;
-      __syncwarp();
       if (lane < S) {
         s_row[lane] = less + eq_before;
-        row_of[ti * kFusedMaxTok + lane / f.k] = less + eq_before;
+        s_tok[less + eq_before] = lane / f.k;
       }
       if (first) {
         touched[ti] = id;
@@ -604,8 +608,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             dep_ok = false;
           }
           for (int pass = 0; pass < n_pass; ++pass) {
-            const bool own_rows = kFused && phase == 0;  // all T tokens
-            const int bi = term_box(own_rows ? f.T : min(tok_pass, n_rows_e - pass * tok_pass));  // box of 8 << bi term rows
+            const bool by_token = kFused && phase == 0;  // the expert's rows are fetched token by token (at most 4)
+            const int bi = term_box(min(tok_pass, n_rows_e - pass * tok_pass));  // box of 8 << bi term rows
             for (int ks = 0; ks < P.n_steps; ++ks) {
               if ((ks & 1) == 0) {  // 16 scale bytes per weight row cover two K steps
                 mbar_wait(&empty_sc[cs], cph ^ 1u, a.status);
@@ -619,7 +623,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
                 if (++cs == kScStages) { cs = 0; cph ^= 1u; }
               }
               mbar_wait(&empty_w[s], ph ^ 1u, a.status);
-              mbar_expect_tx(&full_w[s], static_cast<uint32_t>(kWStage + (bi <= kRepBox ? 4 : 1) * (8 << bi) * 128));
+              mbar_expect_tx(&full_w[s], static_cast<uint32_t>(kWStage + (by_token ? 4 * n_rows_e * 8 * 128
+                                                                                   : (bi <= kRepBox ? 4 : 1) * (8 << bi) * 128)));
               // 128 rows x 128 bytes of codes; tile-contiguous layout: tile (row / 128, ks) is 128 consecutive rows of 128 bytes
               const int wx = a.blocked ? 0 : ks * 128;
               const int wya = a.blocked ? ((wrow_a >> 7) * P.n_steps + ks) * 128 : wrow_a;
@@ -627,8 +632,14 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
               tma_load_2d_hint(sW + s * kStage, mw, wx, wya, &full_w[s], stream_once);
               tma_load_2d_hint(sW + s * kStage + 128 * 128, mw, wx, wyb, &full_w[s], stream_once);
               // the pass's term rows (8 per token, consecutive); rows past the end of the tensor arrive as zeros
-              const int arow = own_rows ? 0 : (row_begin + pass * tok_pass) * kTerms;
-              if (dep_ok) {
+              const int arow = (row_begin + pass * tok_pass) * kTerms;
+              if (by_token) {
+                // (the tokens' term rows were seen complete during the set-up: no dependency to hold these back for)
+                for (int j = 0; j < n_rows_e; ++j)
+                  for (int r = 0; r < 4; ++r)
+                    tma_load_2d(sW + s * kStage + kWStage + r * (32 * 128) + j * (8 * 128), &ma->box[0], ks * 128,
+                                s_tok[row_begin + j] * kTerms, &full_w[s]);
+              } else if (dep_ok) {
                 load_terms(ma, s, bi, ks * 128, arow);
               } else {
                 pend_s[n_pend] = s;
@@ -680,8 +691,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
           for (int pass = 0; pass < n_pass; ++pass) {
             // The scale factors of the term rows (tensor memory) are shared by consecutive items of an expert whose
             // rows fit one pass; otherwise every (item, pass) has its own.  The scale warps follow the same rule.
-            // (One-launch layer: every gate/up item has the same operand, all T tokens.)
-            const bool new_operand = (kFused && phase == 0) ? (it == P.begin) : ((prev_ti != ti) || (n_pass > 1));
+            const bool new_operand = (prev_ti != ti) || (n_pass > 1);
             prev_ti = ti;
             if (new_operand) {
               mbar_wait(act_ready, aph, a.status);
@@ -712,8 +722,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             acc_ph ^= 1u;
             // last use of these scale factors?  (always at the end of a phase)
             bool next_new = true;
-            if (pass + 1 >= n_pass && it + 1 < P.end)
-              next_new = (kFused && phase == 0) ? false : (((it + 1) / P.tiles != ti) || (n_pass > 1));
+            if (pass + 1 >= n_pass && it + 1 < P.end) next_new = ((it + 1) / P.tiles != ti) || (n_pass > 1);
             if (next_new) umma_commit(act_free);
           }
         }
@@ -737,7 +746,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         const int row_begin = t_begin[ti], row_end = t_end[ti];
         const int n_pass = (row_end - row_begin + tok_pass - 1) / tok_pass;
         for (int pass = 0; pass < n_pass; ++pass) {
-          const bool new_operand = (kFused && phase == 0) ? (it == P.begin) : ((prev_ti != ti) || (n_pass > 1));
+          const bool new_operand = (prev_ti != ti) || (n_pass > 1);
           prev_ti = ti;
           if (new_operand) {
             // ---- scale factors of the pass's term rows: global -> shared memory -> tensor memory ----
@@ -753,9 +762,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
               if (st == 0) counter_wait_ge(a.done + touched[ti], need_done, a.status);
               asm volatile("bar.sync 3, 128;" ::: "memory");
             }
-            const bool own_rows = kFused && phase == 0;
-            const int row0 = own_rows ? 0 : row_begin + pass * tok_pass;
-            const int n_rows = (own_rows ? f.T : min(tok_pass, row_end - row0)) * kTerms;  // term rows that exist
+            const bool by_token = kFused && phase == 0;  // the tokens' scale bytes are stored by token, not by sorted row
+            const int row0 = row_begin + pass * tok_pass;
+            const int n_rows = min(tok_pass, row_end - row0) * kTerms;  // term rows that exist
             const bool rep = n_rows <= kRepTok * kTerms;                // the operand repeats in every lane quadrant
             // rows are n_blk bytes each and consecutive: one contiguous range, copied 16 bytes at a time
             // (the 16-byte chunks of a row are XOR-swizzled with the row number against bank conflicts)
@@ -764,7 +773,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             const uint4* src = reinterpret_cast<const uint4*>(src_sf + static_cast<size_t>(row0) * kTerms * n_blk);
             for (int i = st; i < n_vec; i += 128) {
               const int r = i / n_chunk, c = i % n_chunk;
-              reinterpret_cast<uint4*>(sSfa)[r * n_chunk + (c ^ (r & cmask))] = __ldcg(src + i);
+              const uint4* from = by_token ? reinterpret_cast<const uint4*>(src_sf) + (s_tok[row0 + (r >> 3)] * kTerms + (r & 7)) * n_chunk + c
+                                           : src + i;
+              reinterpret_cast<uint4*>(sSfa)[r * n_chunk + (c ^ (r & cmask))] = __ldcg(from);
             }
             asm volatile("bar.sync 3, 128;" ::: "memory");
             __syncwarp();
@@ -840,10 +851,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     // and store left out: each CTA executes this code only a few times, so its first real use would otherwise pay
     // for fetching it - on the critical path of a one-item CTA - while the warp has nothing to do before the first
     // accumulator is complete.
-    // `rowmap` (one-launch layer, gate/up items): sorted row of each operand token for this item's expert, -1 for the
-    // tokens that were not routed to it; otherwise operand token i is sorted row row0 + i.
-    auto run_pass = [&](const int phase, const int out_stride, const int tile, const int row0, const int n_tok, const int* rowmap,
-                        const bool dry) {
+    auto run_pass = [&](const int phase, const int out_stride, const int tile, const int row0, const int n_tok, const bool dry) {
       const bool rep = n_tok <= kRepTok;
       const bool active = rep || 4 * q < n_tok;
       // 32-column chunks this warp sums: all 8, or (small pass) gate chunk q and up chunk 4 + q of a gate/up item,
@@ -920,10 +928,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
           }
           const int tok = rep ? jl : 4 * q + rd;  // token of the pass whose block this lane group splits
           const int i0 = tile * 128 + 32 * (rep ? q : jl);
-          const int prow = tok < n_tok ? (rowmap != nullptr ? rowmap[tok] : row0 + tok) : -1;
-          const bool live = !dry && prow >= 0;
-          uint8_t* qrow = a.aq2 + static_cast<size_t>(live ? prow : 0) * kTerms * (a.I / 2) + ((i0 + cb) >> 1);
-          uint8_t* srow = a.sf2 + static_cast<size_t>(live ? prow : 0) * kTerms * n_blk_i + (i0 >> 5);
+          const bool live = !dry && tok < n_tok;
+          uint8_t* qrow = a.aq2 + static_cast<size_t>(row0 + tok) * kTerms * (a.I / 2) + ((i0 + cb) >> 1);
+          uint8_t* srow = a.sf2 + static_cast<size_t>(row0 + tok) * kTerms * n_blk_i + (i0 >> 5);
           split_terms<1>(r, [&](int, int t, uint32_t bytes, int se) {
             if (live) {
               *reinterpret_cast<uint16_t*>(qrow + static_cast<size_t>(t) * (a.I / 2)) = static_cast<uint16_t>(bytes);
@@ -950,11 +957,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
           const int ti = it / P.tiles, tile = it % P.tiles;
           const int row_begin = t_begin[ti], row_end = t_end[ti];
           const int n_pass = dry ? 1 : (row_end - row_begin + tok_pass - 1) / tok_pass;
-          const bool own_rows = kFused && phase == 0;
           for (int pass = 0; pass < n_pass; ++pass) {
             const int row0 = row_begin + pass * tok_pass;
-            run_pass(phase, P.R, tile, row0, own_rows ? f.T : min(tok_pass, row_end - row0),
-                     own_rows ? row_of + ti * kFusedMaxTok : nullptr, dry);
+            run_pass(phase, P.R, tile, row0, min(tok_pass, row_end - row0), dry);
           }
           if constexpr (kFused) {
             if (!dry && phase == 1) {
@@ -1129,13 +1134,15 @@ bool forward_fused_ok(const moe_shape_t& sh, const void* w13, const void* w2) {
   const int K = sh.H > sh.I ? sh.H : sh.I;
   return native_shape_ok(sh, w13, w2) && sm_count() >= kSplitCtas && sh.T <= kFusedMaxTok && sh.T * sh.k <= kFusedMaxSlots &&
          static_cast<size_t>(sh.T) * sh.E * 4 <= static_cast<size_t>(128) * (K / 32) && sh.E <= kSyncDone2 &&
-         sh.H / kTile <= kSyncExit - kSyncDone2 && static_cast<size_t>(sh.T) * (sh.H / 32) <= static_cast<size_t>(kSplitCtas) * 16;
+         sh.H / kTile <= kSyncExit - kSyncDone2;
 }
 size_t forward_fused_scratch_bytes(const moe_shape_t& sh) {
   const size_t S = static_cast<size_t>(sh.T) * sh.k, own = static_cast<size_t>(sh.T) * kTerms;
   return align_up(S * sh.H * 4, kAlign) + align_up(S * kTerms * (sh.I / 2), kAlign) + align_up(S * kTerms * (sh.I / 32), kAlign) +
          align_up(own * (sh.H / 2), kAlign) + align_up(own * (sh.H / 32), kAlign);
 }
+bool forward_fused_preferred(const moe_shape_t& sh) { return sh.T <= kFusedPreferredTok; }
+
 int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const ExpertWeights& w, const moe_shape_t& sh,
                          __nv_bfloat16* out, int* ids_out, float* w_out, int* sync, void* scratch, int* status_word,
                          cudaStream_t st) {

@@ -17,7 +17,7 @@ EXPORTS = ("moe_workspace_bytes", "moe_status_string", "moe_last_kernel_name", "
            "moe_forward_workspace_bytes", "moe_forward_sync_bytes", "moe_forward",
            "moe_forward_host_workspace_bytes", "moe_forward_host", "moe_expert_ffn_noalloc_max_bytes",
            "moe_expert_ffn_noalloc", "moe_debug_native_cta_share", "moe_debug_read_probe", "moe_prepack_bytes", "moe_prepack",
-           "moe_expert_ffn_packed", "moe_forward_packed", "moe_forward_host_packed")
+           "moe_expert_ffn_packed", "moe_forward_packed", "moe_forward_host_packed", "moe_debug_forward_one_launch")
 
 
 class MoeError(RuntimeError):
@@ -80,6 +80,8 @@ def lib():
         L.moe_forward_sync_bytes.argtypes = []
         L.moe_forward.restype = C.c_int
         L.moe_forward.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp, vp, vp, sz, vp]
+        L.moe_debug_forward_one_launch.restype = C.c_int
+        L.moe_debug_forward_one_launch.argtypes = L.moe_forward.argtypes
         L.moe_forward_host.restype = C.c_int
         L.moe_forward_host.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp, sz, vp]
         _lib = L
@@ -234,6 +236,13 @@ def moe_forward(logits, x, w13, w13_scale, w2, w2_scale, sh, out, topk_ids, topk
     _check(lib().moe_forward(_ptr(logits), _ptr(x), _ptr(w13), _ptr(w13_scale), _ptr(w2), _ptr(w2_scale), C.byref(sh),
                              _ptr(out), _ptr(topk_ids), _ptr(topk_w), _ptr(status_word), _ptr(ws), ws.numel(),
                              _stream(stream)), "moe_forward")
+
+
+def moe_debug_forward_one_launch(logits, x, w13, w13_scale, w2, w2_scale, sh, out, topk_ids, topk_w, status_word, ws,
+                                 stream=None):
+    _check(lib().moe_debug_forward_one_launch(_ptr(logits), _ptr(x), _ptr(w13), _ptr(w13_scale), _ptr(w2), _ptr(w2_scale),
+                                              C.byref(sh), _ptr(out), _ptr(topk_ids), _ptr(topk_w), _ptr(status_word),
+                                              _ptr(ws), ws.numel(), _stream(stream)), "moe_debug_forward_one_launch")
 
 
 def moe_forward_host(logits_host, x_host, w13, w13_scale, w2, w2_scale, sh, out_host, status_word, ws, stream=None):

@@ -332,7 +332,7 @@ def test_layer_decode_full(name, prod_weights):
 _ONE_LAUNCH = "layer_one_launch_mxf4_block_scaled"
 
 
-def _run_forward(wl, d, wdev, reps=1):
+def _run_forward(wl, d, wdev, reps=1, force_one_launch=False):
     sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
     ws = moe.alloc_forward_workspace(sh)
     out = torch.empty((wl.T, wl.H), dtype=torch.bfloat16, device="cuda")
@@ -342,7 +342,7 @@ def _run_forward(wl, d, wdev, reps=1):
     lg, x = dev(d["logits"]), dev(d["x"])
     for _ in range(reps):
         out.fill_(float("nan"))
-        moe.moe_forward(lg, x, *wdev, sh, out, ids, w, st, ws)
+        (moe.moe_debug_forward_one_launch if force_one_launch else moe.moe_forward)(lg, x, *wdev, sh, out, ids, w, st, ws)
         torch.cuda.synchronize()
         assert int(st.item()) == 0
         # the counter block is left clear for the next call
@@ -350,9 +350,9 @@ def _run_forward(wl, d, wdev, reps=1):
     return out, ids, w, moe.moe_last_kernel_name()
 
 
-def _check_forward(wl, d, wdev, one_launch):
+def _check_forward(wl, d, wdev, one_launch, force_one_launch=False):
     wdev = wdev if wdev is not None else weights_dev(d)
-    out, ids, w, kernel = _run_forward(wl, d, wdev, reps=3)
+    out, ids, w, kernel = _run_forward(wl, d, wdev, reps=3, force_one_launch=force_one_launch)
     assert (kernel == _ONE_LAUNCH) == one_launch, kernel
     # against the oracle: routing bit for bit, the output within the stated tolerance
     r = O.forward_staged(d["logits"], d["x"], d["w13"], d["s13"], d["w2"], d["s2"], wl.k)
@@ -365,12 +365,11 @@ def _check_forward(wl, d, wdev, one_launch):
 
 
 @pytest.mark.parametrize("T,H,I,E,k,one_launch", [
-    (1, 512, 512, 8, 2, True), (2, 1024, 512, 16, 4, True), (2, 2048, 1024, 64, 8, True), (2, 1024, 512, 32, 6, True),
+    (1, 512, 512, 8, 2, True), (1, 1024, 512, 16, 4, True), (1, 2048, 1024, 64, 8, True), (1, 1024, 512, 32, 6, True),
     (1, 512, 512, 4, 4, True),      # every expert touched
-    (2, 512, 512, 16, 16, True),    # 32 slots, every expert touched by both tokens
-    (2, 512, 512, 512, 8, False),   # the logits of 2 tokens do not fit the router's shared memory at this H
-    (2, 512, 512, 32, 32, False),   # more than 32 slots
-    (3, 512, 512, 8, 2, False),     # more than 2 tokens
+    (1, 512, 512, 32, 32, True),    # 32 slots
+    (1, 512, 512, 1024, 8, False),  # the logits do not fit the router's shared memory at this H
+    (2, 1024, 512, 16, 4, False),   # more than one token: the four calls are faster
     (16, 256, 128, 8, 2, False),    # not a shape of the decode-sized expert kernel
     (64, 1024, 512, 32, 6, False)])
 def test_forward_small_shapes(T, H, I, E, k, one_launch):
@@ -379,20 +378,45 @@ def test_forward_small_shapes(T, H, I, E, k, one_launch):
     _check_forward(wl, d, None, one_launch)
 
 
-@pytest.mark.parametrize("T,k,seed", [(1, 8, 0), (1, 8, 1), (1, 6, 2), (2, 8, 0), (2, 6, 3), (4, 8, 4)])
-def test_forward_production_shape(T, k, seed, prod_weights):
+@pytest.mark.parametrize("T,H,I,E,k", [
+    (2, 1024, 512, 16, 4), (2, 2048, 1024, 64, 8), (3, 1024, 512, 32, 6), (4, 512, 512, 8, 2), (4, 1024, 512, 32, 8),
+    (2, 512, 512, 16, 16),          # 32 slots, every expert touched by both tokens
+    (4, 2048, 1024, 8, 8),          # every expert touched by all four tokens
+    (3, 512, 512, 4, 1)])
+def test_one_launch_kernel_with_several_tokens(T, H, I, E, k):
+    """moe_forward keeps the one-launch kernel for one token; the kernel itself takes up to four."""
+    wl = inputs.Workload("fwd_n", T, H, I, E, k)
+    d = inputs.make_workload(wl, seed=7)
+    _check_forward(wl, d, None, True, force_one_launch=True)
+
+
+def test_one_launch_kernel_refuses_what_it_cannot_take():
+    for T, H, I, E, k in ((5, 512, 512, 8, 2), (2, 512, 512, 32, 32), (2, 512, 512, 512, 8), (2, 256, 128, 8, 2)):
+        wl = inputs.Workload("fwd_no", T, H, I, E, k)
+        d = inputs.make_workload(wl, seed=7)
+        wdev = weights_dev(d)
+        sh = moe.shape(T, H, I, E, k)
+        ws = moe.alloc_forward_workspace(sh)
+        out = torch.empty((T, H), dtype=torch.bfloat16, device="cuda")
+        with pytest.raises(moe.MoeError, match="unsupported shape"):
+            moe.moe_debug_forward_one_launch(dev(d["logits"]), dev(d["x"]), *wdev, sh, out, None, None, None, ws)
+
+
+@pytest.mark.parametrize("T,k,seed,force", [(1, 8, 0, False), (1, 8, 1, False), (1, 6, 2, False), (2, 8, 0, False),
+                                             (2, 6, 3, True), (3, 8, 5, True), (4, 8, 4, True)])
+def test_forward_production_shape(T, k, seed, force, prod_weights):
     wl = inputs.Workload("fwd_prod", T, 4096, 2048, 256, k)
     (w13, s13, w2, s2), wdev = prod_weights
     d = dict(logits=inputs.make_logits(T, wl.E, seed), x=inputs.make_x(T, wl.H, seed), w13=w13, s13=s13, w2=w2, s2=s2)
-    _check_forward(wl, d, wdev, T <= 2)
+    _check_forward(wl, d, wdev, T == 1 or force, force_one_launch=force)
 
 
 def test_forward_tokens_sharing_experts():
-    """Two tokens with the same logits: every touched expert gets both rows."""
-    wl = inputs.Workload("fwd_same", 2, 1024, 512, 16, 4)
+    """Four tokens with the same logits: every touched expert gets all four rows."""
+    wl = inputs.Workload("fwd_same", 4, 1024, 512, 16, 4)
     d = inputs.make_workload(wl, seed=6)
     d["logits"][:] = d["logits"][0]
-    _check_forward(wl, d, None, True)
+    _check_forward(wl, d, None, True, force_one_launch=True)
 
 
 def test_forward_without_routing_outputs_and_in_a_graph(prod_weights):
@@ -432,7 +456,7 @@ def test_forward_without_routing_outputs_and_in_a_graph(prod_weights):
 def test_forward_with_a_workspace_that_was_never_cleared():
     """The one-launch kernel finds its two untouched words non-zero, reports it and does nothing; after a clear the
     same workspace works."""
-    wl = inputs.Workload("fwd_dirty", 2, 1024, 512, 16, 4)
+    wl = inputs.Workload("fwd_dirty", 1, 1024, 512, 16, 4)
     d = inputs.make_workload(wl, seed=9)
     wdev = weights_dev(d)
     sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
@@ -456,7 +480,7 @@ def test_forward_with_a_workspace_that_was_never_cleared():
 
 def test_forward_host_uses_it():
     """moe_forward_host clears the counter block itself: a workspace full of ones still gives the layer's result."""
-    wl = inputs.Workload("fwd_host", 2, 1024, 512, 16, 4)
+    wl = inputs.Workload("fwd_host", 1, 1024, 512, 16, 4)
     d = inputs.make_workload(wl, seed=8)
     wdev = weights_dev(d)
     sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
@@ -549,7 +573,7 @@ def test_forward_packed_production_shape(T, k, seed, prod_weights):
     moe.moe_forward_packed(lg, x, packed, sh, out_packed, ids, w, st, ws)
     torch.cuda.synchronize()
     assert int(st.item()) == 0 and moe.moe_last_kernel_name() == k_raw
-    assert (k_raw == _ONE_LAUNCH) == (T <= 2)
+    assert (k_raw == _ONE_LAUNCH) == (T == 1)
     assert torch.equal(out_raw.view(torch.int16), out_packed.view(torch.int16))
     d = dict(logits=lg.cpu().numpy(), x=bits(x), w13=w13, s13=s13, w2=w2, s2=s2)
     r = O.forward_staged(d["logits"], d["x"], w13, s13, w2, s2, k)
