@@ -30,7 +30,7 @@ DECODE = ("decode_c1", "decode_c64")
 # dram__bytes_read.sum + dram__bytes_write.sum per moe_expert_ffn call from one ncu capture of the
 # workload (see profiles/); None until captured.
 NCU_TRAFFIC_BYTES = {
-    "decode_c1_one_launch": 110514000,  # ffn_native_kernel<true>, the whole layer: 107.14 MB read + 3.38 MB written (mean of two launches)
+    "decode_c1_one_launch": 110440700,  # ffn_native_kernel<true>, the whole layer: 107.14 MB read + 3.30 MB written (mean of two launches)
     "decode_c1": 111216000,      # ffn_native_kernel<false>: 107.19 MB read + 4.03 MB written (profiles/ffn_native_decode.md)
     "decode_c64": 3064384880,    # 3057.9 MB read + 6.5 MB written
     "prefill_8k": 5611119000,    # ffn_umma_kernel<true> 2.882 + 0.263 GB, <false> 1.431 + 1.034 GB (profiles/ffn_umma_prefill_8k.md)
