@@ -28,7 +28,49 @@ MOE_DEVINL float exp_fixed(float d) {
 // One warp per token.  row = this warp's copy of the token's logits in shared memory.
 // Returns through lane j (< k) the j-th selected expert and its logit: experts in the order (logit descending by
 // IEEE comparison, so -0 ties with +0; expert id ascending among equals).
+// Up to 256 experts: a lane's eight logits stay in registers as integer keys that order like the floats (-0 counted
+// as +0), so a round is a register max, two warp reductions and a few selects.
+MOE_DEVINL void warp_topk_256(const float* row, int E, int k, int lane, int* my_id, float* my_v) {
+  unsigned key[8];
+  unsigned valid = 0u;  // bit u: element lane + 32*u exists and is not selected yet
+#pragma unroll
+  for (int u = 0; u < 8; ++u) {
+    const int idx = u * 32 + lane;
+    const float v = idx < E ? row[idx] : 0.0f;
+    const unsigned b = __float_as_uint(v == 0.0f ? 0.0f : v);
+    key[u] = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+    valid |= (idx < E ? 1u : 0u) << u;
+  }
+  *my_id = 0;
+  *my_v = 0.0f;
+  for (int j = 0; j < k; ++j) {
+    unsigned best = 0u;
+    bool any = false;
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      if ((valid >> u) & 1u) {
+        best = any ? max(best, key[u]) : key[u];
+        any = true;
+      }
+    const unsigned top = __reduce_max_sync(0xffffffffu, any ? best : 0u);
+    unsigned cand = 0xffffffffu;  // lowest id in this lane that holds the top key
+#pragma unroll
+    for (int u = 7; u >= 0; --u)
+      if (((valid >> u) & 1u) && key[u] == top) cand = static_cast<unsigned>(u * 32 + lane);
+    const unsigned win = __reduce_min_sync(0xffffffffu, cand);
+    if ((win & 31u) == static_cast<unsigned>(lane)) valid &= ~(1u << (win >> 5));
+    if (lane == j) {
+      *my_id = static_cast<int>(win);
+      *my_v = __uint_as_float((top & 0x80000000u) ? (top & 0x7fffffffu) : ~top);
+    }
+  }
+}
+
 MOE_DEVINL void warp_topk(const float* row, int E, int k, int lane, int* my_id, float* my_v) {
+  if (E <= 256) {
+    warp_topk_256(row, E, k, lane, my_id, my_v);
+    return;
+  }
   unsigned taken = 0u;  // bit i: element lane + 32*i already selected
   *my_id = 0;
   *my_v = 0.0f;
