@@ -134,10 +134,13 @@ constexpr int kTermBoxes = 5;
 struct alignas(64) TermMaps {
   CUtensorMap box[kTermBoxes];
 };
-// A pass of at most kRepTok tokens fills one lane quadrant of the accumulator (32 operand rows).  Its term rows are
-// then loaded once per quadrant, so that each of the four epilogue warps finds every token in its own quadrant and
-// takes a quarter of the columns instead of one warp taking them all.
-constexpr int kRepTok = 4, kRepBox = 2;  // boxes 0..kRepBox hold at most kRepTok tokens
+// A pass of one token is loaded once per lane quadrant of the accumulator, so that each of the four epilogue warps finds
+// the token in its own quadrant and takes a quarter of the columns instead of one warp taking them all (decode_c1:
+// every expert has one row, and the epilogues are on the critical path).  The scheme works for up to 4 tokens (one
+// quadrant = 32 operand rows), but every repeated KB of term rows competes with the weight stream: measured on
+// decode_c64 (2.3 rows per expert on average) the expert-FFN call takes 545 us with passes of up to 4 tokens repeated,
+// 526 us with single-token passes only (row-layout weights; 560 against 550 us under the power cap).
+constexpr int kRepBox = 0, kRepTok = 1 << kRepBox;  // boxes 0..kRepBox hold at most kRepTok tokens
 MOE_DEVINL int term_box(int n_tok) { return n_tok <= 1 ? 0 : (n_tok <= 2 ? 1 : (n_tok <= 4 ? 2 : (n_tok <= 8 ? 3 : 4))); }
 
 // One projection as the kernel sees it
@@ -610,6 +613,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
           for (int pass = 0; pass < n_pass; ++pass) {
             const bool by_token = kFused && phase == 0;  // the expert's rows are fetched token by token (at most 4)
             const int bi = term_box(min(tok_pass, n_rows_e - pass * tok_pass));  // box of 8 << bi term rows
+            const int n_rep = bi <= kRepBox ? 4 : 1;
             for (int ks = 0; ks < P.n_steps; ++ks) {
               if ((ks & 1) == 0) {  // 16 scale bytes per weight row cover two K steps
                 mbar_wait(&empty_sc[cs], cph ^ 1u, a.status);
@@ -623,8 +627,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
                 if (++cs == kScStages) { cs = 0; cph ^= 1u; }
               }
               mbar_wait(&empty_w[s], ph ^ 1u, a.status);
-              mbar_expect_tx(&full_w[s], static_cast<uint32_t>(kWStage + (by_token ? 4 * n_rows_e * 8 * 128
-                                                                                   : (bi <= kRepBox ? 4 : 1) * (8 << bi) * 128)));
+              mbar_expect_tx(&full_w[s], static_cast<uint32_t>(kWStage + n_rep * (by_token ? n_rows_e * 8 : 8 << bi) * 128));
               // 128 rows x 128 bytes of codes; tile-contiguous layout: tile (row / 128, ks) is 128 consecutive rows of 128 bytes
               const int wx = a.blocked ? 0 : ks * 128;
               const int wya = a.blocked ? ((wrow_a >> 7) * P.n_steps + ks) * 128 : wrow_a;
@@ -636,7 +639,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
               if (by_token) {
                 // (the tokens' term rows were seen complete during the set-up: no dependency to hold these back for)
                 for (int j = 0; j < n_rows_e; ++j)
-                  for (int r = 0; r < 4; ++r)
+                  for (int r = 0; r < n_rep; ++r)
                     tma_load_2d(sW + s * kStage + kWStage + r * (32 * 128) + j * (8 * 128), &ma->box[0], ks * 128,
                                 s_tok[row_begin + j] * kTerms, &full_w[s]);
               } else if (dep_ok) {
