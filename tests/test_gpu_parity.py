@@ -478,6 +478,33 @@ def test_forward_with_a_workspace_that_was_never_cleared():
     assert np.array_equal(bits(out), bits(out4))
 
 
+def test_forward_bounded_wait_runs_out_and_the_next_call_works():
+    """A wait that nothing can satisfy: the count of CTAs that have split the token (word 1089 of the counter block)
+    starts far below zero, so it never reaches its target.  The wait gives up after its limit (about two seconds), the
+    kernel reports MOE_ERR_TIMEOUT through the status word and runs to its end, the last CTA clears the block as
+    always, and the same workspace then serves a correct call."""
+    wl = inputs.Workload("fwd_wait", 1, 1024, 512, 16, 4)
+    d = inputs.make_workload(wl, seed=10)
+    wdev = weights_dev(d)
+    sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
+    ws = moe.alloc_forward_workspace(sh)
+    ws[:moe.moe_forward_sync_bytes()].view(torch.int32)[1024 + 65] = -1000
+    out = torch.zeros((wl.T, wl.H), dtype=torch.bfloat16, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    lg, x = dev(d["logits"]), dev(d["x"])
+    moe.moe_forward(lg, x, *wdev, sh, out, None, None, st, ws)
+    torch.cuda.synchronize()
+    assert moe.moe_last_kernel_name() == _ONE_LAUNCH
+    assert int(st.item()) == 5                      # MOE_ERR_TIMEOUT
+    assert int(ws[:moe.moe_forward_sync_bytes()].view(torch.int32).abs().sum().item()) == 0
+    st.zero_()
+    moe.moe_forward(lg, x, *wdev, sh, out, None, None, st, ws)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    buf, out4 = run_layer(wl, d, wdev)
+    assert np.array_equal(bits(out), bits(out4))
+
+
 def test_forward_host_uses_it():
     """moe_forward_host clears the counter block itself: a workspace full of ones still gives the layer's result."""
     wl = inputs.Workload("fwd_host", 1, 1024, 512, 16, 4)
