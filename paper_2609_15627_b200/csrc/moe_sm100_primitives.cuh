@@ -73,7 +73,7 @@ MOE_DEVINL void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* b
                "l"(src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
 }
-// 2-D tiled tensor-map load (no multicast); x is the innermost coordinate and x * element size must be a
+// 2-D tiled tensor-map load into this CTA only; x is the innermost coordinate and x * element size must be a
 // multiple of 16 bytes
 MOE_DEVINL void tma_load_2d(void* dst, const void* tmap, int x, int y, uint64_t* bar) {
   asm volatile(
