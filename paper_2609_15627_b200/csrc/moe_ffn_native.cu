@@ -140,13 +140,17 @@ struct alignas(64) TermMaps {
 // quadrant = 32 operand rows), but every repeated KB of term rows competes with the weight stream: measured on
 // decode_c64 (2.3 rows per expert on average) the expert-FFN call takes 545 us with passes of up to 4 tokens repeated,
 // 526 us with single-token passes only (row-layout weights; 560 against 550 us under the power cap).
+// Nor is it worth anything where the epilogue hides behind the next item's MMAs: a CTA repeats only in a phase in which
+// it has at most kRepMaxItems items (another 0.7 % on decode_c64, where a CTA has 24).
 constexpr int kRepBox = 0, kRepTok = 1 << kRepBox;  // boxes 0..kRepBox hold at most kRepTok tokens
+constexpr int kRepMaxItems = 2;
 MOE_DEVINL int term_box(int n_tok) { return n_tok <= 1 ? 0 : (n_tok <= 2 ? 1 : (n_tok <= 4 ? 2 : (n_tok <= 8 ? 3 : 4))); }
 
 // One projection as the kernel sees it
 struct Phase {
   int K, R, n_steps, tiles;  // reduction length, weight rows per expert, K steps, items per expert
   int begin, end;            // this CTA's items (at most 1024 experts x 32 tiles)
+  bool rep_ok;               // few enough of them for single-token passes to be repeated per lane quadrant
 };
 // Items go to CTAs in contiguous shares: gate/up items evenly, per0 each.  A down item of expert t is placed as if it
 // followed that expert's last gate/up item in the gate/up list, its expert's down items spread over the span of the
@@ -187,6 +191,7 @@ MOE_DEVINL Phase phase_of(int ph, const NatArgs& a, const int* shares) {
   p.tiles = p.R / kTile;
   p.begin = shares[2 * ph];
   p.end = shares[2 * ph + 1];
+  p.rep_ok = p.end - p.begin <= kRepMaxItems;
   return p;
 }
 
@@ -570,10 +575,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       bool pdl_done = kFused, dep_ok = kFused;
       if (kFused) fence_proxy_async_all();  // they were written through the generic proxy
       int dep_phase = 0, dep_e = -1;
-      int n_pend = 0, pend_s[kWStages], pend_x[kWStages], pend_y[kWStages], pend_b[kWStages];
-      // term rows of one K step; a pass of at most kRepTok tokens gets them once per lane quadrant of the accumulator
-      auto load_terms = [&](const TermMaps* ma, int stage, int bi, int x, int y) {
-        const int n_rep = bi <= kRepBox ? 4 : 1;
+      int n_pend = 0, pend_s[kWStages], pend_x[kWStages], pend_y[kWStages], pend_b[kWStages], pend_r[kWStages];
+      // term rows of one K step, n_rep times: once, or once per lane quadrant of the accumulator
+      auto load_terms = [&](const TermMaps* ma, int stage, int bi, int n_rep, int x, int y) {
         for (int r = 0; r < n_rep; ++r)
           tma_load_2d(sW + stage * kStage + kWStage + r * (32 * 128), &ma->box[bi], x, y, &full_w[stage]);
       };
@@ -587,7 +591,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
           fence_proxy_async_all();  // the rows were written through the generic proxy, TMA reads through the async one
         }
         const TermMaps* ma = dep_phase == 0 ? &tmap_a1 : &tmap_a2;
-        for (int i = 0; i < n_pend; ++i) load_terms(ma, pend_s[i], pend_b[i], pend_x[i], pend_y[i]);
+        for (int i = 0; i < n_pend; ++i) load_terms(ma, pend_s[i], pend_b[i], pend_r[i], pend_x[i], pend_y[i]);
         n_pend = 0;
         dep_ok = true;
       };
@@ -613,7 +617,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
           for (int pass = 0; pass < n_pass; ++pass) {
             const bool by_token = kFused && phase == 0;  // the expert's rows are fetched token by token (at most 4)
             const int bi = term_box(min(tok_pass, n_rows_e - pass * tok_pass));  // box of 8 << bi term rows
-            const int n_rep = bi <= kRepBox ? 4 : 1;
+            const int n_rep = (P.rep_ok && bi <= kRepBox) ? 4 : 1;
             for (int ks = 0; ks < P.n_steps; ++ks) {
               if ((ks & 1) == 0) {  // 16 scale bytes per weight row cover two K steps
                 mbar_wait(&empty_sc[cs], cph ^ 1u, a.status);
@@ -643,8 +647,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
                     tma_load_2d(sW + s * kStage + kWStage + r * (32 * 128) + j * (8 * 128), &ma->box[0], ks * 128,
                                 s_tok[row_begin + j] * kTerms, &full_w[s]);
               } else if (dep_ok) {
-                load_terms(ma, s, bi, ks * 128, arow);
+                load_terms(ma, s, bi, n_rep, ks * 128, arow);
               } else {
+                pend_r[n_pend] = n_rep;
                 pend_s[n_pend] = s;
                 pend_x[n_pend] = ks * 128;
                 pend_y[n_pend] = arow;
@@ -768,7 +773,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             const bool by_token = kFused && phase == 0;  // the tokens' scale bytes are stored by token, not by sorted row
             const int row0 = row_begin + pass * tok_pass;
             const int n_rows = min(tok_pass, row_end - row0) * kTerms;  // term rows that exist
-            const bool rep = n_rows <= kRepTok * kTerms;                // the operand repeats in every lane quadrant
+            const bool rep = P.rep_ok && n_rows <= kRepTok * kTerms;    // the operand repeats in every lane quadrant
             // rows are n_blk bytes each and consecutive: one contiguous range, copied 16 bytes at a time
             // (the 16-byte chunks of a row are XOR-swizzled with the row number against bank conflicts)
             const int n_chunk = n_blk / 16, cmask = min(n_chunk, 8) - 1;
@@ -854,8 +859,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     // and store left out: each CTA executes this code only a few times, so its first real use would otherwise pay
     // for fetching it - on the critical path of a one-item CTA - while the warp has nothing to do before the first
     // accumulator is complete.
-    auto run_pass = [&](const int phase, const int out_stride, const int tile, const int row0, const int n_tok, const bool dry) {
-      const bool rep = n_tok <= kRepTok;
+    auto run_pass = [&](const int phase, const bool rep_ok, const int out_stride, const int tile, const int row0, const int n_tok,
+                        const bool dry) {
+      const bool rep = rep_ok && n_tok <= kRepTok;
       const bool active = rep || 4 * q < n_tok;
       // 32-column chunks this warp sums: all 8, or (small pass) gate chunk q and up chunk 4 + q of a gate/up item,
       // chunks 2q and 2q + 1 of a down item
@@ -962,7 +968,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
           const int n_pass = dry ? 1 : (row_end - row_begin + tok_pass - 1) / tok_pass;
           for (int pass = 0; pass < n_pass; ++pass) {
             const int row0 = row_begin + pass * tok_pass;
-            run_pass(phase, P.R, tile, row0, min(tok_pass, row_end - row0), dry);
+            run_pass(phase, P.rep_ok, P.R, tile, row0, min(tok_pass, row_end - row0), dry);
           }
           if constexpr (kFused) {
             if (!dry && phase == 1) {
