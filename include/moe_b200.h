@@ -4,7 +4,9 @@
  * The layer (paper, figure "Execution structure" and the accepted large-prefill path in the section
  * "Prefill optimization"): Router Top-k -> route production (expert sorter) -> FP4 routed experts
  * gate/up -> activation rounded to BF16 -> down projection, FP32 per-slot partials, unique-slot
- * stores -> fixed-order Top-k FP32 reduction.  One call per stage, in that order.
+ * stores -> fixed-order Top-k FP32 reduction.  One call per stage, in that order; moe_forward runs the
+ * four stages as one call (one kernel launch for a single token), and moe_prepack re-lays the expert
+ * weights once, byte for byte, for the *_packed forms of the calls that read them.
  *
  * Notation: T tokens, H hidden size, I expert intermediate size, E experts, k experts per token,
  * S = T*k slots, flat slot s = t*k + j (j = rank of the expert for token t, 0 = largest logit).
@@ -14,7 +16,7 @@
  *     row-major array (innermost dimension contiguous).  The caller owns every buffer; the library
  *     allocates, frees and retains nothing.  `ws` is caller-provided scratch of at least
  *     moe_workspace_bytes() bytes, 256-byte aligned; its contents need not survive between calls
- *     and need no initialisation.
+ *     and need no initialisation (moe_forward's workspace has one exception, stated there).
  *   - Every call only enqueues work on `cuda_stream` (a cudaStream_t passed as void*, NULL = the
  *     legacy default stream) and returns; there is no host synchronisation and no device-to-host copy.
  *   - Return value: a moe_status_t.  Argument errors are found on the host before anything is
