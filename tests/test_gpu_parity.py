@@ -614,6 +614,33 @@ def test_forward_packed_production_shape(T, k, seed, prod_weights):
     assert np.array_equal(oh.numpy().view(np.uint16), bits(out_packed))
 
 
+def test_forward_packed_on_the_benchmark_batches(prod_weights):
+    """decode_c1 as bench.py runs it: the 32 seeded batches of its cycle through moe_forward_packed back to back on one
+    workspace (the one-launch kernel), each compared bit for bit with the four calls on the row-layout weights, and
+    the first and last with the oracle."""
+    wl = inputs.WORKLOADS["decode_c1"]
+    (w13, s13, w2, s2), wdev = prod_weights
+    sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
+    packed = moe.moe_prepack(*wdev, sh)
+    ws = moe.alloc_forward_workspace(sh)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    batches = [(inputs.make_logits(wl.T, wl.E, 7000 + i), inputs.make_x(wl.T, wl.H, 7000 + i)) for i in range(32)]
+    dev_batches = [(dev(l), dev(x)) for l, x in batches]
+    outs = [torch.empty((wl.T, wl.H), dtype=torch.bfloat16, device="cuda") for _ in batches]
+    for (lg, x), o in zip(dev_batches, outs):
+        moe.moe_forward_packed(lg, x, packed, sh, o, None, None, st, ws)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0 and moe.moe_last_kernel_name() == _ONE_LAUNCH
+    buf = moe.LayerBuffers(sh)
+    for i, ((lg, x), o) in enumerate(zip(dev_batches, outs)):
+        out4 = moe.moe_layer(lg, x, wdev, buf)
+        torch.cuda.synchronize()
+        assert torch.equal(o.view(torch.int16), out4.view(torch.int16)), "batch %d" % i
+    for i in (0, 31):
+        r = O.forward_staged(batches[i][0], batches[i][1], w13, s13, w2, s2, wl.k)
+        check_out(bits(outs[i]), r["out"], r["out_f32"], "decode_c1 batch %d" % i)
+
+
 def _sample_tokens(wl, ids, off, n):
     """Tokens covering the first and last row of the heaviest expert, a row of many experts, and
     rows at tile boundaries; the rest seeded."""
