@@ -1,11 +1,17 @@
 """Benchmark of the routed FP4 mixture-of-experts layer on B200.
 
 A step is one pass of the whole hot path (moe_route -> moe_permute -> moe_expert_ffn -> moe_combine)
-over one batch of seeded synthetic input.  For a handful of tokens (decode_c1) the library runs that path
+over one batch of seeded synthetic input.  For a single token (decode_c1) the library runs that path
 as ONE kernel launch behind moe_forward; the step is then that call, and the four calls are timed beside
 it.  Prints ONE JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+With no --workload the line's headline keys describe decode_c1 (exactly K timed steps) and a top-level
+`workloads` object carries all four production workloads - decode_c1, decode_c64, prefill_8k,
+prefill_32k_skewed - timed in the same process on the same resident weights, each over regions of at least
+100 ms (three rounds, median reported, every round kept), each with its own roofline, end-to-end figure and
+clock record.  --workload NAME times that one workload only.
 
 N > 1 (launched by torch.distributed.run, one rank per GPU) runs independent replicas: the layer
 does not shard in this build, so there is no data-path collective; the barrier and the max over
@@ -13,6 +19,7 @@ ranks are the only communication.  --impl reference times the CPU oracle (rank 0
 """
 import argparse
 import json
+import math
 import os
 import sys
 import threading
@@ -26,14 +33,19 @@ import numpy as np  # noqa: E402
 
 METRIC = "MoE FP4 layer tokens/s"
 DECODE = ("decode_c1", "decode_c64")
+PRODUCTION = ("decode_c1", "decode_c64", "prefill_8k", "prefill_32k_skewed")
+HEADLINE = "decode_c1"
+MIN_REGION_MS = 100.0   # a timed round of the per-workload figures lasts at least this long
+ROUNDS = 3
+GRAPH_STEPS = 8         # consecutive batches of the cycle per CUDA graph (decode workloads)
 
-# dram__bytes_read.sum + dram__bytes_write.sum per moe_expert_ffn call from one ncu capture of the
-# workload (see profiles/); None until captured.
+# dram__bytes_read.sum + dram__bytes_write.sum per launch (or per two-launch call) from one ncu capture of the
+# workload; which capture, at which commit, is stated in the file under profiles/ named beside each figure.
 NCU_TRAFFIC_BYTES = {
-    "decode_c1_one_launch": 110440700,  # ffn_native_kernel<true>, the whole layer: 107.14 MB read + 3.30 MB written (mean of two launches)
-    "decode_c1": 111216000,      # ffn_native_kernel<false>: 107.19 MB read + 4.03 MB written (profiles/ffn_native_decode.md)
-    "decode_c64": 3064384880,    # 3057.9 MB read + 6.5 MB written
-    "prefill_8k": 5611119000,    # ffn_umma_kernel<true> 2.882 + 0.263 GB, <false> 1.431 + 1.034 GB (profiles/ffn_umma_prefill_8k.md)
+    "decode_c1_one_launch": 110440700,  # ffn_native_kernel<true>, the whole layer (profiles/ffn_native_decode.md)
+    "decode_c1": 111216000,             # ffn_native_kernel<false> (profiles/ffn_native_decode.md)
+    "decode_c64": 3064384880,           # ffn_native_kernel<false> (profiles/ffn_native_decode.md)
+    "prefill_8k": 5611119000,           # ffn_umma_kernel<true> + <false> (profiles/ffn_umma_prefill_8k.md)
 }
 
 
@@ -66,6 +78,18 @@ def load_peaks():
         return dict(hbm=float(p["hbm_gbs"]), tensor_burst=float(p["bf16_tflops"]),
                     tensor_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
     return dict(hbm=6650.0, tensor_burst=1590.0, tensor_sustained=1400.0, source="fallback")
+
+
+def tensor_roofline(flops, ms, region_ms, peaks):
+    """Fraction of the dense bf16 peak: the burst figure for a region shorter than a second (the board has not
+    reached its power limit yet), the sustained one otherwise; both fractions are printed."""
+    achieved = flops / (ms * 1e-3) / 1e12
+    sustained = region_ms >= 1000.0
+    peak = peaks["tensor_sustained"] if sustained else peaks["tensor_burst"]
+    return {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+            "peak_used": "bf16_tflops_sustained" if sustained else "bf16_tflops",
+            "frac_of_burst": achieved / peaks["tensor_burst"], "frac_of_sustained": achieved / peaks["tensor_sustained"],
+            "algorithmic_flops": flops, "ms": ms, "peak_source": peaks["source"]}
 
 
 class ClockSampler(threading.Thread):
@@ -136,6 +160,12 @@ def max_over_ranks(value, world):
     return float(t.item())
 
 
+def steps_for_region(ms_per_step, min_ms=MIN_REGION_MS, multiple=1, at_least=1):
+    """Steps that make a timed round last at least min_ms, rounded up to a multiple (whole graphs)."""
+    n = max(at_least, int(math.ceil(min_ms / max(ms_per_step, 1e-6))))
+    return (n + multiple - 1) // multiple * multiple
+
+
 def oracle_sample(wl, inputs, n_tokens, seed0=1000, weights=None):
     """Time the CPU oracle, as it stands, on n_tokens tokens of the workload (per-token definition).
     `weights`: the full host arrays if the caller has them; else the touched experts are generated here."""
@@ -184,12 +214,392 @@ def run_reference(args, wl, inputs):
     }))
 
 
+class Bench:
+    """The resident model state (one copy of the expert weights) and the timing of one workload on it."""
+
+    def __init__(self, args, rank, world, local):
+        import torch
+        from paper_2609_15627_b200 import inputs, moe
+        self.torch, self.inputs, self.moe = torch, inputs, moe
+        self.args, self.rank, self.world, self.local = args, rank, world, local
+        self.stream = torch.cuda.current_stream()
+        self.peaks = load_peaks()
+        self._weights_key = None
+        self.weights_host = self.weights = self.packed = None
+        self.read_only_gbs = None
+
+    # ---- plumbing ---------------------------------------------------------------------------------------------
+    def dev(self, a):
+        torch = self.torch
+        if a.dtype == np.uint16:
+            return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+        return torch.from_numpy(a).cuda()
+
+    def barrier(self):
+        if self.world > 1:
+            self.torch.distributed.barrier()
+        self.torch.cuda.synchronize()
+
+    def events(self):
+        return self.torch.cuda.Event(enable_timing=True), self.torch.cuda.Event(enable_timing=True)
+
+    def hold(self):
+        """Keep the GPU busy for about 100 us, so that the event and the launches enqueued behind it are already
+        queued when it ends: the region then measures device time, not the host's launch latency."""
+        self.torch.cuda._sleep(200000)
+
+    def load_weights(self, wl):
+        """Weights are model state: generated once per (H, I, E), moved to the device, re-laid by moe_prepack (the
+        one-time load transform, untimed) unless --raw-weights, after which the row-layout tensors are dropped."""
+        key = (wl.H, wl.I, wl.E)
+        if self._weights_key == key:
+            return
+        torch, moe = self.torch, self.moe
+        self.weights = self.packed = None
+        torch.cuda.empty_cache()
+        self.weights_host = self.inputs.make_expert_weights(wl.H, wl.I, wl.E, seed=0)
+        self.weights = tuple(self.dev(a) for a in self.weights_host)
+        if not self.args.raw_weights:
+            self.packed = moe.moe_prepack(*self.weights, moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k))
+            torch.cuda.synchronize()
+            self.weights = None
+        self._weights_key = key
+        self.read_only_gbs = None
+
+    def read_only_stream(self, status):
+        """Read-only ceiling: the decode kernel's load mechanism alone over the resident gate/up weights (2.1 GB at
+        the production shape, larger than L2).  Context for the HBM-bound workloads, not the denominator."""
+        if self.read_only_gbs is not None:
+            return self.read_only_gbs
+        torch, moe = self.torch, self.moe
+        src = self.packed if self.packed is not None else self.weights[0]
+        if src.numel() < (1 << 28):
+            return None
+        sink = torch.empty(4096, dtype=torch.int32, device="cuda")
+        for _ in range(2):
+            moe.moe_debug_read_probe(src, sink, status, self.stream)
+        p0, p1 = self.events()
+        p0.record(self.stream)
+        for _ in range(5):
+            moe.moe_debug_read_probe(src, sink, status, self.stream)
+        p1.record(self.stream)
+        self.barrier()
+        self.read_only_gbs = 5 * src.numel() / (p0.elapsed_time(p1) * 1e-3) / 1e9
+        return self.read_only_gbs
+
+    # ---- one workload -------------------------------------------------------------------------------------------
+    def run(self, wl, exact_steps=None, warmup=3, e2e=True):
+        """Times `wl`.  exact_steps: also time one region of exactly that many steps (the headline's K).
+        Returns the per-workload record; with exact_steps its 'exact' entry holds that region."""
+        torch, moe, inputs, args = self.torch, self.moe, self.inputs, self.args
+        rank, world, stream = self.rank, self.world, self.stream
+        decode = wl.name in DECODE or wl.name == "tiny"
+        self.load_weights(wl)
+        packed, weights = self.packed, self.weights
+        sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
+        n_cycle = 32 if decode else 2
+        batches_host = [(inputs.make_logits(wl.T, wl.E, 7000 + rank * 100 + i, wl.skew),
+                         inputs.make_x(wl.T, wl.H, 7000 + rank * 100 + i)) for i in range(n_cycle)]
+        batches = [(self.dev(l), self.dev(x)) for l, x in batches_host]
+        buf = moe.LayerBuffers(sh)
+        fws = moe.alloc_forward_workspace(sh)
+
+        # experts touched per batch of the cycle (from the library's own routing), for the byte count
+        touched = []
+        for l, x in batches:
+            moe.moe_route(l, wl.k, buf.topk_ids, buf.topk_w, buf.expert_offsets, buf.ws)
+            touched.append(int(np.count_nonzero(np.diff(buf.expert_offsets.cpu().numpy()))))
+
+        def forward(l, x, st):
+            if packed is not None:
+                moe.moe_forward_packed(l, x, packed, sh, buf.out, None, None, buf.status, fws, st)
+            else:
+                moe.moe_forward(l, x, *weights, sh, buf.out, None, None, buf.status, fws, st)
+
+        def expert_ffn(b, st):
+            if packed is not None:
+                moe.moe_expert_ffn_packed(b.x_perm, b.expert_offsets, packed, sh, b.y_perm, b.status, b.ws, st)
+            else:
+                moe.moe_expert_ffn(b.x_perm, b.expert_offsets, *weights, sh, b.y_perm, b.status, b.ws, st)
+
+        # Does moe_forward run this shape as one launch?  (Asked of the library: one call, then the name of its kernel.)
+        forward(batches[0][0], batches[0][1], stream)
+        torch.cuda.synchronize()
+        one_launch = moe.moe_last_kernel_name().startswith("layer_one_launch") and not args.four_calls
+
+        def step4(i, ev=None, st=stream):
+            """The four C-ABI calls on batch i of the cycle (st=None: torch's current stream, used during capture)."""
+            l, x = batches[i % n_cycle]
+            moe.moe_route(l, wl.k, buf.topk_ids, buf.topk_w, buf.expert_offsets, buf.ws, st)
+            moe.moe_permute(x, buf.topk_ids, buf.expert_offsets, sh, buf.x_perm, buf.perm, buf.inv_perm, buf.ws, st)
+            if ev is not None:
+                ev[0].record(st)
+            expert_ffn(buf, st)
+            if ev is not None:
+                ev[1].record(st)
+            moe.moe_combine(buf.y_perm, buf.inv_perm, buf.topk_w, sh, buf.out, st)
+
+        def step1(i, ev=None, st=stream):
+            """The same path as one call (one kernel launch for this shape)."""
+            l, x = batches[i % n_cycle]
+            forward(l, x, st)
+
+        step = step1 if one_launch else step4
+        for i in range(max(warmup, 3)):
+            step(i)
+        self.barrier()
+
+        # Decode-sized steps are a handful of short kernels: like the paper's decode tiers they are replayed as CUDA
+        # graphs (the C-ABI calls captured as they are).  A serving graph holds many layers back to back; here a graph
+        # holds GRAPH_STEPS consecutive batches of the cycle (one layer call each), plus one single-step graph per
+        # batch for a step count that is not a multiple of GRAPH_STEPS.
+        use_graph = decode and not args.no_graph
+
+        def capture(fn, idx):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for i in idx:
+                    fn(i, st=None)
+            return g
+
+        def warm_side(fn):
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            with torch.cuda.stream(side):
+                for i in range(3):
+                    fn(i, st=None)
+            stream.wait_stream(side)
+            self.barrier()
+
+        graphs, multi_graphs, launches_per_step = [], [], None
+        if use_graph:
+            warm_side(step)
+            c0 = moe.moe_launch_count()
+            graphs = [capture(step, [i]) for i in range(n_cycle)]
+            launches_per_step = (moe.moe_launch_count() - c0) // n_cycle
+            multi_graphs = [capture(step, range(i0, i0 + GRAPH_STEPS)) for i0 in range(0, n_cycle, GRAPH_STEPS)]
+            for g in graphs[:3] + multi_graphs:
+                g.replay()
+            self.barrier()
+
+        def play(n, inner=None):
+            """Enqueue n consecutive steps of the cycle."""
+            if use_graph:
+                n_multi = n // GRAPH_STEPS
+                for i in range(n_multi):
+                    multi_graphs[i % len(multi_graphs)].replay()
+                for i in range(n_multi * GRAPH_STEPS, n):
+                    graphs[i % n_cycle].replay()
+            else:
+                for i in range(n):
+                    step(i, inner[i] if inner is not None and i < len(inner) and not one_launch else None)
+
+        def region(n, inner=None):
+            """One timed region of exactly n steps: barrier + synchronize on both sides, CUDA events on the launching
+            stream, max over ranks.  Returns (ms of the region, clock record, launches of the library's kernels)."""
+            e0, e1 = self.events()
+            sampler = ClockSampler(physical_gpu_index(self.local))
+            c0 = moe.moe_launch_count()
+            self.barrier()
+            sampler.start()
+            self.hold()
+            e0.record(stream)
+            play(n, inner)
+            e1.record(stream)
+            self.barrier()
+            clocks = sampler.stop()
+            launches = launches_per_step * n if use_graph else moe.moe_launch_count() - c0
+            assert int(buf.status.item()) == 0, "device-side wait timed out"
+            return max_over_ranks(e0.elapsed_time(e1), world), clocks, launches
+
+        # ---- the headline's region: exactly K steps -------------------------------------------------------------
+        rec = {}
+        if exact_steps is not None:
+            ms, clocks, launches = region(exact_steps)
+            rec["exact"] = {"steps": exact_steps, "ms_total": ms, "ms_per_step": ms / exact_steps, "clocks": clocks,
+                            "gpu_launches": launches,
+                            "experts_touched": float(np.mean([touched[i % n_cycle] for i in range(exact_steps)]))}
+
+        # ---- rounds of at least MIN_REGION_MS ---------------------------------------------------------------------
+        pilot_n = GRAPH_STEPS if use_graph else 2
+        pilot_ms = region(pilot_n)[0] / pilot_n
+        n_steps = steps_for_region(pilot_ms, multiple=GRAPH_STEPS if use_graph else 1, at_least=3)
+        n_inner = 0 if (use_graph or one_launch) else n_steps
+        inner = [self.events() for _ in range(n_inner)]
+        rounds, clock_rounds, reasons, launches = [], [], set(), 0
+        ffn_round_ms = []
+        for _ in range(ROUNDS):
+            ms, clocks, launches = region(n_steps, inner if n_inner else None)
+            rounds.append(ms / n_steps)
+            clock_rounds.append(clocks["sm_mhz"])
+            reasons.update(clocks["reasons"])
+            if n_inner:
+                ffn_round_ms.append(float(np.mean([a.elapsed_time(b) for a, b in inner])))
+        ms_step = float(np.median(rounds))
+        region_ms = ms_step * n_steps
+        mean_touched = float(np.mean([touched[i % n_cycle] for i in range(n_steps)]))
+        rec.update({"ms_per_step": ms_step, "value": wl.T * world / (ms_step * 1e-3), "unit": "tokens/s",
+                    "steps": n_steps, "rounds_ms_per_step": rounds, "region_ms": region_ms,
+                    "gpu_launches": launches,
+                    "clocks": {"sm_mhz": int(np.median([c for c in clock_rounds if c is not None])) if any(
+                        c is not None for c in clock_rounds) else None, "sm_max_mhz": clocks["sm_max_mhz"],
+                        "reasons": sorted(reasons), "sm_mhz_rounds": clock_rounds},
+                    "call": ("moe_forward%s (one kernel launch per step)" if one_launch else
+                             "moe_route, moe_permute, moe_expert_ffn%s, moe_combine") % ("_packed" if packed is not None else ""),
+                    "launch": ("cuda graph replay, %d consecutive batches of the cycle per graph" % GRAPH_STEPS) if use_graph else "eager",
+                    "experts_touched": mean_touched})
+
+        # ---- the expert-FFN call inside eager steps (decode: a second region right after the graph-replayed one) ---
+        ffn_eager_ms, eager_ms_step = (float(np.median(ffn_round_ms)) if ffn_round_ms else None), None
+        if use_graph or one_launch:
+            n_e = min(n_steps, 256)
+            inner_e = [self.events() for _ in range(n_e)]
+            for i in range(3):
+                step4(i)
+            self.barrier()
+            ee0, ee1 = self.events()
+            ee0.record(stream)
+            for i in range(n_e):
+                step4(i, inner_e[i])
+            ee1.record(stream)
+            self.barrier()
+            eager_ms_step = ee0.elapsed_time(ee1) / n_e
+            ffn_eager_ms = float(np.mean([a.elapsed_time(b) for a, b in inner_e]))
+
+        # ---- one-launch workloads: the four calls, graph-replayed the same way, for comparison -----------------------
+        four_calls_ms_step = None
+        if one_launch and use_graph:
+            warm_side(step4)
+            mg4 = [capture(step4, range(i0, i0 + GRAPH_STEPS)) for i0 in range(0, n_cycle, GRAPH_STEPS)]
+            for g in mg4:
+                g.replay()
+            self.barrier()
+            n4 = max(len(mg4), min(n_steps // GRAPH_STEPS, 128))
+            g0, g1 = self.events()
+            self.hold()
+            g0.record(stream)
+            for i in range(n4):
+                mg4[i % len(mg4)].replay()
+            g1.record(stream)
+            self.barrier()
+            four_calls_ms_step = g0.elapsed_time(g1) / (n4 * GRAPH_STEPS)
+            del mg4
+
+        # ---- the expert-FFN call alone, graph-replayed like the step (calls shorter than 100 us) -------------------------
+        # Eager launches of kernels this short leave the GPU idle between the event and the launch, which the bracketing
+        # events count.  So such a call is also captured alone, one graph per batch of the cycle on that batch's own routed
+        # and permuted inputs, and the replays are timed back to back: consecutive calls touch different experts, as in
+        # the step.  Longer calls keep the time between their events inside the eager steps.
+        ffn_graph_ms, n_ffn = None, 0
+        if use_graph and ffn_eager_ms is not None and ffn_eager_ms < 0.1:
+            fbufs = []
+            for i in range(n_cycle):
+                b = moe.LayerBuffers(sh)
+                l, x = batches[i]
+                moe.moe_route(l, wl.k, b.topk_ids, b.topk_w, b.expert_offsets, b.ws, stream)
+                moe.moe_permute(x, b.topk_ids, b.expert_offsets, sh, b.x_perm, b.perm, b.inv_perm, b.ws, stream)
+                fbufs.append(b)
+            self.barrier()
+
+            def ffn_only(i, st=stream):
+                expert_ffn(fbufs[i % n_cycle], st)
+
+            warm_side(ffn_only)
+            fgraphs = [capture(ffn_only, [i]) for i in range(n_cycle)]
+            for i in range(3):
+                fgraphs[i].replay()
+            self.barrier()
+            n_ffn = max(n_cycle, min(n_steps, 1024))
+            f0, f1 = self.events()
+            self.hold()
+            f0.record(stream)
+            for i in range(n_ffn):
+                fgraphs[i % n_cycle].replay()
+            f1.record(stream)
+            self.barrier()
+            ffn_graph_ms = f0.elapsed_time(f1) / n_ffn
+            assert all(int(b.status.item()) == 0 for b in fbufs), "device-side wait timed out"
+            del fgraphs, fbufs
+
+        # ---- roofline of the dominant call (the expert FFN), and of the whole step ---------------------------------
+        peaks = self.peaks
+        ffn_ms = ffn_graph_ms if ffn_graph_ms is not None else ffn_eager_ms
+        timed_in = ("graph replays of the call alone, one graph per batch of the cycle, right after the timed rounds"
+                    if ffn_graph_ms is not None else
+                    ("eager steps right after the graph-replayed rounds" if use_graph or one_launch else
+                     "CUDA events around the call inside every step of the timed rounds"))
+        if decode:
+            alg = ffn_algorithmic_bytes(wl, mean_touched)
+            achieved = alg / (ffn_ms * 1e-3) / 1e9
+            roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"],
+                    "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "algorithmic_bytes": alg, "ms": ffn_ms,
+                    "peak_source": peaks["source"]}
+            alg_step = layer_algorithmic_bytes(wl, mean_touched)
+            step_roof = {"bound": "hbm", "achieved": alg_step / (ms_step * 1e-3) / 1e9, "peak": peaks["hbm"], "unit": "GB/s",
+                         "frac": alg_step / (ms_step * 1e-3) / 1e9 / peaks["hbm"], "algorithmic_bytes": alg_step, "ms": ms_step,
+                         "peak_source": peaks["source"],
+                         "traffic": NCU_TRAFFIC_BYTES.get(wl.name + "_one_launch") if one_launch else None}
+        else:
+            roof = tensor_roofline(ffn_flops(wl), ffn_ms, region_ms, peaks)
+            roof["traffic"] = NCU_TRAFFIC_BYTES.get(wl.name)
+            step_roof = tensor_roofline(ffn_flops(wl), ms_step, region_ms, peaks)
+        roof.update({"kernel": "moe_expert_ffn", "experts_touched": mean_touched, "timed_in": timed_in,
+                     "ms_between_events_in_eager_steps": ffn_eager_ms})
+        step_roof.update({"kernel": "the whole step (%s)" % rec["call"], "timed_in": "the timed rounds"})
+        if one_launch:
+            # the dominant kernel is the step itself: one launch per step, timed by the events of the timed rounds
+            step_roof["four_calls"] = {"ms_per_step": four_calls_ms_step, "eager_ms_per_step": eager_ms_step, "expert_ffn": roof}
+            rec["roofline"] = step_roof
+        else:
+            rec["roofline"] = roof
+            rec["roofline_step"] = step_roof
+            rec["eager_ms_per_step"] = eager_ms_step
+        if decode:
+            gbs = self.read_only_stream(buf.status)
+            if gbs is not None:
+                rec["roofline"]["read_only_stream_gbs"] = gbs
+                rec["roofline"]["frac_of_read_only_stream"] = rec["roofline"]["achieved"] / gbs
+
+        # ---- end to end through the host-buffer entry point ---------------------------------------------------------
+        if e2e and not args.no_e2e:
+            ws_h = moe.alloc_workspace(sh, host_path=True)
+            lh = [torch.from_numpy(l).pin_memory() for l, _ in batches_host]
+            xh = [torch.from_numpy(x.view(np.int16)).pin_memory() for _, x in batches_host]
+            oh = torch.empty((wl.T, wl.H), dtype=torch.int16).pin_memory()
+            n_e2e = max(3, min(exact_steps if exact_steps is not None else n_steps, 200 if decode else 5))
+
+            def forward_host(i):
+                if packed is not None:
+                    moe.moe_forward_host_packed(lh[i % n_cycle], xh[i % n_cycle], packed, sh, oh, buf.status, ws_h, stream)
+                else:
+                    moe.moe_forward_host(lh[i % n_cycle], xh[i % n_cycle], *weights, sh, oh, buf.status, ws_h, stream)
+
+            for i in range(3):
+                forward_host(i)
+            self.barrier()
+            t0 = time.perf_counter()
+            for i in range(n_e2e):
+                forward_host(i)
+            dt = max_over_ranks(time.perf_counter() - t0, world)
+            rec["e2e"] = {"value": wl.T * world * n_e2e / dt, "unit": "tokens/s",
+                          "h2d_bytes_per_step": wl.T * wl.E * 4 + wl.T * wl.H * 2, "d2h_bytes_per_step": wl.T * wl.H * 2,
+                          "steps": n_e2e, "call": "%s (pinned host logits/x in, bf16 out back, weights resident)"
+                                  % ("moe_forward_host_packed" if packed is not None else "moe_forward_host")}
+            del ws_h, lh, xh, oh
+        rec["kernels"] = moe.moe_last_kernel_name()
+        rec["one_launch"] = one_launch
+        rec["n_cycle"] = n_cycle
+        del graphs, multi_graphs, batches, buf, fws
+        torch.cuda.empty_cache()
+        return rec
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--workload", default="decode_c1")
+    ap.add_argument("--workload", default=None, help="time this workload only (default: all four production workloads, headline decode_c1)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -199,17 +609,17 @@ def main():
     args = ap.parse_args()
 
     from paper_2609_15627_b200 import inputs
-    wl = inputs.WORKLOADS[args.workload]
-    decode = wl.name in DECODE or wl.name == "tiny"
+    head = inputs.WORKLOADS[args.workload or HEADLINE]
     if args.impl == "reference":
         args.steps = args.steps if args.steps is not None else 5
         args.warmup = args.warmup if args.warmup is not None else 1
-        run_reference(args, wl, inputs)
+        run_reference(args, head, inputs)
         return
+    head_decode = head.name in DECODE or head.name == "tiny"
     if args.steps is None:
-        args.steps = 2000 if decode else 10
+        args.steps = 2000 if head_decode else 10
     if args.warmup is None:
-        args.warmup = 20 if decode else 3
+        args.warmup = 20 if head_decode else 3
     args.warmup = max(args.warmup, 3)
 
     import torch
@@ -229,334 +639,59 @@ def main():
         torch.distributed.barrier()
     moe.lib()
 
-    # ---- resident inputs: weights once, a cycle of seeded (logits, x) batches -------------------------
-    def dev(a):
-        if a.dtype == np.uint16:
-            return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
-        return torch.from_numpy(a).cuda()
+    bench = Bench(args, rank, world, local)
+    # every rank times the same list, in the same order (the barriers pair up)
+    # (replicas, N > 1: the headline workload only - the scaling figure is the headline's)
+    names = [args.workload] if args.workload else [HEADLINE] + ([n for n in PRODUCTION if n != HEADLINE] if world == 1 else [])
+    records = {}
+    for name in names:
+        wl = inputs.WORKLOADS[name]
+        records[name] = bench.run(wl, exact_steps=args.steps if name == head.name else None, warmup=args.warmup)
+    hr = records[head.name]
+    ex = hr.pop("exact")
 
-    weights_host = inputs.make_expert_weights(wl.H, wl.I, wl.E, seed=0)
-    weights = tuple(dev(a) for a in weights_host)
-    # One-time load transform (untimed, as in the paper's load path): the same bytes in tiles that are contiguous in
-    # memory.  The row-layout tensors are dropped afterwards: one copy of the weights is resident.
-    packed = None
-    if not args.raw_weights:
-        packed = moe.moe_prepack(*weights, moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k))
-        torch.cuda.synchronize()
-        weights = None
-    n_cycle = 32 if decode else 2
-    batches_host = [(inputs.make_logits(wl.T, wl.E, 7000 + rank * 100 + i, wl.skew), inputs.make_x(wl.T, wl.H, 7000 + rank * 100 + i))
-                    for i in range(n_cycle)]
-    batches = [(dev(l), dev(x)) for l, x in batches_host]
-    sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
-    buf = moe.LayerBuffers(sh)
-    stream = torch.cuda.current_stream()
-
-    # experts touched per batch of the cycle (from the library's own routing), for the byte count
-    touched = []
-    for l, x in batches:
-        moe.moe_route(l, wl.k, buf.topk_ids, buf.topk_w, buf.expert_offsets, buf.ws)
-        off = buf.expert_offsets.cpu().numpy()
-        touched.append(int(np.count_nonzero(np.diff(off))))
-
-    # Does moe_forward run this shape as one launch?  (Asked of the library: one call, then the name of its kernel.)
-    fws = moe.alloc_forward_workspace(sh)
-    def forward(l, x, st):
-        if packed is not None:
-            moe.moe_forward_packed(l, x, packed, sh, buf.out, None, None, buf.status, fws, st)
-        else:
-            moe.moe_forward(l, x, *weights, sh, buf.out, None, None, buf.status, fws, st)
-
-    def expert_ffn(b, st):
-        if packed is not None:
-            moe.moe_expert_ffn_packed(b.x_perm, b.expert_offsets, packed, sh, b.y_perm, b.status, b.ws, st)
-        else:
-            moe.moe_expert_ffn(b.x_perm, b.expert_offsets, *weights, sh, b.y_perm, b.status, b.ws, st)
-
-    forward(batches[0][0], batches[0][1], stream)
-    torch.cuda.synchronize()
-    one_launch = moe.moe_last_kernel_name().startswith("layer_one_launch") and not args.four_calls
-
-    def step4(i, ev=None, st=stream):
-        """The four C-ABI calls on batch i of the cycle (st=None: torch's current stream, used during capture)."""
-        l, x = batches[i % n_cycle]
-        moe.moe_route(l, wl.k, buf.topk_ids, buf.topk_w, buf.expert_offsets, buf.ws, st)
-        moe.moe_permute(x, buf.topk_ids, buf.expert_offsets, sh, buf.x_perm, buf.perm, buf.inv_perm, buf.ws, st)
-        if ev is not None:
-            ev[0].record(st)
-        expert_ffn(buf, st)
-        if ev is not None:
-            ev[1].record(st)
-        moe.moe_combine(buf.y_perm, buf.inv_perm, buf.topk_w, sh, buf.out, st)
-
-    def step1(i, ev=None, st=stream):
-        """The same path as one call (one kernel launch for this shape)."""
-        l, x = batches[i % n_cycle]
-        forward(l, x, st)
-
-    step = step1 if one_launch else step4
-
-    def barrier():
-        if world > 1:
-            torch.distributed.barrier()
-        torch.cuda.synchronize()
-
-    for i in range(args.warmup):
-        step(i)
-    barrier()
-
-    # Decode-sized steps are a handful of short kernels: like the paper's decode tiers they are replayed as CUDA
-    # graphs (the four C-ABI calls captured as they are).  A serving graph holds many layers back to back; here a
-    # graph holds kGraphSteps consecutive batches of the cycle (one layer call each), plus one single-step graph per
-    # batch for a step count that is not a multiple of kGraphSteps.
-    use_graph = decode and not args.no_graph
-    kGraphSteps = 8
-    graphs, multi_graphs, launches_per_step = [], [], None
-    if use_graph:
-        side = torch.cuda.Stream()
-        side.wait_stream(stream)
-        with torch.cuda.stream(side):
-            for i in range(3):
-                step(i, st=None)
-        stream.wait_stream(side)
-        barrier()
-        for i in range(n_cycle):
-            g = torch.cuda.CUDAGraph()
-            c0 = moe.moe_launch_count()
-            with torch.cuda.graph(g):
-                step(i, st=None)
-            launches_per_step = moe.moe_launch_count() - c0
-            graphs.append(g)
-        for i0 in range(0, n_cycle, kGraphSteps):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g):
-                for i in range(i0, i0 + kGraphSteps):
-                    step(i, st=None)
-            multi_graphs.append(g)
-        for i in range(max(args.warmup, 3)):
-            graphs[i % n_cycle].replay()
-        for g in multi_graphs:
-            g.replay()
-        barrier()
-
-    # ---- timed region: exactly K steps ---------------------------------------------------------------------
-    n_inner = min(args.steps, 256)  # steps whose expert-FFN call is bracketed by its own events
-    inner = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_inner)]
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(physical_gpu_index(local))
-    launches0 = moe.moe_launch_count()
-    barrier()
-    sampler.start()
-    e0.record(stream)
-    if use_graph:
-        n_multi = args.steps // kGraphSteps
-        for i in range(n_multi):
-            multi_graphs[i % len(multi_graphs)].replay()
-        for i in range(n_multi * kGraphSteps, args.steps):
-            graphs[i % n_cycle].replay()
-    else:
-        for i in range(args.steps):
-            step(i, inner[i] if i < n_inner and not one_launch else None)
-    e1.record(stream)
-    barrier()
-    clocks = sampler.stop()
-    launches = launches_per_step * args.steps if use_graph else moe.moe_launch_count() - launches0
-    assert int(buf.status.item()) == 0, "device-side wait timed out"
-    ms_total = max_over_ranks(e0.elapsed_time(e1), world)
-    ms_step = ms_total / args.steps
-    value = wl.T * world / (ms_step * 1e-3)
-    eager_ms_step = None
-    if use_graph or one_launch:
-        # the expert-FFN call cannot be bracketed by events inside a graph (nor inside the one-launch layer): time it
-        # in a second region of eager steps of the four calls on the same batches, right after the timed one
-        for i in range(3):
-            step4(i)
-        barrier()
-        ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ee0.record(stream)
-        for i in range(n_inner):
-            step4(i, inner[i])
-        ee1.record(stream)
-        barrier()
-        eager_ms_step = ee0.elapsed_time(ee1) / n_inner
-
-    # ---- one-launch workloads: the four calls, graph-replayed the same way, for comparison -----------------------
-    four_calls_ms_step = None
-    if one_launch and use_graph:
-        side = torch.cuda.Stream()
-        side.wait_stream(stream)
-        with torch.cuda.stream(side):
-            for i in range(3):
-                step4(i, st=None)
-        stream.wait_stream(side)
-        barrier()
-        mg4 = []
-        for i0 in range(0, n_cycle, kGraphSteps):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g):
-                for i in range(i0, i0 + kGraphSteps):
-                    step4(i, st=None)
-            mg4.append(g)
-        for g in mg4:
-            g.replay()
-        barrier()
-        n4 = max(len(mg4), min(args.steps // kGraphSteps, 64))
-        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        g0.record(stream)
-        for i in range(n4):
-            mg4[i % len(mg4)].replay()
-        g1.record(stream)
-        barrier()
-        four_calls_ms_step = g0.elapsed_time(g1) / (n4 * kGraphSteps)
-
-    # ---- the expert-FFN call alone, graph-replayed like the step (calls shorter than 100 us) -------------------------
-    # Eager launches of kernels this short leave the GPU idle between the event and the launch, which the bracketing
-    # events count.  So such a call is also captured alone, one graph per batch of the cycle on that batch's own routed
-    # and permuted inputs, and the replays are timed back to back: consecutive calls touch different experts, as in
-    # the step.  Longer calls keep the time between their events inside the eager steps.
-    ffn_graph_ms, n_ffn = None, 0
-    if use_graph and float(np.mean([a.elapsed_time(b) for a, b in inner])) < 0.1:
-        fbufs = []
-        for i in range(n_cycle):
-            b = moe.LayerBuffers(sh)
-            l, x = batches[i]
-            moe.moe_route(l, wl.k, b.topk_ids, b.topk_w, b.expert_offsets, b.ws, stream)
-            moe.moe_permute(x, b.topk_ids, b.expert_offsets, sh, b.x_perm, b.perm, b.inv_perm, b.ws, stream)
-            fbufs.append(b)
-        barrier()
-
-        def ffn_only(b, st=stream):
-            expert_ffn(b, st)
-
-        side = torch.cuda.Stream()
-        side.wait_stream(stream)
-        with torch.cuda.stream(side):
-            ffn_only(fbufs[0], None)
-        stream.wait_stream(side)
-        barrier()
-        fgraphs = []
-        for b in fbufs:
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g):
-                ffn_only(b, None)
-            fgraphs.append(g)
-        for i in range(max(args.warmup, 3)):
-            fgraphs[i % n_cycle].replay()
-        barrier()
-        n_ffn = max(n_cycle, min(args.steps, 512))
-        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        f0.record(stream)
-        for i in range(n_ffn):
-            fgraphs[i % n_cycle].replay()
-        f1.record(stream)
-        barrier()
-        ffn_graph_ms = f0.elapsed_time(f1) / n_ffn
-        assert all(int(b.status.item()) == 0 for b in fbufs), "device-side wait timed out"
-
-    # ---- roofline of the dominant call (the expert FFN) --------------------------------------------------------
-    ffn_eager_ms = float(np.mean([a.elapsed_time(b) for a, b in inner]))
-    ffn_ms = ffn_graph_ms if ffn_graph_ms is not None else ffn_eager_ms
-    n_avg = n_ffn if ffn_graph_ms is not None else n_inner
-    mean_touched = float(np.mean([touched[i % n_cycle] for i in range(n_avg)]))
-    peaks = load_peaks()
-    if decode:
-        alg = ffn_algorithmic_bytes(wl, mean_touched)
-        achieved = alg / (ffn_ms * 1e-3) / 1e9
-        roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"],
-                "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "algorithmic_bytes": alg}
-    else:
-        fl = ffn_flops(wl)
-        achieved = fl / (ffn_ms * 1e-3) / 1e12
-        roof = {"bound": "tensor", "achieved": achieved, "peak": peaks["tensor_sustained"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["tensor_sustained"], "traffic": NCU_TRAFFIC_BYTES.get(wl.name),
-                "algorithmic_flops": fl}
-    roof.update({"kernel": "moe_expert_ffn",
-                 "ms": ffn_ms, "peak_source": peaks["source"], "experts_touched": mean_touched,
-                 "timed_in": ("graph replays of the call alone, one graph per batch of the cycle, right after the timed region"
-                              if ffn_graph_ms is not None else
-                              ("eager steps right after the graph-replayed region" if use_graph or one_launch else "the timed region")),
-                 "ms_between_events_in_eager_steps": ffn_eager_ms})
-    if one_launch:
-        # the dominant kernel is the step itself: one launch per step, timed by the events of the timed region
-        touched_steps = float(np.mean([touched[i % n_cycle] for i in range(args.steps)]))
-        alg = layer_algorithmic_bytes(wl, touched_steps)
+    # ---- the headline: exactly K steps of the headline workload ------------------------------------------------
+    ms_step = ex["ms_per_step"]
+    value = head.T * world / (ms_step * 1e-3)
+    peaks = bench.peaks
+    roof = dict(hr["roofline"])
+    if hr["one_launch"]:
+        alg = layer_algorithmic_bytes(head, ex["experts_touched"])
         achieved = alg / (ms_step * 1e-3) / 1e9
-        roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"],
-                "traffic": NCU_TRAFFIC_BYTES.get(wl.name + "_one_launch"), "algorithmic_bytes": alg,
-                "kernel": "moe_forward (route, term split, expert FFN and combine in one launch)", "ms": ms_step,
-                "peak_source": peaks["source"], "experts_touched": touched_steps, "timed_in": "the timed region",
-                "four_calls": {"ms_per_step": four_calls_ms_step, "eager_ms_per_step": eager_ms_step, "expert_ffn": roof}}
-
-    # ---- read-only ceiling: the decode kernel's load mechanism alone over the resident gate/up weights ------------
-    # (2.1 GB at the production shape, larger than L2; context for the HBM-bound workloads, not the denominator)
-    probe_src = packed if packed is not None else weights[0]
-    if decode and probe_src.numel() >= (1 << 28):
-        sink = torch.empty(4096, dtype=torch.int32, device="cuda")
-        for _ in range(2):
-            moe.moe_debug_read_probe(probe_src, sink, buf.status, stream)
-        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        p0.record(stream)
-        for _ in range(5):
-            moe.moe_debug_read_probe(probe_src, sink, buf.status, stream)
-        p1.record(stream)
-        barrier()
-        read_gbs = 5 * probe_src.numel() / (p0.elapsed_time(p1) * 1e-3) / 1e9
-        roof["read_only_stream_gbs"] = read_gbs
-        roof["frac_of_read_only_stream"] = roof["achieved"] / read_gbs
-
-    # ---- end to end through the host-buffer entry point ---------------------------------------------------------
-    e2e = None
-    if not args.no_e2e:
-        ws_h = moe.alloc_workspace(sh, host_path=True)
-        lh = [torch.from_numpy(l).pin_memory() for l, _ in batches_host]
-        xh = [torch.from_numpy(x.view(np.int16)).pin_memory() for _, x in batches_host]
-        oh = torch.empty((wl.T, wl.H), dtype=torch.int16).pin_memory()
-        n_e2e = max(3, min(args.steps, 200 if decode else 5))
-        def forward_host(i):
-            if packed is not None:
-                moe.moe_forward_host_packed(lh[i % n_cycle], xh[i % n_cycle], packed, sh, oh, buf.status, ws_h, stream)
-            else:
-                moe.moe_forward_host(lh[i % n_cycle], xh[i % n_cycle], *weights, sh, oh, buf.status, ws_h, stream)
-
-        for i in range(3):
-            forward_host(i)
-        barrier()
-        t0 = time.perf_counter()
-        for i in range(n_e2e):
-            forward_host(i)
-        dt = max_over_ranks(time.perf_counter() - t0, world)
-        e2e = {"value": wl.T * world * n_e2e / dt, "unit": "tokens/s",
-               "h2d_bytes_per_step": wl.T * wl.E * 4 + wl.T * wl.H * 2, "d2h_bytes_per_step": wl.T * wl.H * 2,
-               "steps": n_e2e, "call": "%s (pinned host logits/x in, bf16 out back, weights resident)"
-                       % ("moe_forward_host_packed" if packed is not None else "moe_forward_host")}
+        roof.update({"achieved": achieved, "frac": achieved / peaks["hbm"], "algorithmic_bytes": alg, "ms": ms_step,
+                     "experts_touched": ex["experts_touched"], "timed_in": "the timed region"})
+        if "read_only_stream_gbs" in roof:
+            roof["frac_of_read_only_stream"] = achieved / roof["read_only_stream_gbs"]
 
     # ---- the oracle on the host cores (rank 0, N = 1 only) ----------------------------------------------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         # about 10-20 s of host work at the production shape (the oracle does roughly 50 tokens/s on 16 cores)
-        n_tok = {"tiny": 4096}.get(wl.name, 640)
-        v, dt, n, cores = oracle_sample(wl, inputs, n_tok, weights=weights_host)
+        n_tok = {"tiny": 4096}.get(head.name, 640)
+        v, dt, n, cores = oracle_sample(head, inputs, n_tok, weights=bench.weights_host)
         cpu = {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle",
-               "sample": "%d tokens with the %s shape and routing distribution, per-token definition, %.1f s" % (n, wl.name, dt)}
+               "sample": "%d tokens with the %s shape and routing distribution, per-token definition, %.1f s" % (n, head.name, dt)}
 
     if rank == 0:
-        print(json.dumps({
+        line = {
             "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": wl.name, "T": wl.T, "H": wl.H, "I": wl.I, "E": wl.E, "k": wl.k,
-                       "parallelism": "replicas only" if world > 1 else "1 GPU",
-                       "call": ("moe_forward%s (one kernel launch per step)" if one_launch else
-                                "moe_route, moe_permute, moe_expert_ffn%s, moe_combine") % ("_packed" if packed is not None else ""),
-                       "weights": ("moe_prepack's tile-contiguous layout (one-time transform, same bytes)" if packed is not None
-                                   else "checkpoint row layout"),
-                       "launch": "cuda graph replay, %d consecutive batches of the cycle per graph" % kGraphSteps if use_graph else "eager",
-                       "eager_ms_per_step": None if one_launch else eager_ms_step,
+            "config": {"workload": head.name, "T": head.T, "H": head.H, "I": head.I, "E": head.E, "k": head.k,
+                       "parallelism": "replicas only" if world > 1 else "1 GPU", "call": hr["call"],
+                       "weights": ("moe_prepack's tile-contiguous layout (one-time transform, same bytes)"
+                                   if bench.packed is not None else "checkpoint row layout"),
+                       "launch": hr["launch"],
                        "l2": "inputs cycle over %d seeded batches; %.2f GB of expert weights resident (larger than L2)"
-                             % (n_cycle, wl.E * expert_weight_bytes(wl.H, wl.I) / 1e9)},
-            "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
-            "kernels": moe.moe_last_kernel_name(),
-        }))
+                             % (hr["n_cycle"], head.E * expert_weight_bytes(head.H, head.I) / 1e9)},
+            "roofline": roof, "cpu_baseline": cpu, "e2e": hr.get("e2e"), "gpu_launches": ex["gpu_launches"],
+            "clocks": ex["clocks"], "kernels": hr["kernels"],
+            "workloads": {n: {k: v for k, v in r.items() if k not in ("one_launch", "n_cycle")} for n, r in records.items()},
+            "protocol": ("headline: one region of exactly --steps steps; workloads: %d rounds of at least %d ms each, median "
+                         "reported, every round kept; every region is bracketed by a barrier and a synchronize, timed by CUDA "
+                         "events on the launching stream behind a 100 us hold kernel, max over ranks") % (ROUNDS, MIN_REGION_MS),
+        }
+        print(json.dumps(line))
     if world > 1:
         torch.distributed.destroy_process_group()
 

@@ -21,7 +21,13 @@
  *     legacy default stream) and returns; there is no host synchronisation and no device-to-host copy.
  *   - Return value: a moe_status_t.  Argument errors are found on the host before anything is
  *     launched.  A device-side bounded wait that runs out writes MOE_ERR_TIMEOUT to *status_word
- *     (sticky, device memory, may be NULL) and the kernel still terminates normally.
+ *     (sticky, device memory, may be NULL) and the kernel still terminates normally.  Once one wait of a
+ *     call has run out (about two seconds), every later wait of that call gives up after a millisecond, so a
+ *     lost signal costs seconds, not seconds per wait.  With status_word == NULL the kernels keep that rule
+ *     through a word inside the library (one per device, looked up on the first such call on a device - make
+ *     that call outside stream capture - and cleared by each call that uses it); nothing is reported then, and
+ *     NULL-status calls that overlap on the GPU share the word.
+ *   - Diagnostic and measurement exports (moe_debug_*) are declared in moe_b200_debug.h.
  *   - Determinism: identical inputs give bit-identical outputs on every launch.  No invariance is
  *     claimed across different T or batch compositions.
  *   - bf16 arrays are passed as `const void*` / `void*` (16-bit elements, IEEE bfloat16 bit patterns).
@@ -71,24 +77,6 @@ const char* moe_last_kernel_name(void);
 
 /* Host.  Number of kernels launched (memset nodes not counted) by this thread's moe_* calls so far. */
 uint64_t moe_launch_count(void);
-
-/*
- * Measurement aid (no counterpart in the paper): one persistent CTA per SM pulls `bytes` of device memory at `src`
- * (128-byte aligned, at least 32 KB) through a shared-memory ring of 32 KB bulk copies and does nothing with them -
- * the decode-sized expert kernel's weight stream without the tensor-core work.  Timed by the caller with CUDA events
- * over a buffer larger than L2 it gives the read-only bandwidth such a stream can reach on this GPU, which bench.py
- * reports beside the roofline.  `sink` receives one word per CTA (4 * number of SMs bytes at least).  Enqueue only;
- * bounded waits as everywhere.
- */
-int moe_debug_read_probe(const void* src, size_t bytes, void* sink, size_t sink_bytes, int32_t* status_word,
-                         void* cuda_stream);
-
-/* Host, pure, diagnostic.  Work split of the decode-sized expert-FFN kernel: which items (touched expert x tile of
- * 256 weight rows, in expert order) CTA `cta` of `n_ctas` takes when `n_touched` experts have rows.  out4 = first
- * and one-past-last gate/up item, first and one-past-last down item.  A down item waits, on the device, for all
- * gate/up items of its expert; the split keeps those in CTAs with a lower or equal index.  INVALID_ARG on
- * nonsense (cta outside [0, n_ctas), n_touched outside [0, 1024], H or 2I not a multiple of 256). */
-int moe_debug_native_cta_share(int32_t n_ctas, int32_t cta, int32_t n_touched, int32_t H, int32_t I, int32_t* out4);
 
 /*
  * Router Top-k (paper: "Router Top-k"; fixed Top-K membership and order is a stated requirement).
@@ -171,9 +159,12 @@ int moe_validate_scales(const uint8_t* scales, size_t n_bytes, int32_t* bad_coun
  *     along K; the scale bytes likewise in tiles of 128 rows x 16 bytes.  A kernel's pipeline step then reads whole
  *     contiguous runs instead of 128 pieces one row pitch apart.  For every other shape the packed buffer is a plain
  *     copy of the four tensors.
- *   - moe_prepack: device to device, asynchronous on the stream, out of place (packed_out must not overlap the
- *     inputs), 256-byte aligned, packed_bytes >= moe_prepack_bytes() else MOE_ERR_WORKSPACE.  Not part of the timed
- *     path: weights are packed once per model load.  The caller may free the four tensors afterwards.
+ *   - moe_prepack: device to device, out of place (packed_out must not overlap the inputs), 256-byte aligned,
+ *     packed_bytes >= moe_prepack_bytes() else MOE_ERR_WORKSPACE.  Not part of the timed path: weights are packed once
+ *     per model load.  It is also the load check of the scale bytes (the paper's scale-value trap): both scale
+ *     tensors are scanned for bytes outside [0,128], the count is read back, and MOE_ERR_INVALID_ARG is returned -
+ *     with nothing packed - if there is one.  Because of that read-back this call, unlike the others, WAITS for the
+ *     stream and cannot be captured into a CUDA graph.  The caller may free the four tensors afterwards.
  *   - moe_expert_ffn_packed: moe_expert_ffn with `packed` in place of the four weight arguments; same arithmetic, same
  *     result bit for bit.  Kernel choice as moe_expert_ffn, except that shapes with the tiled layout that would fall to
  *     the row-streaming fallback kernel (neither decode-sized nor prefill-sized) run the grouped-GEMM kernel.
@@ -213,14 +204,6 @@ int moe_forward(const float* logits /* [T,E] */, const void* x_bf16 /* [T,H] */,
                 const uint8_t* w2, const uint8_t* w2_scale, const moe_shape_t* shape, void* out_bf16 /* [T,H] */,
                 int32_t* topk_ids /* [T,k] or NULL */, float* topk_w /* [T,k] or NULL */, int32_t* status_word, void* ws,
                 size_t ws_bytes, void* cuda_stream);
-/* Diagnostic: the one-launch kernel of moe_forward for any batch it can take (up to 4 tokens, T*k <= 32), where
- * moe_forward itself would run the four calls because they are faster from 2 tokens on.  Same arguments, workspace and
- * result as moe_forward; MOE_ERR_UNSUPPORTED_SHAPE if the kernel cannot take the shape.  For the tests. */
-int moe_debug_forward_one_launch(const float* logits, const void* x_bf16, const uint8_t* w13, const uint8_t* w13_scale,
-                                 const uint8_t* w2, const uint8_t* w2_scale, const moe_shape_t* shape, void* out_bf16,
-                                 int32_t* topk_ids, float* topk_w, int32_t* status_word, void* ws, size_t ws_bytes,
-                                 void* cuda_stream);
-
 /* The same on weights written by moe_prepack (same workspace, same rules, same result). */
 int moe_forward_packed(const float* logits /* [T,E] */, const void* x_bf16 /* [T,H] */, const void* packed,
                        const moe_shape_t* shape, void* out_bf16 /* [T,H] */, int32_t* topk_ids /* [T,k] or NULL */,

@@ -27,20 +27,52 @@ int check_ws(const void* ws, size_t ws_bytes, size_t need) {
 }
 }  // namespace
 
+namespace {
+// see StatusRef: the word used by calls whose caller passed no status word; one per device that loads the library
+static __device__ int g_status_fallback;
+int* g_status_fallback_addr[kMaxDevices] = {};
+}  // namespace
+
+int resolve_status(int32_t* user_word, StatusRef* out) {
+  if (user_word != nullptr) {
+    *out = StatusRef{user_word, false};
+    return MOE_OK;
+  }
+  const int dev = current_device();
+  if (dev < 0 || dev >= kMaxDevices) return MOE_ERR_CUDA;
+  if (g_status_fallback_addr[dev] == nullptr) {
+    // the name of a __device__ variable is a host-side handle: its device address is looked up per device
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_status_fallback) != cudaSuccess || p == nullptr) return MOE_ERR_CUDA;
+    g_status_fallback_addr[dev] = static_cast<int*>(p);
+  }
+  *out = StatusRef{g_status_fallback_addr[dev], true};
+  return MOE_OK;
+}
+
+// kernels that cannot clear the library's own status word themselves: a memset node before them
+static int clear_own_status(const StatusRef& s, cudaStream_t st) {
+  if (s.own && cudaMemsetAsync(s.word, 0, sizeof(int), st) != cudaSuccess) return MOE_ERR_CUDA;
+  return MOE_OK;
+}
+
 void note_kernel(const char* name, int launches) {
   g_last_kernel = name;
   g_launches += static_cast<uint64_t>(launches);
 }
 
+int current_device() {
+  int dev = -1;
+  return cudaGetDevice(&dev) == cudaSuccess ? dev : -1;
+}
+
 int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        n <= 0)
-      n = 148;
-  }
-  return n;
+  static int n[kMaxDevices] = {};
+  const int dev = current_device();
+  if (dev < 0 || dev >= kMaxDevices) return 148;
+  if (n[dev] == 0 && (cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n[dev] <= 0))
+    n[dev] = 148;
+  return n[dev];
 }
 
 }  // namespace moe
@@ -114,9 +146,13 @@ int expert_ffn_impl(const void* x_perm_bf16, const int32_t* expert_offsets, cons
   // FP4 MMA for decode-sized batches, bf16 grouped GEMM for prefill-sized batches, the register-expansion streaming
   // kernel for every other shape.  The streaming kernel reads whole rows, so with the tile-contiguous weight layout
   // (which only shapes the first two kernels take can have) the grouped GEMM also takes what is left.
-  if (native_shape_ok(*shape, w.w13, w.w2)) return launch_expert_ffn_native(xp, expert_offsets, w, *shape, act, y_perm, status_word, st);
-  if (umma_shape_ok(*shape) || w.blocked) return launch_expert_ffn_umma(xp, expert_offsets, w, *shape, act, y_perm, status_word, st);
-  return launch_expert_ffn_stream(xp, expert_offsets, w.w13, w.s13, w.w2, w.s2, *shape, act, y_perm, status_word, st);
+  StatusRef status;
+  int rc = resolve_status(status_word, &status);
+  if (rc != MOE_OK) return rc;
+  if (native_shape_ok(*shape, w.w13, w.w2)) return launch_expert_ffn_native(xp, expert_offsets, w, *shape, act, y_perm, status, st);
+  if ((rc = clear_own_status(status, st)) != MOE_OK) return rc;
+  if (umma_shape_ok(*shape) || w.blocked) return launch_expert_ffn_umma(xp, expert_offsets, w, *shape, act, y_perm, status.word, st);
+  return launch_expert_ffn_stream(xp, expert_offsets, w.w13, w.s13, w.w2, w.s2, *shape, act, y_perm, status.word, st);
 }
 
 // the four tensors inside a buffer written by moe_prepack
@@ -147,8 +183,26 @@ int moe_prepack(const uint8_t* w13, const uint8_t* w13_scale, const uint8_t* w2,
   if (rc != MOE_OK) return rc;
   if (!aligned(w13, 16) || !aligned(w13_scale, 16) || !aligned(w2, 16) || !aligned(w2_scale, 16)) return MOE_ERR_INVALID_ARG;
   if (!aligned(packed_out, kAlign) || packed_bytes < packed_layout(*shape).total) return MOE_ERR_WORKSPACE;
-  return launch_prepack(w13, w13_scale, w2, w2_scale, *shape, static_cast<uint8_t*>(packed_out),
-                        static_cast<cudaStream_t>(cuda_stream));
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  // load check of the scale bytes (once per model load, so a round trip to the host is affordable): the kernels
+  // take bytes 0..128 only, and a larger one would give silently unspecified values on the hot path
+  StatusRef counter;  // the library's own device word doubles as the counter of this one-time check
+  if (resolve_status(nullptr, &counter) != MOE_OK) return MOE_ERR_CUDA;
+  const size_t n = static_cast<size_t>(shape->E) * shape->H * shape->I;
+  const uint8_t* tensors[2] = {w13_scale, w2_scale};
+  const size_t sizes[2] = {n / 16, n / 32};
+  for (int i = 0; i < 2; ++i) {
+    int bad = 0;
+    if (launch_validate_scales(tensors[i], sizes[i], counter.word, st) != MOE_OK ||
+        cudaMemcpyAsync(&bad, counter.word, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+      return MOE_ERR_CUDA;
+    if (bad != 0) {
+      cudaMemsetAsync(counter.word, 0, sizeof(int), st);
+      return MOE_ERR_INVALID_ARG;
+    }
+  }
+  return launch_prepack(w13, w13_scale, w2, w2_scale, *shape, static_cast<uint8_t*>(packed_out), st);
 }
 
 int moe_expert_ffn_packed(const void* x_perm_bf16, const int32_t* expert_offsets, const void* packed, const moe_shape_t* shape,
@@ -230,10 +284,13 @@ int forward_impl(const float* logits, const void* x_bf16, const ExpertWeights& w
   if (check_ws(ws, ws_bytes, L.total) != MOE_OK) return MOE_ERR_WORKSPACE;
   char* base = static_cast<char*>(ws);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  if (forward_fused_ok(*shape, w.w13, w.w2) && forward_fused_preferred(*shape))
+  if (forward_fused_ok(*shape, w.w13, w.w2) && forward_fused_preferred(*shape)) {
+    StatusRef status;
+    if ((rc = resolve_status(status_word, &status)) != MOE_OK) return rc;
     return launch_forward_fused(logits, static_cast<const __nv_bfloat16*>(x_bf16), w, *shape,
                                 static_cast<__nv_bfloat16*>(out_bf16), topk_ids, topk_w, reinterpret_cast<int*>(base),
-                                base + kForwardSyncBytes, status_word, st);
+                                base + kForwardSyncBytes, status, st);
+  }
   int32_t* d_ids = topk_ids != nullptr ? topk_ids : reinterpret_cast<int32_t*>(base + L.ids);
   float* d_w = topk_w != nullptr ? topk_w : reinterpret_cast<float*>(base + L.w);
   int32_t* d_off = reinterpret_cast<int32_t*>(base + L.offsets);
@@ -273,9 +330,42 @@ int moe_debug_forward_one_launch(const float* logits, const void* x_bf16, const 
   if (!forward_fused_ok(*shape, w13, w2)) return MOE_ERR_UNSUPPORTED_SHAPE;
   if (check_ws(ws, ws_bytes, forward_layout(*shape).total) != MOE_OK) return MOE_ERR_WORKSPACE;
   char* base = static_cast<char*>(ws);
+  StatusRef status;
+  const int rs = resolve_status(status_word, &status);
+  if (rs != MOE_OK) return rs;
   return launch_forward_fused(logits, static_cast<const __nv_bfloat16*>(x_bf16), ExpertWeights{w13, w13_scale, w2, w2_scale, false},
                               *shape, static_cast<__nv_bfloat16*>(out_bf16), topk_ids, topk_w, reinterpret_cast<int*>(base),
-                              base + kForwardSyncBytes, status_word, static_cast<cudaStream_t>(cuda_stream));
+                              base + kForwardSyncBytes, status, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int moe_debug_expert_ffn_variant(const void* x_perm_bf16, const int32_t* expert_offsets, const uint8_t* w13,
+                                 const uint8_t* w13_scale, const uint8_t* w2, const uint8_t* w2_scale, const moe_shape_t* shape,
+                                 float* y_perm, int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream,
+                                 int32_t variant) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (!aligned(x_perm_bf16, 16) || !aligned(expert_offsets, 16) || !aligned(w13, 16) || !aligned(w13_scale, 16) ||
+      !aligned(w2, 16) || !aligned(w2_scale, 16) || !aligned(y_perm, 16) || variant < 0 || variant > 2 ||
+      (status_word != nullptr && !aligned(status_word, 4)))
+    return MOE_ERR_INVALID_ARG;
+  const WsLayout L = ws_layout(*shape);
+  if (check_ws(ws, ws_bytes, L.total) != MOE_OK) return MOE_ERR_WORKSPACE;
+  __nv_bfloat16* act = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(ws) + L.act_off);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const __nv_bfloat16* xp = static_cast<const __nv_bfloat16*>(x_perm_bf16);
+  const ExpertWeights w{w13, w13_scale, w2, w2_scale, false};
+  StatusRef status;
+  if ((rc = resolve_status(status_word, &status)) != MOE_OK) return rc;
+  if (variant == 2) {
+    if (!native_shape_ok(*shape, w13, w2)) return MOE_ERR_UNSUPPORTED_SHAPE;
+    return launch_expert_ffn_native(xp, expert_offsets, w, *shape, act, y_perm, status, st);
+  }
+  if ((rc = clear_own_status(status, st)) != MOE_OK) return rc;
+  if (variant == 1) {
+    if (!blocked_shape(*shape) || !umma_shape_ok(moe_shape_t{1 << 20, shape->H, shape->I, shape->E, 1})) return MOE_ERR_UNSUPPORTED_SHAPE;
+    return launch_expert_ffn_umma(xp, expert_offsets, w, *shape, act, y_perm, status.word, st);
+  }
+  return launch_expert_ffn_stream(xp, expert_offsets, w13, w13_scale, w2, w2_scale, *shape, act, y_perm, status.word, st);
 }
 
 int moe_forward_packed(const float* logits, const void* x_bf16, const void* packed, const moe_shape_t* shape, void* out_bf16,

@@ -7,6 +7,7 @@
 #include <stdint.h>
 
 #include "../../include/moe_b200.h"
+#include "../../include/moe_b200_debug.h"
 
 #define MOE_DEVINL __device__ __forceinline__
 
@@ -95,6 +96,20 @@ inline PackedLayout packed_layout(const moe_shape_t& s) {
 int launch_prepack(const uint8_t* w13, const uint8_t* s13, const uint8_t* w2, const uint8_t* s2, const moe_shape_t& s,
                    uint8_t* packed, cudaStream_t st);
 
+// ---- the status word the kernels report through (host) ---------------------------------------------
+// The caller's, or - when the caller passed NULL - one word inside the library image per device, so that the rule
+// "once one bounded wait has run out, every later wait of the grid gives up after a short spin" holds for every
+// call: without a word to look at, one lost signal would cost the full limit in every wait that follows it.
+// The library's own word is cleared by the call that uses it (`own` tells the launcher to arrange that: by a kernel
+// of the call where one runs before the waits or after them, else by a memset node before the launches); nobody
+// reads it on the host.  Calls that pass NULL and overlap on the GPU share it: a timeout in one may cut short the
+// waits of the other, whose results are then reported nowhere - pass a status word to know.
+struct StatusRef {
+  int* word;
+  bool own;
+};
+int resolve_status(int32_t* user_word, StatusRef* out);  // MOE_OK or MOE_ERR_CUDA
+
 // ---- per-thread call record (host) -----------------------------------------------------------
 void note_kernel(const char* name, int launches);
 
@@ -118,7 +133,7 @@ int launch_validate_scales(const uint8_t* scales, size_t n, int* bad, cudaStream
 // native block-scaled FP4 variant; scratch of native_scratch_bytes
 bool native_shape_ok(const moe_shape_t& s, const void* w13, const void* w2);
 int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& s,
-                             void* scratch, float* y_perm, int* status_word, cudaStream_t st);
+                             void* scratch, float* y_perm, StatusRef status, cudaStream_t st);
 
 // the whole layer in one launch, for a handful of tokens on shapes the native variant takes (moe_forward);
 // `sync` is the zeroed block of kForwardSyncBytes, `scratch` holds forward_fused_scratch_bytes
@@ -127,15 +142,39 @@ bool forward_fused_ok(const moe_shape_t& s, const void* w13, const void* w2);  /
 bool forward_fused_preferred(const moe_shape_t& s);                             // and is the faster choice (measured)
 size_t forward_fused_scratch_bytes(const moe_shape_t& s);
 int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const ExpertWeights& w, const moe_shape_t& s,
-                         __nv_bfloat16* out, int* ids_out, float* w_out, int* sync, void* scratch, int* status_word,
+                         __nv_bfloat16* out, int* ids_out, float* w_out, int* sync, void* scratch, StatusRef status,
                          cudaStream_t st);
 
-int sm_count();
+int sm_count();  // of the current device
+
+// ---- per-device one-time set-up (host) ---------------------------------------------------------------
+// cudaFuncSetAttribute and the SM count belong to a device, not to the process: a process that drives several GPUs
+// through this library sets each kernel's attributes once on every device it calls from.
+constexpr int kMaxDevices = 64;
+int current_device();  // -1 if the runtime cannot tell
+struct PerDeviceFlag {
+  bool done[kMaxDevices] = {};
+};
+template <typename F>
+inline bool once_per_device(PerDeviceFlag& f, F&& set) {
+  const int d = current_device();
+  if (d < 0 || d >= kMaxDevices) return false;
+  if (!f.done[d]) {
+    if (!set()) return false;
+    f.done[d] = true;
+  }
+  return true;
+}
 
 // ---- programmatic dependent launch (host) ------------------------------------------------------
 // The kernel may start while its predecessor in the stream is still running; it must execute
-// griddepcontrol.wait before it touches anything the predecessor writes or reads.  Every kernel launched
-// this way here waits first and only then lets its own dependent start, so at most two neighbours overlap.
+// griddepcontrol.wait before it reads anything the predecessor writes, and before it writes anything at all to
+// global memory.  Most kernels here wait first and then release their own dependent; route_kernel, native_split_kernel
+// and the expert-FFN kernels release theirs BEFORE they wait, so three or four neighbours of a chain (route, permute,
+// split, expert FFN) can be resident together.  That is safe because of the rule above: whatever a kernel does before
+// its wait only reads buffers that no kernel of the chain before it writes (logits, expert_offsets of a completed
+// router, the weights), and every global write comes after the wait, i.e. after everything launched earlier on the
+// stream has completed.
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
   cudaLaunchConfig_t cfg = {};

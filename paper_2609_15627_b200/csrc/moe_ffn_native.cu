@@ -83,7 +83,8 @@ struct NatArgs {
   int* done;                 // [E] epilogue warps that have published a gate/up item of the expert
   const int* offsets;
   float* y;                  // output [S, H]
-  int* status;
+  int* status;               // never null: the caller's word or the library's own (see StatusRef)
+  int own_status;            // the library's own word: the one-launch kernel's last CTA clears it for the next call
   int E, H, I, S;
   int blocked;               // weights in moe_prepack's tile-contiguous layout (see ExpertWeights)
 };
@@ -320,12 +321,15 @@ MOE_DEVINL void split_terms(float (&r)[NB][4], Store store) {
 // grid still occupies delays one of them - with at most (SMs - working FFN CTAs) CTAs here, only idle ones.
 __global__ void __launch_bounds__(1024) native_split_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict__ aq,
                                                            uint8_t* __restrict__ aq_sf, int* __restrict__ done, int S, int H,
-                                                           int E) {
+                                                           int E, int* __restrict__ status_clear) {
   pdl_launch_dependents();  // the FFN grid may set up and start its weight stream; it waits before it reads aq or done
   pdl_wait();               // the sorted token rows of moe_permute are complete, and every earlier kernel on the stream
   const int n_blk = H / 32;
   const long long gt = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (gt < E) done[gt] = 0;
+  // the library's own status word (caller passed none): whatever an earlier call left there is over, and the FFN grid
+  // of this call looks at the word only in waits that have lasted a millisecond
+  if (gt == 0 && status_clear != nullptr) *status_clear = 0;
   const long long task = gt >> 3;  // (row, block); the grid is padded to whole warps, so whole tasks are in or out
   const int sub = static_cast<int>(gt & 7);
   const bool live = task < static_cast<long long>(S) * n_blk;
@@ -681,6 +685,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         if (lane == 0) {
           f.sync[kSyncExit] = 0;
           f.sync[kSyncSplit] = 0;
+          if (a.own_status) *a.status = 0;  // every wait of this call is over; nobody reads this word on the host
         }
       }
     }
@@ -1060,14 +1065,11 @@ bool nat_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint64_t rows
 
 namespace {
 bool nat_attr_once() {
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(ffn_native_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-        cudaFuncSetAttribute(ffn_native_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
-      return false;
-    attr_done = true;
-  }
-  return true;
+  static PerDeviceFlag flag;
+  return once_per_device(flag, [] {
+    return cudaFuncSetAttribute(ffn_native_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess &&
+           cudaFuncSetAttribute(ffn_native_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+  });
 }
 }  // namespace
 
@@ -1095,7 +1097,7 @@ bool native_shape_ok(const moe_shape_t& sh, const void* w13, const void* w2) {
 }
 
 int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& sh,
-                             void* scratch, float* y_perm, int* status_word, cudaStream_t st) {
+                             void* scratch, float* y_perm, StatusRef status, cudaStream_t st) {
   if (!nat_attr_once()) return MOE_ERR_CUDA;
   const size_t S = static_cast<size_t>(sh.T) * sh.k;
   // scratch: term rows of the intermediate and of the token rows, each followed by its scale bytes; the counters
@@ -1113,7 +1115,7 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
   if (!weight_maps(w, sh, &tm_w13, &tm_s13, &tm_w2, &tm_s2)) return MOE_ERR_CUDA;
   const size_t split_threads = S * (sh.H / 32) * 8 > static_cast<size_t>(sh.E) ? S * (sh.H / 32) * 8 : static_cast<size_t>(sh.E);
   if (launch_pdl(native_split_kernel, dim3(static_cast<unsigned>((split_threads + 1023) / 1024)), dim3(1024), 0, st, x_perm, aq1, sf1,
-                 done, static_cast<int>(S), sh.H, sh.E) != cudaSuccess)
+                 done, static_cast<int>(S), sh.H, sh.E, status.own ? status.word : nullptr) != cudaSuccess)
     return MOE_ERR_CUDA;
   NatArgs a;
   a.sf1 = sf1;
@@ -1122,7 +1124,8 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
   a.done = done;
   a.offsets = offsets;
   a.y = y_perm;
-  a.status = status_word;
+  a.status = status.word;
+  a.own_status = 0;
   a.E = sh.E;
   a.H = sh.H;
   a.I = sh.I;
@@ -1153,7 +1156,7 @@ size_t forward_fused_scratch_bytes(const moe_shape_t& sh) {
 bool forward_fused_preferred(const moe_shape_t& sh) { return sh.T <= kFusedPreferredTok; }
 
 int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const ExpertWeights& w, const moe_shape_t& sh,
-                         __nv_bfloat16* out, int* ids_out, float* w_out, int* sync, void* scratch, int* status_word,
+                         __nv_bfloat16* out, int* ids_out, float* w_out, int* sync, void* scratch, StatusRef status,
                          cudaStream_t st) {
   if (!nat_attr_once()) return MOE_ERR_CUDA;
   const size_t S = static_cast<size_t>(sh.T) * sh.k;
@@ -1180,7 +1183,8 @@ int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const Expe
   a.done = sync;
   a.offsets = nullptr;
   a.y = y;
-  a.status = status_word;
+  a.status = status.word;
+  a.own_status = status.own ? 1 : 0;
   a.E = sh.E;
   a.H = sh.H;
   a.I = sh.I;

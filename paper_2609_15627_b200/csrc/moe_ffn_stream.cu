@@ -272,16 +272,15 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const FfnArgs a
 int launch_expert_ffn_stream(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
                       const uint8_t* w2, const uint8_t* s2, const moe_shape_t& sh, __nv_bfloat16* act, float* y_perm,
                       int* status_word, cudaStream_t st) {
-  static bool attr_done = false;
   constexpr int kSmemBudget = 200 * 1024;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(ffn_stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 24 * 1024) !=
-            cudaSuccess ||
-        cudaFuncSetAttribute(ffn_stream_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 24 * 1024) !=
-            cudaSuccess)
-      return MOE_ERR_CUDA;
-    attr_done = true;
-  }
+  static PerDeviceFlag flag;
+  if (!once_per_device(flag, [] {
+        return cudaFuncSetAttribute(ffn_stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 24 * 1024) ==
+                   cudaSuccess &&
+               cudaFuncSetAttribute(ffn_stream_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 24 * 1024) ==
+                   cudaSuccess;
+      }))
+    return MOE_ERR_CUDA;
   const int grid = sm_count();
   auto run = [&](bool stage1) -> bool {
     FfnArgs a;

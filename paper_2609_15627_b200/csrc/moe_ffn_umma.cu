@@ -398,13 +398,12 @@ bool umma_shape_ok(const moe_shape_t& sh) {
 int launch_expert_ffn_umma(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& sh,
                            __nv_bfloat16* act, float* y_perm, int* status_word, cudaStream_t st) {
   const size_t smem = smem_map(sh.E).total + 1024;
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(ffn_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-        cudaFuncSetAttribute(ffn_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
-      return MOE_ERR_CUDA;
-    attr_done = true;
-  }
+  static PerDeviceFlag flag;
+  if (!once_per_device(flag, [] {
+        return cudaFuncSetAttribute(ffn_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess &&
+               cudaFuncSetAttribute(ffn_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+      }))
+    return MOE_ERR_CUDA;
   const uint64_t S = static_cast<uint64_t>(sh.T) * sh.k;
   CUtensorMap tm_x, tm_act, tm_w13, tm_w2;
   if (!make_map_2d(&tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, x_perm, sh.H, S, kBlockK, kTokBox, CU_TENSOR_MAP_SWIZZLE_128B) ||

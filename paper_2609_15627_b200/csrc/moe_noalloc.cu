@@ -8,7 +8,6 @@ namespace moe {
 namespace {
 
 constexpr size_t kStaticScratchBytes = 16u << 20;  // 16 MiB
-constexpr int kMaxDevices = 64;
 
 // Lives in every GPU context that loads the library, until the process exits.
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
@@ -51,6 +50,7 @@ int moe_expert_ffn_noalloc(const void* x_perm_bf16, const int32_t* expert_offset
   if (!aligned16(x_perm_bf16) || !aligned16(expert_offsets) || !aligned16(w13) || !aligned16(w13_scale) || !aligned16(w2) ||
       !aligned16(w2_scale) || !aligned16(y_perm))
     return MOE_ERR_INVALID_ARG;
+  if (status_word != nullptr && (reinterpret_cast<uintptr_t>(status_word) & 3u) != 0) return MOE_ERR_INVALID_ARG;
   // what the chosen kernel keeps between its launches must fit the fixed array: the bf16 intermediate act[T*k, I],
   // or for the native variant the E2M1 term rows and scale bytes of both projections' inputs (4.25 (H + I) bytes per slot)
   const unsigned long long S = static_cast<unsigned long long>(s.T) * s.k;
@@ -58,8 +58,10 @@ int moe_expert_ffn_noalloc(const void* x_perm_bf16, const int32_t* expert_offset
       (native_shape_ok(s, w13, w2) ? static_cast<unsigned long long>(native_scratch_bytes(s)) : S * s.I * 2ULL) + kAlign;
   if (need > kStaticScratchBytes) return MOE_ERR_WORKSPACE;
   void* scratch = nullptr;
-  const int rc = static_scratch(&scratch);  // first call on a device looks the address up
+  int rc = static_scratch(&scratch);  // first call on a device looks the address up
   if (rc != MOE_OK) return rc;
+  StatusRef status;  // the caller's word, or the library's own (a second fixed device word; nothing is allocated)
+  if ((rc = resolve_status(status_word, &status)) != MOE_OK) return rc;
   // Every row of act that stage 2 reads is written by stage 1 of the same call, so nothing in the array has
   // to start at zero.  Same kernels and the same kernel choice as moe_expert_ffn.
   __nv_bfloat16* act = static_cast<__nv_bfloat16*>(scratch);
@@ -67,12 +69,13 @@ int moe_expert_ffn_noalloc(const void* x_perm_bf16, const int32_t* expert_offset
   const ExpertWeights w{w13, w13_scale, w2, w2_scale, false};
   if (native_shape_ok(s, w13, w2))
     return launch_expert_ffn_native(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w, s, scratch, y_perm,
-                                    status_word, st);
+                                    status, st);
+  if (status.own && cudaMemsetAsync(status.word, 0, sizeof(int), st) != cudaSuccess) return MOE_ERR_CUDA;
   if (umma_shape_ok(s))
     return launch_expert_ffn_umma(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w, s, act, y_perm,
-                                  status_word, st);
+                                  status.word, st);
   return launch_expert_ffn_stream(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w13, w13_scale, w2,
-                                  w2_scale, s, act, y_perm, status_word, st);
+                                  w2_scale, s, act, y_perm, status.word, st);
 }
 
 }  // extern "C"

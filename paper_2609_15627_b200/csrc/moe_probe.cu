@@ -59,13 +59,12 @@ extern "C" int moe_debug_read_probe(const void* src, size_t bytes, void* sink, s
   if (src == nullptr || sink == nullptr || (reinterpret_cast<uintptr_t>(src) & 127u) != 0 || bytes < static_cast<size_t>(kProbeChunk) ||
       sink_bytes < static_cast<size_t>(sm_count()) * 4)
     return MOE_ERR_INVALID_ARG;
-  static bool attr_done = false;
   const size_t smem = static_cast<size_t>(kProbeStages) * kProbeChunk + 2 * kProbeStages * 8 + 128;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(read_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
-      return MOE_ERR_CUDA;
-    attr_done = true;
-  }
+  static PerDeviceFlag flag;
+  if (!once_per_device(flag, [smem] {
+        return cudaFuncSetAttribute(read_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) == cudaSuccess;
+      }))
+    return MOE_ERR_CUDA;
   read_probe_kernel<<<sm_count(), 64, smem, static_cast<cudaStream_t>(cuda_stream)>>>(
       static_cast<const uint8_t*>(src), static_cast<long long>(bytes / kProbeChunk), static_cast<unsigned*>(sink), status_word);
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;

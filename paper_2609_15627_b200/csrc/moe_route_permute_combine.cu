@@ -106,12 +106,11 @@ int launch_route(const float* logits, int T, int E, int k, int* ids, float* w, i
   const bool single = T <= 128;
   const int nw = single ? 32 : 8;
   const size_t smem = (static_cast<size_t>(nw) * E + E + 40) * 4;
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
-      return MOE_ERR_CUDA;
-    attr_done = true;
-  }
+  static PerDeviceFlag flag;
+  if (!once_per_device(flag, [] {
+        return cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) == cudaSuccess;
+      }))
+    return MOE_ERR_CUDA;
   int launches = 1;
   if (single) {
     if (launch_pdl(route_kernel, dim3(1), dim3(nw * 32), smem, st, logits, T, E, k, ids, w, offsets, counters, 1) != cudaSuccess)

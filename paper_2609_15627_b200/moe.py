@@ -17,7 +17,8 @@ EXPORTS = ("moe_workspace_bytes", "moe_status_string", "moe_last_kernel_name", "
            "moe_forward_workspace_bytes", "moe_forward_sync_bytes", "moe_forward",
            "moe_forward_host_workspace_bytes", "moe_forward_host", "moe_expert_ffn_noalloc_max_bytes",
            "moe_expert_ffn_noalloc", "moe_debug_native_cta_share", "moe_debug_read_probe", "moe_prepack_bytes", "moe_prepack",
-           "moe_expert_ffn_packed", "moe_forward_packed", "moe_forward_host_packed", "moe_debug_forward_one_launch")
+           "moe_expert_ffn_packed", "moe_forward_packed", "moe_forward_host_packed", "moe_debug_forward_one_launch",
+           "moe_debug_expert_ffn_variant")
 
 
 class MoeError(RuntimeError):
@@ -82,6 +83,8 @@ def lib():
         L.moe_forward.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp, vp, vp, sz, vp]
         L.moe_debug_forward_one_launch.restype = C.c_int
         L.moe_debug_forward_one_launch.argtypes = L.moe_forward.argtypes
+        L.moe_debug_expert_ffn_variant.restype = C.c_int
+        L.moe_debug_expert_ffn_variant.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp, sz, vp, i32]
         L.moe_forward_host.restype = C.c_int
         L.moe_forward_host.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp, sz, vp]
         _lib = L
@@ -144,6 +147,17 @@ def moe_expert_ffn(x_perm, expert_offsets, w13, w13_scale, w2, w2_scale, sh, y_p
     _check(lib().moe_expert_ffn(_ptr(x_perm), _ptr(expert_offsets), _ptr(w13), _ptr(w13_scale), _ptr(w2), _ptr(w2_scale),
                                 C.byref(sh), _ptr(y_perm), _ptr(status_word), _ptr(ws), ws.numel(), _stream(stream)),
            "moe_expert_ffn")
+
+
+VARIANT_STREAM, VARIANT_UMMA, VARIANT_NATIVE = 0, 1, 2
+
+
+def moe_debug_expert_ffn_variant(x_perm, expert_offsets, w13, w13_scale, w2, w2_scale, sh, y_perm, status_word, ws, variant,
+                                 stream=None):
+    """moe_expert_ffn with the kernel variant named by the caller (see include/moe_b200_debug.h)."""
+    _check(lib().moe_debug_expert_ffn_variant(_ptr(x_perm), _ptr(expert_offsets), _ptr(w13), _ptr(w13_scale), _ptr(w2),
+                                              _ptr(w2_scale), C.byref(sh), _ptr(y_perm), _ptr(status_word), _ptr(ws),
+                                              ws.numel(), _stream(stream), int(variant)), "moe_debug_expert_ffn_variant")
 
 
 def moe_expert_ffn_noalloc_max_bytes():

@@ -31,6 +31,17 @@ def run_layer(wl, d, wdev=None):
     return buf, out
 
 
+def bf16_neighbours(f32):
+    """The two bf16 values that bracket each (finite) fp32 value: the truncation towards zero and the next bf16
+    value away from zero, one unit in the last place of the TRUNCATED value's binade further (bf16 bit patterns of
+    one sign are ordered like their magnitudes, so that neighbour is the bit pattern plus one).  Returned as
+    float64 arrays; a value that is itself a bf16 number gets (itself, the next one away from zero)."""
+    f = np.ascontiguousarray(f32, dtype=np.float32)
+    lo_bits = (f.view(np.uint32) >> np.uint32(16)).astype(np.uint16)
+    hi_bits = (lo_bits + np.uint16(1)).astype(np.uint16)
+    return (inputs.bf16_bits_to_f32(lo_bits).astype(np.float64), inputs.bf16_bits_to_f32(hi_bits).astype(np.float64))
+
+
 def check_out(got_bits, ref_bits, ref_f32, what=""):
     """The stated tolerance: rel-Frobenius <= 5e-3 and max|diff| <= 2e-2 * rms(reference).
 
@@ -45,12 +56,9 @@ def check_out(got_bits, ref_bits, ref_f32, what=""):
     over = diff > 2e-2 * rms
     flips = 0
     if over.any():
-        f = ref_f32[over].astype(np.float32)
-        lo = inputs.bf16_bits_to_f32((f.view(np.uint32) >> 16).astype(np.uint16))            # truncation
-        step = np.abs(lo) * 2.0 ** -7
-        hi = lo + np.sign(f) * np.where(step > 0, step, 2.0 ** -133)
+        lo, hi = bf16_neighbours(ref_f32[over])
         g = got[over]
-        ok = (g == lo) | (g == hi.astype(np.float32))
+        ok = (g == lo) | (g == hi)
         assert ok.all(), "%s: %d elements beyond 2e-2*rms that are not bf16 rounding flips (max %g, rms %g)" % (
             what, int((~ok).sum()), diff.max(), rms)
         flips = int(over.sum())

@@ -18,8 +18,10 @@ def L():
 
 
 def test_every_declared_symbol_is_exported(L):
-    header = open(os.path.join(ROOT, "include", "moe_b200.h")).read()
+    header = "".join(open(os.path.join(ROOT, "include", h)).read() for h in ("moe_b200.h", "moe_b200_debug.h"))
     declared = set(re.findall(r"\b(moe_[a-z0-9_]+)\s*\(", header))
+    public = open(os.path.join(ROOT, "include", "moe_b200.h")).read()
+    assert not re.findall(r"\b(moe_debug_[a-z0-9_]+)\s*\(", public)      # diagnostics stay out of the layer's header
     declared -= {"moe_status_t", "moe_shape_t"}
     assert {"moe_route", "moe_permute", "moe_expert_ffn", "moe_combine"} <= declared
     for name in sorted(declared):
