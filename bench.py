@@ -35,7 +35,10 @@ METRIC = "MoE FP4 layer tokens/s"
 DECODE = ("decode_c1", "decode_c64")
 PRODUCTION = ("decode_c1", "decode_c64", "prefill_8k", "prefill_32k_skewed")
 HEADLINE = "decode_c1"
-MIN_REGION_MS = 100.0   # a timed round of the per-workload figures lasts at least this long
+MIN_REGION_MS = 100.0   # a timed round of a decode workload lasts at least this long
+MIN_REGION_MS_PREFILL = 40.0  # prefill rounds: at least this long and at least 3 steps - a burst-length region, to go with
+                              # the burst bf16 peak they are divided by (a single sub-millisecond GEMM, best of ten)
+COOLDOWN_S = 1.0        # idle time before every round: each round starts with the board below its power limit
 ROUNDS = 3
 GRAPH_STEPS = 8         # consecutive batches of the cycle per CUDA graph (decode workloads)
 
@@ -423,12 +426,14 @@ class Bench:
         # ---- rounds of at least MIN_REGION_MS ---------------------------------------------------------------------
         pilot_n = GRAPH_STEPS if use_graph else 2
         pilot_ms = region(pilot_n)[0] / pilot_n
-        n_steps = steps_for_region(pilot_ms, multiple=GRAPH_STEPS if use_graph else 1, at_least=3)
+        n_steps = steps_for_region(pilot_ms, MIN_REGION_MS if decode else MIN_REGION_MS_PREFILL,
+                                   multiple=GRAPH_STEPS if use_graph else 1, at_least=3)
         n_inner = 0 if (use_graph or one_launch) else n_steps
         inner = [self.events() for _ in range(n_inner)]
         rounds, clock_rounds, reasons, launches = [], [], set(), 0
         ffn_round_ms = []
         for _ in range(ROUNDS):
+            time.sleep(COOLDOWN_S)
             ms, clocks, launches = region(n_steps, inner if n_inner else None)
             rounds.append(ms / n_steps)
             clock_rounds.append(clocks["sm_mhz"])
@@ -687,9 +692,10 @@ def main():
             "roofline": roof, "cpu_baseline": cpu, "e2e": hr.get("e2e"), "gpu_launches": ex["gpu_launches"],
             "clocks": ex["clocks"], "kernels": hr["kernels"],
             "workloads": {n: {k: v for k, v in r.items() if k not in ("one_launch", "n_cycle")} for n, r in records.items()},
-            "protocol": ("headline: one region of exactly --steps steps; workloads: %d rounds of at least %d ms each, median "
-                         "reported, every round kept; every region is bracketed by a barrier and a synchronize, timed by CUDA "
-                         "events on the launching stream behind a 100 us hold kernel, max over ranks") % (ROUNDS, MIN_REGION_MS),
+            "protocol": ("headline: one region of exactly --steps steps; workloads: %d rounds of at least %d ms (decode) / %d ms "
+                         "(prefill) each, %.1f s idle before every round, median reported, every round kept; every region is "
+                         "bracketed by a barrier and a synchronize, timed by CUDA events on the launching stream behind a "
+                         "100 us hold kernel, max over ranks") % (ROUNDS, MIN_REGION_MS, MIN_REGION_MS_PREFILL, COOLDOWN_S),
         }
         print(json.dumps(line))
     if world > 1:
