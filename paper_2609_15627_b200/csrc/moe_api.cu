@@ -255,10 +255,11 @@ ForwardLayout forward_layout(const moe_shape_t& s) {
   off += ws_layout(s).total;
   // whether the one-launch kernel applies also depends on the weights' alignment; the size allows for it whenever
   // the shape does
-  const size_t fused = forward_fused_ok(s, reinterpret_cast<const void*>(uintptr_t(256)), reinterpret_cast<const void*>(uintptr_t(256)))
-                           ? kForwardSyncBytes + forward_fused_scratch_bytes(s)
-                           : 0;
+  const void* al = reinterpret_cast<const void*>(uintptr_t(256));
+  const size_t fused = forward_fused_ok(s, al, al) ? kForwardSyncBytes + forward_fused_scratch_bytes(s) : 0;
+  const size_t one = decode_one_ok(s, al, al) ? kForwardSyncBytes + decode_one_scratch_bytes(s) : 0;
   L.total = off > fused ? off : fused;
+  L.total = L.total > one ? L.total : one;
   return L;
 }
 }  // namespace
@@ -284,6 +285,12 @@ int forward_impl(const float* logits, const void* x_bf16, const ExpertWeights& w
   if (check_ws(ws, ws_bytes, L.total) != MOE_OK) return MOE_ERR_WORKSPACE;
   char* base = static_cast<char*>(ws);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (decode_one_ok(*shape, w.w13, w.w2)) {
+    StatusRef status;
+    if ((rc = resolve_status(status_word, &status)) != MOE_OK) return rc;
+    return launch_decode_one(logits, static_cast<const __nv_bfloat16*>(x_bf16), w, *shape, static_cast<__nv_bfloat16*>(out_bf16),
+                             topk_ids, topk_w, reinterpret_cast<int*>(base), base + kForwardSyncBytes, status, st);
+  }
   if (forward_fused_ok(*shape, w.w13, w.w2) && forward_fused_preferred(*shape)) {
     StatusRef status;
     if ((rc = resolve_status(status_word, &status)) != MOE_OK) return rc;

@@ -138,12 +138,27 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
 // the whole layer in one launch, for a handful of tokens on shapes the native variant takes (moe_forward);
 // `sync` is the zeroed block of kForwardSyncBytes, `scratch` holds forward_fused_scratch_bytes
 constexpr size_t kForwardSyncBytes = 8192;
+// int indices inside that block (both one-launch kernels): [0, E) per-expert counters of the general kernel, then
+constexpr int kSyncDone2 = 1024;      // per column tile of the output: warps that have stored their rows of a down item
+constexpr int kSyncExit = 1024 + 64;  // CTAs that are through with the counters; the last one clears the block
+constexpr int kSyncSplit = 1024 + 65; // general kernel: CTAs that have written their share of the tokens' term rows
+// two words that no kernel ever writes: a call that finds one of them non-zero was given a block that was never
+// cleared, reports MOE_ERR_WORKSPACE through the status word and does nothing (every CTA takes the same decision)
+constexpr int kSyncCanary0 = 1024 + 66, kSyncCanary1 = 2047;
 bool forward_fused_ok(const moe_shape_t& s, const void* w13, const void* w2);  // the kernel can take the shape
 bool forward_fused_preferred(const moe_shape_t& s);                             // and is the faster choice (measured)
 size_t forward_fused_scratch_bytes(const moe_shape_t& s);
 int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const ExpertWeights& w, const moe_shape_t& s,
                          __nv_bfloat16* out, int* ids_out, float* w_out, int* sync, void* scratch, StatusRef status,
                          cudaStream_t st);
+
+// the whole layer for one token in one launch with the down projection split along K over pairs of CTAs (moe_forward
+// at T = 1 where the shape allows it); `sync` as above, `scratch` holds decode_one_scratch_bytes
+bool decode_one_ok(const moe_shape_t& s, const void* w13, const void* w2);
+size_t decode_one_scratch_bytes(const moe_shape_t& s);
+int launch_decode_one(const float* logits, const __nv_bfloat16* x, const ExpertWeights& w, const moe_shape_t& s,
+                      __nv_bfloat16* out, int* ids_out, float* w_out, int* sync, void* scratch, StatusRef status,
+                      cudaStream_t st);
 
 int sm_count();  // of the current device
 

@@ -49,6 +49,8 @@
 
 #include <algorithm>
 
+#include "moe_mxf4_device.cuh"
+#include "moe_tmap.cuh"
 #include "moe_route_device.cuh"
 #include "moe_sm100_primitives.cuh"
 
@@ -65,7 +67,6 @@ constexpr int kWStages = 4;
 constexpr int kScStages = 3;          // scale-byte ring: one stage = 256 rows x 16 bytes = 2 K steps
 constexpr int kScStage = kTile * 16;
 constexpr int kSfGroups = 3;          // tensor-memory groups for the weight scale factors: 4 words x 8 columns
-constexpr int kTerms = 8;             // E2M1 terms per activation value
 constexpr int kMaxTokPass = 16;       // tokens per pass (16 x 8 = 128 operand rows)
 constexpr int kMaxK = 4096;           // scale factors of one pass's term rows stay in tensor memory: 8 columns per K step
 constexpr int kNatThreads = 10 * 32;
@@ -105,17 +106,10 @@ struct NatArgs {
 constexpr int kFusedMaxTok = 4;
 constexpr int kFusedPreferredTok = 1;
 constexpr int kFusedMaxSlots = 32; // T * k: one warp sorts them
-constexpr int kSyncDone2 = 1024;   // int index in the sync block: per column tile, warps that stored a down item
-constexpr int kSyncExit = 1024 + 64;  // CTAs that have finished; the last one clears the block
-constexpr int kSyncSplit = 1024 + 65; // CTAs that have written their share of the tokens' term rows
-// These CTAs wait for one another (every other wait in the kernel points to CTAs with a lower index), so the grid
-// needs this many SMs to itself at the start; 16 CTAs x 20 groups of 8 lanes cover the 256 blocks of two 4096-wide rows
-// in one round, more CTAs would not make it shorter.
+// The CTAs that split the token rows wait for one another (every other wait in the kernel points to CTAs with a lower
+// index), so the grid needs this many SMs to itself at the start; 16 CTAs x 20 groups of 8 lanes cover the 256 blocks of
+// two 4096-wide rows in one round, more CTAs would not make it shorter.
 constexpr int kSplitCtas = 16;
-// two words of the sync block that no kernel ever writes: a call that finds one of them non-zero was given a block
-// that was never cleared, reports MOE_ERR_WORKSPACE through the status word and does nothing (every CTA takes the same
-// decision, since nobody changes these words)
-constexpr int kSyncCanary0 = 1024 + 66, kSyncCanary1 = 2047;
 struct FusedArgs {
   const float* logits;       // [T, E]
   const __nv_bfloat16* x;    // [T, H]
@@ -219,99 +213,6 @@ __host__ __device__ inline NatSmem nat_smem(int E, int K) {
   off += 4 * kFusedMaxSlots * 4;
   m.total = off;
   return m;
-}
-
-MOE_DEVINL void tmem_st_32x8(uint32_t taddr, const uint32_t (&r)[8]) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), "r"(r[0]), "r"(r[1]),
-               "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
-               : "memory");
-}
-MOE_DEVINL void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-// D[tmem] (+)= A[smem, E2M1] * B[smem, E2M1]^T, K = 64, two UE8M0 block scales per row held in tensor memory
-MOE_DEVINL void umma_mxf4(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t sfa, uint32_t sfb,
-                          uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-      :
-      : "r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
-      : "memory");
-}
-// instruction descriptor: A and B E2M1, UE8M0 scales, M = 128, N = 256; `half` (0 or 1) picks bytes 0,1 or 2,3 of
-// the scale words
-MOE_DEVINL uint32_t idesc_mxf4(uint32_t half) {
-  return (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24) | ((2u * half) << 29) | ((2u * half) << 4);
-}
-
-// Bounded wait until *p >= need (acquire at GPU scope); same give-up rules as mbar_wait
-MOE_DEVINL void counter_wait_ge(const int* p, int need, int* status) {
-  const long long t0 = clock64();
-  int spins = 0;
-  while (true) {
-    int v;
-    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    if (v >= need) return;
-    const long long waited = clock64() - t0;
-    if (waited > kWaitLimitCycles) {
-      if (status != nullptr) atomicExch(status, static_cast<int>(MOE_ERR_TIMEOUT));
-      return;
-    }
-    if (((++spins) & 63) == 0 && waited > 2000000 && status != nullptr && *reinterpret_cast<volatile int*>(status) != 0) return;
-    __nanosleep(64);
-  }
-}
-// orders this thread's generic-proxy accesses with its asynchronous-proxy (TMA) accesses, global memory included
-MOE_DEVINL void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
-MOE_DEVINL void prefetch_tmap(const void* tmap) { asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory"); }
-
-MOE_DEVINL float pow2f(int e) { return __uint_as_float(static_cast<uint32_t>(e + 127) << 23); }  // e in [-126, 127]
-// Block exponent of a term: the smallest s with amax <= 6 * 2^s (amax > 0), kept inside the UE8M0 range
-MOE_DEVINL int term_exp(float amax) {
-  const uint32_t u = __float_as_uint(amax);
-  const int e = static_cast<int>((u >> 23) & 0xFFu) - 127;
-  const int s = ((u & 0x7FFFFFu) <= 0x400000u) ? e - 2 : e - 1;  // 1.5 * 2^e = 6 * 2^(e-2)
-  return max(-126, min(s, 126));
-}
-// Two values (already divided by the block scale) -> one byte of two E2M1 codes (a in the low nibble) and their
-// decoded values
-MOE_DEVINL uint32_t e2m1_pair(float a, float b, float* qa, float* qb) {
-  const __nv_fp4x2_storage_t c = __nv_cvt_float2_to_fp4x2(make_float2(a, b), __NV_E2M1, cudaRoundNearest);
-  const __half2_raw h = __nv_cvt_fp4x2_to_halfraw2(c, __NV_E2M1);
-  const float2 q = __half22float2(*reinterpret_cast<const __half2*>(&h));
-  *qa = q.x;
-  *qb = q.y;
-  return static_cast<uint32_t>(c);
-}
-
-
-// Eight threads (consecutive lanes) share one 32-element block, four consecutive values each: the 8-term split,
-// for NB independent blocks at once (their dependency chains interleave).  `store(nb, t, bytes, se)` receives
-// term t's two bytes of codes (values 0,1 and 2,3 of this thread) and the block exponent.  All 32 lanes must call
-// it together.
-template <int NB, typename Store>
-MOE_DEVINL void split_terms(float (&r)[NB][4], Store store) {
-#pragma unroll 1
-  for (int t = 0; t < kTerms; ++t) {
-#pragma unroll
-    for (int nb = 0; nb < NB; ++nb) {
-      float amax = fmaxf(fmaxf(fabsf(r[nb][0]), fabsf(r[nb][1])), fmaxf(fabsf(r[nb][2]), fabsf(r[nb][3])));
-      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
-      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
-      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 4));
-      const int se = (amax > 0.0f) ? term_exp(amax) : 0;
-      const float inv = pow2f(-se), sc = pow2f(se);
-      float q0, q1, q2, q3;
-      const uint32_t bytes =
-          e2m1_pair(r[nb][0] * inv, r[nb][1] * inv, &q0, &q1) | (e2m1_pair(r[nb][2] * inv, r[nb][3] * inv, &q2, &q3) << 8);
-      r[nb][0] = fmaf(-q0, sc, r[nb][0]);
-      r[nb][1] = fmaf(-q1, sc, r[nb][1]);
-      r[nb][2] = fmaf(-q2, sc, r[nb][2]);
-      r[nb][3] = fmaf(-q3, sc, r[nb][3]);
-      store(nb, t, bytes, se);
-    }
-  }
 }
 
 }  // namespace
@@ -1073,8 +974,12 @@ bool nat_attr_once() {
 }
 }  // namespace
 
-namespace {
-// tensor maps of the weights and their scale bytes, in either layout
+// byte tensor [rows][row_bytes] with a 128-byte-swizzled box of [box_rows][128 bytes] (declared in moe_tmap.cuh)
+bool term_row_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint64_t rows, uint32_t box_rows) {
+  return nat_map(m, base, row_bytes, rows, 128, box_rows, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+
+// tensor maps of the weights and their scale bytes, in either layout (declared in moe_tmap.cuh)
 bool weight_maps(const ExpertWeights& w, const moe_shape_t& sh, CUtensorMap* tm_w13, CUtensorMap* tm_s13, CUtensorMap* tm_w2,
                  CUtensorMap* tm_s2) {
   const uint64_t r13 = static_cast<uint64_t>(sh.E) * 2 * sh.I, r2 = static_cast<uint64_t>(sh.E) * sh.H;
@@ -1088,7 +993,6 @@ bool weight_maps(const ExpertWeights& w, const moe_shape_t& sh, CUtensorMap* tm_
          nat_map(tm_s13, w.s13, sh.H / 32, r13, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE) &&
          nat_map(tm_s2, w.s2, sh.I / 32, r2, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
 }
-}  // namespace
 
 bool native_shape_ok(const moe_shape_t& sh, const void* w13, const void* w2) {
   return native_batch_ok(sh) && sh.H <= kMaxK && sh.I <= kMaxK && sh.H % 512 == 0 && sh.I % 512 == 0 &&

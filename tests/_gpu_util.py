@@ -74,3 +74,17 @@ def check_y(got, ref, what=""):
     mx = np.abs(got - ref).max() / max(rms, 1e-30)
     assert rel <= 5e-4 and mx <= 2e-2, "%s: y_perm rel %g max/rms %g" % (what, rel, mx)
     return dict(rel=rel, max_over_rms=float(mx))
+
+
+def assert_same_up_to_rounding(got_bits, want_bits, what=""):
+    """Two bf16 results of the same arithmetic up to the summation order inside fp32 dot products: the fp32 values
+    differ in their last bits, so the bf16 roundings agree except where a value sits on a rounding boundary - there
+    by one bf16 unit in the last place, in a small fraction of the elements."""
+    a = np.ascontiguousarray(got_bits, dtype=np.uint16).astype(np.int32)
+    b = np.ascontiguousarray(want_bits, dtype=np.uint16).astype(np.int32)
+    # order-preserving integer of a bf16 bit pattern: distance 1 = neighbouring values (also across zero)
+    ka = np.where(a & 0x8000, -(a & 0x7FFF), a & 0x7FFF)
+    kb = np.where(b & 0x8000, -(b & 0x7FFF), b & 0x7FFF)
+    d = np.abs(ka - kb)
+    assert d.max() <= 1, "%s: bf16 values %d units apart" % (what, int(d.max()))
+    assert (d != 0).mean() <= 0.05, "%s: %.3f of the elements differ" % (what, float((d != 0).mean()))
