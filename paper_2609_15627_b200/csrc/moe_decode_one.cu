@@ -17,7 +17,7 @@
 //     each multiplies the joint 256-wide slice - one 128-byte K step of the packed W2 rows, the same tiles and the same
 //     tensor maps as everywhere else - with half of the expert's H output rows.  The partial sums go to
 //     part[slot][p][H] (fp32, one store per element, no atomics).
-//   * The last H/256 CTAs each own 256 output columns: they wait until every partial of their half of the columns is
+//   * The last H/128 CTAs each own 128 output columns: they wait until every partial of their half of the columns is
 //     stored (one counter per half, release/acquire), sum the I/256 partials of every slot in ascending p, and combine
 //     the k slots in slot order with fma from zero - moe_combine's arithmetic - into the bf16 output row.  Every wait
 //     points to CTAs with a lower or equal index.
@@ -94,11 +94,13 @@ struct OneSmem {
 };
 // A operand of the gate/up projection: the token's 8 term rows of one K step, 4 copies (one per lane quadrant of the
 // accumulator, so that each epilogue warp finds the token in its own quadrant), fetched by TMA with every stage of the
-// weight ring.  Row 32 q + t of ring stage s sits at s * 1 KB + q * 4 KB + t * 128: the four stages interleave inside
-// one 16 KB operand span, each using the 8-row group the others leave empty.  The MMA of a stage reads 128 rows from
-// its own base (up to 3 KB past the span); rows it does not own hold other stages' data and feed accumulator lanes
-// nobody reads.
-__host__ __device__ inline uint32_t a1_bytes(int) { return kATile + 4096; }
+// weight ring.  Row 32 q + t of ring stage s sits at (s / 4) * 16 KB + (s % 4) * 1 KB + q * 4 KB + t * 128: four stages
+// interleave inside one 16 KB operand span, each using the 8-row group the others leave empty.  The MMA of a stage
+// reads 128 rows from its own base (up to 3 KB past the span); rows it does not own hold other stages' data and feed
+// accumulator lanes nobody reads.
+__host__ __device__ inline uint32_t a1_slot(int s) { return static_cast<uint32_t>((s >> 2) * kATile + (s & 3) * 1024); }
+__host__ __device__ inline uint32_t a1_bytes(int) { return static_cast<uint32_t>((kWStages + 3) / 4) * kATile + 4096; }
+constexpr int kA2Bytes = 2048;  // B operand of the down projection: the 8 term rows of one K step (N = 16 reads 16 rows)
 __host__ __device__ inline OneSmem one_smem(int E, int H) {
   OneSmem m;
   uint32_t off = 0;
@@ -106,8 +108,8 @@ __host__ __device__ inline OneSmem one_smem(int E, int H) {
   off += kWStages * kWStage;
   m.a1 = off;
   off += a1_bytes(H);
-  m.a2 = off;  // A operand of the down projection: one K step, rows 32 q + t at q * 4 KB + t * 128
-  off += kATile;
+  m.a2 = off;  // the term rows of the pair's slice of the intermediate, row t at t * 128 (1024-byte aligned)
+  off += kA2Bytes;
   m.sc = off;
   off += kScStages * kScStage;
   m.sf2 = off;  // scale bytes of the intermediate's term rows for the pair's K step [8][8]
@@ -181,7 +183,6 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   const int n_ks0 = a.H / 256;           // K steps of the gate/up projection
   const int npp = a.I / 256;             // K steps of the down projection = pairs of CTAs per slot
   const int n_t1 = a.H / 512;            // 256-row tiles of the down projection per CTA (half of the H rows)
-  const int nct = a.H / 256;             // column tiles of the output, one reducing CTA each
   const int item = static_cast<int>(blockIdx.x);
   const bool has_item = item < a.k * tiles0;
   const int slot = item / tiles0, tile = item % tiles0;
@@ -305,7 +306,7 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             }
 #pragma unroll
             for (int qq = 0; qq < 4; ++qq)
-              tma_load_2d(sA1 + s * 1024 + qq * 4096, &tmap_a1, ks * 128, (item % kCopies) * kTerms, &full_w[s]);
+              tma_load_2d(sA1 + a1_slot(s) + qq * 4096, &tmap_a1, ks * 128, (item % kCopies) * kTerms, &full_w[s]);
           }
           if (++s == kWStages) { s = 0; ph ^= 1u; }
         }
@@ -328,7 +329,7 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         tc_fence_after_sync();
         if (ks == 0) MOE_TP(7);
         const uint32_t w_addr = smem_u32(sW + s * kWStage);
-        const uint32_t a_addr = smem_u32(sA1) + static_cast<uint32_t>(s * 1024);
+        const uint32_t a_addr = smem_u32(sA1) + a1_slot(s);
 #pragma unroll
         for (uint32_t j = 0; j < 4; ++j) {  // K = 64 each; scale word (ks & 1) * 2 + j / 2 of the group, half j & 1
           const uint32_t sf_act = tmem_base + kColSfAct + static_cast<uint32_t>(ks * 8) + (j >> 1) * 4;
@@ -345,31 +346,36 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       }
       umma_commit(&acc_full[0]);
       MOE_TP(8);
-      // ---- down: a single K step per 256-row tile, one accumulator (the instruction takes the same time for 128 weight
-      // rows as for 256, so two alternating half-width accumulators cost twice the tensor-core time) ----
+      // ---- down: a single K step.  The operands change places: the 128 weight rows of a sub-tile are the M side, the
+      // 8 term rows of the pair's slice the N side (N = 16, the smallest; its upper 8 rows are never looked at), so the
+      // accumulator of a sub-tile is 16 columns and those of all H/256 sub-tiles of this CTA sit side by side in the
+      // 256 columns: no accumulator is handed back and forth with the epilogue, which reads them all once at the end ----
       mbar_wait(act_ready, 1u, a.status);
+      mbar_wait(&acc_empty[0], 0u, a.status);  // the gate/up accumulator has been read
       tc_fence_after_sync();
       MOE_TP(9);
       const uint32_t a2_addr = smem_u32(sA2);
       for (int n = 0; n < n_t1; ++n) {
         mbar_wait(&sf_full[slotg], sph, a.status);
         mbar_wait(&full_w[s], ph, a.status);
-        mbar_wait(&acc_empty[0], static_cast<uint32_t>(n & 1), a.status);  // the previous accumulator has been read
         tc_fence_after_sync();
-        const uint32_t w_addr = smem_u32(sW + s * kWStage);
 #pragma unroll
-        for (uint32_t j = 0; j < 4; ++j) {
-          const uint32_t sf_act = tmem_base + kColSfAct + (j >> 1) * 4;
-          const uint32_t sf_w = tmem_base + kColSfW + static_cast<uint32_t>(slotg * 32 + ((pp & 1) * 2 + static_cast<int>(j >> 1)) * 8);
-          umma_mxf4(d_addr, umma_desc_k_sw128(a2_addr + j * 32), umma_desc_k_sw128(w_addr + j * 32), idesc_mxf4(j & 1u), sf_act, sf_w,
-                    j != 0 ? 1u : 0u);
+        for (uint32_t b = 0; b < 2; ++b) {
+          const uint32_t w_addr = smem_u32(sW + s * kWStage) + b * (128u * 128u);
+#pragma unroll
+          for (uint32_t j = 0; j < 4; ++j) {
+            const uint32_t sf_act = tmem_base + kColSfAct + (j >> 1) * 4;
+            const uint32_t sf_w = tmem_base + kColSfW + static_cast<uint32_t>(slotg * 32 + ((pp & 1) * 2 + static_cast<int>(j >> 1)) * 8) + b * 4;
+            umma_mxf4(d_addr + static_cast<uint32_t>(2 * n) * 16u + b * 16u, umma_desc_k_sw128(w_addr + j * 32),
+                      umma_desc_k_sw128(a2_addr + j * 32), idesc_mxf4(j & 1u, 16u), sf_w, sf_act, j != 0 ? 1u : 0u);
+          }
         }
-        umma_commit(&acc_full[0]);
         umma_commit(&empty_w[s]);
         umma_commit(&sf_free[slotg]);
         if (++s == kWStages) { s = 0; ph ^= 1u; }
         if (++slotg == kSfGroups) { slotg = 0; sph ^= 1u; }
       }
+      umma_commit(&acc_full[0]);
       MOE_TP(10);
     }
   } else {
@@ -554,7 +560,7 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         {
           // SwiGLU, bf16 rounding (the intermediate is defined as a bf16 value) and the 8-term split of this warp's block
           // of 32: block q of this CTA's four = 16-byte chunk rank * 4 + q of the pair's 128-byte K step.  The rows go
-          // to this CTA's operand and to the partner's, four copies each.
+          // to this CTA's operand and to the partner's.
           float r[1][4];
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
@@ -565,11 +571,8 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
           split_terms<1>(r, [&](int, int t, uint32_t bytes, int se) {
             if (live) {
               const uint32_t off = static_cast<uint32_t>(t * 128) + ((chunk ^ static_cast<uint32_t>(t)) << 4) + static_cast<uint32_t>(cb >> 1);
-#pragma unroll
-              for (int qq = 0; qq < 4; ++qq) {
-                asm volatile("st.shared.u16 [%0], %1;" ::"r"(sA2_u + off + qq * 4096), "h"(static_cast<unsigned short>(bytes)) : "memory");
-                st_cluster_u16(peer_a2 + off + qq * 4096, bytes);
-              }
+              asm volatile("st.shared.u16 [%0], %1;" ::"r"(sA2_u + off), "h"(static_cast<unsigned short>(bytes)) : "memory");
+              st_cluster_u16(peer_a2 + off, bytes);
               if (tl == 0) {
                 sSf2[t * 8 + static_cast<int>(chunk)] = static_cast<uint8_t>(se + 127);
                 st_cluster_u8(peer_sf2 + static_cast<uint32_t>(t * 8) + chunk, static_cast<uint32_t>(se + 127));
@@ -597,27 +600,24 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             if (lane == 0) mbar_arrive(act_ready);
           }
         }
-        // ---- down accumulators: chunks 2q and 2q + 1 of each 256-row tile -> partial sums ----
-        for (int n = 0; n < (dry ? 1 : n_t1); ++n) {
-          if (!dry) mbar_wait(&acc_full[0], static_cast<uint32_t>((n + 1) & 1), a.status);
-          __syncwarp();
-          tc_fence_after_sync();
-          uint32_t v0[32], v1[32];
-          tmem_ld_32x32(tmem_base + lane_base + kColD + static_cast<uint32_t>(64 * q), v0);
-          tmem_ld_32x32(tmem_base + lane_base + kColD + static_cast<uint32_t>(64 * q + 32), v1);
+        // ---- down accumulators, all sub-tiles at once: lane = weight row of the sub-tile, 16 columns per sub-tile of
+        // which the first 8 are the 8 terms; their sum, in ascending term order, is the row's partial sum ----
+        if (!dry) mbar_wait(&acc_full[0], 1u, a.status);
+        __syncwarp();
+        tc_fence_after_sync();
+        for (int u0 = 0; u0 < (dry ? 2 : 2 * n_t1); u0 += 2) {  // two sub-tiles (32 columns) per load
+          uint32_t v[32];
+          tmem_ld_32x32(tmem_base + lane_base + kColD + static_cast<uint32_t>(u0 * 16), v);
           tmem_ld_wait();
-          tc_fence_before_sync();
-          __syncwarp();
-          if (!dry && lane == 0) mbar_arrive(&acc_empty[0]);  // the sums and the stores overlap the next tile's MMAs
-          float o0[4], o1[4];
-          reduce8(v0, o0);
-          reduce8(v1, o1);
-          if (!dry && jl == 0) {
-            float* dst = prow + n * kTile + 64 * q + cb;
-            *reinterpret_cast<float4*>(dst) = make_float4(o0[0], o0[1], o0[2], o0[3]);
-            *reinterpret_cast<float4*>(dst + 32) = make_float4(o1[0], o1[1], o1[2], o1[3]);
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            float sum = __uint_as_float(v[16 * h]);
+#pragma unroll
+            for (int t = 1; t < kTerms; ++t) sum = __fadd_rn(sum, __uint_as_float(v[16 * h + t]));
+            if (!dry) prow[(u0 + h) * 128 + 32 * q + lane] = sum;
           }
         }
+        tc_fence_before_sync();
         if (!dry) {
           // one release for all of this warp's stores (a release per tile would wait a memory round trip each time),
           // counted for this CTA's half of the output columns
@@ -635,55 +635,48 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   __syncthreads();
   if (!skip && !(has_item && wid >= 6)) cluster_wait();
 
-  // ---- reduction: the last nct CTAs own one column tile each ----
-  const int ct = item - (grid - nct);
+  // ---- reduction: the last H/128 CTAs own 128 output columns each ----
+  constexpr int kRedCols = 128;
+  const int n_red = a.H / kRedCols;
+  const int ct = item - (grid - n_red);
   // y_j[n] = sum over p ascending of part[j][p][n]; out[n] = bf16(fma chain over j = 0..k-1 from zero)
   auto reduce_tile = [&](const bool dry) {
-    float* ys = reinterpret_cast<float*>(sW);  // [k][256], the ring is idle by now
-    const int cg = tid & 63, grp = tid >> 6;   // 64 groups of 4 columns; 4 thread groups (256 threads) share the slots
-    if (grp < 4) {
-      for (int j0 = grp; j0 < a.k; j0 += 8) {  // two slots at a time: 2 * npp independent 16-byte loads in flight
-        float4 acc0 = make_float4(0.f, 0.f, 0.f, 0.f), acc1 = acc0;
-        const int j1 = j0 + 4;
-        const float* p0 = a.part + static_cast<size_t>(j0) * npp * a.H + ct * kTile + cg * 4;
-        const float* p1 = a.part + static_cast<size_t>(j1 < a.k ? j1 : j0) * npp * a.H + ct * kTile + cg * 4;
-        for (int p = 0; p < npp; p += 4) {
-          float4 v0[4], v1[4];
+    float* ys = reinterpret_cast<float*>(sW);  // [k][128], the ring is idle by now
+    const int cg = tid & 31, grp = tid >> 5;   // 32 groups of 4 columns; warp j sums the partials of slot j, j + 8, ...
+    if (grp < 8) {
+      for (int j = grp; j < a.k; j += 8) {
+        const float* p0 = a.part + static_cast<size_t>(j) * npp * a.H + ct * kRedCols + cg * 4;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int p = 0; p < npp; p += 8) {  // eight independent 16-byte loads in flight
+          float4 v[8];
 #pragma unroll
-          for (int u = 0; u < 4; ++u)
-            if (p + u < npp) {
-              v0[u] = __ldcg(reinterpret_cast<const float4*>(p0 + static_cast<size_t>(p + u) * a.H));
-              v1[u] = __ldcg(reinterpret_cast<const float4*>(p1 + static_cast<size_t>(p + u) * a.H));
-            }
+          for (int u = 0; u < 8; ++u)
+            if (p + u < npp) v[u] = __ldcg(reinterpret_cast<const float4*>(p0 + static_cast<size_t>(p + u) * a.H));
 #pragma unroll
-          for (int u = 0; u < 4; ++u)
+          for (int u = 0; u < 8; ++u)
             if (p + u < npp) {
               if (p + u == 0) {
-                acc0 = v0[u];
-                acc1 = v1[u];
+                acc = v[u];
               } else {
-                acc0.x = __fadd_rn(acc0.x, v0[u].x); acc0.y = __fadd_rn(acc0.y, v0[u].y);
-                acc0.z = __fadd_rn(acc0.z, v0[u].z); acc0.w = __fadd_rn(acc0.w, v0[u].w);
-                acc1.x = __fadd_rn(acc1.x, v1[u].x); acc1.y = __fadd_rn(acc1.y, v1[u].y);
-                acc1.z = __fadd_rn(acc1.z, v1[u].z); acc1.w = __fadd_rn(acc1.w, v1[u].w);
+                acc.x = __fadd_rn(acc.x, v[u].x); acc.y = __fadd_rn(acc.y, v[u].y);
+                acc.z = __fadd_rn(acc.z, v[u].z); acc.w = __fadd_rn(acc.w, v[u].w);
               }
             }
         }
-        *reinterpret_cast<float4*>(ys + j0 * kTile + cg * 4) = acc0;
-        if (j1 < a.k) *reinterpret_cast<float4*>(ys + j1 * kTile + cg * 4) = acc1;
+        *reinterpret_cast<float4*>(ys + j * kRedCols + cg * 4) = acc;
       }
     }
     __syncthreads();
-    if (tid < 128) {
+    if (tid < kRedCols / 2) {
       const int col = tid * 2;
       float2 acc = make_float2(0.0f, 0.0f);
       for (int j = 0; j < a.k; ++j) {
         const float wj = s_w[j];
-        const float2 v = *reinterpret_cast<const float2*>(ys + j * kTile + col);
+        const float2 v = *reinterpret_cast<const float2*>(ys + j * kRedCols + col);
         acc.x = __fmaf_rn(wj, v.x, acc.x);
         acc.y = __fmaf_rn(wj, v.y, acc.y);
       }
-      if (!dry) *reinterpret_cast<__nv_bfloat162*>(a.out + ct * kTile + col) = __floats2bfloat162_rn(acc.x, acc.y);
+      if (!dry) *reinterpret_cast<__nv_bfloat162*>(a.out + ct * kRedCols + col) = __floats2bfloat162_rn(acc.x, acc.y);
     }
     __syncthreads();
   };
@@ -691,7 +684,7 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     if (ct >= 0) {
       reduce_tile(true);  // once on whatever the buffer holds, no store: the code is then in place when the count completes
       if (tid == 0) {
-        counter_wait_ge(a.sync + kSyncDone2 + ct / n_t1, 4 * a.k * npp, a.status);  // the half its columns are in
+        counter_wait_ge(a.sync + kSyncDone2 + (2 * ct) / n_red, 4 * a.k * npp, a.status);  // the half its columns are in
         MOE_TP(17);
       }
       __syncthreads();
@@ -731,7 +724,7 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
 bool decode_one_ok(const moe_shape_t& sh, const void* w13, const void* w2) {
   const int grid = sm_count() & ~1;
   return sh.T == 1 && sh.H % 512 == 0 && sh.I % 512 == 0 && sh.H <= 4096 && sh.I <= 4096 && sh.k <= 32 &&
-         sh.k * (sh.I / 128) <= grid && sh.H / 32 <= grid && sh.H / 256 <= kSyncExit - kSyncDone2 &&
+         sh.k * (sh.I / 128) <= grid && sh.H / 32 <= grid && sh.H / 128 <= grid && sh.H / 256 <= kSyncExit - kSyncDone2 &&
          (reinterpret_cast<uintptr_t>(w13) & 15u) == 0 && (reinterpret_cast<uintptr_t>(w2) & 15u) == 0 &&
          one_smem(sh.E, sh.H).total + 1024 <= 227 * 1024;
 }

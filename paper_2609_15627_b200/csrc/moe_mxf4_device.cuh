@@ -79,7 +79,7 @@ MOE_DEVINL uint32_t e2m1_pair(float a, float b, float* qa, float* qb) {
 // Eight threads (consecutive lanes) share one 32-element block, four consecutive values each: the 8-term split,
 // for NB independent blocks at once (their dependency chains interleave).  `store(nb, t, bytes, se)` receives
 // term t's two bytes of codes (values 0,1 and 2,3 of this thread) and the block exponent.  All 32 lanes must call
-// it together.
+// it together.  (With NB > 1 the chains overlap little: the exchanges and the stores keep their program order.)
 template <int NB, typename Store>
 MOE_DEVINL void split_terms(float (&r)[NB][4], Store store) {
 #pragma unroll 1
@@ -103,6 +103,5 @@ MOE_DEVINL void split_terms(float (&r)[NB][4], Store store) {
     }
   }
 }
-
 
 }  // namespace moe

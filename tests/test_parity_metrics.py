@@ -69,3 +69,22 @@ def test_check_out_and_check_y_enforce_the_frobenius_bounds():
     check_y(y * np.float32(1 + 1e-5), y, "close")
     with pytest.raises(AssertionError):
         check_y(y * np.float32(1 + 1e-3), y, "rel 1e-3 > 5e-4")
+
+
+def test_same_up_to_rounding_allows_one_unit_and_cancelled_values_only():
+    from _gpu_util import assert_same_up_to_rounding
+    rng = np.random.default_rng(3)
+    want = _bits((rng.standard_normal(4096) * 8).astype(np.float32))
+    got = want.copy()
+    got[5] += 1                                     # one unit up
+    got[9] = _bits(np.float32(3e-4)); want[9] = _bits(np.float32(1e-4))   # cancelled to almost nothing: many units, tiny difference
+    assert_same_up_to_rounding(got, want, "ok")
+    bad = want.copy()
+    bad[7] += 2                                     # two units at an ordinary magnitude
+    if abs(float(inputs.bf16_bits_to_f32(want[7:8])[0])) > 1.0:
+        with pytest.raises(AssertionError):
+            assert_same_up_to_rounding(bad, want, "two units")
+    many = want.copy()
+    many[:400] ^= 1                                 # every tenth element off by one unit: too many
+    with pytest.raises(AssertionError):
+        assert_same_up_to_rounding(many, want, "many")
