@@ -291,6 +291,46 @@ void oracle_combine(const float* y_perm, const int32_t* inv_perm, const float* w
   }
 }
 
+// ---- the steps either side of the routed path (figure "Execution structure": router scores before the Top-k, the
+// shared expert beside the routed experts, "add partials" after them) ----
+
+// Router projection: logits[t,e] = sum over h ascending of x[t,h] * w_router[e,h], both bf16, accumulated in fp32
+// (each product of two bf16 values is exact in fp32; only the running sum rounds).  The paper kept a vendor BLAS for
+// this step and states no precision; fp32 accumulation of exact products is the reading taken.
+void oracle_router_logits(const uint16_t* x, const uint16_t* w_router, int T, int H, int E, float* logits) {
+#pragma omp parallel for schedule(static)
+  for (int t = 0; t < T; ++t) {
+    for (int e = 0; e < E; ++e) {
+      float acc = 0.0f;
+      for (int h = 0; h < H; ++h) {
+        const float prod = bf16_to_f32(x[static_cast<int64_t>(t) * H + h]) * bf16_to_f32(w_router[static_cast<int64_t>(e) * H + h]);
+        acc = acc + prod;
+      }
+      logits[static_cast<int64_t>(t) * E + e] = acc;
+    }
+  }
+}
+
+// The join: the routed experts' slot-ordered fp32 sum (exactly oracle_combine's recurrence) plus the shared expert's
+// fp32 row, one fp32 addition, then one rounding to bf16.  y_shared[t,:] is the shared expert's down projection of
+// token t (the same expert arithmetic as a routed expert, applied to every token with weight 1).
+void oracle_combine_shared(const float* y_perm, const int32_t* inv_perm, const float* w, const float* y_shared, int T,
+                           int H, int k, uint16_t* out_bf16, float* out_f32) {
+#pragma omp parallel for schedule(static)
+  for (int t = 0; t < T; ++t) {
+    for (int n = 0; n < H; ++n) {
+      float acc = 0.0f;
+      for (int j = 0; j < k; ++j) {
+        const int64_t p = inv_perm[static_cast<int64_t>(t) * k + j];
+        acc = std::fmaf(w[static_cast<int64_t>(t) * k + j], y_perm[p * H + n], acc);
+      }
+      acc = acc + y_shared[static_cast<int64_t>(t) * H + n];
+      out_bf16[static_cast<int64_t>(t) * H + n] = f32_to_bf16(acc);
+      if (out_f32 != nullptr) out_f32[static_cast<int64_t>(t) * H + n] = acc;
+    }
+  }
+}
+
 // The layer by its per-token definition, with no permutation at all: for each
 // listed token route it, evaluate its k experts and reduce in slot order.
 // Outputs are indexed by position in `tokens`.  y_slots (may be NULL) receives

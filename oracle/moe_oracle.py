@@ -181,3 +181,46 @@ def forward_tokens(logits, x, w13, s13, w2, s2, k, tokens, acc64=False):
     lib().oracle_forward_tokens(_p(logits), _p(x), _p(w13), _p(s13), _p(w2), _p(s2), T, H, I, E, k,
                                 int(bool(acc64)), _p(tokens), n, _p(ids), _p(w), _p(act), _p(y), _p(out), _p(out_f32))
     return dict(ids=ids, w=w, act=act, y=y, out=out, out_f32=out_f32)
+
+
+# ---- the steps either side of the routed path: router projection, shared expert, join ----------------------
+
+def router_logits(x, w_router):
+    """logits[T,E] float32 = x[T,H] (bf16 bits) times w_router[E,H] (bf16 bits) transposed, fp32 accumulation, h ascending."""
+    T, H = x.shape
+    E = w_router.shape[0]
+    _chk(x, np.uint16)
+    _chk(w_router, np.uint16, (E, H))
+    logits = np.empty((T, E), np.float32)
+    lib().oracle_router_logits(_p(x), _p(w_router), T, H, E, _p(logits))
+    return logits
+
+
+def combine_shared(y_perm, inv_perm, w, y_shared):
+    S, H = y_perm.shape
+    T, k = w.shape
+    _chk(y_perm, np.float32)
+    _chk(inv_perm, np.int32, (S,))
+    _chk(w, np.float32)
+    _chk(y_shared, np.float32, (T, H))
+    out = np.empty((T, H), np.uint16)
+    out_f32 = np.empty((T, H), np.float32)
+    lib().oracle_combine_shared(_p(y_perm), _p(inv_perm), _p(w), _p(y_shared), T, H, k, _p(out), _p(out_f32))
+    return out, out_f32
+
+
+def shared_expert(x, sw13, ss13, sw2, ss2):
+    """The shared expert on every token: one expert in the routed experts' weight format (tensors with E = 1), weight 1."""
+    T = x.shape[0]
+    return expert_ffn(x, np.array([0, T], np.int32), sw13, ss13, sw2, ss2, 1)
+
+
+def ffn_block(x, w_router, w13, s13, w2, s2, sw13, ss13, sw2, ss2, k, logits=None):
+    """Router projection -> Top-k -> routed experts, beside the shared expert -> join.  `logits`: use these instead of
+    the oracle's own router projection (to compare the steps after it on logits computed elsewhere)."""
+    lg = router_logits(x, w_router) if logits is None else logits
+    r = forward_staged(lg, x, w13, s13, w2, s2, k)
+    y_shared = shared_expert(x, sw13, ss13, sw2, ss2)
+    out, out_f32 = combine_shared(r["y_perm"], r["inv_perm"], r["w"], y_shared)
+    r.update(logits=lg, y_shared=y_shared, routed_out=r["out"], routed_out_f32=r["out_f32"], out=out, out_f32=out_f32)
+    return r
