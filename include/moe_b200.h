@@ -230,6 +230,35 @@ int moe_forward_host_packed(const float* logits_host, const void* x_host_bf16, c
                             size_t ws_bytes, void* cuda_stream);
 
 /*
+ * The steps either side of the routed path (paper, figure "Execution structure": router scores before the Top-k; the
+ * shared expert beside the routed experts; "add partials" after them), and the FFN block they make with it.
+ *
+ *   - moe_router_logits: logits[t,e] = sum_h x[t,h] * w_router[e,h]; x [T,H] and w_router [E,H] bf16, fp32
+ *     accumulation (each product is exact in fp32; the order of the sum is the kernel's), logits [T,E] fp32.  The paper
+ *     states no precision for this step (it kept a vendor BLAS).  H a multiple of 128, E <= 1024.  Up to 16 tokens: one
+ *     warp per expert streams w_router once; more: a tcgen05 GEMM on tiles of 128 tokens x 64 experts.
+ *   - The shared expert is one more expert in the routed experts' weight format, applied to every token with weight 1:
+ *     tensors shaped as the routed ones with E = 1.  It needs no entry point of its own: moe_expert_ffn with x as
+ *     x_perm, offsets {0, T} and shape {T, H, I, 1, 1} gives y_shared [T,H] fp32.
+ *   - moe_combine_shared: out[t,n] = bf16_rne( acc_k + y_shared[t,n] ), acc as in moe_combine (fma over the slots in slot
+ *     order from zero), then one fp32 addition, then one rounding.
+ *   - moe_ffn_block: router projection -> moe_route -> moe_permute -> moe_expert_ffn (routed) -> moe_expert_ffn (shared)
+ *     -> moe_combine_shared on DEVICE buffers, every intermediate in `ws` (moe_ffn_block_workspace_bytes(), 256-byte
+ *     aligned, no initialisation needed).  topk_ids / topk_w [T,k] receive the routing where not NULL.  Enqueue only,
+ *     no allocation, capturable, bounded device-side waits.
+ */
+int moe_router_logits(const void* x_bf16 /* [T,H] */, const void* w_router_bf16 /* [E,H] */, int32_t T, int32_t H, int32_t E,
+                      float* logits /* [T,E] */, int32_t* status_word, void* cuda_stream);
+int moe_combine_shared(const float* y_perm, const int32_t* inv_perm, const float* topk_w, const float* y_shared /* [T,H] */,
+                       const moe_shape_t* shape, void* out_bf16 /* [T,H] */, void* cuda_stream);
+size_t moe_ffn_block_workspace_bytes(const moe_shape_t* shape);
+int moe_ffn_block(const void* x_bf16 /* [T,H] */, const void* w_router_bf16 /* [E,H] */, const uint8_t* w13,
+                  const uint8_t* w13_scale, const uint8_t* w2, const uint8_t* w2_scale, const uint8_t* shared_w13 /* [1,2I,H/2] */,
+                  const uint8_t* shared_w13_scale, const uint8_t* shared_w2 /* [1,H,I/2] */, const uint8_t* shared_w2_scale,
+                  const moe_shape_t* shape, void* out_bf16 /* [T,H] */, int32_t* topk_ids /* [T,k] or NULL */,
+                  float* topk_w /* [T,k] or NULL */, int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * moe_expert_ffn without a workspace argument, for callers that cannot allocate device memory
  * (the paper has no counterpart: this is a packaging variant of moe_expert_ffn, same arithmetic).
  *

@@ -224,6 +224,114 @@ int moe_combine(const float* y_perm, const int32_t* inv_perm, const float* topk_
                         static_cast<cudaStream_t>(cuda_stream));
 }
 
+// ---- router projection, shared expert, join: the whole FFN block ---------------------------------------------
+int moe_router_logits(const void* x_bf16, const void* w_router_bf16, int32_t T, int32_t H, int32_t E, float* logits,
+                      int32_t* status_word, void* cuda_stream) {
+  if (T < 1 || H < 1 || E < 1) return MOE_ERR_INVALID_ARG;
+  if (H % 128 != 0 || E > 1024) return MOE_ERR_UNSUPPORTED_SHAPE;
+  if (!aligned(x_bf16, 16) || !aligned(w_router_bf16, 16) || !aligned(logits, 16) ||
+      (status_word != nullptr && !aligned(status_word, 4)))
+    return MOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  StatusRef status;
+  int rc = resolve_status(status_word, &status);
+  if (rc != MOE_OK) return rc;
+  if ((rc = clear_own_status(status, st)) != MOE_OK) return rc;
+  return launch_router_logits(static_cast<const __nv_bfloat16*>(x_bf16), static_cast<const __nv_bfloat16*>(w_router_bf16), T, H, E,
+                              logits, status.word, st);
+}
+
+int moe_combine_shared(const float* y_perm, const int32_t* inv_perm, const float* topk_w, const float* y_shared,
+                       const moe_shape_t* shape, void* out_bf16, void* cuda_stream) {
+  const int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (!aligned(y_perm, 16) || !aligned(inv_perm, 16) || !aligned(topk_w, 16) || !aligned(y_shared, 16) || !aligned(out_bf16, 16))
+    return MOE_ERR_INVALID_ARG;
+  return launch_combine_shared(y_perm, inv_perm, topk_w, y_shared, *shape, static_cast<__nv_bfloat16*>(out_bf16),
+                               static_cast<cudaStream_t>(cuda_stream));
+}
+
+namespace {
+// ws of moe_ffn_block = [ logits | ids | w | offsets | shared offsets | x_perm | perm | inv_perm | y_perm | y_shared |
+//                         the expert-FFN calls' workspace (the routed call's and the shared call's, used one after the other) ]
+struct BlockLayout {
+  size_t logits, ids, w, offsets, offsets2, x_perm, perm, inv_perm, y_perm, y_shared, inner, inner_bytes, total;
+};
+moe_shape_t shared_shape(const moe_shape_t& s) { return moe_shape_t{s.T, s.H, s.I, 1, 1}; }
+BlockLayout block_layout(const moe_shape_t& s) {
+  BlockLayout L;
+  const size_t S = static_cast<size_t>(s.T) * s.k;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t o = off;
+    off += align_up(bytes, kAlign);
+    return o;
+  };
+  L.logits = take(static_cast<size_t>(s.T) * s.E * 4);
+  L.ids = take(S * 4);
+  L.w = take(S * 4);
+  L.offsets = take((static_cast<size_t>(s.E) + 1) * 4);
+  L.offsets2 = take(16);
+  L.x_perm = take(S * s.H * 2);
+  L.perm = take(S * 4);
+  L.inv_perm = take(S * 4);
+  L.y_perm = take(S * s.H * 4);
+  L.y_shared = take(static_cast<size_t>(s.T) * s.H * 4);
+  L.inner = off;
+  const size_t a = ws_layout(s).total, b = ws_layout(shared_shape(s)).total;
+  L.inner_bytes = a > b ? a : b;
+  off += L.inner_bytes;
+  L.total = off;
+  return L;
+}
+}  // namespace
+
+size_t moe_ffn_block_workspace_bytes(const moe_shape_t* shape) {
+  if (check_shape(shape) != MOE_OK) return 0;
+  return block_layout(*shape).total;
+}
+
+int moe_ffn_block(const void* x_bf16, const void* w_router_bf16, const uint8_t* w13, const uint8_t* w13_scale, const uint8_t* w2,
+                  const uint8_t* w2_scale, const uint8_t* shared_w13, const uint8_t* shared_w13_scale, const uint8_t* shared_w2,
+                  const uint8_t* shared_w2_scale, const moe_shape_t* shape, void* out_bf16, int32_t* topk_ids, float* topk_w,
+                  int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (!aligned(x_bf16, 16) || !aligned(w_router_bf16, 16) || !aligned(out_bf16, 16) || !aligned(shared_w13, 16) ||
+      !aligned(shared_w13_scale, 16) || !aligned(shared_w2, 16) || !aligned(shared_w2_scale, 16) ||
+      (topk_ids != nullptr && !aligned(topk_ids, 16)) || (topk_w != nullptr && !aligned(topk_w, 16)))
+    return MOE_ERR_INVALID_ARG;
+  const moe_shape_t& s = *shape;
+  const BlockLayout L = block_layout(s);
+  if (check_ws(ws, ws_bytes, L.total) != MOE_OK) return MOE_ERR_WORKSPACE;
+  char* base = static_cast<char*>(ws);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  float* d_logits = reinterpret_cast<float*>(base + L.logits);
+  int32_t* d_ids = topk_ids != nullptr ? topk_ids : reinterpret_cast<int32_t*>(base + L.ids);
+  float* d_w = topk_w != nullptr ? topk_w : reinterpret_cast<float*>(base + L.w);
+  int32_t* d_off = reinterpret_cast<int32_t*>(base + L.offsets);
+  int32_t* d_off2 = reinterpret_cast<int32_t*>(base + L.offsets2);
+  void* d_xp = base + L.x_perm;
+  int32_t* d_perm = reinterpret_cast<int32_t*>(base + L.perm);
+  int32_t* d_inv = reinterpret_cast<int32_t*>(base + L.inv_perm);
+  float* d_y = reinterpret_cast<float*>(base + L.y_perm);
+  float* d_ys = reinterpret_cast<float*>(base + L.y_shared);
+  void* inner = base + L.inner;
+  const moe_shape_t sh1 = shared_shape(s);
+  // router scores -> Top-k -> route production -> routed experts; the shared expert on every token (its sorted rows are
+  // the token rows themselves); the join
+  if ((rc = moe_router_logits(x_bf16, w_router_bf16, s.T, s.H, s.E, d_logits, status_word, st)) != MOE_OK) return rc;
+  if ((rc = launch_shared_offsets(d_off2, s.T, st)) != MOE_OK) return rc;
+  if ((rc = moe_route(d_logits, s.T, s.E, s.k, d_ids, d_w, d_off, inner, L.inner_bytes, st)) != MOE_OK) return rc;
+  if ((rc = moe_permute(x_bf16, d_ids, d_off, shape, d_xp, d_perm, d_inv, inner, L.inner_bytes, st)) != MOE_OK) return rc;
+  if ((rc = moe_expert_ffn(d_xp, d_off, w13, w13_scale, w2, w2_scale, shape, d_y, status_word, inner, L.inner_bytes, st)) != MOE_OK)
+    return rc;
+  if ((rc = moe_expert_ffn(x_bf16, d_off2, shared_w13, shared_w13_scale, shared_w2, shared_w2_scale, &sh1, d_ys, status_word, inner,
+                           L.inner_bytes, st)) != MOE_OK)
+    return rc;
+  return moe_combine_shared(d_y, d_inv, d_w, d_ys, shape, out_bf16, st);
+}
+
 int moe_validate_scales(const uint8_t* scales, size_t n_bytes, int32_t* bad_count, void* cuda_stream) {
   if (scales == nullptr || n_bytes == 0 || !aligned(bad_count, 4)) return MOE_ERR_INVALID_ARG;
   return launch_validate_scales(scales, n_bytes, bad_count, static_cast<cudaStream_t>(cuda_stream));

@@ -160,6 +160,13 @@ int launch_decode_one(const float* logits, const __nv_bfloat16* x, const ExpertW
                       __nv_bfloat16* out, int* ids_out, float* w_out, int* sync, void* scratch, StatusRef status,
                       cudaStream_t st);
 
+// router projection, join with the shared expert, and the shared expert's offsets {0, T} (moe_block.cu)
+int launch_router_logits(const __nv_bfloat16* x, const __nv_bfloat16* w_router, int T, int H, int E, float* logits, int* status,
+                         cudaStream_t st);
+int launch_combine_shared(const float* y_perm, const int* inv_perm, const float* w, const float* y_shared, const moe_shape_t& s,
+                          __nv_bfloat16* out, cudaStream_t st);
+int launch_shared_offsets(int* offsets2, int T, cudaStream_t st);
+
 int sm_count();  // of the current device
 
 // ---- per-device one-time set-up (host) ---------------------------------------------------------------

@@ -979,6 +979,18 @@ bool term_row_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint64_t
   return nat_map(m, base, row_bytes, rows, 128, box_rows, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
+// bf16 matrix [rows][inner], 128-byte-swizzled box of [box_rows][box_inner]; rows past the end read as zeros
+bool bf16_map_2d(CUtensorMap* m, const void* base, uint64_t inner, uint64_t rows, uint32_t box_inner, uint32_t box_rows) {
+  EncodeTiledFn fn = nat_encode_fn();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[2] = {inner, rows};
+  const cuuint64_t strides[1] = {inner * 2};
+  const cuuint32_t box[2] = {box_inner, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // tensor maps of the weights and their scale bytes, in either layout (declared in moe_tmap.cuh)
 bool weight_maps(const ExpertWeights& w, const moe_shape_t& sh, CUtensorMap* tm_w13, CUtensorMap* tm_s13, CUtensorMap* tm_w2,
                  CUtensorMap* tm_s2) {

@@ -18,7 +18,8 @@ EXPORTS = ("moe_workspace_bytes", "moe_status_string", "moe_last_kernel_name", "
            "moe_forward_host_workspace_bytes", "moe_forward_host", "moe_expert_ffn_noalloc_max_bytes",
            "moe_expert_ffn_noalloc", "moe_debug_native_cta_share", "moe_debug_read_probe", "moe_prepack_bytes", "moe_prepack",
            "moe_expert_ffn_packed", "moe_forward_packed", "moe_forward_host_packed", "moe_debug_forward_one_launch",
-           "moe_debug_expert_ffn_variant")
+           "moe_debug_expert_ffn_variant", "moe_router_logits", "moe_combine_shared", "moe_ffn_block_workspace_bytes",
+           "moe_ffn_block")
 
 
 class MoeError(RuntimeError):
@@ -85,6 +86,14 @@ def lib():
         L.moe_debug_forward_one_launch.argtypes = L.moe_forward.argtypes
         L.moe_debug_expert_ffn_variant.restype = C.c_int
         L.moe_debug_expert_ffn_variant.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp, sz, vp, i32]
+        L.moe_router_logits.restype = C.c_int
+        L.moe_router_logits.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
+        L.moe_combine_shared.restype = C.c_int
+        L.moe_combine_shared.argtypes = [vp, vp, vp, vp, C.POINTER(Shape), vp, vp]
+        L.moe_ffn_block_workspace_bytes.restype = sz
+        L.moe_ffn_block_workspace_bytes.argtypes = [C.POINTER(Shape)]
+        L.moe_ffn_block.restype = C.c_int
+        L.moe_ffn_block.argtypes = [vp] * 10 + [C.POINTER(Shape), vp, vp, vp, vp, vp, sz, vp]
         L.moe_forward_host.restype = C.c_int
         L.moe_forward_host.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp, sz, vp]
         _lib = L
@@ -263,6 +272,33 @@ def moe_forward_host(logits_host, x_host, w13, w13_scale, w2, w2_scale, sh, out_
     _check(lib().moe_forward_host(_ptr(logits_host), _ptr(x_host), _ptr(w13), _ptr(w13_scale), _ptr(w2), _ptr(w2_scale),
                                   C.byref(sh), _ptr(out_host), _ptr(status_word), _ptr(ws), ws.numel(), _stream(stream)),
            "moe_forward_host")
+
+
+def moe_router_logits(x, w_router, logits, status_word=None, stream=None):
+    T, H = x.shape
+    E = w_router.shape[0]
+    _check(lib().moe_router_logits(_ptr(x), _ptr(w_router), T, H, E, _ptr(logits), _ptr(status_word), _stream(stream)),
+           "moe_router_logits")
+
+
+def moe_combine_shared(y_perm, inv_perm, topk_w, y_shared, sh, out, stream=None):
+    _check(lib().moe_combine_shared(_ptr(y_perm), _ptr(inv_perm), _ptr(topk_w), _ptr(y_shared), C.byref(sh), _ptr(out),
+                                    _stream(stream)), "moe_combine_shared")
+
+
+def alloc_block_workspace(sh, device="cuda"):
+    n = int(lib().moe_ffn_block_workspace_bytes(C.byref(sh)))
+    if n == 0:
+        raise MoeError("unsupported shape")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def moe_ffn_block(x, w_router, routed, shared, sh, out, topk_ids, topk_w, status_word, ws, stream=None):
+    """The FFN block: router projection, routed experts, shared expert, join (see include/moe_b200.h).
+    `routed` and `shared` are (w13, w13_scale, w2, w2_scale) tuples; the shared tensors have E = 1."""
+    _check(lib().moe_ffn_block(_ptr(x), _ptr(w_router), *[_ptr(a) for a in routed], *[_ptr(a) for a in shared], C.byref(sh),
+                               _ptr(out), _ptr(topk_ids), _ptr(topk_w), _ptr(status_word), _ptr(ws), ws.numel(),
+                               _stream(stream)), "moe_ffn_block")
 
 
 class LayerBuffers:
