@@ -45,7 +45,7 @@ GRAPH_STEPS = 8         # consecutive batches of the cycle per CUDA graph (decod
 # dram__bytes_read.sum + dram__bytes_write.sum per launch (or per two-launch call) from one ncu capture of the
 # workload; which capture, at which commit, is stated in the file under profiles/ named beside each figure.
 NCU_TRAFFIC_BYTES = {
-    "decode_c1_one_launch": 110440700,  # ffn_native_kernel<true>, the whole layer (profiles/ffn_native_decode.md)
+    "decode_c1_one_launch": 111113000,  # decode_one_kernel, the whole layer (profiles/decode_one_kernel_decode_c1.md)
     "decode_c1": 111216000,             # ffn_native_kernel<false> (profiles/ffn_native_decode.md)
     "decode_c64": 3064384880,           # ffn_native_kernel<false> (profiles/ffn_native_decode.md)
     "prefill_8k": 5611119000,           # ffn_umma_kernel<true> + <false> (profiles/ffn_umma_prefill_8k.md)
@@ -228,7 +228,7 @@ class Bench:
         self.stream = torch.cuda.current_stream()
         self.peaks = load_peaks()
         self._weights_key = None
-        self.weights_host = self.weights = self.packed = None
+        self.weights_host = self.weights = self.packed = self.raw = None
         self.read_only_gbs = None
 
     # ---- plumbing ---------------------------------------------------------------------------------------------
@@ -251,9 +251,10 @@ class Bench:
         queued when it ends: the region then measures device time, not the host's launch latency."""
         self.torch.cuda._sleep(200000)
 
-    def load_weights(self, wl):
+    def load_weights(self, wl, keep_raw=False):
         """Weights are model state: generated once per (H, I, E), moved to the device, re-laid by moe_prepack (the
-        one-time load transform, untimed) unless --raw-weights, after which the row-layout tensors are dropped."""
+        one-time load transform, untimed) unless --raw-weights, after which the row-layout tensors are dropped
+        (keep_raw: not yet - the FFN-block timing, which takes the row layout, runs first and drops them)."""
         key = (wl.H, wl.I, wl.E)
         if self._weights_key == key:
             return
@@ -265,9 +266,85 @@ class Bench:
         if not self.args.raw_weights:
             self.packed = moe.moe_prepack(*self.weights, moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k))
             torch.cuda.synchronize()
+            if keep_raw:
+                self.raw = self.weights
             self.weights = None
         self._weights_key = key
         self.read_only_gbs = None
+
+    def run_block(self, wl, min_ms=50.0):
+        """The FFN block around the routed path (moe_ffn_block: router projection, routed experts, shared expert, join)
+        on the same routed weights in the checkpoint's row layout, seeded router and shared-expert weights, a cycle of
+        seeded token batches: one round of at least min_ms, CUDA events, graphs of GRAPH_STEPS steps for decode."""
+        torch, moe, inputs = self.torch, self.moe, self.inputs
+        stream = self.stream
+        decode = wl.name in DECODE
+        routed = self.raw if self.raw is not None else self.weights
+        sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
+        n_cycle = 32 if decode else 2
+        xs = [self.dev(inputs.make_x(wl.T, wl.H, 7000 + self.rank * 100 + i)) for i in range(n_cycle)]
+        w_router = self.dev(inputs.f32_to_bf16_bits(inputs.bf16_bits_to_f32(inputs.make_x(wl.E, wl.H, 31)) * np.float32(0.03)))
+        shared = tuple(self.dev(a) for a in inputs.make_expert_weights(wl.H, wl.I, 1, seed=21))
+        ws = moe.alloc_block_workspace(sh)
+        out = torch.empty((wl.T, wl.H), dtype=torch.bfloat16, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+        def step(i, st=stream):
+            moe.moe_ffn_block(xs[i % n_cycle], w_router, routed, shared, sh, out, None, None, status, ws, st)
+
+        c0 = moe.moe_launch_count()
+        step(0)
+        launches_per_step = moe.moe_launch_count() - c0
+        for i in range(3):
+            step(i)
+        self.barrier()
+        graphs = []
+        if decode:
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            with torch.cuda.stream(side):
+                step(0, None)
+            stream.wait_stream(side)
+            self.barrier()
+            for i0 in range(0, n_cycle, GRAPH_STEPS):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    for i in range(i0, i0 + GRAPH_STEPS):
+                        step(i, None)
+                graphs.append(g)
+            for g in graphs:
+                g.replay()
+            self.barrier()
+
+        def play(n):
+            if decode:
+                for i in range(n // GRAPH_STEPS):
+                    graphs[i % len(graphs)].replay()
+            else:
+                for i in range(n):
+                    step(i)
+
+        def timed(n):
+            e0, e1 = self.events()
+            self.barrier()
+            self.hold()
+            e0.record(stream)
+            play(n)
+            e1.record(stream)
+            self.barrier()
+            return max_over_ranks(e0.elapsed_time(e1), self.world)
+
+        pilot_n = GRAPH_STEPS if decode else 2
+        pilot = timed(pilot_n) / pilot_n
+        n = steps_for_region(pilot, min_ms, multiple=GRAPH_STEPS if decode else 1, at_least=3)
+        time.sleep(COOLDOWN_S)
+        ms = timed(n) / n
+        assert int(status.item()) == 0, "device-side wait timed out"
+        del graphs, xs, ws, shared
+        torch.cuda.empty_cache()
+        return {"ms_per_step": ms, "value": wl.T * self.world / (ms * 1e-3), "unit": "tokens/s", "steps": n,
+                "gpu_launches_per_step": launches_per_step, "call": "moe_ffn_block (row-layout weights)",
+                "launch": ("cuda graph replay, %d steps per graph" % GRAPH_STEPS) if decode else "eager"}
 
     def read_only_stream(self, status):
         """Read-only ceiling: the decode kernel's load mechanism alone over the resident gate/up weights (2.1 GB at
@@ -354,8 +431,8 @@ class Bench:
 
         # Decode-sized steps are a handful of short kernels: like the paper's decode tiers they are replayed as CUDA
         # graphs (the C-ABI calls captured as they are).  A serving graph holds many layers back to back; here a graph
-        # holds GRAPH_STEPS consecutive batches of the cycle (one layer call each), plus one single-step graph per
-        # batch for a step count that is not a multiple of GRAPH_STEPS.
+        # holds GRAPH_STEPS consecutive batches of the cycle (one layer call each); a step count that is not a multiple of
+        # GRAPH_STEPS ends with one graph of the remaining steps.
         use_graph = decode and not args.no_graph
 
         def capture(fn, idx):
@@ -378,12 +455,24 @@ class Bench:
         if use_graph:
             warm_side(step)
             c0 = moe.moe_launch_count()
-            graphs = [capture(step, [i]) for i in range(n_cycle)]
-            launches_per_step = (moe.moe_launch_count() - c0) // n_cycle
+            graphs = [capture(step, [0])]
+            launches_per_step = moe.moe_launch_count() - c0
             multi_graphs = [capture(step, range(i0, i0 + GRAPH_STEPS)) for i0 in range(0, n_cycle, GRAPH_STEPS)]
-            for g in graphs[:3] + multi_graphs:
+            for g in graphs + multi_graphs:
                 g.replay()
             self.barrier()
+
+        rem_graphs = {}
+
+        def prepare(n):
+            """A step count that is not a multiple of GRAPH_STEPS ends with ONE graph of the remaining steps (captured
+            here, before the timed region)."""
+            r = n % GRAPH_STEPS
+            if use_graph and r and r not in rem_graphs:
+                i0 = (n // GRAPH_STEPS) * GRAPH_STEPS
+                rem_graphs[r] = capture(step, range(i0, i0 + r))
+                rem_graphs[r].replay()
+                self.barrier()
 
         def play(n, inner=None):
             """Enqueue n consecutive steps of the cycle."""
@@ -391,8 +480,8 @@ class Bench:
                 n_multi = n // GRAPH_STEPS
                 for i in range(n_multi):
                     multi_graphs[i % len(multi_graphs)].replay()
-                for i in range(n_multi * GRAPH_STEPS, n):
-                    graphs[i % n_cycle].replay()
+                if n % GRAPH_STEPS:
+                    rem_graphs[n % GRAPH_STEPS].replay()
             else:
                 for i in range(n):
                     step(i, inner[i] if inner is not None and i < len(inner) and not one_launch else None)
@@ -400,6 +489,7 @@ class Bench:
         def region(n, inner=None):
             """One timed region of exactly n steps: barrier + synchronize on both sides, CUDA events on the launching
             stream, max over ranks.  Returns (ms of the region, clock record, launches of the library's kernels)."""
+            prepare(n)
             e0, e1 = self.events()
             sampler = ClockSampler(physical_gpu_index(self.local))
             c0 = moe.moe_launch_count()
@@ -609,6 +699,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="decode workloads: launch the calls eagerly instead of replaying CUDA graphs")
+    ap.add_argument("--no-block", action="store_true", help="skip the timing of moe_ffn_block")
     ap.add_argument("--four-calls", action="store_true", help="time the four calls even where moe_forward is one launch")
     ap.add_argument("--raw-weights", action="store_true", help="read the weights in the checkpoint's row layout instead of moe_prepack's tiles")
     args = ap.parse_args()
@@ -648,6 +739,13 @@ def main():
     # every rank times the same list, in the same order (the barriers pair up)
     # (replicas, N > 1: the headline workload only - the scaling figure is the headline's)
     names = [args.workload] if args.workload else [HEADLINE] + ([n for n in PRODUCTION if n != HEADLINE] if world == 1 else [])
+    # the FFN block around the routed path (router projection, shared expert, join), beside the headline (N = 1, default run)
+    block = None
+    if world == 1 and not args.workload and not args.raw_weights and not args.no_block:
+        bench.load_weights(head, keep_raw=True)
+        block = {n: bench.run_block(inputs.WORKLOADS[n]) for n in ("decode_c1", "decode_c64", "prefill_8k")}
+        bench.raw = None
+        torch.cuda.empty_cache()
     records = {}
     for name in names:
         wl = inputs.WORKLOADS[name]
@@ -692,6 +790,7 @@ def main():
             "roofline": roof, "cpu_baseline": cpu, "e2e": hr.get("e2e"), "gpu_launches": ex["gpu_launches"],
             "clocks": ex["clocks"], "kernels": hr["kernels"],
             "workloads": {n: {k: v for k, v in r.items() if k not in ("one_launch", "n_cycle")} for n, r in records.items()},
+            "ffn_block": block,
             "protocol": ("headline: one region of exactly --steps steps; workloads: %d rounds of at least %d ms (decode) / %d ms "
                          "(prefill) each, %.1f s idle before every round, median reported, every round kept; every region is "
                          "bracketed by a barrier and a synchronize, timed by CUDA events on the launching stream behind a "
