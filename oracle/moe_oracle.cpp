@@ -150,17 +150,73 @@ void route_token(const float* l, int E, int k, int32_t* ids, float* w) {
   for (int j = 0; j < k; ++j) w[j] = ex[j] / s;
 }
 
+// ---- online activation quantisation (variant) --------------------------------
+//
+// The paper's historical decode route quantises the BF16 activations online to INT8, one scale per 32 elements,
+// so that an integer dot product can consume them.  The analogue on the hardware this repository targets is the
+// weights' own format: E2M1 codes with one E8M0 scale byte per 32 consecutive elements (reading G18).  One block:
+//   amax = max |v|;  amax = 0 -> byte 127, every code a signed zero;
+//   s    = the smallest integer in [-126, 126] with amax <= 6 * 2^s  (6 = largest E2M1 magnitude: nothing saturates,
+//          and a smaller s would);  scale byte = s + 127;
+//   code = sign bit of v, magnitude = the E2M1 magnitude nearest to |v| / 2^s, a tie going to the magnitude whose
+//          mantissa bit is 0 (round to nearest even); dequantised value = E2M1(code) * 2^s.
+// |v| / 2^s is formed in double, where it is exact for every bf16 v.  Domain: |v| <= 2^126, so that every decoded
+// value is an fp32 number (above it 4 * 2^126 or 6 * 2^126 would not be); activations never come near it.
+inline void quant_block(const float* v, uint8_t* codes /* 32, one per byte */, uint8_t* scale_byte) {
+  double amax = 0.0;
+  for (int j = 0; j < 32; ++j) amax = std::fmax(amax, std::fabs(static_cast<double>(v[j])));
+  int s = 0;
+  if (amax > 0.0) {
+    s = -126;
+    while (s < 126 && amax > 6.0 * std::ldexp(1.0, s)) s += 1;
+  }
+  *scale_byte = static_cast<uint8_t>(s + 127);
+  for (int j = 0; j < 32; ++j) {
+    const double m = std::fabs(static_cast<double>(v[j])) / std::ldexp(1.0, s);
+    unsigned best = 0;
+    double best_d = m;  // distance to magnitude code 0 (value 0)
+    for (unsigned c = 1; c < 8; ++c) {
+      const double d = std::fabs(m - static_cast<double>(e2m1_value(c)));
+      if (d < best_d || (d == best_d && (c & 1u) == 0u)) {
+        best = c;
+        best_d = d;
+      }
+    }
+    codes[j] = static_cast<uint8_t>(best | (std::signbit(v[j]) ? 8u : 0u));
+  }
+}
+
+// A row of K bf16 values -> the values its quantised form decodes to (what the contraction then consumes), and
+// optionally the packed codes (element 2j in the low nibble of byte j, as the weights) and scale bytes.
+inline void quant_row(const uint16_t* row, int64_t K, float* deq, uint8_t* packed /* K/2 or NULL */,
+                      uint8_t* scales /* K/32 or NULL */) {
+  for (int64_t b = 0; b < K / 32; ++b) {
+    float v[32];
+    uint8_t codes[32], sb;
+    for (int j = 0; j < 32; ++j) v[j] = bf16_to_f32(row[b * 32 + j]);
+    quant_block(v, codes, &sb);
+    for (int j = 0; j < 32; ++j) deq[b * 32 + j] = e2m1_value(codes[j]) * e8m0_value(sb);
+    if (packed != nullptr)
+      for (int j = 0; j < 16; ++j) packed[b * 16 + j] = static_cast<uint8_t>(codes[2 * j] | (codes[2 * j + 1] << 4));
+    if (scales != nullptr) scales[b] = sb;
+  }
+}
+
 // ---- one slot of the expert FFN ---------------------------------------------
 
 // act[i] = bf16( silu(g_i) * u_i ), g = W1 x, u = W3 x, W1 = rows [0,I) of w13,
 // W3 = rows [I,2I) (reading G4); g and u are not rounded before the
 // activation (reading G6); y[n] = sum_i W2[n,i] act[i].  Accumulation in
 // ascending index order in ACC (float or double).
+//
+// quant = true is the quantised-activation variant: both contractions consume the quantised form of their input row
+// (quant_row: the token row; the intermediate after its rounding to bf16), everything else unchanged.
 template <typename ACC>
 void ffn_slot(const uint16_t* x_row, const uint8_t* w13, const uint8_t* s13, const uint8_t* w2, const uint8_t* s2,
-              int64_t H, int64_t I, uint16_t* act_row /* [I] */, float* y_row /* [H] */) {
+              int64_t H, int64_t I, uint16_t* act_row /* [I] */, float* y_row /* [H] */, bool quant = false) {
   std::vector<float> xf(static_cast<size_t>(H));
   for (int64_t h = 0; h < H; ++h) xf[h] = bf16_to_f32(x_row[h]);
+  if (quant) quant_row(x_row, H, xf.data(), nullptr, nullptr);
   for (int64_t i = 0; i < I; ++i) {
     ACC g = 0, u = 0;
     for (int64_t h = 0; h < H; ++h) {
@@ -173,6 +229,7 @@ void ffn_slot(const uint16_t* x_row, const uint8_t* w13, const uint8_t* s13, con
   }
   std::vector<float> af(static_cast<size_t>(I));
   for (int64_t i = 0; i < I; ++i) af[i] = bf16_to_f32(act_row[i]);
+  if (quant) quant_row(act_row, I, af.data(), nullptr, nullptr);
   for (int64_t n = 0; n < H; ++n) {
     ACC acc = 0;
     for (int64_t i = 0; i < I; ++i)
@@ -250,9 +307,9 @@ void oracle_permute(const uint16_t* x, const int32_t* ids, const int32_t* offset
 
 // Steps a5-a7 over sorted rows.  act may be NULL.  Weight tensors are the
 // logical ones: w13[E,2I,H/2], s13[E,2I,H/32], w2[E,H,I/2], s2[E,H,I/32].
-void oracle_expert_ffn(const uint16_t* x_perm, const int32_t* offsets, const uint8_t* w13, const uint8_t* s13,
-                       const uint8_t* w2, const uint8_t* s2, int T, int H, int I, int E, int k, int acc64,
-                       uint16_t* act /* [T*k, I] or NULL */, float* y_perm /* [T*k, H] */) {
+static void expert_ffn_rows(const uint16_t* x_perm, const int32_t* offsets, const uint8_t* w13, const uint8_t* s13,
+                            const uint8_t* w2, const uint8_t* s2, int T, int H, int I, int E, int k, int acc64, bool quant,
+                            uint16_t* act /* [T*k, I] or NULL */, float* y_perm /* [T*k, H] */) {
   const int64_t S = static_cast<int64_t>(T) * k;
   std::vector<int32_t> expert_of(static_cast<size_t>(S));
   for (int e = 0; e < E; ++e)
@@ -265,11 +322,37 @@ void oracle_expert_ffn(const uint16_t* x_perm, const int32_t* offsets, const uin
     std::vector<uint16_t> act_row(static_cast<size_t>(I));
     if (acc64)
       ffn_slot<double>(x_perm + p * H, w13 + e * w13_e, s13 + e * s13_e, w2 + e * w2_e, s2 + e * s2_e, H, I,
-                       act_row.data(), y_perm + p * H);
+                       act_row.data(), y_perm + p * H, quant);
     else
       ffn_slot<float>(x_perm + p * H, w13 + e * w13_e, s13 + e * s13_e, w2 + e * w2_e, s2 + e * s2_e, H, I,
-                      act_row.data(), y_perm + p * H);
+                      act_row.data(), y_perm + p * H, quant);
     if (act != nullptr) std::memcpy(act + p * I, act_row.data(), static_cast<size_t>(I) * 2);
+  }
+}
+
+void oracle_expert_ffn(const uint16_t* x_perm, const int32_t* offsets, const uint8_t* w13, const uint8_t* s13,
+                       const uint8_t* w2, const uint8_t* s2, int T, int H, int I, int E, int k, int acc64,
+                       uint16_t* act /* [T*k, I] or NULL */, float* y_perm /* [T*k, H] */) {
+  expert_ffn_rows(x_perm, offsets, w13, s13, w2, s2, T, H, I, E, k, acc64, false, act, y_perm);
+}
+
+// The quantised-activation variant of steps a5-a7 (see quant_block).  `act` receives the intermediate as bf16, i.e.
+// before its quantisation.
+void oracle_expert_ffn_q(const uint16_t* x_perm, const int32_t* offsets, const uint8_t* w13, const uint8_t* s13,
+                         const uint8_t* w2, const uint8_t* s2, int T, int H, int I, int E, int k, int acc64,
+                         uint16_t* act /* [T*k, I] or NULL */, float* y_perm /* [T*k, H] */) {
+  expert_ffn_rows(x_perm, offsets, w13, s13, w2, s2, T, H, I, E, k, acc64, true, act, y_perm);
+}
+
+// Rows of K bf16 values (K a multiple of 32) -> packed codes [rows, K/2], scale bytes [rows, K/32] and the decoded
+// values [rows, K]; any output may be NULL.
+void oracle_quant_act(const uint16_t* v, int64_t rows, int64_t K, uint8_t* packed, uint8_t* scales, float* deq) {
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r) {
+    std::vector<float> d(static_cast<size_t>(K));
+    quant_row(v + r * K, K, d.data(), packed != nullptr ? packed + r * (K / 2) : nullptr,
+              scales != nullptr ? scales + r * (K / 32) : nullptr);
+    if (deq != nullptr) std::memcpy(deq + r * K, d.data(), static_cast<size_t>(K) * 4);
   }
 }
 

@@ -137,6 +137,39 @@ def expert_ffn(x_perm, offsets, w13, s13, w2, s2, k, acc64=False, want_act=False
     return (y, act) if want_act else y
 
 
+def expert_ffn_q(x_perm, offsets, w13, s13, w2, s2, k, acc64=False, want_act=False):
+    """The quantised-activation variant of expert_ffn: both contractions consume E2M1 codes with one E8M0 scale per
+    32 elements (quant_act) instead of bf16 values; `act` is the bf16 intermediate before its quantisation."""
+    S, H = x_perm.shape
+    E, twoI, _ = w13.shape
+    I = twoI // 2
+    T = S // k
+    _chk(x_perm, np.uint16)
+    _chk(offsets, np.int32, (E + 1,))
+    _chk(w13, np.uint8, (E, 2 * I, H // 2))
+    _chk(s13, np.uint8, (E, 2 * I, H // 32))
+    _chk(w2, np.uint8, (E, H, I // 2))
+    _chk(s2, np.uint8, (E, H, I // 32))
+    y = np.empty((S, H), np.float32)
+    act = np.empty((S, I), np.uint16) if want_act else None
+    lib().oracle_expert_ffn_q(_p(x_perm), _p(offsets), _p(w13), _p(s13), _p(w2), _p(s2), T, H, I, E, k,
+                              int(bool(acc64)), _p(act), _p(y))
+    return (y, act) if want_act else y
+
+
+def quant_act(v):
+    """Rows of bf16 bit patterns [rows, K] -> (packed E2M1 codes [rows, K/2], scale bytes [rows, K/32], decoded
+    values [rows, K] float32): the online activation quantisation of the variant, one scale per 32 elements."""
+    rows, K = v.shape
+    assert K % 32 == 0
+    _chk(v, np.uint16)
+    packed = np.empty((rows, K // 2), np.uint8)
+    scales = np.empty((rows, K // 32), np.uint8)
+    deq = np.empty((rows, K), np.float32)
+    lib().oracle_quant_act(_p(v), C.c_int64(rows), C.c_int64(K), _p(packed), _p(scales), _p(deq))
+    return packed, scales, deq
+
+
 def combine(y_perm, inv_perm, w):
     S, H = y_perm.shape
     T, k = w.shape
