@@ -259,6 +259,31 @@ int moe_ffn_block(const void* x_bf16 /* [T,H] */, const void* w_router_bf16 /* [
                   float* topk_w /* [T,k] or NULL */, int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Quantised-activation variant of moe_expert_ffn (paper, "historical TP4/EP1 decode route": the BF16 activations are
+ * quantised online, one scale per 32 elements, so that a low-precision dot product consumes them; the paper's target is
+ * INT8, this library's is the weights' own format, which the block-scaled FP4 tensor-core instruction takes directly).
+ *
+ *   - Quantiser, applied to every row of x_perm along H and to every row of the bf16 intermediate along I, per block of
+ *     32 consecutive elements: amax = max |v|; s = the smallest integer in [-126, 126] with amax <= 6 * 2^s (s = 0 for
+ *     an all-zero block); code = E2M1 value nearest to v / 2^s, ties to the even code; the contraction consumes
+ *     E2M1(code) * 2^s.  Everything else as moe_expert_ffn: g, u in fp32, act = bf16_rne(silu(g) * u), y_perm fp32.
+ *     Inputs with |v| > 2^126 are outside the domain.
+ *   - Result: y_perm differs from moe_expert_ffn's by the quantisation error (about a quarter of the output's norm on
+ *     the benchmark's inputs: one E2M1 term keeps two to three significant bits); against this variant's own oracle the
+ *     result is the same up to fp32 summation order and the roundings that order can flip.
+ *   - Weights: the four logical tensors with packed = NULL, or packed = the buffer of moe_prepack with the four NULL.
+ *   - Shapes: H and I multiples of 512 and at most 4096; otherwise MOE_ERR_UNSUPPORTED_SHAPE.  Any T * k: one kernel
+ *     serves decode and prefill (a pass holds 128 tokens of an expert, against 16 in moe_expert_ffn's kernel).
+ *   - `ws`: moe_expert_ffn_q_workspace_bytes(), 256-byte aligned, no initialisation needed.  Enqueue only, no
+ *     allocation, capturable, bounded device-side waits and status_word as moe_expert_ffn.
+ */
+size_t moe_expert_ffn_q_workspace_bytes(const moe_shape_t* shape);
+int moe_expert_ffn_q(const void* x_perm_bf16 /* [T*k,H] */, const int32_t* expert_offsets, const uint8_t* w13,
+                     const uint8_t* w13_scale, const uint8_t* w2, const uint8_t* w2_scale, const void* packed,
+                     const moe_shape_t* shape, float* y_perm /* [T*k,H] */, int32_t* status_word, void* ws, size_t ws_bytes,
+                     void* cuda_stream);
+
+/*
  * moe_expert_ffn without a workspace argument, for callers that cannot allocate device memory
  * (the paper has no counterpart: this is a packaging variant of moe_expert_ffn, same arithmetic).
  *

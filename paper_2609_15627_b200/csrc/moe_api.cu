@@ -286,6 +286,35 @@ BlockLayout block_layout(const moe_shape_t& s) {
 }
 }  // namespace
 
+size_t moe_expert_ffn_q_workspace_bytes(const moe_shape_t* shape) {
+  if (check_shape(shape) != MOE_OK) return 0;
+  return native_q_scratch_bytes(*shape) + kAlign;
+}
+
+int moe_expert_ffn_q(const void* x_perm_bf16, const int32_t* expert_offsets, const uint8_t* w13, const uint8_t* w13_scale,
+                     const uint8_t* w2, const uint8_t* w2_scale, const void* packed, const moe_shape_t* shape, float* y_perm,
+                     int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  const bool raw = w13 != nullptr || w13_scale != nullptr || w2 != nullptr || w2_scale != nullptr;
+  if (raw == (packed != nullptr)) return MOE_ERR_INVALID_ARG;  // exactly one form of the weights
+  if (packed != nullptr && !aligned(packed, kAlign)) return MOE_ERR_INVALID_ARG;
+  const ExpertWeights w = packed != nullptr ? packed_view(packed, *shape) : ExpertWeights{w13, w13_scale, w2, w2_scale, false};
+  if (w.w13 == nullptr || w.s13 == nullptr || w.w2 == nullptr || w.s2 == nullptr || x_perm_bf16 == nullptr ||
+      expert_offsets == nullptr || y_perm == nullptr)
+    return MOE_ERR_INVALID_ARG;
+  if (!aligned(x_perm_bf16, 16) || !aligned(expert_offsets, 16) || !aligned(w.w13, 16) || !aligned(w.s13, 16) ||
+      !aligned(w.w2, 16) || !aligned(w.s2, 16) || !aligned(y_perm, 16))
+    return MOE_ERR_INVALID_ARG;
+  if (status_word != nullptr && !aligned(status_word, 4)) return MOE_ERR_INVALID_ARG;
+  if (!native_q_shape_ok(*shape, w.w13, w.w2)) return MOE_ERR_UNSUPPORTED_SHAPE;
+  if (check_ws(ws, ws_bytes, native_q_scratch_bytes(*shape)) != MOE_OK) return MOE_ERR_WORKSPACE;
+  StatusRef status;
+  if ((rc = resolve_status(status_word, &status)) != MOE_OK) return rc;
+  return launch_expert_ffn_native_q(static_cast<const __nv_bfloat16*>(x_perm_bf16), expert_offsets, w, *shape, ws, y_perm, status,
+                                    static_cast<cudaStream_t>(cuda_stream));
+}
+
 size_t moe_ffn_block_workspace_bytes(const moe_shape_t* shape) {
   if (check_shape(shape) != MOE_OK) return 0;
   return block_layout(*shape).total;

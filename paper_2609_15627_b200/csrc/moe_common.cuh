@@ -43,6 +43,14 @@ inline size_t native_scratch_bytes(const moe_shape_t& s) {
          align_up(8 * S * (s.H / 32), kAlign) + align_up(static_cast<size_t>(s.E) * 4, kAlign);
 }
 
+// scratch of the quantised-activation variant: one operand row per sorted row (codes and scale bytes of the token rows
+// and of the intermediate) and the per-expert counters
+inline size_t native_q_scratch_bytes(const moe_shape_t& s) {
+  const size_t S = static_cast<size_t>(s.T) * s.k;
+  return align_up(S * (s.I / 2), kAlign) + align_up(S * (s.I / 32), kAlign) + align_up(S * (s.H / 2), kAlign) +
+         align_up(S * (s.H / 32), kAlign) + align_up(static_cast<size_t>(s.E) * 4, kAlign);
+}
+
 inline WsLayout ws_layout(const moe_shape_t& s) {
   WsLayout L;
   const size_t S = static_cast<size_t>(s.T) * s.k;
@@ -132,6 +140,10 @@ int launch_validate_scales(const uint8_t* scales, size_t n, int* bad, cudaStream
 
 // native block-scaled FP4 variant; scratch of native_scratch_bytes
 bool native_shape_ok(const moe_shape_t& s, const void* w13, const void* w2);
+// the quantised-activation variant of the same kernel: any batch size; scratch of native_q_scratch_bytes
+bool native_q_shape_ok(const moe_shape_t& s, const void* w13, const void* w2);
+int launch_expert_ffn_native_q(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& s,
+                               void* scratch, float* y_perm, StatusRef status, cudaStream_t st);
 int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& s,
                              void* scratch, float* y_perm, StatusRef status, cudaStream_t st);
 

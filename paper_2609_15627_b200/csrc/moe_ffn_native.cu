@@ -68,6 +68,7 @@ constexpr int kScStages = 3;          // scale-byte ring: one stage = 256 rows x
 constexpr int kScStage = kTile * 16;
 constexpr int kSfGroups = 3;          // tensor-memory groups for the weight scale factors: 4 words x 8 columns
 constexpr int kMaxTokPass = 16;       // tokens per pass (16 x 8 = 128 operand rows)
+constexpr int kQOneLaunchRows = 64;   // quantised-activation variant: up to this many rows per expert on average, one launch
 constexpr int kMaxK = 4096;           // scale factors of one pass's term rows stay in tensor memory: 8 columns per K step
 constexpr int kNatThreads = 10 * 32;
 constexpr int kEpiWarp = 6;           // warps 6..9: warp % 4 = 2, 3, 0, 1 -> one tensor-memory lane quadrant each
@@ -88,6 +89,8 @@ struct NatArgs {
   int own_status;            // the library's own word: the one-launch kernel's last CTA clears it for the next call
   int E, H, I, S;
   int blocked;               // weights in moe_prepack's tile-contiguous layout (see ExpertWeights)
+  int ph_lo, ph_hi;          // projections this launch runs: [0, 2) = both; the large-batch schedule runs one per launch
+  int by_pass;               // large-batch schedule: CTAs get equal numbers of passes, not of items (see unit_shares)
 };
 
 // The one-launch layer (moe_forward on a handful of tokens): what the kernel needs beyond the expert FFN's arguments.
@@ -139,12 +142,13 @@ struct alignas(64) TermMaps {
 // it has at most kRepMaxItems items (another 0.7 % on decode_c64, where a CTA has 24).
 constexpr int kRepBox = 0, kRepTok = 1 << kRepBox;  // boxes 0..kRepBox hold at most kRepTok tokens
 constexpr int kRepMaxItems = 2;
-MOE_DEVINL int term_box(int n_tok) { return n_tok <= 1 ? 0 : (n_tok <= 2 ? 1 : (n_tok <= 4 ? 2 : (n_tok <= 8 ? 3 : 4))); }
+MOE_DEVINL int op_box(int n_rows) { return n_rows <= 8 ? 0 : (n_rows <= 16 ? 1 : (n_rows <= 32 ? 2 : (n_rows <= 64 ? 3 : 4))); }
 
 // One projection as the kernel sees it
 struct Phase {
   int K, R, n_steps, tiles;  // reduction length, weight rows per expert, K steps, items per expert
   int begin, end;            // this CTA's items (at most 1024 experts x 32 tiles)
+  int pb, pe;                // of item `begin` the passes from pb on, of item `end - 1` the passes before pe
   bool rep_ok;               // few enough of them for single-token passes to be repeated per lane quadrant
 };
 // Items go to CTAs in contiguous shares: gate/up items evenly, per0 each.  A down item of expert t is placed as if it
@@ -178,6 +182,32 @@ __host__ __device__ inline void cta_shares(int grid, int c, int n_touched, int t
   out[2] = total1 == 0 ? 0 : first_down_item_of_cta(c, total1, tiles0, tiles1, per0);
   out[3] = total1 == 0 ? 0 : (c + 1 >= grid ? total1 : first_down_item_of_cta(c + 1, total1, tiles0, tiles1, per0));
 }
+// Large-batch schedule (one projection per launch, so no item waits for another): the passes of all items, in the order
+// (touched expert, tile, pass), are cut into gridDim.x equal contiguous shares - an expert with many rows has many
+// passes per item, and equal item counts would leave its CTAs far behind.  out: first item, item after the last, first
+// pass of the first item, pass after the last of the last item.
+MOE_DEVINL void pass_shares(int grid, int c, int n_touched, const int* t_begin, const int* t_end, int tok_pass, int tiles,
+                            int* out) {
+  long long total = 0;
+  for (int ti = 0; ti < n_touched; ++ti) total += static_cast<long long>((t_end[ti] - t_begin[ti] + tok_pass - 1) / tok_pass) * tiles;
+  const long long lo = total * c / grid, hi = total * (c + 1) / grid;
+  out[0] = out[1] = out[2] = out[3] = 0;
+  if (lo >= hi) return;
+  long long cum = 0;
+  for (int ti = 0; ti < n_touched; ++ti) {
+    const int n_pass = (t_end[ti] - t_begin[ti] + tok_pass - 1) / tok_pass;
+    const long long next = cum + static_cast<long long>(n_pass) * tiles;
+    if (lo >= cum && lo < next) {
+      out[0] = ti * tiles + static_cast<int>((lo - cum) / n_pass);
+      out[2] = static_cast<int>((lo - cum) % n_pass);
+    }
+    if (hi - 1 >= cum && hi - 1 < next) {
+      out[1] = ti * tiles + static_cast<int>((hi - 1 - cum) / n_pass) + 1;
+      out[3] = static_cast<int>((hi - 1 - cum) % n_pass) + 1;
+    }
+    cum = next;
+  }
+}
 MOE_DEVINL Phase phase_of(int ph, const NatArgs& a, const int* shares) {
   Phase p;
   p.K = ph == 0 ? a.H : a.I;
@@ -186,6 +216,8 @@ MOE_DEVINL Phase phase_of(int ph, const NatArgs& a, const int* shares) {
   p.tiles = p.R / kTile;
   p.begin = shares[2 * ph];
   p.end = shares[2 * ph + 1];
+  p.pb = shares[5 + 2 * ph];  // (shares[4] is another word of the set-up)
+  p.pe = shares[6 + 2 * ph];
   p.rep_ok = p.end - p.begin <= kRepMaxItems;
   return p;
 }
@@ -208,7 +240,7 @@ __host__ __device__ inline NatSmem nat_smem(int E, int K) {
   m.misc = off;
   off += 64;
   m.touched = off;  // touched experts: id, first row, end row
-  off += (3 * static_cast<uint32_t>(E) + 8) * 4;
+  off += (3 * static_cast<uint32_t>(E) + 16) * 4;
   m.route = off;    // one-launch layer: expert and weight of every slot, sorted row of every slot, row of (touched expert, token)
   off += 4 * kFusedMaxSlots * 4;
   m.total = off;
@@ -220,6 +252,8 @@ __host__ __device__ inline NatSmem nat_smem(int E, int K) {
 // ---- split kernel: bf16 token rows -> 8 E2M1 term rows with their scale bytes; 8 threads per 32-element block ----
 // Few, large CTAs: the FFN grid's CTAs need a whole SM each and are handed out in blockIdx order, so every SM this
 // grid still occupies delays one of them - with at most (SMs - working FFN CTAs) CTAs here, only idle ones.
+// kQ (quantised-activation variant): one term per row, operand row = token row.
+template <bool kQ>
 __global__ void __launch_bounds__(1024) native_split_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict__ aq,
                                                            uint8_t* __restrict__ aq_sf, int* __restrict__ done, int S, int H,
                                                            int E, int* __restrict__ status_clear) {
@@ -238,9 +272,10 @@ __global__ void __launch_bounds__(1024) native_split_kernel(const __nv_bfloat16*
   const uint2 v = __ldcg(reinterpret_cast<const uint2*>(x + static_cast<size_t>(p) * H + b * 32 + sub * 4));
   float r[1][4] = {{__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u), __uint_as_float(v.y << 16),
                    __uint_as_float(v.y & 0xFFFF0000u)}};
-  split_terms<1>(r, [&](int, int t, uint32_t bytes, int se) {
+  constexpr int nt = kQ ? 1 : kTerms;
+  split_terms<1, nt>(r, [&](int, int t, uint32_t bytes, int se) {
     if (live) {
-      const size_t row = static_cast<size_t>(p) * kTerms + t;
+      const size_t row = static_cast<size_t>(p) * nt + t;
       *reinterpret_cast<uint16_t*>(aq + row * (H / 2) + b * 16 + sub * 2) = static_cast<uint16_t>(bytes);
       if (sub == 0) aq_sf[row * n_blk + b] = static_cast<uint8_t>(se + 127);
     }
@@ -250,7 +285,10 @@ __global__ void __launch_bounds__(1024) native_split_kernel(const __nv_bfloat16*
 // kFused = false: the expert FFN (moe_expert_ffn).  kFused = true: the whole layer in this one launch (see FusedArgs);
 // the differences are the set-up, where the gate/up items' operand rows come from, which rows their epilogue writes,
 // and the reduction over slots after the down items.
-template <bool kFused>
+// kQ = true: the quantised-activation variant of the expert FFN.  Every operand row is one token's single E2M1 term
+// (the first term of the split: smallest block scale without saturation, round to nearest even), so a pass holds up to
+// 128 tokens, nothing is summed over lanes, and the gate/up epilogue quantises the bf16 intermediate the same way.
+template <bool kFused, bool kQ = false>
 __global__ void __launch_bounds__(kNatThreads, 1)
 ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_constant__ CUtensorMap tmap_s13,
                   const __grid_constant__ TermMaps tmap_a1, const __grid_constant__ CUtensorMap tmap_w2,
@@ -285,7 +323,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   int* s_tok = s_row + kFusedMaxSlots;                                  // [T * k] token of every sorted row
 
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  constexpr int tok_pass = kMaxTokPass;
+  static_assert(!(kFused && kQ), "the one-launch layer has no quantised-activation variant");
+  constexpr int nt = kQ ? 1 : kTerms;                 // operand rows per token
+  constexpr int tok_pass = kQ ? 128 : kMaxTokPass;    // tokens per pass: 128 operand rows
   const int need_done = 4 * (2 * a.I / kTile);  // four epilogue warps publish each gate/up item of an expert
 
   // ---- setup: touched experts, barriers, tensor memory ----
@@ -324,9 +364,23 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       }
       run += tot;
     }
+    __syncwarp();
     if (lane == 0) {
       s_misc[0] = run;
       cta_shares(static_cast<int>(gridDim.x), static_cast<int>(blockIdx.x), run, 2 * a.I / kTile, a.H / kTile, s_misc + 1);
+      s_misc[6] = s_misc[8] = 0;
+      s_misc[7] = s_misc[9] = 1 << 30;
+      if (a.by_pass) {
+        for (int ph = 0; ph < 2; ++ph) {
+          int r[4];
+          pass_shares(static_cast<int>(gridDim.x), static_cast<int>(blockIdx.x), run, t_begin, t_end, tok_pass,
+                      ph == 0 ? 2 * a.I / kTile : a.H / kTile, r);
+          s_misc[1 + 2 * ph] = r[0];
+          s_misc[2 + 2 * ph] = r[1];
+          s_misc[6 + 2 * ph] = r[2];
+          s_misc[7 + 2 * ph] = r[3];
+        }
+      }
     }
   }
   if (tid == 0) {
@@ -459,6 +513,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       if (lane == 0) {
         s_misc[0] = n_t;
         cta_shares(static_cast<int>(gridDim.x), static_cast<int>(blockIdx.x), n_t, 2 * a.I / kTile, a.H / kTile, s_misc + 1);
+        s_misc[6] = s_misc[8] = 0;
+        s_misc[7] = s_misc[9] = 1 << 30;
       }
     }
     __syncthreads();
@@ -472,7 +528,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     if (lane == 0) {
       int s = 0, cs = 0;
       uint32_t ph = 0, cph = 0;
-      const uint64_t stream_once = l2_policy_evict_first();  // every weight byte is read once per call
+      // every weight byte is read once per call - unless items have several passes, each of which reads it again
+      const uint64_t stream_once = a.by_pass ? l2_policy_evict_normal() : l2_policy_evict_first();
       // The weights depend on nothing, the term rows do: on the split kernel (phase 0) or on the gate/up items of
       // their expert (phase 1).  While a dependency is open, the weight loads go out and the term-row loads of up to
       // kWStages steps are held back; they follow once the dependency is met.
@@ -500,7 +557,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         n_pend = 0;
         dep_ok = true;
       };
-      for (int phase = 0; phase < 2; ++phase) {
+      for (int phase = a.ph_lo; phase < a.ph_hi; ++phase) {
         const Phase P = phase_of(phase, a, s_misc + 1);
         const CUtensorMap* mw = phase == 0 ? &tmap_w13 : &tmap_w2;
         const CUtensorMap* msc = phase == 0 ? &tmap_s13 : &tmap_s2;
@@ -519,10 +576,10 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             dep_e = e;
             dep_ok = false;
           }
-          for (int pass = 0; pass < n_pass; ++pass) {
+          for (int pass = (it == P.begin ? P.pb : 0); pass < (it == P.end - 1 ? min(n_pass, P.pe) : n_pass); ++pass) {
             const bool by_token = kFused && phase == 0;  // the expert's rows are fetched token by token (at most 4)
-            const int bi = term_box(min(tok_pass, n_rows_e - pass * tok_pass));  // box of 8 << bi term rows
-            const int n_rep = (P.rep_ok && bi <= kRepBox) ? 4 : 1;
+            const int bi = op_box(min(tok_pass, n_rows_e - pass * tok_pass) * nt);  // box of 8 << bi operand rows
+            const int n_rep = (!kQ && P.rep_ok && bi <= kRepBox) ? 4 : 1;
             for (int ks = 0; ks < P.n_steps; ++ks) {
               if ((ks & 1) == 0) {  // 16 scale bytes per weight row cover two K steps
                 mbar_wait(&empty_sc[cs], cph ^ 1u, a.status);
@@ -544,7 +601,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
               tma_load_2d_hint(sW + s * kStage, mw, wx, wya, &full_w[s], stream_once);
               tma_load_2d_hint(sW + s * kStage + 128 * 128, mw, wx, wyb, &full_w[s], stream_once);
               // the pass's term rows (8 per token, consecutive); rows past the end of the tensor arrive as zeros
-              const int arow = (row_begin + pass * tok_pass) * kTerms;
+              const int arow = (row_begin + pass * tok_pass) * nt;
               if (by_token) {
                 // (the tokens' term rows were seen complete during the set-up: no dependency to hold these back for)
                 for (int j = 0; j < n_rows_e; ++j)
@@ -596,13 +653,13 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       int s = 0, slot = 0;
       uint32_t ph = 0, sph = 0, aph = 0, acc_ph = 0;
       const uint32_t d_addr = tmem_base + kColD;
-      for (int phase = 0; phase < 2; ++phase) {
+      for (int phase = a.ph_lo; phase < a.ph_hi; ++phase) {
         const Phase P = phase_of(phase, a, s_misc + 1);
         int prev_ti = -1;
         for (int it = P.begin; it < P.end; ++it) {
           const int ti = it / P.tiles;
           const int n_pass = (t_end[ti] - t_begin[ti] + tok_pass - 1) / tok_pass;
-          for (int pass = 0; pass < n_pass; ++pass) {
+          for (int pass = (it == P.begin ? P.pb : 0); pass < (it == P.end - 1 ? min(n_pass, P.pe) : n_pass); ++pass) {
             // The scale factors of the term rows (tensor memory) are shared by consecutive items of an expert whose
             // rows fit one pass; otherwise every (item, pass) has its own.  The scale warps follow the same rule.
             const bool new_operand = (prev_ti != ti) || (n_pass > 1);
@@ -650,7 +707,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     int cs = 0, slot = 0;
     uint32_t cph = 0, sfree_ph = 0, afree_ph = 0;
     bool first_op = true;
-    for (int phase = 0; phase < 2; ++phase) {
+    for (int phase = a.ph_lo; phase < a.ph_hi; ++phase) {
       const Phase P = phase_of(phase, a, s_misc + 1);
       const int n_blk = P.K / 32;
       const uint8_t* src_sf = phase == 0 ? (kFused ? f.sf1 : a.sf1) : a.sf2;
@@ -659,7 +716,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         const int ti = it / P.tiles;
         const int row_begin = t_begin[ti], row_end = t_end[ti];
         const int n_pass = (row_end - row_begin + tok_pass - 1) / tok_pass;
-        for (int pass = 0; pass < n_pass; ++pass) {
+        for (int pass = (it == P.begin ? P.pb : 0); pass < (it == P.end - 1 ? min(n_pass, P.pe) : n_pass); ++pass) {
           const bool new_operand = (prev_ti != ti) || (n_pass > 1);
           prev_ti = ti;
           if (new_operand) {
@@ -678,13 +735,13 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             }
             const bool by_token = kFused && phase == 0;  // the tokens' scale bytes are stored by token, not by sorted row
             const int row0 = row_begin + pass * tok_pass;
-            const int n_rows = min(tok_pass, row_end - row0) * kTerms;  // term rows that exist
-            const bool rep = P.rep_ok && n_rows <= kRepTok * kTerms;    // the operand repeats in every lane quadrant
+            const int n_rows = min(tok_pass, row_end - row0) * nt;  // operand rows that exist
+            const bool rep = !kQ && P.rep_ok && n_rows <= kRepTok * kTerms;  // the operand repeats in every lane quadrant
             // rows are n_blk bytes each and consecutive: one contiguous range, copied 16 bytes at a time
             // (the 16-byte chunks of a row are XOR-swizzled with the row number against bank conflicts)
             const int n_chunk = n_blk / 16, cmask = min(n_chunk, 8) - 1;
             const int n_vec = n_rows * n_chunk;
-            const uint4* src = reinterpret_cast<const uint4*>(src_sf + static_cast<size_t>(row0) * kTerms * n_blk);
+            const uint4* src = reinterpret_cast<const uint4*>(src_sf + static_cast<size_t>(row0) * nt * n_blk);
             for (int i = st; i < n_vec; i += 128) {
               const int r = i / n_chunk, c = i % n_chunk;
               const uint4* from = by_token ? reinterpret_cast<const uint4*>(src_sf) + (s_tok[row0 + (r >> 3)] * kTerms + (r & 7)) * n_chunk + c
@@ -863,18 +920,103 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         }
       }
     };
-    for (int sweep = 0; sweep < 2; ++sweep) {  // sweep 0 is the dry run of this CTA's first pass, through the one call site below
+    // Quantised-activation variant: accumulator lane = operand row = token.  The warp of quadrant q owns tokens
+    // 32q..32q+31 of the pass and all 256 columns of theirs; nothing is summed across lanes.
+    auto run_pass_q = [&](const int phase, const int out_stride, const int tile, const int row0, const int n_tok) {
+      const bool active = 32 * q < n_tok;
+      const int tok = 32 * q + lane;
+      const bool live = tok < n_tok;
+      mbar_wait(acc_full, acc_ph, a.status);
+      acc_ph ^= 1u;
+      __syncwarp();  // tcgen05.ld is warp-collective
+      tc_fence_after_sync();
+      if (phase == 0) {
+        // columns 0..127 gate, 128..255 up of i = tile * 128 + column; SwiGLU and the rounding to bf16 while the
+        // accumulator is read (two values per register), its quantisation after the accumulator is handed back
+        uint32_t pk[64];
+        if (active) {
+#pragma unroll
+          for (int b = 0; b < 4; ++b) {
+            uint32_t g[32], u[32];
+            tmem_ld_32x32(tmem_base + lane_base + kColD + static_cast<uint32_t>(32 * b), g);
+            tmem_ld_32x32(tmem_base + lane_base + kColD + static_cast<uint32_t>(32 * (4 + b)), u);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const float g0 = __uint_as_float(g[2 * j]), g1 = __uint_as_float(g[2 * j + 1]);
+              const float v0 = __fdividef(g0, 1.0f + __expf(-g0)) * __uint_as_float(u[2 * j]);
+              const float v1 = __fdividef(g1, 1.0f + __expf(-g1)) * __uint_as_float(u[2 * j + 1]);
+              const __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);  // the intermediate is defined as a bf16 value
+              pk[16 * b + j] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+          }
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_empty);  // the rest overlaps the next pass's MMAs
+        if (!active) return;
+        const int n_blk_i = a.I / 32;
+        uint8_t* qrow = a.aq2 + static_cast<size_t>(row0 + tok) * (a.I / 2) + tile * 64;
+        uint8_t* srow = a.sf2 + static_cast<size_t>(row0 + tok) * n_blk_i + tile * 4;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {  // one block of 32 consecutive i: block scale, then 32 codes = 16 bytes
+          float amax = 0.0f;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const uint32_t w = pk[16 * b + j];
+            amax = fmaxf(amax, fmaxf(fabsf(__uint_as_float(w << 16)), fabsf(__uint_as_float(w & 0xFFFF0000u))));
+          }
+          const int se = (amax > 0.0f) ? term_exp(amax) : 0;
+          const float inv = pow2f(-se);
+          uint32_t w4[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const uint32_t w = pk[16 * b + j];
+            float qa, qb;
+            w4[j >> 2] |= e2m1_pair(__uint_as_float(w << 16) * inv, __uint_as_float(w & 0xFFFF0000u) * inv, &qa, &qb) << (8 * (j & 3));
+          }
+          if (live) {
+            *reinterpret_cast<uint4*>(qrow + 16 * b) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+            srow[b] = static_cast<uint8_t>(se + 127);
+          }
+        }
+      } else {
+        if (active) {
+          float* dst = a.y + static_cast<size_t>(row0 + tok) * out_stride + tile * kTile;
+#pragma unroll 1
+          for (int m = 0; m < 8; ++m) {
+            uint32_t v[32];
+            tmem_ld_32x32(tmem_base + lane_base + kColD + static_cast<uint32_t>(32 * m), v);
+            tmem_ld_wait();
+            if (live) {
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<float4*>(dst + 32 * m + 4 * j) =
+                    make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
+                                __uint_as_float(v[4 * j + 3]));
+            }
+          }
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_empty);
+      }
+    };
+    for (int sweep = kQ ? 1 : 0; sweep < 2; ++sweep) {  // sweep 0 is the dry run of this CTA's first pass, through the one call site below
       const bool dry = sweep == 0;
-      for (int phase = 0; phase < (dry ? 1 : 2); ++phase) {
+      for (int phase = dry ? 0 : a.ph_lo; phase < (dry ? 1 : a.ph_hi); ++phase) {
         const Phase P = phase_of(phase, a, s_misc + 1);
         const int it_end = dry ? min(P.begin + 1, P.end) : P.end;
         for (int it = P.begin; it < it_end; ++it) {
           const int ti = it / P.tiles, tile = it % P.tiles;
           const int row_begin = t_begin[ti], row_end = t_end[ti];
           const int n_pass = dry ? 1 : (row_end - row_begin + tok_pass - 1) / tok_pass;
-          for (int pass = 0; pass < n_pass; ++pass) {
+          for (int pass = (it == P.begin ? P.pb : 0); pass < (it == P.end - 1 ? min(n_pass, P.pe) : n_pass); ++pass) {
             const int row0 = row_begin + pass * tok_pass;
-            run_pass(phase, P.rep_ok, P.R, tile, row0, min(tok_pass, row_end - row0), dry);
+            if constexpr (kQ)
+              run_pass_q(phase, P.R, tile, row0, min(tok_pass, row_end - row0));
+            else
+              run_pass(phase, P.rep_ok, P.R, tile, row0, min(tok_pass, row_end - row0), dry);
           }
           if constexpr (kFused) {
             if (!dry && phase == 1) {
@@ -969,7 +1111,8 @@ bool nat_attr_once() {
   static PerDeviceFlag flag;
   return once_per_device(flag, [] {
     return cudaFuncSetAttribute(ffn_native_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess &&
-           cudaFuncSetAttribute(ffn_native_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
+           cudaFuncSetAttribute(ffn_native_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess &&
+           cudaFuncSetAttribute(ffn_native_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
   });
 }
 }  // namespace
@@ -1006,32 +1149,42 @@ bool weight_maps(const ExpertWeights& w, const moe_shape_t& sh, CUtensorMap* tm_
          nat_map(tm_s2, w.s2, sh.I / 32, r2, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
 }
 
+bool native_q_shape_ok(const moe_shape_t& sh, const void* w13, const void* w2) {
+  return sh.H <= kMaxK && sh.I <= kMaxK && sh.H % 512 == 0 && sh.I % 512 == 0 &&
+         (reinterpret_cast<uintptr_t>(w13) & 15u) == 0 && (reinterpret_cast<uintptr_t>(w2) & 15u) == 0 &&
+         nat_smem(sh.E, sh.H > sh.I ? sh.H : sh.I).total + 1024 <= 227 * 1024;
+}
+
 bool native_shape_ok(const moe_shape_t& sh, const void* w13, const void* w2) {
   return native_batch_ok(sh) && sh.H <= kMaxK && sh.I <= kMaxK && sh.H % 512 == 0 && sh.I % 512 == 0 &&
          (reinterpret_cast<uintptr_t>(w13) & 15u) == 0 && (reinterpret_cast<uintptr_t>(w2) & 15u) == 0 &&
          nat_smem(sh.E, sh.H > sh.I ? sh.H : sh.I).total + 1024 <= 227 * 1024;
 }
 
-int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& sh,
-                             void* scratch, float* y_perm, StatusRef status, cudaStream_t st) {
+namespace {
+// kQ: the quantised-activation variant (one operand row per token instead of kTerms)
+template <bool kQ>
+int launch_native_ffn(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& sh,
+                      void* scratch, float* y_perm, StatusRef status, cudaStream_t st) {
   if (!nat_attr_once()) return MOE_ERR_CUDA;
   const size_t S = static_cast<size_t>(sh.T) * sh.k;
-  // scratch: term rows of the intermediate and of the token rows, each followed by its scale bytes; the counters
+  const size_t rows = S * (kQ ? 1 : kTerms);  // operand rows
+  // scratch: operand rows of the intermediate and of the token rows, each followed by its scale bytes; the counters
   uint8_t* aq2 = static_cast<uint8_t*>(scratch);
-  uint8_t* sf2 = aq2 + align_up(S * kTerms * (sh.I / 2), kAlign);
-  uint8_t* aq1 = sf2 + align_up(S * kTerms * (sh.I / 32), kAlign);
-  uint8_t* sf1 = aq1 + align_up(S * kTerms * (sh.H / 2), kAlign);
-  int* done = reinterpret_cast<int*>(sf1 + align_up(S * kTerms * (sh.H / 32), kAlign));
+  uint8_t* sf2 = aq2 + align_up(rows * (sh.I / 2), kAlign);
+  uint8_t* aq1 = sf2 + align_up(rows * (sh.I / 32), kAlign);
+  uint8_t* sf1 = aq1 + align_up(rows * (sh.H / 2), kAlign);
+  int* done = reinterpret_cast<int*>(sf1 + align_up(rows * (sh.H / 32), kAlign));
   CUtensorMap tm_w13, tm_w2, tm_s13, tm_s2;
   TermMaps tm_a1, tm_a2;
   for (int i = 0; i < kTermBoxes; ++i)
-    if (!nat_map(&tm_a1.box[i], aq1, sh.H / 2, S * kTerms, 128, 8u << i, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !nat_map(&tm_a2.box[i], aq2, sh.I / 2, S * kTerms, 128, 8u << i, CU_TENSOR_MAP_SWIZZLE_128B))
+    if (!nat_map(&tm_a1.box[i], aq1, sh.H / 2, rows, 128, 8u << i, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !nat_map(&tm_a2.box[i], aq2, sh.I / 2, rows, 128, 8u << i, CU_TENSOR_MAP_SWIZZLE_128B))
       return MOE_ERR_CUDA;
   if (!weight_maps(w, sh, &tm_w13, &tm_s13, &tm_w2, &tm_s2)) return MOE_ERR_CUDA;
   const size_t split_threads = S * (sh.H / 32) * 8 > static_cast<size_t>(sh.E) ? S * (sh.H / 32) * 8 : static_cast<size_t>(sh.E);
-  if (launch_pdl(native_split_kernel, dim3(static_cast<unsigned>((split_threads + 1023) / 1024)), dim3(1024), 0, st, x_perm, aq1, sf1,
-                 done, static_cast<int>(S), sh.H, sh.E, status.own ? status.word : nullptr) != cudaSuccess)
+  if (launch_pdl(native_split_kernel<kQ>, dim3(static_cast<unsigned>((split_threads + 1023) / 1024)), dim3(1024), 0, st, x_perm, aq1,
+                 sf1, done, static_cast<int>(S), sh.H, sh.E, status.own ? status.word : nullptr) != cudaSuccess)
     return MOE_ERR_CUDA;
   NatArgs a;
   a.sf1 = sf1;
@@ -1047,12 +1200,29 @@ int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, co
   a.I = sh.I;
   a.S = static_cast<int>(S);
   a.blocked = w.blocked ? 1 : 0;
-  if (launch_pdl(ffn_native_kernel<false>, dim3(sm_count()), dim3(kNatThreads),
-                 nat_smem(sh.E, sh.H > sh.I ? sh.H : sh.I).total + 1024, st, tm_w13, tm_s13, tm_a1, tm_w2, tm_s2, tm_a2, a,
-                 FusedArgs{}) != cudaSuccess)
-    return MOE_ERR_CUDA;
-  note_kernel("ffn_native_mxf4_block_scaled", 2);
+  // Batches whose experts have several passes: one launch per projection, shares balanced by passes (see pass_shares)
+  const bool two = kQ && S > static_cast<size_t>(kQOneLaunchRows) * sh.E;
+  a.by_pass = two ? 1 : 0;
+  for (int l = 0; l < (two ? 2 : 1); ++l) {
+    a.ph_lo = two ? l : 0;
+    a.ph_hi = two ? l + 1 : 2;
+    if (launch_pdl(ffn_native_kernel<false, kQ>, dim3(sm_count()), dim3(kNatThreads),
+                   nat_smem(sh.E, sh.H > sh.I ? sh.H : sh.I).total + 1024, st, tm_w13, tm_s13, tm_a1, tm_w2, tm_s2, tm_a2, a,
+                   FusedArgs{}) != cudaSuccess)
+      return MOE_ERR_CUDA;
+  }
+  note_kernel(kQ ? "ffn_native_mxf4_quantised_activations" : "ffn_native_mxf4_block_scaled", two ? 3 : 2);
   return MOE_OK;
+}
+}  // namespace
+
+int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& sh,
+                             void* scratch, float* y_perm, StatusRef status, cudaStream_t st) {
+  return launch_native_ffn<false>(x_perm, offsets, w, sh, scratch, y_perm, status, st);
+}
+int launch_expert_ffn_native_q(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& sh,
+                               void* scratch, float* y_perm, StatusRef status, cudaStream_t st) {
+  return launch_native_ffn<true>(x_perm, offsets, w, sh, scratch, y_perm, status, st);
 }
 
 // ---- the one-launch layer ----
@@ -1106,6 +1276,9 @@ int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const Expe
   a.I = sh.I;
   a.S = static_cast<int>(S);
   a.blocked = w.blocked ? 1 : 0;
+  a.ph_lo = 0;
+  a.ph_hi = 2;
+  a.by_pass = 0;
   FusedArgs f;
   f.logits = logits;
   f.x = x;

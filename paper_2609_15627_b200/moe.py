@@ -55,6 +55,10 @@ def lib():
         L.moe_permute.argtypes = [vp, vp, vp, C.POINTER(Shape), vp, vp, vp, vp, sz, vp]
         L.moe_expert_ffn.restype = C.c_int
         L.moe_expert_ffn.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp, sz, vp]
+        L.moe_expert_ffn_q_workspace_bytes.restype = sz
+        L.moe_expert_ffn_q_workspace_bytes.argtypes = [C.POINTER(Shape)]
+        L.moe_expert_ffn_q.restype = C.c_int
+        L.moe_expert_ffn_q.argtypes = [vp, vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp, sz, vp]
         L.moe_combine.restype = C.c_int
         L.moe_combine.argtypes = [vp, vp, vp, C.POINTER(Shape), vp, vp]
         L.moe_validate_scales.restype = C.c_int
@@ -216,6 +220,23 @@ def moe_prepack(w13, w13_scale, w2, w2_scale, sh, stream=None):
 def moe_expert_ffn_packed(x_perm, expert_offsets, packed, sh, y_perm, status_word, ws, stream=None):
     _check(lib().moe_expert_ffn_packed(_ptr(x_perm), _ptr(expert_offsets), _ptr(packed), C.byref(sh), _ptr(y_perm),
                                        _ptr(status_word), _ptr(ws), ws.numel(), _stream(stream)), "moe_expert_ffn_packed")
+
+
+def alloc_ffn_q_workspace(sh, device="cuda"):
+    n = lib().moe_expert_ffn_q_workspace_bytes(C.byref(sh))
+    if n == 0:
+        raise MoeError("unsupported shape")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def moe_expert_ffn_q(x_perm, expert_offsets, weights, sh, y_perm, status_word, ws, stream=None):
+    """The quantised-activation variant; `weights` is the tuple (w13, w13_scale, w2, w2_scale) or the one tensor
+    written by moe_prepack."""
+    raw = tuple(weights) if isinstance(weights, (tuple, list)) else (None, None, None, None)
+    packed = None if isinstance(weights, (tuple, list)) else weights
+    _check(lib().moe_expert_ffn_q(_ptr(x_perm), _ptr(expert_offsets), _ptr(raw[0]), _ptr(raw[1]), _ptr(raw[2]), _ptr(raw[3]),
+                                  _ptr(packed), C.byref(sh), _ptr(y_perm), _ptr(status_word), _ptr(ws), ws.numel(),
+                                  _stream(stream)), "moe_expert_ffn_q")
 
 
 def moe_forward_packed(logits, x, packed, sh, out, topk_ids, topk_w, status_word, ws, stream=None):
