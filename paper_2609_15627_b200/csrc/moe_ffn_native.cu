@@ -90,7 +90,7 @@ struct NatArgs {
   int E, H, I, S;
   int blocked;               // weights in moe_prepack's tile-contiguous layout (see ExpertWeights)
   int ph_lo, ph_hi;          // projections this launch runs: [0, 2) = both; the large-batch schedule runs one per launch
-  int by_pass;               // large-batch schedule: CTAs get equal numbers of passes, not of items (see unit_shares)
+  int by_pass;               // large-batch schedule: the list of experts is a list of (expert, pass) entries (see the set-up)
 };
 
 // The one-launch layer (moe_forward on a handful of tokens): what the kernel needs beyond the expert FFN's arguments.
@@ -148,7 +148,6 @@ MOE_DEVINL int op_box(int n_rows) { return n_rows <= 8 ? 0 : (n_rows <= 16 ? 1 :
 struct Phase {
   int K, R, n_steps, tiles;  // reduction length, weight rows per expert, K steps, items per expert
   int begin, end;            // this CTA's items (at most 1024 experts x 32 tiles)
-  int pb, pe;                // of item `begin` the passes from pb on, of item `end - 1` the passes before pe
   bool rep_ok;               // few enough of them for single-token passes to be repeated per lane quadrant
 };
 // Items go to CTAs in contiguous shares: gate/up items evenly, per0 each.  A down item of expert t is placed as if it
@@ -182,32 +181,6 @@ __host__ __device__ inline void cta_shares(int grid, int c, int n_touched, int t
   out[2] = total1 == 0 ? 0 : first_down_item_of_cta(c, total1, tiles0, tiles1, per0);
   out[3] = total1 == 0 ? 0 : (c + 1 >= grid ? total1 : first_down_item_of_cta(c + 1, total1, tiles0, tiles1, per0));
 }
-// Large-batch schedule (one projection per launch, so no item waits for another): the passes of all items, in the order
-// (touched expert, tile, pass), are cut into gridDim.x equal contiguous shares - an expert with many rows has many
-// passes per item, and equal item counts would leave its CTAs far behind.  out: first item, item after the last, first
-// pass of the first item, pass after the last of the last item.
-MOE_DEVINL void pass_shares(int grid, int c, int n_touched, const int* t_begin, const int* t_end, int tok_pass, int tiles,
-                            int* out) {
-  long long total = 0;
-  for (int ti = 0; ti < n_touched; ++ti) total += static_cast<long long>((t_end[ti] - t_begin[ti] + tok_pass - 1) / tok_pass) * tiles;
-  const long long lo = total * c / grid, hi = total * (c + 1) / grid;
-  out[0] = out[1] = out[2] = out[3] = 0;
-  if (lo >= hi) return;
-  long long cum = 0;
-  for (int ti = 0; ti < n_touched; ++ti) {
-    const int n_pass = (t_end[ti] - t_begin[ti] + tok_pass - 1) / tok_pass;
-    const long long next = cum + static_cast<long long>(n_pass) * tiles;
-    if (lo >= cum && lo < next) {
-      out[0] = ti * tiles + static_cast<int>((lo - cum) / n_pass);
-      out[2] = static_cast<int>((lo - cum) % n_pass);
-    }
-    if (hi - 1 >= cum && hi - 1 < next) {
-      out[1] = ti * tiles + static_cast<int>((hi - 1 - cum) / n_pass) + 1;
-      out[3] = static_cast<int>((hi - 1 - cum) % n_pass) + 1;
-    }
-    cum = next;
-  }
-}
 MOE_DEVINL Phase phase_of(int ph, const NatArgs& a, const int* shares) {
   Phase p;
   p.K = ph == 0 ? a.H : a.I;
@@ -216,12 +189,12 @@ MOE_DEVINL Phase phase_of(int ph, const NatArgs& a, const int* shares) {
   p.tiles = p.R / kTile;
   p.begin = shares[2 * ph];
   p.end = shares[2 * ph + 1];
-  p.pb = shares[5 + 2 * ph];  // (shares[4] is another word of the set-up)
-  p.pe = shares[6 + 2 * ph];
   p.rep_ok = p.end - p.begin <= kRepMaxItems;
   return p;
 }
 
+// entries of the list of experts with rows that a CTA keeps
+__host__ __device__ inline int touched_cap(int E) { return E > 32 ? E : 32; }
 struct NatSmem {
   uint32_t act, w, sc, sfa, bars, misc, touched, route, total;
 };
@@ -240,7 +213,7 @@ __host__ __device__ inline NatSmem nat_smem(int E, int K) {
   m.misc = off;
   off += 64;
   m.touched = off;  // touched experts: id, first row, end row
-  off += (3 * static_cast<uint32_t>(E) + 16) * 4;
+  off += (3 * static_cast<uint32_t>(touched_cap(E)) + 8) * 4;
   m.route = off;    // one-launch layer: expert and weight of every slot, sorted row of every slot, row of (touched expert, token)
   off += 4 * kFusedMaxSlots * 4;
   m.total = off;
@@ -314,9 +287,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   uint64_t* ctr_done = act_free + 1;             // one-launch layer: epilogue warps that are through with the global counters
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + sm.misc);
   int* touched = reinterpret_cast<int*>(smem + sm.touched);  // ids of the experts that have rows
-  int* t_begin = touched + a.E;                              // their first sorted row
-  int* t_end = t_begin + a.E;                                // and the row after their last
-  int* s_misc = t_end + a.E;
+  int* t_begin = touched + touched_cap(a.E);                 // their first sorted row
+  int* t_end = t_begin + touched_cap(a.E);                   // and the row after their last
+  int* s_misc = t_end + touched_cap(a.E);
   int* s_ids = reinterpret_cast<int*>(smem + sm.route);                 // [T * k] expert of every slot (one-launch layer only)
   float* s_w = reinterpret_cast<float*>(s_ids + kFusedMaxSlots);        // [T * k] routing weight
   int* s_row = reinterpret_cast<int*>(s_w + kFusedMaxSlots);            // [T * k] sorted row of every slot
@@ -339,7 +312,52 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       prefetch_tmap(&tmap_a2.box[i]);
     }
   }
-  if (!kFused && wid == 2) {
+  if (!kFused && a.by_pass && wid == 2) {
+    // Large-batch schedule (one projection per launch, so no item waits for another).  An expert with many rows would
+    // make its items many passes long, and equal item counts would leave its CTAs far behind.  So the list of experts
+    // becomes a list of (expert, pass) entries of at most tok_pass rows each: every item is one pass, consecutive items
+    // of an entry share the operand's scale factors in tensor memory, and equal item counts are equal work.  A CTA
+    // keeps only the entries its own items belong to.
+    const int tiles = a.ph_lo == 0 ? 2 * a.I / kTile : a.H / kTile;
+    const int n_it = (a.E + 31) / 32;
+    int n_ent = 0;
+    for (int i = 0; i < n_it; ++i) {
+      const int e = i * 32 + lane;
+      const int rows = (e < a.E) ? __ldg(a.offsets + e + 1) - __ldg(a.offsets + e) : 0;
+      int tot;
+      warp_excl_scan((rows + tok_pass - 1) / tok_pass, lane, &tot);
+      n_ent += tot;
+    }
+    const long long total = static_cast<long long>(n_ent) * tiles;
+    const long long per = (total + gridDim.x - 1) / gridDim.x;
+    const long long begin = min(static_cast<long long>(blockIdx.x) * per, total), end = min(begin + per, total);
+    const int v_lo = static_cast<int>(begin / tiles);
+    const int v_hi = end > begin ? static_cast<int>((end - 1) / tiles) + 1 : v_lo;
+    int run = 0;
+    for (int i = 0; i < n_it; ++i) {
+      const int e = i * 32 + lane;
+      const int lo = (e < a.E) ? __ldg(a.offsets + e) : 0;
+      const int hi = (e < a.E) ? __ldg(a.offsets + e + 1) : 0;
+      const int v = (hi - lo + tok_pass - 1) / tok_pass;
+      int tot;
+      const int first = run + warp_excl_scan(v, lane, &tot);
+      for (int vi = max(first, v_lo); vi < min(first + v, v_hi); ++vi) {
+        const int idx = vi - v_lo;
+        if (idx < touched_cap(a.E)) {  // (the host chooses this schedule only where the window fits)
+          touched[idx] = e;
+          t_begin[idx] = lo + (vi - first) * tok_pass;
+          t_end[idx] = min(hi, lo + (vi - first + 1) * tok_pass);
+        }
+      }
+      run += tot;
+    }
+    if (lane == 0) {
+      s_misc[0] = v_hi - v_lo;
+      s_misc[1] = s_misc[2] = s_misc[3] = s_misc[4] = 0;
+      s_misc[1 + 2 * a.ph_lo] = static_cast<int>(begin - static_cast<long long>(v_lo) * tiles);
+      s_misc[2 + 2 * a.ph_lo] = static_cast<int>(end - static_cast<long long>(v_lo) * tiles);
+    }
+  } else if (!kFused && wid == 2) {
     // lane l looks at experts l, l + 32, ...: all loads are issued before any is used (one memory round trip);
     // the second loop's loads hit L1.  expert_offsets was complete before the permute kernel let this chain start.
     const int n_it = (a.E + 31) / 32;
@@ -364,23 +382,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       }
       run += tot;
     }
-    __syncwarp();
     if (lane == 0) {
       s_misc[0] = run;
       cta_shares(static_cast<int>(gridDim.x), static_cast<int>(blockIdx.x), run, 2 * a.I / kTile, a.H / kTile, s_misc + 1);
-      s_misc[6] = s_misc[8] = 0;
-      s_misc[7] = s_misc[9] = 1 << 30;
-      if (a.by_pass) {
-        for (int ph = 0; ph < 2; ++ph) {
-          int r[4];
-          pass_shares(static_cast<int>(gridDim.x), static_cast<int>(blockIdx.x), run, t_begin, t_end, tok_pass,
-                      ph == 0 ? 2 * a.I / kTile : a.H / kTile, r);
-          s_misc[1 + 2 * ph] = r[0];
-          s_misc[2 + 2 * ph] = r[1];
-          s_misc[6 + 2 * ph] = r[2];
-          s_misc[7 + 2 * ph] = r[3];
-        }
-      }
     }
   }
   if (tid == 0) {
@@ -513,8 +517,6 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       if (lane == 0) {
         s_misc[0] = n_t;
         cta_shares(static_cast<int>(gridDim.x), static_cast<int>(blockIdx.x), n_t, 2 * a.I / kTile, a.H / kTile, s_misc + 1);
-        s_misc[6] = s_misc[8] = 0;
-        s_misc[7] = s_misc[9] = 1 << 30;
       }
     }
     __syncthreads();
@@ -576,7 +578,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             dep_e = e;
             dep_ok = false;
           }
-          for (int pass = (it == P.begin ? P.pb : 0); pass < (it == P.end - 1 ? min(n_pass, P.pe) : n_pass); ++pass) {
+          for (int pass = 0; pass < n_pass; ++pass) {
             const bool by_token = kFused && phase == 0;  // the expert's rows are fetched token by token (at most 4)
             const int bi = op_box(min(tok_pass, n_rows_e - pass * tok_pass) * nt);  // box of 8 << bi operand rows
             const int n_rep = (!kQ && P.rep_ok && bi <= kRepBox) ? 4 : 1;
@@ -659,7 +661,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         for (int it = P.begin; it < P.end; ++it) {
           const int ti = it / P.tiles;
           const int n_pass = (t_end[ti] - t_begin[ti] + tok_pass - 1) / tok_pass;
-          for (int pass = (it == P.begin ? P.pb : 0); pass < (it == P.end - 1 ? min(n_pass, P.pe) : n_pass); ++pass) {
+          for (int pass = 0; pass < n_pass; ++pass) {
             // The scale factors of the term rows (tensor memory) are shared by consecutive items of an expert whose
             // rows fit one pass; otherwise every (item, pass) has its own.  The scale warps follow the same rule.
             const bool new_operand = (prev_ti != ti) || (n_pass > 1);
@@ -716,7 +718,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         const int ti = it / P.tiles;
         const int row_begin = t_begin[ti], row_end = t_end[ti];
         const int n_pass = (row_end - row_begin + tok_pass - 1) / tok_pass;
-        for (int pass = (it == P.begin ? P.pb : 0); pass < (it == P.end - 1 ? min(n_pass, P.pe) : n_pass); ++pass) {
+        for (int pass = 0; pass < n_pass; ++pass) {
           const bool new_operand = (prev_ti != ti) || (n_pass > 1);
           prev_ti = ti;
           if (new_operand) {
@@ -1011,7 +1013,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
           const int ti = it / P.tiles, tile = it % P.tiles;
           const int row_begin = t_begin[ti], row_end = t_end[ti];
           const int n_pass = dry ? 1 : (row_end - row_begin + tok_pass - 1) / tok_pass;
-          for (int pass = (it == P.begin ? P.pb : 0); pass < (it == P.end - 1 ? min(n_pass, P.pe) : n_pass); ++pass) {
+          for (int pass = 0; pass < n_pass; ++pass) {
             const int row0 = row_begin + pass * tok_pass;
             if constexpr (kQ)
               run_pass_q(phase, P.R, tile, row0, min(tok_pass, row_end - row0));
@@ -1201,7 +1203,10 @@ int launch_native_ffn(const __nv_bfloat16* x_perm, const int* offsets, const Exp
   a.S = static_cast<int>(S);
   a.blocked = w.blocked ? 1 : 0;
   // Batches whose experts have several passes: one launch per projection, shares balanced by passes (see pass_shares)
-  const bool two = kQ && S > static_cast<size_t>(kQOneLaunchRows) * sh.E;
+  // (a CTA's window of (expert, pass) entries must fit the list it keeps: its items / tiles + 2 entries at most)
+  const size_t ent_max = S / (kQ ? 128 : kMaxTokPass) + sh.E, grid_n = static_cast<size_t>(sm_count());
+  const bool two = kQ && S > static_cast<size_t>(kQOneLaunchRows) * sh.E &&
+                   (ent_max + grid_n - 1) / grid_n + 3 <= static_cast<size_t>(touched_cap(sh.E));
   a.by_pass = two ? 1 : 0;
   for (int l = 0; l < (two ? 2 : 1); ++l) {
     a.ph_lo = two ? l : 0;
