@@ -35,6 +35,7 @@ METRIC = "MoE FP4 layer tokens/s"
 DECODE = ("decode_c1", "decode_c64")
 PRODUCTION = ("decode_c1", "decode_c64", "prefill_8k", "prefill_32k_skewed")
 HEADLINE = "decode_c1"
+QUANT_WORKLOADS = ("decode_c64", "prefill_8k", "prefill_32k_skewed")  # also timed with moe_expert_ffn_q
 MIN_REGION_MS = 100.0   # a timed round of a decode workload lasts at least this long
 MIN_REGION_MS_PREFILL = 40.0  # prefill rounds: at least this long and at least 3 steps - a burst-length region, to go with
                               # the burst bf16 peak they are divided by (a single sub-millisecond GEMM, best of ten)
@@ -345,6 +346,112 @@ class Bench:
         return {"ms_per_step": ms, "value": wl.T * self.world / (ms * 1e-3), "unit": "tokens/s", "steps": n,
                 "gpu_launches_per_step": launches_per_step, "call": "moe_ffn_block (row-layout weights)",
                 "launch": ("cuda graph replay, %d steps per graph" % GRAPH_STEPS) if decode else "eager"}
+
+    def run_quant(self, wl, min_ms=50.0):
+        """The quantised-activation variant (moe_expert_ffn_q in place of moe_expert_ffn in the four calls) on the weights
+        already resident: one round of at least min_ms of whole steps, and the FFN call between its own events in eager
+        steps.  Roofline of the call: HBM bytes for decode batches; for prefill batches the FP4 tensor peak (the
+        measured bf16 peak times the nominal ratio of 4)."""
+        torch, moe, inputs = self.torch, self.moe, self.inputs
+        stream = self.stream
+        decode = wl.name in DECODE
+        weights = self.packed if self.packed is not None else self.weights
+        sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
+        n_cycle = 32 if decode else 2
+        batches = [(self.dev(inputs.make_logits(wl.T, wl.E, 7000 + self.rank * 100 + i, wl.skew)),
+                    self.dev(inputs.make_x(wl.T, wl.H, 7000 + self.rank * 100 + i))) for i in range(n_cycle)]
+        buf = moe.LayerBuffers(sh)
+        qws = moe.alloc_ffn_q_workspace(sh)
+        touched = []
+        for l, x in batches:
+            moe.moe_route(l, wl.k, buf.topk_ids, buf.topk_w, buf.expert_offsets, buf.ws)
+            touched.append(int(np.count_nonzero(np.diff(buf.expert_offsets.cpu().numpy()))))
+
+        def step(i, ev=None, st=stream):
+            l, x = batches[i % n_cycle]
+            moe.moe_route(l, wl.k, buf.topk_ids, buf.topk_w, buf.expert_offsets, buf.ws, st)
+            moe.moe_permute(x, buf.topk_ids, buf.expert_offsets, sh, buf.x_perm, buf.perm, buf.inv_perm, buf.ws, st)
+            if ev is not None:
+                ev[0].record(st)
+            moe.moe_expert_ffn_q(buf.x_perm, buf.expert_offsets, weights, sh, buf.y_perm, buf.status, qws, st)
+            if ev is not None:
+                ev[1].record(st)
+            moe.moe_combine(buf.y_perm, buf.inv_perm, buf.topk_w, sh, buf.out, st)
+
+        c0 = moe.moe_launch_count()
+        step(0)
+        launches_per_step = moe.moe_launch_count() - c0
+        for i in range(3):
+            step(i)
+        self.barrier()
+        graphs = []
+        if decode:
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            with torch.cuda.stream(side):
+                step(0, None, None)
+            stream.wait_stream(side)
+            self.barrier()
+            for i0 in range(0, n_cycle, GRAPH_STEPS):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    for i in range(i0, i0 + GRAPH_STEPS):
+                        step(i, None, None)
+                graphs.append(g)
+            for g in graphs:
+                g.replay()
+            self.barrier()
+
+        def timed(n, inner=None):
+            e0, e1 = self.events()
+            self.barrier()
+            self.hold()
+            e0.record(stream)
+            if decode and inner is None:
+                for i in range(n // GRAPH_STEPS):
+                    graphs[i % len(graphs)].replay()
+            else:
+                for i in range(n):
+                    step(i, inner[i] if inner is not None else None)
+            e1.record(stream)
+            self.barrier()
+            return max_over_ranks(e0.elapsed_time(e1), self.world)
+
+        pilot_n = GRAPH_STEPS if decode else 2
+        pilot = timed(pilot_n) / pilot_n
+        n = steps_for_region(pilot, min_ms, multiple=GRAPH_STEPS if decode else 1, at_least=3)
+        time.sleep(COOLDOWN_S)
+        ms = timed(n) / n
+        n_e = min(n, 64)
+        inner = [self.events() for _ in range(n_e)]
+        timed(n_e, inner)
+        ffn_ms = float(np.mean([a.elapsed_time(b) for a, b in inner]))
+        assert int(buf.status.item()) == 0, "device-side wait timed out"
+        peaks = self.peaks
+        mean_touched = float(np.mean(touched))
+        if decode:
+            # weights of the touched experts once, token rows in, fp32 rows out; the quantised rows are 1/4 of the bf16 ones
+            alg = ffn_algorithmic_bytes(wl, mean_touched)
+            achieved = alg / (ffn_ms * 1e-3) / 1e9
+            roof = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"],
+                    "traffic": None, "algorithmic_bytes": alg, "ms": ffn_ms, "peak_source": peaks["source"]}
+        else:
+            achieved = ffn_flops(wl) / (ffn_ms * 1e-3) / 1e12
+            peak = 4.0 * peaks["tensor_burst"]
+            roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                    "traffic": None, "ms": ffn_ms,
+                    "peak_source": "4 x the measured bf16 burst peak (nominal FP4 : bf16 ratio); " + peaks["source"]}
+        roof.update({"kernel": "moe_expert_ffn_q", "experts_touched": mean_touched,
+                     "timed_in": "CUDA events around the call in eager steps right after the timed round"})
+        kernels = moe.moe_last_kernel_name()
+        del graphs, batches, buf, qws
+        torch.cuda.empty_cache()
+        return {"ms_per_step": ms, "value": wl.T * self.world / (ms * 1e-3), "unit": "tokens/s", "steps": n,
+                "gpu_launches_per_step": launches_per_step, "roofline": roof,
+                "call": "moe_route, moe_permute, moe_expert_ffn_q, moe_combine",
+                "launch": ("cuda graph replay, %d steps per graph" % GRAPH_STEPS) if decode else "eager",
+                "numerics": "E2M1 activations with one E8M0 scale per 32 elements: a different result from the bf16-activation "
+                            "workloads (its own oracle), about 0.2 of the output norm away"}
 
     def read_only_stream(self, status):
         """Read-only ceiling: the decode kernel's load mechanism alone over the resident gate/up weights (2.1 GB at
@@ -700,6 +807,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="decode workloads: launch the calls eagerly instead of replaying CUDA graphs")
     ap.add_argument("--no-block", action="store_true", help="skip the timing of moe_ffn_block")
+    ap.add_argument("--no-quant", action="store_true", help="skip the quantised-activation variant (moe_expert_ffn_q)")
     ap.add_argument("--four-calls", action="store_true", help="time the four calls even where moe_forward is one launch")
     ap.add_argument("--raw-weights", action="store_true", help="read the weights in the checkpoint's row layout instead of moe_prepack's tiles")
     args = ap.parse_args()
@@ -746,10 +854,13 @@ def main():
         block = {n: bench.run_block(inputs.WORKLOADS[n]) for n in ("decode_c1", "decode_c64", "prefill_8k")}
         bench.raw = None
         torch.cuda.empty_cache()
-    records = {}
+    records, quant = {}, {}
     for name in names:
         wl = inputs.WORKLOADS[name]
         records[name] = bench.run(wl, exact_steps=args.steps if name == head.name else None, warmup=args.warmup)
+        # the quantised-activation variant of the same workload, on the weights this workload has just loaded
+        if world == 1 and not args.no_quant and name in QUANT_WORKLOADS:
+            quant[name + "_q"] = bench.run_quant(wl)
     hr = records[head.name]
     ex = hr.pop("exact")
 
@@ -791,6 +902,7 @@ def main():
             "clocks": ex["clocks"], "kernels": hr["kernels"],
             "workloads": {n: {k: v for k, v in r.items() if k not in ("one_launch", "n_cycle")} for n, r in records.items()},
             "ffn_block": block,
+            "quantised_activations": quant or None,
             "protocol": ("headline: one region of exactly --steps steps; workloads: %d rounds of at least %d ms (decode) / %d ms "
                          "(prefill) each, %.1f s idle before every round, median reported, every round kept; every region is "
                          "bracketed by a barrier and a synchronize, timed by CUDA events on the launching stream behind a "

@@ -1,0 +1,183 @@
+"""GPU parity of the quantised-activation variant (moe_expert_ffn_q) against its own oracle (oracle.expert_ffn_q).
+
+Tolerance.  Every product of the variant is an E2M1 value times an E2M1 value times a power of two; the fp32 sums of such
+terms are exact, whatever their order, as long as the terms of one sum span fewer than 24 bits - which is the rule on the
+seeded inputs, so most rows are bit-identical to the oracle.  Where a sum does round, the kernel's order may differ from
+the oracle's ascending order by a few units in the last place (relative 1e-6), and such a difference can flip the bf16
+rounding of an intermediate value and, rarely, the E2M1 code it quantises to - one element of a contraction of I, a change
+of up to the block's unit in one of I terms.  The test therefore asks: at least 95 % of the rows within 1e-5 of the row's
+rms, element by element, and every row within 3e-2 of it."""
+import numpy as np
+import pytest
+import torch
+
+from _gpu_util import dev
+from oracle import moe_oracle as O
+from paper_2609_15627_b200 import inputs, moe
+
+pytestmark = pytest.mark.gpu
+
+_INVALID_ARG, _UNSUPPORTED_SHAPE, _WORKSPACE = 1, 2, 3   # moe_status_t
+
+
+def _check_rows(got, want, what):
+    assert not np.isnan(got).any(), what
+    rms = np.sqrt((want.astype(np.float64) ** 2).mean(axis=1, keepdims=True)) + 1e-30
+    rel = (np.abs(got.astype(np.float64) - want) / rms).max(axis=1)
+    assert rel.max() <= 3e-2, (what, float(rel.max()))
+    assert (rel <= 1e-5).mean() >= 0.95, (what, float((rel <= 1e-5).mean()))
+
+
+def _problem(T, H, I, E, k, seed, logits=None):
+    w = inputs.make_expert_weights(H, I, E, seed=seed)
+    x = inputs.make_x(T, H, seed + 1)
+    lg = inputs.make_logits(T, E, seed + 2) if logits is None else logits
+    ids, wt, off = O.route(lg, k)
+    xp, perm, inv = O.permute(x, ids, off)
+    return w, xp, off
+
+
+def _run(w_dev, xp, off, sh, status=True):
+    ws = moe.alloc_ffn_q_workspace(sh)
+    y = torch.full((sh.T * sh.k, sh.H), float("nan"), dtype=torch.float32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda") if status else None
+    moe.moe_expert_ffn_q(dev(xp), dev(off), w_dev, sh, y, st, ws)
+    torch.cuda.synchronize()
+    if status:
+        assert int(st.item()) == 0
+    return y.cpu().numpy()
+
+
+# (T, H, I, E, k): one row; ragged small batch; an expert with three passes of 128 rows (large-batch schedule: one launch per
+# projection); many experts, most of them empty; H != 2I and a long reduction; rows per expert straddling the 64-row
+# boundary between the two schedules
+_CASES = [(1, 512, 512, 4, 2), (7, 512, 1024, 8, 2), (300, 512, 512, 2, 2), (3, 1024, 512, 200, 2), (5, 4096, 1024, 16, 4),
+          (129, 512, 512, 4, 2), (65, 1024, 512, 2, 2)]
+
+
+@pytest.mark.parametrize("case", _CASES)
+@pytest.mark.parametrize("packed", [False, True])
+def test_ffn_q_matches_its_oracle(case, packed):
+    T, H, I, E, k = case
+    w, xp, off = _problem(T, H, I, E, k, seed=sum(case))
+    sh = moe.shape(T, H, I, E, k)
+    wd = tuple(dev(a) for a in w)
+    got = _run(moe.moe_prepack(*wd, sh) if packed else wd, xp, off, sh)
+    _check_rows(got, O.expert_ffn_q(xp, off, *w, k), (case, packed))
+
+
+def test_ffn_q_all_rows_on_one_expert_and_empty_batch_edges():
+    T, H, I, E, k = 200, 512, 512, 6, 1
+    lg = np.full((T, E), -5.0, np.float32)
+    lg[:, 4] = 5.0                                   # every row on expert 4: two passes there, five experts empty
+    w, xp, off = _problem(T, H, I, E, k, seed=3, logits=lg)
+    assert off.tolist() == [0, 0, 0, 0, 0, T, T]
+    sh = moe.shape(T, H, I, E, k)
+    got = _run(tuple(dev(a) for a in w), xp, off, sh)
+    _check_rows(got, O.expert_ffn_q(xp, off, *w, k), "one expert")
+
+
+def test_ffn_q_structured_scales_and_zero_blocks():
+    # scale bytes that depend on (expert, row, block); token rows with all-zero blocks and with one huge element per block
+    T, H, I, E, k = 9, 512, 512, 3, 2
+    w13, s13, w2, s2 = inputs.make_expert_weights(H, I, E, seed=12)
+    s13 = inputs.index_scales(2 * I, H, E)
+    s2 = inputs.index_scales(H, I, E, lo=117)
+    x = inputs.bf16_bits_to_f32(inputs.make_x(T, H, 13)).copy()
+    x[:, 64:96] = 0.0
+    x[2, 128] = 3.0e4
+    x[3, :] = 0.0
+    xb = inputs.f32_to_bf16_bits(x.astype(np.float32))
+    ids, wt, off = O.route(inputs.make_logits(T, E, 14), k)
+    xp, _, _ = O.permute(xb, ids, off)
+    sh = moe.shape(T, H, I, E, k)
+    got = _run(tuple(dev(a) for a in (w13, s13, w2, s2)), xp, off, sh)
+    _check_rows(got, O.expert_ffn_q(xp, off, w13, s13, w2, s2, k), "structured")
+
+
+def test_ffn_q_without_a_status_word_and_replayed_as_a_graph():
+    T, H, I, E, k = 33, 512, 512, 4, 2
+    w, xp, off = _problem(T, H, I, E, k, seed=5)
+    sh = moe.shape(T, H, I, E, k)
+    wd = tuple(dev(a) for a in w)
+    first = _run(wd, xp, off, sh, status=False)
+    _check_rows(first, O.expert_ffn_q(xp, off, *w, k), "no status word")
+    ws = moe.alloc_ffn_q_workspace(sh)
+    xd, od = dev(xp), dev(off)
+    y = torch.empty((T * k, H), dtype=torch.float32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        moe.moe_expert_ffn_q(xd, od, wd, sh, y, st, ws, side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        moe.moe_expert_ffn_q(xd, od, wd, sh, y, st, ws, torch.cuda.current_stream())
+    for _ in range(20):
+        y.fill_(float("nan"))
+        g.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(y.cpu().numpy(), first)
+    assert int(st.item()) == 0
+
+
+def test_ffn_q_argument_checks():
+    T, H, I, E, k = 4, 512, 512, 2, 1
+    w, xp, off = _problem(T, H, I, E, k, seed=1)
+    sh = moe.shape(T, H, I, E, k)
+    wd = tuple(dev(a) for a in w)
+    ws = moe.alloc_ffn_q_workspace(sh)
+    y = torch.empty((T * k, H), dtype=torch.float32, device="cuda")
+    xd, od = dev(xp), dev(off)
+    lib, C = moe.lib(), __import__("ctypes")
+    p = lambda t: None if t is None else C.c_void_p(t.data_ptr())
+    stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    packed = moe.moe_prepack(*wd, sh)
+
+    def call(weights4, pk, shape, ws_t=ws, n=None):
+        return lib.moe_expert_ffn_q(p(xd), p(od), *(p(t) for t in weights4), p(pk), C.byref(shape), p(y), None, p(ws_t),
+                                    ws_t.numel() if n is None else n, stream)
+
+    none4 = (None, None, None, None)
+    assert call(wd, None, sh) == 0 and call(none4, packed, sh) == 0
+    assert call(wd, packed, sh) == _INVALID_ARG          # both forms of the weights
+    assert call(none4, None, sh) == _INVALID_ARG        # neither
+    assert call((wd[0], None, wd[2], wd[3]), None, sh) == _INVALID_ARG
+    assert call(wd, None, sh, n=ws.numel() // 2) == _WORKSPACE
+    assert call(wd, None, moe.shape(T, 384, I, E, k)) == _UNSUPPORTED_SHAPE   # H not a multiple of 512
+    assert call(wd, None, moe.shape(T, H, 256, E, k)) == _UNSUPPORTED_SHAPE
+    torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("name", ["decode_c64", "prefill_8k"])
+def test_ffn_q_at_the_benchmark_shapes_on_sampled_rows(name):
+    """The launch configuration bench.py times (prepacked weights, the library's own routing and permutation), checked on
+    sampled sorted rows: first and last row, rows either side of expert boundaries, random rows."""
+    wl = inputs.WORKLOADS[name]
+    T, H, I, E, k = wl.T, wl.H, wl.I, wl.E, wl.k
+    w = inputs.make_expert_weights(H, I, E, seed=0)
+    sh = moe.shape(T, H, I, E, k)
+    wd = tuple(dev(a) for a in w)
+    packed = moe.moe_prepack(*wd, sh)
+    del wd
+    buf = moe.LayerBuffers(sh)
+    moe.moe_route(dev(inputs.make_logits(T, E, 1, wl.skew)), k, buf.topk_ids, buf.topk_w, buf.expert_offsets, buf.ws)
+    moe.moe_permute(dev(inputs.make_x(T, H, 1)), buf.topk_ids, buf.expert_offsets, sh, buf.x_perm, buf.perm, buf.inv_perm, buf.ws)
+    ws = moe.alloc_ffn_q_workspace(sh)
+    buf.y_perm.fill_(float("nan"))
+    moe.moe_expert_ffn_q(buf.x_perm, buf.expert_offsets, packed, sh, buf.y_perm, buf.status, ws)
+    torch.cuda.synchronize()
+    assert int(buf.status.item()) == 0
+    assert not torch.isnan(buf.y_perm).any()
+    off = buf.expert_offsets.cpu().numpy()
+    S = T * k
+    rng = np.random.default_rng(0)
+    edges = off[np.r_[1:4, E // 2, E - 2]]
+    rows = np.unique(np.clip(np.concatenate([rng.integers(0, S, 40), [0, S - 1], edges - 1, edges, edges + 127, edges + 128]), 0, S - 1))
+    expert_of = np.searchsorted(off, rows, side="right") - 1
+    idx = torch.from_numpy(rows).cuda()
+    xs = np.ascontiguousarray(buf.x_perm[idx].cpu().view(torch.int16).numpy().view(np.uint16))
+    so = np.zeros(E + 1, np.int64)
+    np.add.at(so, expert_of + 1, 1)
+    want = O.expert_ffn_q(xs, np.cumsum(so).astype(np.int32), *w, 1)
+    _check_rows(buf.y_perm[idx].cpu().numpy(), want, name)
