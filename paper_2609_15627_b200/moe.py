@@ -19,7 +19,7 @@ EXPORTS = ("moe_workspace_bytes", "moe_status_string", "moe_last_kernel_name", "
            "moe_expert_ffn_noalloc", "moe_debug_native_cta_share", "moe_debug_read_probe", "moe_prepack_bytes", "moe_prepack",
            "moe_expert_ffn_packed", "moe_forward_packed", "moe_forward_host_packed", "moe_debug_forward_one_launch",
            "moe_debug_expert_ffn_variant", "moe_router_logits", "moe_combine_shared", "moe_ffn_block_workspace_bytes",
-           "moe_ffn_block")
+           "moe_ffn_block", "moe_expert_ffn_q_workspace_bytes", "moe_expert_ffn_q")
 
 
 class MoeError(RuntimeError):
