@@ -984,19 +984,37 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         }
       } else {
         if (active) {
+          // each lane writes its own row: 32 bytes per store where the output allows it (whole sectors), and the next
+          // chunk's tensor-memory load in flight during the stores of the current one
           float* dst = a.y + static_cast<size_t>(row0 + tok) * out_stride + tile * kTile;
-#pragma unroll 1
-          for (int m = 0; m < 8; ++m) {
-            uint32_t v[32];
-            tmem_ld_32x32(tmem_base + lane_base + kColD + static_cast<uint32_t>(32 * m), v);
-            tmem_ld_wait();
-            if (live) {
+          const bool wide = (reinterpret_cast<uintptr_t>(a.y) & 31u) == 0;  // rows are multiples of 2 KB apart
+          auto put = [&](const uint32_t (&v)[32], int m) {
+            if (!live) return;
+            if (wide) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst + 32 * m + 8 * j), "r"(v[8 * j]),
+                             "r"(v[8 * j + 1]), "r"(v[8 * j + 2]), "r"(v[8 * j + 3]), "r"(v[8 * j + 4]), "r"(v[8 * j + 5]),
+                             "r"(v[8 * j + 6]), "r"(v[8 * j + 7])
+                             : "memory");
+            } else {
 #pragma unroll
               for (int j = 0; j < 8; ++j)
-                *reinterpret_cast<float4*>(dst + 32 * m + 4 * j) =
-                    make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
-                                __uint_as_float(v[4 * j + 3]));
+                *reinterpret_cast<uint4*>(dst + 32 * m + 4 * j) = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
             }
+          };
+          const uint32_t col = tmem_base + lane_base + kColD;
+          uint32_t va[32], vb[32];
+          tmem_ld_32x32(col, va);
+          tmem_ld_wait();
+#pragma unroll 1
+          for (int m = 0; m < 8; m += 2) {
+            tmem_ld_32x32(col + static_cast<uint32_t>(32 * (m + 1)), vb);
+            put(va, m);
+            tmem_ld_wait();
+            if (m + 2 < 8) tmem_ld_32x32(col + static_cast<uint32_t>(32 * (m + 2)), va);
+            put(vb, m + 1);
+            if (m + 2 < 8) tmem_ld_wait();
           }
         }
         tc_fence_before_sync();
