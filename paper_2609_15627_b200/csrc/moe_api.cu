@@ -550,6 +550,7 @@ size_t moe_forward_host_workspace_bytes(const moe_shape_t* shape) {
 }
 
 namespace {
+constexpr size_t kDirectOutBytes = 64 * 1024;  // outputs up to this size are written to pinned host memory by the kernel
 int forward_host_impl(const float* logits_host, const void* x_host_bf16, const ExpertWeights& w, const moe_shape_t* shape,
                       void* out_host_bf16, int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
   int rc;
@@ -562,6 +563,20 @@ int forward_host_impl(const float* logits_host, const void* x_host_bf16, const E
   float* d_logits = reinterpret_cast<float*>(base + L.logits);
   void* d_x = base + L.x;
   void* d_out = base + L.out;
+  // A small output goes straight to the caller's buffer where the device can address it (pinned host memory under
+  // unified addressing): the last kernel's stores cross the bus instead of a copy operation enqueued after it.
+  bool direct = false;
+  const size_t out_bytes = static_cast<size_t>(s.T) * s.H * 2;
+  if (out_bytes <= kDirectOutBytes) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, out_host_bf16) == cudaSuccess && at.type == cudaMemoryTypeHost &&
+        at.devicePointer != nullptr && aligned(at.devicePointer, 16)) {
+      d_out = at.devicePointer;
+      direct = true;
+    } else {
+      cudaGetLastError();  // pageable memory: not an error of this call
+    }
+  }
   // this call owns its workspace's contents: it clears the sync block of moe_forward itself
   if (cudaMemsetAsync(base + L.inner, 0, kForwardSyncBytes, st) != cudaSuccess ||
       cudaMemcpyAsync(d_logits, logits_host, static_cast<size_t>(s.T) * s.E * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
@@ -570,7 +585,7 @@ int forward_host_impl(const float* logits_host, const void* x_host_bf16, const E
   if ((rc = forward_impl(d_logits, d_x, w, shape, d_out, nullptr, nullptr, status_word, base + L.inner, ws_bytes - L.inner,
                          st)) != MOE_OK)
     return rc;
-  if (cudaMemcpyAsync(out_host_bf16, d_out, static_cast<size_t>(s.T) * s.H * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+  if (!direct && cudaMemcpyAsync(out_host_bf16, d_out, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return MOE_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return MOE_ERR_CUDA;
   return MOE_OK;
