@@ -273,7 +273,7 @@ int moe_ffn_block(const void* x_bf16 /* [T,H] */, const void* w_router_bf16 /* [
  *     the benchmark's inputs: one E2M1 term keeps two to three significant bits); against this variant's own oracle the
  *     result is the same up to fp32 summation order and the roundings that order can flip.
  *   - Weights: the four logical tensors with packed = NULL, or packed = the buffer of moe_prepack with the four NULL.
- *   - Shapes: H and I multiples of 512 and at most 4096; otherwise MOE_ERR_UNSUPPORTED_SHAPE.  Any T * k: one kernel
+ *   - Shapes: H and I multiples of 256 and at most 4096; otherwise MOE_ERR_UNSUPPORTED_SHAPE.  Any T * k: one kernel
  *     serves decode and prefill (a pass holds 128 tokens of an expert, against 16 in moe_expert_ffn's kernel).
  *   - `ws`: moe_expert_ffn_q_workspace_bytes(), 256-byte aligned, no initialisation needed.  Enqueue only, no
  *     allocation, capturable, bounded device-side waits and status_word as moe_expert_ffn.

@@ -48,6 +48,7 @@
 #include <cuda_fp4.h>
 
 #include <algorithm>
+#include <cstring>
 
 #include "moe_mxf4_device.cuh"
 #include "moe_tmap.cuh"
@@ -89,6 +90,8 @@ struct NatArgs {
   int own_status;            // the library's own word: the one-launch kernel's last CTA clears it for the next call
   int E, H, I, S;
   int blocked;               // weights in moe_prepack's tile-contiguous layout (see ExpertWeights)
+  const uint8_t* s13;        // the weights' scale bytes in the row layout, for reductions that are not multiples of 512:
+  const uint8_t* s2;         //   their rows are then not multiples of 16 bytes, which a tensor map cannot address
   int ph_lo, ph_hi;          // projections this launch runs: [0, 2) = both; the large-batch schedule runs one per launch
   int by_pass;               // large-batch schedule: the list of experts is a list of (expert, pass) entries (see the set-up)
 };
@@ -148,6 +151,7 @@ MOE_DEVINL int op_box(int n_rows) { return n_rows <= 8 ? 0 : (n_rows <= 16 ? 1 :
 struct Phase {
   int K, R, n_steps, tiles;  // reduction length, weight rows per expert, K steps, items per expert
   int begin, end;            // this CTA's items (at most 1024 experts x 32 tiles)
+  bool direct;               // K is not a multiple of 512: scale bytes come by plain loads (see NatArgs::s13)
   bool rep_ok;               // few enough of them for single-token passes to be repeated per lane quadrant
 };
 // Items go to CTAs in contiguous shares: gate/up items evenly, per0 each.  A down item of expert t is placed as if it
@@ -186,6 +190,7 @@ MOE_DEVINL Phase phase_of(int ph, const NatArgs& a, const int* shares) {
   p.K = ph == 0 ? a.H : a.I;
   p.R = ph == 0 ? 2 * a.I : a.H;
   p.n_steps = p.K / kKStep;
+  p.direct = (p.K % 512) != 0;
   p.tiles = p.R / kTile;
   p.begin = shares[2 * ph];
   p.end = shares[2 * ph + 1];
@@ -583,7 +588,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             const int bi = op_box(min(tok_pass, n_rows_e - pass * tok_pass) * nt);  // box of 8 << bi operand rows
             const int n_rep = (!kQ && P.rep_ok && bi <= kRepBox) ? 4 : 1;
             for (int ks = 0; ks < P.n_steps; ++ks) {
-              if ((ks & 1) == 0) {  // 16 scale bytes per weight row cover two K steps
+              if (!P.direct && (ks & 1) == 0) {  // 16 scale bytes per weight row cover two K steps
                 mbar_wait(&empty_sc[cs], cph ^ 1u, a.status);
                 mbar_expect_tx(&full_sc[cs], kScStage);
                 // 128 rows x 16 scale bytes; tile-contiguous layout: tile (row / 128, ks / 2) is 128 consecutive rows of 16 bytes
@@ -686,7 +691,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
               }
               umma_commit(&empty_w[s]);
               if (++s == kWStages) { s = 0; ph ^= 1u; }
-              if ((ks & 1) == 1) {
+              if ((ks & 1) == 1 || ks == P.n_steps - 1) {
                 umma_commit(&sf_free[slot]);
                 if (++slot == kSfGroups) { slot = 0; sph ^= 1u; }
               }
@@ -744,6 +749,10 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             const int n_chunk = n_blk / 16, cmask = min(n_chunk, 8) - 1;
             const int n_vec = n_rows * n_chunk;
             const uint4* src = reinterpret_cast<const uint4*>(src_sf + static_cast<size_t>(row0) * nt * n_blk);
+            if (P.direct) {  // rows of n_blk = 8 (mod 16) bytes: 8 bytes at a time, rows plainly one after the other
+              const uint2* src8 = reinterpret_cast<const uint2*>(src_sf + static_cast<size_t>(row0) * nt * n_blk);
+              for (int i = st; i < n_rows * (n_blk / 8); i += 128) reinterpret_cast<uint2*>(sSfa)[i] = __ldcg(src8 + i);
+            } else
             for (int i = st; i < n_vec; i += 128) {
               const int r = i / n_chunk, c = i % n_chunk;
               const uint4* from = by_token ? reinterpret_cast<const uint4*>(src_sf) + (s_tok[row0 + (r >> 3)] * kTerms + (r & 7)) * n_chunk + c
@@ -759,7 +768,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
 #pragma unroll
               for (int c = 0; c < 4; ++c) {
                 const int r = rep ? lane : 32 * c + lane;
-                const uint2 v = *reinterpret_cast<const uint2*>(sSfa + (r * n_chunk + ((ks >> 1) ^ (r & cmask))) * 16 + (ks & 1) * 8);
+                const uint2 v = P.direct ? reinterpret_cast<const uint2*>(sSfa)[r * (n_blk / 8) + ks]
+                                         : *reinterpret_cast<const uint2*>(sSfa + (r * n_chunk + ((ks >> 1) ^ (r & cmask))) * 16 + (ks & 1) * 8);
                 w[c] = v.x;
                 w[4 + c] = v.y;
               }
@@ -772,13 +782,30 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
           }
           // ---- weight scale factors: one scale stage (256 rows x 16 bytes = 2 K steps) -> one 32-column group ----
           for (int ks = 0; ks < P.n_steps; ks += 2) {
-            mbar_wait(&full_sc[cs], cph, a.status);
+            uint4 r[8];
+            if (P.direct) {
+              // 8 scale bytes per weight row and K step, straight from the row layout; issued before the wait below
+              const int e = touched[ti], tile = it % P.tiles;
+              const int wrow_a = phase == 0 ? e * P.R + tile * 128 : e * P.R + tile * kTile;
+              const int wrow_b = phase == 0 ? e * P.R + a.I + tile * 128 : wrow_a + 128;
+              const uint8_t* sc = phase == 0 ? a.s13 : a.s2;
+#pragma unroll
+              for (int c = 0; c < 8; ++c) {
+                const uint2* p = reinterpret_cast<const uint2*>(sc + static_cast<size_t>((c < 4 ? wrow_a : wrow_b) + lane + 32 * (c & 3)) * n_blk) + ks;
+                const uint2 lo = __ldg(p);
+                const uint2 hi = ks + 1 < P.n_steps ? __ldg(p + 1) : make_uint2(0u, 0u);
+                r[c] = make_uint4(lo.x, lo.y, hi.x, hi.y);
+              }
+            } else {
+              mbar_wait(&full_sc[cs], cph, a.status);
+            }
             mbar_wait(&sf_free[slot], sfree_ph ^ 1u, a.status);
             __syncwarp();  // the spins may leave lanes diverged; tcgen05.st is warp-collective
             const unsigned char* blk = sSc + cs * kScStage;
-            uint4 r[8];
+            if (!P.direct) {
 #pragma unroll
-            for (int c = 0; c < 8; ++c) r[c] = *reinterpret_cast<const uint4*>(blk + (lane + 32 * c) * 16);
+              for (int c = 0; c < 8; ++c) r[c] = *reinterpret_cast<const uint4*>(blk + (lane + 32 * c) * 16);
+            }
             // column 8t + c of the group: scale word t (K blocks 4t..4t+3 of the 16) for weight row lane + 32c
             asm volatile(
                 "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
@@ -794,9 +821,9 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             __syncwarp();
             if (lane == 0) {
               mbar_arrive(&sf_full[slot]);
-              mbar_arrive(&empty_sc[cs]);
+              if (!P.direct) mbar_arrive(&empty_sc[cs]);
             }
-            if (++cs == kScStages) { cs = 0; cph ^= 1u; }
+            if (!P.direct && ++cs == kScStages) { cs = 0; cph ^= 1u; }
             if (++slot == kSfGroups) { slot = 0; sfree_ph ^= 1u; }
           }
         }
@@ -1163,20 +1190,23 @@ bool weight_maps(const ExpertWeights& w, const moe_shape_t& sh, CUtensorMap* tm_
            nat_map(tm_w2, w.w2, 128, r2 * (sh.I / 256), 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
            nat_map(tm_s13, w.s13, 16, r13 * (sh.H / 512), 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE) &&
            nat_map(tm_s2, w.s2, 16, r2 * (sh.I / 512), 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
+  // (scale rows that are not multiples of 16 bytes get no tensor map: the kernel loads them itself)
+  std::memset(tm_s13, 0, sizeof(*tm_s13));
+  std::memset(tm_s2, 0, sizeof(*tm_s2));
   return nat_map(tm_w13, w.w13, sh.H / 2, r13, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
          nat_map(tm_w2, w.w2, sh.I / 2, r2, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B) &&
-         nat_map(tm_s13, w.s13, sh.H / 32, r13, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE) &&
-         nat_map(tm_s2, w.s2, sh.I / 32, r2, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE);
+         (sh.H % 512 != 0 || nat_map(tm_s13, w.s13, sh.H / 32, r13, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE)) &&
+         (sh.I % 512 != 0 || nat_map(tm_s2, w.s2, sh.I / 32, r2, 16, 128, CU_TENSOR_MAP_SWIZZLE_NONE));
 }
 
 bool native_q_shape_ok(const moe_shape_t& sh, const void* w13, const void* w2) {
-  return sh.H <= kMaxK && sh.I <= kMaxK && sh.H % 512 == 0 && sh.I % 512 == 0 &&
+  return sh.H <= kMaxK && sh.I <= kMaxK && sh.H % 256 == 0 && sh.I % 256 == 0 &&
          (reinterpret_cast<uintptr_t>(w13) & 15u) == 0 && (reinterpret_cast<uintptr_t>(w2) & 15u) == 0 &&
          nat_smem(sh.E, sh.H > sh.I ? sh.H : sh.I).total + 1024 <= 227 * 1024;
 }
 
 bool native_shape_ok(const moe_shape_t& sh, const void* w13, const void* w2) {
-  return native_batch_ok(sh) && sh.H <= kMaxK && sh.I <= kMaxK && sh.H % 512 == 0 && sh.I % 512 == 0 &&
+  return native_batch_ok(sh) && sh.H <= kMaxK && sh.I <= kMaxK && sh.H % 256 == 0 && sh.I % 256 == 0 &&
          (reinterpret_cast<uintptr_t>(w13) & 15u) == 0 && (reinterpret_cast<uintptr_t>(w2) & 15u) == 0 &&
          nat_smem(sh.E, sh.H > sh.I ? sh.H : sh.I).total + 1024 <= 227 * 1024;
 }
@@ -1220,6 +1250,8 @@ int launch_native_ffn(const __nv_bfloat16* x_perm, const int* offsets, const Exp
   a.I = sh.I;
   a.S = static_cast<int>(S);
   a.blocked = w.blocked ? 1 : 0;
+  a.s13 = w.s13;
+  a.s2 = w.s2;
   // Batches whose experts have several passes: one launch per projection, shares balanced by passes (see pass_shares)
   // (a CTA's window of (expert, pass) entries must fit the list it keeps: its items / tiles + 2 entries at most)
   const size_t ent_max = S / (kQ ? 128 : kMaxTokPass) + sh.E, grid_n = static_cast<size_t>(sm_count());
@@ -1253,7 +1285,7 @@ int launch_expert_ffn_native_q(const __nv_bfloat16* x_perm, const int* offsets, 
 // borrows the shared memory that later holds the term rows' scale bytes.
 bool forward_fused_ok(const moe_shape_t& sh, const void* w13, const void* w2) {
   const int K = sh.H > sh.I ? sh.H : sh.I;
-  return native_shape_ok(sh, w13, w2) && sm_count() >= kSplitCtas && sh.T <= kFusedMaxTok && sh.T * sh.k <= kFusedMaxSlots &&
+  return native_shape_ok(sh, w13, w2) && sh.H % 512 == 0 && sh.I % 512 == 0 && sm_count() >= kSplitCtas && sh.T <= kFusedMaxTok && sh.T * sh.k <= kFusedMaxSlots &&
          static_cast<size_t>(sh.T) * sh.E * 4 <= static_cast<size_t>(128) * (K / 32) && sh.E <= kSyncDone2 &&
          sh.H / kTile <= kSyncExit - kSyncDone2;
 }
@@ -1299,6 +1331,8 @@ int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const Expe
   a.I = sh.I;
   a.S = static_cast<int>(S);
   a.blocked = w.blocked ? 1 : 0;
+  a.s13 = w.s13;
+  a.s2 = w.s2;
   a.ph_lo = 0;
   a.ph_hi = 2;
   a.by_pass = 0;

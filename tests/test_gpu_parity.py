@@ -951,7 +951,7 @@ def test_kernel_choice_is_a_function_of_the_shape():
         assert moe.moe_last_kernel_name() == want
 
 
-# ---- the native block-scaled FP4 expert FFN, reached when T*k <= 32*E (decode-sized) and H, I are multiples of 512 ----
+# ---- the native block-scaled FP4 expert FFN, reached when T*k <= 32*E (decode-sized) and H, I are multiples of 256 ----
 
 @pytest.mark.parametrize("T,H,I,E,k,hot,seed", [
     (16, 512, 512, 8, 2, False, 0),      # a few rows per expert: term-row boxes of 16 to 64 rows
@@ -960,6 +960,10 @@ def test_kernel_choice_is_a_function_of_the_shape():
     (64, 1024, 512, 8, 2, False, 2),     # ~16 rows per expert: 128-row boxes, some experts need two passes of 16 tokens
     (64, 512, 512, 4, 2, False, 5),      # ~32 rows per expert: two or three passes each
     (40, 512, 1024, 8, 1, True, 3),      # one hot expert with most rows, several empty experts
+    (8, 512, 256, 8, 2, False, 6),       # I = 256 (the paper's TP8 shard of the intermediate): one K step in the down
+    (12, 768, 256, 4, 2, False, 7),      #   projection, scale rows of 8 bytes; H = 768: three K steps, rows of 24 bytes
+    (5, 1280, 768, 6, 3, False, 8),      # both reductions odd multiples of 256
+    (33, 4096, 256, 16, 4, False, 9),    # the model's H with the TP8 shard
 ])
 def test_ffn_native_fp4_path_against_oracle(T, H, I, E, k, hot, seed):
     w = inputs.make_expert_weights(H, I, E, seed=seed)

@@ -52,7 +52,7 @@ def _run(w_dev, xp, off, sh, status=True):
 # projection); many experts, most of them empty; H != 2I and a long reduction; rows per expert straddling the 64-row
 # boundary between the two schedules
 _CASES = [(1, 512, 512, 4, 2), (7, 512, 1024, 8, 2), (300, 512, 512, 2, 2), (3, 1024, 512, 200, 2), (5, 4096, 1024, 16, 4),
-          (129, 512, 512, 4, 2), (65, 1024, 512, 2, 2)]
+          (129, 512, 512, 4, 2), (65, 1024, 512, 2, 2), (9, 768, 256, 4, 2), (200, 1280, 256, 2, 1)]
 
 
 @pytest.mark.parametrize("case", _CASES)
@@ -144,8 +144,8 @@ def test_ffn_q_argument_checks():
     assert call(none4, None, sh) == _INVALID_ARG        # neither
     assert call((wd[0], None, wd[2], wd[3]), None, sh) == _INVALID_ARG
     assert call(wd, None, sh, n=ws.numel() // 2) == _WORKSPACE
-    assert call(wd, None, moe.shape(T, 384, I, E, k)) == _UNSUPPORTED_SHAPE   # H not a multiple of 512
-    assert call(wd, None, moe.shape(T, H, 256, E, k)) == _UNSUPPORTED_SHAPE
+    assert call(wd, None, moe.shape(T, 384, I, E, k)) == _UNSUPPORTED_SHAPE   # H not a multiple of 256
+    assert call(wd, None, moe.shape(T, H, 128, E, k)) == _UNSUPPORTED_SHAPE
     torch.cuda.synchronize()
 
 
