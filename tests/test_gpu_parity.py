@@ -935,7 +935,8 @@ def test_ffn_tensor_core_path_against_oracle(T, H, I, E, k, hot, seed):
 
 def test_kernel_choice_is_a_function_of_the_shape():
     for (T, H, I, E, k, want) in [(16, 256, 128, 8, 2, "ffn_stream_bulk_ring_mma16816"),
-                                  (64, 512, 256, 8, 2, "ffn_stream_bulk_ring_mma16816"),
+                                  (64, 512, 256, 8, 2, "ffn_native_mxf4_block_scaled"),   # I = 256: native since H, I % 256
+                                  (64, 512, 384, 8, 2, "ffn_stream_bulk_ring_mma16816"),
                                   (64, 512, 512, 8, 2, "ffn_native_mxf4_block_scaled"),
                                   (512, 512, 512, 8, 2, "ffn_umma_tcgen05_grouped"),
                                   (512, 512, 256, 8, 2, "ffn_stream_bulk_ring_mma16816")]:
