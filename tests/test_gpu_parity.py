@@ -354,7 +354,8 @@ def test_layer_tiny():
 
 @pytest.mark.parametrize("T,H,I,E,k,kernel", [
     (8, 1024, 512, 32, 6, "ffn_native_mxf4_block_scaled"),   # the paper's own top-k (6), decode-sized
-    (24, 512, 256, 16, 6, "ffn_stream_bulk_ring_mma16816"),  # top-6 with I = 256, the paper's TP8 shard of I
+    (24, 512, 256, 16, 6, "ffn_native_mxf4_block_scaled"),   # top-6 with I = 256, the paper's TP8 shard of I
+    (24, 512, 384, 16, 6, "ffn_stream_bulk_ring_mma16816"),  # an I the tensor-core kernels do not take
     (256, 512, 512, 8, 6, "ffn_umma_tcgen05_grouped"),       # top-6, prefill-sized
 ])
 def test_layer_full_with_top6(T, H, I, E, k, kernel):
