@@ -117,8 +117,8 @@ int moe_permute(const void* x_bf16, const int32_t* topk_ids, const int32_t* expe
  * The summation order inside a dot product is the kernel's; everything else is as written.
  *   status_word: device int32, may be NULL; see the common rules.
  * Three kernel variants, chosen by the shape alone (moe_last_kernel_name names the one that ran): for
- * decode-sized batches (T*k <= 32*E and <= 6144; H and I multiples of 512 up to 4096; E up to about 400 at
- * H = 4096, where shared memory runs out) the packed weights feed the block-scaled FP4
+ * decode-sized batches (T*k <= 32*E and <= 6144; H and I multiples of 256 up to 4096 - so also the I = 256 shard of
+ * the paper's TP8 layout; E up to about 400 at H = 4096, where shared memory runs out) the packed weights feed the block-scaled FP4
  * tensor-core instruction directly and each bf16 activation row is written as a sum of eight E2M1 rows with their
  * own block scales (exact for elements within 2^-10 of their 32-block's largest magnitude; the others are off by
  * less than 2^-16 of that magnitude);
