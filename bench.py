@@ -808,6 +808,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="decode workloads: launch the calls eagerly instead of replaying CUDA graphs")
     ap.add_argument("--no-block", action="store_true", help="skip the timing of moe_ffn_block")
     ap.add_argument("--no-quant", action="store_true", help="skip the quantised-activation variant (moe_expert_ffn_q)")
+    ap.add_argument("--only-quant", action="store_true", help="time only the quantised-activation variant of --workload")
+    ap.add_argument("--min-ms", type=float, default=50.0, help="with --only-quant: length of the timed round")
     ap.add_argument("--four-calls", action="store_true", help="time the four calls even where moe_forward is one launch")
     ap.add_argument("--raw-weights", action="store_true", help="read the weights in the checkpoint's row layout instead of moe_prepack's tiles")
     args = ap.parse_args()
@@ -844,6 +846,12 @@ def main():
     moe.lib()
 
     bench = Bench(args, rank, world, local)
+    if args.only_quant:
+        # the variant alone (for a profiler capture: nothing else launches before it but the routing and the load transform)
+        assert world == 1 and head.name in QUANT_WORKLOADS
+        bench.load_weights(head)
+        print(json.dumps({"quantised_activations": {head.name + "_q": bench.run_quant(head, min_ms=args.min_ms)}}))
+        return
     # every rank times the same list, in the same order (the barriers pair up)
     # (replicas, N > 1: the headline workload only - the scaling figure is the headline's)
     names = [args.workload] if args.workload else [HEADLINE] + ([n for n in PRODUCTION if n != HEADLINE] if world == 1 else [])
