@@ -149,7 +149,7 @@ MOE_DEVINL int op_box(int n_rows) { return n_rows <= 8 ? 0 : (n_rows <= 16 ? 1 :
 
 // One projection as the kernel sees it
 struct Phase {
-  int K, R, n_steps, tiles;  // reduction length, weight rows per expert, K steps, items per expert
+  int K, R, n_steps, tiles;  // reduction length, weight rows per expert, K steps, items per entry of the expert list
   int begin, end;            // this CTA's items (at most 1024 experts x 32 tiles)
   bool direct;               // K is not a multiple of 512: scale bytes come by plain loads (see NatArgs::s13)
   bool rep_ok;               // few enough of them for single-token passes to be repeated per lane quadrant
@@ -185,13 +185,15 @@ __host__ __device__ inline void cta_shares(int grid, int c, int n_touched, int t
   out[2] = total1 == 0 ? 0 : first_down_item_of_cta(c, total1, tiles0, tiles1, per0);
   out[3] = total1 == 0 ? 0 : (c + 1 >= grid ? total1 : first_down_item_of_cta(c + 1, total1, tiles0, tiles1, per0));
 }
+// Large-batch schedule: consecutive tiles of one (expert, pass) entry that a CTA takes in one go
+__host__ __device__ inline int block_tiles(int tiles) { return tiles % 4 == 0 ? 4 : (tiles % 2 == 0 ? 2 : 1); }
 MOE_DEVINL Phase phase_of(int ph, const NatArgs& a, const int* shares) {
   Phase p;
   p.K = ph == 0 ? a.H : a.I;
   p.R = ph == 0 ? 2 * a.I : a.H;
   p.n_steps = p.K / kKStep;
   p.direct = (p.K % 512) != 0;
-  p.tiles = p.R / kTile;
+  p.tiles = a.by_pass ? block_tiles(p.R / kTile) : p.R / kTile;
   p.begin = shares[2 * ph];
   p.end = shares[2 * ph + 1];
   p.rep_ok = p.end - p.begin <= kRepMaxItems;
@@ -218,7 +220,7 @@ __host__ __device__ inline NatSmem nat_smem(int E, int K) {
   m.misc = off;
   off += 64;
   m.touched = off;  // touched experts: id, first row, end row
-  off += (3 * static_cast<uint32_t>(touched_cap(E)) + 8) * 4;
+  off += (4 * static_cast<uint32_t>(touched_cap(E)) + 8) * 4;
   m.route = off;    // one-launch layer: expert and weight of every slot, sorted row of every slot, row of (touched expert, token)
   off += 4 * kFusedMaxSlots * 4;
   m.total = off;
@@ -294,7 +296,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   int* touched = reinterpret_cast<int*>(smem + sm.touched);  // ids of the experts that have rows
   int* t_begin = touched + touched_cap(a.E);                 // their first sorted row
   int* t_end = t_begin + touched_cap(a.E);                   // and the row after their last
-  int* s_misc = t_end + touched_cap(a.E);
+  int* t_tile = t_end + touched_cap(a.E);                    // first tile of the entry's items (0 outside the large-batch schedule)
+  int* s_misc = t_tile + touched_cap(a.E);
   int* s_ids = reinterpret_cast<int*>(smem + sm.route);                 // [T * k] expert of every slot (one-launch layer only)
   float* s_w = reinterpret_cast<float*>(s_ids + kFusedMaxSlots);        // [T * k] routing weight
   int* s_row = reinterpret_cast<int*>(s_w + kFusedMaxSlots);            // [T * k] sorted row of every slot
@@ -318,26 +321,18 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     }
   }
   if (!kFused && a.by_pass && wid == 2) {
-    // Large-batch schedule (one projection per launch, so no item waits for another).  An expert with many rows would
-    // make its items many passes long, and equal item counts would leave its CTAs far behind.  So the list of experts
-    // becomes a list of (expert, pass) entries of at most tok_pass rows each: every item is one pass, consecutive items
-    // of an entry share the operand's scale factors in tensor memory, and equal item counts are equal work.  A CTA
-    // keeps only the entries its own items belong to.
+    // Large-batch schedule (one projection per launch, so no item waits for another).  The list of experts becomes a
+    // list of (expert, pass) entries of at most tok_pass rows, each cut into blocks of a few consecutive tiles
+    // (block_tiles); block b goes to CTA b mod gridDim.x.  So every item is one pass and equal block counts are equal
+    // work (an expert with many rows would otherwise make its items many passes long); the items of a block share the
+    // operand's scale factors in tensor memory; and at any moment the grid works on neighbouring blocks - a few experts'
+    // weights and token rows, which stay in L2 for the other passes and tiles that need them (with one contiguous share
+    // per CTA every pass re-read its expert's weights from DRAM: 7 GB instead of 2.3 in the gate/up launch at
+    // prefill_8k).  A CTA keeps one list entry per block of its own: slot j = block blockIdx.x + j * gridDim.x.
     const int tiles = a.ph_lo == 0 ? 2 * a.I / kTile : a.H / kTile;
+    const int bt = block_tiles(tiles), bpe = tiles / bt;  // tiles per block, blocks per entry
+    const int grid = static_cast<int>(gridDim.x), c = static_cast<int>(blockIdx.x);
     const int n_it = (a.E + 31) / 32;
-    int n_ent = 0;
-    for (int i = 0; i < n_it; ++i) {
-      const int e = i * 32 + lane;
-      const int rows = (e < a.E) ? __ldg(a.offsets + e + 1) - __ldg(a.offsets + e) : 0;
-      int tot;
-      warp_excl_scan((rows + tok_pass - 1) / tok_pass, lane, &tot);
-      n_ent += tot;
-    }
-    const long long total = static_cast<long long>(n_ent) * tiles;
-    const long long per = (total + gridDim.x - 1) / gridDim.x;
-    const long long begin = min(static_cast<long long>(blockIdx.x) * per, total), end = min(begin + per, total);
-    const int v_lo = static_cast<int>(begin / tiles);
-    const int v_hi = end > begin ? static_cast<int>((end - 1) / tiles) + 1 : v_lo;
     int run = 0;
     for (int i = 0; i < n_it; ++i) {
       const int e = i * 32 + lane;
@@ -346,21 +341,26 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       const int v = (hi - lo + tok_pass - 1) / tok_pass;
       int tot;
       const int first = run + warp_excl_scan(v, lane, &tot);
-      for (int vi = max(first, v_lo); vi < min(first + v, v_hi); ++vi) {
-        const int idx = vi - v_lo;
-        if (idx < touched_cap(a.E)) {  // (the host chooses this schedule only where the window fits)
-          touched[idx] = e;
-          t_begin[idx] = lo + (vi - first) * tok_pass;
-          t_end[idx] = min(hi, lo + (vi - first + 1) * tok_pass);
+      // blocks [first * bpe, (first + v) * bpe) belong to this expert; mine are those = c (mod grid)
+      const long long b_lo = static_cast<long long>(first) * bpe, b_hi = static_cast<long long>(first + v) * bpe;
+      long long b = b_lo <= c ? c : c + (b_lo - c + grid - 1) / grid * grid;
+      for (; b < b_hi; b += grid) {
+        const int slot = static_cast<int>((b - c) / grid), vi = static_cast<int>(b / bpe) - first;
+        if (slot < touched_cap(a.E)) {  // (the host chooses this schedule only where the list fits)
+          touched[slot] = e;
+          t_tile[slot] = static_cast<int>(b % bpe) * bt;
+          t_begin[slot] = lo + vi * tok_pass;
+          t_end[slot] = min(hi, lo + (vi + 1) * tok_pass);
         }
       }
       run += tot;
     }
     if (lane == 0) {
-      s_misc[0] = v_hi - v_lo;
+      const long long n_blocks = static_cast<long long>(run) * bpe;
+      const int n_slots = n_blocks > c ? static_cast<int>((n_blocks - c + grid - 1) / grid) : 0;
+      s_misc[0] = n_slots;
       s_misc[1] = s_misc[2] = s_misc[3] = s_misc[4] = 0;
-      s_misc[1 + 2 * a.ph_lo] = static_cast<int>(begin - static_cast<long long>(v_lo) * tiles);
-      s_misc[2 + 2 * a.ph_lo] = static_cast<int>(end - static_cast<long long>(v_lo) * tiles);
+      s_misc[2 + 2 * a.ph_lo] = min(n_slots, touched_cap(a.E)) * bt;
     }
   } else if (!kFused && wid == 2) {
     // lane l looks at experts l, l + 32, ...: all loads are issued before any is used (one memory round trip);
@@ -382,6 +382,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       if (has) {
         const int e = i * 32 + lane;
         touched[run + ex] = e;
+        t_tile[run + ex] = 0;
         t_begin[run + ex] = __ldg(a.offsets + e);
         t_end[run + ex] = __ldg(a.offsets + e + 1);
       }
@@ -516,6 +517,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       }
       if (first) {
         touched[ti] = id;
+        t_tile[ti] = 0;
         t_begin[ti] = less;
         t_end[ti] = less + eq_all;
       }
@@ -571,7 +573,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         const TermMaps* ma = phase == 0 ? &tmap_a1 : &tmap_a2;
         for (int it = P.begin; it < P.end; ++it) {
           const int ti = it / P.tiles, e = touched[ti];
-          const int tile = it % P.tiles;
+          const int tile = t_tile[ti] + it % P.tiles;
           const int row_begin = t_begin[ti];
           const int n_rows_e = t_end[ti] - row_begin;
           const int n_pass = (n_rows_e + tok_pass - 1) / tok_pass;
@@ -785,7 +787,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
             uint4 r[8];
             if (P.direct) {
               // 8 scale bytes per weight row and K step, straight from the row layout; issued before the wait below
-              const int e = touched[ti], tile = it % P.tiles;
+              const int e = touched[ti], tile = t_tile[ti] + it % P.tiles;
               const int wrow_a = phase == 0 ? e * P.R + tile * 128 : e * P.R + tile * kTile;
               const int wrow_b = phase == 0 ? e * P.R + a.I + tile * 128 : wrow_a + 128;
               const uint8_t* sc = phase == 0 ? a.s13 : a.s2;
@@ -1055,7 +1057,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         const Phase P = phase_of(phase, a, s_misc + 1);
         const int it_end = dry ? min(P.begin + 1, P.end) : P.end;
         for (int it = P.begin; it < it_end; ++it) {
-          const int ti = it / P.tiles, tile = it % P.tiles;
+          const int ti = it / P.tiles, tile = t_tile[ti] + it % P.tiles;
           const int row_begin = t_begin[ti], row_end = t_end[ti];
           const int n_pass = dry ? 1 : (row_end - row_begin + tok_pass - 1) / tok_pass;
           for (int pass = 0; pass < n_pass; ++pass) {
@@ -1253,10 +1255,11 @@ int launch_native_ffn(const __nv_bfloat16* x_perm, const int* offsets, const Exp
   a.s13 = w.s13;
   a.s2 = w.s2;
   // Batches whose experts have several passes: one launch per projection, shares balanced by passes (see pass_shares)
-  // (a CTA's window of (expert, pass) entries must fit the list it keeps: its items / tiles + 2 entries at most)
+  // (a CTA's blocks, one list entry each, must fit the list it keeps)
   const size_t ent_max = S / (kQ ? 128 : kMaxTokPass) + sh.E, grid_n = static_cast<size_t>(sm_count());
+  const size_t bpe_max = static_cast<size_t>(std::max(2 * sh.I / kTile / block_tiles(2 * sh.I / kTile), sh.H / kTile / block_tiles(sh.H / kTile)));
   const bool two = kQ && S > static_cast<size_t>(kQOneLaunchRows) * sh.E &&
-                   (ent_max + grid_n - 1) / grid_n + 3 <= static_cast<size_t>(touched_cap(sh.E));
+                   (ent_max * bpe_max + grid_n - 1) / grid_n + 1 <= static_cast<size_t>(touched_cap(sh.E));
   a.by_pass = two ? 1 : 0;
   for (int l = 0; l < (two ? 2 : 1); ++l) {
     a.ph_lo = two ? l : 0;
