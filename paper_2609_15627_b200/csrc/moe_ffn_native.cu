@@ -262,6 +262,45 @@ __global__ void __launch_bounds__(1024) native_split_kernel(const __nv_bfloat16*
   });
 }
 
+// ---- the quantised-activation variant's split: bf16 token rows -> one E2M1 row with its scale bytes.  Four threads per
+// 32-element block, eight consecutive values each (16-byte loads, 4-byte stores: a warp writes 128 contiguous bytes) ----
+__global__ void __launch_bounds__(1024) native_quant_rows_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict__ aq,
+                                                                uint8_t* __restrict__ aq_sf, int* __restrict__ done, int S, int H,
+                                                                int E, int* __restrict__ status_clear) {
+  pdl_launch_dependents();  // as native_split_kernel
+  pdl_wait();
+  const long long gt = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (gt < E) done[gt] = 0;
+  if (gt == 0 && status_clear != nullptr) *status_clear = 0;
+  const long long n_grp = static_cast<long long>(S) * (H / 8);  // a multiple of 4: whole blocks are in or out
+  const bool live = gt < n_grp;
+  const uint4 v = live ? __ldcg(reinterpret_cast<const uint4*>(x) + gt) : make_uint4(0u, 0u, 0u, 0u);
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+  float f[8];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    f[2 * j] = __uint_as_float(w[j] << 16);
+    f[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+  }
+  float amax = 0.0f;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) amax = fmaxf(amax, fabsf(f[j]));
+  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+  const int se = (amax > 0.0f) ? term_exp(amax) : 0;
+  const float inv = pow2f(-se);
+  uint32_t codes = 0u;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    float qa, qb;
+    codes |= e2m1_pair(f[2 * j] * inv, f[2 * j + 1] * inv, &qa, &qb) << (8 * j);
+  }
+  if (live) {
+    reinterpret_cast<uint32_t*>(aq)[gt] = codes;                 // row p, bytes 4 * (group in the row): the same index
+    if ((gt & 3) == 0) aq_sf[gt >> 2] = static_cast<uint8_t>(se + 127);  // [row][block]: the same index again
+  }
+}
+
 // kFused = false: the expert FFN (moe_expert_ffn).  kFused = true: the whole layer in this one launch (see FusedArgs);
 // the differences are the set-up, where the gate/up items' operand rows come from, which rows their epilogue writes,
 // and the reduction over slots after the down items.
@@ -1234,9 +1273,13 @@ int launch_native_ffn(const __nv_bfloat16* x_perm, const int* offsets, const Exp
         !nat_map(&tm_a2.box[i], aq2, sh.I / 2, rows, 128, 8u << i, CU_TENSOR_MAP_SWIZZLE_128B))
       return MOE_ERR_CUDA;
   if (!weight_maps(w, sh, &tm_w13, &tm_s13, &tm_w2, &tm_s2)) return MOE_ERR_CUDA;
-  const size_t split_threads = S * (sh.H / 32) * 8 > static_cast<size_t>(sh.E) ? S * (sh.H / 32) * 8 : static_cast<size_t>(sh.E);
-  if (launch_pdl(native_split_kernel<kQ>, dim3(static_cast<unsigned>((split_threads + 1023) / 1024)), dim3(1024), 0, st, x_perm, aq1,
-                 sf1, done, static_cast<int>(S), sh.H, sh.E, status.own ? status.word : nullptr) != cudaSuccess)
+  const size_t per_block = kQ ? 4 : 8;  // threads per 32-element block
+  const size_t split_threads = S * (sh.H / 32) * per_block > static_cast<size_t>(sh.E) ? S * (sh.H / 32) * per_block : static_cast<size_t>(sh.E);
+  const dim3 split_grid(static_cast<unsigned>((split_threads + 1023) / 1024));
+  int* own_word = status.own ? status.word : nullptr;
+  if ((kQ ? launch_pdl(native_quant_rows_kernel, split_grid, dim3(1024), 0, st, x_perm, aq1, sf1, done, static_cast<int>(S), sh.H, sh.E, own_word)
+          : launch_pdl(native_split_kernel<false>, split_grid, dim3(1024), 0, st, x_perm, aq1, sf1, done, static_cast<int>(S), sh.H, sh.E, own_word)) !=
+      cudaSuccess)
     return MOE_ERR_CUDA;
   NatArgs a;
   a.sf1 = sf1;
