@@ -41,9 +41,17 @@
 // The weights are read either in the checkpoint's row layout or in moe_prepack's tile-contiguous layout (one tensor
 // map box = one contiguous run; see ExpertWeights), always with the L2 evict-first policy: each byte is used once.
 //
+// Reductions that are multiples of 256 but not of 512 (the I = 256 shard): the scale bytes' rows are then not multiples
+// of 16 bytes, which no tensor map addresses; the scale warps fetch them with plain loads instead (Phase::direct).
+//
 // The same kernel, instantiated with kFused = true, is the whole layer in one launch for a handful of tokens
-// (moe_forward uses it for one): it routes, sorts the slots and splits the token rows itself, and reduces over the slots at the end
-// (see FusedArgs).
+// (where the one-token kernel does not take the shape): it routes, sorts the slots and splits the token rows itself, and
+// reduces over the slots at the end (see FusedArgs).
+//
+// Instantiated with kQ = true it is the quantised-activation variant (moe_expert_ffn_q): one operand row per token - the
+// activation quantised online to E2M1 with one scale per 32 elements, as the paper's historical decode route does to
+// INT8 - so a pass holds 128 tokens and the epilogues sum nothing across lanes.  Large batches run one projection per
+// launch over blocks of (expert, pass, four tiles) dealt round-robin to the CTAs (see the set-up).
 #include <cuda.h>
 #include <cuda_fp4.h>
 
@@ -232,8 +240,6 @@ __host__ __device__ inline NatSmem nat_smem(int E, int K) {
 // ---- split kernel: bf16 token rows -> 8 E2M1 term rows with their scale bytes; 8 threads per 32-element block ----
 // Few, large CTAs: the FFN grid's CTAs need a whole SM each and are handed out in blockIdx order, so every SM this
 // grid still occupies delays one of them - with at most (SMs - working FFN CTAs) CTAs here, only idle ones.
-// kQ (quantised-activation variant): one term per row, operand row = token row.
-template <bool kQ>
 __global__ void __launch_bounds__(1024) native_split_kernel(const __nv_bfloat16* __restrict__ x, uint8_t* __restrict__ aq,
                                                            uint8_t* __restrict__ aq_sf, int* __restrict__ done, int S, int H,
                                                            int E, int* __restrict__ status_clear) {
@@ -252,10 +258,9 @@ __global__ void __launch_bounds__(1024) native_split_kernel(const __nv_bfloat16*
   const uint2 v = __ldcg(reinterpret_cast<const uint2*>(x + static_cast<size_t>(p) * H + b * 32 + sub * 4));
   float r[1][4] = {{__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u), __uint_as_float(v.y << 16),
                    __uint_as_float(v.y & 0xFFFF0000u)}};
-  constexpr int nt = kQ ? 1 : kTerms;
-  split_terms<1, nt>(r, [&](int, int t, uint32_t bytes, int se) {
+  split_terms<1>(r, [&](int, int t, uint32_t bytes, int se) {
     if (live) {
-      const size_t row = static_cast<size_t>(p) * nt + t;
+      const size_t row = static_cast<size_t>(p) * kTerms + t;
       *reinterpret_cast<uint16_t*>(aq + row * (H / 2) + b * 16 + sub * 2) = static_cast<uint16_t>(bytes);
       if (sub == 0) aq_sf[row * n_blk + b] = static_cast<uint8_t>(se + 127);
     }
@@ -1278,7 +1283,7 @@ int launch_native_ffn(const __nv_bfloat16* x_perm, const int* offsets, const Exp
   const dim3 split_grid(static_cast<unsigned>((split_threads + 1023) / 1024));
   int* own_word = status.own ? status.word : nullptr;
   if ((kQ ? launch_pdl(native_quant_rows_kernel, split_grid, dim3(1024), 0, st, x_perm, aq1, sf1, done, static_cast<int>(S), sh.H, sh.E, own_word)
-          : launch_pdl(native_split_kernel<false>, split_grid, dim3(1024), 0, st, x_perm, aq1, sf1, done, static_cast<int>(S), sh.H, sh.E, own_word)) !=
+          : launch_pdl(native_split_kernel, split_grid, dim3(1024), 0, st, x_perm, aq1, sf1, done, static_cast<int>(S), sh.H, sh.E, own_word)) !=
       cudaSuccess)
     return MOE_ERR_CUDA;
   NatArgs a;

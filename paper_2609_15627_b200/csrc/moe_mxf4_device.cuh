@@ -80,11 +80,10 @@ MOE_DEVINL uint32_t e2m1_pair(float a, float b, float* qa, float* qb) {
 // for NB independent blocks at once (their dependency chains interleave).  `store(nb, t, bytes, se)` receives
 // term t's two bytes of codes (values 0,1 and 2,3 of this thread) and the block exponent.  All 32 lanes must call
 // it together.  (With NB > 1 the chains overlap little: the exchanges and the stores keep their program order.)
-// NT < kTerms stops after the first NT terms (the quantised-activation variant keeps one).
-template <int NB, int NT = kTerms, typename Store>
+template <int NB, typename Store>
 MOE_DEVINL void split_terms(float (&r)[NB][4], Store store) {
 #pragma unroll 1
-  for (int t = 0; t < NT; ++t) {
+  for (int t = 0; t < kTerms; ++t) {
 #pragma unroll
     for (int nb = 0; nb < NB; ++nb) {
       float amax = fmaxf(fmaxf(fabsf(r[nb][0]), fabsf(r[nb][1])), fmaxf(fabsf(r[nb][2]), fabsf(r[nb][3])));
