@@ -246,7 +246,9 @@ int moe_forward_host_packed(const float* logits_host, const void* x_host_bf16, c
  *   - moe_ffn_block: router projection -> moe_route -> moe_permute -> moe_expert_ffn (routed) -> moe_expert_ffn (shared)
  *     -> moe_combine_shared on DEVICE buffers, every intermediate in `ws` (moe_ffn_block_workspace_bytes(), 256-byte
  *     aligned, no initialisation needed).  topk_ids / topk_w [T,k] receive the routing where not NULL.  Enqueue only,
- *     no allocation, capturable, bounded device-side waits.
+ *     no allocation, capturable, bounded device-side waits.  One token (on shapes moe_forward runs as one launch, with
+ *     room for one more expert's CTAs): the router projection, then one launch - the shared expert is an extra slot of
+ *     the one-token kernel, added with weight 1 after the routed slots (the same order of operations).
  */
 int moe_router_logits(const void* x_bf16 /* [T,H] */, const void* w_router_bf16 /* [E,H] */, int32_t T, int32_t H, int32_t E,
                       float* logits /* [T,E] */, int32_t* status_word, void* cuda_stream);

@@ -255,7 +255,7 @@ namespace {
 // ws of moe_ffn_block = [ logits | ids | w | offsets | shared offsets | x_perm | perm | inv_perm | y_perm | y_shared |
 //                         the expert-FFN calls' workspace (the routed call's and the shared call's, used one after the other) ]
 struct BlockLayout {
-  size_t logits, ids, w, offsets, offsets2, x_perm, perm, inv_perm, y_perm, y_shared, inner, inner_bytes, total;
+  size_t logits, ids, w, offsets, offsets2, x_perm, perm, inv_perm, y_perm, y_shared, inner, inner_bytes, one_sync, one_scratch, total;
 };
 moe_shape_t shared_shape(const moe_shape_t& s) { return moe_shape_t{s.T, s.H, s.I, 1, 1}; }
 BlockLayout block_layout(const moe_shape_t& s) {
@@ -281,6 +281,11 @@ BlockLayout block_layout(const moe_shape_t& s) {
   const size_t a = ws_layout(s).total, b = ws_layout(shared_shape(s)).total;
   L.inner_bytes = a > b ? a : b;
   off += L.inner_bytes;
+  // one token: the counter block and the scratch of the one-launch kernel with the shared expert as an extra slot
+  // (whether that kernel applies also depends on the weights' alignment; the size allows for it whenever the shape does)
+  const void* al = reinterpret_cast<const void*>(uintptr_t(256));
+  L.one_sync = take(kForwardSyncBytes);
+  L.one_scratch = take(decode_one_ok(s, al, al, 1) ? decode_one_scratch_bytes(s, 1) : 0);
   L.total = off;
   return L;
 }
@@ -349,6 +354,19 @@ int moe_ffn_block(const void* x_bf16, const void* w_router_bf16, const uint8_t* 
   const moe_shape_t sh1 = shared_shape(s);
   // router scores -> Top-k -> route production -> routed experts; the shared expert on every token (its sorted rows are
   // the token rows themselves); the join
+  if (decode_one_ok(s, w13, w2, 1) && aligned(shared_w13, 16) && aligned(shared_w2, 16) && s.H % 512 == 0 && s.I % 512 == 0) {
+    // One token: the router projection, then ONE launch for everything else - the shared expert is one more slot of the
+    // one-token kernel (its weights depend on no routing, so its stream starts first), added with weight 1 after the
+    // routed slots' recurrence.  The kernel needs its counter block clear; this call owns the block.
+    if (cudaMemsetAsync(base + L.one_sync, 0, kForwardSyncBytes, st) != cudaSuccess) return MOE_ERR_CUDA;
+    if ((rc = moe_router_logits(x_bf16, w_router_bf16, s.T, s.H, s.E, d_logits, status_word, st)) != MOE_OK) return rc;
+    StatusRef status;
+    if ((rc = resolve_status(status_word, &status)) != MOE_OK) return rc;
+    const ExpertWeights shared{shared_w13, shared_w13_scale, shared_w2, shared_w2_scale, false};
+    return launch_decode_one(d_logits, static_cast<const __nv_bfloat16*>(x_bf16), ExpertWeights{w13, w13_scale, w2, w2_scale, false}, s,
+                             static_cast<__nv_bfloat16*>(out_bf16), topk_ids, topk_w, reinterpret_cast<int*>(base + L.one_sync),
+                             base + L.one_scratch, status, st, &shared);
+  }
   if ((rc = moe_router_logits(x_bf16, w_router_bf16, s.T, s.H, s.E, d_logits, status_word, st)) != MOE_OK) return rc;
   if ((rc = launch_shared_offsets(d_off2, s.T, st)) != MOE_OK) return rc;
   if ((rc = moe_route(d_logits, s.T, s.E, s.k, d_ids, d_w, d_off, inner, L.inner_bytes, st)) != MOE_OK) return rc;

@@ -166,11 +166,11 @@ int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const Expe
 
 // the whole layer for one token in one launch with the down projection split along K over pairs of CTAs (moe_forward
 // at T = 1 where the shape allows it); `sync` as above, `scratch` holds decode_one_scratch_bytes
-bool decode_one_ok(const moe_shape_t& s, const void* w13, const void* w2);
-size_t decode_one_scratch_bytes(const moe_shape_t& s);
+bool decode_one_ok(const moe_shape_t& s, const void* w13, const void* w2, int n_shared = 0);
+size_t decode_one_scratch_bytes(const moe_shape_t& s, int n_shared = 0);
 int launch_decode_one(const float* logits, const __nv_bfloat16* x, const ExpertWeights& w, const moe_shape_t& s,
                       __nv_bfloat16* out, int* ids_out, float* w_out, int* sync, void* scratch, StatusRef status,
-                      cudaStream_t st);
+                      cudaStream_t st, const ExpertWeights* shared = nullptr);
 
 // router projection, join with the shared expert, and the shared expert's offsets {0, T} (moe_block.cu)
 int launch_router_logits(const __nv_bfloat16* x, const __nv_bfloat16* w_router, int T, int H, int E, float* logits, int* status,

@@ -79,7 +79,7 @@ struct OneArgs {
   __nv_bfloat16* out;       // [H]
   int* ids_out;             // [k] or null
   float* w_out;             // [k] or null
-  float* part;              // [k][I/256][H] partial sums of the down projection
+  float* part;              // [k + n_shared][I/256][H] partial sums of the down projection
   uint8_t* aq1;             // [kCopies][8][H/2] E2M1 term rows of the token, written by the CTAs that split it
   uint8_t* sf1;             // [kCopies][8][H/32] their scale bytes
   int* sync;                // counter block, zero between calls
@@ -87,6 +87,8 @@ struct OneArgs {
   int own_status;           // the library's own status word: the last CTA clears it
   int E, H, I, k;
   int blocked;              // weights in moe_prepack's tile-contiguous layout
+  int n_shared;             // 1: slot k is the shared expert (its own tensor maps, expert 0 of them), added with weight 1
+  int blocked_shared;       //    and its weights' layout
 };
 
 struct OneSmem {
@@ -151,7 +153,9 @@ MOE_DEVINL void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::
 __global__ void __launch_bounds__(kOneThreads, 1)
 decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_constant__ CUtensorMap tmap_s13,
                   const __grid_constant__ CUtensorMap tmap_w2, const __grid_constant__ CUtensorMap tmap_s2,
-                  const __grid_constant__ CUtensorMap tmap_a1, const OneArgs a) {
+                  const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_sw13,
+                  const __grid_constant__ CUtensorMap tmap_ss13, const __grid_constant__ CUtensorMap tmap_sw2,
+                  const __grid_constant__ CUtensorMap tmap_ss2, const OneArgs a) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   const OneSmem sm = one_smem(a.E, a.H);
@@ -184,7 +188,8 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   const int npp = a.I / 256;             // K steps of the down projection = pairs of CTAs per slot
   const int n_t1 = a.H / 512;            // 256-row tiles of the down projection per CTA (half of the H rows)
   const int item = static_cast<int>(blockIdx.x);
-  const bool has_item = item < a.k * tiles0;
+  const int n_slots = a.k + a.n_shared;  // routed slots, then the shared expert (figure "Execution structure": it runs beside them)
+  const bool has_item = item < n_slots * tiles0;
   const int slot = item / tiles0, tile = item % tiles0;
   const int pp = tile >> 1;
   const uint32_t rank = cluster_ctarank();  // = tile & 1 for a CTA with an item (tiles0 is even, clusters are (2c, 2c + 1))
@@ -202,6 +207,12 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     prefetch_tmap(&tmap_w2);
     prefetch_tmap(&tmap_s2);
     prefetch_tmap(&tmap_a1);
+    if (a.n_shared) {
+      prefetch_tmap(&tmap_sw13);
+      prefetch_tmap(&tmap_ss13);
+      prefetch_tmap(&tmap_sw2);
+      prefetch_tmap(&tmap_ss2);
+    }
   }
   if (tid == 0) {
     for (int s = 0; s < kWStages; ++s) { mbar_init(&full_w[s], 1); mbar_init(&empty_w[s], 1); }
@@ -264,14 +275,16 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
   } else if (wid == 0) {
     // =========================== producer: all TMA loads of both projections ===========================
     if (lane == 0 && has_item) {
-      mbar_wait(route_ready, 0u, a.status);
-      const int e = s_ids[slot];
+      const bool shared = slot >= a.k;  // the shared expert's weights depend on no routing: its stream starts at once
+      if (!shared) mbar_wait(route_ready, 0u, a.status);
+      const int e = shared ? 0 : s_ids[slot];
+      const int blocked = shared ? a.blocked_shared : a.blocked;
       int s = 0, cs = 0;
       uint32_t ph = 0, cph = 0;
       const uint64_t stream_once = l2_policy_evict_first();  // every weight byte is read once per call
       for (int phase = 0; phase < 2; ++phase) {
-        const CUtensorMap* mw = phase == 0 ? &tmap_w13 : &tmap_w2;
-        const CUtensorMap* msc = phase == 0 ? &tmap_s13 : &tmap_s2;
+        const CUtensorMap* mw = phase == 0 ? (shared ? &tmap_sw13 : &tmap_w13) : (shared ? &tmap_sw2 : &tmap_w2);
+        const CUtensorMap* msc = phase == 0 ? (shared ? &tmap_ss13 : &tmap_s13) : (shared ? &tmap_ss2 : &tmap_s2);
         const int n_steps = phase == 0 ? n_ks0 : npp;  // K steps of the projection (tile geometry of the packed layout)
         const int n_it = phase == 0 ? n_ks0 : n_t1;
         for (int it = 0; it < n_it; ++it) {
@@ -283,18 +296,18 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
           if (phase == 1 || (it & 1) == 0) {  // 16 scale bytes per weight row cover two K steps
             mbar_wait(&empty_sc[cs], cph ^ 1u, a.status);
             mbar_expect_tx(&full_sc[cs], kScStage);
-            const int sx = a.blocked ? 0 : (ks >> 1) * 16;
-            const int sya = a.blocked ? ((wrow_a >> 7) * (n_steps >> 1) + (ks >> 1)) * 128 : wrow_a;
-            const int syb = a.blocked ? ((wrow_b >> 7) * (n_steps >> 1) + (ks >> 1)) * 128 : wrow_b;
+            const int sx = blocked ? 0 : (ks >> 1) * 16;
+            const int sya = blocked ? ((wrow_a >> 7) * (n_steps >> 1) + (ks >> 1)) * 128 : wrow_a;
+            const int syb = blocked ? ((wrow_b >> 7) * (n_steps >> 1) + (ks >> 1)) * 128 : wrow_b;
             tma_load_2d_hint(sSc + cs * kScStage, msc, sx, sya, &full_sc[cs], stream_once);
             tma_load_2d_hint(sSc + cs * kScStage + 128 * 16, msc, sx, syb, &full_sc[cs], stream_once);
             if (++cs == kScStages) { cs = 0; cph ^= 1u; }
           }
           mbar_wait(&empty_w[s], ph ^ 1u, a.status);
           mbar_expect_tx(&full_w[s], phase == 0 ? kWStage + 4 * 1024 : kWStage);
-          const int wx = a.blocked ? 0 : ks * 128;
-          const int wya = a.blocked ? ((wrow_a >> 7) * n_steps + ks) * 128 : wrow_a;
-          const int wyb = a.blocked ? ((wrow_b >> 7) * n_steps + ks) * 128 : wrow_b;
+          const int wx = blocked ? 0 : ks * 128;
+          const int wya = blocked ? ((wrow_a >> 7) * n_steps + ks) * 128 : wrow_a;
+          const int wyb = blocked ? ((wrow_b >> 7) * n_steps + ks) * 128 : wrow_b;
           tma_load_2d_hint(sW + s * kWStage, mw, wx, wya, &full_w[s], stream_once);
           tma_load_2d_hint(sW + s * kWStage + 128 * 128, mw, wx, wyb, &full_w[s], stream_once);
           if (it == 0) MOE_TP(5 + phase);
@@ -644,7 +657,7 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     float* ys = reinterpret_cast<float*>(sW);  // [k][128], the ring is idle by now
     const int cg = tid & 31, grp = tid >> 5;   // 32 groups of 4 columns; warp j sums the partials of slot j, j + 8, ...
     if (grp < 8) {
-      for (int j = grp; j < a.k; j += 8) {
+      for (int j = grp; j < n_slots; j += 8) {
         const float* p0 = a.part + static_cast<size_t>(j) * npp * a.H + ct * kRedCols + cg * 4;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int p = 0; p < npp; p += 8) {  // eight independent 16-byte loads in flight
@@ -676,6 +689,11 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         acc.x = __fmaf_rn(wj, v.x, acc.x);
         acc.y = __fmaf_rn(wj, v.y, acc.y);
       }
+      if (a.n_shared) {  // the join: one fp32 addition of the shared expert's row after the routed slots' recurrence
+        const float2 v = *reinterpret_cast<const float2*>(ys + a.k * kRedCols + col);
+        acc.x = __fadd_rn(acc.x, v.x);
+        acc.y = __fadd_rn(acc.y, v.y);
+      }
       if (!dry) *reinterpret_cast<__nv_bfloat162*>(a.out + ct * kRedCols + col) = __floats2bfloat162_rn(acc.x, acc.y);
     }
     __syncthreads();
@@ -684,7 +702,7 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
     if (ct >= 0) {
       reduce_tile(true);  // once on whatever the buffer holds, no store: the code is then in place when the count completes
       if (tid == 0) {
-        counter_wait_ge(a.sync + kSyncDone2 + (2 * ct) / n_red, 4 * a.k * npp, a.status);  // the half its columns are in
+        counter_wait_ge(a.sync + kSyncDone2 + (2 * ct) / n_red, 4 * n_slots * npp, a.status);  // the half its columns are in
         MOE_TP(17);
       }
       __syncthreads();
@@ -721,21 +739,21 @@ decode_one_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
 // ---- host side ---------------------------------------------------------------------------------------
 // Shapes: one token; H and I multiples of 512 up to 4096 (whole 256-row tiles, whole pairs); one gate/up item and one
 // reducing CTA per SM at most; the routing row and the operands fit shared memory.
-bool decode_one_ok(const moe_shape_t& sh, const void* w13, const void* w2) {
+bool decode_one_ok(const moe_shape_t& sh, const void* w13, const void* w2, int n_shared) {
   const int grid = sm_count() & ~1;
   return sh.T == 1 && sh.H % 512 == 0 && sh.I % 512 == 0 && sh.H <= 4096 && sh.I <= 4096 && sh.k <= 32 &&
-         sh.k * (sh.I / 128) <= grid && sh.H / 32 <= grid && sh.H / 128 <= grid && sh.H / 256 <= kSyncExit - kSyncDone2 &&
+         (sh.k + n_shared) * (sh.I / 128) <= grid && sh.H / 32 <= grid && sh.H / 128 <= grid && sh.H / 256 <= kSyncExit - kSyncDone2 &&
          (reinterpret_cast<uintptr_t>(w13) & 15u) == 0 && (reinterpret_cast<uintptr_t>(w2) & 15u) == 0 &&
          one_smem(sh.E, sh.H).total + 1024 <= 227 * 1024;
 }
-size_t decode_one_scratch_bytes(const moe_shape_t& sh) {
-  return align_up(static_cast<size_t>(sh.k) * (sh.I / 256) * sh.H * 4, kAlign) +
+size_t decode_one_scratch_bytes(const moe_shape_t& sh, int n_shared) {
+  return align_up(static_cast<size_t>(sh.k + n_shared) * (sh.I / 256) * sh.H * 4, kAlign) +
          align_up(static_cast<size_t>(kCopies) * kTerms * (sh.H / 2), kAlign) + align_up(static_cast<size_t>(kCopies) * kTerms * (sh.H / 32), kAlign);
 }
 
 int launch_decode_one(const float* logits, const __nv_bfloat16* x, const ExpertWeights& w, const moe_shape_t& sh,
                       __nv_bfloat16* out, int* ids_out, float* w_out, int* sync, void* scratch, StatusRef status,
-                      cudaStream_t st) {
+                      cudaStream_t st, const ExpertWeights* shared) {
   static PerDeviceFlag flag;
   if (!once_per_device(flag, [] {
         return cudaFuncSetAttribute(decode_one_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) == cudaSuccess;
@@ -743,6 +761,10 @@ int launch_decode_one(const float* logits, const __nv_bfloat16* x, const ExpertW
     return MOE_ERR_CUDA;
   CUtensorMap tm_w13, tm_w2, tm_s13, tm_s2;
   if (!weight_maps(w, sh, &tm_w13, &tm_s13, &tm_w2, &tm_s2)) return MOE_ERR_CUDA;
+  // the shared expert, where there is one: tensors shaped as the routed ones with a single expert
+  CUtensorMap tm_sw13 = tm_w13, tm_sw2 = tm_w2, tm_ss13 = tm_s13, tm_ss2 = tm_s2;
+  const int n_shared = shared != nullptr ? 1 : 0;
+  if (shared != nullptr && !weight_maps(*shared, moe_shape_t{1, sh.H, sh.I, 1, 1}, &tm_sw13, &tm_ss13, &tm_sw2, &tm_ss2)) return MOE_ERR_CUDA;
   OneArgs a;
   a.logits = logits;
   a.x = x;
@@ -750,7 +772,7 @@ int launch_decode_one(const float* logits, const __nv_bfloat16* x, const ExpertW
   a.ids_out = ids_out;
   a.w_out = w_out;
   a.part = static_cast<float*>(scratch);
-  a.aq1 = static_cast<uint8_t*>(scratch) + align_up(static_cast<size_t>(sh.k) * (sh.I / 256) * sh.H * 4, kAlign);
+  a.aq1 = static_cast<uint8_t*>(scratch) + align_up(static_cast<size_t>(sh.k + n_shared) * (sh.I / 256) * sh.H * 4, kAlign);
   a.sf1 = a.aq1 + align_up(static_cast<size_t>(kCopies) * kTerms * (sh.H / 2), kAlign);
   a.sync = sync;
   a.status = status.word;
@@ -760,6 +782,8 @@ int launch_decode_one(const float* logits, const __nv_bfloat16* x, const ExpertW
   a.I = sh.I;
   a.k = sh.k;
   a.blocked = w.blocked ? 1 : 0;
+  a.n_shared = n_shared;
+  a.blocked_shared = (shared != nullptr && shared->blocked) ? 1 : 0;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(sm_count() & ~1));
   cfg.blockDim = dim3(kOneThreads);
@@ -776,8 +800,9 @@ int launch_decode_one(const float* logits, const __nv_bfloat16* x, const ExpertW
   cfg.numAttrs = 2;
   CUtensorMap tm_a1;  // the token's 8 term rows [8][H/2 bytes], one box = 8 rows x one K step
   if (!term_row_map(&tm_a1, a.aq1, sh.H / 2, kCopies * kTerms, 8)) return MOE_ERR_CUDA;
-  if (cudaLaunchKernelEx(&cfg, decode_one_kernel, tm_w13, tm_s13, tm_w2, tm_s2, tm_a1, a) != cudaSuccess) return MOE_ERR_CUDA;
-  note_kernel("layer_one_launch_mxf4_pair_split_k", 1);
+  if (cudaLaunchKernelEx(&cfg, decode_one_kernel, tm_w13, tm_s13, tm_w2, tm_s2, tm_a1, tm_sw13, tm_ss13, tm_sw2, tm_ss2, a) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  note_kernel(n_shared ? "block_one_launch_mxf4_pair_split_k" : "layer_one_launch_mxf4_pair_split_k", 1);
   return MOE_OK;
 }
 

@@ -109,15 +109,22 @@ def _check_block(wl, seed, routed=None, rdev=None, sample=None):
     (4, 512, 512, 8, 2),       # decode-sized kernel, router by warps
     (24, 1024, 512, 32, 6),    # decode-sized routed call, shared call of 24 rows on one expert
     (512, 512, 512, 8, 2),     # prefill-sized routed call, router GEMM
-    (1100, 512, 512, 16, 6)])  # prefill-sized kernel for both calls
+    (1100, 512, 512, 16, 6),   # prefill-sized kernel for both calls
+    (1, 512, 512, 8, 2),       # one token: the router projection, then one launch with the shared expert as a third slot
+    (1, 1024, 512, 16, 6),
+    (1, 512, 1024, 4, 4)])
 def test_ffn_block_small_shapes(T, H, I, E, k):
     _check_block(inputs.Workload("block", T, H, I, E, k), seed=5)
+    if T == 1:
+        assert moe.moe_last_kernel_name() == "block_one_launch_mxf4_pair_split_k"
 
 
 @pytest.mark.parametrize("name", ["decode_c1", "decode_c64"])
 def test_ffn_block_production_decode(name):
     wl = inputs.WORKLOADS[name]
     _check_block(wl, seed=7)
+    if wl.T == 1:   # 9 slots x 16 CTAs on 144 of the 148 SMs
+        assert moe.moe_last_kernel_name() == "block_one_launch_mxf4_pair_split_k"
 
 
 def test_ffn_block_prefill_8k_sampled():
