@@ -41,7 +41,7 @@ MIN_REGION_MS_PREFILL = 40.0  # prefill rounds: at least this long and at least 
                               # the burst bf16 peak they are divided by (a single sub-millisecond GEMM, best of ten)
 COOLDOWN_S = 1.0        # idle time before every round: each round starts with the board below its power limit
 ROUNDS = 3
-GRAPH_STEPS = 8         # consecutive batches of the cycle per CUDA graph (decode workloads)
+GRAPH_STEPS = 32  # decode steps per CUDA graph: the whole cycle of seeded batches (a serving graph holds dozens of layer calls)
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch (or per two-launch call) from one ncu capture of the
 # workload; which capture, at which commit, is stated in the file under profiles/ named beside each figure.
@@ -569,11 +569,18 @@ class Bench:
                 g.replay()
             self.barrier()
 
-        rem_graphs = {}
+        rem_graphs, whole_graphs = {}, {}
 
-        def prepare(n):
+        def prepare(n, whole=False):
             """A step count that is not a multiple of GRAPH_STEPS ends with ONE graph of the remaining steps (captured
-            here, before the timed region)."""
+            here, before the timed region).  whole: the region of exactly --steps steps is ONE graph of all its steps
+            (up to 4096), so that no gap between graph launches falls inside a region of a few hundred microseconds."""
+            if use_graph and whole and n <= 4096:
+                if n not in whole_graphs:
+                    whole_graphs[n] = capture(step, range(n))
+                    whole_graphs[n].replay()
+                    self.barrier()
+                return
             r = n % GRAPH_STEPS
             if use_graph and r and r not in rem_graphs:
                 i0 = (n // GRAPH_STEPS) * GRAPH_STEPS
@@ -581,9 +588,11 @@ class Bench:
                 rem_graphs[r].replay()
                 self.barrier()
 
-        def play(n, inner=None):
+        def play(n, inner=None, whole=False):
             """Enqueue n consecutive steps of the cycle."""
-            if use_graph:
+            if use_graph and whole and n in whole_graphs:
+                whole_graphs[n].replay()
+            elif use_graph:
                 n_multi = n // GRAPH_STEPS
                 for i in range(n_multi):
                     multi_graphs[i % len(multi_graphs)].replay()
@@ -593,10 +602,15 @@ class Bench:
                 for i in range(n):
                     step(i, inner[i] if inner is not None and i < len(inner) and not one_launch else None)
 
-        def region(n, inner=None):
+        def region(n, inner=None, whole=False):
             """One timed region of exactly n steps: barrier + synchronize on both sides, CUDA events on the launching
             stream, max over ranks.  Returns (ms of the region, clock record, launches of the library's kernels)."""
-            prepare(n)
+            prepare(n, whole)
+            if whole and use_graph:
+                # a region this short is over before the clocks have come up from idle: run about 20 ms of the same
+                # steps, untimed, right in front of it
+                for _ in range(max(1, int(20.0 / max(n * 0.03, 0.01)))):
+                    play(n, None, whole)
             e0, e1 = self.events()
             sampler = ClockSampler(physical_gpu_index(self.local))
             c0 = moe.moe_launch_count()
@@ -604,7 +618,7 @@ class Bench:
             sampler.start()
             self.hold()
             e0.record(stream)
-            play(n, inner)
+            play(n, inner, whole)
             e1.record(stream)
             self.barrier()
             clocks = sampler.stop()
@@ -615,7 +629,7 @@ class Bench:
         # ---- the headline's region: exactly K steps -------------------------------------------------------------
         rec = {}
         if exact_steps is not None:
-            ms, clocks, launches = region(exact_steps)
+            ms, clocks, launches = region(exact_steps, whole=True)
             rec["exact"] = {"steps": exact_steps, "ms_total": ms, "ms_per_step": ms / exact_steps, "clocks": clocks,
                             "gpu_launches": launches,
                             "experts_touched": float(np.mean([touched[i % n_cycle] for i in range(exact_steps)]))}
@@ -648,7 +662,8 @@ class Bench:
                         "reasons": sorted(reasons), "sm_mhz_rounds": clock_rounds},
                     "call": ("moe_forward%s (one kernel launch per step)" if one_launch else
                              "moe_route, moe_permute, moe_expert_ffn%s, moe_combine") % ("_packed" if packed is not None else ""),
-                    "launch": ("cuda graph replay, %d consecutive batches of the cycle per graph" % GRAPH_STEPS) if use_graph else "eager",
+                    "launch": ("cuda graph replay, %d consecutive batches of the cycle per graph (the region of exactly --steps "
+                               "steps: one graph of all its steps)" % GRAPH_STEPS) if use_graph else "eager",
                     "experts_touched": mean_touched})
 
         # ---- the expert-FFN call inside eager steps (decode: a second region right after the graph-replayed one) ---
@@ -791,7 +806,7 @@ class Bench:
         rec["kernels"] = moe.moe_last_kernel_name()
         rec["one_launch"] = one_launch
         rec["n_cycle"] = n_cycle
-        del graphs, multi_graphs, batches, buf, fws
+        del graphs, multi_graphs, whole_graphs, rem_graphs, batches, buf, fws
         torch.cuda.empty_cache()
         return rec
 
