@@ -251,6 +251,32 @@ def moe_forward_host_packed(logits_host, x_host, packed, sh, out_host, status_wo
            "moe_forward_host_packed")
 
 
+class BoundCall:
+    """One C-ABI call with its arguments marshalled once: calling the object makes the call again on the same buffers
+    (which it keeps alive) - a serving loop that reuses its buffers need not rebuild the argument list every step."""
+
+    def __init__(self, name, fn, args, keep):
+        self.name, self.fn, self.args, self.keep = name, fn, args, keep
+
+    def __call__(self):
+        rc = self.fn(*self.args)
+        if rc != 0:
+            _check(rc, self.name)
+
+
+def bind_forward_host(logits_host, x_host, weights, sh, out_host, status_word, ws, stream=None):
+    """moe_forward_host (weights = the four tensors) or moe_forward_host_packed (weights = moe_prepack's tensor) as a
+    BoundCall."""
+    tensors = (logits_host, x_host, weights, sh, out_host, status_word, ws, stream)
+    if isinstance(weights, (tuple, list)):
+        args = (_ptr(logits_host), _ptr(x_host), *(_ptr(t) for t in weights), C.byref(sh), _ptr(out_host), _ptr(status_word),
+                _ptr(ws), ws.numel(), _stream(stream))
+        return BoundCall("moe_forward_host", lib().moe_forward_host, args, tensors)
+    args = (_ptr(logits_host), _ptr(x_host), _ptr(weights), C.byref(sh), _ptr(out_host), _ptr(status_word), _ptr(ws),
+            ws.numel(), _stream(stream))
+    return BoundCall("moe_forward_host_packed", lib().moe_forward_host_packed, args, tensors)
+
+
 def moe_debug_read_probe(src, sink, status_word, stream=None):
     """Enqueue one read-only pass over the tensor `src` (see the header); time it with events around the call."""
     _check(lib().moe_debug_read_probe(_ptr(src), src.numel() * src.element_size(), _ptr(sink),
