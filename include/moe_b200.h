@@ -213,8 +213,11 @@ int moe_forward_packed(const float* logits /* [T,E] */, const void* x_bf16 /* [T
 /*
  * moe_forward with HOST input and output for one batch: copies logits_host [T,E] and x_host [T,H] to
  * device buffers carved from `ws`, clears moe_forward's counters, runs moe_forward on `cuda_stream`,
- * copies out [T,H] bf16 back into out_host and waits for the stream.  An output of at most 64 KB in page-locked
- * memory that the device can address is written there by the last kernel itself (no copy operation after it).
+ * copies out [T,H] bf16 back into out_host and waits for the stream.  Fewer stream operations where the sizes allow: an
+ * output of at most 64 KB in page-locked memory that the device can address is written there by the last kernel itself;
+ * a single token row in such memory is read there by the kernel; logits of at most 64 KB travel in one copy with the
+ * zeros of moe_forward's counter block, through a page-locked staging buffer that the library allocates once per host
+ * thread (the only allocation any entry point makes, on its first call).
  * Weights stay device-resident (they are model state, not per-batch input).  For page-locked host
  * buffers the copies are asynchronous until the final wait.  ws must hold
  * moe_forward_host_workspace_bytes() bytes.  No counterpart in the paper: it is the end-to-end

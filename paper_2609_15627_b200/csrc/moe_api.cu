@@ -552,9 +552,11 @@ HostLayout host_layout(const moe_shape_t& s) {
     off += align_up(bytes, kAlign);
     return o;
   };
-  L.logits = take(static_cast<size_t>(s.T) * s.E * 4);
+  // (the logits sit right in front of moe_forward's workspace, whose first bytes are its counter block: small logits
+  // and the block's zeros arrive in one copy)
   L.x = take(static_cast<size_t>(s.T) * s.H * 2);
   L.out = take(static_cast<size_t>(s.T) * s.H * 2);
+  L.logits = take(static_cast<size_t>(s.T) * s.E * 4);
   L.inner = off;
   off += forward_layout(s).total;
   L.total = off;
@@ -568,6 +570,23 @@ size_t moe_forward_host_workspace_bytes(const moe_shape_t* shape) {
 }
 
 namespace {
+constexpr size_t kStageLogitsBytes = 64 * 1024;  // logits up to this size travel together with the counter block's zeros
+// [kStageLogitsBytes of logits][kForwardSyncBytes of zeros], page-locked, one per host thread (never freed)
+unsigned char* logits_staging() {
+  thread_local unsigned char* buf = nullptr;
+  thread_local bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    if (cudaHostAlloc(&p, kStageLogitsBytes + kForwardSyncBytes, cudaHostAllocDefault) == cudaSuccess) {
+      buf = static_cast<unsigned char*>(p);
+      memset(buf, 0, kStageLogitsBytes + kForwardSyncBytes);
+    } else {
+      cudaGetLastError();
+    }
+  }
+  return buf;
+}
 constexpr size_t kDirectOutBytes = 64 * 1024;  // outputs up to this size are written to pinned host memory by the kernel
 int forward_host_impl(const float* logits_host, const void* x_host_bf16, const ExpertWeights& w, const moe_shape_t* shape,
                       void* out_host_bf16, int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
@@ -595,10 +614,33 @@ int forward_host_impl(const float* logits_host, const void* x_host_bf16, const E
       cudaGetLastError();  // pageable memory: not an error of this call
     }
   }
-  // this call owns its workspace's contents: it clears the sync block of moe_forward itself
-  if (cudaMemsetAsync(base + L.inner, 0, kForwardSyncBytes, st) != cudaSuccess ||
-      cudaMemcpyAsync(d_logits, logits_host, static_cast<size_t>(s.T) * s.E * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(d_x, x_host_bf16, static_cast<size_t>(s.T) * s.H * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+  // Likewise a single token row is read where it lies: the few CTAs that split it fetch 512 bytes each across the bus,
+  // which costs the kernel less than a copy operation in front of it costs the call.
+  bool x_direct = false;
+  if (s.T == 1 && decode_one_ok(s, w.w13, w.w2)) {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, x_host_bf16) == cudaSuccess && at.type == cudaMemoryTypeHost && at.devicePointer != nullptr &&
+        aligned(at.devicePointer, 16)) {
+      d_x = at.devicePointer;
+      x_direct = true;
+    } else {
+      cudaGetLastError();
+    }
+  }
+  // This call owns its workspace's contents: it clears the counter block of moe_forward itself.  Small logits go through
+  // a page-locked staging buffer of this thread that ends in zeros, so that one copy brings both (the call waits for the
+  // stream before it returns, so the buffer is free again by then).
+  const size_t lg_bytes = static_cast<size_t>(s.T) * s.E * 4, lg_span = L.inner - L.logits;
+  unsigned char* stage = lg_span <= kStageLogitsBytes ? logits_staging() : nullptr;
+  if (stage != nullptr) {
+    memcpy(stage, logits_host, lg_bytes);
+    memset(stage + lg_bytes, 0, lg_span - lg_bytes + kForwardSyncBytes);  // (an earlier, larger batch may have left logits there)
+    if (cudaMemcpyAsync(d_logits, stage, lg_span + kForwardSyncBytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return MOE_ERR_CUDA;
+  } else if (cudaMemsetAsync(base + L.inner, 0, kForwardSyncBytes, st) != cudaSuccess ||
+             cudaMemcpyAsync(d_logits, logits_host, lg_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    return MOE_ERR_CUDA;
+  }
+  if ((!x_direct && cudaMemcpyAsync(d_x, x_host_bf16, static_cast<size_t>(s.T) * s.H * 2, cudaMemcpyHostToDevice, st) != cudaSuccess))
     return MOE_ERR_CUDA;
   if ((rc = forward_impl(d_logits, d_x, w, shape, d_out, nullptr, nullptr, status_word, base + L.inner, ws_bytes - L.inner,
                          st)) != MOE_OK)
