@@ -613,6 +613,30 @@ def test_forward_host_uses_it():
     assert_same_up_to_rounding(oh.numpy().view(np.uint16), bits(out4))
 
 
+def test_forward_host_sequence_of_shapes_and_pageable_buffers():
+    """The host entry point on one thread: a batch whose logits fill the staging buffer, then a single token (whose
+    counter block's zeros travel behind 1 KB of logits in the same buffer), twice, then the same from pageable memory
+    (no page-locked buffer for the kernel to read or write in place)."""
+    big = inputs.Workload("host_big", 64, 512, 512, 256, 4)     # 64 KB of logits
+    one = inputs.Workload("host_one", 1, 1024, 512, 256, 4)
+    for pinned in (True, False):
+        for wl in (big, one, big, one):
+            d = inputs.make_workload(wl, seed=11)
+            wdev = weights_dev(d)
+            sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
+            ws = moe.alloc_workspace(sh, host_path=True)
+            ws.fill_(0x5A)
+            st = torch.zeros(1, dtype=torch.int32, device="cuda")
+            lh, xh = torch.from_numpy(d["logits"].copy()), torch.from_numpy(d["x"].view(np.int16).copy())
+            oh = torch.zeros((wl.T, wl.H), dtype=torch.int16)
+            if pinned:
+                lh, xh, oh = lh.pin_memory(), xh.pin_memory(), oh.pin_memory()
+            moe.moe_forward_host(lh, xh, *wdev, sh, oh, st, ws)
+            assert int(st.item()) == 0
+            buf, out4 = run_layer(wl, d, wdev)
+            assert_same_up_to_rounding(oh.numpy().view(np.uint16), bits(out4))
+
+
 # ---- moe_prepack and the calls that take its result ------------------------------------------------------
 
 def _tiles(a, tile_bytes):
