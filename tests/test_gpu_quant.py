@@ -149,7 +149,7 @@ def test_ffn_q_argument_checks():
     torch.cuda.synchronize()
 
 
-@pytest.mark.parametrize("name", ["decode_c64", "prefill_8k"])
+@pytest.mark.parametrize("name", ["decode_c64", "prefill_8k", "prefill_32k_skewed"])
 def test_ffn_q_at_the_benchmark_shapes_on_sampled_rows(name):
     """The launch configuration bench.py times (prepacked weights, the library's own routing and permutation), checked on
     sampled sorted rows: first and last row, rows either side of expert boundaries, random rows."""
@@ -172,7 +172,8 @@ def test_ffn_q_at_the_benchmark_shapes_on_sampled_rows(name):
     off = buf.expert_offsets.cpu().numpy()
     S = T * k
     rng = np.random.default_rng(0)
-    edges = off[np.r_[1:4, E // 2, E - 2]]
+    heavy = int(np.argmax(np.diff(off)))                      # the expert with the most rows: the most passes
+    edges = np.concatenate([off[np.r_[1:4, E // 2, E - 2]], [off[heavy], off[heavy + 1] - 130]])
     rows = np.unique(np.clip(np.concatenate([rng.integers(0, S, 40), [0, S - 1], edges - 1, edges, edges + 127, edges + 128]), 0, S - 1))
     expert_of = np.searchsorted(off, rows, side="right") - 1
     idx = torch.from_numpy(rows).cuda()
