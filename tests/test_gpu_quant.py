@@ -182,3 +182,26 @@ def test_ffn_q_at_the_benchmark_shapes_on_sampled_rows(name):
     np.add.at(so, expert_of + 1, 1)
     want = O.expert_ffn_q(xs, np.cumsum(so).astype(np.int32), *w, 1)
     _check_rows(buf.y_perm[idx].cpu().numpy(), want, name)
+
+
+def test_ffn_q_whole_tensor_agrees_between_weight_layouts_at_prefill_8k():
+    """Every row of the output, not a sample: the call on the checkpoint's row layout and the call on moe_prepack's tiles
+    read different bytes through different tensor maps and must give the same bits (the sampled rows above tie one of
+    them to the oracle)."""
+    wl = inputs.WORKLOADS["prefill_8k"]
+    T, H, I, E, k = wl.T, wl.H, wl.I, wl.E, wl.k
+    sh = moe.shape(T, H, I, E, k)
+    wd = tuple(dev(a) for a in inputs.make_expert_weights(H, I, E, seed=0))
+    packed = moe.moe_prepack(*wd, sh)
+    buf = moe.LayerBuffers(sh)
+    moe.moe_route(dev(inputs.make_logits(T, E, 2, wl.skew)), k, buf.topk_ids, buf.topk_w, buf.expert_offsets, buf.ws)
+    moe.moe_permute(dev(inputs.make_x(T, H, 2)), buf.topk_ids, buf.expert_offsets, sh, buf.x_perm, buf.perm, buf.inv_perm, buf.ws)
+    ws = moe.alloc_ffn_q_workspace(sh)
+    y2 = torch.full_like(buf.y_perm, float("nan"))
+    buf.y_perm.fill_(float("nan"))
+    moe.moe_expert_ffn_q(buf.x_perm, buf.expert_offsets, wd, sh, buf.y_perm, buf.status, ws)
+    moe.moe_expert_ffn_q(buf.x_perm, buf.expert_offsets, packed, sh, y2, buf.status, ws)
+    torch.cuda.synchronize()
+    assert int(buf.status.item()) == 0
+    assert not torch.isnan(y2).any()
+    assert torch.equal(buf.y_perm, y2)
