@@ -95,8 +95,9 @@ def test_ffn_q_structured_scales_and_zero_blocks():
     _check_rows(got, O.expert_ffn_q(xp, off, w13, s13, w2, s2, k), "structured")
 
 
-def test_ffn_q_without_a_status_word_and_replayed_as_a_graph():
-    T, H, I, E, k = 33, 512, 512, 4, 2
+@pytest.mark.parametrize("T,H,I,E,k", [(33, 512, 512, 4, 2),      # one launch for both projections
+                                       (300, 512, 512, 2, 2)])    # large-batch schedule: one launch per projection
+def test_ffn_q_without_a_status_word_and_replayed_as_a_graph(T, H, I, E, k):
     w, xp, off = _problem(T, H, I, E, k, seed=5)
     sh = moe.shape(T, H, I, E, k)
     wd = tuple(dev(a) for a in w)
