@@ -290,6 +290,34 @@ int moe_expert_ffn_q(const void* x_perm_bf16 /* [T*k,H] */, const int32_t* exper
                      void* cuda_stream);
 
 /*
+ * Expert-parallel sharding of the routed layer over `world` GPUs, one process each (the paper compares a tensor-parallel
+ * layout with expert-parallel ones, "TP8/EP1" against "TP4/EP4"; outside the single-GPU workloads this library is
+ * measured on).  Rank r holds the weights of the experts [e_begin, e_end) and finishes the tokens
+ * [r * tpr, (r + 1) * tpr), tpr = ceil(T / world).  Every rank runs moe_route and moe_permute on ALL tokens (identical
+ * results everywhere); its experts' rows are one contiguous range of the sorted order.  Then
+ *   - moe_ep_row_table fills row_dst[p], for the sorted rows p of this rank's experts, with the address of row
+ *     (token - owner * tpr) * k + slot of owner_y[owner], owner = token / tpr: owner_y is a DEVICE array of `world`
+ *     pointers to the ranks' buffers [tpr * k, H] fp32 - peer memory for the other ranks (the caller maps it: CUDA IPC,
+ *     symmetric memory; the library only stores through the pointers);
+ *   - moe_ep_expert_ffn is moe_expert_ffn on this rank's experts (weights [e_end - e_begin, ...], the GLOBAL
+ *     expert_offsets and shape), whose down projection stores every output row through row_dst instead of into a local
+ *     y_perm: the exchange ("combine" in expert-parallel terms) happens in the kernel's epilogue, row by row;
+ *   - after a barrier between the ranks (the caller's: all stores of all ranks complete), each rank runs moe_combine on
+ *     its buffer with the identity as inv_perm and its tokens' rows of topk_w: the same fp32 rows in the same slot order
+ *     as on one GPU, so the result is bit-identical to the unsharded layer.
+ * e_begin must be a multiple of 4 (alignment of the shifted offsets); `ws` as for moe_expert_ffn on the global shape.
+ * Enqueue only, no allocation, capturable, bounded device-side waits; no kernel of one rank waits for another rank.
+ */
+int moe_ep_row_table(const int32_t* perm, const int32_t* expert_offsets, const moe_shape_t* shape, int32_t e_begin,
+                     int32_t e_end, float* const* owner_y /* device, [world] */, int32_t world,
+                     float** row_dst /* device, [T*k] */, void* cuda_stream);
+int moe_ep_expert_ffn(const void* x_perm_bf16 /* [T*k,H] */, const int32_t* expert_offsets /* [E+1], all experts */,
+                      const uint8_t* w13_local, const uint8_t* w13_scale_local, const uint8_t* w2_local,
+                      const uint8_t* w2_scale_local, const moe_shape_t* shape /* global */, int32_t e_begin, int32_t e_end,
+                      float* const* row_dst /* device, [T*k] */, int32_t* status_word, void* ws, size_t ws_bytes,
+                      void* cuda_stream);
+
+/*
  * moe_expert_ffn without a workspace argument, for callers that cannot allocate device memory
  * (the paper has no counterpart: this is a packaging variant of moe_expert_ffn, same arithmetic).
  *

@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmoe_b200.so")
-SOURCES = ["moe_api.cu", "moe_route_permute_combine.cu", "moe_ffn_stream.cu", "moe_ffn_umma.cu", "moe_ffn_native.cu", "moe_decode_one.cu", "moe_block.cu", "moe_noalloc.cu", "moe_probe.cu", "moe_prepack.cu"]
+SOURCES = ["moe_api.cu", "moe_route_permute_combine.cu", "moe_ffn_stream.cu", "moe_ffn_umma.cu", "moe_ffn_native.cu", "moe_decode_one.cu", "moe_block.cu", "moe_ep.cu", "moe_noalloc.cu", "moe_probe.cu", "moe_prepack.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-shared",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

@@ -132,12 +132,16 @@ int moe_permute(const void* x_bf16, const int32_t* topk_ids, const int32_t* expe
 
 namespace {
 int expert_ffn_impl(const void* x_perm_bf16, const int32_t* expert_offsets, const ExpertWeights& w, const moe_shape_t* shape,
-                    float* y_perm, int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
+                    float* y_perm, int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream,
+                    float* const* row_dst = nullptr, const moe_shape_t* choice = nullptr) {
+  // `choice`: the shape that picks the kernel where it is not `shape` itself - a rank of an expert-parallel job runs the
+  // kernel the unsharded layer would run, so that the sharded result has the same bits
+  if (choice == nullptr) choice = shape;
   if (!aligned(x_perm_bf16, 16) || !aligned(expert_offsets, 16) || !aligned(w.w13, 16) || !aligned(w.s13, 16) ||
-      !aligned(w.w2, 16) || !aligned(w.s2, 16) || !aligned(y_perm, 16))
-    return MOE_ERR_INVALID_ARG;
+      !aligned(w.w2, 16) || !aligned(w.s2, 16) || (row_dst == nullptr ? !aligned(y_perm, 16) : !aligned(row_dst, 8)))
+    return MOE_ERR_INVALID_ARG;  // (with a table of output rows there is no y_perm)
   if (status_word != nullptr && !aligned(status_word, 4)) return MOE_ERR_INVALID_ARG;
-  const WsLayout L = ws_layout(*shape);
+  const WsLayout L = ws_layout(*choice);  // (the scratch of the kernel that `choice` picks, same row count)
   if (check_ws(ws, ws_bytes, L.total) != MOE_OK) return MOE_ERR_WORKSPACE;
   __nv_bfloat16* act = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(ws) + L.act_off);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -149,10 +153,12 @@ int expert_ffn_impl(const void* x_perm_bf16, const int32_t* expert_offsets, cons
   StatusRef status;
   int rc = resolve_status(status_word, &status);
   if (rc != MOE_OK) return rc;
-  if (native_shape_ok(*shape, w.w13, w.w2)) return launch_expert_ffn_native(xp, expert_offsets, w, *shape, act, y_perm, status, st);
+  if (native_shape_ok(*choice, w.w13, w.w2))
+    return launch_expert_ffn_native(xp, expert_offsets, w, *shape, act, y_perm, status, st, row_dst);
   if ((rc = clear_own_status(status, st)) != MOE_OK) return rc;
-  if (umma_shape_ok(*shape) || w.blocked) return launch_expert_ffn_umma(xp, expert_offsets, w, *shape, act, y_perm, status.word, st);
-  return launch_expert_ffn_stream(xp, expert_offsets, w.w13, w.s13, w.w2, w.s2, *shape, act, y_perm, status.word, st);
+  if (umma_shape_ok(*choice) || w.blocked)
+    return launch_expert_ffn_umma(xp, expert_offsets, w, *shape, act, y_perm, status.word, st, row_dst);
+  return launch_expert_ffn_stream(xp, expert_offsets, w.w13, w.s13, w.w2, w.s2, *shape, act, y_perm, status.word, st, row_dst);
 }
 
 // the four tensors inside a buffer written by moe_prepack
@@ -290,6 +296,41 @@ BlockLayout block_layout(const moe_shape_t& s) {
   return L;
 }
 }  // namespace
+
+// ---- expert-parallel sharding ------------------------------------------------------------------------
+namespace {
+int check_ep(const moe_shape_t& s, int e_begin, int e_end, int world) {
+  if (world < 1 || e_begin < 0 || e_end <= e_begin || e_end > s.E) return MOE_ERR_INVALID_ARG;
+  if (e_begin % 4 != 0) return MOE_ERR_INVALID_ARG;  // the shifted offsets array keeps its 16-byte alignment
+  return MOE_OK;
+}
+}  // namespace
+
+int moe_ep_row_table(const int32_t* perm, const int32_t* expert_offsets, const moe_shape_t* shape, int32_t e_begin, int32_t e_end,
+                     float* const* owner_y, int32_t world, float** row_dst, void* cuda_stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if ((rc = check_ep(*shape, e_begin, e_end, world)) != MOE_OK) return rc;
+  if (perm == nullptr || expert_offsets == nullptr || owner_y == nullptr || row_dst == nullptr) return MOE_ERR_INVALID_ARG;
+  const int tpr = (shape->T + world - 1) / world;
+  return launch_ep_row_table(perm, expert_offsets, shape->k, shape->H, e_begin, e_end, owner_y, world, tpr, row_dst,
+                             static_cast<cudaStream_t>(cuda_stream), shape->T * shape->k);
+}
+
+int moe_ep_expert_ffn(const void* x_perm_bf16, const int32_t* expert_offsets, const uint8_t* w13_local, const uint8_t* w13_scale_local,
+                      const uint8_t* w2_local, const uint8_t* w2_scale_local, const moe_shape_t* shape, int32_t e_begin, int32_t e_end,
+                      float* const* row_dst, int32_t* status_word, void* ws, size_t ws_bytes, void* cuda_stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if ((rc = check_ep(*shape, e_begin, e_end, 1)) != MOE_OK) return rc;
+  if (row_dst == nullptr || expert_offsets == nullptr) return MOE_ERR_INVALID_ARG;
+  // the kernels see this rank's experts only: their rows are the range [offsets[e_begin], offsets[e_end]) of the sorted
+  // order, and the shifted offsets array describes exactly that; x_perm and the table are indexed by sorted row as ever
+  moe_shape_t local = *shape;
+  local.E = e_end - e_begin;  // (k stays: it only sizes buffers and tensor maps, T * k rows)
+  return expert_ffn_impl(x_perm_bf16, expert_offsets + e_begin, ExpertWeights{w13_local, w13_scale_local, w2_local, w2_scale_local, false},
+                         &local, nullptr, status_word, ws, ws_bytes, cuda_stream, row_dst, shape);
+}
 
 size_t moe_expert_ffn_q_workspace_bytes(const moe_shape_t* shape) {
   if (check_shape(shape) != MOE_OK) return 0;

@@ -129,11 +129,11 @@ int launch_permute(const __nv_bfloat16* x, const int* ids, const int* offsets, c
 // weight-streaming variant (any shape; the one for decode-sized batches)
 int launch_expert_ffn_stream(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
                              const uint8_t* w2, const uint8_t* s2, const moe_shape_t& s, __nv_bfloat16* act, float* y_perm,
-                             int* status_word, cudaStream_t st);
+                             int* status_word, cudaStream_t st, float* const* row_dst = nullptr);
 // tcgen05 grouped-GEMM variant (prefill-sized batches); umma_shape_ok says whether it applies
 bool umma_shape_ok(const moe_shape_t& s);
 int launch_expert_ffn_umma(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& s,
-                           __nv_bfloat16* act, float* y_perm, int* status_word, cudaStream_t st);
+                           __nv_bfloat16* act, float* y_perm, int* status_word, cudaStream_t st, float* const* row_dst = nullptr);
 int launch_combine(const float* y_perm, const int* inv_perm, const float* w, const moe_shape_t& s,
                    __nv_bfloat16* out, cudaStream_t st);
 int launch_validate_scales(const uint8_t* scales, size_t n, int* bad, cudaStream_t st);
@@ -143,9 +143,9 @@ bool native_shape_ok(const moe_shape_t& s, const void* w13, const void* w2);
 // the quantised-activation variant of the same kernel: any batch size; scratch of native_q_scratch_bytes
 bool native_q_shape_ok(const moe_shape_t& s, const void* w13, const void* w2);
 int launch_expert_ffn_native_q(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& s,
-                               void* scratch, float* y_perm, StatusRef status, cudaStream_t st);
+                               void* scratch, float* y_perm, StatusRef status, cudaStream_t st, float* const* row_dst = nullptr);
 int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& s,
-                             void* scratch, float* y_perm, StatusRef status, cudaStream_t st);
+                             void* scratch, float* y_perm, StatusRef status, cudaStream_t st, float* const* row_dst = nullptr);
 
 // the whole layer in one launch, for a handful of tokens on shapes the native variant takes (moe_forward);
 // `sync` is the zeroed block of kForwardSyncBytes, `scratch` holds forward_fused_scratch_bytes
@@ -175,6 +175,9 @@ int launch_decode_one(const float* logits, const __nv_bfloat16* x, const ExpertW
 // router projection, join with the shared expert, and the shared expert's offsets {0, T} (moe_block.cu)
 int launch_router_logits(const __nv_bfloat16* x, const __nv_bfloat16* w_router, int T, int H, int E, float* logits, int* status,
                          cudaStream_t st);
+// expert-parallel sharding: the table of output rows (see moe_ep_row_table)
+int launch_ep_row_table(const int* perm, const int* offsets, int k, int H, int e_begin, int e_end, float* const* owner_y, int world,
+                        int tokens_per_rank, float** row_dst, cudaStream_t st, int max_rows);
 int launch_combine_shared(const float* y_perm, const int* inv_perm, const float* w, const float* y_shared, const moe_shape_t& s,
                           __nv_bfloat16* out, cudaStream_t st);
 int launch_shared_offsets(int* offsets2, int T, cudaStream_t st);

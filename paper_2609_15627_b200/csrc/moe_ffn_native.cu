@@ -94,6 +94,7 @@ struct NatArgs {
   int* done;                 // [E] epilogue warps that have published a gate/up item of the expert
   const int* offsets;
   float* y;                  // output [S, H]
+  float* const* row_dst;     // or null; else output row p goes to row_dst[p] (see y_row)
   int* status;               // never null: the caller's word or the library's own (see StatusRef)
   int own_status;            // the library's own word: the one-launch kernel's last CTA clears it for the next call
   int E, H, I, S;
@@ -988,7 +989,7 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
       } else {
         const int tok = rep ? jl : 4 * q + jl;
         if (!dry && tok < n_tok) {
-          float* dst = a.y + static_cast<size_t>(row0 + tok) * out_stride + tile * kTile + 32 * ch0 + cb;
+          float* dst = y_row(a.y, a.row_dst, static_cast<size_t>(row0 + tok), out_stride) + tile * kTile + 32 * ch0 + cb;
 #pragma unroll
           for (int mm = 0; mm < 8; ++mm)
             if (mm < n_ch) *reinterpret_cast<float4*>(dst + 32 * mm) = make_float4(acc[mm][0], acc[mm][1], acc[mm][2], acc[mm][3]);
@@ -1059,8 +1060,8 @@ ffn_native_kernel(const __grid_constant__ CUtensorMap tmap_w13, const __grid_con
         if (active) {
           // each lane writes its own row: 32 bytes per store where the output allows it (whole sectors), and the next
           // chunk's tensor-memory load in flight during the stores of the current one
-          float* dst = a.y + static_cast<size_t>(row0 + tok) * out_stride + tile * kTile;
-          const bool wide = (reinterpret_cast<uintptr_t>(a.y) & 31u) == 0;  // rows are multiples of 2 KB apart
+          float* dst = y_row(a.y, a.row_dst, static_cast<size_t>(live ? row0 + tok : row0), out_stride) + tile * kTile;
+          const bool wide = (reinterpret_cast<uintptr_t>(dst) & 31u) == 0;
           auto put = [&](const uint32_t (&v)[32], int m) {
             if (!live) return;
             if (wide) {
@@ -1261,7 +1262,7 @@ namespace {
 // kQ: the quantised-activation variant (one operand row per token instead of kTerms)
 template <bool kQ>
 int launch_native_ffn(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& sh,
-                      void* scratch, float* y_perm, StatusRef status, cudaStream_t st) {
+                      void* scratch, float* y_perm, StatusRef status, cudaStream_t st, float* const* row_dst) {
   if (!nat_attr_once()) return MOE_ERR_CUDA;
   const size_t S = static_cast<size_t>(sh.T) * sh.k;
   const size_t rows = S * (kQ ? 1 : kTerms);  // operand rows
@@ -1293,6 +1294,7 @@ int launch_native_ffn(const __nv_bfloat16* x_perm, const int* offsets, const Exp
   a.done = done;
   a.offsets = offsets;
   a.y = y_perm;
+  a.row_dst = row_dst;
   a.status = status.word;
   a.own_status = 0;
   a.E = sh.E;
@@ -1323,12 +1325,12 @@ int launch_native_ffn(const __nv_bfloat16* x_perm, const int* offsets, const Exp
 }  // namespace
 
 int launch_expert_ffn_native(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& sh,
-                             void* scratch, float* y_perm, StatusRef status, cudaStream_t st) {
-  return launch_native_ffn<false>(x_perm, offsets, w, sh, scratch, y_perm, status, st);
+                             void* scratch, float* y_perm, StatusRef status, cudaStream_t st, float* const* row_dst) {
+  return launch_native_ffn<false>(x_perm, offsets, w, sh, scratch, y_perm, status, st, row_dst);
 }
 int launch_expert_ffn_native_q(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& sh,
-                               void* scratch, float* y_perm, StatusRef status, cudaStream_t st) {
-  return launch_native_ffn<true>(x_perm, offsets, w, sh, scratch, y_perm, status, st);
+                               void* scratch, float* y_perm, StatusRef status, cudaStream_t st, float* const* row_dst) {
+  return launch_native_ffn<true>(x_perm, offsets, w, sh, scratch, y_perm, status, st, row_dst);
 }
 
 // ---- the one-launch layer ----
@@ -1375,6 +1377,7 @@ int launch_forward_fused(const float* logits, const __nv_bfloat16* x, const Expe
   a.done = sync;
   a.offsets = nullptr;
   a.y = y;
+  a.row_dst = nullptr;
   a.status = status.word;
   a.own_status = status.own ? 1 : 0;
   a.E = sh.E;

@@ -31,6 +31,7 @@ struct FfnArgs {
   const int* offsets;         // [E+1]
   __nv_bfloat16* act;         // stage 1 output [S, I]
   float* y;                   // stage 2 output [S, Hout]
+  float* const* row_dst;      // or null; else output row p goes to row_dst[p] (see y_row)
   int* status;
   uint32_t k1, k2;         // 0x1040, 0x0104: multipliers of the E2M1 expansion, kept opaque to the compiler
   int E, K, R, I;             // R rows per expert (2I for stage 1, H for stage 2); I used by stage 1 only
@@ -248,12 +249,14 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const FfnArgs a
           } else {
             const int n = tile * 16 + g;
             if (r_a < row_end) {
-              a.y[static_cast<size_t>(r_a) * a.R + n] = s.x;
-              a.y[static_cast<size_t>(r_a) * a.R + n + 8] = s.z;
+              float* ya = y_row(a.y, a.row_dst, static_cast<size_t>(r_a), a.R);
+              ya[n] = s.x;
+              ya[n + 8] = s.z;
             }
             if (r_b < row_end) {
-              a.y[static_cast<size_t>(r_b) * a.R + n] = s.y;
-              a.y[static_cast<size_t>(r_b) * a.R + n + 8] = s.w;
+              float* yb = y_row(a.y, a.row_dst, static_cast<size_t>(r_b), a.R);
+              yb[n] = s.y;
+              yb[n + 8] = s.w;
             }
           }
         }
@@ -271,7 +274,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_stream_kernel(const FfnArgs a
 
 int launch_expert_ffn_stream(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
                       const uint8_t* w2, const uint8_t* s2, const moe_shape_t& sh, __nv_bfloat16* act, float* y_perm,
-                      int* status_word, cudaStream_t st) {
+                      int* status_word, cudaStream_t st, float* const* row_dst) {
   constexpr int kSmemBudget = 200 * 1024;
   static PerDeviceFlag flag;
   if (!once_per_device(flag, [] {
@@ -287,6 +290,7 @@ int launch_expert_ffn_stream(const __nv_bfloat16* x_perm, const int* offsets, co
     a.offsets = offsets;
     a.act = act;
     a.y = y_perm;
+    a.row_dst = row_dst;
     a.status = status_word;
   a.k1 = 0x1040u;
   a.k2 = 0x0104u;

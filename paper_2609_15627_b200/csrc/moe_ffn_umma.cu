@@ -51,6 +51,7 @@ struct UmmaArgs {
   const int* offsets;      // [E+1]
   __nv_bfloat16* act;      // stage 1 output [S, I]
   float* y;                // stage 2 output [S, R]
+  float* const* row_dst;   // or null; else output row p goes to row_dst[p] (see y_row)
   int* status;
   uint32_t k1, k2;         // 0x1040, 0x0104: multipliers of the E2M1 expansion, kept opaque to the compiler
   int E, K, R, I;          // R weight rows per expert (2I or H)
@@ -335,7 +336,7 @@ ffn_umma_kernel(const __grid_constant__ CUtensorMap tmap_tok, const __grid_const
             tmem_ld_wait();
 #pragma unroll
             for (int jj = 0; jj < 32; ++jj)
-              if (c0 + jj < ntok) a.y[static_cast<size_t>(row0 + c0 + jj) * a.R + n] = __uint_as_float(v[jj]);
+              if (c0 + jj < ntok) y_row(a.y, a.row_dst, static_cast<size_t>(row0 + c0 + jj), a.R)[n] = __uint_as_float(v[jj]);
           }
         }
       }
@@ -396,7 +397,7 @@ bool umma_shape_ok(const moe_shape_t& sh) {
 }
 
 int launch_expert_ffn_umma(const __nv_bfloat16* x_perm, const int* offsets, const ExpertWeights& w, const moe_shape_t& sh,
-                           __nv_bfloat16* act, float* y_perm, int* status_word, cudaStream_t st) {
+                           __nv_bfloat16* act, float* y_perm, int* status_word, cudaStream_t st, float* const* row_dst) {
   const size_t smem = smem_map(sh.E).total + 1024;
   static PerDeviceFlag flag;
   if (!once_per_device(flag, [] {
@@ -420,6 +421,7 @@ int launch_expert_ffn_umma(const __nv_bfloat16* x_perm, const int* offsets, cons
   a.offsets = offsets;
   a.act = act;
   a.y = y_perm;
+  a.row_dst = row_dst;
   a.status = status_word;
   a.k1 = 0x1040u;
   a.k2 = 0x0104u;

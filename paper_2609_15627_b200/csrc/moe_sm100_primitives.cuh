@@ -101,6 +101,11 @@ MOE_DEVINL void tma_load_2d_hint(void* dst, const void* tmap, int x, int y, uint
       "l"(tmap), "r"(smem_u32(bar)), "r"(x), "r"(y), "l"(policy)
       : "memory");
 }
+// Output row `row` of the expert FFN: in the caller's y_perm [rows, stride], or - expert-parallel sharding - wherever the
+// table says (a row of the buffer of the rank that finishes the row's token, possibly in a peer GPU's memory)
+MOE_DEVINL float* y_row(float* y, float* const* row_dst, size_t row, int stride) {
+  return row_dst != nullptr ? row_dst[row] : y + row * static_cast<size_t>(stride);
+}
 // make generic-proxy shared-memory writes visible to the asynchronous proxy (TMA, tcgen05.mma)
 MOE_DEVINL void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 

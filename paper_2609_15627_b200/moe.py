@@ -19,7 +19,8 @@ EXPORTS = ("moe_workspace_bytes", "moe_status_string", "moe_last_kernel_name", "
            "moe_expert_ffn_noalloc", "moe_debug_native_cta_share", "moe_debug_read_probe", "moe_prepack_bytes", "moe_prepack",
            "moe_expert_ffn_packed", "moe_forward_packed", "moe_forward_host_packed", "moe_debug_forward_one_launch",
            "moe_debug_expert_ffn_variant", "moe_router_logits", "moe_combine_shared", "moe_ffn_block_workspace_bytes",
-           "moe_ffn_block", "moe_expert_ffn_q_workspace_bytes", "moe_expert_ffn_q")
+           "moe_ffn_block", "moe_expert_ffn_q_workspace_bytes", "moe_expert_ffn_q",
+           "moe_ep_row_table", "moe_ep_expert_ffn")
 
 
 class MoeError(RuntimeError):
@@ -59,6 +60,10 @@ def lib():
         L.moe_expert_ffn_q_workspace_bytes.argtypes = [C.POINTER(Shape)]
         L.moe_expert_ffn_q.restype = C.c_int
         L.moe_expert_ffn_q.argtypes = [vp, vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp, sz, vp]
+        L.moe_ep_row_table.restype = C.c_int
+        L.moe_ep_row_table.argtypes = [vp, vp, C.POINTER(Shape), i32, i32, vp, i32, vp, vp]
+        L.moe_ep_expert_ffn.restype = C.c_int
+        L.moe_ep_expert_ffn.argtypes = [vp, vp, vp, vp, vp, vp, C.POINTER(Shape), i32, i32, vp, vp, vp, sz, vp]
         L.moe_combine.restype = C.c_int
         L.moe_combine.argtypes = [vp, vp, vp, C.POINTER(Shape), vp, vp]
         L.moe_validate_scales.restype = C.c_int
@@ -237,6 +242,19 @@ def moe_expert_ffn_q(x_perm, expert_offsets, weights, sh, y_perm, status_word, w
     _check(lib().moe_expert_ffn_q(_ptr(x_perm), _ptr(expert_offsets), _ptr(raw[0]), _ptr(raw[1]), _ptr(raw[2]), _ptr(raw[3]),
                                   _ptr(packed), C.byref(sh), _ptr(y_perm), _ptr(status_word), _ptr(ws), ws.numel(),
                                   _stream(stream)), "moe_expert_ffn_q")
+
+
+def moe_ep_row_table(perm, expert_offsets, sh, e_begin, e_end, owner_y, world, row_dst, stream=None):
+    """owner_y: int64 device tensor of `world` addresses; row_dst: int64 device tensor [T*k] (receives addresses)."""
+    _check(lib().moe_ep_row_table(_ptr(perm), _ptr(expert_offsets), C.byref(sh), e_begin, e_end, _ptr(owner_y), world,
+                                  _ptr(row_dst), _stream(stream)), "moe_ep_row_table")
+
+
+def moe_ep_expert_ffn(x_perm, expert_offsets, w_local, sh, e_begin, e_end, row_dst, status_word, ws, stream=None):
+    w13, s13, w2, s2 = w_local
+    _check(lib().moe_ep_expert_ffn(_ptr(x_perm), _ptr(expert_offsets), _ptr(w13), _ptr(s13), _ptr(w2), _ptr(s2), C.byref(sh),
+                                   e_begin, e_end, _ptr(row_dst), _ptr(status_word), _ptr(ws), ws.numel(), _stream(stream)),
+           "moe_ep_expert_ffn")
 
 
 def moe_forward_packed(logits, x, packed, sh, out, topk_ids, topk_w, status_word, ws, stream=None):
