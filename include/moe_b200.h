@@ -293,8 +293,8 @@ int moe_expert_ffn_q(const void* x_perm_bf16 /* [T*k,H] */, const int32_t* exper
  * Expert-parallel sharding of the routed layer over `world` GPUs, one process each (the paper compares a tensor-parallel
  * layout with expert-parallel ones, "TP8/EP1" against "TP4/EP4"; outside the single-GPU workloads this library is
  * measured on).  Rank r holds the weights of the experts [e_begin, e_end) and finishes the tokens
- * [r * tpr, (r + 1) * tpr), tpr = ceil(T / world).  Every rank runs moe_route and moe_permute on ALL tokens (identical
- * results everywhere); its experts' rows are one contiguous range of the sorted order.  Then
+ * [r * tpr, (r + 1) * tpr), tpr = ceil(T / world).  Every rank runs moe_route and moe_ep_permute on ALL tokens (identical
+ * routing and order everywhere); its experts' rows are one contiguous range of the sorted order.  Then
  *   - moe_ep_row_table fills row_dst[p], for the sorted rows p of this rank's experts, with the address of row
  *     (token - owner * tpr) * k + slot of owner_y[owner], owner = token / tpr: owner_y is a DEVICE array of `world`
  *     pointers to the ranks' buffers [tpr * k, H] fp32 - peer memory for the other ranks (the caller maps it: CUDA IPC,
@@ -308,6 +308,11 @@ int moe_expert_ffn_q(const void* x_perm_bf16 /* [T*k,H] */, const int32_t* exper
  * e_begin must be a multiple of 4 (alignment of the shifted offsets); `ws` as for moe_expert_ffn on the global shape.
  * Enqueue only, no allocation, capturable, bounded device-side waits; no kernel of one rank waits for another rank.
  */
+/* moe_permute of which a rank needs the order (perm, inv_perm: complete) but only its own experts' rows of x_perm: for
+ * batches of more than 4096 slots only those rows are copied (smaller batches: all, the copy is part of one small kernel) */
+int moe_ep_permute(const void* x_bf16, const int32_t* topk_ids, const int32_t* expert_offsets, const moe_shape_t* shape,
+                   int32_t e_begin, int32_t e_end, void* x_perm_bf16, int32_t* perm, int32_t* inv_perm, void* ws,
+                   size_t ws_bytes, void* cuda_stream);
 int moe_ep_row_table(const int32_t* perm, const int32_t* expert_offsets, const moe_shape_t* shape, int32_t e_begin,
                      int32_t e_end, float* const* owner_y /* device, [world] */, int32_t world,
                      float** row_dst /* device, [T*k] */, void* cuda_stream);

@@ -306,6 +306,22 @@ int check_ep(const moe_shape_t& s, int e_begin, int e_end, int world) {
 }
 }  // namespace
 
+int moe_ep_permute(const void* x_bf16, const int32_t* topk_ids, const int32_t* expert_offsets, const moe_shape_t* shape, int32_t e_begin,
+                   int32_t e_end, void* x_perm_bf16, int32_t* perm, int32_t* inv_perm, void* ws, size_t ws_bytes, void* cuda_stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if ((rc = check_ep(*shape, e_begin, e_end, 1)) != MOE_OK) return rc;
+  if (!aligned(x_bf16, 16) || !aligned(topk_ids, 16) || !aligned(expert_offsets, 16) || !aligned(x_perm_bf16, 16) ||
+      !aligned(perm, 16) || !aligned(inv_perm, 16))
+    return MOE_ERR_INVALID_ARG;
+  const WsLayout L = ws_layout(*shape);
+  if (check_ws(ws, ws_bytes, L.total) != MOE_OK) return MOE_ERR_WORKSPACE;
+  int* block_counts = reinterpret_cast<int*>(static_cast<char*>(ws) + L.permute_off);
+  return launch_permute(static_cast<const __nv_bfloat16*>(x_bf16), topk_ids, expert_offsets, *shape,
+                        static_cast<__nv_bfloat16*>(x_perm_bf16), perm, inv_perm, block_counts, static_cast<cudaStream_t>(cuda_stream),
+                        expert_offsets + e_begin, expert_offsets + e_end);
+}
+
 int moe_ep_row_table(const int32_t* perm, const int32_t* expert_offsets, const moe_shape_t* shape, int32_t e_begin, int32_t e_end,
                      float* const* owner_y, int32_t world, float** row_dst, void* cuda_stream) {
   int rc = check_shape(shape);

@@ -125,7 +125,8 @@ void note_kernel(const char* name, int launches);
 int launch_route(const float* logits, int T, int E, int k, int* ids, float* w, int* offsets, int* counters,
                  cudaStream_t st);
 int launch_permute(const __nv_bfloat16* x, const int* ids, const int* offsets, const moe_shape_t& s,
-                   __nv_bfloat16* x_perm, int* perm, int* inv_perm, int* block_counts, cudaStream_t st);
+                   __nv_bfloat16* x_perm, int* perm, int* inv_perm, int* block_counts, cudaStream_t st,
+                   const int* range_lo = nullptr, const int* range_hi = nullptr);
 // weight-streaming variant (any shape; the one for decode-sized batches)
 int launch_expert_ffn_stream(const __nv_bfloat16* x_perm, const int* offsets, const uint8_t* w13, const uint8_t* s13,
                              const uint8_t* w2, const uint8_t* s2, const moe_shape_t& s, __nv_bfloat16* act, float* y_perm,

@@ -248,19 +248,24 @@ __global__ void __launch_bounds__(256) permute_scatter_kernel(const int* __restr
 }
 
 // Large S, pass 4: gather rows, one warp per sorted row.
+// range: null, or two device words {first sorted row, row after the last} - only those rows are copied (a rank of an
+// expert-parallel job needs the rows of its own experts only)
 __global__ void __launch_bounds__(256) permute_gather_kernel(const __nv_bfloat16* __restrict__ x,
                                                              const int* __restrict__ perm, int S, int H, int k,
-                                                             __nv_bfloat16* __restrict__ x_perm) {
+                                                             __nv_bfloat16* __restrict__ x_perm, const int* __restrict__ range_lo,
+                                                             const int* __restrict__ range_hi) {
   const int lane = threadIdx.x & 31;
   const int wpb = blockDim.x >> 5;
-  for (int p = blockIdx.x * wpb + (threadIdx.x >> 5); p < S; p += gridDim.x * wpb) {
+  const int p_lo = range_lo != nullptr ? *range_lo : 0, p_hi = range_hi != nullptr ? *range_hi : S;
+  for (int p = p_lo + blockIdx.x * wpb + (threadIdx.x >> 5); p < p_hi; p += gridDim.x * wpb) {
     const int s = perm[p];
     warp_copy_row(x + static_cast<size_t>(s / k) * H, x_perm + static_cast<size_t>(p) * H, H, lane);
   }
 }
 
 int launch_permute(const __nv_bfloat16* x, const int* ids, const int* offsets, const moe_shape_t& sh,
-                   __nv_bfloat16* x_perm, int* perm, int* inv_perm, int* block_counts, cudaStream_t st) {
+                   __nv_bfloat16* x_perm, int* perm, int* inv_perm, int* block_counts, cudaStream_t st, const int* range_lo,
+                   const int* range_hi) {
   const int S = sh.T * sh.k;
   if (S <= 4096) {
     if (launch_pdl(permute_small_kernel, dim3((S + 7) / 8), dim3(256), 0, st, x, ids, offsets, S, sh.H, sh.k, x_perm, perm,
@@ -273,7 +278,7 @@ int launch_permute(const __nv_bfloat16* x, const int* ids, const int* offsets, c
     permute_scan_kernel<<<(sh.E + 7) / 8, 256, 0, st>>>(offsets, sh.E, nblk, block_counts);
     permute_scatter_kernel<<<nblk, 256, 8 * sh.E * 4, st>>>(ids, S, sh.E, block_counts, perm, inv_perm);
     const int grid = min((S + 7) / 8, sm_count() * 16);
-    permute_gather_kernel<<<grid, 256, 0, st>>>(x, perm, S, sh.H, sh.k, x_perm);
+    permute_gather_kernel<<<grid, 256, 0, st>>>(x, perm, S, sh.H, sh.k, x_perm, range_lo, range_hi);
     note_kernel("permute_chunked_scan", 4);
   }
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;

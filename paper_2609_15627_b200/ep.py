@@ -58,7 +58,7 @@ def compute(moe, buf, logits, x, w_local, stream=None):
     epilogue stores into the owners' buffers)."""
     sh, L = buf.sh, buf.layer
     moe.moe_route(logits, sh.k, L.topk_ids, L.topk_w, L.expert_offsets, L.ws, stream)
-    moe.moe_permute(x, L.topk_ids, L.expert_offsets, sh, L.x_perm, L.perm, L.inv_perm, L.ws, stream)
+    moe.moe_ep_permute(x, L.topk_ids, L.expert_offsets, sh, buf.e_begin, buf.e_end, L.x_perm, L.perm, L.inv_perm, L.ws, stream)
     moe.moe_ep_row_table(L.perm, L.expert_offsets, sh, buf.e_begin, buf.e_end, buf.owner_y, buf.world, buf.row_dst, stream)
     moe.moe_ep_expert_ffn(L.x_perm, L.expert_offsets, w_local, sh, buf.e_begin, buf.e_end, buf.row_dst, L.status, L.ws, stream)
 

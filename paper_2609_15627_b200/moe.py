@@ -20,7 +20,7 @@ EXPORTS = ("moe_workspace_bytes", "moe_status_string", "moe_last_kernel_name", "
            "moe_expert_ffn_packed", "moe_forward_packed", "moe_forward_host_packed", "moe_debug_forward_one_launch",
            "moe_debug_expert_ffn_variant", "moe_router_logits", "moe_combine_shared", "moe_ffn_block_workspace_bytes",
            "moe_ffn_block", "moe_expert_ffn_q_workspace_bytes", "moe_expert_ffn_q",
-           "moe_ep_row_table", "moe_ep_expert_ffn")
+           "moe_ep_permute", "moe_ep_row_table", "moe_ep_expert_ffn")
 
 
 class MoeError(RuntimeError):
@@ -60,6 +60,8 @@ def lib():
         L.moe_expert_ffn_q_workspace_bytes.argtypes = [C.POINTER(Shape)]
         L.moe_expert_ffn_q.restype = C.c_int
         L.moe_expert_ffn_q.argtypes = [vp, vp, vp, vp, vp, vp, vp, C.POINTER(Shape), vp, vp, vp, sz, vp]
+        L.moe_ep_permute.restype = C.c_int
+        L.moe_ep_permute.argtypes = [vp, vp, vp, C.POINTER(Shape), i32, i32, vp, vp, vp, vp, sz, vp]
         L.moe_ep_row_table.restype = C.c_int
         L.moe_ep_row_table.argtypes = [vp, vp, C.POINTER(Shape), i32, i32, vp, i32, vp, vp]
         L.moe_ep_expert_ffn.restype = C.c_int
@@ -242,6 +244,11 @@ def moe_expert_ffn_q(x_perm, expert_offsets, weights, sh, y_perm, status_word, w
     _check(lib().moe_expert_ffn_q(_ptr(x_perm), _ptr(expert_offsets), _ptr(raw[0]), _ptr(raw[1]), _ptr(raw[2]), _ptr(raw[3]),
                                   _ptr(packed), C.byref(sh), _ptr(y_perm), _ptr(status_word), _ptr(ws), ws.numel(),
                                   _stream(stream)), "moe_expert_ffn_q")
+
+
+def moe_ep_permute(x, topk_ids, expert_offsets, sh, e_begin, e_end, x_perm, perm, inv_perm, ws, stream=None):
+    _check(lib().moe_ep_permute(_ptr(x), _ptr(topk_ids), _ptr(expert_offsets), C.byref(sh), e_begin, e_end, _ptr(x_perm),
+                                _ptr(perm), _ptr(inv_perm), _ptr(ws), ws.numel(), _stream(stream)), "moe_ep_permute")
 
 
 def moe_ep_row_table(perm, expert_offsets, sh, e_begin, e_end, owner_y, world, row_dst, stream=None):
