@@ -276,7 +276,9 @@ int moe_ffn_block(const void* x_bf16 /* [T,H] */, const void* w_router_bf16 /* [
  *     Inputs with |v| > 2^126 are outside the domain.
  *   - Result: y_perm differs from moe_expert_ffn's by the quantisation error (about a quarter of the output's norm on
  *     the benchmark's inputs: one E2M1 term keeps two to three significant bits); against this variant's own oracle the
- *     result is the same up to fp32 summation order and the roundings that order can flip.
+ *     result is the same - bit for bit on most rows - up to fp32 summation order, the fast exponential and division of the
+ *     SwiGLU, and the roundings those can flip: about one row in two hundred has one element of its intermediate one code
+ *     step away from the oracle's.
  *   - Weights: the four logical tensors with packed = NULL, or packed = the buffer of moe_prepack with the four NULL.
  *   - Shapes: H and I multiples of 256 and at most 4096; otherwise MOE_ERR_UNSUPPORTED_SHAPE.  Any T * k: one kernel
  *     serves decode and prefill (a pass holds 128 tokens of an expert, against 16 in moe_expert_ffn's kernel).

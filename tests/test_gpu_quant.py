@@ -3,10 +3,14 @@
 Tolerance.  Every product of the variant is an E2M1 value times an E2M1 value times a power of two; the fp32 sums of such
 terms are exact, whatever their order, as long as the terms of one sum span fewer than 24 bits - which is the rule on the
 seeded inputs, so most rows are bit-identical to the oracle.  Where a sum does round, the kernel's order may differ from
-the oracle's ascending order by a few units in the last place (relative 1e-6), and such a difference can flip the bf16
-rounding of an intermediate value and, rarely, the E2M1 code it quantises to - one element of a contraction of I, a change
-of up to the block's unit in one of I terms.  The test therefore asks: at least 95 % of the rows within 1e-5 of the row's
-rms, element by element, and every row within 3e-2 of it."""
+the oracle's ascending order by a few units in the last place, and the kernel's SwiGLU uses the fast exponential and
+division (relative 1e-6).  Such a difference can flip the bf16 rounding of an intermediate value (about 3e-4 of the
+elements) and then, where the value sits at a rounding boundary of the 4-bit format, its E2M1 code (about 1 % of those):
+about one row in two hundred has one element of its intermediate off by one code step - up to a third of its block's
+largest magnitude - and every output of that row moves by that step times a weight (seen: 0.13 of the row's rms, on one
+row of 774).  The comparison therefore asks: every row within 0.25 of its rms, element by element, and all rows but one
+(or 3 % of them) within 1e-5 of it.  `test_ffn_q_stage_by_stage` takes the call apart instead: the token rows' codes
+bit-exact, the intermediate's codes equal up to such flips, the down projection exact on the kernel's own codes."""
 import numpy as np
 import pytest
 import torch
@@ -24,8 +28,9 @@ def _check_rows(got, want, what):
     assert not np.isnan(got).any(), what
     rms = np.sqrt((want.astype(np.float64) ** 2).mean(axis=1, keepdims=True)) + 1e-30
     rel = (np.abs(got.astype(np.float64) - want) / rms).max(axis=1)
-    assert rel.max() <= 3e-2, (what, float(rel.max()))
-    assert (rel <= 1e-5).mean() >= 0.95, (what, float((rel <= 1e-5).mean()))
+    assert rel.max() <= 0.25, (what, float(rel.max()))
+    n_off = int((rel > 1e-5).sum())
+    assert n_off <= max(1, int(0.03 * len(rel))), (what, n_off, len(rel))
 
 
 def _problem(T, H, I, E, k, seed, logits=None):
@@ -206,3 +211,59 @@ def test_ffn_q_whole_tensor_agrees_between_weight_layouts_at_prefill_8k():
     assert int(buf.status.item()) == 0
     assert not torch.isnan(y2).any()
     assert torch.equal(buf.y_perm, y2)
+
+
+def _unpack_codes(packed):
+    return np.stack([packed & 0xF, packed >> 4], axis=-1).reshape(packed.shape[0], -1)
+
+
+@pytest.mark.parametrize("T,H,I,E,k", [(129, 256, 1024, 32, 6), (64, 512, 512, 8, 2), (300, 512, 256, 2, 2)])
+def test_ffn_q_stage_by_stage(T, H, I, E, k):
+    """The call taken apart through its scratch (layout of the variant's workspace: codes of the intermediate [S, I/2],
+    its scale bytes [S, I/32], codes of the token rows [S, H/2], their scale bytes [S, H/32], each region padded to 256
+    bytes).  (1) The token rows' quantisation involves no sum: bit-exact against the oracle's quantiser.  (2) The
+    intermediate's codes: equal to the oracle's except where a last-bit difference before the rounding to bf16 moved
+    a value across a rounding boundary - a handful of elements, each one code step away.  (3) The down projection on
+    the kernel's OWN codes, recomputed in float64: equal to the kernel's output to fp32 rounding."""
+    w, xp, off = _problem(T, H, I, E, k, seed=7)
+    sh = moe.shape(T, H, I, E, k)
+    S = T * k
+    ws = moe.alloc_ffn_q_workspace(sh)
+    y = torch.empty((S, H), dtype=torch.float32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    moe.moe_expert_ffn_q(dev(xp), dev(off), tuple(dev(a) for a in w), sh, y, st, ws)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    al = lambda n: (n + 255) // 256 * 256
+    raw = ws.cpu().numpy()
+    o = 0
+    aq2 = raw[o:o + S * I // 2].reshape(S, I // 2); o += al(S * I // 2)
+    sf2 = raw[o:o + S * I // 32].reshape(S, I // 32); o += al(S * I // 32)
+    aq1 = raw[o:o + S * H // 2].reshape(S, H // 2); o += al(S * H // 2)
+    sf1 = raw[o:o + S * H // 32].reshape(S, H // 32)
+    # (1)
+    q1, s1, _ = O.quant_act(xp)
+    assert np.array_equal(aq1, q1) and np.array_equal(sf1, s1)
+    # (2)
+    want, act = O.expert_ffn_q(xp, off, *w, k, want_act=True)
+    q2, s2, _ = O.quant_act(act)
+    same_scale = sf2 == s2
+    c_gpu, c_ref = _unpack_codes(aq2).astype(np.int64), _unpack_codes(q2).astype(np.int64)
+    diff = (c_gpu != c_ref) & np.repeat(same_scale, 32, axis=1)
+    n_elem = S * I
+    assert (~same_scale).sum() <= max(1, n_elem // 32 // 20000)          # a block's largest value crossing a scale boundary
+    assert diff.sum() <= max(2, n_elem // 20000), int(diff.sum())
+    mag = lambda c: np.where(c >= 8, c - 8, c)
+    assert np.all(np.abs(mag(c_gpu[diff]) - mag(c_ref[diff])) <= 1)       # one step of the 4-bit format
+    # (3)
+    mags = np.array([0, .5, 1, 1.5, 2, 3, 4, 6], np.float64)
+    table = np.concatenate([mags, -mags])
+    a_gpu = table[c_gpu] * np.repeat(np.ldexp(1.0, sf2.astype(np.int64) - 127), 32, axis=1)
+    w2, s2w = w[2], w[3]
+    expert_of = np.repeat(np.arange(E), np.diff(off))
+    got = y.cpu().numpy()
+    for e in np.unique(expert_of):
+        rows = np.nonzero(expert_of == e)[0]
+        W2 = table[_unpack_codes(w2[e]).astype(np.int64)] * np.repeat(np.ldexp(1.0, s2w[e].astype(np.int64) - 127), 32, axis=1)
+        ref = a_gpu[rows] @ W2.T
+        assert np.allclose(got[rows], ref, rtol=2e-6, atol=2e-6 * np.abs(ref).max())
