@@ -453,6 +453,75 @@ class Bench:
                 "numerics": "E2M1 activations with one E8M0 scale per 32 elements: a different result from the bf16-activation "
                             "workloads (its own oracle), about 0.2 of the output norm away"}
 
+    def run_ep_emulated(self, wl, world=8, min_ms=20.0):
+        """Expert-parallel sharding, ONE rank's step as this GPU would run it in a job of `world` GPUs: routing and sort of
+        all tokens, the row table, the rank's experts (their down projection storing through the table - here into
+        buffers on the same GPU, so the links are not in the figure), the combine of the rank's tokens.  Row-layout
+        weights of the rank's experts; CUDA graph of eight steps for decode."""
+        torch, moe, inputs = self.torch, self.moe, self.inputs
+        from paper_2609_15627_b200 import ep
+        stream = self.stream
+        decode = wl.name in DECODE
+        sh = moe.shape(wl.T, wl.H, wl.I, wl.E, wl.k)
+        e0, e1, _, _, _ = ep.partition(wl.T, wl.E, world, 0)
+        w_local = tuple(self.dev(np.ascontiguousarray(a[e0:e1]))
+                        for a in inputs.make_expert_weights(wl.H, wl.I, wl.E, seed=0, experts=range(e0, e1)))
+        n_cycle = 8 if decode else 2
+        batches = [(self.dev(inputs.make_logits(wl.T, wl.E, 7000 + i, wl.skew)), self.dev(inputs.make_x(wl.T, wl.H, 7000 + i)))
+                   for i in range(n_cycle)]
+        ranks = [ep.RankBuffers(torch, moe, sh, world, 0)]
+        others = [torch.empty_like(ranks[0].y_own) for _ in range(world - 1)]  # the other ranks' buffers (never read here)
+        ptrs = torch.tensor([ranks[0].y_own.data_ptr()] + [t.data_ptr() for t in others], dtype=torch.int64, device="cuda")
+        ranks[0].owner_y.copy_(ptrs)
+        out = torch.empty((wl.T, wl.H), dtype=torch.bfloat16, device="cuda")
+        b = ranks[0]
+
+        def step(i, st=stream):
+            l, x = batches[i % n_cycle]
+            ep.compute(moe, b, l, x, w_local, st)
+            ep.finish(moe, b, out, st)
+
+        for i in range(3):
+            step(i)
+        self.barrier()
+        g = None
+        if decode:
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            with torch.cuda.stream(side):
+                step(0, None)
+            stream.wait_stream(side)
+            self.barrier()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for i in range(n_cycle):
+                    step(i, None)
+            g.replay()
+            self.barrier()
+
+        def timed(n):
+            e_0, e_1 = self.events()
+            self.barrier()
+            self.hold()
+            e_0.record(stream)
+            for i in range(n):
+                if g is not None:
+                    g.replay()
+                else:
+                    step(i)
+            e_1.record(stream)
+            self.barrier()
+            return e_0.elapsed_time(e_1) / (n * (n_cycle if g is not None else 1))
+
+        pilot = timed(2)
+        n = max(3, int(min_ms / max(pilot * (n_cycle if g is not None else 1), 1e-3)))
+        ms = timed(n)
+        assert int(b.layer.status.item()) == 0, "device-side wait timed out"
+        del g, ranks, others, batches, w_local
+        torch.cuda.empty_cache()
+        return {"world": world, "rank_ms_per_step": ms, "experts_per_rank": e1 - e0,
+                "note": "one rank's step on one GPU; the stores that would cross the links land in local buffers"}
+
     def read_only_stream(self, status):
         """Read-only ceiling: the decode kernel's load mechanism alone over the resident gate/up weights (2.1 GB at
         the production shape, larger than L2).  Context for the HBM-bound workloads, not the denominator."""
@@ -885,6 +954,13 @@ def main():
         # the quantised-activation variant of the same workload, on the weights this workload has just loaded
         if world == 1 and not args.no_quant and name in QUANT_WORKLOADS:
             quant[name + "_q"] = bench.run_quant(wl)
+    # expert-parallel sharding: one emulated rank of eight (N = 1, default run)
+    ep_emulated = None
+    packed_layout = bench.packed is not None
+    if world == 1 and not args.workload and not args.no_block:
+        bench.weights = bench.packed = None
+        torch.cuda.empty_cache()
+        ep_emulated = {n: bench.run_ep_emulated(inputs.WORKLOADS[n]) for n in ("decode_c64", "prefill_8k")}
     hr = records[head.name]
     ex = hr.pop("exact")
 
@@ -918,7 +994,7 @@ def main():
             "config": {"workload": head.name, "T": head.T, "H": head.H, "I": head.I, "E": head.E, "k": head.k,
                        "parallelism": "replicas only" if world > 1 else "1 GPU", "call": hr["call"],
                        "weights": ("moe_prepack's tile-contiguous layout (one-time transform, same bytes)"
-                                   if bench.packed is not None else "checkpoint row layout"),
+                                   if packed_layout else "checkpoint row layout"),
                        "launch": hr["launch"],
                        "l2": "inputs cycle over %d seeded batches; %.2f GB of expert weights resident (larger than L2)"
                              % (hr["n_cycle"], head.E * expert_weight_bytes(head.H, head.I) / 1e9)},
@@ -927,6 +1003,7 @@ def main():
             "workloads": {n: {k: v for k, v in r.items() if k not in ("one_launch", "n_cycle")} for n, r in records.items()},
             "ffn_block": block,
             "quantised_activations": quant or None,
+            "expert_parallel_emulated": ep_emulated,
             "protocol": ("headline: one region of exactly --steps steps; workloads: %d rounds of at least %d ms (decode) / %d ms "
                          "(prefill) each, %.1f s idle before every round, median reported, every round kept; every region is "
                          "bracketed by a barrier and a synchronize, timed by CUDA events on the launching stream behind a "
